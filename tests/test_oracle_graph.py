@@ -1,0 +1,138 @@
+"""Pins for topology construction and the pair sampler (Section 2 system model, Algorithm 1)."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import swarm_oracle as o
+
+
+def laplacian(adj, n):
+    Lm = np.zeros((n, n))
+    for i in range(n):
+        for j in adj[i]:
+            Lm[i, j] -= 1
+            Lm[i, i] += 1
+    return Lm
+
+
+def check_simple_regular(adj, n, k):
+    assert adj.shape == (n, k)
+    for i in range(n):
+        row = adj[i].tolist()
+        assert i not in row
+        assert len(set(row)) == k
+        for j in row:
+            assert i in adj[j].tolist()
+    # connected (BFS)
+    seen, frontier = {0}, [0]
+    while frontier:
+        nxt = []
+        for u in frontier:
+            for v in adj[u]:
+                if int(v) not in seen:
+                    seen.add(int(v))
+                    nxt.append(int(v))
+        frontier = nxt
+    assert len(seen) == n
+
+
+@pytest.mark.parametrize("n", [2, 3, 8, 16])
+def test_complete_graph(n):
+    s = o.OracleSwarm(n, 4, "complete")
+    check_simple_regular(s.adj, n, n - 1)
+    for i in range(n):
+        assert s.adj[i].tolist() == [j for j in range(n) if j != i]
+    lam = np.linalg.eigvalsh(laplacian(s.adj, n))
+    assert abs(lam[1] - n) < 1e-9            # lambda_2 of the complete graph is n
+
+
+@pytest.mark.parametrize("n", [3, 8, 15])
+def test_ring(n):
+    s = o.OracleSwarm(n, 4, "ring")
+    for i in range(n):
+        assert s.adj[i].tolist() == [(i - 1) % n, (i + 1) % n]
+    lam = np.linalg.eigvalsh(laplacian(s.adj, n))
+    assert abs(lam[1] - (2 - 2 * math.cos(2 * math.pi / n))) < 1e-9
+    with pytest.raises(ValueError):
+        o.OracleSwarm(2, 4, "ring")
+
+
+@pytest.mark.parametrize("n,k,seed", [(32, 4, 3), (16, 8, 5), (256, 8, 5), (9, 4, 1), (5, 2, 9)])
+def test_random_regular(n, k, seed):
+    s = o.OracleSwarm(n, 4, "regular", degree=k, seed=seed)
+    check_simple_regular(s.adj, n, k)
+    for i in range(n):
+        assert s.adj[i].tolist() == sorted(s.adj[i].tolist())
+    s2 = o.OracleSwarm(n, 4, "regular", degree=k, seed=seed + 1)
+    if n > k + 1:
+        assert not np.array_equal(s.adj, s2.adj)
+    for bad in (3, 0, n):
+        with pytest.raises(ValueError):
+            o.OracleSwarm(n, 4, "regular", degree=bad, seed=seed)
+
+
+def test_first_cycle_is_the_fisher_yates_permutation():
+    n, seed = 9, 11
+    s = o.OracleSwarm(n, 4, "regular", degree=2, seed=seed)
+    perm = list(range(n))
+    for i in range(n - 1, 0, -1):
+        wd = o.philox([i // 4, 0, 0, 6], [seed, 0])[i % 4]
+        j = o.uniform_int(wd, i + 1)
+        perm[i], perm[j] = perm[j], perm[i]
+    for t in range(n):
+        u, v = perm[t], perm[(t + 1) % n]
+        assert v in s.adj[u].tolist() and u in s.adj[v].tolist()
+
+
+@pytest.mark.parametrize("topo,k,n", [("ring", 0, 64), ("regular", 4, 32), ("complete", 0, 16)])
+def test_sampled_pairs_are_disjoint_and_adjacent(topo, k, n):
+    s = o.OracleSwarm(n, 4, topo, degree=k, seed=2)
+    total = 0
+    for launch in range(50):
+        pairs = s.sample_pairs(n // 2)
+        assert int(s.launch[0]) == launch + 1
+        nodes = pairs.reshape(-1).tolist()
+        assert len(nodes) == len(set(nodes))
+        for a, b in pairs:
+            assert b in s.adj[a].tolist()
+        total += len(pairs)
+    assert total > 50 * n // 4
+
+
+def test_single_pair_follows_the_edge_law():
+    """With one pair per launch the draw is Algorithm 1's: P[(i -> j)] = 1 / (n * rho_i)."""
+    n, k = 6, 2
+    s = o.OracleSwarm(n, 4, "ring", seed=4)
+    T = 24000
+    counts = {}
+    for _ in range(T):
+        (a, b), = s.sample_pairs(1)
+        counts[(int(a), int(b))] = counts.get((int(a), int(b)), 0) + 1
+    assert len(counts) == n * k
+    expected = T / (n * k)
+    chi2 = sum((c - expected) ** 2 / expected for c in counts.values())
+    assert chi2 < 40.0          # 11 dof
+    # first draw of launch 0 restated from the counter layout
+    s2 = o.OracleSwarm(n, 4, "ring", seed=4)
+    wd = o.philox([0, 0, 0, 7], [4, 0])
+    i = o.uniform_int(wd[0], n)
+    j = int(s2.adj[i][o.uniform_int(wd[1], 2)])
+    assert s2.sample_pairs(1).tolist() == [[i, j]]
+
+
+def test_staleness_clock_bound():
+    """tau resets for the initiator and grows by one for everybody else; the analysis bounds
+    sum_i E[tau_i^2] by 5 n^3 (here: time average over a long schedule)."""
+    n = 8
+    s = o.OracleSwarm(n, 4, "complete", seed=1)
+    tau = np.zeros(n)
+    acc = 0.0
+    T = 4000
+    for _ in range(T):
+        (a, b), = s.sample_pairs(1)
+        tau += 1
+        tau[a] = 0
+        acc += (tau**2).sum()
+    assert acc / T <= 5 * n**3
+    assert acc / T > n            # and it is not trivially zero

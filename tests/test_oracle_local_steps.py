@@ -1,0 +1,135 @@
+"""Pins for the local SGD steps (Section 3 "The Communication Procedure": H sequential stochastic
+gradients, each taken at the running iterate) on the two synthetic objectives."""
+import numpy as np
+import pytest
+
+from oracle import swarm_oracle as o
+
+
+def lsq(n=3, d=24, m=10, batch=4, dtype=0, groups=0, noise=0.0, seed=1):
+    s = o.OracleSwarm(n, d, "complete", seed=seed)
+    s.configure(objective=2, lsq_m=m, lsq_batch=batch, lsq_dtype=dtype, lsq_groups=groups, lsq_noise_std=noise)
+    return s
+
+
+def test_lsq_data_recipe():
+    s = lsq(n=4, d=4000, m=6, noise=float(np.sqrt(0.1)), seed=2)
+    A = s.A
+    assert A.shape == (4, 6, 4000)
+    assert abs(A.std() * np.sqrt(4000) - 1) < 0.02          # N(0, 1/d)
+    assert abs(s.xstar.std() - 1) < 0.05
+    assert np.all(np.abs(s.shift) <= 1)
+    clean = np.einsum("grk,k->gr", A.astype(np.float64), s.xstar.astype(np.float64))
+    resid = s.bvec - clean - s.shift[:, None]
+    assert abs(resid.std() - np.sqrt(0.1)) < 0.15            # 24 samples of the label noise
+    s = lsq(n=4, d=64, m=6, groups=2, dtype=1)
+    assert s.A.shape == (2, 6, 64)
+    import torch
+    a = torch.from_numpy(s.A.copy())
+    assert torch.equal(a, a.to(torch.bfloat16).to(torch.float32))   # stored values are bf16-representable
+
+
+def test_lsq_single_step_by_hand():
+    """H = 1, batch 1: x' = x - lr * (<a, x> - b) * a for the sampled row a."""
+    s = lsq(n=2, d=5, m=3, batch=1)
+    x0 = s.X[1].astype(np.float64).copy()
+    row = int(s.minibatch_rows(1, 0)[0])
+    a = s.A[1, row].astype(np.float64)
+    assert s.local_steps([1], 1, 0.25) == 0
+    want = x0 - 0.25 * (a @ x0 - float(s.bvec[1, row])) * a
+    assert np.array_equal(s.X[1], want.astype(np.float32))
+    assert s.ls.tolist() == [0, 1]
+    fresh = o.OracleSwarm(2, 5, "complete", seed=1)
+    assert np.array_equal(s.X[0], fresh.X[0])                 # other node untouched
+
+
+def test_lsq_step_is_minus_lr_times_minibatch_gradient_by_finite_differences():
+    s = lsq(n=2, d=8, m=12, batch=5, noise=0.3)
+    rows = s.minibatch_rows(0, 0)
+    x0 = s.X[0].astype(np.float64).copy()
+    A = s.A[0].astype(np.float64)[rows]
+    b = s.bvec[0].astype(np.float64)[rows]
+
+    def f(x):                                  # minibatch objective (1/2B) sum (a_s x - b_s)^2
+        return 0.5 * ((A @ x - b) ** 2).mean()
+    g = np.zeros(8)
+    for k in range(8):
+        h = np.zeros(8)
+        h[k] = 1e-6
+        g[k] = (f(x0 + h) - f(x0 - h)) / 2e-6
+    s.local_steps([0], 1, 0.1)
+    assert np.abs((s.X[0] - x0) / -0.1 - g).max() < 1e-5 * max(1.0, np.abs(g).max())
+
+
+def test_lsq_rows_are_uniform_with_replacement_and_shared_inside_a_data_group():
+    s = lsq(n=4, d=8, m=7, batch=6, groups=2)
+    counts = np.zeros(7)
+    for ev in range(2000):
+        r = s.minibatch_rows(0, ev)
+        assert r.min() >= 0 and r.max() < 7
+        counts[r] += 1
+        assert np.array_equal(r, s.minibatch_rows(1, ev))        # same group, same event
+    assert not np.array_equal(s.minibatch_rows(0, 0), s.minibatch_rows(2, 0))
+    exp = counts.sum() / 7
+    assert ((counts - exp) ** 2 / exp).sum() < 30
+    # restated from the counter layout: word t of stream 8, row id = data group, event = step counter
+    wd = o.philox([1, 1, 5, 8], [1, 0])
+    assert s.minibatch_rows(3, 5)[4] == o.uniform_int(wd[0], 7)
+
+
+def test_lsq_sgd_converges_on_a_consistent_system():
+    """No label noise, no shift: the system A x = b is consistent (m < d), so randomized row-action
+    SGD drives the residual to zero (Kaczmarz-type convergence)."""
+    s = lsq(n=2, d=40, m=8, batch=4, noise=0.0)
+    s.shift[:] = 0
+    A = s.A.astype(np.float64)
+    s.bvec[:] = np.einsum("grk,k->gr", A, s.xstar.astype(np.float64)).astype(np.float32)
+    r0 = np.linalg.norm(A[0] @ s.X[0] - s.bvec[0])
+    s.local_steps([0], 4000, 0.5)
+    r1 = np.linalg.norm(A[0] @ s.X[0] - s.bvec[0])
+    assert r1 < 1e-4 * r0
+    assert int(s.ls[0]) == 4000 and int(s.ls[1]) == 0
+
+
+def test_each_local_step_uses_the_running_iterate():
+    s1, s2 = lsq(seed=4), lsq(seed=4)
+    s1.local_steps([2], 3, 0.2)
+    for _ in range(3):
+        s2.local_steps([2], 1, 0.2)
+    assert np.array_equal(s1.X, s2.X)
+    assert s1.ls.tolist() == [0, 0, 3]
+
+
+def test_synthetic_gradient_moments_and_op_order():
+    n, d = 2, 40000
+    s = o.OracleSwarm(n, d, "complete", seed=6)
+    s.configure(objective=1, grad_std=float(np.sqrt(1e-3)), drift_std=float(np.sqrt(0.05)))
+    x0 = s.X.copy()
+    lr = 0.05
+    s.local_steps([1], 1, lr)
+    upd = (s.X[1].astype(np.float64) - x0[1])
+    c = float(s.drift[1])
+    assert abs(upd.mean() + lr * c) < 5 * lr * np.sqrt(1e-3 / d) + 1e-8
+    assert abs(upd.var() - lr**2 * 1e-3) < 0.03 * lr**2 * 1e-3
+    assert np.array_equal(s.X[0], x0[0])
+    # element 0 restated from the counter layout with the unfused fp32 operation order
+    wd = o.philox([0, 1, 0, 9], [6, 0])
+    z = np.float32(o.normal_pair(wd[0], wd[1])[0])
+    p = np.float32(s.cfg.grad_std) * z
+    g = np.float32(c) + p
+    st = np.float32(lr) * g
+    assert s.X[1, 0] == x0[1, 0] - st
+    # second step draws fresh noise (event counter advanced)
+    x1 = s.X[1].copy()
+    s.local_steps([1], 1, lr)
+    assert abs(np.corrcoef(s.X[1] - x1, x1 - x0[1])[0, 1]) < 0.03
+
+
+def test_local_step_validation():
+    s = o.OracleSwarm(3, 8, "complete")
+    assert s.local_steps([0], 1, 0.1) == -1          # no objective configured
+    s.configure(objective=1, grad_std=0.1)
+    assert s.local_steps([0, 0], 1, 0.1) == -1       # node listed twice
+    assert s.local_steps([3], 1, 0.1) == -2
+    assert s.local_steps([], 2, 0.1) == 0
+    assert s.local_steps([1], 0, 0.1) == 0 and int(s.ls[1]) == 0
