@@ -1,0 +1,180 @@
+/*
+ * swarm.h -- C ABI of the B200 SwarmSGD gossip-interaction library.
+ *
+ * Paper: Alistarh et al., "Asynchronous Decentralized SGD with Quantized and Local
+ * Updates" (SwarmSGD). n node models X^1..X^n in R^d live side by side in one GPU's
+ * memory; time is counted in pairwise interactions over the edges of a graph G
+ * (Section 2, "The Distributed System Model").
+ *
+ * General conventions
+ *   - Every call returns SWARM_OK (0) or a negative SWARM_E* code; nothing aborts or
+ *     throws across this boundary. swarm_strerror() names a code; for SWARM_ECUDA
+ *     swarm_last_cuda_error() returns the CUDA error of the failing call.
+ *   - The context owns every device buffer. Pointers named *_host are host memory,
+ *     *_dev device memory; both stay owned by the caller and are only read or
+ *     written during the call unless stated otherwise.
+ *   - Arguments are validated on the host before anything is launched: a rejected
+ *     call changes no state and no counter.
+ *   - Device work is asynchronous on the context's stream and ordered by call order.
+ *     swarm_potential, swarm_get_tensor, swarm_sample_pairs and swarm_sync wait for it.
+ *   - One context is bound to the CUDA device that was current at swarm_init and is
+ *     not thread-safe.
+ *   - All kernels are compiled for sm_100a only; there is no CPU path.
+ *
+ * Memory layout (row-major, every row padded to a multiple of 1024 elements)
+ *   X[n][pitch]   fp32 live models
+ *   B[n][pitch]   fp32 base snapshots (non-blocking mode only): the model a node
+ *                 adopted at its last initiation (Algorithm 1: \hat X^i)
+ *   codes[n][nblk*1024] bytes: the node's communication buffer; at b bits per
+ *                 coordinate the first nblk*128*b bytes are meaningful. Within a
+ *                 1024-coordinate block the code of local coordinate k occupies bits
+ *                 [(k mod (8/b))*b, +b) of byte (k*b) div 8; codes past d are zero.
+ *   exps[n][nblk] int8 lattice exponents e (step 2^e) of each block of the buffer
+ *   nblk = ceil(d / 1024)
+ */
+#ifndef SWARM_B200_H
+#define SWARM_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct swarm_ctx swarm_ctx;
+
+/* A directed interaction: a = initiator, b = responder (Section 2; Algorithm 1, sampling lines). */
+typedef struct { int32_t a, b; } swarm_pair;
+
+/* Communication graph G (Section 2). degree is read for SWARM_TOPO_REGULAR only (even, 2..n-1). */
+typedef struct { int32_t kind, degree; } swarm_topology;
+enum { SWARM_TOPO_COMPLETE = 0, SWARM_TOPO_RING = 1, SWARM_TOPO_REGULAR = 2 };
+
+enum { SWARM_BLOCKING = 0, SWARM_NONBLOCKING = 1 };
+enum { SWARM_OBJ_NONE = 0, SWARM_OBJ_SYNTH = 1, SWARM_OBJ_LSQ = 2 };
+enum { SWARM_F32 = 0, SWARM_BF16 = 1 };
+
+enum {
+  SWARM_OK = 0,
+  SWARM_EINVAL = -1,  /* bad n, d, bits, mode, H, count, NULL pointer, size mismatch          */
+  SWARM_ERANGE = -2,  /* node id outside [0, n)                                                */
+  SWARM_EPAIR  = -3,  /* pairs not disjoint, a == b, or (a, b) not an edge of G                */
+  SWARM_ESTATE = -4,  /* e.g. non-blocking mode without base snapshots, local steps without an objective */
+  SWARM_ENOMEM = -5,  /* device or host allocation failed                                      */
+  SWARM_ECUDA  = -6   /* a CUDA call failed                                                    */
+};
+
+/* Workload description (everything the paper leaves to the experiment). Standard deviations,
+ * not variances. Applying it re-creates the whole state from the seed. */
+typedef struct {
+  int32_t objective;     /* SWARM_OBJ_*                                                           */
+  int32_t nonblocking;   /* 1: keep base snapshots B and allow SWARM_NONBLOCKING                  */
+  float   init_std;      /* X^i[k] = init_std * z + o_i                                           */
+  float   offset_std;    /* per-node scalar o_i ~ N(0, offset_std^2)                              */
+  float   grad_std;      /* SYNTH: stochastic gradient = c_i + grad_std * z                       */
+  float   drift_std;     /* SYNTH: per-node scalar c_i ~ N(0, drift_std^2) (non-IID term)         */
+  int32_t lsq_m;         /* LSQ: rows of each data matrix                                         */
+  int32_t lsq_batch;     /* LSQ: minibatch size (rows drawn uniformly with replacement)           */
+  int32_t lsq_dtype;     /* LSQ: SWARM_F32 or SWARM_BF16 storage of the data matrices             */
+  int32_t lsq_groups;    /* LSQ: number of data matrices; 0 = one per node, else must divide n    */
+  float   lsq_noise_std; /* LSQ: label noise; labels = A x* + mu_i + noise, mu_i ~ U(-1, 1)       */
+} swarm_config;
+
+/* Optional device allocator (e.g. a framework's caching allocator). Must be installed before
+ * swarm_init; applies to contexts created afterwards. alloc returns NULL on failure. */
+typedef void *(*swarm_alloc_fn)(size_t bytes, void *user);
+typedef void (*swarm_free_fn)(void *ptr, void *user);
+int swarm_set_allocator(swarm_alloc_fn alloc_fn, swarm_free_fn free_fn, void *user);
+
+/* ------------------------------------------------------------------------------------------
+ * The five core calls
+ * ---------------------------------------------------------------------------------------- */
+
+/* Section 2 / Section 3: create n >= 2 node models of dimension d >= 1 on graph `topo`, with
+ * the counter-based generator keyed by `seed`. Defaults: init_std = 0.1, no objective, no base
+ * snapshots (see swarm_configure). *out receives the context (caller destroys it).
+ * Errors: EINVAL (n, d, topology; regular graph not constructible), ENOMEM, ECUDA. */
+int swarm_init(swarm_ctx **out, int32_t n, int64_t d, swarm_topology topo, uint64_t seed);
+
+/* Section 3, "The Communication Procedure": each listed node takes H sequential stochastic
+ * gradient steps of size lr on its own objective, every gradient evaluated at the running
+ * iterate (\tilde h^q = \tilde g_i(X - sum_{s<q} lr \tilde h^s)); the steps are applied in
+ * place to X^i. node_ids_host: `count` distinct ids (host). H >= 0.
+ * Errors: ESTATE (no objective), EINVAL (H < 0, count < 0, duplicate id), ERANGE. */
+int swarm_local_steps(swarm_ctx *ctx, const int32_t *node_ids_host, int32_t count, int32_t H, float lr);
+
+/* Algorithm 1, interaction lines; Corollary 1 for Enc/Dec. `pairs_host` holds npairs disjoint
+ * directed edges of G. bits in {2, 4, 8}: lattice quantizer with that many bits per
+ * coordinate; bits = 32 (blocking only): identity quantizer (Corollary 2).
+ *   SWARM_BLOCKING: per 1024-block the common exponent e is taken from the exact range of
+ *     X^a - X^b; both models are encoded into their own buffers, each side decodes the
+ *     partner's buffer with its own model as key, and both adopt Q(X^a)/2 + Q(X^b)/2.
+ *   SWARM_NONBLOCKING: the initiator decodes its own and the responder's buffer with its base
+ *     snapshot as key, averages, subtracts its pending local update B^a - X^a, adopts the
+ *     result as model and snapshot, and writes Enc(new model) to its own buffer and Enc(average)
+ *     to the responder's; the responder's model is not touched. Buffers are (re)published from
+ *     the snapshots first if they do not hold `bits`-bit codes or a blocking call intervened.
+ * Errors: EINVAL (bits, mode, npairs < 0, NULL), ERANGE, EPAIR, ESTATE. */
+int swarm_interact(swarm_ctx *ctx, const swarm_pair *pairs_host, int32_t npairs, int32_t bits, int32_t mode);
+
+/* Section 4: mu = (1/n) sum_i X^i, written to out_dev (d floats, device memory). */
+int swarm_mean_model(swarm_ctx *ctx, float *out_dev);
+
+/* Section 4: Gamma = sum_i ||X^i - mu||^2, written to *out_gamma_host. Synchronises. */
+int swarm_potential(swarm_ctx *ctx, double *out_gamma_host);
+
+/* ------------------------------------------------------------------------------------------
+ * Auxiliary calls
+ * ---------------------------------------------------------------------------------------- */
+
+/* Apply a workload description and rebuild the state from the seed (models, per-node scalars,
+ * data, counters). Errors: EINVAL, ENOMEM, ECUDA. */
+int swarm_configure(swarm_ctx *ctx, const swarm_config *cfg_host);
+
+/* Algorithm 1, sampling lines: draw up to max_pairs disjoint pairs for the next launch
+ * (initiator uniform over nodes, responder uniform over its neighbours, draws that touch an
+ * already paired node rejected, at most 16*max_pairs draws). Runs on the device, synchronises,
+ * advances the launch counter. out_pairs_host has room for max_pairs entries. */
+int swarm_sample_pairs(swarm_ctx *ctx, int32_t max_pairs, swarm_pair *out_pairs_host, int32_t *out_count_host);
+
+/* Fill all communication buffers with `bits`-bit encodings of the base snapshots (see
+ * swarm_interact, SWARM_NONBLOCKING). Errors: ESTATE without base snapshots, EINVAL. */
+int swarm_publish(swarm_ctx *ctx, int32_t bits);
+
+/* State access (checkpointing, test injection). `which` selects the array, `node` the row
+ * (ignored for whole-context arrays). bytes must equal the row size exactly. Both synchronise. */
+enum {
+  SWARM_T_X = 0,        /* d floats                                  */
+  SWARM_T_B = 1,        /* d floats (ESTATE without snapshots)       */
+  SWARM_T_CODES = 2,    /* nblk*1024 bytes                           */
+  SWARM_T_EXPS = 3,     /* nblk int8                                 */
+  SWARM_T_ADJ = 4,      /* degree int32 (read-only)                  */
+  SWARM_T_A = 5,        /* node = data-matrix id; lsq_m*d floats (bf16 storage is widened/rounded) */
+  SWARM_T_BVEC = 6,     /* lsq_m floats                              */
+  SWARM_T_XSTAR = 7,    /* d floats, node ignored                    */
+  SWARM_T_SCALARS = 8,  /* 3 floats: offset o_i, drift c_i, shift mu_i */
+  SWARM_T_COUNTERS = 9  /* 3 uint32: buffer write counter, local-step counter, code width of the buffer */
+};
+int swarm_get_tensor(swarm_ctx *ctx, int32_t which, int32_t node, void *dst_host, size_t bytes);
+int swarm_set_tensor(swarm_ctx *ctx, int32_t which, int32_t node, const void *src_host, size_t bytes);
+
+/* Whole-context counters: launch counter of the pair sampler and the "snapshots stale" flag. */
+int swarm_get_state(swarm_ctx *ctx, uint32_t *launch_host, int32_t *b_stale_host);
+int swarm_set_state(swarm_ctx *ctx, uint32_t launch, int32_t b_stale);
+
+/* Device pointer and row pitch (in elements) of X, for callers that consume models in place.
+ * Valid until the next swarm_configure / swarm_destroy. */
+int swarm_model_ptr(swarm_ctx *ctx, float **x_dev, int64_t *pitch);
+
+int swarm_set_stream(swarm_ctx *ctx, void *cuda_stream);   /* cudaStream_t; NULL = default stream */
+int swarm_sync(swarm_ctx *ctx);
+int64_t swarm_kernel_launches(swarm_ctx *ctx);             /* kernels launched so far by this context */
+int swarm_last_cuda_error(swarm_ctx *ctx);                 /* cudaError_t of the last SWARM_ECUDA       */
+const char *swarm_strerror(int code);
+void swarm_destroy(swarm_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SWARM_B200_H */

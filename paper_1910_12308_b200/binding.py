@@ -1,0 +1,265 @@
+"""Thin ctypes binding of the C ABI declared in include/swarm.h.
+
+Argument marshalling only: every step of the method runs in the CUDA library. PyTorch supplies
+device memory (through the allocator hook) and the stream. There is no CPU path: the binding
+raises at import if the shared library is missing and cannot be built.
+"""
+import ctypes as C
+import os
+
+import numpy as np
+
+from . import build as _build
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+
+BLOCKING, NONBLOCKING = 0, 1
+TOPO_COMPLETE, TOPO_RING, TOPO_REGULAR = 0, 1, 2
+OBJ_NONE, OBJ_SYNTH, OBJ_LSQ = 0, 1, 2
+F32, BF16 = 0, 1
+T_X, T_B, T_CODES, T_EXPS, T_ADJ, T_A, T_BVEC, T_XSTAR, T_SCALARS, T_COUNTERS = range(10)
+TOPOLOGY = {"complete": TOPO_COMPLETE, "ring": TOPO_RING, "regular": TOPO_REGULAR}
+
+EXPORTS = [
+    "swarm_set_allocator", "swarm_init", "swarm_local_steps", "swarm_interact", "swarm_mean_model",
+    "swarm_potential", "swarm_configure", "swarm_sample_pairs", "swarm_publish", "swarm_get_tensor",
+    "swarm_set_tensor", "swarm_get_state", "swarm_set_state", "swarm_model_ptr", "swarm_set_stream",
+    "swarm_sync", "swarm_kernel_launches", "swarm_last_cuda_error", "swarm_strerror", "swarm_destroy",
+]
+
+
+class SwarmPair(C.Structure):
+    _fields_ = [("a", C.c_int32), ("b", C.c_int32)]
+
+
+class SwarmTopology(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("degree", C.c_int32)]
+
+
+class SwarmConfig(C.Structure):
+    _fields_ = [
+        ("objective", C.c_int32), ("nonblocking", C.c_int32),
+        ("init_std", C.c_float), ("offset_std", C.c_float),
+        ("grad_std", C.c_float), ("drift_std", C.c_float),
+        ("lsq_m", C.c_int32), ("lsq_batch", C.c_int32), ("lsq_dtype", C.c_int32), ("lsq_groups", C.c_int32),
+        ("lsq_noise_std", C.c_float),
+    ]
+
+
+ALLOC_FN = C.CFUNCTYPE(C.c_void_p, C.c_size_t, C.c_void_p)
+FREE_FN = C.CFUNCTYPE(None, C.c_void_p, C.c_void_p)
+
+_lib = None
+
+
+class SwarmError(RuntimeError):
+    def __init__(self, code, what=""):
+        self.code = code
+        msg = load().swarm_strerror(code).decode()
+        super().__init__(f"{what}: {msg} ({code})" if what else f"{msg} ({code})")
+
+
+def library_path():
+    return os.path.join(_HERE, "libswarm_b200.so")
+
+
+def load():
+    """Load (building first if the sources are newer) the CUDA library. Never falls back."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = library_path()
+    if not os.path.exists(path) or os.environ.get("SWARM_REBUILD"):
+        path = _build.build()
+    L = C.CDLL(path)
+    vp, i32, i64, u32, u64, f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32, C.c_uint64, C.c_float
+    sig = {
+        "swarm_set_allocator": (C.c_int, [ALLOC_FN, FREE_FN, vp]),
+        "swarm_init": (C.c_int, [C.POINTER(vp), i32, i64, SwarmTopology, u64]),
+        "swarm_local_steps": (C.c_int, [vp, C.POINTER(i32), i32, i32, f32]),
+        "swarm_interact": (C.c_int, [vp, C.POINTER(SwarmPair), i32, i32, i32]),
+        "swarm_mean_model": (C.c_int, [vp, vp]),
+        "swarm_potential": (C.c_int, [vp, C.POINTER(C.c_double)]),
+        "swarm_configure": (C.c_int, [vp, C.POINTER(SwarmConfig)]),
+        "swarm_sample_pairs": (C.c_int, [vp, i32, C.POINTER(SwarmPair), C.POINTER(i32)]),
+        "swarm_publish": (C.c_int, [vp, i32]),
+        "swarm_get_tensor": (C.c_int, [vp, i32, i32, vp, C.c_size_t]),
+        "swarm_set_tensor": (C.c_int, [vp, i32, i32, vp, C.c_size_t]),
+        "swarm_get_state": (C.c_int, [vp, C.POINTER(u32), C.POINTER(i32)]),
+        "swarm_set_state": (C.c_int, [vp, u32, i32]),
+        "swarm_model_ptr": (C.c_int, [vp, C.POINTER(vp), C.POINTER(i64)]),
+        "swarm_set_stream": (C.c_int, [vp, vp]),
+        "swarm_sync": (C.c_int, [vp]),
+        "swarm_kernel_launches": (i64, [vp]),
+        "swarm_last_cuda_error": (C.c_int, [vp]),
+        "swarm_strerror": (C.c_char_p, [C.c_int]),
+        "swarm_destroy": (None, [vp]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(L, name)
+        fn.restype = res
+        fn.argtypes = args
+    _lib = L
+    return L
+
+
+# ---- torch-backed device memory ---------------------------------------------------------------
+_torch_blocks = {}
+_alloc_cb = None
+_free_cb = None
+
+
+def use_torch_allocator():
+    """Route the library's device allocations through PyTorch's caching allocator."""
+    global _alloc_cb, _free_cb
+    import torch
+
+    def _alloc(nbytes, _user):
+        try:
+            t = torch.empty(int(nbytes), dtype=torch.uint8, device="cuda")
+        except Exception:
+            return None
+        _torch_blocks[t.data_ptr()] = t
+        return t.data_ptr()
+
+    def _free(ptr, _user):
+        _torch_blocks.pop(ptr, None)
+
+    _alloc_cb, _free_cb = ALLOC_FN(_alloc), FREE_FN(_free)
+    rc = load().swarm_set_allocator(_alloc_cb, _free_cb, None)
+    if rc != 0:
+        raise SwarmError(rc, "swarm_set_allocator")
+
+
+def _pairs_array(pairs):
+    pairs = np.ascontiguousarray(pairs, dtype=np.int32).reshape(-1, 2)
+    return pairs, pairs.ctypes.data_as(C.POINTER(SwarmPair))
+
+
+class Swarm:
+    """One swarm context on the current CUDA device. Methods mirror the C entry points."""
+
+    def __init__(self, n, d, topology="complete", degree=0, seed=0, torch_memory=True, stream=None):
+        L = load()
+        if torch_memory:
+            import torch
+            if not torch.cuda.is_available():
+                raise RuntimeError("swarm: no CUDA device; this library has no CPU path")
+            if _alloc_cb is None:
+                use_torch_allocator()
+        kind = TOPOLOGY[topology] if isinstance(topology, str) else int(topology)
+        h = C.c_void_p()
+        rc = L.swarm_init(C.byref(h), n, d, SwarmTopology(kind, degree), seed)
+        if rc != 0:
+            raise SwarmError(rc, "swarm_init")
+        self._h, self._L = h, L
+        self.n, self.d, self.seed = n, d, seed
+        self.nblk = (d + 1023) // 1024
+        self.cfg = SwarmConfig(OBJ_NONE, 0, 0.1, 0.0, 0.0, 0.0, 0, 0, 0, 0, 0.0)
+        self.degree = {TOPO_COMPLETE: n - 1, TOPO_RING: 2}.get(kind, degree)
+        if stream is not None:
+            self.set_stream(stream)
+
+    # -- lifetime
+    def close(self):
+        if getattr(self, "_h", None):
+            self._L.swarm_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, rc, what):
+        if rc != 0:
+            raise SwarmError(rc, what)
+
+    # -- the five core calls
+    def local_steps(self, nodes, H, lr):
+        nodes = np.ascontiguousarray(nodes, dtype=np.int32)
+        return self._L.swarm_local_steps(self._h, nodes.ctypes.data_as(C.POINTER(C.c_int32)), len(nodes), H, lr)
+
+    def interact(self, pairs, bits, mode=BLOCKING):
+        arr, ptr = _pairs_array(pairs)
+        return self._L.swarm_interact(self._h, ptr, len(arr), bits, mode)
+
+    def mean_model(self, out=None):
+        import torch
+        if out is None:
+            out = torch.empty(self.d, dtype=torch.float32, device="cuda")
+        self._check(self._L.swarm_mean_model(self._h, out.data_ptr()), "swarm_mean_model")
+        return out
+
+    def potential(self):
+        g = C.c_double()
+        self._check(self._L.swarm_potential(self._h, C.byref(g)), "swarm_potential")
+        return g.value
+
+    # -- auxiliary
+    def configure(self, **kw):
+        for k, v in kw.items():
+            if not hasattr(self.cfg, k):
+                raise KeyError(k)
+            setattr(self.cfg, k, v)
+        self._check(self._L.swarm_configure(self._h, C.byref(self.cfg)), "swarm_configure")
+
+    def sample_pairs(self, max_pairs):
+        out = np.zeros((max(max_pairs, 1), 2), dtype=np.int32)
+        cnt = C.c_int32()
+        self._check(self._L.swarm_sample_pairs(self._h, max_pairs, out.ctypes.data_as(C.POINTER(SwarmPair)),
+                                               C.byref(cnt)), "swarm_sample_pairs")
+        return out[: cnt.value].copy()
+
+    def publish(self, bits):
+        return self._L.swarm_publish(self._h, bits)
+
+    def set_stream(self, stream):
+        ptr = getattr(stream, "cuda_stream", stream)
+        self._check(self._L.swarm_set_stream(self._h, ptr), "swarm_set_stream")
+
+    def sync(self):
+        self._check(self._L.swarm_sync(self._h), "swarm_sync")
+
+    def kernel_launches(self):
+        return int(self._L.swarm_kernel_launches(self._h))
+
+    def model_ptr(self):
+        p, pitch = C.c_void_p(), C.c_int64()
+        self._check(self._L.swarm_model_ptr(self._h, C.byref(p), C.byref(pitch)), "swarm_model_ptr")
+        return p.value, pitch.value
+
+    # -- state access
+    def _row_spec(self, which):
+        m = self.cfg.lsq_m
+        return {
+            T_X: (np.float32, self.d), T_B: (np.float32, self.d), T_CODES: (np.uint8, self.nblk * 1024),
+            T_EXPS: (np.int8, self.nblk), T_ADJ: (np.int32, self.degree), T_A: (np.float32, m * self.d),
+            T_BVEC: (np.float32, m), T_XSTAR: (np.float32, self.d), T_SCALARS: (np.float32, 3),
+            T_COUNTERS: (np.uint32, 3),
+        }[which]
+
+    def get(self, which, node=0):
+        dt, count = self._row_spec(which)
+        out = np.empty(count, dtype=dt)
+        self._check(self._L.swarm_get_tensor(self._h, which, node, out.ctypes.data, out.nbytes), "swarm_get_tensor")
+        return out
+
+    def set(self, which, node, values):
+        dt, count = self._row_spec(which)
+        arr = np.ascontiguousarray(values, dtype=dt).reshape(-1)
+        if arr.size != count:
+            raise ValueError(f"expected {count} elements, got {arr.size}")
+        self._check(self._L.swarm_set_tensor(self._h, which, node, arr.ctypes.data, arr.nbytes), "swarm_set_tensor")
+
+    def get_all(self, which):
+        return np.stack([self.get(which, i) for i in range(self.n)])
+
+    def get_state(self):
+        launch, stale = C.c_uint32(), C.c_int32()
+        self._check(self._L.swarm_get_state(self._h, C.byref(launch), C.byref(stale)), "swarm_get_state")
+        return launch.value, stale.value
+
+    def set_state(self, launch, b_stale):
+        self._check(self._L.swarm_set_state(self._h, launch, b_stale), "swarm_set_state")

@@ -1,0 +1,655 @@
+// C ABI and host scheduler: context, device store, argument validation, counters, staging of
+// pair / node descriptors and kernel launches. All arithmetic of the method runs in the kernels.
+#include <algorithm>
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/swarm.h"
+#include "swarm_dev.cuh"
+#include "swarm_internal.h"
+
+using namespace swarm;
+
+namespace {
+
+swarm_alloc_fn g_alloc = nullptr;
+swarm_free_fn g_free = nullptr;
+void* g_alloc_user = nullptr;
+
+constexpr int kStageSlots = 8;
+
+}  // namespace
+
+struct swarm_ctx {
+  int32_t n = 0;
+  int64_t d = 0, pitch = 0, nblk = 0;
+  int32_t topo_kind = 0, degree = 0;
+  uint64_t seed = 0;
+  int device = 0;
+  cudaStream_t stream = nullptr;
+  swarm_config cfg{};
+  int last_cuda = 0;
+  int64_t launches = 0;
+  bool custom_alloc = false;
+  swarm_alloc_fn alloc_fn = nullptr;
+  swarm_free_fn free_fn = nullptr;
+  void* alloc_user = nullptr;
+
+  // host mirrors
+  std::vector<int32_t> adj;          // n * degree
+  std::vector<uint32_t> w, ls;       // buffer write counters, local-step counters
+  std::vector<int32_t> pbits;        // code width currently held by each buffer (0 = none)
+  uint32_t launch_ctr = 0;
+  int32_t b_stale = 0;
+  int32_t groups = 0, nodes_per_group = 0;
+
+  // device store
+  float* X = nullptr;
+  float* B = nullptr;
+  uint8_t* codes = nullptr;
+  int8_t* exps = nullptr;
+  int32_t* adj_dev = nullptr;
+  float* scalars = nullptr;          // n * 3
+  void* A = nullptr;
+  float* bvec = nullptr;
+  float* xstar = nullptr;
+  float* lsq_partial = nullptr;      // n * batch * chunks
+  double* pot_partial = nullptr;
+  double* pot_out = nullptr;
+  int32_t* pairs_out_dev = nullptr;  // 2 * n/2 + 1 (sampler result, count last)
+  uint8_t* used_dev = nullptr;       // n
+  float* convert_tmp = nullptr;      // pitch floats (bf16 row conversion)
+
+  // staging ring for descriptors (pinned host + device), guarded by events
+  void* stage_host = nullptr;
+  void* stage_dev = nullptr;
+  size_t stage_slot_bytes = 0;
+  cudaEvent_t stage_event[kStageSlots] = {};
+  int stage_next = 0;
+  double* pot_host = nullptr;        // pinned
+  int32_t* pairs_out_host = nullptr; // pinned
+};
+
+namespace {
+
+struct DeviceGuard {
+  int prev = 0;
+  explicit DeviceGuard(int dev) { cudaGetDevice(&prev); if (prev != dev) cudaSetDevice(dev); else prev = -1; }
+  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+int fail_cuda(swarm_ctx* c, cudaError_t e) { c->last_cuda = (int)e; return SWARM_ECUDA; }
+
+#define SW_CUDA(ctx, call)                                   \
+  do {                                                       \
+    cudaError_t e__ = (call);                                \
+    if (e__ != cudaSuccess) return fail_cuda((ctx), e__);    \
+  } while (0)
+
+void* dev_alloc(swarm_ctx* c, size_t bytes) {
+  if (bytes == 0) bytes = 256;
+  void* p = nullptr;
+  if (c->custom_alloc) p = c->alloc_fn(bytes, c->alloc_user);
+  else if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); p = nullptr; }
+  return p;
+}
+void dev_free(swarm_ctx* c, void* p) {
+  if (!p) return;
+  if (c->custom_alloc) c->free_fn(p, c->alloc_user); else cudaFree(p);
+}
+
+StoreView view_of(const swarm_ctx* c) {
+  StoreView s;
+  s.X = c->X; s.B = c->B; s.codes = c->codes; s.exps = c->exps;
+  s.pitch = c->pitch; s.d = c->d; s.nblk = c->nblk; s.n = c->n;
+  s.key0 = (uint32_t)c->seed; s.key1 = (uint32_t)(c->seed >> 32);
+  return s;
+}
+LsqView lsq_of(const swarm_ctx* c) {
+  LsqView l;
+  l.A = c->A; l.bvec = c->bvec; l.m = c->cfg.lsq_m; l.batch = c->cfg.lsq_batch; l.dtype = c->cfg.lsq_dtype;
+  l.groups = c->groups; l.nodes_per_group = c->nodes_per_group;
+  return l;
+}
+
+// Communication graph (Section 2). Random k-regular graphs are unions of k/2 Hamiltonian
+// cycles; a cycle comes from a Fisher-Yates shuffle driven by the topology stream, and a draw
+// that would repeat an existing edge is discarded and redrawn.
+bool build_graph(swarm_ctx* c) {
+  const int n = c->n;
+  auto& adj = c->adj;
+  if (c->topo_kind == SWARM_TOPO_COMPLETE) {
+    c->degree = n - 1;
+    adj.clear();
+    for (int i = 0; i < n; ++i)
+      for (int j = 0; j < n; ++j)
+        if (j != i) adj.push_back(j);
+    return true;
+  }
+  if (c->topo_kind == SWARM_TOPO_RING) {
+    if (n < 3) return false;
+    c->degree = 2;
+    adj.clear();
+    for (int i = 0; i < n; ++i) { adj.push_back((i + n - 1) % n); adj.push_back((i + 1) % n); }
+    return true;
+  }
+  if (c->topo_kind != SWARM_TOPO_REGULAR) return false;
+  const int k = c->degree;
+  if (n < 3 || k < 2 || (k & 1) || k > n - 1) return false;
+  std::vector<std::vector<int>> nb(n);
+  auto linked = [&](int u, int v) { return std::find(nb[u].begin(), nb[u].end(), v) != nb[u].end(); };
+  const uint32_t key0 = (uint32_t)c->seed, key1 = (uint32_t)(c->seed >> 32);
+  std::vector<int> order(n);
+  int accepted = 0;
+  for (uint32_t attempt = 0; accepted < k / 2; ++attempt) {
+    if (attempt >= 4096) return false;
+    for (int i = 0; i < n; ++i) order[i] = i;
+    uint4 words = make_uint4(0, 0, 0, 0);
+    int have = -1;
+    for (int i = n - 1; i > 0; --i) {
+      if (i / 4 != have) { have = i / 4; words = philox4x32_10((uint32_t)have, 0u, attempt, kStreamTopology, key0, key1); }
+      const uint32_t wd = (i & 3) == 0 ? words.x : (i & 3) == 1 ? words.y : (i & 3) == 2 ? words.z : words.w;
+      std::swap(order[i], order[uniform_int(wd, (uint32_t)i + 1u)]);
+    }
+    bool repeat = false;
+    for (int t = 0; t < n; ++t)
+      if (linked(order[t], order[(t + 1) % n])) { repeat = true; break; }
+    if (repeat) continue;
+    for (int t = 0; t < n; ++t) {
+      const int u = order[t], v = order[(t + 1) % n];
+      nb[u].push_back(v);
+      nb[v].push_back(u);
+    }
+    ++accepted;
+  }
+  adj.clear();
+  for (int i = 0; i < n; ++i) {
+    std::sort(nb[i].begin(), nb[i].end());
+    if ((int)nb[i].size() != k) return false;
+    adj.insert(adj.end(), nb[i].begin(), nb[i].end());
+  }
+  return true;
+}
+
+void free_objective(swarm_ctx* c) {
+  dev_free(c, c->A); c->A = nullptr;
+  dev_free(c, c->bvec); c->bvec = nullptr;
+  dev_free(c, c->xstar); c->xstar = nullptr;
+  dev_free(c, c->lsq_partial); c->lsq_partial = nullptr;
+  dev_free(c, c->convert_tmp); c->convert_tmp = nullptr;
+  dev_free(c, c->B); c->B = nullptr;
+  c->groups = 0; c->nodes_per_group = 0;
+}
+
+// Acquire a staging slot: returns host pointer and device pointer of the slot.
+int stage_acquire(swarm_ctx* c, size_t bytes, void** host, void** dev, int* slot) {
+  if (bytes > c->stage_slot_bytes) return SWARM_EINVAL;
+  const int sidx = c->stage_next;
+  c->stage_next = (sidx + 1) % kStageSlots;
+  SW_CUDA(c, cudaEventSynchronize(c->stage_event[sidx]));
+  *host = (char*)c->stage_host + (size_t)sidx * c->stage_slot_bytes;
+  *dev = (char*)c->stage_dev + (size_t)sidx * c->stage_slot_bytes;
+  *slot = sidx;
+  return SWARM_OK;
+}
+int stage_commit(swarm_ctx* c, int slot, size_t bytes) {
+  void* host = (char*)c->stage_host + (size_t)slot * c->stage_slot_bytes;
+  void* dev = (char*)c->stage_dev + (size_t)slot * c->stage_slot_bytes;
+  SW_CUDA(c, cudaMemcpyAsync(dev, host, bytes, cudaMemcpyHostToDevice, c->stream));
+  return SWARM_OK;
+}
+int stage_release(swarm_ctx* c, int slot) {
+  SW_CUDA(c, cudaEventRecord(c->stage_event[slot], c->stream));
+  return SWARM_OK;
+}
+
+int apply_config(swarm_ctx* c, const swarm_config& cfg) {
+  free_objective(c);
+  c->cfg = cfg;
+  const int n = c->n;
+  const size_t row_bytes = (size_t)c->pitch * sizeof(float);
+  int nl = 0;
+  if (cfg.nonblocking) {
+    c->B = (float*)dev_alloc(c, (size_t)n * row_bytes);
+    if (!c->B) return SWARM_ENOMEM;
+  }
+  if (cfg.objective == SWARM_OBJ_LSQ) {
+    c->groups = cfg.lsq_groups > 0 ? cfg.lsq_groups : n;
+    c->nodes_per_group = n / c->groups;
+    const size_t esz = cfg.lsq_dtype == SWARM_BF16 ? 2 : 4;
+    c->A = dev_alloc(c, (size_t)c->groups * cfg.lsq_m * c->pitch * esz);
+    c->bvec = (float*)dev_alloc(c, (size_t)n * cfg.lsq_m * sizeof(float));
+    c->xstar = (float*)dev_alloc(c, row_bytes);
+    c->lsq_partial = (float*)dev_alloc(c, (size_t)n * cfg.lsq_batch * lsq_chunks(c->d) * sizeof(float));
+    c->convert_tmp = (float*)dev_alloc(c, row_bytes);
+    if (!c->A || !c->bvec || !c->xstar || !c->lsq_partial || !c->convert_tmp) return SWARM_ENOMEM;
+  }
+  StoreView s = view_of(c);
+  SW_CUDA(c, cudaMemsetAsync(c->X, 0, (size_t)n * row_bytes, c->stream));
+  SW_CUDA(c, cudaMemsetAsync(c->codes, 0, (size_t)n * c->nblk * kBlockCoords, c->stream));
+  SW_CUDA(c, cudaMemsetAsync(c->exps, 0, (size_t)n * c->nblk, c->stream));
+  SW_CUDA(c, launch_node_scalars(c->scalars, n, cfg.offset_std, cfg.drift_std, s.key0, s.key1, c->stream, &nl));
+  SW_CUDA(c, launch_init_models(s, c->scalars, cfg.init_std, c->stream, &nl));
+  if (c->B) SW_CUDA(c, cudaMemcpyAsync(c->B, c->X, (size_t)n * row_bytes, cudaMemcpyDeviceToDevice, c->stream));
+  if (cfg.objective == SWARM_OBJ_LSQ) {
+    LsqView l = lsq_of(c);
+    SW_CUDA(c, launch_lsq_data(s, l, c->A, c->xstar, c->bvec, c->scalars, cfg.lsq_noise_std, c->stream, &nl));
+  }
+  c->launches += nl;
+  std::fill(c->w.begin(), c->w.end(), 0u);
+  std::fill(c->ls.begin(), c->ls.end(), 0u);
+  std::fill(c->pbits.begin(), c->pbits.end(), 0);
+  c->launch_ctr = 0;
+  c->b_stale = 0;
+  return SWARM_OK;
+}
+
+int validate_config(const swarm_ctx* c, const swarm_config* cfg) {
+  if (cfg->objective < SWARM_OBJ_NONE || cfg->objective > SWARM_OBJ_LSQ) return SWARM_EINVAL;
+  if (cfg->nonblocking != 0 && cfg->nonblocking != 1) return SWARM_EINVAL;
+  if (!(cfg->init_std >= 0.0f) || !(cfg->offset_std >= 0.0f) || !(cfg->grad_std >= 0.0f) || !(cfg->drift_std >= 0.0f))
+    return SWARM_EINVAL;
+  if (cfg->objective == SWARM_OBJ_LSQ) {
+    if (cfg->lsq_m < 1 || cfg->lsq_batch < 1 || cfg->lsq_batch > 256) return SWARM_EINVAL;
+    if (cfg->lsq_dtype != SWARM_F32 && cfg->lsq_dtype != SWARM_BF16) return SWARM_EINVAL;
+    if (cfg->lsq_groups < 0 || cfg->lsq_groups > c->n) return SWARM_EINVAL;
+    if (cfg->lsq_groups > 0 && (c->n % cfg->lsq_groups) != 0) return SWARM_EINVAL;
+    const int npg = cfg->lsq_groups > 0 ? c->n / cfg->lsq_groups : 1;
+    if (npg > 256) return SWARM_EINVAL;
+    if (!(cfg->lsq_noise_std >= 0.0f)) return SWARM_EINVAL;
+  }
+  return SWARM_OK;
+}
+
+int validate_pairs(const swarm_ctx* c, const swarm_pair* pairs, int npairs) {
+  std::vector<uint8_t> used((size_t)c->n, 0);
+  for (int p = 0; p < npairs; ++p) {
+    const int a = pairs[p].a, b = pairs[p].b;
+    if (a < 0 || a >= c->n || b < 0 || b >= c->n) return SWARM_ERANGE;
+  }
+  for (int p = 0; p < npairs; ++p) {
+    const int a = pairs[p].a, b = pairs[p].b;
+    if (a == b || used[a] || used[b]) return SWARM_EPAIR;
+    const int32_t* row = c->adj.data() + (size_t)a * c->degree;
+    if (std::find(row, row + c->degree, b) == row + c->degree) return SWARM_EPAIR;
+    used[a] = used[b] = 1;
+  }
+  return SWARM_OK;
+}
+
+int do_publish(swarm_ctx* c, int bits) {
+  const size_t row_bytes = (size_t)c->pitch * sizeof(float);
+  if (c->b_stale) {
+    SW_CUDA(c, cudaMemcpyAsync(c->B, c->X, (size_t)c->n * row_bytes, cudaMemcpyDeviceToDevice, c->stream));
+    c->b_stale = 0;
+  }
+  void *host, *dev;
+  int slot;
+  int rc = stage_acquire(c, (size_t)c->n * sizeof(uint32_t), &host, &dev, &slot);
+  if (rc != SWARM_OK) return rc;
+  std::memcpy(host, c->w.data(), (size_t)c->n * sizeof(uint32_t));
+  rc = stage_commit(c, slot, (size_t)c->n * sizeof(uint32_t));
+  if (rc != SWARM_OK) return rc;
+  int nl = 0;
+  SW_CUDA(c, launch_publish(view_of(c), (const uint32_t*)dev, bits, c->stream, &nl));
+  c->launches += nl;
+  rc = stage_release(c, slot);
+  if (rc != SWARM_OK) return rc;
+  for (int i = 0; i < c->n; ++i) { c->w[i] += 1; c->pbits[i] = bits; }
+  return SWARM_OK;
+}
+
+}  // namespace
+
+// =============================================================================================
+extern "C" {
+
+int swarm_set_allocator(swarm_alloc_fn alloc_fn, swarm_free_fn free_fn, void* user) {
+  if ((alloc_fn == nullptr) != (free_fn == nullptr)) return SWARM_EINVAL;
+  g_alloc = alloc_fn; g_free = free_fn; g_alloc_user = user;
+  return SWARM_OK;
+}
+
+const char* swarm_strerror(int code) {
+  switch (code) {
+    case SWARM_OK: return "ok";
+    case SWARM_EINVAL: return "invalid argument";
+    case SWARM_ERANGE: return "node id out of range";
+    case SWARM_EPAIR: return "pairs not disjoint, self-pair, or not an edge of the graph";
+    case SWARM_ESTATE: return "call not valid in the current configuration";
+    case SWARM_ENOMEM: return "out of memory";
+    case SWARM_ECUDA: return "CUDA error (see swarm_last_cuda_error)";
+    default: return "unknown error";
+  }
+}
+
+void swarm_destroy(swarm_ctx* c) {
+  if (!c) return;
+  DeviceGuard guard(c->device);
+  cudaStreamSynchronize(c->stream);
+  free_objective(c);
+  dev_free(c, c->X); dev_free(c, c->codes); dev_free(c, c->exps); dev_free(c, c->adj_dev);
+  dev_free(c, c->scalars); dev_free(c, c->pot_partial); dev_free(c, c->pot_out);
+  dev_free(c, c->pairs_out_dev); dev_free(c, c->used_dev); dev_free(c, c->stage_dev);
+  if (c->stage_host) cudaFreeHost(c->stage_host);
+  if (c->pot_host) cudaFreeHost(c->pot_host);
+  if (c->pairs_out_host) cudaFreeHost(c->pairs_out_host);
+  for (auto& ev : c->stage_event) if (ev) cudaEventDestroy(ev);
+  delete c;
+}
+
+int swarm_init(swarm_ctx** out, int32_t n, int64_t d, swarm_topology topo, uint64_t seed) {
+  if (!out) return SWARM_EINVAL;
+  *out = nullptr;
+  if (n < 2 || d < 1 || d > ((int64_t)1 << 34)) return SWARM_EINVAL;
+  swarm_ctx* c = new (std::nothrow) swarm_ctx();
+  if (!c) return SWARM_ENOMEM;
+  if (cudaGetDevice(&c->device) != cudaSuccess) { c->last_cuda = (int)cudaGetLastError(); delete c; return SWARM_ECUDA; }
+  c->n = n; c->d = d; c->seed = seed;
+  c->nblk = (d + kBlockCoords - 1) / kBlockCoords;
+  c->pitch = c->nblk * kBlockCoords;
+  c->topo_kind = topo.kind; c->degree = topo.degree;
+  c->custom_alloc = g_alloc != nullptr;
+  c->alloc_fn = g_alloc; c->free_fn = g_free; c->alloc_user = g_alloc_user;
+  if (!build_graph(c)) { delete c; return SWARM_EINVAL; }
+  c->w.assign(n, 0); c->ls.assign(n, 0); c->pbits.assign(n, 0);
+
+  const size_t row_bytes = (size_t)c->pitch * sizeof(float);
+  const size_t max_pairs = (size_t)n / 2;
+  c->stage_slot_bytes = std::max({max_pairs * sizeof(PairDesc), (size_t)n * sizeof(NodeDesc), (size_t)n * sizeof(uint32_t)});
+  c->stage_slot_bytes = (c->stage_slot_bytes + 255) / 256 * 256;
+  c->X = (float*)dev_alloc(c, (size_t)n * row_bytes);
+  c->codes = (uint8_t*)dev_alloc(c, (size_t)n * c->nblk * kBlockCoords);
+  c->exps = (int8_t*)dev_alloc(c, (size_t)n * c->nblk);
+  c->adj_dev = (int32_t*)dev_alloc(c, c->adj.size() * sizeof(int32_t));
+  c->scalars = (float*)dev_alloc(c, (size_t)n * 3 * sizeof(float));
+  c->pot_partial = (double*)dev_alloc(c, (size_t)potential_partials(d) * sizeof(double));
+  c->pot_out = (double*)dev_alloc(c, sizeof(double));
+  c->pairs_out_dev = (int32_t*)dev_alloc(c, (2 * max_pairs + 1) * sizeof(int32_t));
+  c->used_dev = (uint8_t*)dev_alloc(c, (size_t)n);
+  c->stage_dev = dev_alloc(c, c->stage_slot_bytes * kStageSlots);
+  bool ok = c->X && c->codes && c->exps && c->adj_dev && c->scalars && c->pot_partial && c->pot_out &&
+            c->pairs_out_dev && c->used_dev && c->stage_dev;
+  ok = ok && cudaMallocHost(&c->stage_host, c->stage_slot_bytes * kStageSlots) == cudaSuccess;
+  ok = ok && cudaMallocHost((void**)&c->pot_host, sizeof(double)) == cudaSuccess;
+  ok = ok && cudaMallocHost((void**)&c->pairs_out_host, (2 * max_pairs + 1) * sizeof(int32_t)) == cudaSuccess;
+  for (int i = 0; ok && i < kStageSlots; ++i)
+    ok = cudaEventCreateWithFlags(&c->stage_event[i], cudaEventDisableTiming) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); swarm_destroy(c); return SWARM_ENOMEM; }
+
+  cudaError_t e = cudaMemcpyAsync(c->adj_dev, c->adj.data(), c->adj.size() * sizeof(int32_t), cudaMemcpyHostToDevice,
+                                  c->stream);
+  if (e != cudaSuccess) { swarm_destroy(c); return SWARM_ECUDA; }
+  swarm_config def{};
+  def.objective = SWARM_OBJ_NONE; def.nonblocking = 0; def.init_std = 0.1f;
+  int rc = apply_config(c, def);
+  if (rc == SWARM_OK && cudaStreamSynchronize(c->stream) != cudaSuccess) rc = SWARM_ECUDA;
+  if (rc != SWARM_OK) { swarm_destroy(c); return rc; }
+  *out = c;
+  return SWARM_OK;
+}
+
+int swarm_configure(swarm_ctx* c, const swarm_config* cfg) {
+  if (!c || !cfg) return SWARM_EINVAL;
+  int rc = validate_config(c, cfg);
+  if (rc != SWARM_OK) return rc;
+  DeviceGuard guard(c->device);
+  SW_CUDA(c, cudaStreamSynchronize(c->stream));
+  rc = apply_config(c, *cfg);
+  if (rc != SWARM_OK) return rc;
+  SW_CUDA(c, cudaStreamSynchronize(c->stream));
+  return SWARM_OK;
+}
+
+int swarm_set_stream(swarm_ctx* c, void* cuda_stream) {
+  if (!c) return SWARM_EINVAL;
+  DeviceGuard guard(c->device);
+  SW_CUDA(c, cudaStreamSynchronize(c->stream));
+  c->stream = (cudaStream_t)cuda_stream;
+  return SWARM_OK;
+}
+
+int swarm_sync(swarm_ctx* c) {
+  if (!c) return SWARM_EINVAL;
+  DeviceGuard guard(c->device);
+  SW_CUDA(c, cudaStreamSynchronize(c->stream));
+  return SWARM_OK;
+}
+
+int64_t swarm_kernel_launches(swarm_ctx* c) { return c ? c->launches : 0; }
+int swarm_last_cuda_error(swarm_ctx* c) { return c ? c->last_cuda : 0; }
+
+int swarm_model_ptr(swarm_ctx* c, float** x_dev, int64_t* pitch) {
+  if (!c || !x_dev || !pitch) return SWARM_EINVAL;
+  *x_dev = c->X; *pitch = c->pitch;
+  return SWARM_OK;
+}
+
+int swarm_local_steps(swarm_ctx* c, const int32_t* node_ids, int32_t count, int32_t H, float lr) {
+  if (!c || count < 0 || H < 0 || (count > 0 && !node_ids)) return SWARM_EINVAL;
+  if (c->cfg.objective == SWARM_OBJ_NONE) return SWARM_ESTATE;
+  if (count > c->n) return SWARM_EINVAL;
+  {
+    std::vector<uint8_t> seen((size_t)c->n, 0);
+    for (int t = 0; t < count; ++t)
+      if (node_ids[t] < 0 || node_ids[t] >= c->n) return SWARM_ERANGE;
+    for (int t = 0; t < count; ++t) {
+      if (seen[node_ids[t]]) return SWARM_EINVAL;
+      seen[node_ids[t]] = 1;
+    }
+  }
+  if (count == 0 || H == 0) return SWARM_OK;
+  DeviceGuard guard(c->device);
+  void *host, *dev;
+  int slot;
+  int rc = stage_acquire(c, (size_t)count * sizeof(NodeDesc), &host, &dev, &slot);
+  if (rc != SWARM_OK) return rc;
+  NodeDesc* nd = (NodeDesc*)host;
+  for (int t = 0; t < count; ++t) { nd[t].node = node_ids[t]; nd[t].event = c->ls[node_ids[t]]; }
+  rc = stage_commit(c, slot, (size_t)count * sizeof(NodeDesc));
+  if (rc != SWARM_OK) return rc;
+  int nl = 0;
+  const StoreView s = view_of(c);
+  if (c->cfg.objective == SWARM_OBJ_SYNTH) {
+    SW_CUDA(c, launch_local_synth(s, (const NodeDesc*)dev, count, H, lr, c->cfg.grad_std, c->scalars, c->stream, &nl));
+  } else {
+    SW_CUDA(c, launch_local_lsq(s, lsq_of(c), (const NodeDesc*)dev, count, H, lr, c->lsq_partial, c->stream, &nl));
+  }
+  c->launches += nl;
+  rc = stage_release(c, slot);
+  if (rc != SWARM_OK) return rc;
+  for (int t = 0; t < count; ++t) c->ls[node_ids[t]] += (uint32_t)H;
+  return SWARM_OK;
+}
+
+int swarm_interact(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, int32_t bits, int32_t mode) {
+  if (!c || npairs < 0 || (npairs > 0 && !pairs)) return SWARM_EINVAL;
+  if (mode != SWARM_BLOCKING && mode != SWARM_NONBLOCKING) return SWARM_EINVAL;
+  const bool quant = bits == 2 || bits == 4 || bits == 8;
+  if (!(quant || (bits == 32 && mode == SWARM_BLOCKING))) return SWARM_EINVAL;
+  if (mode == SWARM_NONBLOCKING && !c->cfg.nonblocking) return SWARM_ESTATE;
+  if (npairs > c->n / 2) return SWARM_EPAIR;
+  int rc = validate_pairs(c, pairs, npairs);
+  if (rc != SWARM_OK) return rc;
+  DeviceGuard guard(c->device);
+  if (mode == SWARM_NONBLOCKING) {
+    bool need = c->b_stale != 0;
+    for (int i = 0; i < c->n && !need; ++i) need = c->pbits[i] != bits;
+    if (need) { rc = do_publish(c, bits); if (rc != SWARM_OK) return rc; }
+  }
+  if (npairs == 0) return SWARM_OK;
+  void *host, *dev;
+  int slot;
+  rc = stage_acquire(c, (size_t)npairs * sizeof(PairDesc), &host, &dev, &slot);
+  if (rc != SWARM_OK) return rc;
+  PairDesc* pd = (PairDesc*)host;
+  for (int p = 0; p < npairs; ++p) {
+    pd[p].a = pairs[p].a; pd[p].b = pairs[p].b;
+    pd[p].wa = c->w[pairs[p].a]; pd[p].wb = c->w[pairs[p].b];
+  }
+  rc = stage_commit(c, slot, (size_t)npairs * sizeof(PairDesc));
+  if (rc != SWARM_OK) return rc;
+  int nl = 0;
+  if (mode == SWARM_BLOCKING) SW_CUDA(c, launch_interact_blocking(view_of(c), (const PairDesc*)dev, npairs, bits, c->stream, &nl));
+  else SW_CUDA(c, launch_interact_nonblocking(view_of(c), (const PairDesc*)dev, npairs, bits, c->stream, &nl));
+  c->launches += nl;
+  rc = stage_release(c, slot);
+  if (rc != SWARM_OK) return rc;
+  if (bits != 32) {
+    for (int p = 0; p < npairs; ++p) {
+      c->w[pairs[p].a] += 1; c->w[pairs[p].b] += 1;
+      if (mode == SWARM_BLOCKING) { c->pbits[pairs[p].a] = bits; c->pbits[pairs[p].b] = bits; }
+    }
+  }
+  if (mode == SWARM_BLOCKING && c->cfg.nonblocking) c->b_stale = 1;
+  return SWARM_OK;
+}
+
+int swarm_publish(swarm_ctx* c, int32_t bits) {
+  if (!c || !(bits == 2 || bits == 4 || bits == 8)) return SWARM_EINVAL;
+  if (!c->cfg.nonblocking) return SWARM_ESTATE;
+  DeviceGuard guard(c->device);
+  return do_publish(c, bits);
+}
+
+int swarm_mean_model(swarm_ctx* c, float* out_dev) {
+  if (!c || !out_dev) return SWARM_EINVAL;
+  DeviceGuard guard(c->device);
+  int nl = 0;
+  SW_CUDA(c, launch_mean_model(view_of(c), out_dev, c->stream, &nl));
+  c->launches += nl;
+  return SWARM_OK;
+}
+
+int swarm_potential(swarm_ctx* c, double* out_gamma) {
+  if (!c || !out_gamma) return SWARM_EINVAL;
+  DeviceGuard guard(c->device);
+  int nl = 0;
+  SW_CUDA(c, launch_potential(view_of(c), c->pot_partial, c->pot_out, c->stream, &nl));
+  c->launches += nl;
+  SW_CUDA(c, cudaMemcpyAsync(c->pot_host, c->pot_out, sizeof(double), cudaMemcpyDeviceToHost, c->stream));
+  SW_CUDA(c, cudaStreamSynchronize(c->stream));
+  *out_gamma = *c->pot_host;
+  return SWARM_OK;
+}
+
+int swarm_sample_pairs(swarm_ctx* c, int32_t max_pairs, swarm_pair* out_pairs, int32_t* out_count) {
+  if (!c || !out_pairs || !out_count || max_pairs < 1) return SWARM_EINVAL;
+  DeviceGuard guard(c->device);
+  const size_t max_slots = (size_t)(c->n / 2);
+  int nl = 0;
+  // the draw budget is 16 * max_pairs even when max_pairs exceeds n/2; acceptance stops at n/2 anyway
+  SW_CUDA(c, launch_sample_pairs(c->adj_dev, c->n, c->degree, max_pairs, c->launch_ctr, (uint32_t)c->seed,
+                                 (uint32_t)(c->seed >> 32), c->pairs_out_dev, c->pairs_out_dev + 2 * max_slots,
+                                 c->used_dev, c->stream, &nl));
+  c->launches += nl;
+  SW_CUDA(c, cudaMemcpyAsync(c->pairs_out_host, c->pairs_out_dev, (2 * max_slots + 1) * sizeof(int32_t),
+                             cudaMemcpyDeviceToHost, c->stream));
+  SW_CUDA(c, cudaStreamSynchronize(c->stream));
+  const int count = c->pairs_out_host[2 * max_slots];
+  for (int p = 0; p < count; ++p) { out_pairs[p].a = c->pairs_out_host[2 * p]; out_pairs[p].b = c->pairs_out_host[2 * p + 1]; }
+  *out_count = count;
+  c->launch_ctr += 1;
+  return SWARM_OK;
+}
+
+int swarm_get_state(swarm_ctx* c, uint32_t* launch, int32_t* b_stale) {
+  if (!c || !launch || !b_stale) return SWARM_EINVAL;
+  *launch = c->launch_ctr; *b_stale = c->b_stale;
+  return SWARM_OK;
+}
+int swarm_set_state(swarm_ctx* c, uint32_t launch, int32_t b_stale) {
+  if (!c || (b_stale != 0 && b_stale != 1)) return SWARM_EINVAL;
+  if (b_stale && !c->cfg.nonblocking) return SWARM_ESTATE;
+  c->launch_ctr = launch; c->b_stale = b_stale;
+  return SWARM_OK;
+}
+
+static int tensor_access(swarm_ctx* c, int32_t which, int32_t node, void* host, size_t bytes, bool write) {
+  if (!c || !host) return SWARM_EINVAL;
+  const bool per_node = which != SWARM_T_XSTAR && which != SWARM_T_A;
+  if (per_node && (node < 0 || node >= c->n)) return SWARM_ERANGE;
+  DeviceGuard guard(c->device);
+  const size_t d = (size_t)c->d;
+  void* dev = nullptr;
+  size_t want = 0;
+  switch (which) {
+    case SWARM_T_X: dev = c->X + (size_t)node * c->pitch; want = d * 4; break;
+    case SWARM_T_B:
+      if (!c->B) return SWARM_ESTATE;
+      dev = c->B + (size_t)node * c->pitch; want = d * 4; break;
+    case SWARM_T_CODES: dev = c->codes + (size_t)node * c->nblk * kBlockCoords; want = (size_t)c->nblk * kBlockCoords; break;
+    case SWARM_T_EXPS: dev = c->exps + (size_t)node * c->nblk; want = (size_t)c->nblk; break;
+    case SWARM_T_ADJ:
+      if (write) return SWARM_EINVAL;
+      if (bytes != (size_t)c->degree * 4) return SWARM_EINVAL;
+      std::memcpy(host, c->adj.data() + (size_t)node * c->degree, bytes);
+      return SWARM_OK;
+    case SWARM_T_BVEC:
+      if (!c->bvec) return SWARM_ESTATE;
+      dev = c->bvec + (size_t)node * c->cfg.lsq_m; want = (size_t)c->cfg.lsq_m * 4; break;
+    case SWARM_T_XSTAR:
+      if (!c->xstar) return SWARM_ESTATE;
+      dev = c->xstar; want = d * 4; break;
+    case SWARM_T_SCALARS: dev = c->scalars + (size_t)node * 3; want = 12; break;
+    case SWARM_T_COUNTERS: {
+      if (bytes != 12) return SWARM_EINVAL;
+      uint32_t* v = (uint32_t*)host;
+      if (write) {
+        if (!(v[2] == 0 || v[2] == 2 || v[2] == 4 || v[2] == 8)) return SWARM_EINVAL;
+        c->w[node] = v[0]; c->ls[node] = v[1]; c->pbits[node] = (int32_t)v[2];
+      } else {
+        v[0] = c->w[node]; v[1] = c->ls[node]; v[2] = (uint32_t)c->pbits[node];
+      }
+      return SWARM_OK;
+    }
+    case SWARM_T_A: {
+      if (!c->A) return SWARM_ESTATE;
+      if (node < 0 || node >= c->groups) return SWARM_ERANGE;
+      const size_t m = (size_t)c->cfg.lsq_m;
+      if (bytes != m * d * 4) return SWARM_EINVAL;
+      SW_CUDA(c, cudaStreamSynchronize(c->stream));
+      int nl = 0;
+      for (size_t r = 0; r < m; ++r) {
+        char* hrow = (char*)host + r * d * 4;
+        if (c->cfg.lsq_dtype == SWARM_F32) {
+          float* drow = (float*)c->A + ((size_t)node * m + r) * c->pitch;
+          if (write) SW_CUDA(c, cudaMemcpyAsync(drow, hrow, d * 4, cudaMemcpyHostToDevice, c->stream));
+          else SW_CUDA(c, cudaMemcpyAsync(hrow, drow, d * 4, cudaMemcpyDeviceToHost, c->stream));
+        } else {
+          uint16_t* drow = (uint16_t*)c->A + ((size_t)node * m + r) * c->pitch;
+          if (write) {
+            SW_CUDA(c, cudaMemcpyAsync(c->convert_tmp, hrow, d * 4, cudaMemcpyHostToDevice, c->stream));
+            SW_CUDA(c, launch_f32_to_bf16(c->convert_tmp, drow, (int64_t)d, c->stream, &nl));
+          } else {
+            SW_CUDA(c, launch_bf16_to_f32(drow, c->convert_tmp, (int64_t)d, c->stream, &nl));
+            SW_CUDA(c, cudaMemcpyAsync(hrow, c->convert_tmp, d * 4, cudaMemcpyDeviceToHost, c->stream));
+          }
+          SW_CUDA(c, cudaStreamSynchronize(c->stream));   // convert_tmp and pageable host memory are reused per row
+        }
+      }
+      c->launches += nl;
+      SW_CUDA(c, cudaStreamSynchronize(c->stream));
+      return SWARM_OK;
+    }
+    default: return SWARM_EINVAL;
+  }
+  if (bytes != want) return SWARM_EINVAL;
+  SW_CUDA(c, cudaStreamSynchronize(c->stream));
+  if (write) SW_CUDA(c, cudaMemcpyAsync(dev, host, bytes, cudaMemcpyHostToDevice, c->stream));
+  else SW_CUDA(c, cudaMemcpyAsync(host, dev, bytes, cudaMemcpyDeviceToHost, c->stream));
+  SW_CUDA(c, cudaStreamSynchronize(c->stream));
+  return SWARM_OK;
+}
+
+int swarm_get_tensor(swarm_ctx* c, int32_t which, int32_t node, void* dst, size_t bytes) {
+  return tensor_access(c, which, node, dst, bytes, false);
+}
+int swarm_set_tensor(swarm_ctx* c, int32_t which, int32_t node, const void* src, size_t bytes) {
+  return tensor_access(c, which, node, const_cast<void*>(src), bytes, true);
+}
+
+}  // extern "C"

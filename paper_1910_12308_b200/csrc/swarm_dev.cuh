@@ -1,0 +1,179 @@
+// Device-side primitives shared by the kernels: counter-based generator, normals,
+// lattice quantizer (constructive form of Corollary 1), 256-bit global accesses and
+// warp reductions. sm_100a only.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace swarm {
+
+constexpr int kBlockCoords = 1024;   // coordinates sharing one lattice exponent
+constexpr int kExpMin = -126;
+constexpr int kExpMax = 119;
+
+// Generator stream ids (fourth counter word).
+enum : uint32_t {
+  kStreamInit = 1, kStreamDataA = 2, kStreamDataNoise = 3, kStreamXStar = 4,
+  kStreamNodeScalars = 5, kStreamTopology = 6, kStreamPairs = 7,
+  kStreamMinibatch = 8, kStreamSynthGrad = 9, kStreamRounding = 10
+};
+
+// ---------------------------------------------------------------------------------------
+// Philox-4x32, 10 rounds (Salmon et al., SC'11). Two 32x32->64 multiplies per round.
+// ---------------------------------------------------------------------------------------
+__host__ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                        uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+    const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+    c1 = (uint32_t)p1;
+    c3 = (uint32_t)p0;
+    c0 = n0;
+    c2 = n2;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return make_uint4(c0, c1, c2, c3);
+}
+
+__host__ __device__ __forceinline__ uint32_t uniform_int(uint32_t word, uint32_t m) {
+  return (uint32_t)(((uint64_t)word * m) >> 32);
+}
+
+__device__ __forceinline__ float uniform_float(uint32_t word) { return (float)(word >> 8) * 0x1p-24f; }
+
+// Box-Muller on two generator words: u1 in (0, 1], u2 in [0, 1).
+__device__ __forceinline__ void normal_pair(uint32_t w0, uint32_t w1, float& z0, float& z1) {
+  const float u1 = (float)((w0 >> 8) + 1u) * 0x1p-24f;
+  const float u2 = (float)(w1 >> 8) * 0x1p-24f;
+  const float r = sqrtf(-2.0f * logf(u1));
+  float s, c;
+  sincospif(2.0f * u2, &s, &c);
+  z0 = r * c;
+  z1 = r * s;
+}
+
+// Four normals of generator call (group, row, event, stream).
+__device__ __forceinline__ void normal4(uint32_t group, uint32_t row, uint32_t event, uint32_t stream,
+                                        uint32_t k0, uint32_t k1, float z[4]) {
+  const uint4 w = philox4x32_10(group, row, event, stream, k0, k1);
+  normal_pair(w.x, w.y, z[0], z[1]);
+  normal_pair(w.z, w.w, z[2], z[3]);
+}
+
+// ---------------------------------------------------------------------------------------
+// Quantizer: lattice of step 2^e, colour = index mod 2^b, L = 2^(b-1) - 1.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ float pow2f_exact(int e) {   // e in [-126, 127]
+  return __uint_as_float((uint32_t)(e + 127) << 23);
+}
+
+// Least e with L * 2^e >= rho, raised so that M * 2^-e < 2^23, clamped to [-126, 119].
+// rho = m * 2^E with m in [0.5, 1): L * 2^(E-b+1) = 2^E (1 - 2^(1-b)) covers rho iff
+// m <= 1 - 2^(1-b), i.e. iff the 23-bit mantissa field is <= 2^23 - 2^(25-b); otherwise
+// one more doubling is needed. Subnormal or zero rho ends at the lower clamp.
+template <int BITS>
+__device__ __forceinline__ int exponent_rule(float rho, float M) {
+  const uint32_t rb = __float_as_uint(rho);
+  int e = kExpMin;
+  if (rb >= 0x00800000u) {
+    const int E = (int)(rb >> 23) - 126;
+    const uint32_t man = rb & 0x007FFFFFu;
+    constexpr uint32_t lim = (1u << 23) - (1u << (25 - BITS));
+    e = E - BITS + (man <= lim ? 1 : 2);
+  }
+  const uint32_t mb = __float_as_uint(M);
+  if (mb >= 0x00800000u) e = max(e, (int)(mb >> 23) - 126 - 23);
+  e = max(e, kExpMin);
+  e = min(e, kExpMax);
+  return e;
+}
+
+// Stochastic rounding onto the lattice with a 16-bit uniform: up with probability
+// floor(frac * 2^16) / 2^16. Returns the lattice index; `cell` receives floor(x * 2^-e).
+__device__ __forceinline__ int32_t encode_index(float x, float inv_step, uint32_t u16, int32_t& cell) {
+  const float t = __fmul_rn(x, inv_step);
+  const float f = floorf(t);
+  const float frac = __fsub_rn(t, f);
+  const uint32_t thr = __float2uint_rz(__fmul_rn(frac, 65536.0f));
+  cell = __float2int_rd(t);                     // saturating, like the reference definition
+  return (int32_t)((uint32_t)cell + (u16 < thr ? 1u : 0u));
+}
+
+// Lattice index congruent to colour c (mod 2^b) in the window [cell - L, cell + L + 1]
+// around the key's cell.
+template <int BITS>
+__device__ __forceinline__ int32_t decode_index(uint32_t c, int32_t cell) {
+  constexpr uint32_t mask = (1u << BITS) - 1u;
+  int32_t delta = (int32_t)((c - (uint32_t)cell) & mask);
+  if (delta > (1 << (BITS - 1))) delta -= (1 << BITS);
+  return (int32_t)((uint32_t)cell + (uint32_t)delta);
+}
+
+template <int BITS>
+__device__ __forceinline__ float decode_value(float key, uint32_t c, float inv_step, float step) {
+  const int32_t cell = __float2int_rd(__fmul_rn(key, inv_step));
+  return __fmul_rn(__int2float_rn(decode_index<BITS>(c, cell)), step);
+}
+
+// 16-bit rounding uniform i (0..7) of a generator call covering 8 consecutive coordinates.
+__device__ __forceinline__ uint32_t sr_u16(const uint4& w, int i) {
+  const uint32_t word = (i < 2) ? w.x : (i < 4) ? w.y : (i < 6) ? w.z : w.w;
+  return (i & 1) ? (word >> 16) : (word & 0xFFFFu);
+}
+
+// ---------------------------------------------------------------------------------------
+// 256-bit global accesses (one lane moves 8 consecutive floats; 32-byte aligned).
+// ---------------------------------------------------------------------------------------
+struct alignas(32) f8 { float v[8]; };
+
+__device__ __forceinline__ f8 ld256(const float* p) {
+  f8 r;
+  asm volatile("ld.global.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]),
+                 "=f"(r.v[4]), "=f"(r.v[5]), "=f"(r.v[6]), "=f"(r.v[7])
+               : "l"(p));
+  return r;
+}
+
+__device__ __forceinline__ void st256(float* p, const f8& r) {
+  asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+               :: "l"(p), "f"(r.v[0]), "f"(r.v[1]), "f"(r.v[2]), "f"(r.v[3]),
+                  "f"(r.v[4]), "f"(r.v[5]), "f"(r.v[6]), "f"(r.v[7])
+               : "memory");
+}
+
+// Eight packed codes of one lane: BITS bytes at `p` (aligned to BITS bytes).
+template <int BITS>
+__device__ __forceinline__ void store_codes(uint8_t* p, uint64_t packed) {
+  if constexpr (BITS == 8) *reinterpret_cast<uint2*>(p) = make_uint2((uint32_t)packed, (uint32_t)(packed >> 32));
+  else if constexpr (BITS == 4) *reinterpret_cast<uint32_t*>(p) = (uint32_t)packed;
+  else *reinterpret_cast<uint16_t*>(p) = (uint16_t)packed;
+}
+template <int BITS>
+__device__ __forceinline__ uint64_t load_codes(const uint8_t* p) {
+  if constexpr (BITS == 8) { const uint2 v = *reinterpret_cast<const uint2*>(p); return (uint64_t)v.x | ((uint64_t)v.y << 32); }
+  else if constexpr (BITS == 4) return *reinterpret_cast<const uint32_t*>(p);
+  else return *reinterpret_cast<const uint16_t*>(p);
+}
+
+// Warp-wide maximum of non-negative floats (bit pattern order equals value order).
+__device__ __forceinline__ float warp_max_nonneg(float v) {
+  return __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, __float_as_uint(v)));
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  return v;
+}
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  return v;
+}
+
+}  // namespace swarm

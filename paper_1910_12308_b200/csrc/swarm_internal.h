@@ -1,0 +1,76 @@
+// Host-side view of the kernels: launch wrappers implemented in the .cu files and the
+// plain-data descriptors they take. No CUDA types beyond cudaStream_t cross this header.
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace swarm {
+
+// One interaction of a launch, with the write counters that index the rounding uniforms.
+struct PairDesc {
+  int32_t a, b;        // initiator, responder
+  uint32_t wa, wb;     // write counters of the two buffers before this interaction
+};
+
+// One node of a local-step launch.
+struct NodeDesc {
+  int32_t node;
+  uint32_t event;      // local-step counter before this call
+};
+
+struct StoreView {
+  float* X;            // [n][pitch]
+  float* B;            // [n][pitch] or nullptr
+  uint8_t* codes;      // [n][nblk * 1024]
+  int8_t* exps;        // [n][nblk]
+  int64_t pitch;       // elements per row, multiple of 1024
+  int64_t d;
+  int64_t nblk;
+  int32_t n;
+  uint32_t key0, key1; // generator key (seed low / high word)
+};
+
+struct LsqView {
+  const void* A;       // [groups][m][pitch] fp32 or bf16
+  const float* bvec;   // [n][m]
+  int32_t m, batch, dtype, groups, nodes_per_group;
+};
+
+// --- swarm_interact.cu -------------------------------------------------------------------
+cudaError_t launch_interact_blocking(const StoreView& s, const PairDesc* pairs_dev, int npairs, int bits,
+                                     cudaStream_t st, int* launches);
+cudaError_t launch_interact_nonblocking(const StoreView& s, const PairDesc* pairs_dev, int npairs, int bits,
+                                        cudaStream_t st, int* launches);
+// wctr_dev: n write counters (uint32) used for the rounding uniforms of each node's buffer.
+cudaError_t launch_publish(const StoreView& s, const uint32_t* wctr_dev, int bits, cudaStream_t st, int* launches);
+
+// --- swarm_local.cu ----------------------------------------------------------------------
+cudaError_t launch_init_models(const StoreView& s, const float* scalars_dev, float init_std, cudaStream_t st,
+                               int* launches);
+cudaError_t launch_node_scalars(float* scalars_dev, int n, float offset_std, float drift_std, uint32_t key0,
+                                uint32_t key1, cudaStream_t st, int* launches);
+cudaError_t launch_lsq_data(const StoreView& s, const LsqView& l, void* A, float* xstar, float* bvec,
+                            const float* scalars_dev, float noise_std, cudaStream_t st, int* launches);
+cudaError_t launch_local_synth(const StoreView& s, const NodeDesc* nodes_dev, int count, int H, float lr,
+                               float grad_std, const float* scalars_dev, cudaStream_t st, int* launches);
+// partial_dev: scratch of count * batch * lsq_chunks(d) floats.
+cudaError_t launch_local_lsq(const StoreView& s, const LsqView& l, const NodeDesc* nodes_dev, int count, int H,
+                             float lr, float* partial_dev, cudaStream_t st, int* launches);
+int64_t lsq_chunks(int64_t d);
+cudaError_t launch_sample_pairs(const int32_t* adj_dev, int n, int degree, int max_pairs, uint32_t launch_ctr,
+                                uint32_t key0, uint32_t key1, int32_t* out_pairs_dev, int32_t* out_count_dev,
+                                uint8_t* used_dev, cudaStream_t st, int* launches);
+
+// --- swarm_reduce.cu ---------------------------------------------------------------------
+cudaError_t launch_mean_model(const StoreView& s, float* out_dev, cudaStream_t st, int* launches);
+// partial_dev: potential_partials(d) doubles of scratch; out_dev: one double.
+cudaError_t launch_potential(const StoreView& s, double* partial_dev, double* out_dev, cudaStream_t st,
+                             int* launches);
+int64_t potential_partials(int64_t d);
+
+// Row conversion helpers for get/set of bf16 data.
+cudaError_t launch_bf16_to_f32(const void* src, float* dst, int64_t count, cudaStream_t st, int* launches);
+cudaError_t launch_f32_to_bf16(const float* src, void* dst, int64_t count, cudaStream_t st, int* launches);
+
+}  // namespace swarm

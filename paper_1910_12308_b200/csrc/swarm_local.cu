@@ -1,0 +1,370 @@
+// State generation, local SGD steps (Section 3, "The Communication Procedure": H sequential
+// stochastic gradient steps, each at the running iterate) and the pair sampler (Algorithm 1,
+// sampling lines).
+#include <cuda_bf16.h>
+
+#include "swarm_dev.cuh"
+#include "swarm_internal.h"
+
+namespace swarm {
+
+// -----------------------------------------------------------------------------------------
+// Per-node scalars: offset o_i, drift c_i (normals), label shift mu_i ~ U(-1, 1).
+// scalars[i*3 + {0,1,2}].
+// -----------------------------------------------------------------------------------------
+__global__ void node_scalars_kernel(float* scalars, int n, float offset_std, float drift_std, uint32_t k0,
+                                    uint32_t k1) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const uint4 w = philox4x32_10(0u, (uint32_t)i, 0u, kStreamNodeScalars, k0, k1);
+  float z0, z1;
+  normal_pair(w.x, w.y, z0, z1);
+  scalars[i * 3 + 0] = __fmul_rn(offset_std, z0);
+  scalars[i * 3 + 1] = __fmul_rn(drift_std, z1);
+  scalars[i * 3 + 2] = __fsub_rn(__fmul_rn(2.0f, uniform_float(w.z)), 1.0f);
+}
+
+// X^i[k] = init_std * z(stream init, row i, k) + o_i ; one thread per 4 coordinates.
+__global__ void init_models_kernel(StoreView s, const float* __restrict__ scalars, float init_std) {
+  const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int i = blockIdx.y;
+  if (g * 4 >= s.d) return;
+  float z[4];
+  normal4((uint32_t)g, (uint32_t)i, 0u, kStreamInit, s.key0, s.key1, z);
+  const float off = scalars[i * 3 + 0];
+  float4 v;
+  float* o = &v.x;
+#pragma unroll
+  for (int t = 0; t < 4; ++t) o[t] = (g * 4 + t < s.d) ? __fadd_rn(__fmul_rn(init_std, z[t]), off) : 0.0f;
+  *reinterpret_cast<float4*>(s.X + (int64_t)i * s.pitch + g * 4) = v;
+}
+
+// -----------------------------------------------------------------------------------------
+// Least-squares data: A_g[r][k] = z / sqrt(d) (rounded to bf16 when stored so), x*[k] = z,
+// labels b_i[r] = <A_g(i)[r], x*> + mu_i + noise_std * z.
+// -----------------------------------------------------------------------------------------
+template <typename T>
+__global__ void lsq_matrix_kernel(T* A, int64_t pitch, int64_t d, int m, float inv_sqrt_d, uint32_t k0, uint32_t k1) {
+  const int64_t g4 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int r = blockIdx.y, grp = blockIdx.z;
+  if (g4 * 4 >= pitch) return;
+  float z[4];
+  normal4((uint32_t)g4, (uint32_t)grp, (uint32_t)r, kStreamDataA, k0, k1, z);
+  T* row = A + ((int64_t)grp * m + r) * pitch + g4 * 4;
+#pragma unroll
+  for (int t = 0; t < 4; ++t) {
+    const float v = (g4 * 4 + t < d) ? __fmul_rn(z[t], inv_sqrt_d) : 0.0f;
+    if constexpr (sizeof(T) == 2) row[t] = __float2bfloat16_rn(v); else row[t] = v;
+  }
+}
+
+__global__ void xstar_kernel(float* xstar, int64_t pitch, int64_t d, uint32_t k0, uint32_t k1) {
+  const int64_t g4 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (g4 * 4 >= pitch) return;
+  float z[4];
+  normal4((uint32_t)g4, 0u, 0u, kStreamXStar, k0, k1, z);
+#pragma unroll
+  for (int t = 0; t < 4; ++t) xstar[g4 * 4 + t] = (g4 * 4 + t < d) ? z[t] : 0.0f;
+}
+
+__device__ __forceinline__ float load_as_float(const float* p) { return *p; }
+__device__ __forceinline__ float load_as_float(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+
+// One CTA per (row r, data matrix g): dot(A_g[r], x*) in double, then the labels of the
+// nodes that own matrix g.
+template <typename T>
+__global__ void __launch_bounds__(256)
+lsq_labels_kernel(const T* __restrict__ A, const float* __restrict__ xstar, float* bvec, const float* __restrict__ scalars,
+                  int64_t pitch, int64_t d, int m, int nodes_per_group, float noise_std, uint32_t k0, uint32_t k1) {
+  const int r = blockIdx.x, grp = blockIdx.y;
+  const T* row = A + ((int64_t)grp * m + r) * pitch;
+  double acc = 0.0;
+  for (int64_t k = threadIdx.x; k < d; k += blockDim.x) acc += (double)load_as_float(row + k) * (double)xstar[k];
+  __shared__ double part[8];
+  acc = warp_sum(acc);
+  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x < nodes_per_group) {
+    double dot = 0.0;
+    for (int w = 0; w < 8; ++w) dot += part[w];
+    const int node = grp * nodes_per_group + threadIdx.x;
+    float z[4];
+    normal4((uint32_t)(r / 4), (uint32_t)node, 0u, kStreamDataNoise, k0, k1, z);
+    const float noise = __fmul_rn(noise_std, z[r % 4]);
+    bvec[(int64_t)node * m + r] = (float)(dot + (double)scalars[node * 3 + 2] + (double)noise);
+  }
+}
+
+// -----------------------------------------------------------------------------------------
+// Synthetic-gradient local steps: x <- x - lr * (c_i + grad_std * z), H times in one memory
+// pass; each step is its own sequence of rounded fp32 operations (no fusion across steps).
+// One thread per 4 coordinates (one generator call per step).
+// -----------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+local_synth_kernel(StoreView s, const NodeDesc* __restrict__ nodes, int H, float lr, float grad_std,
+                   const float* __restrict__ scalars) {
+  const int64_t g4 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (g4 * 4 >= s.d) return;
+  const NodeDesc nd = nodes[blockIdx.y];
+  const float c = scalars[nd.node * 3 + 1];
+  float* p = s.X + (int64_t)nd.node * s.pitch + g4 * 4;
+  float4 v = *reinterpret_cast<const float4*>(p);
+  float* x = &v.x;
+  for (int q = 0; q < H; ++q) {
+    float z[4];
+    normal4((uint32_t)g4, (uint32_t)nd.node, nd.event + (uint32_t)q, kStreamSynthGrad, s.key0, s.key1, z);
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      const float grad = __fadd_rn(c, __fmul_rn(grad_std, z[t]));
+      x[t] = __fsub_rn(x[t], __fmul_rn(lr, grad));
+    }
+  }
+#pragma unroll
+  for (int t = 0; t < 4; ++t) if (g4 * 4 + t >= s.d) x[t] = 0.0f;    // keep the row padding zero
+  *reinterpret_cast<float4*>(p) = v;
+}
+
+// -----------------------------------------------------------------------------------------
+// Least-squares local step, general d: two kernels per step.
+//   residual partials: CTA (chunk c, node t) computes for every minibatch row s the partial
+//     dot product of A[r_s] and x over its chunk of kLsqChunk coordinates;
+//   update: CTA (chunk c, node t) first sums the partials of each row in chunk order (a fixed
+//     order, so results do not depend on scheduling), forms resid_s = <A[r_s], x> - b[r_s], then
+//     x[k] -= (lr / B) * sum_s resid_s * A[r_s][k] on its chunk.
+// -----------------------------------------------------------------------------------------
+constexpr int kLsqThreads = 256;
+constexpr int kLsqPerThread = 8;
+constexpr int kLsqChunk = kLsqThreads * kLsqPerThread;   // 2048 coordinates per CTA
+constexpr int kLsqMaxBatch = 256;
+
+int64_t lsq_chunks(int64_t d) { return (d + kLsqChunk - 1) / kLsqChunk; }
+
+__device__ __forceinline__ int minibatch_row(int s_idx, int group, uint32_t event, int m, uint32_t k0, uint32_t k1) {
+  const uint4 w = philox4x32_10((uint32_t)(s_idx / 4), (uint32_t)group, event, kStreamMinibatch, k0, k1);
+  const int t = s_idx & 3;
+  const uint32_t word = t == 0 ? w.x : t == 1 ? w.y : t == 2 ? w.z : w.w;
+  return (int)uniform_int(word, (uint32_t)m);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kLsqThreads)
+lsq_residual_kernel(StoreView s, LsqView l, const NodeDesc* __restrict__ nodes, int step, float* __restrict__ partial,
+                    int64_t nchunks) {
+  const NodeDesc nd = nodes[blockIdx.y];
+  const int group = nd.node / l.nodes_per_group;
+  const uint32_t event = nd.event + (uint32_t)step;
+  const int64_t k0 = (int64_t)blockIdx.x * kLsqChunk + threadIdx.x * kLsqPerThread;
+  const float* xrow = s.X + (int64_t)nd.node * s.pitch;
+  const T* A = reinterpret_cast<const T*>(l.A) + (int64_t)group * l.m * s.pitch;
+
+  __shared__ int rows[kLsqMaxBatch];
+  __shared__ float red[kLsqThreads / 32];
+  if (threadIdx.x < l.batch) rows[threadIdx.x] = minibatch_row(threadIdx.x, group, event, l.m, s.key0, s.key1);
+  float x[kLsqPerThread];
+#pragma unroll
+  for (int t = 0; t < kLsqPerThread; ++t) x[t] = (k0 + t < s.pitch) ? xrow[k0 + t] : 0.0f;
+  __syncthreads();
+  for (int si = 0; si < l.batch; ++si) {
+    const T* row = A + (int64_t)rows[si] * s.pitch;
+    float acc = 0.0f;
+    if (k0 < s.pitch) {
+#pragma unroll
+      for (int t = 0; t < kLsqPerThread; ++t) acc = fmaf(load_as_float(row + k0 + t), x[t], acc);
+    }
+    acc = warp_sum(acc);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float tot = 0.0f;
+#pragma unroll
+      for (int w = 0; w < kLsqThreads / 32; ++w) tot += red[w];
+      partial[((int64_t)blockIdx.y * l.batch + si) * nchunks + blockIdx.x] = tot;
+    }
+    __syncthreads();
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kLsqThreads)
+lsq_update_kernel(StoreView s, LsqView l, const NodeDesc* __restrict__ nodes, int step, float lr,
+                  const float* __restrict__ partial, int64_t nchunks) {
+  const NodeDesc nd = nodes[blockIdx.y];
+  const int group = nd.node / l.nodes_per_group;
+  const uint32_t event = nd.event + (uint32_t)step;
+  const int64_t k0 = (int64_t)blockIdx.x * kLsqChunk + threadIdx.x * kLsqPerThread;
+  float* xrow = s.X + (int64_t)nd.node * s.pitch;
+  const T* A = reinterpret_cast<const T*>(l.A) + (int64_t)group * l.m * s.pitch;
+
+  __shared__ int rows[kLsqMaxBatch];
+  __shared__ float resid[kLsqMaxBatch];
+  // sum the chunk partials of each minibatch row in chunk order: one warp per row, lanes
+  // stride the chunks, then a fixed-shape shuffle tree
+  for (int si = threadIdx.x >> 5; si < l.batch; si += kLsqThreads / 32) {
+    const float* p = partial + ((int64_t)blockIdx.y * l.batch + si) * nchunks;
+    float acc = 0.0f;
+    for (int64_t c = threadIdx.x & 31; c < nchunks; c += 32) acc += p[c];
+    acc = warp_sum(acc);
+    if ((threadIdx.x & 31) == 0) {
+      const int r = minibatch_row(si, group, event, l.m, s.key0, s.key1);
+      rows[si] = r;
+      resid[si] = acc - l.bvec[(int64_t)nd.node * l.m + r];
+    }
+  }
+  __syncthreads();
+  if (k0 >= s.d) return;
+  float g[kLsqPerThread];
+#pragma unroll
+  for (int t = 0; t < kLsqPerThread; ++t) g[t] = 0.0f;
+  for (int si = 0; si < l.batch; ++si) {
+    const T* row = A + (int64_t)rows[si] * s.pitch + k0;
+    const float rs = resid[si];
+#pragma unroll
+    for (int t = 0; t < kLsqPerThread; ++t) g[t] = fmaf(rs, load_as_float(row + t), g[t]);
+  }
+  const float scale = lr / (float)l.batch;
+#pragma unroll
+  for (int t = 0; t < kLsqPerThread; ++t)
+    if (k0 + t < s.d) xrow[k0 + t] -= scale * g[t];
+}
+
+// -----------------------------------------------------------------------------------------
+// Pair sampler: draws are generated in parallel (one per thread), accepted sequentially in
+// draw order by thread 0 so that the result equals the sequential rejection procedure.
+// -----------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+sample_pairs_kernel(const int32_t* __restrict__ adj, int n, int degree, int max_pairs, uint32_t launch_ctr, uint32_t k0,
+                    uint32_t k1, int32_t* out_pairs, int32_t* out_count, uint8_t* used) {
+  __shared__ int cand_i[256], cand_j[256];
+  __shared__ int count_sh;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) used[i] = 0;
+  if (threadIdx.x == 0) count_sh = 0;
+  __syncthreads();
+  const int64_t max_attempts = 16LL * max_pairs;
+  for (int64_t base = 0; base < max_attempts; base += 256) {
+    const int64_t attempt = base + threadIdx.x;
+    if (attempt < max_attempts) {
+      const uint4 w = philox4x32_10((uint32_t)attempt, 0u, launch_ctr, kStreamPairs, k0, k1);
+      const int i = (int)uniform_int(w.x, (uint32_t)n);
+      cand_i[threadIdx.x] = i;
+      cand_j[threadIdx.x] = adj[(int64_t)i * degree + uniform_int(w.y, (uint32_t)degree)];
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int count = count_sh;
+      const int lim = (int)min((int64_t)256, max_attempts - base);
+      for (int t = 0; t < lim && count < max_pairs; ++t) {
+        const int i = cand_i[t], j = cand_j[t];
+        if (used[i] || used[j]) continue;
+        used[i] = used[j] = 1;
+        out_pairs[2 * count] = i;
+        out_pairs[2 * count + 1] = j;
+        ++count;
+      }
+      count_sh = count;
+    }
+    __syncthreads();
+    if (count_sh >= max_pairs) break;
+  }
+  if (threadIdx.x == 0) *out_count = count_sh;
+}
+
+__global__ void bf16_to_f32_kernel(const __nv_bfloat16* src, float* dst, int64_t count) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < count) dst[i] = __bfloat162float(src[i]);
+}
+__global__ void f32_to_bf16_kernel(const float* src, __nv_bfloat16* dst, int64_t count) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < count) dst[i] = __float2bfloat16_rn(src[i]);
+}
+
+// -----------------------------------------------------------------------------------------
+// Launch wrappers
+// -----------------------------------------------------------------------------------------
+static inline unsigned cdiv(int64_t a, int64_t b) { return (unsigned)((a + b - 1) / b); }
+
+cudaError_t launch_node_scalars(float* scalars_dev, int n, float offset_std, float drift_std, uint32_t key0,
+                                uint32_t key1, cudaStream_t st, int* launches) {
+  node_scalars_kernel<<<cdiv(n, 128), 128, 0, st>>>(scalars_dev, n, offset_std, drift_std, key0, key1);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_init_models(const StoreView& s, const float* scalars_dev, float init_std, cudaStream_t st,
+                               int* launches) {
+  const dim3 grid(cdiv((s.d + 3) / 4, 256), s.n);
+  init_models_kernel<<<grid, 256, 0, st>>>(s, scalars_dev, init_std);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_lsq_data(const StoreView& s, const LsqView& l, void* A, float* xstar, float* bvec,
+                            const float* scalars_dev, float noise_std, cudaStream_t st, int* launches) {
+  const float inv_sqrt_d = (float)(1.0 / sqrt((double)s.d));
+  const dim3 grid_a(cdiv(s.pitch / 4, 256), l.m, l.groups);
+  const dim3 grid_l(l.m, l.groups);
+  if (l.nodes_per_group > 256) return cudaErrorInvalidValue;
+  xstar_kernel<<<cdiv(s.pitch / 4, 256), 256, 0, st>>>(xstar, s.pitch, s.d, s.key0, s.key1);
+  if (l.dtype == 1) {
+    auto* Ab = reinterpret_cast<__nv_bfloat16*>(A);
+    lsq_matrix_kernel<<<grid_a, 256, 0, st>>>(Ab, s.pitch, s.d, l.m, inv_sqrt_d, s.key0, s.key1);
+    lsq_labels_kernel<<<grid_l, 256, 0, st>>>(Ab, xstar, bvec, scalars_dev, s.pitch, s.d, l.m, l.nodes_per_group,
+                                               noise_std, s.key0, s.key1);
+  } else {
+    auto* Af = reinterpret_cast<float*>(A);
+    lsq_matrix_kernel<<<grid_a, 256, 0, st>>>(Af, s.pitch, s.d, l.m, inv_sqrt_d, s.key0, s.key1);
+    lsq_labels_kernel<<<grid_l, 256, 0, st>>>(Af, xstar, bvec, scalars_dev, s.pitch, s.d, l.m, l.nodes_per_group,
+                                               noise_std, s.key0, s.key1);
+  }
+  *launches += 3;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_local_synth(const StoreView& s, const NodeDesc* nodes_dev, int count, int H, float lr,
+                               float grad_std, const float* scalars_dev, cudaStream_t st, int* launches) {
+  if (count == 0 || H == 0) return cudaSuccess;
+  const dim3 grid(cdiv((s.d + 3) / 4, 256), count);
+  local_synth_kernel<<<grid, 256, 0, st>>>(s, nodes_dev, H, lr, grad_std, scalars_dev);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_local_lsq(const StoreView& s, const LsqView& l, const NodeDesc* nodes_dev, int count, int H,
+                             float lr, float* partial_dev, cudaStream_t st, int* launches) {
+  if (count == 0 || H == 0) return cudaSuccess;
+  if (l.batch > kLsqMaxBatch) return cudaErrorInvalidValue;
+  const int64_t nchunks = lsq_chunks(s.d);
+  const dim3 grid((unsigned)nchunks, count);
+  for (int q = 0; q < H; ++q) {
+    if (l.dtype == 1) {
+      lsq_residual_kernel<__nv_bfloat16><<<grid, kLsqThreads, 0, st>>>(s, l, nodes_dev, q, partial_dev, nchunks);
+      lsq_update_kernel<__nv_bfloat16><<<grid, kLsqThreads, 0, st>>>(s, l, nodes_dev, q, lr, partial_dev, nchunks);
+    } else {
+      lsq_residual_kernel<float><<<grid, kLsqThreads, 0, st>>>(s, l, nodes_dev, q, partial_dev, nchunks);
+      lsq_update_kernel<float><<<grid, kLsqThreads, 0, st>>>(s, l, nodes_dev, q, lr, partial_dev, nchunks);
+    }
+    *launches += 2;
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_sample_pairs(const int32_t* adj_dev, int n, int degree, int max_pairs, uint32_t launch_ctr,
+                                uint32_t key0, uint32_t key1, int32_t* out_pairs_dev, int32_t* out_count_dev,
+                                uint8_t* used_dev, cudaStream_t st, int* launches) {
+  sample_pairs_kernel<<<1, 256, 0, st>>>(adj_dev, n, degree, max_pairs, launch_ctr, key0, key1, out_pairs_dev,
+                                         out_count_dev, used_dev);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_bf16_to_f32(const void* src, float* dst, int64_t count, cudaStream_t st, int* launches) {
+  bf16_to_f32_kernel<<<cdiv(count, 256), 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(src), dst, count);
+  ++*launches;
+  return cudaGetLastError();
+}
+cudaError_t launch_f32_to_bf16(const float* src, void* dst, int64_t count, cudaStream_t st, int* launches) {
+  f32_to_bf16_kernel<<<cdiv(count, 256), 256, 0, st>>>(src, reinterpret_cast<__nv_bfloat16*>(dst), count);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+}  // namespace swarm

@@ -1,0 +1,118 @@
+// Mean model mu = (1/n) sum_i X^i and potential Gamma = sum_i ||X^i - mu||^2 (Section 4).
+// Both stream X[n][d] once: a thread owns 4 adjacent columns and walks down the n rows.
+#include "swarm_dev.cuh"
+#include "swarm_internal.h"
+
+namespace swarm {
+
+constexpr int kRedThreads = 128;
+constexpr int kRowUnroll = 8;
+
+// mu[k]: rows summed in double in row order, divided by n, rounded once.
+__global__ void __launch_bounds__(kRedThreads)
+mean_model_kernel(StoreView s, float* __restrict__ out) {
+  const int64_t c4 = (int64_t)blockIdx.x * kRedThreads + threadIdx.x;
+  if (c4 * 4 >= s.d) return;
+  const float* col = s.X + c4 * 4;
+  double acc[4] = {0.0, 0.0, 0.0, 0.0};
+  int i = 0;
+  for (; i + kRowUnroll <= s.n; i += kRowUnroll) {
+    float4 v[kRowUnroll];
+#pragma unroll
+    for (int u = 0; u < kRowUnroll; ++u) v[u] = *reinterpret_cast<const float4*>(col + (int64_t)(i + u) * s.pitch);
+#pragma unroll
+    for (int u = 0; u < kRowUnroll; ++u) {
+      acc[0] += (double)v[u].x; acc[1] += (double)v[u].y; acc[2] += (double)v[u].z; acc[3] += (double)v[u].w;
+    }
+  }
+  for (; i < s.n; ++i) {
+    const float4 v = *reinterpret_cast<const float4*>(col + (int64_t)i * s.pitch);
+    acc[0] += (double)v.x; acc[1] += (double)v.y; acc[2] += (double)v.z; acc[3] += (double)v.w;
+  }
+  const double inv = (double)s.n;
+#pragma unroll
+  for (int t = 0; t < 4; ++t)
+    if (c4 * 4 + t < s.d) out[c4 * 4 + t] = (float)(acc[t] / inv);
+}
+
+// Per column, with the first row as shift (exact in double): s_i = x_i - x_0,
+// Gamma_col = sum s_i^2 - (sum s_i)^2 / n. The shift keeps the subtraction benign when the
+// models are close to each other but far from the origin. CTA partials go to scratch and are
+// summed by a second, single-CTA kernel in index order.
+__global__ void __launch_bounds__(kRedThreads)
+potential_partial_kernel(StoreView s, double* __restrict__ partial) {
+  const int64_t c4 = (int64_t)blockIdx.x * kRedThreads + threadIdx.x;
+  double gamma = 0.0;
+  if (c4 * 4 < s.d) {
+    const float* col = s.X + c4 * 4;
+    const float4 x0 = *reinterpret_cast<const float4*>(col);
+    const double b0 = x0.x, b1 = x0.y, b2 = x0.z, b3 = x0.w;
+    double sm[4] = {0.0, 0.0, 0.0, 0.0}, sq[4] = {0.0, 0.0, 0.0, 0.0};
+    int i = 1;
+    for (; i + kRowUnroll <= s.n; i += kRowUnroll) {
+      float4 v[kRowUnroll];
+#pragma unroll
+      for (int u = 0; u < kRowUnroll; ++u) v[u] = *reinterpret_cast<const float4*>(col + (int64_t)(i + u) * s.pitch);
+#pragma unroll
+      for (int u = 0; u < kRowUnroll; ++u) {
+        const double d0 = (double)v[u].x - b0, d1 = (double)v[u].y - b1, d2 = (double)v[u].z - b2, d3 = (double)v[u].w - b3;
+        sm[0] += d0; sm[1] += d1; sm[2] += d2; sm[3] += d3;
+        sq[0] = fma(d0, d0, sq[0]); sq[1] = fma(d1, d1, sq[1]); sq[2] = fma(d2, d2, sq[2]); sq[3] = fma(d3, d3, sq[3]);
+      }
+    }
+    for (; i < s.n; ++i) {
+      const float4 v = *reinterpret_cast<const float4*>(col + (int64_t)i * s.pitch);
+      const double d0 = (double)v.x - b0, d1 = (double)v.y - b1, d2 = (double)v.z - b2, d3 = (double)v.w - b3;
+      sm[0] += d0; sm[1] += d1; sm[2] += d2; sm[3] += d3;
+      sq[0] = fma(d0, d0, sq[0]); sq[1] = fma(d1, d1, sq[1]); sq[2] = fma(d2, d2, sq[2]); sq[3] = fma(d3, d3, sq[3]);
+    }
+    const double inv_n = 1.0 / (double)s.n;
+#pragma unroll
+    for (int t = 0; t < 4; ++t)                      // padding columns are all-zero: contribute 0
+      gamma += sq[t] - sm[t] * sm[t] * inv_n;
+  }
+  __shared__ double red[kRedThreads / 32];
+  gamma = warp_sum(gamma);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = gamma;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double tot = 0.0;
+#pragma unroll
+    for (int w = 0; w < kRedThreads / 32; ++w) tot += red[w];
+    partial[blockIdx.x] = tot;
+  }
+}
+
+__global__ void __launch_bounds__(1024)
+potential_final_kernel(const double* __restrict__ partial, int64_t count, double* __restrict__ out) {
+  double acc = 0.0;
+  for (int64_t i = threadIdx.x; i < count; i += 1024) acc += partial[i];
+  __shared__ double red[32];
+  acc = warp_sum(acc);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    double v = red[threadIdx.x];
+    v = warp_sum(v);
+    if (threadIdx.x == 0) *out = v;
+  }
+}
+
+int64_t potential_partials(int64_t d) { return ((d + 3) / 4 + kRedThreads - 1) / kRedThreads; }
+
+cudaError_t launch_mean_model(const StoreView& s, float* out_dev, cudaStream_t st, int* launches) {
+  mean_model_kernel<<<(unsigned)potential_partials(s.d), kRedThreads, 0, st>>>(s, out_dev);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_potential(const StoreView& s, double* partial_dev, double* out_dev, cudaStream_t st,
+                             int* launches) {
+  const int64_t parts = potential_partials(s.d);
+  potential_partial_kernel<<<(unsigned)parts, kRedThreads, 0, st>>>(s, partial_dev);
+  potential_final_kernel<<<1, 1024, 0, st>>>(partial_dev, parts, out_dev);
+  *launches += 2;
+  return cudaGetLastError();
+}
+
+}  // namespace swarm

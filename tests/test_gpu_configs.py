@@ -1,0 +1,92 @@
+"""Parity at the sizes of the benchmark configurations, in the launch shapes the benchmark uses.
+The oracle runs either the whole launch (where it finishes in seconds) or a sample of the pairs."""
+import numpy as np
+import pytest
+
+from oracle import swarm_oracle as o
+from paper_1910_12308_b200 import binding as g
+from tests.parity import rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+def ring_matching(n, parity, flip_bits):
+    pairs = []
+    for t in range(n // 2):
+        a, b = (2 * t + parity) % n, (2 * t + 1 + parity) % n
+        pairs.append((b, a) if (flip_bits >> t) & 1 else (a, b))
+    return np.array(pairs, dtype=np.int32)
+
+
+def test_config2_full_launch_bit_exact():
+    """n = 64, d = 2^20, ring, 32 disjoint pairs per launch, 4-bit, averaging only."""
+    n, d, bits = 64, 1 << 20, 4
+    gpu = g.Swarm(n, d, "ring", seed=2)
+    gpu.configure(offset_std=float(np.sqrt(0.1)))
+    orc = o.OracleSwarm(n, d, "ring", seed=2)
+    for i in range(n):                       # the CUDA-generated state is the common input
+        orc.X[i] = gpu.get(g.T_X, i)
+    assert abs(float(orc.X.std()) - np.sqrt(0.01 + 0.1)) < 0.1
+    for launch in range(2):
+        pairs = ring_matching(n, launch & 1, 0x5A5A5A5A >> launch)
+        assert gpu.interact(pairs, bits) == 0
+        assert orc.interact(pairs, bits, threads=8) == 0
+    for i in range(n):
+        assert np.array_equal(gpu.get(g.T_X, i).view(np.uint32), orc.X[i].view(np.uint32))
+        assert np.array_equal(gpu.get(g.T_CODES, i)[: orc.nblk * 128 * bits], orc.packed_codes(i, bits))
+        assert np.array_equal(gpu.get(g.T_EXPS, i), orc.exps[i])
+    assert abs(gpu.potential() - orc.potential()) <= 1e-9 * orc.potential()
+
+
+@pytest.mark.parametrize("d,bits,mode", [(11_689_512, 8, 1), (25_557_032, 4, 0), (25_557_032, 8, 0)])
+def test_large_model_sampled_pair_bit_exact(d, bits, mode):
+    """ResNet-18 / ResNet-50 sized vectors (ragged tail blocks of 552 and 40 coordinates): the CUDA
+    path runs a full launch, the oracle recomputes one of its pairs."""
+    n = 4
+    cfg = dict(objective=1, nonblocking=mode, grad_std=float(np.sqrt(1e-3)), drift_std=float(np.sqrt(0.05)))
+    gpu = g.Swarm(n, d, "complete", seed=3)
+    gpu.configure(**cfg)
+    orc = o.OracleSwarm(n, d, "complete", seed=3)
+    orc.configure(objective=1, nonblocking=mode, grad_std=0.0, drift_std=0.0, init_std=0.0)
+    assert gpu.local_steps([0, 1, 2, 3], 2, 0.05) == 0
+    if mode == 1:
+        assert gpu.publish(bits) == 0
+        assert gpu.local_steps([0, 1, 2, 3], 1, 0.05) == 0
+    for i in range(n):
+        orc.X[i] = gpu.get(g.T_X, i)
+        if mode == 1:
+            orc.B[i] = gpu.get(g.T_B, i)
+            orc.codes[i] = gpu.get(g.T_CODES, i)
+            orc.exps[i] = gpu.get(g.T_EXPS, i)
+            orc.pbits[i] = bits
+        orc.w[i] = gpu.get(g.T_COUNTERS, i)[0]
+    assert gpu.interact([[2, 0], [1, 3]], bits, mode) == 0
+    assert orc.interact([[1, 3]], bits, mode) == 0            # one of the launch's pairs
+    for i in (1, 3):
+        assert np.array_equal(gpu.get(g.T_X, i).view(np.uint32), orc.X[i].view(np.uint32))
+        assert np.array_equal(gpu.get(g.T_CODES, i)[: orc.nblk * 128 * bits], orc.packed_codes(i, bits))
+        assert np.array_equal(gpu.get(g.T_EXPS, i), orc.exps[i])
+        if mode == 1:
+            assert np.array_equal(gpu.get(g.T_B, i).view(np.uint32), orc.B[i].view(np.uint32))
+    # tail padding of the communication buffer stays zero
+    assert not gpu.get(g.T_CODES, 1)[d * bits // 8: orc.nblk * 128 * bits].any()
+
+
+def test_config1_trajectory_teacher_forced():
+    """n = 8, d = 4096, least squares 64 x 4096, H = 2, batch 16, lr = 0.05, 8-bit, one pair per
+    interaction, seed 0: local steps within tolerance, interactions bit-exact."""
+    from tests.parity import assert_store_equal, inject, make_pair
+    cfg = dict(objective=2, lsq_m=64, lsq_batch=16, lsq_dtype=0, lsq_groups=0, lsq_noise_std=float(np.sqrt(0.1)))
+    orc, gpu = make_pair(8, 4096, "complete", seed=0, **cfg)
+    inject(orc, gpu)
+    for t in range(40):
+        pairs = orc.sample_pairs(1)
+        assert np.array_equal(gpu.sample_pairs(1), pairs)
+        nodes = pairs.reshape(-1)
+        assert orc.local_steps(nodes, 2, 0.05) == 0 and gpu.local_steps(nodes, 2, 0.05) == 0
+        for i in nodes:
+            assert rel_err(gpu.get(g.T_X, i), orc.X[i]) < 1e-6
+        inject(orc, gpu, what=("X",))
+        assert orc.interact(pairs, 8) == 0 and gpu.interact(pairs, 8) == 0
+    assert_store_equal(orc, gpu, 8)
+    assert abs(gpu.potential() - orc.potential()) <= 1e-9 * orc.potential()

@@ -1,0 +1,265 @@
+"""Parity of the CUDA path against the CPU oracle, through the C ABI, on identical seeded inputs.
+
+Bar: bit-exact for codes, packed bytes, exponents, counters, pair schedules and the fp32 outputs of
+the interaction (every operation there is a single IEEE operation on both sides); max relative
+error 1e-6 (max |diff| / max |ref| per row) for what involves transcendental functions or long
+fp32 accumulations (normals, local steps, generated data)."""
+import numpy as np
+import pytest
+
+from oracle import swarm_oracle as o
+from paper_1910_12308_b200 import binding as g
+from tests.parity import assert_store_equal, inject, make_pair, rel_err
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-6
+
+
+def disjoint_pairs(orc, rng, count):
+    """Random disjoint directed edges of the oracle's graph."""
+    used, out = set(), []
+    order = rng.permutation(orc.n)
+    for a in order:
+        if a in used:
+            continue
+        nbrs = [int(b) for b in orc.adj[a] if int(b) not in used and int(b) != a]
+        if not nbrs:
+            continue
+        b = nbrs[int(rng.integers(len(nbrs)))]
+        out.append((int(a), b))
+        used.update((int(a), b))
+        if len(out) == count:
+            break
+    return np.array(out, dtype=np.int32)
+
+
+# ---- state generation ----------------------------------------------------------------------------
+
+@pytest.mark.parametrize("topo,deg,n", [("complete", 0, 5), ("ring", 0, 9), ("regular", 4, 32), ("regular", 8, 256)])
+def test_topology_matches(topo, deg, n):
+    orc, gpu = make_pair(n, 8, topo, deg, seed=11)
+    assert np.array_equal(gpu.get_all(g.T_ADJ), orc.adj)
+
+
+def test_initial_state_matches_within_tolerance():
+    orc, gpu = make_pair(6, 5003, seed=3, init_std=0.1, offset_std=0.3, drift_std=0.2, objective=1, grad_std=0.03,
+                         nonblocking=1)
+    for i in range(6):
+        assert rel_err(gpu.get(g.T_X, i), orc.X[i]) < TOL
+        assert rel_err(gpu.get(g.T_B, i), orc.B[i]) < TOL
+        sc = gpu.get(g.T_SCALARS, i)
+        assert abs(sc[0] - orc.offset[i]) <= 1e-6 * 0.3 * 4 and abs(sc[1] - orc.drift[i]) <= 1e-6 * 0.2 * 4
+        assert sc[2] == orc.shift[i]
+
+
+@pytest.mark.parametrize("dtype,groups", [(0, 0), (1, 2)])
+def test_lsq_data_matches_within_tolerance(dtype, groups):
+    orc, gpu = make_pair(4, 3000, seed=5, objective=2, lsq_m=6, lsq_batch=4, lsq_dtype=dtype, lsq_groups=groups,
+                         lsq_noise_std=float(np.sqrt(0.1)))
+    assert rel_err(gpu.get(g.T_XSTAR), orc.xstar) < TOL
+    for grp in range(orc.groups):
+        got = gpu.get(g.T_A, grp).reshape(6, 3000)
+        if dtype == 0:
+            assert rel_err(got, orc.A[grp]) < TOL
+        else:   # bf16 storage: a 1-ulp fp32 difference before rounding may flip a bf16 rounding
+            diff = np.abs(got - orc.A[grp])
+            assert (diff > 0).mean() < 1e-3 and diff.max() <= 2.0**-8 * np.abs(orc.A[grp]).max()
+    for i in range(4):
+        assert rel_err(gpu.get(g.T_BVEC, i), orc.bvec[i]) < 5e-6 if dtype else rel_err(gpu.get(g.T_BVEC, i), orc.bvec[i]) < TOL
+
+
+# ---- pair schedule -------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("topo,deg,n,P", [("ring", 0, 64, 32), ("regular", 4, 32, 16), ("complete", 0, 16, 8),
+                                          ("regular", 8, 256, 128), ("complete", 0, 8, 1), ("ring", 0, 5, 7)])
+def test_pair_schedule_is_bit_exact(topo, deg, n, P):
+    orc, gpu = make_pair(n, 8, topo, deg, seed=2)
+    for _ in range(12):
+        assert np.array_equal(gpu.sample_pairs(P), orc.sample_pairs(P))
+    assert gpu.get_state()[0] == 12
+
+
+# ---- blocking interaction ------------------------------------------------------------------------
+
+@pytest.mark.parametrize("bits", [2, 4, 8, 32])
+@pytest.mark.parametrize("d", [1, 7, 1024, 1030, 2049, 5000])
+def test_blocking_interaction_bit_exact(bits, d):
+    n = 6
+    orc, gpu = make_pair(n, d, "complete", seed=100 + d, offset_std=0.05)
+    inject(orc, gpu)
+    rng = np.random.default_rng(d + bits)
+    for rnd in range(4):
+        pairs = disjoint_pairs(orc, rng, int(rng.integers(1, 4)))
+        assert orc.interact(pairs, bits) == 0
+        assert gpu.interact(pairs, bits) == 0
+        assert_store_equal(orc, gpu, bits)
+
+
+@pytest.mark.parametrize("bits", [2, 4, 8])
+def test_blocking_interaction_special_values(bits):
+    """Identical models, zeros, huge and tiny magnitudes, and widely separated models."""
+    n, d = 4, 3000
+    orc, gpu = make_pair(n, d, "complete", seed=1)
+    rng = np.random.default_rng(bits)
+    X = orc.X
+    X[1] = X[0]                                   # rho = 0: magnitude clamp only
+    X[2] = 0.0
+    X[3] = 0.0
+    X[3, 5] = 1e-40                               # subnormal range
+    inject(orc, gpu)
+    for pairs in ([[0, 1], [2, 3]], [[0, 2], [1, 3]]):
+        assert orc.interact(pairs, bits) == 0 and gpu.interact(pairs, bits) == 0
+        assert_store_equal(orc, gpu, bits)
+    X[0] = (rng.normal(size=d) * 1e30).astype(np.float32)
+    X[1] = (rng.normal(size=d) * 1e-30).astype(np.float32)
+    X[2] = (rng.normal(size=d) * 1e37).astype(np.float32)
+    X[3] = X[2] * np.float32(1 + 2.0**-20)
+    X[2, 100:200] = np.float32(2.0) ** rng.integers(-126, 100, 100)      # exact powers of two
+    inject(orc, gpu, what=("X",))
+    for pairs in ([[0, 1], [2, 3]], [[1, 2], [3, 0]]):
+        assert orc.interact(pairs, bits) == 0 and gpu.interact(pairs, bits) == 0
+        assert_store_equal(orc, gpu, bits)
+
+
+def test_blocking_interaction_on_ring_and_many_rounds():
+    n, d, bits = 8, 2500, 4
+    orc, gpu = make_pair(n, d, "ring", seed=8, offset_std=0.1)
+    inject(orc, gpu)
+    for rnd in range(12):
+        pairs = orc.sample_pairs(4)
+        assert np.array_equal(gpu.sample_pairs(4), pairs)
+        assert orc.interact(pairs, bits) == 0 and gpu.interact(pairs, bits) == 0
+    assert_store_equal(orc, gpu, bits)
+    assert abs(gpu.potential() - orc.potential()) <= 1e-9 * orc.potential()
+
+
+# ---- non-blocking interaction --------------------------------------------------------------------
+
+@pytest.mark.parametrize("bits", [2, 4, 8])
+@pytest.mark.parametrize("d", [5, 1024, 3001])
+def test_publish_and_nonblocking_interaction_bit_exact(bits, d):
+    n = 6
+    cfg = dict(objective=1, nonblocking=1, grad_std=0.03, drift_std=0.1, offset_std=0.02)
+    orc, gpu = make_pair(n, d, "regular", 4, seed=40 + d, **cfg)
+    inject(orc, gpu)
+    assert orc.publish(bits) == 0 and gpu.publish(bits) == 0
+    assert_store_equal(orc, gpu, bits)
+    rng = np.random.default_rng(bits * 1000 + d)
+    for rnd in range(5):
+        nodes = rng.permutation(n)[: int(rng.integers(1, n + 1))]
+        assert orc.local_steps(nodes, 2, 0.05) == 0 and gpu.local_steps(nodes, 2, 0.05) == 0
+        for i in nodes:
+            assert rel_err(gpu.get(g.T_X, i), orc.X[i]) < TOL
+        inject(orc, gpu, what=("X",))                      # teacher forcing after the transcendental step
+        pairs = disjoint_pairs(orc, rng, int(rng.integers(1, 4)))
+        assert orc.interact(pairs, bits, o.NONBLOCKING) == 0
+        assert gpu.interact(pairs, bits, g.NONBLOCKING) == 0
+        assert_store_equal(orc, gpu, bits)
+
+
+def test_nonblocking_auto_publish_and_mode_switch():
+    n, d = 4, 2100
+    cfg = dict(objective=1, nonblocking=1, grad_std=0.0, drift_std=0.0, offset_std=0.05)
+    orc, gpu = make_pair(n, d, "complete", seed=7, **cfg)
+    inject(orc, gpu)
+    seq = [([[0, 1]], 8, 1), ([[2, 3], [1, 0]], 8, 1), ([[0, 2]], 8, 0), ([[3, 1]], 4, 1), ([[1, 2]], 4, 1),
+           ([[0, 3]], 32, 0), ([[2, 0]], 4, 1)]
+    for pairs, bits, mode in seq:
+        assert orc.interact(pairs, bits, mode) == 0 and gpu.interact(pairs, bits, mode) == 0
+        assert_store_equal(orc, gpu, bits)
+
+
+def test_nonblocking_far_key_alias_matches():
+    """A key outside the decode window is defined behaviour (a lattice point of the same colour
+    near the key); both sides must produce the same alias, including saturated conversions."""
+    n, d, bits = 4, 1500, 4
+    cfg = dict(objective=1, nonblocking=1, grad_std=0.0, drift_std=0.0)
+    orc, gpu = make_pair(n, d, "complete", seed=9, **cfg)
+    orc.publish(bits)
+    orc.B[0] += np.float32(3.0)                  # move one snapshot far from what its buffer encodes
+    orc.X[0] = orc.B[0]
+    orc.B[1, :700] = np.float32(1e30)            # key * 2^-e overflows int32
+    orc.X[1] = orc.B[1]
+    inject(orc, gpu)
+    for pairs in ([[0, 2]], [[1, 3]], [[2, 0], [3, 1]]):
+        assert orc.interact(pairs, bits, o.NONBLOCKING) == 0 and gpu.interact(pairs, bits, g.NONBLOCKING) == 0
+        assert_store_equal(orc, gpu, bits)
+
+
+# ---- local steps ---------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("d,H", [(3, 1), (4099, 3)])
+def test_synthetic_gradient_steps_within_tolerance(d, H):
+    cfg = dict(objective=1, grad_std=float(np.sqrt(1e-3)), drift_std=float(np.sqrt(0.05)))
+    orc, gpu = make_pair(5, d, seed=21, **cfg)
+    inject(orc, gpu)
+    for rnd in range(3):
+        assert orc.local_steps([4, 1, 2], H, 0.05) == 0 and gpu.local_steps([4, 1, 2], H, 0.05) == 0
+        for i in range(5):
+            assert rel_err(gpu.get(g.T_X, i), orc.X[i]) < TOL
+        assert [gpu.get(g.T_COUNTERS, i)[1] for i in range(5)] == orc.ls.tolist()
+    # untouched nodes are bit-identical
+    assert np.array_equal(gpu.get(g.T_X, 0), orc.X[0]) and np.array_equal(gpu.get(g.T_X, 3), orc.X[3])
+
+
+@pytest.mark.parametrize("d,m,batch,dtype,groups", [(4096, 64, 16, 0, 0), (5000, 12, 5, 0, 0), (9000, 32, 64, 1, 2),
+                                                   (300, 8, 3, 1, 0)])
+def test_least_squares_steps_within_tolerance(d, m, batch, dtype, groups):
+    cfg = dict(objective=2, lsq_m=m, lsq_batch=batch, lsq_dtype=dtype, lsq_groups=groups,
+               lsq_noise_std=float(np.sqrt(0.1)))
+    orc, gpu = make_pair(4, d, seed=31, **cfg)
+    inject(orc, gpu)
+    for rnd in range(3):
+        nodes = [0, 3, 1] if rnd else [2]
+        assert orc.local_steps(nodes, 2, 0.05) == 0 and gpu.local_steps(nodes, 2, 0.05) == 0
+        for i in range(4):
+            assert rel_err(gpu.get(g.T_X, i), orc.X[i]) < TOL, (rnd, i)
+        inject(orc, gpu, what=("X",))
+
+
+# ---- mean model and potential ----------------------------------------------------------------------
+
+@pytest.mark.parametrize("n,d", [(2, 1), (3, 1027), (8, 4096), (17, 2500), (64, 3000)])
+def test_mean_model_and_potential(n, d):
+    orc, gpu = make_pair(n, d, seed=n, offset_std=0.5)
+    inject(orc, gpu)
+    mu = gpu.mean_model().cpu().numpy()
+    assert np.array_equal(mu, orc.mean_model())
+    assert abs(gpu.potential() - orc.potential()) <= 1e-12 * orc.potential()
+    # models far from the origin but close together: the subtraction must stay benign
+    orc.X[:] = (1000.0 + 1e-3 * np.random.default_rng(0).normal(size=(n, d))).astype(np.float32)
+    inject(orc, gpu, what=("X",))
+    assert abs(gpu.potential() - orc.potential()) <= 1e-9 * orc.potential()
+    orc.X[:] = orc.X[0]
+    inject(orc, gpu, what=("X",))
+    assert gpu.potential() == 0.0 and orc.potential() == 0.0
+
+
+# ---- error behaviour -------------------------------------------------------------------------------
+
+def test_rejected_calls_change_nothing():
+    orc, gpu = make_pair(6, 2000, "ring", seed=4, objective=1, grad_std=0.1)
+    inject(orc, gpu)
+    before = gpu.get_all(g.T_X)
+    launches = gpu.kernel_launches()
+    assert gpu.interact([[0, 1], [1, 2]], 8) == -3
+    assert gpu.interact([[0, 0]], 8) == -3
+    assert gpu.interact([[0, 3]], 8) == -3
+    assert gpu.interact([[0, 6]], 8) == -2
+    assert gpu.interact([[0, 1]], 3) == -1
+    assert gpu.interact([[0, 1]], 8, 2) == -1
+    assert gpu.interact([[0, 1]], 32, g.NONBLOCKING) == -1
+    assert gpu.interact([[0, 1]], 8, g.NONBLOCKING) == -4
+    assert gpu.publish(8) == -4
+    assert gpu.local_steps([0, 0], 1, 0.1) == -1
+    assert gpu.local_steps([6], 1, 0.1) == -2
+    assert gpu.local_steps([0], -1, 0.1) == -1
+    assert gpu.kernel_launches() == launches
+    assert np.array_equal(gpu.get_all(g.T_X), before)
+    assert [tuple(gpu.get(g.T_COUNTERS, i)) for i in range(6)] == [(0, 0, 0)] * 6
+    gpu2 = g.Swarm(4, 16)
+    assert gpu2.local_steps([0], 1, 0.1) == -4
+    for bad in (dict(topology="ring", n=2), dict(topology="regular", n=8, degree=3)):
+        with pytest.raises(g.SwarmError):
+            g.Swarm(bad["n"], 16, bad["topology"], bad.get("degree", 0))
+    assert gpu.interact([], 8) == 0 and gpu.local_steps([], 3, 0.1) == 0
