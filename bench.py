@@ -1,0 +1,383 @@
+"""Benchmark of the pairwise gossip interaction path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+A step is one launch of the hot path over one batch of disjoint pairs: (local steps, if the
+workload has them) -> fused quantize / exchange / average over all pairs of the launch. The metric is
+gossip interactions per second (pairs processed / time); the roofline object reports the fused
+interaction kernel against the measured HBM copy bandwidth. With N > 1 every rank runs an independent
+replica of the workload on its own GPU (the method is single-GPU: no data-path collective).
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "gossip interactions/sec and fused-interaction HBM GB/s (% of B200 peak) at 1 GPU"
+UNIT = "interactions/s"
+
+# Synthetic workloads shaped like the paper's (flat model vectors, 8..256 nodes, 2..8-bit codes).
+WORKLOADS = {
+    # n = 64 nodes, d = 2^20, ring, 32 disjoint pairs per launch, 4-bit codes, averaging only.
+    "ring64_d1m_b4": dict(n=64, d=1 << 20, topology="ring", degree=0, pairs=32, bits=4, mode=0, H=0, lr=0.0, seed=2,
+                          cfg=dict(offset_std=float(np.sqrt(0.1)))),
+    # n = 16 nodes, d = 25,557,032 (ResNet-50 sized), complete graph, 8 pairs, synthetic-gradient steps.
+    "complete16_resnet50_b8": dict(n=16, d=25_557_032, topology="complete", degree=0, pairs=8, bits=8, mode=0, H=2,
+                                   lr=0.05, seed=4, cfg=dict(objective=1, grad_std=float(np.sqrt(1e-3)),
+                                                             drift_std=float(np.sqrt(0.05)))),
+    "complete16_resnet50_b4": dict(n=16, d=25_557_032, topology="complete", degree=0, pairs=8, bits=4, mode=0, H=2,
+                                   lr=0.05, seed=4, cfg=dict(objective=1, grad_std=float(np.sqrt(1e-3)),
+                                                             drift_std=float(np.sqrt(0.05)))),
+    # n = 32 nodes, d = 11,689,512 (ResNet-18 sized), random 4-regular graph, non-blocking, 8-bit.
+    "regular32_resnet18_b8_nb": dict(n=32, d=11_689_512, topology="regular", degree=4, pairs=16, bits=8, mode=1, H=3,
+                                     lr=0.05, seed=3, cfg=dict(objective=1, nonblocking=1,
+                                                               grad_std=float(np.sqrt(1e-3)))),
+    # small case the CPU checker finishes in seconds
+    "complete8_d4096_b8_lsq": dict(n=8, d=4096, topology="complete", degree=0, pairs=1, bits=8, mode=0, H=2, lr=0.05,
+                                   seed=0, cfg=dict(objective=2, lsq_m=64, lsq_batch=16, lsq_dtype=0, lsq_groups=0,
+                                                    lsq_noise_std=float(np.sqrt(0.1)))),
+}
+DEFAULT_WORKLOAD = "ring64_d1m_b4"
+
+
+def interaction_bytes(d, bits, mode):
+    """Algorithmic bytes one interaction must move: blocking reads two models, writes two models and
+    two packed buffers; non-blocking reads model + snapshot + two buffers and writes the same."""
+    nblk = (d + 1023) // 1024
+    if mode == 0:
+        return d * 16 + 2 * d * bits // 8 + 2 * nblk
+    return d * 16 + 4 * d * bits // 8 + 4 * nblk
+
+
+class PairSchedule:
+    """Deterministic full matchings for the launch shapes of the workloads (host-side list making
+    only; the library validates disjointness and adjacency)."""
+
+    def __init__(self, wl, adj):
+        self.wl, self.adj, self.rng = wl, adj, np.random.default_rng(wl["seed"])
+        self.step = 0
+
+    def next(self):
+        wl, n, P = self.wl, self.wl["n"], self.wl["pairs"]
+        if wl["topology"] == "ring":
+            parity = self.step & 1
+            flips = self.rng.integers(0, 2, P)
+            pairs = []
+            for t in range(P):
+                a, b = (2 * t + parity) % n, (2 * t + 1 + parity) % n
+                pairs.append((b, a) if flips[t] else (a, b))
+        elif wl["topology"] == "complete":
+            perm = self.rng.permutation(n)
+            pairs = [(int(perm[2 * t]), int(perm[2 * t + 1])) for t in range(P)]
+        else:   # greedy random matching on the graph
+            used, pairs = set(), []
+            for a in self.rng.permutation(n):
+                if int(a) in used:
+                    continue
+                free = [int(b) for b in self.adj[a] if int(b) not in used]
+                if not free:
+                    continue
+                b = free[int(self.rng.integers(len(free)))]
+                used.update((int(a), b))
+                pairs.append((int(a), b))
+                if len(pairs) == P:
+                    break
+        self.step += 1
+        return np.array(pairs, dtype=np.int32)
+
+
+class ClockSampler(threading.Thread):
+    """Polls SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
+        self._halt = threading.Event()
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        names = {
+            nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap",
+            nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+            nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+            nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+            nv.nvmlClocksThrottleReasonHwPowerBrakeSlowdown: "hw_power_brake",
+        }
+        while not self._halt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.005)
+
+    def stop(self):
+        self._halt.set()
+        self.join(timeout=2)
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+# ---------------------------------------------------------------------------------------------------
+# CPU checker timing (reported baseline; also the whole of --impl reference)
+# ---------------------------------------------------------------------------------------------------
+def time_oracle(wl, budget_s, max_launches, threads=None):
+    from oracle import swarm_oracle as o
+    cores = len(os.sched_getaffinity(0))
+    T = min(wl["pairs"], cores) if threads is None else threads
+    orc = o.OracleSwarm(wl["n"], wl["d"], wl["topology"], wl["degree"], wl["seed"])
+    if wl["cfg"]:
+        orc.configure(**wl["cfg"])
+    sched = PairSchedule(wl, orc.adj)
+    done, t_total, launches = 0, 0.0, 0
+    while launches < max_launches and (t_total < budget_s or launches == 0):
+        pairs = sched.next()
+        t0 = time.perf_counter()
+        if wl["H"] > 0:
+            orc.local_steps(pairs.reshape(-1), wl["H"], wl["lr"])
+        rc = orc.interact(pairs, wl["bits"], wl["mode"], threads=T)
+        t_total += time.perf_counter() - t0
+        assert rc == 0
+        done += len(pairs)
+        launches += 1
+    return done / t_total, T, launches, t_total
+
+
+def run_reference(args, wl, name):
+    """Times the CPU checker as it stands. Every step is a bounded sample of one launch: the first
+    p pairs of the launch's pair list at full d, p chosen from a calibration interaction so that K
+    steps end within a few minutes."""
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    K, W = args.steps, args.warmup
+    from oracle import swarm_oracle as o
+    cores = len(os.sched_getaffinity(0))
+    orc = o.OracleSwarm(wl["n"], wl["d"], wl["topology"], wl["degree"], wl["seed"])
+    if wl["cfg"]:
+        orc.configure(**wl["cfg"])
+    sched = PairSchedule(wl, orc.adj)
+
+    def step(p, T):
+        pairs = sched.next()[:p]
+        if wl["H"] > 0:
+            orc.local_steps(pairs.reshape(-1), wl["H"], wl["lr"])
+        assert orc.interact(pairs, wl["bits"], wl["mode"], threads=T) == 0
+        return len(pairs)
+    t0 = time.perf_counter()
+    step(1, 1)                                     # calibration (also the first warm-up step)
+    t1 = time.perf_counter() - t0
+    budget = 150.0
+    p = int(max(1, min(wl["pairs"], cores, budget / (K * t1))))
+    T = p
+    for _ in range(min(W, 3) - 1):
+        step(p, T)
+    t0 = time.perf_counter()
+    done = sum(step(p, T) for _ in range(K))
+    dt = time.perf_counter() - t0
+    value = done / dt
+    sample = (f"each step = the first {p} of the launch's {wl['pairs']} pairs at full d on {T} host threads "
+              f"(std::thread over disjoint pairs); {K} steps")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": K,
+        "warmup": min(W, 3), "ms_per_step": 1e3 * dt / K, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": name, **{k: wl[k] for k in ("n", "d", "topology", "pairs", "bits", "mode", "H")}},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": T, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ---------------------------------------------------------------------------------------------------
+# CUDA arm
+# ---------------------------------------------------------------------------------------------------
+def run_ours(args, wl, name):
+    import torch
+    from paper_1910_12308_b200 import binding as g
+
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench: no CUDA device (the library has no CPU path)")
+    torch.cuda.set_device(local_rank)
+    use_dist = world > 1
+    if use_dist:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    stream = torch.cuda.current_stream()
+    sw = g.Swarm(wl["n"], wl["d"], wl["topology"], wl["degree"], wl["seed"] + 1000 * rank, stream=stream)
+    if wl["cfg"]:
+        sw.configure(**wl["cfg"])
+    adj = sw.get_all(g.T_ADJ)
+    sched = PairSchedule(wl, adj)
+    K, W = args.steps, args.warmup
+    launches = [sched.next() for _ in range(K + W)]
+    npairs_total = sum(len(p) for p in launches[W:])
+
+    def step(pairs):
+        if wl["H"] > 0:
+            rc = sw.local_steps(pairs.reshape(-1), wl["H"], wl["lr"])
+            assert rc == 0, rc
+        rc = sw.interact(pairs, wl["bits"], wl["mode"])
+        assert rc == 0, rc
+
+    def barrier():
+        if use_dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing
+    for pairs in launches[:W]:
+        step(pairs)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    l0 = sw.kernel_launches()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev_mid = []
+    ev0.record(stream)
+    for pairs in launches[W:]:
+        if wl["H"] > 0:
+            assert sw.local_steps(pairs.reshape(-1), wl["H"], wl["lr"]) == 0
+            e_a, e_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e_a.record(stream)
+            assert sw.interact(pairs, wl["bits"], wl["mode"]) == 0
+            e_b.record(stream)
+            ev_mid.append((e_a, e_b))
+        else:
+            assert sw.interact(pairs, wl["bits"], wl["mode"]) == 0
+    ev1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    gpu_launches = sw.kernel_launches() - l0
+    ms = ev0.elapsed_time(ev1)
+    if use_dist:
+        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    value = world * npairs_total / (ms * 1e-3)
+
+    # fused interaction kernel: average launch duration inside the timed region
+    if ev_mid:
+        kern_ms = sum(a.elapsed_time(b) for a, b in ev_mid) / len(ev_mid)
+    else:
+        kern_ms = ms / K
+    per_launch_bytes = interaction_bytes(wl["d"], wl["bits"], wl["mode"]) * npairs_total / K
+    achieved = per_launch_bytes / (kern_ms * 1e-3) / 1e9
+    peak, peak_kind = measured_peak()
+
+    # ---- end to end through the C ABI with host buffers: pair lists come from pinned host memory,
+    # the step's result (block exponents of the first initiator) is read back every step, the potential
+    # every 32 steps.
+    e2e_steps = min(K, 2000)
+    pinned = [torch.from_numpy(p.copy()).pin_memory() for p in launches[W:W + e2e_steps]]
+    barrier()
+    d2h = 0
+    t0 = time.perf_counter()
+    ev0.record(stream)
+    for i, pt in enumerate(pinned):
+        pairs = pt.numpy()
+        step(pairs)
+        ex = sw.get(g.T_EXPS, int(pairs[0, 0]))
+        d2h += ex.nbytes
+        if i % 32 == 31:
+            sw.potential()
+            d2h += 8
+    ev1.record(stream)
+    barrier()
+    e2e_ms = ev0.elapsed_time(ev1)
+    wall_ms = (time.perf_counter() - t0) * 1e3
+    e2e_ms = max(e2e_ms, wall_ms)
+    if use_dist:
+        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_pairs = sum(len(p) for p in launches[W:W + e2e_steps])
+    e2e = {"value": world * e2e_pairs / (e2e_ms * 1e-3), "unit": UNIT,
+           "h2d_bytes_per_step": int(np.mean([len(p) * 16 for p in launches[W:W + e2e_steps]])),
+           "d2h_bytes_per_step": int(d2h / e2e_steps)}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": name, **{k: wl[k] for k in ("n", "d", "topology", "pairs", "bits", "mode", "H")},
+                   "l2": "inputs larger than L2: every launch streams all models it touches from HBM",
+                   "replicas": world},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(gpu_launches),
+        "roofline": {"bound": "hbm", "kernel": "interact_blocking_kernel" if wl["mode"] == 0 else "interact_nonblocking_kernel",
+                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": peak_kind, "frac_of_8000": achieved / 8000.0, "traffic": TRAFFIC.get(name),
+                     "algorithmic_bytes_per_launch": per_launch_bytes, "kernel_ms": kern_ms},
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, T, nl, tt = time_oracle(wl, budget_s=10.0, max_launches=40)
+        v1, _, nl1, tt1 = time_oracle(wl, budget_s=3.0, max_launches=1, threads=1)
+        out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": T, "kind": "oracle",
+                               "sample": f"{nl} launches of {wl['pairs']} pairs at full d ({tt:.1f} s) on {T} host threads",
+                               "single_thread_value": v1}
+    if use_dist:
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(out))
+
+
+# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel (see profiles/);
+# None until a capture of the current kernel exists.
+TRAFFIC = {"ring64_d1m_b4": 512.1e6}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    wl = WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl, args.workload)
+    else:
+        run_ours(args, wl, args.workload)
+
+
+if __name__ == "__main__":
+    main()
