@@ -167,6 +167,26 @@ int swarm_set_state(swarm_ctx *ctx, uint32_t launch, int32_t b_stale);
  * Valid until the next swarm_configure / swarm_destroy. */
 int swarm_model_ptr(swarm_ctx *ctx, float **x_dev, int64_t *pitch);
 
+/* Potential of caller-held models with no allocation of any kind (the paper has no counterpart: this
+ * exists for callers that are not allowed to allocate). Meant for code that owns all its device memory
+ * up front -- a process with a fixed memory pool, a hook running inside another component's step, a host
+ * framework that passes only raw pointers -- and therefore cannot create a context (contexts allocate
+ * their scratch) or tolerate cudaMalloc's device-wide synchronisation and late failure.
+ *   x_dev          n rows of d floats, row i at x_dev + i*pitch (device memory, read only; pitch >= d,
+ *                  in elements; rows 16-byte aligned and pitch a multiple of 4 take the fast path)
+ *   out_gamma_dev  one double in device memory, written asynchronously on cuda_stream
+ *   cuda_stream    cudaStream_t (NULL = default stream) on the current device
+ * Gamma = sum_i ||X^i - mu||^2 as in swarm_potential, same arithmetic. The per-CTA partial sums live in a
+ * fixed 512 KiB array inside the library image (every GPU that loads the library holds it until the
+ * process exits), which caps the size: d <= SWARM_STATIC_MAX_D, otherwise SWARM_EINVAL and nothing is
+ * launched. All calls share that array: calls on one stream are ordered and safe, calls that may overlap
+ * on the same GPU race on it. The first call made with a given device current looks up the array's
+ * device address (no allocation); make that first call before starting any stream capture.
+ * Errors: EINVAL (NULL pointer, n < 2, d < 1, pitch < d, d > SWARM_STATIC_MAX_D), ECUDA. */
+#define SWARM_STATIC_MAX_D 33554432
+int swarm_potential_static(const float *x_dev, int32_t n, int64_t d, int64_t pitch, double *out_gamma_dev,
+                           void *cuda_stream);
+
 int swarm_set_stream(swarm_ctx *ctx, void *cuda_stream);   /* cudaStream_t; NULL = default stream */
 int swarm_sync(swarm_ctx *ctx);
 int64_t swarm_kernel_launches(swarm_ctx *ctx);             /* kernels launched so far by this context */

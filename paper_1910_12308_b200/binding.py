@@ -24,7 +24,7 @@ EXPORTS = [
     "swarm_set_allocator", "swarm_init", "swarm_local_steps", "swarm_interact", "swarm_mean_model",
     "swarm_potential", "swarm_configure", "swarm_sample_pairs", "swarm_publish", "swarm_get_tensor",
     "swarm_set_tensor", "swarm_get_state", "swarm_set_state", "swarm_model_ptr", "swarm_set_stream",
-    "swarm_sync", "swarm_kernel_launches", "swarm_last_cuda_error", "swarm_strerror", "swarm_destroy",
+    "swarm_sync", "swarm_potential_static", "swarm_kernel_launches", "swarm_last_cuda_error", "swarm_strerror", "swarm_destroy",
 ]
 
 
@@ -88,6 +88,7 @@ def load():
         "swarm_get_state": (C.c_int, [vp, C.POINTER(u32), C.POINTER(i32)]),
         "swarm_set_state": (C.c_int, [vp, u32, i32]),
         "swarm_model_ptr": (C.c_int, [vp, C.POINTER(vp), C.POINTER(i64)]),
+        "swarm_potential_static": (C.c_int, [vp, i32, i64, i64, vp, vp]),
         "swarm_set_stream": (C.c_int, [vp, vp]),
         "swarm_sync": (C.c_int, [vp]),
         "swarm_kernel_launches": (i64, [vp]),
@@ -263,3 +264,14 @@ class Swarm:
 
     def set_state(self, launch, b_stale):
         self._check(self._L.swarm_set_state(self._h, launch, b_stale), "swarm_set_state")
+
+
+STATIC_MAX_D = 33554432
+
+
+def potential_static(x_ptr, n, d, pitch, out_ptr, stream=None):
+    """Gamma of n caller-held rows (device pointer x_ptr, row pitch in elements) into the device double at
+    out_ptr, through the entry point that allocates nothing (for callers that must not allocate: fixed
+    memory pools, hooks inside another component's step). Asynchronous on `stream`; returns the C code."""
+    ptr = getattr(stream, "cuda_stream", stream)
+    return load().swarm_potential_static(x_ptr, n, d, pitch, out_ptr, ptr)
