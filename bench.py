@@ -36,6 +36,10 @@ WORKLOADS = {
     "complete16_resnet50_b4": dict(n=16, d=25_557_032, topology="complete", degree=0, pairs=8, bits=4, mode=0, H=2,
                                    lr=0.05, seed=4, cfg=dict(objective=1, grad_std=float(np.sqrt(1e-3)),
                                                              drift_std=float(np.sqrt(0.05)))),
+    # reduced copy of the workload above (4 nodes, 2 pairs) for profiler captures that must stay small
+    "complete4_resnet50_b8": dict(n=4, d=25_557_032, topology="complete", degree=0, pairs=2, bits=8, mode=0, H=2,
+                                  lr=0.05, seed=4, cfg=dict(objective=1, grad_std=float(np.sqrt(1e-3)),
+                                                            drift_std=float(np.sqrt(0.05)))),
     # n = 32 nodes, d = 11,689,512 (ResNet-18 sized), random 4-regular graph, non-blocking, 8-bit.
     "regular32_resnet18_b8_nb": dict(n=32, d=11_689_512, topology="regular", degree=4, pairs=16, bits=8, mode=1, H=3,
                                      lr=0.05, seed=3, cfg=dict(objective=1, nonblocking=1,

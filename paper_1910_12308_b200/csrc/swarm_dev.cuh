@@ -56,6 +56,33 @@ __device__ __forceinline__ void normal_pair(uint32_t w0, uint32_t w1, float& z0,
   z1 = r * s;
 }
 
+// Box-Muller with the hardware approximations (lg2, sqrt, sin, cos on the special-function unit),
+// for the local-step gradient noise only. Absolute error of a normal: a few 1e-6 (sin/cos: 2^-20.9
+// absolute times a radius <= 5.8; radius: relative 4e-6). The noise enters a model coordinate
+// multiplied by lr * grad_std, so the model error is lr * grad_std * 4e-6 per step.
+//   -ln(u1) for u1 close to 1 comes from the series of -ln(1 - v), v = 1 - u1 (exact in fp32), because
+//   lg2 of a number next to 1 has no relative accuracy; the angle 2*pi*u2 is folded to [-pi, pi).
+__device__ __forceinline__ void normal_pair_fast(uint32_t w0, uint32_t w1, float& z0, float& z1) {
+  const uint32_t m1 = w0 >> 8;
+  const float u1 = (float)(m1 + 1u) * 0x1p-24f;
+  const float v = (float)(0x00FFFFFFu - m1) * 0x1p-24f;
+  const float series = v * fmaf(v, fmaf(v, fmaf(v, 0.25f, 0.33333334f), 0.5f), 1.0f);
+  const float viaLg2 = -0.69314718f * __log2f(u1);
+  const float nl = v < 0x1p-6f ? series : viaLg2;
+  float r;
+  asm("sqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(2.0f * nl));
+  const float ang = (float)(int32_t)(w1 & 0xFFFFFF00u) * (6.2831853071795865f * 0x1p-32f);
+  z0 = r * __cosf(ang);
+  z1 = r * __sinf(ang);
+}
+
+__device__ __forceinline__ void normal4_fast(uint32_t group, uint32_t row, uint32_t event, uint32_t stream,
+                                             uint32_t k0, uint32_t k1, float z[4]) {
+  const uint4 w = philox4x32_10(group, row, event, stream, k0, k1);
+  normal_pair_fast(w.x, w.y, z[0], z[1]);
+  normal_pair_fast(w.z, w.w, z[2], z[3]);
+}
+
 // Four normals of generator call (group, row, event, stream).
 __device__ __forceinline__ void normal4(uint32_t group, uint32_t row, uint32_t event, uint32_t stream,
                                         uint32_t k0, uint32_t k1, float z[4]) {

@@ -112,7 +112,7 @@ local_synth_kernel(StoreView s, const NodeDesc* __restrict__ nodes, int H, float
   float* x = &v.x;
   for (int q = 0; q < H; ++q) {
     float z[4];
-    normal4((uint32_t)g4, (uint32_t)nd.node, nd.event + (uint32_t)q, kStreamSynthGrad, s.key0, s.key1, z);
+    normal4_fast((uint32_t)g4, (uint32_t)nd.node, nd.event + (uint32_t)q, kStreamSynthGrad, s.key0, s.key1, z);
 #pragma unroll
     for (int t = 0; t < 4; ++t) {
       const float grad = __fadd_rn(c, __fmul_rn(grad_std, z[t]));

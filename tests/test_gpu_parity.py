@@ -202,6 +202,25 @@ def test_synthetic_gradient_steps_within_tolerance(d, H):
     assert np.array_equal(gpu.get(g.T_X, 0), orc.X[0]) and np.array_equal(gpu.get(g.T_X, 3), orc.X[3])
 
 
+def test_gradient_noise_accuracy():
+    """The local-step kernel draws its normals with the hardware approximations of lg2/sqrt/sin/cos.
+    With x0 = 0, lr = grad_std = 1 and no drift the model after one step is -z, which exposes the
+    absolute error of the normals: it must stay at a few 1e-6 (including u1 next to 1, where the
+    radius comes from a series)."""
+    cfg = dict(objective=1, grad_std=1.0, drift_std=0.0, init_std=0.0)
+    orc, gpu = make_pair(2, 400_000, seed=77, **cfg)
+    assert orc.local_steps([0, 1], 1, 1.0) == 0 and gpu.local_steps([0, 1], 1, 1.0) == 0
+    for i in range(2):
+        got, ref = gpu.get(g.T_X, i), orc.X[i]
+        err = np.abs(got - ref)
+        print("normal abs error: max %.3e mean %.3e" % (err.max(), err.mean()))
+        assert err.max() < 1e-5
+        assert np.abs(ref).max() > 4.0
+        # exact zeros of the reference (u1 = 1 or angle 0) aside, tiny normals keep their sign and scale
+        tiny = (np.abs(ref) < 1e-3) & (ref != 0)
+        assert tiny.sum() > 100 and np.all(np.sign(got[tiny]) == np.sign(ref[tiny]))
+
+
 @pytest.mark.parametrize("d,m,batch,dtype,groups", [(4096, 64, 16, 0, 0), (5000, 12, 5, 0, 0), (9000, 32, 64, 1, 2),
                                                    (300, 8, 3, 1, 0)])
 def test_least_squares_steps_within_tolerance(d, m, batch, dtype, groups):
