@@ -44,6 +44,12 @@ WORKLOADS = {
     "regular32_resnet18_b8_nb": dict(n=32, d=11_689_512, topology="regular", degree=4, pairs=16, bits=8, mode=1, H=3,
                                      lr=0.05, seed=3, cfg=dict(objective=1, nonblocking=1,
                                                                grad_std=float(np.sqrt(1e-3)))),
+    # n = 256 nodes, d = 2^20, least squares on bf16 data (512 x 2^20 per data group, 16 groups of 16 nodes),
+    # random 8-regular graph, 128 pairs per launch, 2-bit codes, non-blocking, H = 4 steps of batch 64.
+    "regular256_d1m_b2_lsq_nb": dict(n=256, d=1 << 20, topology="regular", degree=8, pairs=128, bits=2, mode=1, H=4,
+                                     lr=0.05, seed=5, cfg=dict(objective=2, nonblocking=1, lsq_m=512, lsq_batch=64,
+                                                               lsq_dtype=1, lsq_groups=16,
+                                                               lsq_noise_std=float(np.sqrt(0.1)))),
     # small case the CPU checker finishes in seconds
     "complete8_d4096_b8_lsq": dict(n=8, d=4096, topology="complete", degree=0, pairs=1, bits=8, mode=0, H=2, lr=0.05,
                                    seed=0, cfg=dict(objective=2, lsq_m=64, lsq_batch=16, lsq_dtype=0, lsq_groups=0,

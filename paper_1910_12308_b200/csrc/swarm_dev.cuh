@@ -62,18 +62,21 @@ __device__ __forceinline__ void normal_pair(uint32_t w0, uint32_t w1, float& z0,
 // multiplied by lr * grad_std, so the model error is lr * grad_std * 4e-6 per step.
 //   -ln(u1) for u1 close to 1 comes from the series of -ln(1 - v), v = 1 - u1 (exact in fp32), because
 //   lg2 of a number next to 1 has no relative accuracy; the angle 2*pi*u2 is folded to [-pi, pi).
+__device__ __forceinline__ float mufu_lg2(float x) { float r; asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
+__device__ __forceinline__ float mufu_sqrt(float x) { float r; asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
+__device__ __forceinline__ float mufu_sin(float x) { float r; asm("sin.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
+__device__ __forceinline__ float mufu_cos(float x) { float r; asm("cos.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
+
 __device__ __forceinline__ void normal_pair_fast(uint32_t w0, uint32_t w1, float& z0, float& z1) {
-  const uint32_t m1 = w0 >> 8;
-  const float u1 = (float)(m1 + 1u) * 0x1p-24f;
-  const float v = (float)(0x00FFFFFFu - m1) * 0x1p-24f;
+  const float u1 = fmaf((float)(w0 >> 8), 0x1p-24f, 0x1p-24f);     // ((w0 >> 8) + 1) * 2^-24, exact
+  const float v = 1.0f - u1;                                        // exact: both are multiples of 2^-24
   const float series = v * fmaf(v, fmaf(v, fmaf(v, 0.25f, 0.33333334f), 0.5f), 1.0f);
-  const float viaLg2 = -0.69314718f * __log2f(u1);
+  const float viaLg2 = -0.69314718f * mufu_lg2(u1);                 // u1 >= 2^-24 is a normal float
   const float nl = v < 0x1p-6f ? series : viaLg2;
-  float r;
-  asm("sqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(2.0f * nl));
+  const float r = mufu_sqrt(2.0f * nl);                             // 0 or >= 3.4e-4: no subnormals
   const float ang = (float)(int32_t)(w1 & 0xFFFFFF00u) * (6.2831853071795865f * 0x1p-32f);
-  z0 = r * __cosf(ang);
-  z1 = r * __sinf(ang);
+  z0 = r * mufu_cos(ang);
+  z1 = r * mufu_sin(ang);
 }
 
 __device__ __forceinline__ void normal4_fast(uint32_t group, uint32_t row, uint32_t event, uint32_t stream,
