@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libswarm_b200.so")
 OBJ_DIR = os.path.join(HERE, "_build")
-SOURCES = ["swarm_api.cu", "swarm_interact.cu", "swarm_local.cu", "swarm_reduce.cu", "swarm_noalloc.cu"]
+SOURCES = ["swarm_api.cu", "swarm_interact.cu", "swarm_local.cu", "swarm_reduce.cu", "swarm_noalloc.cu", "swarm_lsq_tc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

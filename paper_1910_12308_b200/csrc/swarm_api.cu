@@ -57,6 +57,10 @@ struct swarm_ctx {
   float* bvec = nullptr;
   float* xstar = nullptr;
   float* lsq_partial = nullptr;      // n * batch * chunks
+  float* tc_partial = nullptr;       // tensor-core path: split-K partials of the residuals
+  void* tc_resid = nullptr;          // tensor-core path: residuals as bf16 hi / lo
+  int* kernel_status = nullptr;      // set by a kernel whose bounded wait expired
+  int* kernel_status_host = nullptr; // pinned
   double* pot_partial = nullptr;
   double* pot_out = nullptr;
   int32_t* pairs_out_dev = nullptr;  // 2 * n/2 + 1 (sampler result, count last)
@@ -179,6 +183,8 @@ void free_objective(swarm_ctx* c) {
   dev_free(c, c->bvec); c->bvec = nullptr;
   dev_free(c, c->xstar); c->xstar = nullptr;
   dev_free(c, c->lsq_partial); c->lsq_partial = nullptr;
+  dev_free(c, c->tc_partial); c->tc_partial = nullptr;
+  dev_free(c, c->tc_resid); c->tc_resid = nullptr;
   dev_free(c, c->convert_tmp); c->convert_tmp = nullptr;
   dev_free(c, c->B); c->B = nullptr;
   c->groups = 0; c->nodes_per_group = 0;
@@ -226,6 +232,11 @@ int apply_config(swarm_ctx* c, const swarm_config& cfg) {
     c->lsq_partial = (float*)dev_alloc(c, (size_t)n * cfg.lsq_batch * lsq_chunks(c->d) * sizeof(float));
     c->convert_tmp = (float*)dev_alloc(c, row_bytes);
     if (!c->A || !c->bvec || !c->xstar || !c->lsq_partial || !c->convert_tmp) return SWARM_ENOMEM;
+    if (cfg.lsq_dtype == SWARM_BF16 && cfg.lsq_batch <= 64) {
+      c->tc_partial = (float*)dev_alloc(c, lsq_tc_partial_bytes(c->pitch, n));
+      c->tc_resid = dev_alloc(c, lsq_tc_resid_bytes(n));
+      if (!c->tc_partial || !c->tc_resid) return SWARM_ENOMEM;
+    }
   }
   StoreView s = view_of(c);
   SW_CUDA(c, cudaMemsetAsync(c->X, 0, (size_t)n * row_bytes, c->stream));
@@ -333,7 +344,8 @@ void swarm_destroy(swarm_ctx* c) {
   free_objective(c);
   dev_free(c, c->X); dev_free(c, c->codes); dev_free(c, c->exps); dev_free(c, c->adj_dev);
   dev_free(c, c->scalars); dev_free(c, c->pot_partial); dev_free(c, c->pot_out);
-  dev_free(c, c->pairs_out_dev); dev_free(c, c->used_dev); dev_free(c, c->stage_dev);
+  dev_free(c, c->pairs_out_dev); dev_free(c, c->used_dev); dev_free(c, c->stage_dev); dev_free(c, c->kernel_status);
+  if (c->kernel_status_host) cudaFreeHost(c->kernel_status_host);
   if (c->stage_host) cudaFreeHost(c->stage_host);
   if (c->pot_host) cudaFreeHost(c->pot_host);
   if (c->pairs_out_host) cudaFreeHost(c->pairs_out_host);
@@ -359,7 +371,8 @@ int swarm_init(swarm_ctx** out, int32_t n, int64_t d, swarm_topology topo, uint6
 
   const size_t row_bytes = (size_t)c->pitch * sizeof(float);
   const size_t max_pairs = (size_t)n / 2;
-  c->stage_slot_bytes = std::max({max_pairs * sizeof(PairDesc), (size_t)n * sizeof(NodeDesc), (size_t)n * sizeof(uint32_t)});
+  c->stage_slot_bytes = std::max({max_pairs * sizeof(PairDesc), (size_t)n * sizeof(NodeDesc), (size_t)n * sizeof(uint32_t),
+                                  (size_t)n * sizeof(LsqUnit)});
   c->stage_slot_bytes = (c->stage_slot_bytes + 255) / 256 * 256;
   c->X = (float*)dev_alloc(c, (size_t)n * row_bytes);
   c->codes = (uint8_t*)dev_alloc(c, (size_t)n * c->nblk * kBlockCoords);
@@ -370,11 +383,14 @@ int swarm_init(swarm_ctx** out, int32_t n, int64_t d, swarm_topology topo, uint6
   c->pot_out = (double*)dev_alloc(c, sizeof(double));
   c->pairs_out_dev = (int32_t*)dev_alloc(c, (2 * max_pairs + 1) * sizeof(int32_t));
   c->used_dev = (uint8_t*)dev_alloc(c, (size_t)n);
+  c->kernel_status = (int*)dev_alloc(c, sizeof(int));
   c->stage_dev = dev_alloc(c, c->stage_slot_bytes * kStageSlots);
   bool ok = c->X && c->codes && c->exps && c->adj_dev && c->scalars && c->pot_partial && c->pot_out &&
-            c->pairs_out_dev && c->used_dev && c->stage_dev;
+            c->pairs_out_dev && c->used_dev && c->stage_dev && c->kernel_status;
   ok = ok && cudaMallocHost(&c->stage_host, c->stage_slot_bytes * kStageSlots) == cudaSuccess;
   ok = ok && cudaMallocHost((void**)&c->pot_host, sizeof(double)) == cudaSuccess;
+  ok = ok && cudaMallocHost((void**)&c->kernel_status_host, sizeof(int)) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(c->kernel_status, 0, sizeof(int), c->stream) == cudaSuccess;
   ok = ok && cudaMallocHost((void**)&c->pairs_out_host, (2 * max_pairs + 1) * sizeof(int32_t)) == cudaSuccess;
   for (int i = 0; ok && i < kStageSlots; ++i)
     ok = cudaEventCreateWithFlags(&c->stage_event[i], cudaEventDisableTiming) == cudaSuccess;
@@ -415,7 +431,9 @@ int swarm_set_stream(swarm_ctx* c, void* cuda_stream) {
 int swarm_sync(swarm_ctx* c) {
   if (!c) return SWARM_EINVAL;
   DeviceGuard guard(c->device);
+  SW_CUDA(c, cudaMemcpyAsync(c->kernel_status_host, c->kernel_status, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
   SW_CUDA(c, cudaStreamSynchronize(c->stream));
+  if (*c->kernel_status_host != 0) return fail_cuda(c, cudaErrorLaunchTimeout);   // a bounded device wait expired
   return SWARM_OK;
 }
 
@@ -445,6 +463,39 @@ int swarm_local_steps(swarm_ctx* c, const int32_t* node_ids, int32_t count, int3
   DeviceGuard guard(c->device);
   void *host, *dev;
   int slot;
+  if (c->cfg.objective == SWARM_OBJ_LSQ && c->tc_partial) {
+    // bf16 data: batch the listed nodes that share a data matrix and a step counter (hence the
+    // minibatch) into units of up to 16 for the tensor-core kernels
+    std::vector<LsqUnit> units;
+    std::vector<int> order(node_ids, node_ids + count);
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+      const int ga = a / c->nodes_per_group, gb = b / c->nodes_per_group;
+      return ga != gb ? ga < gb : c->ls[a] < c->ls[b];
+    });
+    for (int node : order) {
+      const int g = node / c->nodes_per_group;
+      if (units.empty() || units.back().group != g || units.back().event != c->ls[node] || units.back().count == 16) {
+        LsqUnit u{};
+        u.group = g; u.event = c->ls[node]; u.count = 0;
+        units.push_back(u);
+      }
+      units.back().nodes[units.back().count++] = node;
+    }
+    const size_t bytes = units.size() * sizeof(LsqUnit);
+    int rc = stage_acquire(c, bytes, &host, &dev, &slot);
+    if (rc != SWARM_OK) return rc;
+    std::memcpy(host, units.data(), bytes);
+    rc = stage_commit(c, slot, bytes);
+    if (rc != SWARM_OK) return rc;
+    int nl = 0;
+    SW_CUDA(c, launch_local_lsq_tc(view_of(c), lsq_of(c), (const LsqUnit*)dev, (int)units.size(), H, lr, c->tc_partial,
+                                   c->tc_resid, c->kernel_status, c->stream, &nl));
+    c->launches += nl;
+    rc = stage_release(c, slot);
+    if (rc != SWARM_OK) return rc;
+    for (int t = 0; t < count; ++t) c->ls[node_ids[t]] += (uint32_t)H;
+    return SWARM_OK;
+  }
   int rc = stage_acquire(c, (size_t)count * sizeof(NodeDesc), &host, &dev, &slot);
   if (rc != SWARM_OK) return rc;
   NodeDesc* nd = (NodeDesc*)host;

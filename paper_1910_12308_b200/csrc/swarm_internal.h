@@ -19,6 +19,16 @@ struct NodeDesc {
   uint32_t event;      // local-step counter before this call
 };
 
+// Up to 16 nodes that share a data matrix and a local-step counter (hence a minibatch): one batched
+// tensor-core least-squares step.
+struct LsqUnit {
+  int32_t group;
+  uint32_t event;      // local-step counter of these nodes before this call
+  int32_t count;       // nodes in use (1..16)
+  int32_t nodes[16];
+  int32_t pad;
+};
+
 struct StoreView {
   float* X;            // [n][pitch]
   float* B;            // [n][pitch] or nullptr
@@ -58,6 +68,14 @@ cudaError_t launch_local_synth(const StoreView& s, const NodeDesc* nodes_dev, in
 cudaError_t launch_local_lsq(const StoreView& s, const LsqView& l, const NodeDesc* nodes_dev, int count, int H,
                              float lr, float* partial_dev, cudaStream_t st, int* launches);
 int64_t lsq_chunks(int64_t d);
+
+// --- swarm_lsq_tc.cu (bf16 data, batch <= 64) ----------------------------------------------
+size_t lsq_tc_partial_bytes(int64_t pitch, int units);
+size_t lsq_tc_resid_bytes(int units);
+// status_dev: one int, set to 1 if a bounded wait inside a kernel expired.
+cudaError_t launch_local_lsq_tc(const StoreView& s, const LsqView& l, const LsqUnit* units_dev, int nunits, int H,
+                                float lr, float* partial_dev, void* resid_dev, int* status_dev, cudaStream_t st,
+                                int* launches);
 cudaError_t launch_sample_pairs(const int32_t* adj_dev, int n, int degree, int max_pairs, uint32_t launch_ctr,
                                 uint32_t key0, uint32_t key1, int32_t* out_pairs_dev, int32_t* out_count_dev,
                                 uint8_t* used_dev, cudaStream_t st, int* launches);

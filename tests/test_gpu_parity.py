@@ -236,6 +236,26 @@ def test_least_squares_steps_within_tolerance(d, m, batch, dtype, groups):
         inject(orc, gpu, what=("X",))
 
 
+@pytest.mark.parametrize("n,groups,d,m,batch", [(20, 1, 9000, 40, 64), (6, 3, 40000, 16, 7), (32, 2, 33000, 128, 64),
+                                                (4, 0, 1500, 9, 33)])
+def test_batched_tensor_core_least_squares_steps(n, groups, d, m, batch):
+    """bf16 data: nodes that share a data matrix and a step counter are batched into tensor-core units of up
+    to 16 (here: more than 16 per matrix, ragged units, mixed counters, batches below the 64-row tile,
+    several k-chunks)."""
+    cfg = dict(objective=2, lsq_m=m, lsq_batch=batch, lsq_dtype=1, lsq_groups=groups, lsq_noise_std=0.3)
+    orc, gpu = make_pair(n, d, seed=51, **cfg)
+    inject(orc, gpu)
+    rng = np.random.default_rng(n)
+    schedule = [list(range(n)), sorted(rng.permutation(n)[: max(1, n // 2)].tolist()), list(range(n))[::-1]]
+    for nodes in schedule:
+        assert orc.local_steps(nodes, 3, 0.05) == 0 and gpu.local_steps(nodes, 3, 0.05) == 0
+        gpu.sync()
+        for i in range(n):
+            assert rel_err(gpu.get(g.T_X, i), orc.X[i]) < TOL, i
+            assert gpu.get(g.T_COUNTERS, i)[1] == orc.ls[i]
+        inject(orc, gpu, what=("X",))
+
+
 # ---- mean model and potential ----------------------------------------------------------------------
 
 @pytest.mark.parametrize("n,d", [(2, 1), (3, 1027), (8, 4096), (17, 2500), (64, 3000)])
