@@ -46,16 +46,30 @@ WORKLOADS = {
                                                                grad_std=float(np.sqrt(1e-3)))),
     # n = 256 nodes, d = 2^20, least squares on bf16 data (512 x 2^20 per data group, 16 groups of 16 nodes),
     # random 8-regular graph, 128 pairs per launch, 2-bit codes, non-blocking, H = 4 steps of batch 64.
+    # every node takes its H steps in every launch (all nodes compute between interactions), which keeps the
+    # step counters of a data group equal so that its 16 nodes share minibatches and are batched.
     "regular256_d1m_b2_lsq_nb": dict(n=256, d=1 << 20, topology="regular", degree=8, pairs=128, bits=2, mode=1, H=4,
-                                     lr=0.05, seed=5, cfg=dict(objective=2, nonblocking=1, lsq_m=512, lsq_batch=64,
-                                                               lsq_dtype=1, lsq_groups=16,
-                                                               lsq_noise_std=float(np.sqrt(0.1)))),
+                                     lr=0.05, seed=5, step_all=True,
+                                     cfg=dict(objective=2, nonblocking=1, lsq_m=512, lsq_batch=64, lsq_dtype=1,
+                                              lsq_groups=16, lsq_noise_std=float(np.sqrt(0.1)))),
+    # reduced copy (2 data groups) for profiler captures that must stay small
+    "regular32_d1m_b2_lsq_nb": dict(n=32, d=1 << 20, topology="regular", degree=8, pairs=16, bits=2, mode=1, H=4,
+                                    lr=0.05, seed=5, step_all=True,
+                                    cfg=dict(objective=2, nonblocking=1, lsq_m=512, lsq_batch=64, lsq_dtype=1,
+                                             lsq_groups=2, lsq_noise_std=float(np.sqrt(0.1)))),
     # small case the CPU checker finishes in seconds
     "complete8_d4096_b8_lsq": dict(n=8, d=4096, topology="complete", degree=0, pairs=1, bits=8, mode=0, H=2, lr=0.05,
                                    seed=0, cfg=dict(objective=2, lsq_m=64, lsq_batch=16, lsq_dtype=0, lsq_groups=0,
                                                     lsq_noise_std=float(np.sqrt(0.1)))),
 }
 DEFAULT_WORKLOAD = "ring64_d1m_b4"
+
+
+def stepping_nodes(wl, pairs):
+    """Nodes that take local steps before this launch's interactions."""
+    if wl.get("step_all"):
+        return np.arange(wl["n"], dtype=np.int32)
+    return pairs.reshape(-1)
 
 
 def interaction_bytes(d, bits, mode):
@@ -179,7 +193,7 @@ def time_oracle(wl, budget_s, max_launches, threads=None):
         pairs = sched.next()
         t0 = time.perf_counter()
         if wl["H"] > 0:
-            orc.local_steps(pairs.reshape(-1), wl["H"], wl["lr"])
+            orc.local_steps(stepping_nodes(wl, pairs), wl["H"], wl["lr"])
         rc = orc.interact(pairs, wl["bits"], wl["mode"], threads=T)
         t_total += time.perf_counter() - t0
         assert rc == 0
@@ -206,7 +220,7 @@ def run_reference(args, wl, name):
     def step(p, T):
         pairs = sched.next()[:p]
         if wl["H"] > 0:
-            orc.local_steps(pairs.reshape(-1), wl["H"], wl["lr"])
+            orc.local_steps(stepping_nodes(wl, pairs), wl["H"], wl["lr"])
         assert orc.interact(pairs, wl["bits"], wl["mode"], threads=T) == 0
         return len(pairs)
     t0 = time.perf_counter()
@@ -260,7 +274,7 @@ def run_ours(args, wl, name):
 
     def step(pairs):
         if wl["H"] > 0:
-            rc = sw.local_steps(pairs.reshape(-1), wl["H"], wl["lr"])
+            rc = sw.local_steps(stepping_nodes(wl, pairs), wl["H"], wl["lr"])
             assert rc == 0, rc
         rc = sw.interact(pairs, wl["bits"], wl["mode"])
         assert rc == 0, rc
@@ -282,7 +296,7 @@ def run_ours(args, wl, name):
     ev0.record(stream)
     for pairs in launches[W:]:
         if wl["H"] > 0:
-            assert sw.local_steps(pairs.reshape(-1), wl["H"], wl["lr"]) == 0
+            assert sw.local_steps(stepping_nodes(wl, pairs), wl["H"], wl["lr"]) == 0
             e_a, e_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e_a.record(stream)
             assert sw.interact(pairs, wl["bits"], wl["mode"]) == 0

@@ -120,26 +120,28 @@ __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bflo
 }  // namespace
 
 // =================================================================================================
-// Residual partials. Tile = 256 coordinates (4 swizzle atoms of 64). Shared memory per stage:
-//   A    : 4 atoms x [64 rows x 128 B]   (K-major, 128B swizzle, 8-row groups 1024 B apart)  32 KiB
-//   Xraw : 16 rows x 256 fp32                                                               16 KiB
-// plus two operand buffers Xhi/Xlo: 4 atoms x [16 rows x 128 B] each.
+// Residual partials. Tile = 128 coordinates (2 swizzle atoms of 64). Shared memory per stage:
+//   A    : 2 atoms x [64 rows x 128 B]   (K-major, 128B swizzle, 8-row groups 1024 B apart)  16 KiB
+//   Xraw : 16 rows x 128 fp32                                                                8 KiB
+// plus two operand buffers Xhi/Xlo: 2 atoms x [16 rows x 128 B] each. Three stages: 89 KiB per CTA,
+// two CTAs per SM so that one CTA's barriers and operand conversion hide behind the other's copies.
 // =================================================================================================
-constexpr int kResTile = 256;
+constexpr int kResTile = 128;
+constexpr int kResAtoms = kResTile / 64;
 constexpr int kResStages = 3;
-constexpr int kResABytes = 4 * kTcBatch * 128;                 // 32768
-constexpr int kResXrawBytes = kUnitNodes * kResTile * 4;       // 16384
-constexpr int kResXopBytes = 4 * kUnitNodes * 128;             // 8192 (one of hi / lo)
+constexpr int kResABytes = kResAtoms * kTcBatch * 128;         // 16384
+constexpr int kResXrawBytes = kUnitNodes * kResTile * 4;       // 8192
+constexpr int kResXopBytes = kResAtoms * kUnitNodes * 128;     // 4096 (one of hi / lo)
 constexpr int kResSmem = kResStages * (kResABytes + kResXrawBytes) + 2 * 2 * kResXopBytes + 1024 /*align*/ + 64;
 
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kTcThreads, 2)
 lsq_tc_residual_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, int step, float* __restrict__ partial,
                        int64_t chunk_coords, int64_t nchunks, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* sA = smem;                                           // stages of A
   uint8_t* sXraw = sA + kResStages * kResABytes;
-  uint8_t* sXop = sXraw + kResStages * kResXrawBytes;           // [buf][hi|lo][8192]
+  uint8_t* sXop = sXraw + kResStages * kResXrawBytes;           // [buf][hi|lo]
   uint64_t* bars = (uint64_t*)(sXop + 4 * kResXopBytes);        // mma_done[2]
   uint32_t* tmem_slot = (uint32_t*)(bars + 2);
   __shared__ int rows[kTcBatch];
@@ -174,24 +176,24 @@ lsq_tc_residual_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units
     if (tile < ntiles) {
       const int st = tile % kResStages;
       const int64_t k0 = kbase + (int64_t)tile * kResTile;
-      // A: 64 rows x 32 chunks of 16 B; thread -> (row = idx / 32, chunk = idx % 32)
+      // A: 64 rows x 16 chunks of 16 B; thread -> (row = idx / 16, chunk = idx % 16)
       const uint32_t a_base = smem_u32(sA + st * kResABytes);
 #pragma unroll
-      for (int it = 0; it < kTcBatch * 32 / kTcThreads; ++it) {
+      for (int it = 0; it < kTcBatch * 16 / kTcThreads; ++it) {
         const int idx = it * kTcThreads + tid;
-        const int r = idx >> 5, c = idx & 31;               // c: 16-byte chunk within the 512-byte row slice
+        const int r = idx >> 4, c = idx & 15;               // c: 16-byte chunk within the 256-byte row slice
         if (r < l.batch) {
           const int atom = c >> 3, cc = c & 7;
           const uint32_t dst = a_base + atom * (kTcBatch * 128) + (r >> 3) * 1024 + (r & 7) * 128 + ((cc ^ (r & 7)) << 4);
           cp_async16(dst, A + (int64_t)rows[r] * s.pitch + k0 + c * 8);
         }
       }
-      // X: 16 rows x 64 chunks of 16 B (fp32), plain row-major staging
+      // X: 16 rows x 32 chunks of 16 B (fp32), plain row-major staging
       const uint32_t x_base = smem_u32(sXraw + st * kResXrawBytes);
 #pragma unroll
-      for (int it = 0; it < kUnitNodes * 64 / kTcThreads; ++it) {
+      for (int it = 0; it < kUnitNodes * 32 / kTcThreads; ++it) {
         const int idx = it * kTcThreads + tid;
-        const int r = idx >> 6, c = idx & 63;
+        const int r = idx >> 5, c = idx & 31;
         if (r < u.count) cp_async16(x_base + r * (kResTile * 4) + c * 16, s.X + (int64_t)unodes[r] * s.pitch + k0 + c * 4);
       }
     }
@@ -206,28 +208,23 @@ lsq_tc_residual_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units
     cp_async_wait<kResStages - 2>();
     __syncthreads();                                        // tile t has landed for every thread
     if (t >= 2) ok = mbar_wait(smem_u32(&bars[buf]), ((t >> 1) - 1) & 1);   // operand buffer free again
-    // fp32 -> bf16 hi/lo into the swizzled operand layout: thread -> (row = tid / 16, 16 coordinates)
+    // fp32 -> bf16 hi/lo into the swizzled operand layout: thread -> (row = tid / 16, 8 coordinates)
     {
-      const int r = tid >> 4, c16 = tid & 15;
-      const float4* src = reinterpret_cast<const float4*>(sXraw + st * kResXrawBytes + r * (kResTile * 4) + c16 * 64);
-      __align__(16) __nv_bfloat16 hi[16], lo[16];
+      const int r = tid >> 4, c8 = tid & 15;                // c8: group of 8 coordinates = one 16-byte bf16 chunk
+      const float4* src = reinterpret_cast<const float4*>(sXraw + st * kResXrawBytes + r * (kResTile * 4) + c8 * 32);
+      __align__(16) __nv_bfloat16 hi[8], lo[8];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
+      for (int q = 0; q < 2; ++q) {
         const float4 v = src[q];
         split_bf16(v.x, hi[q * 4 + 0], lo[q * 4 + 0]);
         split_bf16(v.y, hi[q * 4 + 1], lo[q * 4 + 1]);
         split_bf16(v.z, hi[q * 4 + 2], lo[q * 4 + 2]);
         split_bf16(v.w, hi[q * 4 + 3], lo[q * 4 + 3]);
       }
-      const int atom = c16 >> 2;                            // 64 coordinates per atom = 4 groups of 16
-      uint8_t* base_hi = sXop + (buf * 2 + 0) * kResXopBytes + atom * (kUnitNodes * 128) + (r >> 3) * 1024 + (r & 7) * 128;
-      uint8_t* base_lo = sXop + (buf * 2 + 1) * kResXopBytes + atom * (kUnitNodes * 128) + (r >> 3) * 1024 + (r & 7) * 128;
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const int cc = (c16 & 3) * 2 + h;                   // 16-byte chunk within the 128-byte row
-        *reinterpret_cast<uint4*>(base_hi + ((cc ^ (r & 7)) << 4)) = *reinterpret_cast<const uint4*>(hi + h * 8);
-        *reinterpret_cast<uint4*>(base_lo + ((cc ^ (r & 7)) << 4)) = *reinterpret_cast<const uint4*>(lo + h * 8);
-      }
+      const int atom = c8 >> 3, cc = c8 & 7;
+      const int off = atom * (kUnitNodes * 128) + (r >> 3) * 1024 + (r & 7) * 128 + ((cc ^ (r & 7)) << 4);
+      *reinterpret_cast<uint4*>(sXop + (buf * 2 + 0) * kResXopBytes + off) = *reinterpret_cast<const uint4*>(hi);
+      *reinterpret_cast<uint4*>(sXop + (buf * 2 + 1) * kResXopBytes + off) = *reinterpret_cast<const uint4*>(lo);
     }
     fence_proxy_async();                                    // generic-proxy writes (cp.async, st.shared) -> MMA reads
     tc_fence_before();
@@ -238,7 +235,7 @@ lsq_tc_residual_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units
       const uint32_t h_base = smem_u32(sXop + (buf * 2 + 0) * kResXopBytes);
       const uint32_t l_base = smem_u32(sXop + (buf * 2 + 1) * kResXopBytes);
 #pragma unroll
-      for (int atom = 0; atom < 4; ++atom)
+      for (int atom = 0; atom < kResAtoms; ++atom)
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks) {                    // 16 coordinates (32 bytes) per MMA
           const uint64_t da = smem_desc_sw128(a_base + atom * (kTcBatch * 128) + ks * 32, 16, 1024);
@@ -287,7 +284,8 @@ lsq_tc_finalize_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units
   const int sidx = threadIdx.x / kUnitNodes, j = threadIdx.x % kUnitNodes;
   const float* p = partial + (int64_t)blockIdx.x * nchunks * (kTcBatch * kUnitNodes) + threadIdx.x;
   float acc = 0.0f;
-  for (int64_t c = 0; c < nchunks; ++c) acc += p[c * (kTcBatch * kUnitNodes)];
+#pragma unroll 8
+  for (int64_t c = 0; c < nchunks; ++c) acc += p[c * (kTcBatch * kUnitNodes)];   // chunk order: fixed summation order
   float r = 0.0f;
   if (sidx < l.batch && j < u.count) {
     const int row = tc_minibatch_row(sidx, u.group, u.event + (uint32_t)step, l.m, s.key0, s.key1);
