@@ -496,22 +496,34 @@ int swarm_local_steps(swarm_ctx* c, const int32_t* node_ids, int32_t count, int3
     for (int t = 0; t < count; ++t) c->ls[node_ids[t]] += (uint32_t)H;
     return SWARM_OK;
   }
-  int rc = stage_acquire(c, (size_t)count * sizeof(NodeDesc), &host, &dev, &slot);
-  if (rc != SWARM_OK) return rc;
-  NodeDesc* nd = (NodeDesc*)host;
+  NodeList list{};
+  list.n = count;
+  int rc = SWARM_OK;
+  slot = -1;
+  NodeDesc* nd = list.inl;
+  if (count > kInlineNodes) {
+    rc = stage_acquire(c, (size_t)count * sizeof(NodeDesc), &host, &dev, &slot);
+    if (rc != SWARM_OK) return rc;
+    nd = (NodeDesc*)host;
+    list.ptr = (const NodeDesc*)dev;
+  }
   for (int t = 0; t < count; ++t) { nd[t].node = node_ids[t]; nd[t].event = c->ls[node_ids[t]]; }
-  rc = stage_commit(c, slot, (size_t)count * sizeof(NodeDesc));
-  if (rc != SWARM_OK) return rc;
+  if (slot >= 0) {
+    rc = stage_commit(c, slot, (size_t)count * sizeof(NodeDesc));
+    if (rc != SWARM_OK) return rc;
+  }
   int nl = 0;
   const StoreView s = view_of(c);
   if (c->cfg.objective == SWARM_OBJ_SYNTH) {
-    SW_CUDA(c, launch_local_synth(s, (const NodeDesc*)dev, count, H, lr, c->cfg.grad_std, c->scalars, c->stream, &nl));
+    SW_CUDA(c, launch_local_synth(s, list, count, H, lr, c->cfg.grad_std, c->scalars, c->stream, &nl));
   } else {
-    SW_CUDA(c, launch_local_lsq(s, lsq_of(c), (const NodeDesc*)dev, count, H, lr, c->lsq_partial, c->stream, &nl));
+    SW_CUDA(c, launch_local_lsq(s, lsq_of(c), list, count, H, lr, c->lsq_partial, c->stream, &nl));
   }
   c->launches += nl;
-  rc = stage_release(c, slot);
-  if (rc != SWARM_OK) return rc;
+  if (slot >= 0) {
+    rc = stage_release(c, slot);
+    if (rc != SWARM_OK) return rc;
+  }
   for (int t = 0; t < count; ++t) c->ls[node_ids[t]] += (uint32_t)H;
   return SWARM_OK;
 }
@@ -533,22 +545,32 @@ int swarm_interact(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, int32_
   }
   if (npairs == 0) return SWARM_OK;
   void *host, *dev;
-  int slot;
-  rc = stage_acquire(c, (size_t)npairs * sizeof(PairDesc), &host, &dev, &slot);
-  if (rc != SWARM_OK) return rc;
-  PairDesc* pd = (PairDesc*)host;
+  int slot = -1;
+  PairList list{};
+  list.n = npairs;
+  PairDesc* pd = list.inl;
+  if (npairs > kInlinePairs) {
+    rc = stage_acquire(c, (size_t)npairs * sizeof(PairDesc), &host, &dev, &slot);
+    if (rc != SWARM_OK) return rc;
+    pd = (PairDesc*)host;
+    list.ptr = (const PairDesc*)dev;
+  }
   for (int p = 0; p < npairs; ++p) {
     pd[p].a = pairs[p].a; pd[p].b = pairs[p].b;
     pd[p].wa = c->w[pairs[p].a]; pd[p].wb = c->w[pairs[p].b];
   }
-  rc = stage_commit(c, slot, (size_t)npairs * sizeof(PairDesc));
-  if (rc != SWARM_OK) return rc;
+  if (slot >= 0) {
+    rc = stage_commit(c, slot, (size_t)npairs * sizeof(PairDesc));
+    if (rc != SWARM_OK) return rc;
+  }
   int nl = 0;
-  if (mode == SWARM_BLOCKING) SW_CUDA(c, launch_interact_blocking(view_of(c), (const PairDesc*)dev, npairs, bits, c->stream, &nl));
-  else SW_CUDA(c, launch_interact_nonblocking(view_of(c), (const PairDesc*)dev, npairs, bits, c->stream, &nl));
+  if (mode == SWARM_BLOCKING) SW_CUDA(c, launch_interact_blocking(view_of(c), list, npairs, bits, c->stream, &nl));
+  else SW_CUDA(c, launch_interact_nonblocking(view_of(c), list, npairs, bits, c->stream, &nl));
   c->launches += nl;
-  rc = stage_release(c, slot);
-  if (rc != SWARM_OK) return rc;
+  if (slot >= 0) {
+    rc = stage_release(c, slot);
+    if (rc != SWARM_OK) return rc;
+  }
   if (bits != 32) {
     for (int p = 0; p < npairs; ++p) {
       c->w[pairs[p].a] += 1; c->w[pairs[p].b] += 1;

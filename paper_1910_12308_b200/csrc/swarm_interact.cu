@@ -24,13 +24,13 @@ constexpr int kSubCoords = 256;  // coordinates per sub-block
 // -----------------------------------------------------------------------------------------
 template <int BITS>
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
-interact_blocking_kernel(StoreView s, const PairDesc* __restrict__ pairs, int64_t total_warps) {
+interact_blocking_kernel(StoreView s, const PairList pairs, int64_t total_warps) {
   const int lane = threadIdx.x & 31;
   const int64_t warp = (int64_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
   if (warp >= total_warps) return;
   const int64_t pair = warp / s.nblk;
   const int64_t blk = warp - pair * s.nblk;
-  const PairDesc pd = pairs[pair];
+  const PairDesc pd = pairs.get(pair);
 
   float* xa = s.X + (int64_t)pd.a * s.pitch + blk * kBlockCoords + lane * 8;
   float* xb = s.X + (int64_t)pd.b * s.pitch + blk * kBlockCoords + lane * 8;
@@ -92,13 +92,13 @@ interact_blocking_kernel(StoreView s, const PairDesc* __restrict__ pairs, int64_
 
 // Identity quantizer (Corollary 2): plain averaging, buffers untouched.
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
-interact_identity_kernel(StoreView s, const PairDesc* __restrict__ pairs, int64_t total_warps) {
+interact_identity_kernel(StoreView s, const PairList pairs, int64_t total_warps) {
   const int lane = threadIdx.x & 31;
   const int64_t warp = (int64_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
   if (warp >= total_warps) return;
   const int64_t pair = warp / s.nblk;
   const int64_t blk = warp - pair * s.nblk;
-  const PairDesc pd = pairs[pair];
+  const PairDesc pd = pairs.get(pair);
   float* xa = s.X + (int64_t)pd.a * s.pitch + blk * kBlockCoords + lane * 8;
   float* xb = s.X + (int64_t)pd.b * s.pitch + blk * kBlockCoords + lane * 8;
   f8 va[kSub], vb[kSub];
@@ -127,13 +127,13 @@ interact_identity_kernel(StoreView s, const PairDesc* __restrict__ pairs, int64_
 // -----------------------------------------------------------------------------------------
 template <int BITS>
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
-interact_nonblocking_kernel(StoreView s, const PairDesc* __restrict__ pairs, int64_t total_warps) {
+interact_nonblocking_kernel(StoreView s, const PairList pairs, int64_t total_warps) {
   const int lane = threadIdx.x & 31;
   const int64_t warp = (int64_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
   if (warp >= total_warps) return;
   const int64_t pair = warp / s.nblk;
   const int64_t blk = warp - pair * s.nblk;
-  const PairDesc pd = pairs[pair];
+  const PairDesc pd = pairs.get(pair);
 
   float* xa = s.X + (int64_t)pd.a * s.pitch + blk * kBlockCoords + lane * 8;
   float* ba = s.B + (int64_t)pd.a * s.pitch + blk * kBlockCoords + lane * 8;
@@ -279,31 +279,31 @@ publish_encode_kernel(StoreView s, const uint32_t* __restrict__ wctr, int64_t to
 // -----------------------------------------------------------------------------------------
 static inline unsigned ctas_for(int64_t warps) { return (unsigned)((warps + kWarpsPerCta - 1) / kWarpsPerCta); }
 
-cudaError_t launch_interact_blocking(const StoreView& s, const PairDesc* pairs_dev, int npairs, int bits,
+cudaError_t launch_interact_blocking(const StoreView& s, const PairList& pairs, int npairs, int bits,
                                      cudaStream_t st, int* launches) {
   if (npairs == 0) return cudaSuccess;
   const int64_t warps = (int64_t)npairs * s.nblk;
   const dim3 grid(ctas_for(warps)), block(kWarpsPerCta * 32);
   switch (bits) {
-    case 2: interact_blocking_kernel<2><<<grid, block, 0, st>>>(s, pairs_dev, warps); break;
-    case 4: interact_blocking_kernel<4><<<grid, block, 0, st>>>(s, pairs_dev, warps); break;
-    case 8: interact_blocking_kernel<8><<<grid, block, 0, st>>>(s, pairs_dev, warps); break;
-    case 32: interact_identity_kernel<<<grid, block, 0, st>>>(s, pairs_dev, warps); break;
+    case 2: interact_blocking_kernel<2><<<grid, block, 0, st>>>(s, pairs, warps); break;
+    case 4: interact_blocking_kernel<4><<<grid, block, 0, st>>>(s, pairs, warps); break;
+    case 8: interact_blocking_kernel<8><<<grid, block, 0, st>>>(s, pairs, warps); break;
+    case 32: interact_identity_kernel<<<grid, block, 0, st>>>(s, pairs, warps); break;
     default: return cudaErrorInvalidValue;
   }
   ++*launches;
   return cudaGetLastError();
 }
 
-cudaError_t launch_interact_nonblocking(const StoreView& s, const PairDesc* pairs_dev, int npairs, int bits,
+cudaError_t launch_interact_nonblocking(const StoreView& s, const PairList& pairs, int npairs, int bits,
                                         cudaStream_t st, int* launches) {
   if (npairs == 0) return cudaSuccess;
   const int64_t warps = (int64_t)npairs * s.nblk;
   const dim3 grid(ctas_for(warps)), block(kWarpsPerCta * 32);
   switch (bits) {
-    case 2: interact_nonblocking_kernel<2><<<grid, block, 0, st>>>(s, pairs_dev, warps); break;
-    case 4: interact_nonblocking_kernel<4><<<grid, block, 0, st>>>(s, pairs_dev, warps); break;
-    case 8: interact_nonblocking_kernel<8><<<grid, block, 0, st>>>(s, pairs_dev, warps); break;
+    case 2: interact_nonblocking_kernel<2><<<grid, block, 0, st>>>(s, pairs, warps); break;
+    case 4: interact_nonblocking_kernel<4><<<grid, block, 0, st>>>(s, pairs, warps); break;
+    case 8: interact_nonblocking_kernel<8><<<grid, block, 0, st>>>(s, pairs, warps); break;
     default: return cudaErrorInvalidValue;
   }
   ++*launches;

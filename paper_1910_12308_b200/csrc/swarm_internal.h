@@ -19,6 +19,27 @@ struct NodeDesc {
   uint32_t event;      // local-step counter before this call
 };
 
+// Descriptor lists travel either inline in the kernel parameters (short lists: no copy engine
+// involved, which matters when a launch is only a few microseconds long) or through device memory.
+constexpr int kInlinePairs = 8;
+constexpr int kInlineNodes = 16;
+struct PairList {
+  const PairDesc* ptr;
+  int32_t n;
+  PairDesc inl[kInlinePairs];
+#ifdef __CUDACC__
+  __device__ __forceinline__ PairDesc get(int64_t i) const { return n <= kInlinePairs ? inl[i] : ptr[i]; }
+#endif
+};
+struct NodeList {
+  const NodeDesc* ptr;
+  int32_t n;
+  NodeDesc inl[kInlineNodes];
+#ifdef __CUDACC__
+  __device__ __forceinline__ NodeDesc get(int i) const { return n <= kInlineNodes ? inl[i] : ptr[i]; }
+#endif
+};
+
 // Up to 16 nodes that share a data matrix and a local-step counter (hence a minibatch): one batched
 // tensor-core least-squares step.
 struct LsqUnit {
@@ -48,9 +69,9 @@ struct LsqView {
 };
 
 // --- swarm_interact.cu -------------------------------------------------------------------
-cudaError_t launch_interact_blocking(const StoreView& s, const PairDesc* pairs_dev, int npairs, int bits,
+cudaError_t launch_interact_blocking(const StoreView& s, const PairList& pairs, int npairs, int bits,
                                      cudaStream_t st, int* launches);
-cudaError_t launch_interact_nonblocking(const StoreView& s, const PairDesc* pairs_dev, int npairs, int bits,
+cudaError_t launch_interact_nonblocking(const StoreView& s, const PairList& pairs, int npairs, int bits,
                                         cudaStream_t st, int* launches);
 // wctr_dev: n write counters (uint32) used for the rounding uniforms of each node's buffer.
 cudaError_t launch_publish(const StoreView& s, const uint32_t* wctr_dev, int bits, cudaStream_t st, int* launches);
@@ -62,10 +83,10 @@ cudaError_t launch_node_scalars(float* scalars_dev, int n, float offset_std, flo
                                 uint32_t key1, cudaStream_t st, int* launches);
 cudaError_t launch_lsq_data(const StoreView& s, const LsqView& l, void* A, float* xstar, float* bvec,
                             const float* scalars_dev, float noise_std, cudaStream_t st, int* launches);
-cudaError_t launch_local_synth(const StoreView& s, const NodeDesc* nodes_dev, int count, int H, float lr,
+cudaError_t launch_local_synth(const StoreView& s, const NodeList& nodes, int count, int H, float lr,
                                float grad_std, const float* scalars_dev, cudaStream_t st, int* launches);
 // partial_dev: scratch of count * batch * lsq_chunks(d) floats.
-cudaError_t launch_local_lsq(const StoreView& s, const LsqView& l, const NodeDesc* nodes_dev, int count, int H,
+cudaError_t launch_local_lsq(const StoreView& s, const LsqView& l, const NodeList& nodes, int count, int H,
                              float lr, float* partial_dev, cudaStream_t st, int* launches);
 int64_t lsq_chunks(int64_t d);
 

@@ -101,11 +101,11 @@ lsq_labels_kernel(const T* __restrict__ A, const float* __restrict__ xstar, floa
 // One thread per 4 coordinates (one generator call per step).
 // -----------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
-local_synth_kernel(StoreView s, const NodeDesc* __restrict__ nodes, int H, float lr, float grad_std,
+local_synth_kernel(StoreView s, const NodeList nodes, int H, float lr, float grad_std,
                    const float* __restrict__ scalars) {
   const int64_t g4 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (g4 * 4 >= s.d) return;
-  const NodeDesc nd = nodes[blockIdx.y];
+  const NodeDesc nd = nodes.get(blockIdx.y);
   const float c = scalars[nd.node * 3 + 1];
   float* p = s.X + (int64_t)nd.node * s.pitch + g4 * 4;
   float4 v = *reinterpret_cast<const float4*>(p);
@@ -148,9 +148,9 @@ __device__ __forceinline__ int minibatch_row(int s_idx, int group, uint32_t even
 
 template <typename T>
 __global__ void __launch_bounds__(kLsqThreads)
-lsq_residual_kernel(StoreView s, LsqView l, const NodeDesc* __restrict__ nodes, int step, float* __restrict__ partial,
+lsq_residual_kernel(StoreView s, LsqView l, const NodeList nodes, int step, float* __restrict__ partial,
                     int64_t nchunks) {
-  const NodeDesc nd = nodes[blockIdx.y];
+  const NodeDesc nd = nodes.get(blockIdx.y);
   const int group = nd.node / l.nodes_per_group;
   const uint32_t event = nd.event + (uint32_t)step;
   const int64_t k0 = (int64_t)blockIdx.x * kLsqChunk + threadIdx.x * kLsqPerThread;
@@ -186,9 +186,9 @@ lsq_residual_kernel(StoreView s, LsqView l, const NodeDesc* __restrict__ nodes, 
 
 template <typename T>
 __global__ void __launch_bounds__(kLsqThreads)
-lsq_update_kernel(StoreView s, LsqView l, const NodeDesc* __restrict__ nodes, int step, float lr,
+lsq_update_kernel(StoreView s, LsqView l, const NodeList nodes, int step, float lr,
                   const float* __restrict__ partial, int64_t nchunks) {
-  const NodeDesc nd = nodes[blockIdx.y];
+  const NodeDesc nd = nodes.get(blockIdx.y);
   const int group = nd.node / l.nodes_per_group;
   const uint32_t event = nd.event + (uint32_t)step;
   const int64_t k0 = (int64_t)blockIdx.x * kLsqChunk + threadIdx.x * kLsqPerThread;
@@ -225,6 +225,105 @@ lsq_update_kernel(StoreView s, LsqView l, const NodeDesc* __restrict__ nodes, in
 #pragma unroll
   for (int t = 0; t < kLsqPerThread; ++t)
     if (k0 + t < s.d) xrow[k0 + t] -= scale * g[t];
+}
+
+// -----------------------------------------------------------------------------------------
+// Least-squares local steps for short models (row pitch <= 8192, batch <= 32): one CTA per node
+// runs all H steps in one launch with the model in registers. Per step: every thread forms its
+// share of the B dot products, a shuffle + shared-memory reduction in fixed order gives the
+// residuals, then the sampled rows are read again (from L2) for the update.
+// -----------------------------------------------------------------------------------------
+constexpr int kSmallThreads = 256;
+constexpr int kSmallMaxChunks = 8;        // 8 x 1024 coordinates
+constexpr int kSmallMaxBatch = 32;
+
+template <typename T>
+__device__ __forceinline__ float4 load4_as_float(const T* p);
+template <>
+__device__ __forceinline__ float4 load4_as_float<float>(const float* p) { return *reinterpret_cast<const float4*>(p); }
+template <>
+__device__ __forceinline__ float4 load4_as_float<__nv_bfloat16>(const __nv_bfloat16* p) {
+  const uint2 raw = *reinterpret_cast<const uint2*>(p);
+  return make_float4(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xFFFF0000u),
+                     __uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xFFFF0000u));
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kSmallThreads)
+lsq_small_kernel(StoreView s, LsqView l, const NodeList nodes, int H, float lr) {
+  const NodeDesc nd = nodes.get(blockIdx.x);
+  const int group = nd.node / l.nodes_per_group;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int nchunk = (int)(s.pitch / kBlockCoords);
+  float* xrow = s.X + (int64_t)nd.node * s.pitch;
+  const T* A = reinterpret_cast<const T*>(l.A) + (int64_t)group * l.m * s.pitch;
+  const float* labels = l.bvec + (int64_t)nd.node * l.m;
+
+  __shared__ int rows[kSmallMaxBatch];
+  __shared__ float red[kSmallThreads / 32][kSmallMaxBatch];
+  __shared__ float resid[kSmallMaxBatch];
+
+  float4 x[kSmallMaxChunks];
+#pragma unroll
+  for (int c = 0; c < kSmallMaxChunks; ++c)
+    x[c] = c < nchunk ? *reinterpret_cast<const float4*>(xrow + c * kBlockCoords + tid * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+  const float scale = lr / (float)l.batch;
+
+  for (int q = 0; q < H; ++q) {
+    if (tid < l.batch) rows[tid] = minibatch_row(tid, group, nd.event + (uint32_t)q, l.m, s.key0, s.key1);
+    __syncthreads();
+    for (int si = 0; si < l.batch; ++si) {
+      const T* row = A + (int64_t)rows[si] * s.pitch + tid * 4;
+      float acc = 0.0f;
+#pragma unroll
+      for (int c = 0; c < kSmallMaxChunks; ++c)
+        if (c < nchunk) {
+          const float4 a = load4_as_float<T>(row + c * kBlockCoords);
+          acc = fmaf(a.x, x[c].x, acc); acc = fmaf(a.y, x[c].y, acc);
+          acc = fmaf(a.z, x[c].z, acc); acc = fmaf(a.w, x[c].w, acc);
+        }
+      acc = warp_sum(acc);
+      if (lane == 0) red[warp][si] = acc;
+    }
+    __syncthreads();
+    if (tid < l.batch) {
+      float tot = 0.0f;
+#pragma unroll
+      for (int w = 0; w < kSmallThreads / 32; ++w) tot += red[w][tid];
+      resid[tid] = tot - labels[rows[tid]];
+    }
+    __syncthreads();
+    float4 g[kSmallMaxChunks];
+#pragma unroll
+    for (int c = 0; c < kSmallMaxChunks; ++c) g[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int si = 0; si < l.batch; ++si) {
+      const T* row = A + (int64_t)rows[si] * s.pitch + tid * 4;
+      const float rs = resid[si];
+#pragma unroll
+      for (int c = 0; c < kSmallMaxChunks; ++c)
+        if (c < nchunk) {
+          const float4 a = load4_as_float<T>(row + c * kBlockCoords);
+          g[c].x = fmaf(rs, a.x, g[c].x); g[c].y = fmaf(rs, a.y, g[c].y);
+          g[c].z = fmaf(rs, a.z, g[c].z); g[c].w = fmaf(rs, a.w, g[c].w);
+        }
+    }
+#pragma unroll
+    for (int c = 0; c < kSmallMaxChunks; ++c) {
+      x[c].x -= scale * g[c].x; x[c].y -= scale * g[c].y; x[c].z -= scale * g[c].z; x[c].w -= scale * g[c].w;
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int c = 0; c < kSmallMaxChunks; ++c)
+    if (c < nchunk) {
+      const int64_t k = (int64_t)c * kBlockCoords + tid * 4;
+      float4 v = x[c];
+      if (k + 0 >= s.d) v.x = 0.f;                    // data rows are zero past d, so these are zero already
+      if (k + 1 >= s.d) v.y = 0.f;
+      if (k + 2 >= s.d) v.z = 0.f;
+      if (k + 3 >= s.d) v.w = 0.f;
+      *reinterpret_cast<float4*>(xrow + k) = v;
+    }
 }
 
 // -----------------------------------------------------------------------------------------
@@ -319,28 +418,34 @@ cudaError_t launch_lsq_data(const StoreView& s, const LsqView& l, void* A, float
   return cudaGetLastError();
 }
 
-cudaError_t launch_local_synth(const StoreView& s, const NodeDesc* nodes_dev, int count, int H, float lr,
+cudaError_t launch_local_synth(const StoreView& s, const NodeList& nodes, int count, int H, float lr,
                                float grad_std, const float* scalars_dev, cudaStream_t st, int* launches) {
   if (count == 0 || H == 0) return cudaSuccess;
   const dim3 grid(cdiv((s.d + 3) / 4, 256), count);
-  local_synth_kernel<<<grid, 256, 0, st>>>(s, nodes_dev, H, lr, grad_std, scalars_dev);
+  local_synth_kernel<<<grid, 256, 0, st>>>(s, nodes, H, lr, grad_std, scalars_dev);
   ++*launches;
   return cudaGetLastError();
 }
 
-cudaError_t launch_local_lsq(const StoreView& s, const LsqView& l, const NodeDesc* nodes_dev, int count, int H,
+cudaError_t launch_local_lsq(const StoreView& s, const LsqView& l, const NodeList& nodes, int count, int H,
                              float lr, float* partial_dev, cudaStream_t st, int* launches) {
   if (count == 0 || H == 0) return cudaSuccess;
   if (l.batch > kLsqMaxBatch) return cudaErrorInvalidValue;
+  if (s.pitch <= (int64_t)kSmallMaxChunks * kBlockCoords && l.batch <= kSmallMaxBatch) {
+    if (l.dtype == 1) lsq_small_kernel<__nv_bfloat16><<<count, kSmallThreads, 0, st>>>(s, l, nodes, H, lr);
+    else lsq_small_kernel<float><<<count, kSmallThreads, 0, st>>>(s, l, nodes, H, lr);
+    ++*launches;
+    return cudaGetLastError();
+  }
   const int64_t nchunks = lsq_chunks(s.d);
   const dim3 grid((unsigned)nchunks, count);
   for (int q = 0; q < H; ++q) {
     if (l.dtype == 1) {
-      lsq_residual_kernel<__nv_bfloat16><<<grid, kLsqThreads, 0, st>>>(s, l, nodes_dev, q, partial_dev, nchunks);
-      lsq_update_kernel<__nv_bfloat16><<<grid, kLsqThreads, 0, st>>>(s, l, nodes_dev, q, lr, partial_dev, nchunks);
+      lsq_residual_kernel<__nv_bfloat16><<<grid, kLsqThreads, 0, st>>>(s, l, nodes, q, partial_dev, nchunks);
+      lsq_update_kernel<__nv_bfloat16><<<grid, kLsqThreads, 0, st>>>(s, l, nodes, q, lr, partial_dev, nchunks);
     } else {
-      lsq_residual_kernel<float><<<grid, kLsqThreads, 0, st>>>(s, l, nodes_dev, q, partial_dev, nchunks);
-      lsq_update_kernel<float><<<grid, kLsqThreads, 0, st>>>(s, l, nodes_dev, q, lr, partial_dev, nchunks);
+      lsq_residual_kernel<float><<<grid, kLsqThreads, 0, st>>>(s, l, nodes, q, partial_dev, nchunks);
+      lsq_update_kernel<float><<<grid, kLsqThreads, 0, st>>>(s, l, nodes, q, lr, partial_dev, nchunks);
     }
     *launches += 2;
   }
