@@ -44,6 +44,10 @@ WORKLOADS = {
     "regular32_resnet18_b8_nb": dict(n=32, d=11_689_512, topology="regular", degree=4, pairs=16, bits=8, mode=1, H=3,
                                      lr=0.05, seed=3, cfg=dict(objective=1, nonblocking=1,
                                                                grad_std=float(np.sqrt(1e-3)))),
+    # reduced copy (8 nodes, 4 pairs) for profiler captures that must stay small
+    "regular8_resnet18_b8_nb": dict(n=8, d=11_689_512, topology="regular", degree=4, pairs=4, bits=8, mode=1, H=3,
+                                    lr=0.05, seed=3, cfg=dict(objective=1, nonblocking=1,
+                                                              grad_std=float(np.sqrt(1e-3)))),
     # n = 256 nodes, d = 2^20, least squares on bf16 data (512 x 2^20 per data group, 16 groups of 16 nodes),
     # random 8-regular graph, 128 pairs per launch, 2-bit codes, non-blocking, H = 4 steps of batch 64.
     # every node takes its H steps in every launch (all nodes compute between interactions), which keeps the
@@ -171,6 +175,19 @@ def measured_peak():
         except Exception:
             pass
     return 6650.0, "fallback"
+
+
+def aggregate_over_ranks(ms_local, pairs_local, dist=None, device="cpu"):
+    """Whole-job figure for independent replicas: time = max over ranks, work = sum over ranks.
+    Returns (ms_max, pairs_total). `dist` is an initialised torch.distributed module or None."""
+    if dist is None:
+        return ms_local, pairs_local
+    import torch
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    p = torch.tensor([pairs_local], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(p, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(p.item())
 
 
 def dist_env():
@@ -308,18 +325,15 @@ def run_ours(args, wl, name):
     barrier()
     clocks = sampler.stop()
     gpu_launches = sw.kernel_launches() - l0
-    ms = ev0.elapsed_time(ev1)
-    if use_dist:
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = world * npairs_total / (ms * 1e-3)
+    ms_local = ev0.elapsed_time(ev1)
+    ms, pairs_all = aggregate_over_ranks(ms_local, npairs_total, dist if use_dist else None, "cuda")
+    value = pairs_all / (ms * 1e-3)
 
     # fused interaction kernel: average launch duration inside the timed region
     if ev_mid:
         kern_ms = sum(a.elapsed_time(b) for a, b in ev_mid) / len(ev_mid)
     else:
-        kern_ms = ms / K
+        kern_ms = ms_local / K
     per_launch_bytes = interaction_bytes(wl["d"], wl["bits"], wl["mode"]) * npairs_total / K
     achieved = per_launch_bytes / (kern_ms * 1e-3) / 1e9
     peak, peak_kind = measured_peak()
@@ -346,12 +360,9 @@ def run_ours(args, wl, name):
     e2e_ms = ev0.elapsed_time(ev1)
     wall_ms = (time.perf_counter() - t0) * 1e3
     e2e_ms = max(e2e_ms, wall_ms)
-    if use_dist:
-        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
     e2e_pairs = sum(len(p) for p in launches[W:W + e2e_steps])
-    e2e = {"value": world * e2e_pairs / (e2e_ms * 1e-3), "unit": UNIT,
+    e2e_ms, e2e_pairs_all = aggregate_over_ranks(e2e_ms, e2e_pairs, dist if use_dist else None, "cuda")
+    e2e = {"value": e2e_pairs_all / (e2e_ms * 1e-3), "unit": UNIT,
            "h2d_bytes_per_step": int(np.mean([len(p) * 16 for p in launches[W:W + e2e_steps]])),
            "d2h_bytes_per_step": int(d2h / e2e_steps)}
 
