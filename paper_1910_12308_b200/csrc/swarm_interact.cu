@@ -13,6 +13,14 @@
 namespace swarm {
 
 constexpr int kWarpsPerCta = 4;
+
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may become
+// resident while its predecessor in the stream drains; it must not touch global memory before
+// grid_dependency_wait() returns (predecessor complete and flushed). Signalling early lets the
+// successor's CTAs occupy SM slots as soon as this grid has none left to schedule, which hides the
+// launch latency between back-to-back interaction launches.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_signal() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 constexpr int kSub = 4;          // sub-blocks per block
 constexpr int kSubCoords = 256;  // coordinates per sub-block
 
@@ -25,6 +33,8 @@ constexpr int kSubCoords = 256;  // coordinates per sub-block
 template <int BITS>
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
 interact_blocking_kernel(StoreView s, const PairList pairs, int64_t total_warps) {
+  grid_dependency_signal();
+  grid_dependency_wait();
   const int lane = threadIdx.x & 31;
   const int64_t warp = (int64_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
   if (warp >= total_warps) return;
@@ -128,6 +138,8 @@ interact_identity_kernel(StoreView s, const PairList pairs, int64_t total_warps)
 template <int BITS>
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
 interact_nonblocking_kernel(StoreView s, const PairList pairs, int64_t total_warps) {
+  grid_dependency_signal();
+  grid_dependency_wait();
   const int lane = threadIdx.x & 31;
   const int64_t warp = (int64_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
   if (warp >= total_warps) return;
@@ -279,20 +291,37 @@ publish_encode_kernel(StoreView s, const uint32_t* __restrict__ wctr, int64_t to
 // -----------------------------------------------------------------------------------------
 static inline unsigned ctas_for(int64_t warps) { return (unsigned)((warps + kWarpsPerCta - 1) / kWarpsPerCta); }
 
+template <typename Kernel>
+static cudaError_t launch_dependent(Kernel kernel, dim3 grid, dim3 block, cudaStream_t st, const StoreView& s,
+                                    const PairList& pairs, int64_t warps) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, s, pairs, warps);
+}
+
 cudaError_t launch_interact_blocking(const StoreView& s, const PairList& pairs, int npairs, int bits,
                                      cudaStream_t st, int* launches) {
   if (npairs == 0) return cudaSuccess;
   const int64_t warps = (int64_t)npairs * s.nblk;
   const dim3 grid(ctas_for(warps)), block(kWarpsPerCta * 32);
+  cudaError_t e = cudaSuccess;
   switch (bits) {
-    case 2: interact_blocking_kernel<2><<<grid, block, 0, st>>>(s, pairs, warps); break;
-    case 4: interact_blocking_kernel<4><<<grid, block, 0, st>>>(s, pairs, warps); break;
-    case 8: interact_blocking_kernel<8><<<grid, block, 0, st>>>(s, pairs, warps); break;
+    case 2: e = launch_dependent(interact_blocking_kernel<2>, grid, block, st, s, pairs, warps); break;
+    case 4: e = launch_dependent(interact_blocking_kernel<4>, grid, block, st, s, pairs, warps); break;
+    case 8: e = launch_dependent(interact_blocking_kernel<8>, grid, block, st, s, pairs, warps); break;
     case 32: interact_identity_kernel<<<grid, block, 0, st>>>(s, pairs, warps); break;
     default: return cudaErrorInvalidValue;
   }
   ++*launches;
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_interact_nonblocking(const StoreView& s, const PairList& pairs, int npairs, int bits,
@@ -300,14 +329,15 @@ cudaError_t launch_interact_nonblocking(const StoreView& s, const PairList& pair
   if (npairs == 0) return cudaSuccess;
   const int64_t warps = (int64_t)npairs * s.nblk;
   const dim3 grid(ctas_for(warps)), block(kWarpsPerCta * 32);
+  cudaError_t e = cudaSuccess;
   switch (bits) {
-    case 2: interact_nonblocking_kernel<2><<<grid, block, 0, st>>>(s, pairs, warps); break;
-    case 4: interact_nonblocking_kernel<4><<<grid, block, 0, st>>>(s, pairs, warps); break;
-    case 8: interact_nonblocking_kernel<8><<<grid, block, 0, st>>>(s, pairs, warps); break;
+    case 2: e = launch_dependent(interact_nonblocking_kernel<2>, grid, block, st, s, pairs, warps); break;
+    case 4: e = launch_dependent(interact_nonblocking_kernel<4>, grid, block, st, s, pairs, warps); break;
+    case 8: e = launch_dependent(interact_nonblocking_kernel<8>, grid, block, st, s, pairs, warps); break;
     default: return cudaErrorInvalidValue;
   }
   ++*launches;
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_publish(const StoreView& s, const uint32_t* wctr_dev, int bits, cudaStream_t st, int* launches) {

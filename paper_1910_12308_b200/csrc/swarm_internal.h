@@ -21,8 +21,8 @@ struct NodeDesc {
 
 // Descriptor lists travel either inline in the kernel parameters (short lists: no copy engine
 // involved, which matters when a launch is only a few microseconds long) or through device memory.
-constexpr int kInlinePairs = 8;
-constexpr int kInlineNodes = 16;
+constexpr int kInlinePairs = 64;
+constexpr int kInlineNodes = 64;
 struct PairList {
   const PairDesc* ptr;
   int32_t n;
