@@ -197,17 +197,33 @@ def dist_env():
 # ---------------------------------------------------------------------------------------------------
 # CPU checker timing (reported baseline; also the whole of --impl reference)
 # ---------------------------------------------------------------------------------------------------
+def oracle_sample(wl, max_pairs):
+    """A bounded sample of the workload for the CPU checker: the same d, objective and code width, but only
+    as many nodes as the sampled pairs need (complete graph among them, one data matrix), because the
+    checker's cost per interaction does not depend on n while its set-up (Philox normals in double) does."""
+    p = max(1, min(wl["pairs"], max_pairs))
+    if wl["n"] * wl["d"] <= (1 << 27):
+        return dict(wl), wl["pairs"]
+    small = dict(wl, n=2 * p, topology="complete", degree=0, pairs=p)
+    cfg = dict(wl["cfg"])
+    if cfg.get("lsq_groups", 0) > 0:
+        cfg["lsq_groups"] = 1
+    small["cfg"] = cfg
+    return small, p
+
+
 def time_oracle(wl, budget_s, max_launches, threads=None):
     from oracle import swarm_oracle as o
     cores = len(os.sched_getaffinity(0))
-    T = min(wl["pairs"], cores) if threads is None else threads
+    wl, P = oracle_sample(wl, cores if threads is None else threads)
+    T = min(P, cores) if threads is None else threads
     orc = o.OracleSwarm(wl["n"], wl["d"], wl["topology"], wl["degree"], wl["seed"])
     if wl["cfg"]:
         orc.configure(**wl["cfg"])
     sched = PairSchedule(wl, orc.adj)
     done, t_total, launches = 0, 0.0, 0
     while launches < max_launches and (t_total < budget_s or launches == 0):
-        pairs = sched.next()
+        pairs = sched.next()[:P]
         t0 = time.perf_counter()
         if wl["H"] > 0:
             orc.local_steps(stepping_nodes(wl, pairs), wl["H"], wl["lr"])
@@ -216,7 +232,7 @@ def time_oracle(wl, budget_s, max_launches, threads=None):
         assert rc == 0
         done += len(pairs)
         launches += 1
-    return done / t_total, T, launches, t_total
+    return done / t_total, T, launches, t_total, wl
 
 
 def run_reference(args, wl, name):
@@ -380,10 +396,13 @@ def run_ours(args, wl, name):
                      "algorithmic_bytes_per_launch": per_launch_bytes, "kernel_ms": kern_ms},
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        v, T, nl, tt = time_oracle(wl, budget_s=10.0, max_launches=40)
-        v1, _, nl1, tt1 = time_oracle(wl, budget_s=3.0, max_launches=1, threads=1)
+        v, T, nl, tt, swl = time_oracle(wl, budget_s=10.0, max_launches=40)
+        v1, _, nl1, tt1, _ = time_oracle(wl, budget_s=3.0, max_launches=1, threads=1)
+        what = ("the workload itself" if swl["n"] == wl["n"]
+                else f"a {swl['n']}-node sample of the workload (same d, objective, bits)")
         out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": T, "kind": "oracle",
-                               "sample": f"{nl} launches of {wl['pairs']} pairs at full d ({tt:.1f} s) on {T} host threads",
+                               "sample": f"{nl} launches of {swl['pairs']} pairs at full d ({tt:.1f} s) on {T} host "
+                                         f"threads, {what}; local steps included where the workload has them",
                                "single_thread_value": v1}
     if use_dist:
         dist.destroy_process_group()
