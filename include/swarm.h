@@ -104,6 +104,15 @@ int swarm_init(swarm_ctx **out, int32_t n, int64_t d, swarm_topology topo, uint6
  * Errors: ESTATE (no objective), EINVAL (H < 0, count < 0, duplicate id), ERANGE. */
 int swarm_local_steps(swarm_ctx *ctx, const int32_t *node_ids_host, int32_t count, int32_t H, float lr);
 
+/* Section 3, "Sequential model": as swarm_local_steps, but every listed node takes a geometric number
+ * of steps with mean mean_H (the analysis' stand-in for Poisson-clock activation; E[H_i^2] = 2H^2 - H).
+ * The count of node i is the index of the first success in Bernoulli(1/mean_H) trials drawn from the
+ * counter-based generator (stream 11, row i, event = the node's step counter), capped at 1024.
+ * out_steps_host (may be NULL) receives the `count` step counts.
+ * Errors: as swarm_local_steps; EINVAL for mean_H < 1. */
+int swarm_local_steps_geometric(swarm_ctx *ctx, const int32_t *node_ids_host, int32_t count, int32_t mean_H, float lr,
+                                int32_t *out_steps_host);
+
 /* Algorithm 1, interaction lines; Corollary 1 for Enc/Dec. `pairs_host` holds npairs disjoint
  * directed edges of G. bits in {2, 4, 8}: lattice quantizer with that many bits per
  * coordinate; bits = 32 (blocking only): identity quantizer (Corollary 2).

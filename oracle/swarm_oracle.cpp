@@ -61,7 +61,7 @@ constexpr uint32_t kWeyl0 = 0x9E3779B9u, kWeyl1 = 0xBB67AE85u;
 enum Stream : uint32_t {
   kStreamInit = 1, kStreamDataA = 2, kStreamDataNoise = 3, kStreamXStar = 4,
   kStreamNodeScalars = 5, kStreamTopology = 6, kStreamPairs = 7,
-  kStreamMinibatch = 8, kStreamSynthGrad = 9, kStreamRounding = 10
+  kStreamMinibatch = 8, kStreamSynthGrad = 9, kStreamRounding = 10, kStreamStepCount = 11
 };
 
 void philox(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
@@ -430,6 +430,19 @@ void local_step_lsq(Swarm& s, int i, float lr) {
   }
 }
 
+// Number of local steps of a node as a geometric random variable of mean H (Section 3, "Sequential
+// model"): Bernoulli trials with success probability 1/H, the count is the index of the first
+// success. Trial t of node i at step counter e uses word t of stream 11; capped at 1024 trials.
+constexpr int kMaxGeometricTrials = 1024;
+int geometric_steps(const Swarm& s, int node, uint32_t event, int mean_h) {
+  for (int t = 0; t < kMaxGeometricTrials; ++t) {
+    uint32_t wd[4];
+    s.rng.words((uint32_t)(t / 4), (uint32_t)node, event, kStreamStepCount, wd);
+    if (uniform_int(wd[t % 4], (uint32_t)mean_h) == 0) return t + 1;
+  }
+  return kMaxGeometricTrials;
+}
+
 // ---------------------------------------------------------------------------
 // Interactions
 // ---------------------------------------------------------------------------
@@ -685,6 +698,28 @@ int orc_local_steps(void* h, const int32_t* nodes, int32_t count, int32_t H, flo
   for (int t = 0; t < count; ++t) {
     const int i = nodes[t];
     for (int q = 0; q < H; ++q) {
+      if (s.cfg.objective == 1) local_step_synth(s, i, lr); else local_step_lsq(s, i, lr);
+      s.ls[i] += 1;
+    }
+  }
+  return 0;
+}
+
+// Local steps with a geometric number of steps per node (mean mean_h); out_steps receives the counts.
+int orc_local_steps_geometric(void* h, const int32_t* nodes, int32_t count, int32_t mean_h, float lr, int32_t* out_steps) {
+  Swarm& s = *(Swarm*)h;
+  if (s.cfg.objective == 0 || mean_h < 1 || count < 0) return -1;
+  std::vector<uint8_t> seen(s.n, 0);
+  for (int t = 0; t < count; ++t) {
+    if (nodes[t] < 0 || nodes[t] >= s.n) return -2;
+    if (seen[nodes[t]]) return -1;
+    seen[nodes[t]] = 1;
+  }
+  for (int t = 0; t < count; ++t) {
+    const int i = nodes[t];
+    const int steps = geometric_steps(s, i, s.ls[i], mean_h);
+    if (out_steps) out_steps[t] = steps;
+    for (int q = 0; q < steps; ++q) {
       if (s.cfg.objective == 1) local_step_synth(s, i, lr); else local_step_lsq(s, i, lr);
       s.ls[i] += 1;
     }

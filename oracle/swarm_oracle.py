@@ -60,6 +60,7 @@ def lib():
         "orc_minibatch_rows": (C.c_int, [vp, C.c_int32, C.c_uint32, i32p]),
         "orc_sample_pairs": (C.c_int, [vp, C.c_int32, i32p, i32p]),
         "orc_local_steps": (C.c_int, [vp, i32p, C.c_int32, C.c_int32, C.c_float]),
+        "orc_local_steps_geometric": (C.c_int, [vp, i32p, C.c_int32, C.c_int32, C.c_float, i32p]),
         "orc_interact": (C.c_int, [vp, i32p, C.c_int32, C.c_int32, C.c_int32, C.c_int32]),
         "orc_publish": (C.c_int, [vp, C.c_int32]),
         "orc_mean_model": (None, [vp, f32p]),
@@ -280,6 +281,14 @@ class OracleSwarm:
     def local_steps(self, nodes, H, lr):
         nodes = np.ascontiguousarray(nodes, dtype=np.int32)
         return int(lib().orc_local_steps(self._h, nodes.ctypes.data_as(C.POINTER(C.c_int32)), len(nodes), H, lr))
+
+    def local_steps_geometric(self, nodes, mean_h, lr):
+        """Returns (rc, steps taken per listed node)."""
+        nodes = np.ascontiguousarray(nodes, dtype=np.int32)
+        steps = np.zeros(len(nodes), dtype=np.int32)
+        rc = int(lib().orc_local_steps_geometric(self._h, nodes.ctypes.data_as(C.POINTER(C.c_int32)), len(nodes), mean_h,
+                                                 lr, steps.ctypes.data_as(C.POINTER(C.c_int32))))
+        return rc, steps
 
     def interact(self, pairs, bits, mode=BLOCKING, threads=1):
         pairs = np.ascontiguousarray(pairs, dtype=np.int32).reshape(-1, 2)

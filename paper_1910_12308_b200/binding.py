@@ -21,7 +21,7 @@ T_X, T_B, T_CODES, T_EXPS, T_ADJ, T_A, T_BVEC, T_XSTAR, T_SCALARS, T_COUNTERS = 
 TOPOLOGY = {"complete": TOPO_COMPLETE, "ring": TOPO_RING, "regular": TOPO_REGULAR}
 
 EXPORTS = [
-    "swarm_set_allocator", "swarm_init", "swarm_local_steps", "swarm_interact", "swarm_mean_model",
+    "swarm_set_allocator", "swarm_init", "swarm_local_steps", "swarm_local_steps_geometric", "swarm_interact", "swarm_mean_model",
     "swarm_potential", "swarm_configure", "swarm_sample_pairs", "swarm_publish", "swarm_get_tensor",
     "swarm_set_tensor", "swarm_get_state", "swarm_set_state", "swarm_model_ptr", "swarm_set_stream",
     "swarm_sync", "swarm_potential_static", "swarm_kernel_launches", "swarm_last_cuda_error", "swarm_strerror", "swarm_destroy",
@@ -77,6 +77,7 @@ def load():
         "swarm_set_allocator": (C.c_int, [ALLOC_FN, FREE_FN, vp]),
         "swarm_init": (C.c_int, [C.POINTER(vp), i32, i64, SwarmTopology, u64]),
         "swarm_local_steps": (C.c_int, [vp, C.POINTER(i32), i32, i32, f32]),
+        "swarm_local_steps_geometric": (C.c_int, [vp, C.POINTER(i32), i32, i32, f32, C.POINTER(i32)]),
         "swarm_interact": (C.c_int, [vp, C.POINTER(SwarmPair), i32, i32, i32]),
         "swarm_mean_model": (C.c_int, [vp, vp]),
         "swarm_potential": (C.c_int, [vp, C.POINTER(C.c_double)]),
@@ -181,6 +182,14 @@ class Swarm:
     def local_steps(self, nodes, H, lr):
         nodes = np.ascontiguousarray(nodes, dtype=np.int32)
         return self._L.swarm_local_steps(self._h, nodes.ctypes.data_as(C.POINTER(C.c_int32)), len(nodes), H, lr)
+
+    def local_steps_geometric(self, nodes, mean_h, lr):
+        """Returns (rc, steps taken per listed node)."""
+        nodes = np.ascontiguousarray(nodes, dtype=np.int32)
+        steps = np.zeros(len(nodes), dtype=np.int32)
+        rc = self._L.swarm_local_steps_geometric(self._h, nodes.ctypes.data_as(C.POINTER(C.c_int32)), len(nodes), mean_h,
+                                                 lr, steps.ctypes.data_as(C.POINTER(C.c_int32)))
+        return rc, steps
 
     def interact(self, pairs, bits, mode=BLOCKING):
         arr, ptr = _pairs_array(pairs)

@@ -528,6 +528,49 @@ int swarm_local_steps(swarm_ctx* c, const int32_t* node_ids, int32_t count, int3
   return SWARM_OK;
 }
 
+int swarm_local_steps_geometric(swarm_ctx* c, const int32_t* node_ids, int32_t count, int32_t mean_H, float lr,
+                                int32_t* out_steps) {
+  if (!c || count < 0 || mean_H < 1 || (count > 0 && !node_ids)) return SWARM_EINVAL;
+  if (c->cfg.objective == SWARM_OBJ_NONE) return SWARM_ESTATE;
+  if (count > c->n) return SWARM_EINVAL;
+  {
+    std::vector<uint8_t> seen((size_t)c->n, 0);
+    for (int t = 0; t < count; ++t)
+      if (node_ids[t] < 0 || node_ids[t] >= c->n) return SWARM_ERANGE;
+    for (int t = 0; t < count; ++t) {
+      if (seen[node_ids[t]]) return SWARM_EINVAL;
+      seen[node_ids[t]] = 1;
+    }
+  }
+  // step counts: first success among Bernoulli(1/mean_H) trials, one generator word per trial
+  const uint32_t key0 = (uint32_t)c->seed, key1 = (uint32_t)(c->seed >> 32);
+  std::vector<int32_t> steps((size_t)count);
+  int32_t max_steps = 0;
+  for (int t = 0; t < count; ++t) {
+    const uint32_t node = (uint32_t)node_ids[t], event = c->ls[node_ids[t]];
+    int32_t h = 1024;
+    for (int trial = 0; trial < 1024; ++trial) {
+      const uint4 w = philox4x32_10((uint32_t)(trial >> 2), node, event, kStreamStepCount, key0, key1);
+      const uint32_t word = (trial & 3) == 0 ? w.x : (trial & 3) == 1 ? w.y : (trial & 3) == 2 ? w.z : w.w;
+      if (uniform_int(word, (uint32_t)mean_H) == 0) { h = trial + 1; break; }
+    }
+    steps[t] = h;
+    max_steps = std::max(max_steps, h);
+  }
+  // one launch sequence per distinct count (nodes with equal counts travel together)
+  std::vector<int32_t> bucket;
+  for (int32_t h = 1; h <= max_steps; ++h) {
+    bucket.clear();
+    for (int t = 0; t < count; ++t)
+      if (steps[t] == h) bucket.push_back(node_ids[t]);
+    if (bucket.empty()) continue;
+    const int rc = swarm_local_steps(c, bucket.data(), (int32_t)bucket.size(), h, lr);
+    if (rc != SWARM_OK) return rc;
+  }
+  if (out_steps) std::copy(steps.begin(), steps.end(), out_steps);
+  return SWARM_OK;
+}
+
 int swarm_interact(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, int32_t bits, int32_t mode) {
   if (!c || npairs < 0 || (npairs > 0 && !pairs)) return SWARM_EINVAL;
   if (mode != SWARM_BLOCKING && mode != SWARM_NONBLOCKING) return SWARM_EINVAL;

@@ -256,6 +256,23 @@ def test_batched_tensor_core_least_squares_steps(n, groups, d, m, batch):
         inject(orc, gpu, what=("X",))
 
 
+def test_geometric_step_counts_match():
+    cfg = dict(objective=1, grad_std=0.03, drift_std=0.1)
+    orc, gpu = make_pair(12, 3000, seed=61, **cfg)
+    inject(orc, gpu)
+    for rnd in range(4):
+        nodes = list(range(12)) if rnd % 2 == 0 else [5, 1, 9]
+        rc_o, steps_o = orc.local_steps_geometric(nodes, 3, 0.05)
+        rc_g, steps_g = gpu.local_steps_geometric(nodes, 3, 0.05)
+        assert rc_o == 0 and rc_g == 0
+        assert np.array_equal(steps_o, steps_g)                    # integer draws: bit-exact
+        for i in range(12):
+            assert rel_err(gpu.get(g.T_X, i), orc.X[i]) < TOL
+            assert gpu.get(g.T_COUNTERS, i)[1] == orc.ls[i]
+        inject(orc, gpu, what=("X",))
+    assert gpu.local_steps_geometric([0], 0, 0.1)[0] == -1
+
+
 # ---- mean model and potential ----------------------------------------------------------------------
 
 @pytest.mark.parametrize("n,d", [(2, 1), (3, 1027), (8, 4096), (17, 2500), (64, 3000)])

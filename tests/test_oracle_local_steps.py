@@ -133,3 +133,41 @@ def test_local_step_validation():
     assert s.local_steps([3], 1, 0.1) == -2
     assert s.local_steps([], 2, 0.1) == 0
     assert s.local_steps([1], 0, 0.1) == 0 and int(s.ls[1]) == 0
+
+
+def test_geometric_step_counts_have_the_stated_moments():
+    """Section 3 (sequential model): H_i geometric with mean H; the analysis uses E[H_i^2] = 2H^2 - H."""
+    for H in (1, 2, 4):
+        s = o.OracleSwarm(64, 4, "complete", seed=H)
+        s.configure(objective=1, grad_std=0.0)
+        draws = []
+        for _ in range(120):
+            rc, steps = s.local_steps_geometric(list(range(64)), H, 0.0)
+            assert rc == 0
+            draws.extend(steps.tolist())
+        draws = np.array(draws, dtype=np.float64)
+        N = len(draws)
+        assert draws.min() >= 1
+        if H == 1:
+            assert np.all(draws == 1)
+            continue
+        var = H * H - H                                  # variance of the geometric law
+        assert abs(draws.mean() - H) < 5 * np.sqrt(var / N)
+        assert abs((draws**2).mean() - (2 * H * H - H)) < 0.08 * (2 * H * H - H)
+        assert abs((draws == 1).mean() - 1 / H) < 5 * np.sqrt((1 / H) * (1 - 1 / H) / N)
+        assert abs((draws == 2).mean() - (1 - 1 / H) / H) < 5 * np.sqrt(0.25 / N)
+
+
+def test_geometric_steps_equal_that_many_plain_steps():
+    s1, s2 = lsq(seed=9), lsq(seed=9)
+    rc, steps = s1.local_steps_geometric([0, 2], 3, 0.1)
+    assert rc == 0 and s1.ls.tolist() == [int(steps[0]), 0, int(steps[1])]
+    s2.local_steps([0], int(steps[0]), 0.1)
+    s2.local_steps([2], int(steps[1]), 0.1)
+    assert np.array_equal(s1.X, s2.X)
+    # the draw restated from the counter layout: first trial whose word maps to 0 under uniform_int(., mean)
+    t = 0
+    while o.uniform_int(o.philox([t // 4, 2, 0, 11], [9, 0])[t % 4], 3) != 0:
+        t += 1
+    assert steps[1] == t + 1
+    assert s1.local_steps_geometric([0], 0, 0.1)[0] == -1
