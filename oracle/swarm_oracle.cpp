@@ -61,7 +61,7 @@ constexpr uint32_t kWeyl0 = 0x9E3779B9u, kWeyl1 = 0xBB67AE85u;
 enum Stream : uint32_t {
   kStreamInit = 1, kStreamDataA = 2, kStreamDataNoise = 3, kStreamXStar = 4,
   kStreamNodeScalars = 5, kStreamTopology = 6, kStreamPairs = 7,
-  kStreamMinibatch = 8, kStreamSynthGrad = 9, kStreamRounding = 10, kStreamStepCount = 11
+  kStreamMinibatch = 8, kStreamSynthGrad = 9, kStreamRounding = 10, kStreamStepCount = 11, kStreamOwnRounding = 12
 };
 
 void philox(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
@@ -217,7 +217,7 @@ uint32_t get_code(const uint8_t* block_bytes, int k, int bits) {
 // ---------------------------------------------------------------------------
 struct Config {
   int32_t objective;      // 0 none, 1 synthetic gradient, 2 least squares
-  int32_t nonblocking;    // 1: base snapshots exist
+  int32_t nonblocking;    // 1: base snapshots exist; 2: also the nodes' own registers (two-register protocol)
   float init_std, offset_std;
   float grad_std, drift_std;
   int32_t lsq_m, lsq_batch, lsq_dtype, lsq_groups;
@@ -250,6 +250,13 @@ struct Swarm {
   std::vector<uint32_t> w, ls;       // write counters, local-step counters
   uint32_t launch = 0;
   int32_t b_stale = 0;
+  // two-register protocol (Section 3, "The Communication Registers"): the register a node writes
+  // itself holds a 16-bit encoding of its snapshot; `codes` is then the register others write.
+  std::vector<uint16_t> own;         // n * d
+  std::vector<int8_t> oexps;         // n * nblk
+  std::vector<uint32_t> wo;          // write counters of the own registers
+  std::vector<uint32_t> tau;         // interactions since the node last initiated
+  int32_t p_mode = 0;                // convention the buffers were last written in: 0 none/blocking, 1 single buffer, 2 registers
   // objective data
   std::vector<float> offset, drift, shift;   // per-node scalars
   std::vector<float> A;              // groups * m * d
@@ -351,7 +358,10 @@ void init_state(Swarm& s) {
   s.exps.assign((size_t)n * s.nblk, 0);
   s.pbits.assign(n, 0);
   s.w.assign(n, 0); s.ls.assign(n, 0);
-  s.launch = 0; s.b_stale = 0;
+  s.launch = 0; s.b_stale = 0; s.p_mode = 0;
+  s.tau.assign(n, 0); s.wo.assign(n, 0);
+  if (c.nonblocking == 2) { s.own.assign((size_t)n * d, 0); s.oexps.assign((size_t)n * s.nblk, 0); }
+  else { s.own.clear(); s.oexps.clear(); }
 
   s.A.clear(); s.bvec.clear(); s.xstar.clear(); s.groups = 0;
   if (c.objective == 2) {
@@ -518,10 +528,11 @@ void publish(Swarm& s, int bits) {
     }
   }
   for (int i = 0; i < n; ++i) { s.w[i] += 1; s.pbits[i] = bits; }
+  s.p_mode = 1;
 }
 
-bool needs_publish(const Swarm& s, int bits) {
-  if (s.b_stale) return true;
+bool needs_publish(const Swarm& s, int bits, int mode) {
+  if (s.b_stale || s.p_mode != mode) return true;
   for (int i = 0; i < s.n; ++i) if (s.pbits[i] != bits) return true;
   return false;
 }
@@ -565,6 +576,121 @@ void interact_nonblocking(Swarm& s, int a, int b, int bits) {
     for (int k = 0; k < len; ++k) { xa[k0 + k] = new_x[k]; ba[k0 + k] = new_x[k]; }
   }
   s.w[a] += 1; s.w[b] += 1;
+}
+
+// ---------------------------------------------------------------------------
+// Two-register protocol: Algorithm 1 with its chain of three decodes.
+//   own register of node k      O_k = Enc16(X^_k)    written only by k, 16 bits per coordinate,
+//                                                    step of an 8-bit code of the guard distance
+//                                                    (the writer does not know its readers' keys)
+//   current register of node k  P_k = Enc_b(X_k)     written by whoever last interacted with k,
+//                                                    scaled by the exact distance to its decoding
+//                                                    key Q(X^_k) (the writer knows that key)
+// ---------------------------------------------------------------------------
+constexpr int kOwnBits = 16;
+constexpr int kOwnResolutionBits = 8;
+
+uint32_t own_uniform(const Rng& rng, uint32_t owner, uint32_t w, int64_t k) {
+  uint32_t words[4];
+  rng.words((uint32_t)(k / 8), owner, w, kStreamOwnRounding, words);
+  const uint32_t word = words[(k % 8) / 2];
+  return (k % 2 == 0) ? (word & 0xFFFFu) : (word >> 16);
+}
+
+// Write O_i = Enc16(v) for one block with exponent eo, return the written lattice points in qhat.
+void write_own_block(Swarm& s, int i, int64_t blk, const float* v, int len, int eo, float* qhat) {
+  const int64_t k0 = blk * kBlock;
+  uint16_t* o = s.own.data() + (int64_t)i * s.d + k0;
+  for (int k = 0; k < len; ++k) {
+    const int32_t q = enc_q(v[k], eo, own_uniform(s.rng, (uint32_t)i, s.wo[i], k0 + k));
+    o[k] = (uint16_t)code_of(q, kOwnBits);
+    qhat[k] = (float)q * pow2f(eo);
+  }
+  s.oexps[(int64_t)i * s.nblk + blk] = (int8_t)eo;
+}
+
+// Write P_i = Enc_b(v) for one block, scaled by the exact distance to the key `key`.
+void write_current_block(Swarm& s, int i, int64_t blk, const float* v, const float* key, int len, int bits) {
+  const int64_t k0 = blk * kBlock;
+  float rho = 0.0f, M = 0.0f;
+  for (int k = 0; k < len; ++k) {
+    rho = std::max(rho, std::fabs(v[k] - key[k]));
+    M = std::max(M, std::max(std::fabs(v[k]), std::fabs(key[k])));
+  }
+  const int e = exponent_rule(rho, M, bits);
+  const size_t block_bytes = (size_t)kBlock * bits / 8;
+  uint8_t* c = s.code_row(i) + blk * block_bytes;
+  std::memset(c, 0, block_bytes);
+  for (int k = 0; k < len; ++k)
+    put_code(c, k, code_of(enc_q(v[k], e, sr_uniform(s.rng, (uint32_t)i, s.w[i], k0 + k)), bits), bits);
+  s.exp_row(i)[blk] = (int8_t)e;
+}
+
+// Initial register contents: every node's registers hold encodings of its snapshot.
+void register_publish(Swarm& s, int bits) {
+  const int n = s.n; const int64_t d = s.d;
+  if (s.b_stale) { s.B = s.X; s.b_stale = 0; }
+  std::vector<float> qhat(kBlock);
+  for (int64_t blk = 0; blk < s.nblk; ++blk) {
+    const int64_t k0 = blk * kBlock;
+    const int len = (int)std::min<int64_t>(kBlock, d - k0);
+    float rho = 0.0f, M = 0.0f;
+    for (int k = 0; k < len; ++k) {
+      float lo = s.base(0)[k0 + k], hi = lo;
+      for (int i = 0; i < n; ++i) {
+        const float v = s.base(i)[k0 + k];
+        lo = std::min(lo, v); hi = std::max(hi, v);
+        M = std::max(M, std::fabs(v));
+      }
+      rho = std::max(rho, hi - lo);
+    }
+    const int eo = exponent_rule(rho, M, kOwnResolutionBits);
+    for (int i = 0; i < n; ++i) {
+      write_own_block(s, i, blk, s.base(i) + k0, len, eo, qhat.data());
+      write_current_block(s, i, blk, s.base(i) + k0, qhat.data(), len, bits);
+    }
+  }
+  for (int i = 0; i < n; ++i) { s.wo[i] += 1; s.w[i] += 1; s.pbits[i] = bits; }
+  s.p_mode = 2;
+}
+
+void interact_registers(Swarm& s, int a, int b, int bits) {
+  const int64_t d = s.d;
+  float* xa = s.x(a); float* ba = s.base(a);
+  const size_t block_bytes = (size_t)kBlock * bits / 8;
+  std::vector<float> new_x(kBlock), avg(kBlock), qhat_b(kBlock), qhat_new(kBlock);
+  for (int64_t blk = 0; blk < s.nblk; ++blk) {
+    const int64_t k0 = blk * kBlock;
+    const int len = (int)std::min<int64_t>(kBlock, d - k0);
+    const uint8_t* ca = s.code_row(a) + blk * block_bytes;
+    const uint8_t* cb = s.code_row(b) + blk * block_bytes;
+    const uint16_t* oa = s.own.data() + (int64_t)a * d + k0;
+    const uint16_t* ob = s.own.data() + (int64_t)b * d + k0;
+    const int eoa = s.oexps[(int64_t)a * s.nblk + blk], eob = s.oexps[(int64_t)b * s.nblk + blk];
+    const int epa = s.exp_row(a)[blk], epb = s.exp_row(b)[blk];
+    float spread = 0.0f, dmax = 0.0f, M = 0.0f;
+    for (int k = 0; k < len; ++k) {
+      const float snap = ba[k0 + k];
+      const float qhat_a = dec(snap, oa[k], eoa, kOwnBits);                   // Q(X^_a): local, key = own snapshot
+      const float Qa = dec(qhat_a, get_code(ca, k, bits), epa, bits);         // Q(X_a)  <- Dec(Q(X^_a), Enc(X_a))
+      qhat_b[k] = dec(snap, ob[k], eob, kOwnBits);                            // Q(X^_b) <- Dec(X^_a, Enc(X^_b))
+      const float Qb = dec(qhat_b[k], get_code(cb, k, bits), epb, bits);      // Q(X_b)  <- Dec(Q(X^_b), Enc(X_b))
+      const float av = 0.5f * (Qa + Qb);
+      const float D = snap - xa[k0 + k];                                      // pending local update (eta * h)
+      const float nx = av - D;
+      avg[k] = av; new_x[k] = nx;
+      spread = std::max(spread, std::fabs(Qa - Qb));
+      dmax = std::max(dmax, std::fabs(D));
+      M = std::max(M, std::max(std::fabs(nx), std::fabs(av)));
+    }
+    const float rho = 2.0f * spread + dmax;
+    const int eo = exponent_rule(rho, M, kOwnResolutionBits);
+    write_own_block(s, a, blk, new_x.data(), len, eo, qhat_new.data());       // own register of a
+    write_current_block(s, a, blk, new_x.data(), qhat_new.data(), len, bits); // current register of a
+    write_current_block(s, b, blk, avg.data(), qhat_b.data(), len, bits);     // current register of b
+    for (int k = 0; k < len; ++k) { xa[k0 + k] = new_x[k]; ba[k0 + k] = new_x[k]; }
+  }
+  s.wo[a] += 1; s.w[a] += 1; s.w[b] += 1;
 }
 
 int validate_pairs(const Swarm& s, const int32_t* pairs, int npairs) {
@@ -626,7 +752,7 @@ void orc_destroy(void* h) { delete (Swarm*)h; }
 
 int orc_configure(void* h, const Config* c) {
   Swarm& s = *(Swarm*)h;
-  if (c->objective < 0 || c->objective > 2) return -1;
+  if (c->objective < 0 || c->objective > 2 || c->nonblocking < 0 || c->nonblocking > 2) return -1;
   if (c->objective == 2) {
     if (c->lsq_m < 1 || c->lsq_batch < 1 || c->lsq_dtype < 0 || c->lsq_dtype > 1) return -1;
     if (c->lsq_groups < 0 || (c->lsq_groups > 0 && s.n % c->lsq_groups != 0)) return -1;
@@ -731,15 +857,18 @@ int orc_local_steps_geometric(void* h, const int32_t* nodes, int32_t count, int3
 // independent) pairs over plain std::thread workers.
 int orc_interact(void* h, const int32_t* pairs, int32_t npairs, int32_t bits, int32_t mode, int32_t threads) {
   Swarm& s = *(Swarm*)h;
-  if (npairs < 0 || (mode != 0 && mode != 1)) return -1;
+  if (npairs < 0 || mode < 0 || mode > 2) return -1;
   if (!(bits == 2 || bits == 4 || bits == 8 || (bits == 32 && mode == 0))) return -1;
   if (mode == 1 && !s.cfg.nonblocking) return -4;
+  if (mode == 2 && s.cfg.nonblocking != 2) return -4;
   const int v = validate_pairs(s, pairs, npairs);
   if (v != 0) return v;
-  if (mode == 1 && needs_publish(s, bits)) publish(s, bits);
+  if (mode == 1 && needs_publish(s, bits, 1)) publish(s, bits);
+  if (mode == 2 && needs_publish(s, bits, 2)) register_publish(s, bits);
   auto run = [&](int p) {
     if (mode == 0) interact_blocking(s, pairs[2 * p], pairs[2 * p + 1], bits);
-    else interact_nonblocking(s, pairs[2 * p], pairs[2 * p + 1], bits);
+    else if (mode == 1) interact_nonblocking(s, pairs[2 * p], pairs[2 * p + 1], bits);
+    else interact_registers(s, pairs[2 * p], pairs[2 * p + 1], bits);
   };
   if (threads <= 1 || npairs <= 1) {
     for (int p = 0; p < npairs; ++p) run(p);
@@ -750,10 +879,31 @@ int orc_interact(void* h, const int32_t* pairs, int32_t npairs, int32_t bits, in
       pool.emplace_back([&, t]() { for (int p = t; p < npairs; p += T) run(p); });
     for (auto& th : pool) th.join();
   }
-  // a blocking exchange moves X without refreshing the base snapshots
+  // a blocking exchange moves X without refreshing the base snapshots and leaves the buffers in its
+  // own convention (keys = partner models)
+  if (mode == 0 && npairs > 0 && bits != 32) s.p_mode = 0;
   if (mode == 0 && s.cfg.nonblocking && npairs > 0) s.b_stale = 1;
+  // staleness clocks (appendix, "Notation and Auxiliary Potential Functions"): the interactions of a
+  // launch are taken in list order; an interaction resets its initiator and ages everybody else
+  for (int p = 0; p < npairs; ++p) {
+    for (int i = 0; i < s.n; ++i) s.tau[i] += 1;
+    s.tau[pairs[2 * p]] = 0;
+  }
   return 0;
 }
+
+int orc_register_publish(void* h, int32_t bits) {
+  Swarm& s = *(Swarm*)h;
+  if (s.cfg.nonblocking != 2 || !(bits == 2 || bits == 4 || bits == 8)) return -1;
+  register_publish(s, bits);
+  return 0;
+}
+
+uint16_t* orc_own(void* h) { Swarm& s = *(Swarm*)h; return s.own.empty() ? nullptr : s.own.data(); }
+int8_t* orc_oexps(void* h) { Swarm& s = *(Swarm*)h; return s.oexps.empty() ? nullptr : s.oexps.data(); }
+uint32_t* orc_wo(void* h) { return ((Swarm*)h)->wo.data(); }
+uint32_t* orc_tau(void* h) { return ((Swarm*)h)->tau.data(); }
+int32_t* orc_p_mode(void* h) { return &((Swarm*)h)->p_mode; }
 
 int orc_publish(void* h, int32_t bits) {
   Swarm& s = *(Swarm*)h;

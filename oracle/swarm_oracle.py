@@ -63,6 +63,9 @@ def lib():
         "orc_local_steps_geometric": (C.c_int, [vp, i32p, C.c_int32, C.c_int32, C.c_float, i32p]),
         "orc_interact": (C.c_int, [vp, i32p, C.c_int32, C.c_int32, C.c_int32, C.c_int32]),
         "orc_publish": (C.c_int, [vp, C.c_int32]),
+        "orc_register_publish": (C.c_int, [vp, C.c_int32]),
+        "orc_own": (u16p, [vp]), "orc_oexps": (i8p, [vp]), "orc_wo": (u32p, [vp]), "orc_tau": (u32p, [vp]),
+        "orc_p_mode": (i32p, [vp]),
         "orc_mean_model": (None, [vp, f32p]),
         "orc_potential": (C.c_double, [vp]),
     }
@@ -151,7 +154,7 @@ def unpack_block(packed, count, bits):
 # ---- swarm state ---------------------------------------------------------------------------
 
 TOPOLOGY = {"complete": 0, "ring": 1, "regular": 2}
-BLOCKING, NONBLOCKING = 0, 1
+BLOCKING, NONBLOCKING, REGISTERS = 0, 1, 2
 
 
 class OracleSwarm:
@@ -230,6 +233,26 @@ class OracleSwarm:
         return _view(lib().orc_b_stale(self._h), (1,), np.int32)
 
     @property
+    def own(self):
+        return _view(lib().orc_own(self._h), (self.n, self.d), np.uint16)
+
+    @property
+    def oexps(self):
+        return _view(lib().orc_oexps(self._h), (self.n, self.nblk), np.int8)
+
+    @property
+    def wo(self):
+        return _view(lib().orc_wo(self._h), (self.n,), np.uint32)
+
+    @property
+    def tau(self):
+        return _view(lib().orc_tau(self._h), (self.n,), np.uint32)
+
+    @property
+    def p_mode(self):
+        return _view(lib().orc_p_mode(self._h), (1,), np.int32)
+
+    @property
     def groups(self):
         return int(lib().orc_groups(self._h))
 
@@ -297,6 +320,9 @@ class OracleSwarm:
 
     def publish(self, bits):
         return int(lib().orc_publish(self._h, bits))
+
+    def register_publish(self, bits):
+        return int(lib().orc_register_publish(self._h, bits))
 
     def mean_model(self):
         out = np.zeros(self.d, dtype=np.float32)

@@ -1,0 +1,118 @@
+"""Pins for the two-register protocol: Algorithm 1 with its chain of three decodes
+(Section 3, "The Communication Registers" and "The Communication Procedure")."""
+import numpy as np
+import pytest
+
+from oracle import swarm_oracle as o
+
+
+def make(n=4, d=2100, seed=1, topo="complete", **kw):
+    s = o.OracleSwarm(n, d, topo, seed=seed)
+    cfg = dict(objective=1, nonblocking=2, grad_std=0.03, drift_std=0.2)
+    cfg.update(kw)
+    s.configure(**cfg)
+    return s
+
+
+def decode_own(s, reader, owner):
+    """Q(X^_owner) as `reader` obtains it: own register of `owner` decoded with reader's snapshot as key."""
+    out = np.zeros(s.d, dtype=np.float32)
+    for k in range(s.d):
+        out[k] = o.dec(float(s.B[reader, k]), int(s.own[owner, k]), int(s.oexps[owner, k // 1024]), 16)
+    return out
+
+
+def decode_current(s, key, owner, bits):
+    out = np.zeros(s.d, dtype=np.float32)
+    for blk in range(s.nblk):
+        k0, k1 = blk * 1024, min(s.d, (blk + 1) * 1024)
+        codes = o.unpack_block(s.packed_codes(owner, bits)[blk * 128 * bits:(blk + 1) * 128 * bits], k1 - k0, bits)
+        e = int(s.exps[owner, blk])
+        out[k0:k1] = [o.dec(float(key[k0 + t]), int(codes[t]), e, bits) for t in range(k1 - k0)]
+    return out
+
+
+def steps(exps, d):
+    return np.repeat(2.0 ** exps.astype(np.float64), 1024)[:d]
+
+
+@pytest.mark.parametrize("bits", [2, 4, 8])
+def test_register_publish_chain_decodes_every_snapshot(bits):
+    s = make(offset_std=0.3)
+    assert s.register_publish(bits) == 0
+    assert int(s.p_mode[0]) == 2 and s.wo.tolist() == [1] * 4 and s.w.tolist() == [1] * 4
+    for blk in range(s.nblk):
+        assert np.all(s.oexps[:, blk] == s.oexps[0, blk])            # one step per block for the own registers
+    for reader, owner in ((0, 1), (3, 2), (2, 2)):
+        qhat = decode_own(s, reader, owner)
+        assert np.all(np.abs(qhat.astype(np.float64) - s.B[owner]) < steps(s.oexps[owner], s.d))
+        assert np.array_equal(qhat, decode_own(s, owner, owner))    # every in-range reader sees the same point
+        cur = decode_current(s, qhat, owner, bits)
+        assert np.all(np.abs(cur.astype(np.float64) - s.B[owner]) < steps(s.exps[owner], s.d))
+    # the current register is scaled by the distance to its own key: far finer than the own register's range
+    assert np.all(s.exps.astype(int) <= s.oexps.astype(int) - (bits - 2))
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_register_interaction_follows_algorithm_1(bits):
+    s = make(offset_std=0.1)
+    s.local_steps([0, 1, 2, 3], 2, 0.05)
+    s.register_publish(bits)
+    s.local_steps([1], 2, 0.05)
+    X0, B0, own0, codes0 = s.X.copy(), s.B.copy(), s.own.copy(), s.codes.copy()
+    Qa = decode_current(s, decode_own(s, 1, 1), 1, bits)            # Q(X_a)  <- Dec(Q(X^_a), Enc(X_a))
+    qhat_b = decode_own(s, 1, 3)                                    # Q(X^_b) <- Dec(X^_a, Enc(X^_b))
+    Qb = decode_current(s, qhat_b, 3, bits)                         # Q(X_b)  <- Dec(Q(X^_b), Enc(X_b))
+    assert s.interact([[1, 3]], bits, o.REGISTERS) == 0
+    avg = np.float32(0.5) * (Qa + Qb)
+    D = B0[1] - X0[1]
+    assert np.array_equal(s.X[1], avg - D)                          # X_a <- Q(X_a)/2 + Q(X_b)/2 - eta h
+    assert np.array_equal(s.B[1], s.X[1])
+    # one-way: the responder's model, snapshot and own register are untouched; bystanders entirely
+    for i in (0, 2, 3):
+        assert np.array_equal(s.X[i], X0[i]) and np.array_equal(s.B[i], B0[i]) and np.array_equal(s.own[i], own0[i])
+    for i in (0, 2):
+        assert np.array_equal(s.codes[i], codes0[i])
+    # registers written: both of a hold its new model, the current register of b holds the average,
+    # decodable by b with its own (unchanged) Q(X^_b)
+    qa_new = decode_own(s, 1, 1)
+    assert np.all(np.abs(qa_new.astype(np.float64) - s.X[1]) < steps(s.oexps[1], s.d))
+    assert np.all(np.abs(decode_current(s, qa_new, 1, bits).astype(np.float64) - s.X[1]) < steps(s.exps[1], s.d))
+    assert np.array_equal(decode_own(s, 3, 3), qhat_b)
+    assert np.all(np.abs(decode_current(s, qhat_b, 3, bits).astype(np.float64) - avg) < steps(s.exps[3], s.d))
+    assert s.wo.tolist() == [1, 2, 1, 1] and s.w.tolist() == [1, 2, 1, 2]
+    assert s.tau.tolist() == [1, 0, 1, 1]
+
+
+def test_registers_remove_the_aliasing_plateau_of_the_single_buffer_form():
+    """With per-node offsets far larger than the per-coordinate spread, the single-buffer form stalls at a
+    large Gamma (keys leave the decode window for good); the register chain keeps every current-register
+    decode inside its window, so the swarm contracts to its quantisation floor."""
+    results = {}
+    for mode, nb in ((o.NONBLOCKING, 1), (o.REGISTERS, 2)):
+        s = make(n=8, d=1024, seed=3, nonblocking=nb, offset_std=0.3, grad_std=0.0, drift_std=0.0)
+        g0 = s.potential()
+        for _ in range(600):
+            s.interact(s.sample_pairs(1), 8, mode)
+        results[mode] = s.potential() / g0
+    assert results[o.NONBLOCKING] > 0.05          # the documented plateau
+    assert results[o.REGISTERS] < 1e-4
+
+
+def test_staleness_clocks_and_mode_switches():
+    s = make(n=5, d=64)
+    s.interact([[0, 1], [2, 3]], 8, o.REGISTERS)
+    assert s.tau.tolist() == [1, 2, 0, 2, 2]
+    assert int(s.p_mode[0]) == 2
+    s.interact([[4, 0]], 8, o.NONBLOCKING)           # other convention: buffers are re-published first
+    assert int(s.p_mode[0]) == 1 and s.tau.tolist() == [2, 3, 1, 3, 0]
+    w_before = s.w.copy()
+    s.interact([[1, 2]], 8, o.REGISTERS)
+    assert int(s.p_mode[0]) == 2
+    assert np.all(s.w >= w_before + 1)               # register_publish rewrote every current register
+    s.interact([[3, 4]], 8, o.BLOCKING)
+    assert int(s.p_mode[0]) == 0 and int(s.b_stale[0]) == 1
+    plain = o.OracleSwarm(4, 16, "complete")
+    plain.configure(objective=1, nonblocking=1)
+    assert plain.interact([[0, 1]], 8, o.REGISTERS) == -4
+    assert plain.register_publish(8) == -1
