@@ -51,7 +51,7 @@ typedef struct { int32_t a, b; } swarm_pair;
 typedef struct { int32_t kind, degree; } swarm_topology;
 enum { SWARM_TOPO_COMPLETE = 0, SWARM_TOPO_RING = 1, SWARM_TOPO_REGULAR = 2 };
 
-enum { SWARM_BLOCKING = 0, SWARM_NONBLOCKING = 1 };
+enum { SWARM_BLOCKING = 0, SWARM_NONBLOCKING = 1, SWARM_REGISTERS = 2 };
 enum { SWARM_OBJ_NONE = 0, SWARM_OBJ_SYNTH = 1, SWARM_OBJ_LSQ = 2 };
 enum { SWARM_F32 = 0, SWARM_BF16 = 1 };
 
@@ -69,7 +69,8 @@ enum {
  * not variances. Applying it re-creates the whole state from the seed. */
 typedef struct {
   int32_t objective;     /* SWARM_OBJ_*                                                           */
-  int32_t nonblocking;   /* 1: keep base snapshots B and allow SWARM_NONBLOCKING                  */
+  int32_t nonblocking;   /* 1: keep base snapshots B and allow SWARM_NONBLOCKING; 2: also keep the nodes'
+                            own registers (16 bits per coordinate) and allow SWARM_REGISTERS       */
   float   init_std;      /* X^i[k] = init_std * z + o_i                                           */
   float   offset_std;    /* per-node scalar o_i ~ N(0, offset_std^2)                              */
   float   grad_std;      /* SYNTH: stochastic gradient = c_i + grad_std * z                       */
@@ -124,6 +125,16 @@ int swarm_local_steps_geometric(swarm_ctx *ctx, const int32_t *node_ids_host, in
  *     result as model and snapshot, and writes Enc(new model) to its own buffer and Enc(average)
  *     to the responder's; the responder's model is not touched. Buffers are (re)published from
  *     the snapshots first if they do not hold `bits`-bit codes or a blocking call intervened.
+ *   SWARM_REGISTERS: the two-register protocol of Section 3 ("The Communication Registers") with
+ *     Algorithm 1's chain of three decodes. Each node has an own register (16-bit encoding of its
+ *     snapshot, written only by the node, with the step of an 8-bit code of the guard distance) and a
+ *     current register (b-bit, written by its last interaction partner, scaled by the exact distance to
+ *     its decoding key). The initiator a computes Q(X^a) = Dec(B^a, own_a), Q(X_a) = Dec(Q(X^a), cur_a),
+ *     Q(X^b) = Dec(B^a, own_b), Q(X_b) = Dec(Q(X^b), cur_b), adopts Q(X_a)/2 + Q(X_b)/2 - (B^a - X^a) as
+ *     model and snapshot, rewrites both of its registers and writes Enc(average) to cur_b. Registers are
+ *     (re)initialised from the snapshots first when they are not in this convention at `bits` bits.
+ * Every call advances the staleness clocks: interactions of a launch are taken in list order, each
+ * resets its initiator's clock and ages all other nodes by one.
  * Errors: EINVAL (bits, mode, npairs < 0, NULL), ERANGE, EPAIR, ESTATE. */
 int swarm_interact(swarm_ctx *ctx, const swarm_pair *pairs_host, int32_t npairs, int32_t bits, int32_t mode);
 
@@ -151,6 +162,10 @@ int swarm_sample_pairs(swarm_ctx *ctx, int32_t max_pairs, swarm_pair *out_pairs_
  * swarm_interact, SWARM_NONBLOCKING). Errors: ESTATE without base snapshots, EINVAL. */
 int swarm_publish(swarm_ctx *ctx, int32_t bits);
 
+/* Initialise both registers of every node from the snapshots (see swarm_interact, SWARM_REGISTERS).
+ * Errors: ESTATE unless configured with nonblocking = 2, EINVAL. */
+int swarm_register_publish(swarm_ctx *ctx, int32_t bits);
+
 /* State access (checkpointing, test injection). `which` selects the array, `node` the row
  * (ignored for whole-context arrays). bytes must equal the row size exactly. Both synchronise. */
 enum {
@@ -163,7 +178,10 @@ enum {
   SWARM_T_BVEC = 6,     /* lsq_m floats                              */
   SWARM_T_XSTAR = 7,    /* d floats, node ignored                    */
   SWARM_T_SCALARS = 8,  /* 3 floats: offset o_i, drift c_i, shift mu_i */
-  SWARM_T_COUNTERS = 9  /* 3 uint32: buffer write counter, local-step counter, code width of the buffer */
+  SWARM_T_COUNTERS = 9, /* 3 uint32: buffer write counter, local-step counter, code width of the buffer */
+  SWARM_T_OWN = 10,     /* d uint16: own register (ESTATE unless nonblocking = 2)                           */
+  SWARM_T_OEXPS = 11,   /* nblk int8: exponents of the own register                                         */
+  SWARM_T_CLOCKS = 12   /* 2 uint32: write counter of the own register, staleness clock tau                 */
 };
 int swarm_get_tensor(swarm_ctx *ctx, int32_t which, int32_t node, void *dst_host, size_t bytes);
 int swarm_set_tensor(swarm_ctx *ctx, int32_t which, int32_t node, const void *src_host, size_t bytes);
@@ -171,6 +189,10 @@ int swarm_set_tensor(swarm_ctx *ctx, int32_t which, int32_t node, const void *sr
 /* Whole-context counters: launch counter of the pair sampler and the "snapshots stale" flag. */
 int swarm_get_state(swarm_ctx *ctx, uint32_t *launch_host, int32_t *b_stale_host);
 int swarm_set_state(swarm_ctx *ctx, uint32_t launch, int32_t b_stale);
+/* Convention the communication buffers were last written in: 0 none / blocking, 1 single buffer
+ * (SWARM_NONBLOCKING), 2 registers (SWARM_REGISTERS). */
+int swarm_get_buffer_mode(swarm_ctx *ctx, int32_t *mode_host);
+int swarm_set_buffer_mode(swarm_ctx *ctx, int32_t mode);
 
 /* Device pointer and row pitch (in elements) of X, for callers that consume models in place.
  * Valid until the next swarm_configure / swarm_destroy. */

@@ -13,16 +13,17 @@ from . import build as _build
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 
-BLOCKING, NONBLOCKING = 0, 1
+BLOCKING, NONBLOCKING, REGISTERS = 0, 1, 2
 TOPO_COMPLETE, TOPO_RING, TOPO_REGULAR = 0, 1, 2
 OBJ_NONE, OBJ_SYNTH, OBJ_LSQ = 0, 1, 2
 F32, BF16 = 0, 1
-T_X, T_B, T_CODES, T_EXPS, T_ADJ, T_A, T_BVEC, T_XSTAR, T_SCALARS, T_COUNTERS = range(10)
+T_X, T_B, T_CODES, T_EXPS, T_ADJ, T_A, T_BVEC, T_XSTAR, T_SCALARS, T_COUNTERS, T_OWN, T_OEXPS, T_CLOCKS = range(13)
 TOPOLOGY = {"complete": TOPO_COMPLETE, "ring": TOPO_RING, "regular": TOPO_REGULAR}
 
 EXPORTS = [
     "swarm_set_allocator", "swarm_init", "swarm_local_steps", "swarm_local_steps_geometric", "swarm_interact", "swarm_mean_model",
-    "swarm_potential", "swarm_configure", "swarm_sample_pairs", "swarm_publish", "swarm_get_tensor",
+    "swarm_potential", "swarm_configure", "swarm_sample_pairs", "swarm_publish", "swarm_register_publish", "swarm_get_buffer_mode",
+    "swarm_set_buffer_mode", "swarm_get_tensor",
     "swarm_set_tensor", "swarm_get_state", "swarm_set_state", "swarm_model_ptr", "swarm_set_stream",
     "swarm_sync", "swarm_potential_static", "swarm_kernel_launches", "swarm_last_cuda_error", "swarm_strerror", "swarm_destroy",
 ]
@@ -84,6 +85,9 @@ def load():
         "swarm_configure": (C.c_int, [vp, C.POINTER(SwarmConfig)]),
         "swarm_sample_pairs": (C.c_int, [vp, i32, C.POINTER(SwarmPair), C.POINTER(i32)]),
         "swarm_publish": (C.c_int, [vp, i32]),
+        "swarm_register_publish": (C.c_int, [vp, i32]),
+        "swarm_get_buffer_mode": (C.c_int, [vp, C.POINTER(i32)]),
+        "swarm_set_buffer_mode": (C.c_int, [vp, i32]),
         "swarm_get_tensor": (C.c_int, [vp, i32, i32, vp, C.c_size_t]),
         "swarm_set_tensor": (C.c_int, [vp, i32, i32, vp, C.c_size_t]),
         "swarm_get_state": (C.c_int, [vp, C.POINTER(u32), C.POINTER(i32)]),
@@ -225,6 +229,17 @@ class Swarm:
     def publish(self, bits):
         return self._L.swarm_publish(self._h, bits)
 
+    def register_publish(self, bits):
+        return self._L.swarm_register_publish(self._h, bits)
+
+    def get_buffer_mode(self):
+        m = C.c_int32()
+        self._check(self._L.swarm_get_buffer_mode(self._h, C.byref(m)), "swarm_get_buffer_mode")
+        return m.value
+
+    def set_buffer_mode(self, mode):
+        self._check(self._L.swarm_set_buffer_mode(self._h, mode), "swarm_set_buffer_mode")
+
     def set_stream(self, stream):
         ptr = getattr(stream, "cuda_stream", stream)
         self._check(self._L.swarm_set_stream(self._h, ptr), "swarm_set_stream")
@@ -247,7 +262,8 @@ class Swarm:
             T_X: (np.float32, self.d), T_B: (np.float32, self.d), T_CODES: (np.uint8, self.nblk * 1024),
             T_EXPS: (np.int8, self.nblk), T_ADJ: (np.int32, self.degree), T_A: (np.float32, m * self.d),
             T_BVEC: (np.float32, m), T_XSTAR: (np.float32, self.d), T_SCALARS: (np.float32, 3),
-            T_COUNTERS: (np.uint32, 3),
+            T_COUNTERS: (np.uint32, 3), T_OWN: (np.uint16, self.d), T_OEXPS: (np.int8, self.nblk),
+            T_CLOCKS: (np.uint32, 2),
         }[which]
 
     def get(self, which, node=0):

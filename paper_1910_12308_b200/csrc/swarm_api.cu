@@ -42,6 +42,8 @@ struct swarm_ctx {
   std::vector<int32_t> adj;          // n * degree
   std::vector<uint32_t> w, ls;       // buffer write counters, local-step counters
   std::vector<int32_t> pbits;        // code width currently held by each buffer (0 = none)
+  std::vector<uint32_t> wo, tau;     // own-register write counters, staleness clocks
+  int32_t p_mode = 0;                // convention the buffers were last written in (0 none, 1 single buffer, 2 registers)
   uint32_t launch_ctr = 0;
   int32_t b_stale = 0;
   int32_t groups = 0, nodes_per_group = 0;
@@ -51,6 +53,8 @@ struct swarm_ctx {
   float* B = nullptr;
   uint8_t* codes = nullptr;
   int8_t* exps = nullptr;
+  uint16_t* own = nullptr;           // two-register protocol: own registers [n][pitch]
+  int8_t* oexps = nullptr;           // [n][nblk]
   int32_t* adj_dev = nullptr;
   float* scalars = nullptr;          // n * 3
   void* A = nullptr;
@@ -107,7 +111,7 @@ void dev_free(swarm_ctx* c, void* p) {
 
 StoreView view_of(const swarm_ctx* c) {
   StoreView s;
-  s.X = c->X; s.B = c->B; s.codes = c->codes; s.exps = c->exps;
+  s.X = c->X; s.B = c->B; s.codes = c->codes; s.exps = c->exps; s.own = c->own; s.oexps = c->oexps;
   s.pitch = c->pitch; s.d = c->d; s.nblk = c->nblk; s.n = c->n;
   s.key0 = (uint32_t)c->seed; s.key1 = (uint32_t)(c->seed >> 32);
   return s;
@@ -187,6 +191,8 @@ void free_objective(swarm_ctx* c) {
   dev_free(c, c->tc_resid); c->tc_resid = nullptr;
   dev_free(c, c->convert_tmp); c->convert_tmp = nullptr;
   dev_free(c, c->B); c->B = nullptr;
+  dev_free(c, c->own); c->own = nullptr;
+  dev_free(c, c->oexps); c->oexps = nullptr;
   c->groups = 0; c->nodes_per_group = 0;
 }
 
@@ -222,6 +228,11 @@ int apply_config(swarm_ctx* c, const swarm_config& cfg) {
     c->B = (float*)dev_alloc(c, (size_t)n * row_bytes);
     if (!c->B) return SWARM_ENOMEM;
   }
+  if (cfg.nonblocking == 2) {
+    c->own = (uint16_t*)dev_alloc(c, (size_t)n * c->pitch * sizeof(uint16_t));
+    c->oexps = (int8_t*)dev_alloc(c, (size_t)n * c->nblk);
+    if (!c->own || !c->oexps) return SWARM_ENOMEM;
+  }
   if (cfg.objective == SWARM_OBJ_LSQ) {
     c->groups = cfg.lsq_groups > 0 ? cfg.lsq_groups : n;
     c->nodes_per_group = n / c->groups;
@@ -242,6 +253,10 @@ int apply_config(swarm_ctx* c, const swarm_config& cfg) {
   SW_CUDA(c, cudaMemsetAsync(c->X, 0, (size_t)n * row_bytes, c->stream));
   SW_CUDA(c, cudaMemsetAsync(c->codes, 0, (size_t)n * c->nblk * kBlockCoords, c->stream));
   SW_CUDA(c, cudaMemsetAsync(c->exps, 0, (size_t)n * c->nblk, c->stream));
+  if (c->own) {
+    SW_CUDA(c, cudaMemsetAsync(c->own, 0, (size_t)n * c->pitch * sizeof(uint16_t), c->stream));
+    SW_CUDA(c, cudaMemsetAsync(c->oexps, 0, (size_t)n * c->nblk, c->stream));
+  }
   SW_CUDA(c, launch_node_scalars(c->scalars, n, cfg.offset_std, cfg.drift_std, s.key0, s.key1, c->stream, &nl));
   SW_CUDA(c, launch_init_models(s, c->scalars, cfg.init_std, c->stream, &nl));
   if (c->B) SW_CUDA(c, cudaMemcpyAsync(c->B, c->X, (size_t)n * row_bytes, cudaMemcpyDeviceToDevice, c->stream));
@@ -253,14 +268,17 @@ int apply_config(swarm_ctx* c, const swarm_config& cfg) {
   std::fill(c->w.begin(), c->w.end(), 0u);
   std::fill(c->ls.begin(), c->ls.end(), 0u);
   std::fill(c->pbits.begin(), c->pbits.end(), 0);
+  std::fill(c->wo.begin(), c->wo.end(), 0u);
+  std::fill(c->tau.begin(), c->tau.end(), 0u);
   c->launch_ctr = 0;
   c->b_stale = 0;
+  c->p_mode = 0;
   return SWARM_OK;
 }
 
 int validate_config(const swarm_ctx* c, const swarm_config* cfg) {
   if (cfg->objective < SWARM_OBJ_NONE || cfg->objective > SWARM_OBJ_LSQ) return SWARM_EINVAL;
-  if (cfg->nonblocking != 0 && cfg->nonblocking != 1) return SWARM_EINVAL;
+  if (cfg->nonblocking < 0 || cfg->nonblocking > 2) return SWARM_EINVAL;
   if (!(cfg->init_std >= 0.0f) || !(cfg->offset_std >= 0.0f) || !(cfg->grad_std >= 0.0f) || !(cfg->drift_std >= 0.0f))
     return SWARM_EINVAL;
   if (cfg->objective == SWARM_OBJ_LSQ) {
@@ -310,7 +328,40 @@ int do_publish(swarm_ctx* c, int bits) {
   rc = stage_release(c, slot);
   if (rc != SWARM_OK) return rc;
   for (int i = 0; i < c->n; ++i) { c->w[i] += 1; c->pbits[i] = bits; }
+  c->p_mode = 1;
   return SWARM_OK;
+}
+
+int do_register_publish(swarm_ctx* c, int bits) {
+  const size_t row_bytes = (size_t)c->pitch * sizeof(float);
+  if (c->b_stale) {
+    SW_CUDA(c, cudaMemcpyAsync(c->B, c->X, (size_t)c->n * row_bytes, cudaMemcpyDeviceToDevice, c->stream));
+    c->b_stale = 0;
+  }
+  void *host, *dev;
+  int slot;
+  const size_t bytes = (size_t)2 * c->n * sizeof(uint32_t);
+  int rc = stage_acquire(c, bytes, &host, &dev, &slot);
+  if (rc != SWARM_OK) return rc;
+  std::memcpy(host, c->w.data(), bytes / 2);
+  std::memcpy((char*)host + bytes / 2, c->wo.data(), bytes / 2);
+  rc = stage_commit(c, slot, bytes);
+  if (rc != SWARM_OK) return rc;
+  int nl = 0;
+  SW_CUDA(c, launch_register_publish(view_of(c), (const uint32_t*)dev, bits, c->stream, &nl));
+  c->launches += nl;
+  rc = stage_release(c, slot);
+  if (rc != SWARM_OK) return rc;
+  for (int i = 0; i < c->n; ++i) { c->w[i] += 1; c->wo[i] += 1; c->pbits[i] = bits; }
+  c->p_mode = 2;
+  return SWARM_OK;
+}
+
+bool buffers_need_publish(const swarm_ctx* c, int bits, int mode) {
+  if (c->b_stale != 0 || c->p_mode != mode) return true;
+  for (int i = 0; i < c->n; ++i)
+    if (c->pbits[i] != bits) return true;
+  return false;
 }
 
 }  // namespace
@@ -367,11 +418,11 @@ int swarm_init(swarm_ctx** out, int32_t n, int64_t d, swarm_topology topo, uint6
   c->custom_alloc = g_alloc != nullptr;
   c->alloc_fn = g_alloc; c->free_fn = g_free; c->alloc_user = g_alloc_user;
   if (!build_graph(c)) { delete c; return SWARM_EINVAL; }
-  c->w.assign(n, 0); c->ls.assign(n, 0); c->pbits.assign(n, 0);
+  c->w.assign(n, 0); c->ls.assign(n, 0); c->pbits.assign(n, 0); c->wo.assign(n, 0); c->tau.assign(n, 0);
 
   const size_t row_bytes = (size_t)c->pitch * sizeof(float);
   const size_t max_pairs = (size_t)n / 2;
-  c->stage_slot_bytes = std::max({max_pairs * sizeof(PairDesc), (size_t)n * sizeof(NodeDesc), (size_t)n * sizeof(uint32_t),
+  c->stage_slot_bytes = std::max({max_pairs * sizeof(PairDesc), (size_t)n * sizeof(NodeDesc), (size_t)2 * n * sizeof(uint32_t),
                                   (size_t)n * sizeof(LsqUnit)});
   c->stage_slot_bytes = (c->stage_slot_bytes + 255) / 256 * 256;
   c->X = (float*)dev_alloc(c, (size_t)n * row_bytes);
@@ -573,18 +624,22 @@ int swarm_local_steps_geometric(swarm_ctx* c, const int32_t* node_ids, int32_t c
 
 int swarm_interact(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, int32_t bits, int32_t mode) {
   if (!c || npairs < 0 || (npairs > 0 && !pairs)) return SWARM_EINVAL;
-  if (mode != SWARM_BLOCKING && mode != SWARM_NONBLOCKING) return SWARM_EINVAL;
+  if (mode != SWARM_BLOCKING && mode != SWARM_NONBLOCKING && mode != SWARM_REGISTERS) return SWARM_EINVAL;
   const bool quant = bits == 2 || bits == 4 || bits == 8;
   if (!(quant || (bits == 32 && mode == SWARM_BLOCKING))) return SWARM_EINVAL;
   if (mode == SWARM_NONBLOCKING && !c->cfg.nonblocking) return SWARM_ESTATE;
+  if (mode == SWARM_REGISTERS && c->cfg.nonblocking != 2) return SWARM_ESTATE;
   if (npairs > c->n / 2) return SWARM_EPAIR;
   int rc = validate_pairs(c, pairs, npairs);
   if (rc != SWARM_OK) return rc;
   DeviceGuard guard(c->device);
-  if (mode == SWARM_NONBLOCKING) {
-    bool need = c->b_stale != 0;
-    for (int i = 0; i < c->n && !need; ++i) need = c->pbits[i] != bits;
-    if (need) { rc = do_publish(c, bits); if (rc != SWARM_OK) return rc; }
+  if (mode == SWARM_NONBLOCKING && buffers_need_publish(c, bits, 1)) {
+    rc = do_publish(c, bits);
+    if (rc != SWARM_OK) return rc;
+  }
+  if (mode == SWARM_REGISTERS && buffers_need_publish(c, bits, 2)) {
+    rc = do_register_publish(c, bits);
+    if (rc != SWARM_OK) return rc;
   }
   if (npairs == 0) return SWARM_OK;
   void *host, *dev;
@@ -601,6 +656,7 @@ int swarm_interact(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, int32_
   for (int p = 0; p < npairs; ++p) {
     pd[p].a = pairs[p].a; pd[p].b = pairs[p].b;
     pd[p].wa = c->w[pairs[p].a]; pd[p].wb = c->w[pairs[p].b];
+    pd[p].woa = c->wo[pairs[p].a]; pd[p].pad = 0;
   }
   if (slot >= 0) {
     rc = stage_commit(c, slot, (size_t)npairs * sizeof(PairDesc));
@@ -608,7 +664,8 @@ int swarm_interact(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, int32_
   }
   int nl = 0;
   if (mode == SWARM_BLOCKING) SW_CUDA(c, launch_interact_blocking(view_of(c), list, npairs, bits, c->stream, &nl));
-  else SW_CUDA(c, launch_interact_nonblocking(view_of(c), list, npairs, bits, c->stream, &nl));
+  else if (mode == SWARM_NONBLOCKING) SW_CUDA(c, launch_interact_nonblocking(view_of(c), list, npairs, bits, c->stream, &nl));
+  else SW_CUDA(c, launch_interact_registers(view_of(c), list, npairs, bits, c->stream, &nl));
   c->launches += nl;
   if (slot >= 0) {
     rc = stage_release(c, slot);
@@ -620,7 +677,33 @@ int swarm_interact(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, int32_
       if (mode == SWARM_BLOCKING) { c->pbits[pairs[p].a] = bits; c->pbits[pairs[p].b] = bits; }
     }
   }
+  if (mode == SWARM_REGISTERS)
+    for (int p = 0; p < npairs; ++p) c->wo[pairs[p].a] += 1;
+  if (mode == SWARM_BLOCKING && bits != 32) c->p_mode = 0;      // buffers now follow the blocking convention
   if (mode == SWARM_BLOCKING && c->cfg.nonblocking) c->b_stale = 1;
+  // staleness clocks: interactions in list order, each resets its initiator and ages everybody else
+  for (int p = 0; p < npairs; ++p) {
+    for (int i = 0; i < c->n; ++i) c->tau[i] += 1;
+    c->tau[pairs[p].a] = 0;
+  }
+  return SWARM_OK;
+}
+
+int swarm_register_publish(swarm_ctx* c, int32_t bits) {
+  if (!c || !(bits == 2 || bits == 4 || bits == 8)) return SWARM_EINVAL;
+  if (c->cfg.nonblocking != 2) return SWARM_ESTATE;
+  DeviceGuard guard(c->device);
+  return do_register_publish(c, bits);
+}
+
+int swarm_get_buffer_mode(swarm_ctx* c, int32_t* mode) {
+  if (!c || !mode) return SWARM_EINVAL;
+  *mode = c->p_mode;
+  return SWARM_OK;
+}
+int swarm_set_buffer_mode(swarm_ctx* c, int32_t mode) {
+  if (!c || mode < 0 || mode > 2) return SWARM_EINVAL;
+  c->p_mode = mode;
   return SWARM_OK;
 }
 
@@ -711,6 +794,19 @@ static int tensor_access(swarm_ctx* c, int32_t which, int32_t node, void* host, 
       if (!c->xstar) return SWARM_ESTATE;
       dev = c->xstar; want = d * 4; break;
     case SWARM_T_SCALARS: dev = c->scalars + (size_t)node * 3; want = 12; break;
+    case SWARM_T_OWN:
+      if (!c->own) return SWARM_ESTATE;
+      dev = c->own + (size_t)node * c->pitch; want = d * 2; break;
+    case SWARM_T_OEXPS:
+      if (!c->oexps) return SWARM_ESTATE;
+      dev = c->oexps + (size_t)node * c->nblk; want = (size_t)c->nblk; break;
+    case SWARM_T_CLOCKS: {
+      if (bytes != 8) return SWARM_EINVAL;
+      uint32_t* v = (uint32_t*)host;
+      if (write) { c->wo[node] = v[0]; c->tau[node] = v[1]; }
+      else { v[0] = c->wo[node]; v[1] = c->tau[node]; }
+      return SWARM_OK;
+    }
     case SWARM_T_COUNTERS: {
       if (bytes != 12) return SWARM_EINVAL;
       uint32_t* v = (uint32_t*)host;

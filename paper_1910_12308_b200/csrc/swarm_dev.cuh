@@ -15,7 +15,7 @@ constexpr int kExpMax = 119;
 enum : uint32_t {
   kStreamInit = 1, kStreamDataA = 2, kStreamDataNoise = 3, kStreamXStar = 4,
   kStreamNodeScalars = 5, kStreamTopology = 6, kStreamPairs = 7,
-  kStreamMinibatch = 8, kStreamSynthGrad = 9, kStreamRounding = 10, kStreamStepCount = 11
+  kStreamMinibatch = 8, kStreamSynthGrad = 9, kStreamRounding = 10, kStreamStepCount = 11, kStreamOwnRounding = 12
 };
 
 // ---------------------------------------------------------------------------------------

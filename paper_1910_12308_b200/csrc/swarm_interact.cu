@@ -222,7 +222,7 @@ interact_nonblocking_kernel(StoreView s, const PairList pairs, int64_t total_war
 // -----------------------------------------------------------------------------------------
 template <int BITS>
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
-publish_range_kernel(StoreView s) {
+publish_range_kernel(StoreView s, int8_t* __restrict__ out_exps) {
   const int lane = threadIdx.x & 31;
   const int64_t blk = (int64_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
   if (blk >= s.nblk) return;
@@ -252,7 +252,7 @@ publish_range_kernel(StoreView s) {
   rho = warp_max_nonneg(rho);
   M = warp_max_nonneg(M);
   const int e = exponent_rule<BITS>(rho, M);
-  for (int i = lane; i < s.n; i += 32) s.exps[(int64_t)i * s.nblk + blk] = (int8_t)e;
+  for (int i = lane; i < s.n; i += 32) out_exps[(int64_t)i * s.nblk + blk] = (int8_t)e;
 }
 
 template <int BITS>
@@ -284,6 +284,201 @@ publish_encode_kernel(StoreView s, const uint32_t* __restrict__ wctr, int64_t to
     }
     store_codes<BITS>(c + j * (kSubCoords * BITS / 8), pk);
   }
+}
+
+// -----------------------------------------------------------------------------------------
+// Two-register protocol (Section 3, "The Communication Registers"; Algorithm 1 with its chain of
+// three decodes). Node k's own register O_k holds a 16-bit encoding of its snapshot, written only by
+// k with the step of an 8-bit code of the guard distance (its readers' keys are unknown to it); its
+// current register P_k holds a b-bit encoding written by whoever last interacted with k and scaled by
+// the exact distance to its decoding key Q(X^_k), which that writer knows.
+//   Q(X^_a) = Dec16(B_a, O_a)            local
+//   Q(X_a)  = Dec_b(Q(X^_a), P_a)        Algorithm 1, first decode
+//   Q(X^_b) = Dec16(B_a, O_b)            second decode: the partner's own register, key = own snapshot
+//   Q(X_b)  = Dec_b(Q(X^_b), P_b)        third decode
+//   X_a <- Q(X_a)/2 + Q(X_b)/2 - (B_a - X_a);  B_a <- X_a;  O_a, P_a <- Enc(X_a);  P_b <- Enc(average)
+// Traffic per coordinate: 8 + 4 + 2b/8 B read, 8 + 2 + 2b/8 B written.
+// -----------------------------------------------------------------------------------------
+constexpr int kOwnBits = 16;
+constexpr int kOwnResolutionBits = 8;
+
+__device__ __forceinline__ uint32_t own_code(const uint4& v, int i) {
+  const uint32_t word = (i < 2) ? v.x : (i < 4) ? v.y : (i < 6) ? v.z : v.w;
+  return (i & 1) ? (word >> 16) : (word & 0xFFFFu);
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(kWarpsPerCta * 32)
+interact_registers_kernel(StoreView s, const PairList pairs, int64_t total_warps) {
+  grid_dependency_signal();
+  grid_dependency_wait();
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = (int64_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
+  if (warp >= total_warps) return;
+  const int64_t pair = warp / s.nblk;
+  const int64_t blk = warp - pair * s.nblk;
+  const PairDesc pd = pairs.get(pair);
+
+  const int64_t koff = blk * kBlockCoords + lane * 8;
+  float* xa = s.X + (int64_t)pd.a * s.pitch + koff;
+  float* ba = s.B + (int64_t)pd.a * s.pitch + koff;
+  uint16_t* oa = s.own + (int64_t)pd.a * s.pitch + koff;
+  const uint16_t* ob = s.own + (int64_t)pd.b * s.pitch + koff;
+  uint8_t* ca = s.codes + (int64_t)pd.a * s.nblk * kBlockCoords + blk * (kBlockCoords * BITS / 8) + lane * BITS;
+  uint8_t* cb = s.codes + (int64_t)pd.b * s.nblk * kBlockCoords + blk * (kBlockCoords * BITS / 8) + lane * BITS;
+
+  f8 nx[kSub], av[kSub];       // loaded as X^a / B^a, overwritten with new model / average
+  uint4 va[kSub], vb[kSub];
+  uint64_t pa[kSub], pb[kSub];
+#pragma unroll
+  for (int j = 0; j < kSub; ++j) nx[j] = ld256(xa + j * kSubCoords);
+#pragma unroll
+  for (int j = 0; j < kSub; ++j) av[j] = ld256(ba + j * kSubCoords);
+#pragma unroll
+  for (int j = 0; j < kSub; ++j) {
+    va[j] = *reinterpret_cast<const uint4*>(oa + j * kSubCoords);
+    vb[j] = *reinterpret_cast<const uint4*>(ob + j * kSubCoords);
+    pa[j] = load_codes<BITS>(ca + j * (kSubCoords * BITS / 8));
+    pb[j] = load_codes<BITS>(cb + j * (kSubCoords * BITS / 8));
+  }
+  const int eoa = s.oexps[(int64_t)pd.a * s.nblk + blk], eob = s.oexps[(int64_t)pd.b * s.nblk + blk];
+  const int epa = s.exps[(int64_t)pd.a * s.nblk + blk], epb = s.exps[(int64_t)pd.b * s.nblk + blk];
+  const float so_a = pow2f_exact(eoa), io_a = pow2f_exact(-eoa), so_b = pow2f_exact(eob), io_b = pow2f_exact(-eob);
+  const float sp_a = pow2f_exact(epa), ip_a = pow2f_exact(-epa), sp_b = pow2f_exact(epb), ip_b = pow2f_exact(-epb);
+
+  constexpr uint32_t mask = (1u << BITS) - 1u;
+  float spread = 0.0f, dmax = 0.0f, M = 0.0f, rho_b = 0.0f, M_b = 0.0f;
+#pragma unroll
+  for (int j = 0; j < kSub; ++j)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float snap = av[j].v[i];
+      const float qhat_a = decode_value<kOwnBits>(snap, own_code(va[j], i), io_a, so_a);
+      const float Qa = decode_value<BITS>(qhat_a, (uint32_t)(pa[j] >> (i * BITS)) & mask, ip_a, sp_a);
+      const float qhat_b = decode_value<kOwnBits>(snap, own_code(vb[j], i), io_b, so_b);
+      const float Qb = decode_value<BITS>(qhat_b, (uint32_t)(pb[j] >> (i * BITS)) & mask, ip_b, sp_b);
+      const float avg = __fmul_rn(0.5f, __fadd_rn(Qa, Qb));
+      const float D = __fsub_rn(snap, nx[j].v[i]);
+      const float x_new = __fsub_rn(avg, D);
+      spread = fmaxf(spread, fabsf(__fsub_rn(Qa, Qb)));
+      dmax = fmaxf(dmax, fabsf(D));
+      M = fmaxf(M, fmaxf(fabsf(x_new), fabsf(avg)));
+      rho_b = fmaxf(rho_b, fabsf(__fsub_rn(avg, qhat_b)));        // distance of the average to b's decoding key
+      M_b = fmaxf(M_b, fmaxf(fabsf(avg), fabsf(qhat_b)));
+      nx[j].v[i] = x_new;
+      av[j].v[i] = avg;
+    }
+  spread = warp_max_nonneg(spread);
+  dmax = warp_max_nonneg(dmax);
+  M = warp_max_nonneg(M);
+  rho_b = warp_max_nonneg(rho_b);
+  M_b = warp_max_nonneg(M_b);
+  const int eo = exponent_rule<kOwnResolutionBits>(__fadd_rn(__fmul_rn(2.0f, spread), dmax), M);
+  const int ep_b = exponent_rule<BITS>(rho_b, M_b);
+  const float so = pow2f_exact(eo), io = pow2f_exact(-eo), ipb_new = pow2f_exact(-ep_b);
+
+  // own register of a (16 bits) and current register of b; distance of the new model to its own key
+  const uint32_t group0 = (uint32_t)(blk * (kBlockCoords / 8) + lane);
+  float rho_a = 0.0f, M_a = 0.0f;
+#pragma unroll
+  for (int j = 0; j < kSub; ++j) {
+    const uint32_t g = group0 + j * (kSubCoords / 8);
+    const uint4 ro = philox4x32_10(g, (uint32_t)pd.a, pd.woa, kStreamOwnRounding, s.key0, s.key1);
+    const uint4 rb = philox4x32_10(g, (uint32_t)pd.b, pd.wb, kStreamRounding, s.key0, s.key1);
+    uint32_t ow[4] = {0u, 0u, 0u, 0u};
+    uint64_t pkb = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      int32_t cell;
+      const int32_t q = encode_index(nx[j].v[i], io, sr_u16(ro, i), cell);
+      ow[i >> 1] |= ((uint32_t)q & 0xFFFFu) << ((i & 1) * 16);
+      const float qhat_new = __fmul_rn(__int2float_rn(q), so);
+      rho_a = fmaxf(rho_a, fabsf(__fsub_rn(nx[j].v[i], qhat_new)));
+      M_a = fmaxf(M_a, fmaxf(fabsf(nx[j].v[i]), fabsf(qhat_new)));
+      pkb |= (uint64_t)((uint32_t)encode_index(av[j].v[i], ipb_new, sr_u16(rb, i), cell) & mask) << (i * BITS);
+    }
+    *reinterpret_cast<uint4*>(oa + j * kSubCoords) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+    store_codes<BITS>(cb + j * (kSubCoords * BITS / 8), pkb);
+  }
+  rho_a = warp_max_nonneg(rho_a);
+  M_a = warp_max_nonneg(M_a);
+  const int ep_a = exponent_rule<BITS>(rho_a, M_a);
+  const float ipa_new = pow2f_exact(-ep_a);
+#pragma unroll
+  for (int j = 0; j < kSub; ++j) {
+    const uint32_t g = group0 + j * (kSubCoords / 8);
+    const uint4 ra = philox4x32_10(g, (uint32_t)pd.a, pd.wa, kStreamRounding, s.key0, s.key1);
+    uint64_t pka = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      int32_t cell;
+      pka |= (uint64_t)((uint32_t)encode_index(nx[j].v[i], ipa_new, sr_u16(ra, i), cell) & mask) << (i * BITS);
+    }
+    st256(xa + j * kSubCoords, nx[j]);
+    st256(ba + j * kSubCoords, nx[j]);
+    store_codes<BITS>(ca + j * (kSubCoords * BITS / 8), pka);
+  }
+  if (lane == 0) {
+    s.oexps[(int64_t)pd.a * s.nblk + blk] = (int8_t)eo;
+    s.exps[(int64_t)pd.a * s.nblk + blk] = (int8_t)ep_a;
+    s.exps[(int64_t)pd.b * s.nblk + blk] = (int8_t)ep_b;
+  }
+}
+
+// Initial register contents: own register = 16-bit encoding of the snapshot with the block's common
+// exponent (already in oexps), current register = b-bit encoding scaled by the distance to that point.
+template <int BITS>
+__global__ void __launch_bounds__(kWarpsPerCta * 32)
+register_publish_encode_kernel(StoreView s, const uint32_t* __restrict__ wctr, int64_t total_warps) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = (int64_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
+  if (warp >= total_warps) return;
+  const int64_t node = warp / s.nblk;
+  const int64_t blk = warp - node * s.nblk;
+  const int64_t koff = blk * kBlockCoords + lane * 8;
+  const float* row = s.B + node * s.pitch + koff;
+  uint16_t* o = s.own + node * s.pitch + koff;
+  uint8_t* c = s.codes + node * s.nblk * kBlockCoords + blk * (kBlockCoords * BITS / 8) + lane * BITS;
+  const int eo = s.oexps[node * s.nblk + blk];
+  const float so = pow2f_exact(eo), io = pow2f_exact(-eo);
+  const uint32_t w = wctr[node], wo = wctr[s.n + node];
+  constexpr uint32_t mask = (1u << BITS) - 1u;
+  const uint32_t group0 = (uint32_t)(blk * (kBlockCoords / 8) + lane);
+  f8 v[kSub];
+#pragma unroll
+  for (int j = 0; j < kSub; ++j) v[j] = ld256(row + j * kSubCoords);
+  float rho = 0.0f, M = 0.0f;
+#pragma unroll
+  for (int j = 0; j < kSub; ++j) {
+    const uint4 ro = philox4x32_10(group0 + j * (kSubCoords / 8), (uint32_t)node, wo, kStreamOwnRounding, s.key0, s.key1);
+    uint32_t ow[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      int32_t cell;
+      const int32_t q = encode_index(v[j].v[i], io, sr_u16(ro, i), cell);
+      ow[i >> 1] |= ((uint32_t)q & 0xFFFFu) << ((i & 1) * 16);
+      const float qhat = __fmul_rn(__int2float_rn(q), so);
+      rho = fmaxf(rho, fabsf(__fsub_rn(v[j].v[i], qhat)));
+      M = fmaxf(M, fmaxf(fabsf(v[j].v[i]), fabsf(qhat)));
+    }
+    *reinterpret_cast<uint4*>(o + j * kSubCoords) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+  }
+  rho = warp_max_nonneg(rho);
+  M = warp_max_nonneg(M);
+  const int ep = exponent_rule<BITS>(rho, M);
+  const float ip = pow2f_exact(-ep);
+#pragma unroll
+  for (int j = 0; j < kSub; ++j) {
+    const uint4 r = philox4x32_10(group0 + j * (kSubCoords / 8), (uint32_t)node, w, kStreamRounding, s.key0, s.key1);
+    uint64_t pk = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      int32_t cell;
+      pk |= (uint64_t)((uint32_t)encode_index(v[j].v[i], ip, sr_u16(r, i), cell) & mask) << (i * BITS);
+    }
+    store_codes<BITS>(c + j * (kSubCoords * BITS / 8), pk);
+  }
+  if (lane == 0) s.exps[node * s.nblk + blk] = (int8_t)ep;
 }
 
 // -----------------------------------------------------------------------------------------
@@ -347,17 +542,51 @@ cudaError_t launch_publish(const StoreView& s, const uint32_t* wctr_dev, int bit
   const dim3 grid_e(ctas_for(warps));
   switch (bits) {
     case 2:
-      publish_range_kernel<2><<<grid_r, block, 0, st>>>(s);
+      publish_range_kernel<2><<<grid_r, block, 0, st>>>(s, s.exps);
       publish_encode_kernel<2><<<grid_e, block, 0, st>>>(s, wctr_dev, warps);
       break;
     case 4:
-      publish_range_kernel<4><<<grid_r, block, 0, st>>>(s);
+      publish_range_kernel<4><<<grid_r, block, 0, st>>>(s, s.exps);
       publish_encode_kernel<4><<<grid_e, block, 0, st>>>(s, wctr_dev, warps);
       break;
     case 8:
-      publish_range_kernel<8><<<grid_r, block, 0, st>>>(s);
+      publish_range_kernel<8><<<grid_r, block, 0, st>>>(s, s.exps);
       publish_encode_kernel<8><<<grid_e, block, 0, st>>>(s, wctr_dev, warps);
       break;
+    default: return cudaErrorInvalidValue;
+  }
+  *launches += 2;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_interact_registers(const StoreView& s, const PairList& pairs, int npairs, int bits,
+                                      cudaStream_t st, int* launches) {
+  if (npairs == 0) return cudaSuccess;
+  const int64_t warps = (int64_t)npairs * s.nblk;
+  const dim3 grid(ctas_for(warps)), block(kWarpsPerCta * 32);
+  cudaError_t e = cudaSuccess;
+  switch (bits) {
+    case 2: e = launch_dependent(interact_registers_kernel<2>, grid, block, st, s, pairs, warps); break;
+    case 4: e = launch_dependent(interact_registers_kernel<4>, grid, block, st, s, pairs, warps); break;
+    case 8: e = launch_dependent(interact_registers_kernel<8>, grid, block, st, s, pairs, warps); break;
+    default: return cudaErrorInvalidValue;
+  }
+  ++*launches;
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+cudaError_t launch_register_publish(const StoreView& s, const uint32_t* wctr_dev, int bits, cudaStream_t st,
+                                    int* launches) {
+  const dim3 block(kWarpsPerCta * 32);
+  const dim3 grid_r(ctas_for(s.nblk));
+  const int64_t warps = (int64_t)s.n * s.nblk;
+  const dim3 grid_e(ctas_for(warps));
+  // the own registers of a block share the step of an 8-bit code of the spread of all snapshots
+  publish_range_kernel<kOwnResolutionBits><<<grid_r, block, 0, st>>>(s, s.oexps);
+  switch (bits) {
+    case 2: register_publish_encode_kernel<2><<<grid_e, block, 0, st>>>(s, wctr_dev, warps); break;
+    case 4: register_publish_encode_kernel<4><<<grid_e, block, 0, st>>>(s, wctr_dev, warps); break;
+    case 8: register_publish_encode_kernel<8><<<grid_e, block, 0, st>>>(s, wctr_dev, warps); break;
     default: return cudaErrorInvalidValue;
   }
   *launches += 2;

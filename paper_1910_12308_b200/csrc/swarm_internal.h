@@ -11,6 +11,8 @@ namespace swarm {
 struct PairDesc {
   int32_t a, b;        // initiator, responder
   uint32_t wa, wb;     // write counters of the two buffers before this interaction
+  uint32_t woa;        // write counter of the initiator's own register (two-register protocol)
+  uint32_t pad;
 };
 
 // One node of a local-step launch.
@@ -55,6 +57,8 @@ struct StoreView {
   float* B;            // [n][pitch] or nullptr
   uint8_t* codes;      // [n][nblk * 1024]
   int8_t* exps;        // [n][nblk]
+  uint16_t* own;       // [n][pitch] own registers (two-register protocol) or nullptr
+  int8_t* oexps;       // [n][nblk] exponents of the own registers
   int64_t pitch;       // elements per row, multiple of 1024
   int64_t d;
   int64_t nblk;
@@ -75,6 +79,11 @@ cudaError_t launch_interact_nonblocking(const StoreView& s, const PairList& pair
                                         cudaStream_t st, int* launches);
 // wctr_dev: n write counters (uint32) used for the rounding uniforms of each node's buffer.
 cudaError_t launch_publish(const StoreView& s, const uint32_t* wctr_dev, int bits, cudaStream_t st, int* launches);
+// Two-register protocol. wctr_dev: n write counters of the current registers followed by n of the own registers.
+cudaError_t launch_interact_registers(const StoreView& s, const PairList& pairs, int npairs, int bits,
+                                      cudaStream_t st, int* launches);
+cudaError_t launch_register_publish(const StoreView& s, const uint32_t* wctr_dev, int bits, cudaStream_t st,
+                                    int* launches);
 
 // --- swarm_local.cu ----------------------------------------------------------------------
 cudaError_t launch_init_models(const StoreView& s, const float* scalars_dev, float init_std, cudaStream_t st,

@@ -33,8 +33,12 @@ def inject(orc, gpu, what=("X", "B", "P", "counters", "data")):
         if "P" in what:
             gpu.set(g.T_CODES, i, orc.codes[i])
             gpu.set(g.T_EXPS, i, orc.exps[i])
+        if "P" in what and orc.own is not None:
+            gpu.set(g.T_OWN, i, orc.own[i])
+            gpu.set(g.T_OEXPS, i, orc.oexps[i])
         if "counters" in what:
             gpu.set(g.T_COUNTERS, i, [orc.w[i], orc.ls[i], orc.pbits[i]])
+            gpu.set(g.T_CLOCKS, i, [orc.wo[i], orc.tau[i]])
         if "data" in what:
             gpu.set(g.T_SCALARS, i, [orc.offset[i], orc.drift[i], orc.shift[i]])
             if orc.groups:
@@ -44,6 +48,7 @@ def inject(orc, gpu, what=("X", "B", "P", "counters", "data")):
             gpu.set(g.T_A, grp, orc.A[grp])
     if "counters" in what:
         gpu.set_state(int(orc.launch[0]), int(orc.b_stale[0]))
+        gpu.set_buffer_mode(int(orc.p_mode[0]))
 
 
 def assert_store_equal(orc, gpu, bits=None, nodes=None, check_B=True):
@@ -56,9 +61,14 @@ def assert_store_equal(orc, gpu, bits=None, nodes=None, check_B=True):
             assert np.array_equal(gpu.get(g.T_B, i).view(np.uint32), orc.B[i].view(np.uint32)), f"B[{i}] differs"
         w, ls, pb = gpu.get(g.T_COUNTERS, i)
         assert (w, ls, pb) == (orc.w[i], orc.ls[i], orc.pbits[i]), f"counters[{i}]"
+        assert tuple(gpu.get(g.T_CLOCKS, i)) == (orc.wo[i], orc.tau[i]), f"clocks[{i}]"
+        if orc.own is not None and int(orc.p_mode[0]) == 2:
+            assert np.array_equal(gpu.get(g.T_OWN, i), orc.own[i]), f"own register[{i}] differs"
+            assert np.array_equal(gpu.get(g.T_OEXPS, i), orc.oexps[i]), f"own exponents[{i}] differ"
         if bits in (2, 4, 8) and orc.pbits[i] == bits:
             nbytes = orc.nblk * 128 * bits
             assert np.array_equal(gpu.get(g.T_CODES, i)[:nbytes], orc.codes[i, :nbytes]), f"codes[{i}] differ"
             assert np.array_equal(gpu.get(g.T_EXPS, i), orc.exps[i]), f"exps[{i}] differ"
     launch, stale = gpu.get_state()
     assert (launch, stale) == (int(orc.launch[0]), int(orc.b_stale[0]))
+    assert gpu.get_buffer_mode() == int(orc.p_mode[0])

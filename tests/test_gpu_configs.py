@@ -59,6 +59,7 @@ def test_large_model_sampled_pair_bit_exact(d, bits, mode):
             orc.codes[i] = gpu.get(g.T_CODES, i)
             orc.exps[i] = gpu.get(g.T_EXPS, i)
             orc.pbits[i] = bits
+            orc.p_mode[0] = 1                 # buffers were published in the single-buffer convention
         orc.w[i] = gpu.get(g.T_COUNTERS, i)[0]
     assert gpu.interact([[2, 0], [1, 3]], bits, mode) == 0
     assert orc.interact([[1, 3]], bits, mode) == 0            # one of the launch's pairs

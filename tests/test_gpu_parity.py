@@ -186,6 +186,54 @@ def test_nonblocking_far_key_alias_matches():
         assert_store_equal(orc, gpu, bits)
 
 
+# ---- two-register protocol -----------------------------------------------------------------------
+
+@pytest.mark.parametrize("bits", [2, 4, 8])
+@pytest.mark.parametrize("d", [5, 1024, 3001])
+def test_register_protocol_bit_exact(bits, d):
+    n = 6
+    cfg = dict(objective=1, nonblocking=2, grad_std=0.03, drift_std=0.1, offset_std=0.2)
+    orc, gpu = make_pair(n, d, "regular", 4, seed=70 + d, **cfg)
+    inject(orc, gpu)
+    assert orc.register_publish(bits) == 0 and gpu.register_publish(bits) == 0
+    assert_store_equal(orc, gpu, bits)
+    rng = np.random.default_rng(bits * 100 + d)
+    for rnd in range(6):
+        nodes = rng.permutation(n)[: int(rng.integers(1, n + 1))]
+        assert orc.local_steps(nodes, 2, 0.05) == 0 and gpu.local_steps(nodes, 2, 0.05) == 0
+        for i in nodes:
+            assert rel_err(gpu.get(g.T_X, i), orc.X[i]) < TOL
+        inject(orc, gpu, what=("X",))
+        pairs = disjoint_pairs(orc, rng, int(rng.integers(1, 4)))
+        assert orc.interact(pairs, bits, o.REGISTERS) == 0
+        assert gpu.interact(pairs, bits, g.REGISTERS) == 0
+        assert_store_equal(orc, gpu, bits)
+
+
+def test_register_protocol_mode_switches_and_far_snapshots():
+    n, d = 4, 2100
+    cfg = dict(objective=1, nonblocking=2, grad_std=0.0, drift_std=0.0, offset_std=0.05)
+    orc, gpu = make_pair(n, d, "complete", seed=17, **cfg)
+    inject(orc, gpu)
+    seq = [([[0, 1]], 8, 2), ([[2, 3], [1, 0]], 8, 2), ([[0, 2]], 8, 1), ([[3, 1]], 8, 2), ([[1, 2]], 4, 2),
+           ([[0, 3]], 4, 0), ([[2, 0]], 4, 2), ([[1, 3]], 32, 0), ([[3, 2]], 4, 2)]
+    for pairs, bits, mode in seq:
+        assert orc.interact(pairs, bits, mode) == 0 and gpu.interact(pairs, bits, mode) == 0
+        assert_store_equal(orc, gpu, bits)
+    # a snapshot moved outside the 16-bit window of its partner's own register: both sides alias alike
+    orc.B[0] += np.float32(1000.0)
+    orc.X[0] = orc.B[0]
+    orc.B[1, :500] = np.float32(1e30)
+    orc.X[1] = orc.B[1]
+    inject(orc, gpu)
+    for pairs in ([[0, 2]], [[1, 3]], [[2, 0], [3, 1]]):
+        assert orc.interact(pairs, 4, o.REGISTERS) == 0 and gpu.interact(pairs, 4, g.REGISTERS) == 0
+        assert_store_equal(orc, gpu, 4)
+    plain = g.Swarm(4, 64)
+    plain.configure(objective=1, nonblocking=1)
+    assert plain.interact([[0, 1]], 8, g.REGISTERS) == -4 and plain.register_publish(8) == -4
+
+
 # ---- local steps ---------------------------------------------------------------------------------
 
 @pytest.mark.parametrize("d,H", [(3, 1), (4099, 3)])
@@ -303,7 +351,8 @@ def test_rejected_calls_change_nothing():
     assert gpu.interact([[0, 3]], 8) == -3
     assert gpu.interact([[0, 6]], 8) == -2
     assert gpu.interact([[0, 1]], 3) == -1
-    assert gpu.interact([[0, 1]], 8, 2) == -1
+    assert gpu.interact([[0, 1]], 8, 3) == -1
+    assert gpu.interact([[0, 1]], 8, g.REGISTERS) == -4
     assert gpu.interact([[0, 1]], 32, g.NONBLOCKING) == -1
     assert gpu.interact([[0, 1]], 8, g.NONBLOCKING) == -4
     assert gpu.publish(8) == -4
