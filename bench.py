@@ -44,6 +44,10 @@ WORKLOADS = {
     "regular32_resnet18_b8_nb": dict(n=32, d=11_689_512, topology="regular", degree=4, pairs=16, bits=8, mode=1, H=3,
                                      lr=0.05, seed=3, cfg=dict(objective=1, nonblocking=1,
                                                                grad_std=float(np.sqrt(1e-3)))),
+    # the same workload through the two-register protocol (Algorithm 1's chain of three decodes)
+    "regular32_resnet18_b8_reg": dict(n=32, d=11_689_512, topology="regular", degree=4, pairs=16, bits=8, mode=2, H=3,
+                                      lr=0.05, seed=3, cfg=dict(objective=1, nonblocking=2,
+                                                                grad_std=float(np.sqrt(1e-3)))),
     # reduced copy (8 nodes, 4 pairs) for profiler captures that must stay small
     "regular8_resnet18_b8_nb": dict(n=8, d=11_689_512, topology="regular", degree=4, pairs=4, bits=8, mode=1, H=3,
                                     lr=0.05, seed=3, cfg=dict(objective=1, nonblocking=1,
@@ -82,7 +86,11 @@ def interaction_bytes(d, bits, mode):
     nblk = (d + 1023) // 1024
     if mode == 0:
         return d * 16 + 2 * d * bits // 8 + 2 * nblk
-    return d * 16 + 4 * d * bits // 8 + 4 * nblk
+    if mode == 1:
+        return d * 16 + 4 * d * bits // 8 + 4 * nblk
+    # two registers: model + snapshot read and written, two own registers read and one written (16 bits),
+    # two current registers read and written
+    return d * 16 + d * 6 + 4 * d * bits // 8 + 7 * nblk
 
 
 class PairSchedule:
@@ -390,7 +398,7 @@ def run_ours(args, wl, name):
                    "l2": "inputs larger than L2: every launch streams all models it touches from HBM",
                    "replicas": world},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(gpu_launches),
-        "roofline": {"bound": "hbm", "kernel": "interact_blocking_kernel" if wl["mode"] == 0 else "interact_nonblocking_kernel",
+        "roofline": {"bound": "hbm", "kernel": ["interact_blocking_kernel", "interact_nonblocking_kernel", "interact_registers_kernel"][wl["mode"]],
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": peak_kind, "frac_of_8000": achieved / 8000.0, "traffic": TRAFFIC.get(name),
                      "algorithmic_bytes_per_launch": per_launch_bytes, "kernel_ms": kern_ms},
