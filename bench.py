@@ -48,6 +48,9 @@ WORKLOADS = {
     "regular32_resnet18_b8_reg": dict(n=32, d=11_689_512, topology="regular", degree=4, pairs=16, bits=8, mode=2, H=3,
                                       lr=0.05, seed=3, cfg=dict(objective=1, nonblocking=2,
                                                                 grad_std=float(np.sqrt(1e-3)))),
+    "regular8_resnet18_b8_reg": dict(n=8, d=11_689_512, topology="regular", degree=4, pairs=4, bits=8, mode=2, H=3,
+                                     lr=0.05, seed=3, cfg=dict(objective=1, nonblocking=2,
+                                                               grad_std=float(np.sqrt(1e-3)))),
     # reduced copy (8 nodes, 4 pairs) for profiler captures that must stay small
     "regular8_resnet18_b8_nb": dict(n=8, d=11_689_512, topology="regular", degree=4, pairs=4, bits=8, mode=1, H=3,
                                     lr=0.05, seed=3, cfg=dict(objective=1, nonblocking=1,
@@ -420,7 +423,7 @@ def run_ours(args, wl, name):
 
 # ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel (see profiles/);
 # None until a capture of the current kernel exists.
-TRAFFIC = {"ring64_d1m_b4": 512.1e6}
+TRAFFIC = {"ring64_d1m_b4": 512.4e6}
 
 
 def main():
