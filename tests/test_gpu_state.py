@@ -1,0 +1,74 @@
+"""Checkpoint / resume through swarm_get_tensor / swarm_set_tensor, and work on a non-default stream."""
+import numpy as np
+import pytest
+
+from paper_1910_12308_b200 import binding as g
+
+pytestmark = pytest.mark.gpu
+
+ROWS = (g.T_X, g.T_B, g.T_CODES, g.T_EXPS, g.T_OWN, g.T_OEXPS, g.T_COUNTERS, g.T_CLOCKS)
+
+
+def snapshot(sw):
+    state = {which: sw.get_all(which) for which in ROWS}
+    state["ctx"] = sw.get_state() + (sw.get_buffer_mode(),)
+    return state
+
+
+def restore(sw, state):
+    for which in ROWS:
+        for i in range(sw.n):
+            sw.set(which, i, state[which][i])
+    launch, stale, mode = state["ctx"]
+    sw.set_state(launch, stale)
+    sw.set_buffer_mode(mode)
+
+
+def run(sw, rounds):
+    for _ in range(rounds):
+        pairs = sw.sample_pairs(3)
+        assert sw.local_steps(pairs.reshape(-1), 2, 0.05) == 0
+        assert sw.interact(pairs, 8, g.REGISTERS) == 0
+    pairs = sw.sample_pairs(2)
+    assert sw.interact(pairs, 4, g.NONBLOCKING) == 0
+    assert sw.interact(sw.sample_pairs(2), 8, g.BLOCKING) == 0
+
+
+def test_checkpoint_and_resume_reproduce_the_run_bit_for_bit():
+    cfg = dict(objective=1, nonblocking=2, grad_std=0.03, drift_std=0.1, offset_std=0.05)
+    a = g.Swarm(8, 3000, "regular", 4, seed=5)
+    a.configure(**cfg)
+    run(a, 3)
+    saved = snapshot(a)
+    run(a, 4)
+    want = snapshot(a)
+    b = g.Swarm(8, 3000, "regular", 4, seed=5)     # same seed and workload, fresh context
+    b.configure(**cfg)
+    restore(b, saved)
+    run(b, 4)
+    got = snapshot(b)
+    for which in ROWS:
+        assert np.array_equal(got[which].view(np.uint8), want[which].view(np.uint8)), which
+    assert got["ctx"] == want["ctx"]
+    assert abs(a.potential() - b.potential()) == 0.0
+
+
+def test_non_default_stream():
+    import torch
+    stream = torch.cuda.Stream()
+    ref = g.Swarm(6, 5000, "ring", seed=9)
+    sw = g.Swarm(6, 5000, "ring", seed=9, stream=stream)
+    for s in (ref, sw):
+        s.configure(objective=1, grad_std=0.02, offset_std=0.1)
+    with torch.cuda.stream(stream):
+        out = torch.empty(5000, device="cuda")
+        for s in (ref, sw):
+            for r in range(5):
+                pairs = [[0, 1], [2, 3]] if r % 2 == 0 else [[1, 2], [4, 5]]
+                assert s.local_steps([0, 1, 2, 3, 4, 5], 1, 0.05) == 0
+                assert s.interact(pairs, 4) == 0
+        mu = sw.mean_model(out)
+        sw.sync()
+    assert np.array_equal(sw.get_all(g.T_X), ref.get_all(g.T_X))
+    assert np.array_equal(mu.cpu().numpy(), ref.mean_model().cpu().numpy())
+    assert sw.potential() == ref.potential()
