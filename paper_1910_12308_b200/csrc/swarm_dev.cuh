@@ -39,6 +39,31 @@ __host__ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1
   return make_uint4(c0, c1, c2, c3);
 }
 
+// The ten round keys of a generator key, for kernels that call the generator inside a run-time loop
+// (computed once per thread instead of once per call).
+struct PhiloxRoundKeys { uint32_t k0[10], k1[10]; };
+__host__ __device__ __forceinline__ PhiloxRoundKeys philox_round_keys(uint32_t k0, uint32_t k1) {
+  PhiloxRoundKeys rk;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) { rk.k0[r] = k0 + (uint32_t)r * 0x9E3779B9u; rk.k1[r] = k1 + (uint32_t)r * 0xBB67AE85u; }
+  return rk;
+}
+__host__ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                        const PhiloxRoundKeys& rk) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+    const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ rk.k0[r];
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ rk.k1[r];
+    c1 = (uint32_t)p1;
+    c3 = (uint32_t)p0;
+    c0 = n0;
+    c2 = n2;
+  }
+  return make_uint4(c0, c1, c2, c3);
+}
+
 __host__ __device__ __forceinline__ uint32_t uniform_int(uint32_t word, uint32_t m) {
   return (uint32_t)(((uint64_t)word * m) >> 32);
 }
@@ -73,15 +98,15 @@ __device__ __forceinline__ void normal_pair_fast(uint32_t w0, uint32_t w1, float
   const float series = v * fmaf(v, fmaf(v, fmaf(v, 0.25f, 0.33333334f), 0.5f), 1.0f);
   const float viaLg2 = -0.69314718f * mufu_lg2(u1);                 // u1 >= 2^-24 is a normal float
   const float nl = v < 0x1p-6f ? series : viaLg2;
-  const float r = mufu_sqrt(2.0f * nl);                             // 0 or >= 3.4e-4: no subnormals
+  const float r = mufu_sqrt(nl + nl);                               // 0 or >= 3.4e-4: no subnormals
   const float ang = (float)(int32_t)(w1 & 0xFFFFFF00u) * (6.2831853071795865f * 0x1p-32f);
   z0 = r * mufu_cos(ang);
   z1 = r * mufu_sin(ang);
 }
 
 __device__ __forceinline__ void normal4_fast(uint32_t group, uint32_t row, uint32_t event, uint32_t stream,
-                                             uint32_t k0, uint32_t k1, float z[4]) {
-  const uint4 w = philox4x32_10(group, row, event, stream, k0, k1);
+                                             const PhiloxRoundKeys& rk, float z[4]) {
+  const uint4 w = philox4x32_10(group, row, event, stream, rk);
   normal_pair_fast(w.x, w.y, z[0], z[1]);
   normal_pair_fast(w.z, w.w, z[2], z[3]);
 }

@@ -110,9 +110,10 @@ local_synth_kernel(StoreView s, const NodeList nodes, int H, float lr, float gra
   float* p = s.X + (int64_t)nd.node * s.pitch + g4 * 4;
   float4 v = *reinterpret_cast<const float4*>(p);
   float* x = &v.x;
+  const PhiloxRoundKeys rk = philox_round_keys(s.key0, s.key1);
   for (int q = 0; q < H; ++q) {
     float z[4];
-    normal4_fast((uint32_t)g4, (uint32_t)nd.node, nd.event + (uint32_t)q, kStreamSynthGrad, s.key0, s.key1, z);
+    normal4_fast((uint32_t)g4, (uint32_t)nd.node, nd.event + (uint32_t)q, kStreamSynthGrad, rk, z);
 #pragma unroll
     for (int t = 0; t < 4; ++t) {
       const float grad = __fadd_rn(c, __fmul_rn(grad_std, z[t]));

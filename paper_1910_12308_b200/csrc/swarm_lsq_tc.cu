@@ -122,17 +122,17 @@ __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bflo
 // =================================================================================================
 // Residual partials. Tile = 128 coordinates (2 swizzle atoms of 64). Shared memory per stage:
 //   A    : 2 atoms x [64 rows x 128 B]   (K-major, 128B swizzle, 8-row groups 1024 B apart)  16 KiB
-//   Xraw : 16 rows x 128 fp32                                                                8 KiB
-// plus two operand buffers Xhi/Xlo: 2 atoms x [16 rows x 128 B] each. Three stages: 89 KiB per CTA,
-// two CTAs per SM so that one CTA's barriers and operand conversion hide behind the other's copies.
+// plus two operand buffers Xhi/Xlo: 2 atoms x [16 rows x 128 B] each. The fp32 models are loaded one
+// tile ahead into registers (8 coordinates per thread) and converted to bf16 hi/lo straight into the
+// operand buffers. Five stages of A: 97 KiB per CTA, two CTAs per SM so that one CTA's barrier and
+// operand conversion hide behind the other's copies.
 // =================================================================================================
 constexpr int kResTile = 128;
 constexpr int kResAtoms = kResTile / 64;
-constexpr int kResStages = 3;
+constexpr int kResStages = 5;
 constexpr int kResABytes = kResAtoms * kTcBatch * 128;         // 16384
-constexpr int kResXrawBytes = kUnitNodes * kResTile * 4;       // 8192
 constexpr int kResXopBytes = kResAtoms * kUnitNodes * 128;     // 4096 (one of hi / lo)
-constexpr int kResSmem = kResStages * (kResABytes + kResXrawBytes) + 2 * 2 * kResXopBytes + 1024 /*align*/ + 64;
+constexpr int kResSmem = kResStages * kResABytes + 2 * 2 * kResXopBytes + 1024 /*align*/ + 64;
 
 __global__ void __launch_bounds__(kTcThreads, 2)
 lsq_tc_residual_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, int step, float* __restrict__ partial,
@@ -140,8 +140,7 @@ lsq_tc_residual_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* sA = smem;                                           // stages of A
-  uint8_t* sXraw = sA + kResStages * kResABytes;
-  uint8_t* sXop = sXraw + kResStages * kResXrawBytes;           // [buf][hi|lo]
+  uint8_t* sXop = sA + kResStages * kResABytes;                 // [buf][hi|lo]
   uint64_t* bars = (uint64_t*)(sXop + 4 * kResXopBytes);        // mma_done[2]
   uint32_t* tmem_slot = (uint32_t*)(bars + 2);
   __shared__ int rows[kTcBatch];
@@ -164,9 +163,9 @@ lsq_tc_residual_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units
     fence_mbar_init();
   }
   if (warp == 0) { tmem_alloc(smem_u32(tmem_slot), 32); tmem_relinquish(); }
-  // rows of the minibatch tile beyond the batch size and node rows beyond the unit stay zero
-  for (int i = tid; i < kResStages * kResABytes / 16; i += kTcThreads) reinterpret_cast<uint4*>(sA)[i] = make_uint4(0, 0, 0, 0);
-  for (int i = tid; i < kResStages * kResXrawBytes / 16; i += kTcThreads) reinterpret_cast<uint4*>(sXraw)[i] = make_uint4(0, 0, 0, 0);
+  // rows of the minibatch tile beyond the batch size are never copied: they must read as zero
+  if (l.batch < kTcBatch)
+    for (int i = tid; i < kResStages * kResABytes / 16; i += kTcThreads) reinterpret_cast<uint4*>(sA)[i] = make_uint4(0, 0, 0, 0);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -188,34 +187,39 @@ lsq_tc_residual_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units
           cp_async16(dst, A + (int64_t)rows[r] * s.pitch + k0 + c * 8);
         }
       }
-      // X: 16 rows x 32 chunks of 16 B (fp32), plain row-major staging
-      const uint32_t x_base = smem_u32(sXraw + st * kResXrawBytes);
-#pragma unroll
-      for (int it = 0; it < kUnitNodes * 32 / kTcThreads; ++it) {
-        const int idx = it * kTcThreads + tid;
-        const int r = idx >> 5, c = idx & 31;
-        if (r < u.count) cp_async16(x_base + r * (kResTile * 4) + c * 16, s.X + (int64_t)unodes[r] * s.pitch + k0 + c * 4);
-      }
     }
     cp_async_commit();
+  };
+
+  // this thread's slice of the model tile: node row tid / 16, coordinates 8 * (tid % 16) .. +7
+  const int xr = tid >> 4, xc8 = tid & 15;
+  const float* xsrc = s.X + (int64_t)unodes[xr < u.count ? xr : 0] * s.pitch + kbase + xc8 * 8;
+  auto load_x = [&](int tile, float4 v[2]) {
+    if (tile < ntiles && xr < u.count) {
+      v[0] = *reinterpret_cast<const float4*>(xsrc + (int64_t)tile * kResTile);
+      v[1] = *reinterpret_cast<const float4*>(xsrc + (int64_t)tile * kResTile + 4);
+    } else {
+      v[0] = v[1] = make_float4(0.f, 0.f, 0.f, 0.f);          // node rows beyond the unit stay zero
+    }
   };
 
   bool ok = true;
   for (int t = 0; t < kResStages - 1; ++t) issue_loads(t);
   constexpr uint32_t idesc = instr_desc_bf16(kTcBatch, kUnitNodes, 0, 0);
+  float4 xcur[2], xnext[2];
+  load_x(0, xcur);
   for (int t = 0; t < ntiles && ok; ++t) {
     const int st = t % kResStages, buf = t & 1;
-    cp_async_wait<kResStages - 2>();
-    __syncthreads();                                        // tile t has landed for every thread
+    load_x(t + 1, xnext);                                   // consumed one iteration later
+    cp_async_wait<kResStages - 2>();                        // this thread's copies of tile t have landed
     if (t >= 2) ok = mbar_wait(smem_u32(&bars[buf]), ((t >> 1) - 1) & 1);   // operand buffer free again
-    // fp32 -> bf16 hi/lo into the swizzled operand layout: thread -> (row = tid / 16, 8 coordinates)
+    // fp32 -> bf16 hi/lo into the swizzled operand layout
     {
-      const int r = tid >> 4, c8 = tid & 15;                // c8: group of 8 coordinates = one 16-byte bf16 chunk
-      const float4* src = reinterpret_cast<const float4*>(sXraw + st * kResXrawBytes + r * (kResTile * 4) + c8 * 32);
+      const int r = xr, c8 = xc8;                           // c8: group of 8 coordinates = one 16-byte bf16 chunk
       __align__(16) __nv_bfloat16 hi[8], lo[8];
 #pragma unroll
       for (int q = 0; q < 2; ++q) {
-        const float4 v = src[q];
+        const float4 v = xcur[q];
         split_bf16(v.x, hi[q * 4 + 0], lo[q * 4 + 0]);
         split_bf16(v.y, hi[q * 4 + 1], lo[q * 4 + 1]);
         split_bf16(v.z, hi[q * 4 + 2], lo[q * 4 + 2]);
@@ -249,6 +253,7 @@ lsq_tc_residual_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units
     // refill the stage that tile t-1 used (its MMAs were committed one iteration ago)
     if (t >= 1 && ok) ok = mbar_wait(smem_u32(&bars[(t - 1) & 1]), ((t - 1) >> 1) & 1);
     issue_loads(t + kResStages - 1);
+    xcur[0] = xnext[0]; xcur[1] = xnext[1];
   }
   cp_async_wait<0>();
   if (ok && ntiles > 0) ok = mbar_wait(smem_u32(&bars[(ntiles - 1) & 1]), ((ntiles - 1) >> 1) & 1);
@@ -341,7 +346,8 @@ lsq_tc_update_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
     fence_mbar_init();
   }
   if (warp == 0) { tmem_alloc(smem_u32(tmem_slot), 32); tmem_relinquish(); }
-  for (int i = tid; i < kUpdStages * kUpdABytes / 16; i += kTcThreads) reinterpret_cast<uint4*>(sA)[i] = make_uint4(0, 0, 0, 0);
+  if (l.batch < kTcBatch)     // sampled-row slots beyond the batch are never copied: they must read as zero
+    for (int i = tid; i < kUpdStages * kUpdABytes / 16; i += kTcThreads) reinterpret_cast<uint4*>(sA)[i] = make_uint4(0, 0, 0, 0);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
