@@ -850,7 +850,7 @@ static int tensor_access(swarm_ctx* c, int32_t which, int32_t node, void* host, 
     default: return SWARM_EINVAL;
   }
   if (bytes != want) return SWARM_EINVAL;
-  SW_CUDA(c, cudaStreamSynchronize(c->stream));
+  // the copy is ordered after earlier work by the stream; one synchronisation at the end is enough
   if (write) SW_CUDA(c, cudaMemcpyAsync(dev, host, bytes, cudaMemcpyHostToDevice, c->stream));
   else SW_CUDA(c, cudaMemcpyAsync(host, dev, bytes, cudaMemcpyDeviceToHost, c->stream));
   SW_CUDA(c, cudaStreamSynchronize(c->stream));
