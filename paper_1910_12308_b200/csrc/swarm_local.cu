@@ -98,31 +98,33 @@ lsq_labels_kernel(const T* __restrict__ A, const float* __restrict__ xstar, floa
 // -----------------------------------------------------------------------------------------
 // Synthetic-gradient local steps: x <- x - lr * (c_i + grad_std * z), H times in one memory
 // pass; each step is its own sequence of rounded fp32 operations (no fusion across steps).
-// One thread per 4 coordinates (one generator call per step).
 // -----------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 local_synth_kernel(StoreView s, const NodeList nodes, int H, float lr, float grad_std,
                    const float* __restrict__ scalars) {
-  const int64_t g4 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (g4 * 4 >= s.d) return;
+  // one thread per 8 coordinates: one 256-bit load and store, two generator calls per step
+  const int64_t g8 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (g8 * 8 >= s.d) return;
   const NodeDesc nd = nodes.get(blockIdx.y);
   const float c = scalars[nd.node * 3 + 1];
-  float* p = s.X + (int64_t)nd.node * s.pitch + g4 * 4;
-  float4 v = *reinterpret_cast<const float4*>(p);
-  float* x = &v.x;
+  float* p = s.X + (int64_t)nd.node * s.pitch + g8 * 8;
+  f8 v = ld256(p);
   const PhiloxRoundKeys rk = philox_round_keys(s.key0, s.key1);
   for (int q = 0; q < H; ++q) {
-    float z[4];
-    normal4_fast((uint32_t)g4, (uint32_t)nd.node, nd.event + (uint32_t)q, kStreamSynthGrad, rk, z);
+    float z[8];
+    normal4_fast((uint32_t)(2 * g8), (uint32_t)nd.node, nd.event + (uint32_t)q, kStreamSynthGrad, rk, z);
+    normal4_fast((uint32_t)(2 * g8 + 1), (uint32_t)nd.node, nd.event + (uint32_t)q, kStreamSynthGrad, rk, z + 4);
 #pragma unroll
-    for (int t = 0; t < 4; ++t) {
+    for (int t = 0; t < 8; ++t) {
       const float grad = __fadd_rn(c, __fmul_rn(grad_std, z[t]));
-      x[t] = __fsub_rn(x[t], __fmul_rn(lr, grad));
+      v.v[t] = __fsub_rn(v.v[t], __fmul_rn(lr, grad));
     }
   }
+  if (g8 * 8 + 8 > s.d) {                                    // keep the row padding zero
 #pragma unroll
-  for (int t = 0; t < 4; ++t) if (g4 * 4 + t >= s.d) x[t] = 0.0f;    // keep the row padding zero
-  *reinterpret_cast<float4*>(p) = v;
+    for (int t = 0; t < 8; ++t) if (g8 * 8 + t >= s.d) v.v[t] = 0.0f;
+  }
+  st256(p, v);
 }
 
 // -----------------------------------------------------------------------------------------
@@ -422,7 +424,7 @@ cudaError_t launch_lsq_data(const StoreView& s, const LsqView& l, void* A, float
 cudaError_t launch_local_synth(const StoreView& s, const NodeList& nodes, int count, int H, float lr,
                                float grad_std, const float* scalars_dev, cudaStream_t st, int* launches) {
   if (count == 0 || H == 0) return cudaSuccess;
-  const dim3 grid(cdiv((s.d + 3) / 4, 256), count);
+  const dim3 grid(cdiv(s.pitch / 8, 256), count);
   local_synth_kernel<<<grid, 256, 0, st>>>(s, nodes, H, lr, grad_std, scalars_dev);
   ++*launches;
   return cudaGetLastError();
