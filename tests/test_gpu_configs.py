@@ -91,3 +91,26 @@ def test_config1_trajectory_teacher_forced():
         assert orc.interact(pairs, 8) == 0 and gpu.interact(pairs, 8) == 0
     assert_store_equal(orc, gpu, 8)
     assert abs(gpu.potential() - orc.potential()) <= 1e-9 * orc.potential()
+
+
+def test_config5_shape_tensor_core_steps_and_two_bit_interaction():
+    """d = 2^20, bf16 least-squares data shared by groups of 16 nodes, batch 64 (the tensor-core path with
+    128 k-chunks per unit), then a 2-bit non-blocking launch of 16 pairs: reduced in n and in the rows per
+    data matrix (32 nodes, 2 matrices of 64 rows) so that the oracle finishes in under a minute."""
+    from tests.parity import assert_store_equal, inject, make_pair
+    n, d = 32, 1 << 20
+    cfg = dict(objective=2, nonblocking=1, lsq_m=64, lsq_batch=64, lsq_dtype=1, lsq_groups=2,
+               lsq_noise_std=float(np.sqrt(0.1)))
+    orc, gpu = make_pair(n, d, "regular", 8, seed=5, **cfg)
+    inject(orc, gpu)
+    nodes = list(range(n))
+    assert orc.local_steps(nodes, 2, 0.05) == 0 and gpu.local_steps(nodes, 2, 0.05) == 0
+    gpu.sync()
+    for i in range(n):
+        assert rel_err(gpu.get(g.T_X, i), orc.X[i]) < 1e-6, i
+    inject(orc, gpu, what=("X",))
+    pairs = orc.sample_pairs(16)
+    assert np.array_equal(gpu.sample_pairs(16), pairs) and len(pairs) >= 8
+    assert orc.interact(pairs, 2, o.NONBLOCKING, threads=8) == 0 and gpu.interact(pairs, 2, g.NONBLOCKING) == 0
+    assert_store_equal(orc, gpu, 2)
+    assert abs(gpu.potential() - orc.potential()) <= 1e-9 * orc.potential()
