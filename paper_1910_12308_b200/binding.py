@@ -4,8 +4,11 @@ Argument marshalling only: every step of the method runs in the CUDA library. Py
 device memory (through the allocator hook) and the stream. There is no CPU path: the binding
 raises at import if the shared library is missing and cannot be built.
 """
+import atexit
 import ctypes as C
 import os
+import sys
+import weakref
 
 import numpy as np
 
@@ -137,6 +140,20 @@ def use_torch_allocator():
         raise SwarmError(rc, "swarm_set_allocator")
 
 
+# Contexts still alive at interpreter exit are destroyed before the interpreter and the framework that
+# backs the allocator callbacks are torn down (a destroy during finalisation would call back into them).
+_live = weakref.WeakSet()
+
+
+@atexit.register
+def _close_all():
+    for sw in list(_live):
+        try:
+            sw.close()
+        except Exception:
+            pass
+
+
 def _pairs_array(pairs):
     pairs = np.ascontiguousarray(pairs, dtype=np.int32).reshape(-1, 2)
     return pairs, pairs.ctypes.data_as(C.POINTER(SwarmPair))
@@ -159,6 +176,7 @@ class Swarm:
         if rc != 0:
             raise SwarmError(rc, "swarm_init")
         self._h, self._L = h, L
+        _live.add(self)
         self.n, self.d, self.seed = n, d, seed
         self.nblk = (d + 1023) // 1024
         self.cfg = SwarmConfig(OBJ_NONE, 0, 0.1, 0.0, 0.0, 0.0, 0, 0, 0, 0, 0.0)
@@ -174,6 +192,8 @@ class Swarm:
 
     def __del__(self):
         try:
+            if sys is None or sys.is_finalizing():
+                return
             self.close()
         except Exception:
             pass

@@ -1,10 +1,13 @@
 // State generation, local SGD steps (Section 3, "The Communication Procedure": H sequential
 // stochastic gradient steps, each at the running iterate) and the pair sampler (Algorithm 1,
 // sampling lines).
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 
 #include "swarm_dev.cuh"
 #include "swarm_internal.h"
+
+namespace cg = cooperative_groups;
 
 namespace swarm {
 
@@ -231,13 +234,14 @@ lsq_update_kernel(StoreView s, LsqView l, const NodeList nodes, int step, float 
 }
 
 // -----------------------------------------------------------------------------------------
-// Least-squares local steps for short models (row pitch <= 8192, batch <= 32): one CTA per node
-// runs all H steps in one launch with the model in registers. Per step: every thread forms its
-// share of the B dot products, a shuffle + shared-memory reduction in fixed order gives the
-// residuals, then the sampled rows are read again (from L2) for the update.
+// Least-squares local steps for short models (row pitch <= 8192, batch <= 32): all H steps in one
+// launch with the model in registers. A thread-block cluster of up to 8 CTAs owns one node; each CTA
+// holds a 512- or 1024-coordinate slice, forms its share of the B dot products, and the CTAs exchange
+// the partial sums through distributed shared memory (summed in rank order, so results do not depend
+// on scheduling). The cluster barriers are hardware barriers reached by every CTA of the cluster.
 // -----------------------------------------------------------------------------------------
-constexpr int kSmallThreads = 256;
-constexpr int kSmallMaxChunks = 8;        // 8 x 1024 coordinates
+constexpr int kSmallThreads = 128;
+constexpr int kSmallMaxPitch = 8192;
 constexpr int kSmallMaxBatch = 32;
 
 template <typename T>
@@ -253,80 +257,88 @@ __device__ __forceinline__ float4 load4_as_float<__nv_bfloat16>(const __nv_bfloa
 
 template <typename T>
 __global__ void __launch_bounds__(kSmallThreads)
-lsq_small_kernel(StoreView s, LsqView l, const NodeList nodes, int H, float lr) {
-  const NodeDesc nd = nodes.get(blockIdx.x);
+lsq_small_kernel(StoreView s, LsqView l, const NodeList nodes, int H, float lr, int csize, int iters) {
+  cg::cluster_group cluster = cg::this_cluster();
+  const int rank = (int)cluster.block_rank();
+  const NodeDesc nd = nodes.get(blockIdx.x / csize);
   const int group = nd.node / l.nodes_per_group;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int nchunk = (int)(s.pitch / kBlockCoords);
-  float* xrow = s.X + (int64_t)nd.node * s.pitch;
-  const T* A = reinterpret_cast<const T*>(l.A) + (int64_t)group * l.m * s.pitch;
+  const int64_t base = (int64_t)rank * iters * (kSmallThreads * 4) + tid * 4;   // first coordinate of this thread
+  float* xrow = s.X + (int64_t)nd.node * s.pitch + base;
+  const T* A = reinterpret_cast<const T*>(l.A) + (int64_t)group * l.m * s.pitch + base;
   const float* labels = l.bvec + (int64_t)nd.node * l.m;
 
   __shared__ int rows[kSmallMaxBatch];
   __shared__ float red[kSmallThreads / 32][kSmallMaxBatch];
+  __shared__ float part[kSmallMaxBatch];       // this CTA's partial dot products (read by the whole cluster)
   __shared__ float resid[kSmallMaxBatch];
 
-  float4 x[kSmallMaxChunks];
-#pragma unroll
-  for (int c = 0; c < kSmallMaxChunks; ++c)
-    x[c] = c < nchunk ? *reinterpret_cast<const float4*>(xrow + c * kBlockCoords + tid * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+  float4 x[2];
+  x[0] = *reinterpret_cast<const float4*>(xrow);
+  x[1] = iters > 1 ? *reinterpret_cast<const float4*>(xrow + kSmallThreads * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
   const float scale = lr / (float)l.batch;
 
   for (int q = 0; q < H; ++q) {
     if (tid < l.batch) rows[tid] = minibatch_row(tid, group, nd.event + (uint32_t)q, l.m, s.key0, s.key1);
     __syncthreads();
-    for (int si = 0; si < l.batch; ++si) {
-      const T* row = A + (int64_t)rows[si] * s.pitch + tid * 4;
-      float acc = 0.0f;
+    // groups of 8 sampled rows: all loads of a group are issued before the first reduction
+    for (int s0 = 0; s0 < l.batch; s0 += 8) {
+      float4 a0[8], a1[8];
 #pragma unroll
-      for (int c = 0; c < kSmallMaxChunks; ++c)
-        if (c < nchunk) {
-          const float4 a = load4_as_float<T>(row + c * kBlockCoords);
-          acc = fmaf(a.x, x[c].x, acc); acc = fmaf(a.y, x[c].y, acc);
-          acc = fmaf(a.z, x[c].z, acc); acc = fmaf(a.w, x[c].w, acc);
-        }
-      acc = warp_sum(acc);
-      if (lane == 0) red[warp][si] = acc;
+      for (int j = 0; j < 8; ++j) {
+        const bool on = s0 + j < l.batch;
+        const T* row = A + (int64_t)rows[on ? s0 + j : 0] * s.pitch;
+        a0[j] = on ? load4_as_float<T>(row) : make_float4(0.f, 0.f, 0.f, 0.f);
+        a1[j] = (on && iters > 1) ? load4_as_float<T>(row + kSmallThreads * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        float acc = a0[j].x * x[0].x;
+        acc = fmaf(a0[j].y, x[0].y, acc); acc = fmaf(a0[j].z, x[0].z, acc); acc = fmaf(a0[j].w, x[0].w, acc);
+        acc = fmaf(a1[j].x, x[1].x, acc); acc = fmaf(a1[j].y, x[1].y, acc);
+        acc = fmaf(a1[j].z, x[1].z, acc); acc = fmaf(a1[j].w, x[1].w, acc);
+        acc = warp_sum(acc);
+        if (lane == 0 && s0 + j < l.batch) red[warp][s0 + j] = acc;
+      }
     }
     __syncthreads();
     if (tid < l.batch) {
       float tot = 0.0f;
 #pragma unroll
       for (int w = 0; w < kSmallThreads / 32; ++w) tot += red[w][tid];
+      part[tid] = tot;
+    }
+    cluster.sync();                              // every CTA's partial sums are in place
+    if (tid < l.batch) {
+      float tot = 0.0f;
+      for (int r = 0; r < csize; ++r) tot += *cluster.map_shared_rank(&part[tid], r);
       resid[tid] = tot - labels[rows[tid]];
     }
     __syncthreads();
-    float4 g[kSmallMaxChunks];
+    float4 g0 = make_float4(0.f, 0.f, 0.f, 0.f), g1 = g0;
+    for (int s0 = 0; s0 < l.batch; s0 += 8) {
+      float4 a0[8], a1[8];
 #pragma unroll
-    for (int c = 0; c < kSmallMaxChunks; ++c) g[c] = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int si = 0; si < l.batch; ++si) {
-      const T* row = A + (int64_t)rows[si] * s.pitch + tid * 4;
-      const float rs = resid[si];
+      for (int j = 0; j < 8; ++j) {
+        const bool on = s0 + j < l.batch;
+        const T* row = A + (int64_t)rows[on ? s0 + j : 0] * s.pitch;
+        a0[j] = on ? load4_as_float<T>(row) : make_float4(0.f, 0.f, 0.f, 0.f);
+        a1[j] = (on && iters > 1) ? load4_as_float<T>(row + kSmallThreads * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
 #pragma unroll
-      for (int c = 0; c < kSmallMaxChunks; ++c)
-        if (c < nchunk) {
-          const float4 a = load4_as_float<T>(row + c * kBlockCoords);
-          g[c].x = fmaf(rs, a.x, g[c].x); g[c].y = fmaf(rs, a.y, g[c].y);
-          g[c].z = fmaf(rs, a.z, g[c].z); g[c].w = fmaf(rs, a.w, g[c].w);
-        }
+      for (int j = 0; j < 8; ++j) {
+        const float rs = s0 + j < l.batch ? resid[s0 + j] : 0.0f;
+        g0.x = fmaf(rs, a0[j].x, g0.x); g0.y = fmaf(rs, a0[j].y, g0.y); g0.z = fmaf(rs, a0[j].z, g0.z); g0.w = fmaf(rs, a0[j].w, g0.w);
+        g1.x = fmaf(rs, a1[j].x, g1.x); g1.y = fmaf(rs, a1[j].y, g1.y); g1.z = fmaf(rs, a1[j].z, g1.z); g1.w = fmaf(rs, a1[j].w, g1.w);
+      }
     }
-#pragma unroll
-    for (int c = 0; c < kSmallMaxChunks; ++c) {
-      x[c].x -= scale * g[c].x; x[c].y -= scale * g[c].y; x[c].z -= scale * g[c].z; x[c].w -= scale * g[c].w;
-    }
-    __syncthreads();
+    x[0].x -= scale * g0.x; x[0].y -= scale * g0.y; x[0].z -= scale * g0.z; x[0].w -= scale * g0.w;
+    x[1].x -= scale * g1.x; x[1].y -= scale * g1.y; x[1].z -= scale * g1.z; x[1].w -= scale * g1.w;
+    cluster.sync();                              // all remote reads of part[] are done before it is rewritten
   }
-#pragma unroll
-  for (int c = 0; c < kSmallMaxChunks; ++c)
-    if (c < nchunk) {
-      const int64_t k = (int64_t)c * kBlockCoords + tid * 4;
-      float4 v = x[c];
-      if (k + 0 >= s.d) v.x = 0.f;                    // data rows are zero past d, so these are zero already
-      if (k + 1 >= s.d) v.y = 0.f;
-      if (k + 2 >= s.d) v.z = 0.f;
-      if (k + 3 >= s.d) v.w = 0.f;
-      *reinterpret_cast<float4*>(xrow + k) = v;
-    }
+  // data rows are zero past d, so coordinates past d have stayed zero
+  *reinterpret_cast<float4*>(xrow) = x[0];
+  if (iters > 1) *reinterpret_cast<float4*>(xrow + kSmallThreads * 4) = x[1];
 }
 
 // -----------------------------------------------------------------------------------------
@@ -434,11 +446,27 @@ cudaError_t launch_local_lsq(const StoreView& s, const LsqView& l, const NodeLis
                              float lr, float* partial_dev, cudaStream_t st, int* launches) {
   if (count == 0 || H == 0) return cudaSuccess;
   if (l.batch > kLsqMaxBatch) return cudaErrorInvalidValue;
-  if (s.pitch <= (int64_t)kSmallMaxChunks * kBlockCoords && l.batch <= kSmallMaxBatch) {
-    if (l.dtype == 1) lsq_small_kernel<__nv_bfloat16><<<count, kSmallThreads, 0, st>>>(s, l, nodes, H, lr);
-    else lsq_small_kernel<float><<<count, kSmallThreads, 0, st>>>(s, l, nodes, H, lr);
+  if (s.pitch <= kSmallMaxPitch && l.batch <= kSmallMaxBatch) {
+    // cluster of pitch / 512 CTAs (one 512-coordinate slice each) while that is at most 8, else pitch / 1024
+    const int slices512 = (int)(s.pitch / (kSmallThreads * 4));
+    const int csize = slices512 <= 8 ? slices512 : slices512 / 2;
+    const int iters = slices512 <= 8 ? 1 : 2;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(count * csize));
+    cfg.blockDim = dim3(kSmallThreads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)csize;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e;
+    if (l.dtype == 1) e = cudaLaunchKernelEx(&cfg, lsq_small_kernel<__nv_bfloat16>, s, l, nodes, H, lr, csize, iters);
+    else e = cudaLaunchKernelEx(&cfg, lsq_small_kernel<float>, s, l, nodes, H, lr, csize, iters);
     ++*launches;
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
   }
   const int64_t nchunks = lsq_chunks(s.d);
   const dim3 grid((unsigned)nchunks, count);
