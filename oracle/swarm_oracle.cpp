@@ -216,7 +216,7 @@ uint32_t get_code(const uint8_t* block_bytes, int k, int bits) {
 // Swarm state
 // ---------------------------------------------------------------------------
 struct Config {
-  int32_t objective;      // 0 none, 1 synthetic gradient, 2 least squares
+  int32_t objective;      // 0 none, 1 synthetic gradient, 2 least squares, 3 logistic regression (labels in {0, 1})
   int32_t nonblocking;    // 1: base snapshots exist; 2: also the nodes' own registers (two-register protocol)
   float init_std, offset_std;
   float grad_std, drift_std;
@@ -364,7 +364,7 @@ void init_state(Swarm& s) {
   else { s.own.clear(); s.oexps.clear(); }
 
   s.A.clear(); s.bvec.clear(); s.xstar.clear(); s.groups = 0;
-  if (c.objective == 2) {
+  if (c.objective == 2 || c.objective == 3) {
     const int m = c.lsq_m;
     s.groups = c.lsq_groups > 0 ? c.lsq_groups : n;
     const float inv_sqrt_d = (float)(1.0 / std::sqrt((double)d));
@@ -388,7 +388,9 @@ void init_state(Swarm& s) {
         double acc = 0.0;
         for (int64_t k = 0; k < d; ++k) acc += (double)row[k] * (double)s.xstar[k];
         const float noise = c.lsq_noise_std * normal_at(s.rng, kStreamDataNoise, (uint32_t)i, 0, r);
-        s.bvec[(size_t)i * m + r] = (float)(acc + (double)s.shift[i] + (double)noise);
+        const float score = (float)(acc + (double)s.shift[i] + (double)noise);
+        // least squares: real-valued label; logistic regression: its sign as a {0, 1} class
+        s.bvec[(size_t)i * m + r] = c.objective == 3 ? (score > 0.0f ? 1.0f : 0.0f) : score;
       }
     }
   }
@@ -430,7 +432,10 @@ void local_step_lsq(Swarm& s, int i, float lr) {
     const float* row = Ag + (size_t)rows[t] * d;
     double acc = 0.0;
     for (int64_t k = 0; k < d; ++k) acc += (double)row[k] * (double)xi[k];
-    resid[t] = acc - (double)s.bvec[(size_t)i * m + rows[t]];
+    // least squares: f = (1/2m) sum (a.x - b)^2; logistic: f = (1/m) sum log(1 + e^{a.x}) - y a.x.
+    // Either way the stochastic gradient is (1/B) sum_s resid_s a_s with the residual below.
+    const double pred = s.cfg.objective == 3 ? 1.0 / (1.0 + std::exp(-acc)) : acc;
+    resid[t] = pred - (double)s.bvec[(size_t)i * m + rows[t]];
   }
   for (int64_t k = 0; k < d; ++k) {
     double g = 0.0;
@@ -752,8 +757,8 @@ void orc_destroy(void* h) { delete (Swarm*)h; }
 
 int orc_configure(void* h, const Config* c) {
   Swarm& s = *(Swarm*)h;
-  if (c->objective < 0 || c->objective > 2 || c->nonblocking < 0 || c->nonblocking > 2) return -1;
-  if (c->objective == 2) {
+  if (c->objective < 0 || c->objective > 3 || c->nonblocking < 0 || c->nonblocking > 2) return -1;
+  if (c->objective >= 2) {
     if (c->lsq_m < 1 || c->lsq_batch < 1 || c->lsq_dtype < 0 || c->lsq_dtype > 1) return -1;
     if (c->lsq_groups < 0 || (c->lsq_groups > 0 && s.n % c->lsq_groups != 0)) return -1;
   }
@@ -784,7 +789,7 @@ int32_t orc_groups(void* h) { return ((Swarm*)h)->groups; }
 
 int orc_minibatch_rows(void* h, int32_t node, uint32_t event, int32_t* rows) {
   Swarm& s = *(Swarm*)h;
-  if (s.cfg.objective != 2 || node < 0 || node >= s.n) return -1;
+  if (s.cfg.objective < 2 || node < 0 || node >= s.n) return -1;
   minibatch_rows(s, node, event, rows);
   return 0;
 }

@@ -171,3 +171,47 @@ def test_geometric_steps_equal_that_many_plain_steps():
         t += 1
     assert steps[1] == t + 1
     assert s1.local_steps_geometric([0], 0, 0.1)[0] == -1
+
+
+def logistic(n=3, d=24, m=10, batch=4, seed=1, noise=0.2):
+    s = o.OracleSwarm(n, d, "complete", seed=seed)
+    s.configure(objective=3, lsq_m=m, lsq_batch=batch, lsq_dtype=0, lsq_groups=0, lsq_noise_std=noise)
+    return s
+
+
+def test_logistic_labels_and_gradient_by_finite_differences():
+    """Logistic regression as second workload: labels are the sign of the noisy linear score, the step is
+    minus lr times the minibatch gradient of (1/B) sum log(1 + e^{a.x}) - y a.x."""
+    s = logistic(n=2, d=8, m=40, batch=6, seed=3)
+    assert set(np.unique(s.bvec).tolist()) <= {0.0, 1.0} and 0 < s.bvec.mean() < 1
+    score = s.A[0].astype(np.float64) @ s.xstar.astype(np.float64) + float(s.shift[0])
+    sure = np.abs(score) > 0.9                               # label noise (std 0.2) cannot flip these
+    assert sure.sum() >= 3 and np.array_equal(s.bvec[0][sure], (score[sure] > 0).astype(np.float32))
+    rows = s.minibatch_rows(0, 0)
+    x0 = s.X[0].astype(np.float64).copy()
+    A, y = s.A[0].astype(np.float64)[rows], s.bvec[0].astype(np.float64)[rows]
+
+    def f(x):
+        z = A @ x
+        return (np.log1p(np.exp(z)) - y * z).mean()
+    g = np.zeros(8)
+    for k in range(8):
+        h = np.zeros(8)
+        h[k] = 1e-6
+        g[k] = (f(x0 + h) - f(x0 - h)) / 2e-6
+    s.local_steps([0], 1, 0.1)
+    assert np.abs((s.X[0] - x0) / -0.1 - g).max() < 1e-5 * max(1.0, np.abs(g).max())
+
+
+def test_logistic_sgd_reduces_the_loss():
+    s = logistic(n=2, d=30, m=64, batch=16, seed=5, noise=0.0)
+    A, y = s.A[1].astype(np.float64), s.bvec[1].astype(np.float64)
+
+    def loss(x):
+        z = A @ x
+        return (np.log1p(np.exp(z)) - y * z).mean()
+    l0 = loss(s.X[1].astype(np.float64))
+    s.local_steps([1], 400, 0.5)
+    assert loss(s.X[1].astype(np.float64)) < 0.6 * l0
+    pred = (A @ s.X[1].astype(np.float64)) > 0
+    assert (pred == (y > 0.5)).mean() > 0.85
