@@ -52,7 +52,7 @@ typedef struct { int32_t kind, degree; } swarm_topology;
 enum { SWARM_TOPO_COMPLETE = 0, SWARM_TOPO_RING = 1, SWARM_TOPO_REGULAR = 2 };
 
 enum { SWARM_BLOCKING = 0, SWARM_NONBLOCKING = 1, SWARM_REGISTERS = 2 };
-enum { SWARM_OBJ_NONE = 0, SWARM_OBJ_SYNTH = 1, SWARM_OBJ_LSQ = 2 };
+enum { SWARM_OBJ_NONE = 0, SWARM_OBJ_SYNTH = 1, SWARM_OBJ_LSQ = 2, SWARM_OBJ_LOGISTIC = 3 };
 enum { SWARM_F32 = 0, SWARM_BF16 = 1 };
 
 enum {
@@ -79,7 +79,9 @@ typedef struct {
   int32_t lsq_batch;     /* LSQ: minibatch size (rows drawn uniformly with replacement)           */
   int32_t lsq_dtype;     /* LSQ: SWARM_F32 or SWARM_BF16 storage of the data matrices             */
   int32_t lsq_groups;    /* LSQ: number of data matrices; 0 = one per node, else must divide n    */
-  float   lsq_noise_std; /* LSQ: label noise; labels = A x* + mu_i + noise, mu_i ~ U(-1, 1)       */
+  float   lsq_noise_std; /* LSQ: label noise; labels = A x* + mu_i + noise, mu_i ~ U(-1, 1).
+                            SWARM_OBJ_LOGISTIC uses the same lsq_* fields: logistic regression on the same data
+                            with class labels 1[A x* + mu_i + noise > 0], gradient (sigmoid(a.x) - y) a      */
 } swarm_config;
 
 /* Optional device allocator (e.g. a framework's caching allocator). Must be installed before

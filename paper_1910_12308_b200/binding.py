@@ -18,7 +18,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 
 BLOCKING, NONBLOCKING, REGISTERS = 0, 1, 2
 TOPO_COMPLETE, TOPO_RING, TOPO_REGULAR = 0, 1, 2
-OBJ_NONE, OBJ_SYNTH, OBJ_LSQ = 0, 1, 2
+OBJ_NONE, OBJ_SYNTH, OBJ_LSQ, OBJ_LOGISTIC = 0, 1, 2, 3
 F32, BF16 = 0, 1
 T_X, T_B, T_CODES, T_EXPS, T_ADJ, T_A, T_BVEC, T_XSTAR, T_SCALARS, T_COUNTERS, T_OWN, T_OEXPS, T_CLOCKS = range(13)
 TOPOLOGY = {"complete": TOPO_COMPLETE, "ring": TOPO_RING, "regular": TOPO_REGULAR}

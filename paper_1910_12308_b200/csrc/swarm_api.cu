@@ -120,6 +120,7 @@ LsqView lsq_of(const swarm_ctx* c) {
   LsqView l;
   l.A = c->A; l.bvec = c->bvec; l.m = c->cfg.lsq_m; l.batch = c->cfg.lsq_batch; l.dtype = c->cfg.lsq_dtype;
   l.groups = c->groups; l.nodes_per_group = c->nodes_per_group;
+  l.logistic = c->cfg.objective == SWARM_OBJ_LOGISTIC ? 1 : 0;
   return l;
 }
 
@@ -233,7 +234,7 @@ int apply_config(swarm_ctx* c, const swarm_config& cfg) {
     c->oexps = (int8_t*)dev_alloc(c, (size_t)n * c->nblk);
     if (!c->own || !c->oexps) return SWARM_ENOMEM;
   }
-  if (cfg.objective == SWARM_OBJ_LSQ) {
+  if (cfg.objective == SWARM_OBJ_LSQ || cfg.objective == SWARM_OBJ_LOGISTIC) {
     c->groups = cfg.lsq_groups > 0 ? cfg.lsq_groups : n;
     c->nodes_per_group = n / c->groups;
     const size_t esz = cfg.lsq_dtype == SWARM_BF16 ? 2 : 4;
@@ -260,7 +261,7 @@ int apply_config(swarm_ctx* c, const swarm_config& cfg) {
   SW_CUDA(c, launch_node_scalars(c->scalars, n, cfg.offset_std, cfg.drift_std, s.key0, s.key1, c->stream, &nl));
   SW_CUDA(c, launch_init_models(s, c->scalars, cfg.init_std, c->stream, &nl));
   if (c->B) SW_CUDA(c, cudaMemcpyAsync(c->B, c->X, (size_t)n * row_bytes, cudaMemcpyDeviceToDevice, c->stream));
-  if (cfg.objective == SWARM_OBJ_LSQ) {
+  if (cfg.objective == SWARM_OBJ_LSQ || cfg.objective == SWARM_OBJ_LOGISTIC) {
     LsqView l = lsq_of(c);
     SW_CUDA(c, launch_lsq_data(s, l, c->A, c->xstar, c->bvec, c->scalars, cfg.lsq_noise_std, c->stream, &nl));
   }
@@ -277,11 +278,11 @@ int apply_config(swarm_ctx* c, const swarm_config& cfg) {
 }
 
 int validate_config(const swarm_ctx* c, const swarm_config* cfg) {
-  if (cfg->objective < SWARM_OBJ_NONE || cfg->objective > SWARM_OBJ_LSQ) return SWARM_EINVAL;
+  if (cfg->objective < SWARM_OBJ_NONE || cfg->objective > SWARM_OBJ_LOGISTIC) return SWARM_EINVAL;
   if (cfg->nonblocking < 0 || cfg->nonblocking > 2) return SWARM_EINVAL;
   if (!(cfg->init_std >= 0.0f) || !(cfg->offset_std >= 0.0f) || !(cfg->grad_std >= 0.0f) || !(cfg->drift_std >= 0.0f))
     return SWARM_EINVAL;
-  if (cfg->objective == SWARM_OBJ_LSQ) {
+  if (cfg->objective == SWARM_OBJ_LSQ || cfg->objective == SWARM_OBJ_LOGISTIC) {
     if (cfg->lsq_m < 1 || cfg->lsq_batch < 1 || cfg->lsq_batch > 256) return SWARM_EINVAL;
     if (cfg->lsq_dtype != SWARM_F32 && cfg->lsq_dtype != SWARM_BF16) return SWARM_EINVAL;
     if (cfg->lsq_groups < 0 || cfg->lsq_groups > c->n) return SWARM_EINVAL;
@@ -514,7 +515,7 @@ int swarm_local_steps(swarm_ctx* c, const int32_t* node_ids, int32_t count, int3
   DeviceGuard guard(c->device);
   void *host, *dev;
   int slot;
-  if (c->cfg.objective == SWARM_OBJ_LSQ && c->tc_partial) {
+  if (c->cfg.objective >= SWARM_OBJ_LSQ && c->tc_partial) {
     // bf16 data: batch the listed nodes that share a data matrix and a step counter (hence the
     // minibatch) into units of up to 16 for the tensor-core kernels
     std::vector<LsqUnit> units;

@@ -119,6 +119,12 @@ __device__ __forceinline__ void normal4(uint32_t group, uint32_t row, uint32_t e
   normal_pair(w.z, w.w, z[2], z[3]);
 }
 
+// Residual of one sampled row: least squares <a, x> - b, or logistic regression sigmoid(<a, x>) - y.
+__device__ __forceinline__ float row_residual(float dot, float label, int logistic) {
+  const float pred = logistic ? 1.0f / (1.0f + expf(-dot)) : dot;
+  return pred - label;
+}
+
 // ---------------------------------------------------------------------------------------
 // Quantizer: lattice of step 2^e, colour = index mod 2^b, L = 2^(b-1) - 1.
 // ---------------------------------------------------------------------------------------

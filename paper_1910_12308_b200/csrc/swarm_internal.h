@@ -70,6 +70,7 @@ struct LsqView {
   const void* A;       // [groups][m][pitch] fp32 or bf16
   const float* bvec;   // [n][m]
   int32_t m, batch, dtype, groups, nodes_per_group;
+  int32_t logistic;    // 1: residual = sigmoid(<a, x>) - y with labels in {0, 1}; 0: residual = <a, x> - b
 };
 
 // --- swarm_interact.cu -------------------------------------------------------------------

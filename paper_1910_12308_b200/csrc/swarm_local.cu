@@ -78,7 +78,8 @@ __device__ __forceinline__ float load_as_float(const __nv_bfloat16* p) { return 
 template <typename T>
 __global__ void __launch_bounds__(256)
 lsq_labels_kernel(const T* __restrict__ A, const float* __restrict__ xstar, float* bvec, const float* __restrict__ scalars,
-                  int64_t pitch, int64_t d, int m, int nodes_per_group, float noise_std, uint32_t k0, uint32_t k1) {
+                  int64_t pitch, int64_t d, int m, int nodes_per_group, float noise_std, uint32_t k0, uint32_t k1,
+                  int logistic) {
   const int r = blockIdx.x, grp = blockIdx.y;
   const T* row = A + ((int64_t)grp * m + r) * pitch;
   double acc = 0.0;
@@ -94,7 +95,8 @@ lsq_labels_kernel(const T* __restrict__ A, const float* __restrict__ xstar, floa
     float z[4];
     normal4((uint32_t)(r / 4), (uint32_t)node, 0u, kStreamDataNoise, k0, k1, z);
     const float noise = __fmul_rn(noise_std, z[r % 4]);
-    bvec[(int64_t)node * m + r] = (float)(dot + (double)scalars[node * 3 + 2] + (double)noise);
+    const float score = (float)(dot + (double)scalars[node * 3 + 2] + (double)noise);
+    bvec[(int64_t)node * m + r] = logistic ? (score > 0.0f ? 1.0f : 0.0f) : score;   // class label = sign of the score
   }
 }
 
@@ -213,7 +215,7 @@ lsq_update_kernel(StoreView s, LsqView l, const NodeList nodes, int step, float 
     if ((threadIdx.x & 31) == 0) {
       const int r = minibatch_row(si, group, event, l.m, s.key0, s.key1);
       rows[si] = r;
-      resid[si] = acc - l.bvec[(int64_t)nd.node * l.m + r];
+      resid[si] = row_residual(acc, l.bvec[(int64_t)nd.node * l.m + r], l.logistic);
     }
   }
   __syncthreads();
@@ -312,7 +314,7 @@ lsq_small_kernel(StoreView s, LsqView l, const NodeList nodes, int H, float lr, 
     if (tid < l.batch) {
       float tot = 0.0f;
       for (int r = 0; r < csize; ++r) tot += *cluster.map_shared_rank(&part[tid], r);
-      resid[tid] = tot - labels[rows[tid]];
+      resid[tid] = row_residual(tot, labels[rows[tid]], l.logistic);
     }
     __syncthreads();
     float4 g0 = make_float4(0.f, 0.f, 0.f, 0.f), g1 = g0;
@@ -422,12 +424,12 @@ cudaError_t launch_lsq_data(const StoreView& s, const LsqView& l, void* A, float
     auto* Ab = reinterpret_cast<__nv_bfloat16*>(A);
     lsq_matrix_kernel<<<grid_a, 256, 0, st>>>(Ab, s.pitch, s.d, l.m, inv_sqrt_d, s.key0, s.key1);
     lsq_labels_kernel<<<grid_l, 256, 0, st>>>(Ab, xstar, bvec, scalars_dev, s.pitch, s.d, l.m, l.nodes_per_group,
-                                               noise_std, s.key0, s.key1);
+                                               noise_std, s.key0, s.key1, l.logistic);
   } else {
     auto* Af = reinterpret_cast<float*>(A);
     lsq_matrix_kernel<<<grid_a, 256, 0, st>>>(Af, s.pitch, s.d, l.m, inv_sqrt_d, s.key0, s.key1);
     lsq_labels_kernel<<<grid_l, 256, 0, st>>>(Af, xstar, bvec, scalars_dev, s.pitch, s.d, l.m, l.nodes_per_group,
-                                               noise_std, s.key0, s.key1);
+                                               noise_std, s.key0, s.key1, l.logistic);
   }
   *launches += 3;
   return cudaGetLastError();

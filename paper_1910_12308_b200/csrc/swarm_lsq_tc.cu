@@ -294,7 +294,7 @@ lsq_tc_finalize_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units
   float r = 0.0f;
   if (sidx < l.batch && j < u.count) {
     const int row = tc_minibatch_row(sidx, u.group, u.event + (uint32_t)step, l.m, s.key0, s.key1);
-    r = acc - l.bvec[(int64_t)u.nodes[j] * l.m + row];
+    r = row_residual(acc, l.bvec[(int64_t)u.nodes[j] * l.m + row], l.logistic);
   }
   __nv_bfloat16 hi, lo;
   split_bf16(r, hi, lo);

@@ -304,6 +304,27 @@ def test_batched_tensor_core_least_squares_steps(n, groups, d, m, batch):
         inject(orc, gpu, what=("X",))
 
 
+@pytest.mark.parametrize("d,m,batch,dtype,groups", [(4096, 64, 16, 0, 0), (20000, 24, 40, 0, 2), (33000, 64, 64, 1, 2),
+                                                   (700, 12, 5, 1, 0)])
+def test_logistic_regression_steps_within_tolerance(d, m, batch, dtype, groups):
+    """Second objective on the least-squares data: residual sigmoid(<a, x>) - y, through the cluster kernel
+    (short models), the general kernels and the tensor-core kernels."""
+    cfg = dict(objective=3, lsq_m=m, lsq_batch=batch, lsq_dtype=dtype, lsq_groups=groups, lsq_noise_std=0.2,
+               init_std=0.5)
+    orc, gpu = make_pair(4, d, seed=83, **cfg)
+    labels = gpu.get_all(g.T_BVEC)
+    assert set(np.unique(labels).tolist()) <= {0.0, 1.0}
+    assert (labels != orc.bvec).mean() < 0.02                     # a score next to zero may flip a class
+    inject(orc, gpu)
+    for rnd in range(3):
+        nodes = [0, 3, 1] if rnd else [2, 0]
+        assert orc.local_steps(nodes, 2, 0.5) == 0 and gpu.local_steps(nodes, 2, 0.5) == 0
+        gpu.sync()
+        for i in range(4):
+            assert rel_err(gpu.get(g.T_X, i), orc.X[i]) < TOL, (rnd, i)
+        inject(orc, gpu, what=("X",))
+
+
 def test_geometric_step_counts_match():
     cfg = dict(objective=1, grad_std=0.03, drift_std=0.1)
     orc, gpu = make_pair(12, 3000, seed=61, **cfg)
