@@ -406,6 +406,23 @@ def run_ours(args, wl, name):
                      "peak_kind": peak_kind, "frac_of_8000": achieved / 8000.0, "traffic": TRAFFIC.get(name),
                      "algorithmic_bytes_per_launch": per_launch_bytes, "kernel_ms": kern_ms},
     }
+    # mean model and potential (one HBM pass over all n models each), timed on their own
+    reps = 20
+    mu = torch.empty(wl["d"], dtype=torch.float32, device="cuda")
+    L, h = sw._L, sw._h
+    for name_k, call in (("mean_model", lambda: L.swarm_mean_model(h, mu.data_ptr())),
+                         ("potential", lambda: sw.potential())):
+        for _ in range(3):
+            call()
+        barrier()
+        ev0.record(stream)
+        for _ in range(reps):
+            call()
+        ev1.record(stream)
+        barrier()
+        t_ms = ev0.elapsed_time(ev1) / reps
+        out.setdefault("aux_kernels", {})[name_k] = {
+            "ms": t_ms, "GB/s": 4.0 * wl["n"] * wl["d"] / (t_ms * 1e-3) / 1e9, "bytes": 4 * wl["n"] * wl["d"]}
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v, T, nl, tt, swl = time_oracle(wl, budget_s=10.0, max_launches=40)
         v1, _, nl1, tt1, _ = time_oracle(wl, budget_s=3.0, max_launches=1, threads=1)
