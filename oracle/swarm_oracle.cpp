@@ -256,6 +256,11 @@ struct Swarm {
   std::vector<int8_t> oexps;         // n * nblk
   std::vector<uint32_t> wo;          // write counters of the own registers
   std::vector<uint32_t> tau;         // interactions since the node last initiated
+  // auxiliary potentials of the staleness analysis (appendix, "Potential Functions"): per node the mean
+  // model at its last initiation and the squared distance of its snapshot to that mean
+  int32_t track = 0;
+  std::vector<float> mu_hist;        // n * d
+  std::vector<double> a_hist;        // n
   int32_t p_mode = 0;                // convention the buffers were last written in: 0 none/blocking, 1 single buffer, 2 registers
   // objective data
   std::vector<float> offset, drift, shift;   // per-node scalars
@@ -336,6 +341,7 @@ void init_state(Swarm& s) {
   const int64_t d = s.d;
   const Config& c = s.cfg;
   s.offset.assign(n, 0.0f); s.drift.assign(n, 0.0f); s.shift.assign(n, 0.0f);
+  s.track = 0; s.mu_hist.clear(); s.a_hist.clear();
   for (int i = 0; i < n; ++i) {
     uint32_t wd[4];
     s.rng.words(0, (uint32_t)i, 0, kStreamNodeScalars, wd);
@@ -698,6 +704,26 @@ void interact_registers(Swarm& s, int a, int b, int bits) {
   s.wo[a] += 1; s.w[a] += 1; s.w[b] += 1;
 }
 
+// mu = (1/n) sum_i X^i, accumulated in double in node order, rounded once.
+void mean_model(const Swarm& s, float* out) {
+  for (int64_t k = 0; k < s.d; ++k) {
+    double acc = 0.0;
+    for (int i = 0; i < s.n; ++i) acc += (double)s.X[(int64_t)i * s.d + k];
+    out[k] = (float)(acc / (double)s.n);
+  }
+}
+
+// Node i initiated: remember the mean model of that moment and ||X^_i - mu||^2 (one term of A_t).
+void record_initiation(Swarm& s, int i, const float* mu) {
+  double a = 0.0;
+  for (int64_t k = 0; k < s.d; ++k) {
+    s.mu_hist[(int64_t)i * s.d + k] = mu[k];
+    const double t = (double)s.base(i)[k] - (double)mu[k];
+    a += t * t;
+  }
+  s.a_hist[i] = a;
+}
+
 int validate_pairs(const Swarm& s, const int32_t* pairs, int npairs) {
   std::vector<uint8_t> used(s.n, 0);
   for (int p = 0; p < npairs; ++p) {
@@ -866,6 +892,7 @@ int orc_interact(void* h, const int32_t* pairs, int32_t npairs, int32_t bits, in
   if (!(bits == 2 || bits == 4 || bits == 8 || (bits == 32 && mode == 0))) return -1;
   if (mode == 1 && !s.cfg.nonblocking) return -4;
   if (mode == 2 && s.cfg.nonblocking != 2) return -4;
+  if (mode == 0 && s.track) return -4;   // a blocking exchange has no outdated model to track
   const int v = validate_pairs(s, pairs, npairs);
   if (v != 0) return v;
   if (mode == 1 && needs_publish(s, bits, 1)) publish(s, bits);
@@ -894,6 +921,50 @@ int orc_interact(void* h, const int32_t* pairs, int32_t npairs, int32_t bits, in
     for (int i = 0; i < s.n; ++i) s.tau[i] += 1;
     s.tau[pairs[2 * p]] = 0;
   }
+  // the interactions of one launch count as simultaneous for the auxiliary potentials: every initiator
+  // of the launch records the mean model after the launch
+  if (s.track && npairs > 0) {
+    std::vector<float> mu(s.d);
+    mean_model(s, mu.data());
+    for (int p = 0; p < npairs; ++p) record_initiation(s, pairs[2 * p], mu.data());
+  }
+  return 0;
+}
+
+// Start (or stop) tracking the auxiliary potentials: every node counts as having initiated just now.
+int orc_track_staleness(void* h, int32_t enable) {
+  Swarm& s = *(Swarm*)h;
+  if (!enable) { s.track = 0; s.mu_hist.clear(); s.a_hist.clear(); return 0; }
+  if (!s.cfg.nonblocking || s.b_stale) return -4;
+  s.track = 1;
+  s.mu_hist.assign((size_t)s.n * s.d, 0.0f);
+  s.a_hist.assign(s.n, 0.0);
+  std::vector<float> mu(s.d);
+  mean_model(s, mu.data());
+  for (int i = 0; i < s.n; ++i) { record_initiation(s, i, mu.data()); s.tau[i] = 0; }
+  return 0;
+}
+float* orc_mu_hist(void* h) { Swarm& s = *(Swarm*)h; return s.mu_hist.empty() ? nullptr : s.mu_hist.data(); }
+double* orc_a_hist(void* h) { Swarm& s = *(Swarm*)h; return s.a_hist.empty() ? nullptr : s.a_hist.data(); }
+
+// out = { Gamma^_t = sum_i ||X^_i - mu_t||^2,  A_t = sum_i ||X_{t-tau_i} - mu_{t-tau_i}||^2,
+//         B_t = sum_i ||mu_t - mu_{t-tau_i}||^2 }  with X^_i = X_{t-tau_i} the snapshot of node i.
+int orc_aux_potentials(void* h, double* out) {
+  Swarm& s = *(Swarm*)h;
+  if (!s.track) return -4;
+  std::vector<float> mu(s.d);
+  mean_model(s, mu.data());
+  double gh = 0.0, A = 0.0, Bt = 0.0;
+  for (int i = 0; i < s.n; ++i) {
+    for (int64_t k = 0; k < s.d; ++k) {
+      const double t = (double)s.base(i)[k] - (double)mu[k];
+      gh += t * t;
+      const double u = (double)mu[k] - (double)s.mu_hist[(int64_t)i * s.d + k];
+      Bt += u * u;
+    }
+    A += s.a_hist[i];
+  }
+  out[0] = gh; out[1] = A; out[2] = Bt;
   return 0;
 }
 
@@ -918,14 +989,7 @@ int orc_publish(void* h, int32_t bits) {
 }
 
 // mu = (1/n) sum_i X^i, accumulated in double, rounded once.
-void orc_mean_model(void* h, float* out) {
-  Swarm& s = *(Swarm*)h;
-  for (int64_t k = 0; k < s.d; ++k) {
-    double acc = 0.0;
-    for (int i = 0; i < s.n; ++i) acc += (double)s.x(i)[k];
-    out[k] = (float)(acc / (double)s.n);
-  }
-}
+void orc_mean_model(void* h, float* out) { mean_model(*(Swarm*)h, out); }
 
 // Gamma = sum_i ||X^i - mu||^2, two passes in double.
 double orc_potential(void* h) {

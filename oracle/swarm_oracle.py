@@ -68,6 +68,9 @@ def lib():
         "orc_p_mode": (i32p, [vp]),
         "orc_mean_model": (None, [vp, f32p]),
         "orc_potential": (C.c_double, [vp]),
+        "orc_track_staleness": (C.c_int, [vp, C.c_int32]),
+        "orc_mu_hist": (f32p, [vp]), "orc_a_hist": (C.POINTER(C.c_double), [vp]),
+        "orc_aux_potentials": (C.c_int, [vp, C.POINTER(C.c_double)]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(L, name)
@@ -331,3 +334,22 @@ class OracleSwarm:
 
     def potential(self):
         return float(lib().orc_potential(self._h))
+
+    def track_staleness(self, enable=True):
+        return int(lib().orc_track_staleness(self._h, 1 if enable else 0))
+
+    @property
+    def mu_hist(self):
+        return _view(lib().orc_mu_hist(self._h), (self.n, self.d), np.float32)
+
+    @property
+    def a_hist(self):
+        return _view(lib().orc_a_hist(self._h), (self.n,), np.float64)
+
+    def aux_potentials(self):
+        """(Gamma-hat, A_t, B_t) of the staleness analysis; tracking must be on."""
+        out = (C.c_double * 3)()
+        rc = int(lib().orc_aux_potentials(self._h, out))
+        if rc != 0:
+            raise ValueError(rc)
+        return float(out[0]), float(out[1]), float(out[2])
