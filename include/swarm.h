@@ -146,6 +146,22 @@ int swarm_mean_model(swarm_ctx *ctx, float *out_dev);
 /* Section 4: Gamma = sum_i ||X^i - mu||^2, written to *out_gamma_host. Synchronises. */
 int swarm_potential(swarm_ctx *ctx, double *out_gamma_host);
 
+/* Appendix, "Notation and Auxiliary Potential Functions": the potentials that the analysis uses to
+ * control outdated models. With X^_i = X_{t - tau_i} the snapshot B_i of node i (its model right after
+ * its last initiation) and m_i the mean model recorded at that moment,
+ *     Gamma^_t = sum_i ||X^_i - mu_t||^2,   A_t = sum_i ||X^_i - m_i||^2,   B_t = sum_i ||mu_t - m_i||^2,
+ * and Gamma^_t <= 2 A_t + 2 B_t. mu is the fp32 mean model that swarm_mean_model produces; sums in fp64.
+ * swarm_track_staleness(ctx, 1) allocates the records (n * pitch floats of device memory), treats every
+ * node as having initiated just now (records = current mean, clocks tau = 0) and makes every later
+ * non-blocking or register interaction update the records of its initiators; the interactions of one
+ * launch count as simultaneous: all its initiators record the mean model after the launch (one extra
+ * pass over the n models per launch). enable = 0 frees the records.
+ * Errors: ESTATE (configuration without snapshots, snapshots stale after a blocking exchange), ENOMEM.
+ * While tracking is on, swarm_interact in SWARM_BLOCKING mode returns ESTATE. */
+int swarm_track_staleness(swarm_ctx *ctx, int32_t enable);
+/* out3_host receives Gamma^_t, A_t, B_t. Synchronises. ESTATE unless tracking is on. */
+int swarm_aux_potentials(swarm_ctx *ctx, double *out3_host);
+
 /* ------------------------------------------------------------------------------------------
  * Auxiliary calls
  * ---------------------------------------------------------------------------------------- */
@@ -183,7 +199,9 @@ enum {
   SWARM_T_COUNTERS = 9, /* 3 uint32: buffer write counter, local-step counter, code width of the buffer */
   SWARM_T_OWN = 10,     /* d uint16: own register (ESTATE unless nonblocking = 2)                           */
   SWARM_T_OEXPS = 11,   /* nblk int8: exponents of the own register                                         */
-  SWARM_T_CLOCKS = 12   /* 2 uint32: write counter of the own register, staleness clock tau                 */
+  SWARM_T_CLOCKS = 12,  /* 2 uint32: write counter of the own register, staleness clock tau                 */
+  SWARM_T_MU_RECORD = 13, /* d floats: mean model at the node's last initiation (ESTATE unless tracking)    */
+  SWARM_T_A_RECORD = 14   /* 1 double: ||snapshot - mean||^2 at the node's last initiation                  */
 };
 int swarm_get_tensor(swarm_ctx *ctx, int32_t which, int32_t node, void *dst_host, size_t bytes);
 int swarm_set_tensor(swarm_ctx *ctx, int32_t which, int32_t node, const void *src_host, size_t bytes);

@@ -20,12 +20,13 @@ BLOCKING, NONBLOCKING, REGISTERS = 0, 1, 2
 TOPO_COMPLETE, TOPO_RING, TOPO_REGULAR = 0, 1, 2
 OBJ_NONE, OBJ_SYNTH, OBJ_LSQ, OBJ_LOGISTIC = 0, 1, 2, 3
 F32, BF16 = 0, 1
-T_X, T_B, T_CODES, T_EXPS, T_ADJ, T_A, T_BVEC, T_XSTAR, T_SCALARS, T_COUNTERS, T_OWN, T_OEXPS, T_CLOCKS = range(13)
+OK, EINVAL, ERANGE, EPAIR, ESTATE, ENOMEM, ECUDA = 0, -1, -2, -3, -4, -5, -6
+T_X, T_B, T_CODES, T_EXPS, T_ADJ, T_A, T_BVEC, T_XSTAR, T_SCALARS, T_COUNTERS, T_OWN, T_OEXPS, T_CLOCKS, T_MU_RECORD, T_A_RECORD = range(15)
 TOPOLOGY = {"complete": TOPO_COMPLETE, "ring": TOPO_RING, "regular": TOPO_REGULAR}
 
 EXPORTS = [
     "swarm_set_allocator", "swarm_init", "swarm_local_steps", "swarm_local_steps_geometric", "swarm_interact", "swarm_mean_model",
-    "swarm_potential", "swarm_configure", "swarm_sample_pairs", "swarm_publish", "swarm_register_publish", "swarm_get_buffer_mode",
+    "swarm_potential", "swarm_track_staleness", "swarm_aux_potentials", "swarm_configure", "swarm_sample_pairs", "swarm_publish", "swarm_register_publish", "swarm_get_buffer_mode",
     "swarm_set_buffer_mode", "swarm_get_tensor",
     "swarm_set_tensor", "swarm_get_state", "swarm_set_state", "swarm_model_ptr", "swarm_set_stream",
     "swarm_sync", "swarm_potential_static", "swarm_kernel_launches", "swarm_last_cuda_error", "swarm_strerror", "swarm_destroy",
@@ -85,6 +86,8 @@ def load():
         "swarm_interact": (C.c_int, [vp, C.POINTER(SwarmPair), i32, i32, i32]),
         "swarm_mean_model": (C.c_int, [vp, vp]),
         "swarm_potential": (C.c_int, [vp, C.POINTER(C.c_double)]),
+        "swarm_track_staleness": (C.c_int, [vp, i32]),
+        "swarm_aux_potentials": (C.c_int, [vp, C.POINTER(C.c_double)]),
         "swarm_configure": (C.c_int, [vp, C.POINTER(SwarmConfig)]),
         "swarm_sample_pairs": (C.c_int, [vp, i32, C.POINTER(SwarmPair), C.POINTER(i32)]),
         "swarm_publish": (C.c_int, [vp, i32]),
@@ -231,6 +234,16 @@ class Swarm:
         self._check(self._L.swarm_potential(self._h, C.byref(g)), "swarm_potential")
         return g.value
 
+    def track_staleness(self, enable=True):
+        """Start (or stop) recording what the auxiliary potentials need; returns the C code."""
+        return int(self._L.swarm_track_staleness(self._h, 1 if enable else 0))
+
+    def aux_potentials(self):
+        """(Gamma-hat, A_t, B_t) of the staleness analysis."""
+        out = (C.c_double * 3)()
+        self._check(self._L.swarm_aux_potentials(self._h, out), "swarm_aux_potentials")
+        return float(out[0]), float(out[1]), float(out[2])
+
     # -- auxiliary
     def configure(self, **kw):
         for k, v in kw.items():
@@ -283,7 +296,7 @@ class Swarm:
             T_EXPS: (np.int8, self.nblk), T_ADJ: (np.int32, self.degree), T_A: (np.float32, m * self.d),
             T_BVEC: (np.float32, m), T_XSTAR: (np.float32, self.d), T_SCALARS: (np.float32, 3),
             T_COUNTERS: (np.uint32, 3), T_OWN: (np.uint16, self.d), T_OEXPS: (np.int8, self.nblk),
-            T_CLOCKS: (np.uint32, 2),
+            T_CLOCKS: (np.uint32, 2), T_MU_RECORD: (np.float32, self.d), T_A_RECORD: (np.float64, 1),
         }[which]
 
     def get(self, which, node=0):

@@ -66,7 +66,12 @@ struct swarm_ctx {
   int* kernel_status = nullptr;      // set by a kernel whose bounded wait expired
   int* kernel_status_host = nullptr; // pinned
   double* pot_partial = nullptr;
-  double* pot_out = nullptr;
+  double* pot_out = nullptr;         // 4 doubles
+  // auxiliary potentials of the staleness analysis (off until swarm_track_staleness)
+  bool track = false;
+  float* mu_hist = nullptr;          // [n][pitch] mean model at each node's last initiation
+  double* a_hist = nullptr;          // n: ||snapshot - mean||^2 at each node's last initiation
+  double* aux_partial = nullptr;     // max(n, 2) * potential_partials(d)
   int32_t* pairs_out_dev = nullptr;  // 2 * n/2 + 1 (sampler result, count last)
   uint8_t* used_dev = nullptr;       // n
   float* convert_tmp = nullptr;      // pitch floats (bf16 row conversion)
@@ -194,6 +199,10 @@ void free_objective(swarm_ctx* c) {
   dev_free(c, c->B); c->B = nullptr;
   dev_free(c, c->own); c->own = nullptr;
   dev_free(c, c->oexps); c->oexps = nullptr;
+  dev_free(c, c->mu_hist); c->mu_hist = nullptr;
+  dev_free(c, c->a_hist); c->a_hist = nullptr;
+  dev_free(c, c->aux_partial); c->aux_partial = nullptr;
+  c->track = false;
   c->groups = 0; c->nodes_per_group = 0;
 }
 
@@ -358,6 +367,20 @@ int do_register_publish(swarm_ctx* c, int bits) {
   return SWARM_OK;
 }
 
+// The listed nodes initiated just now: store the current mean model as their record and their
+// snapshot's squared distance to it (lists longer than the inline capacity go in slices).
+int record_initiations(swarm_ctx* c, const int32_t* nodes, int count) {
+  int nl = 0;
+  for (int base = 0; base < count; base += kInlineNodes) {
+    NodeList list{};
+    list.n = std::min(kInlineNodes, count - base);
+    for (int t = 0; t < list.n; ++t) { list.inl[t].node = nodes[base + t]; list.inl[t].event = 0; }
+    SW_CUDA(c, launch_staleness_record(view_of(c), c->mu_hist, list, c->aux_partial, c->a_hist, c->stream, &nl));
+  }
+  c->launches += nl;
+  return SWARM_OK;
+}
+
 bool buffers_need_publish(const swarm_ctx* c, int bits, int mode) {
   if (c->b_stale != 0 || c->p_mode != mode) return true;
   for (int i = 0; i < c->n; ++i)
@@ -432,7 +455,7 @@ int swarm_init(swarm_ctx** out, int32_t n, int64_t d, swarm_topology topo, uint6
   c->adj_dev = (int32_t*)dev_alloc(c, c->adj.size() * sizeof(int32_t));
   c->scalars = (float*)dev_alloc(c, (size_t)n * 3 * sizeof(float));
   c->pot_partial = (double*)dev_alloc(c, (size_t)potential_partials(d) * sizeof(double));
-  c->pot_out = (double*)dev_alloc(c, sizeof(double));
+  c->pot_out = (double*)dev_alloc(c, 4 * sizeof(double));
   c->pairs_out_dev = (int32_t*)dev_alloc(c, (2 * max_pairs + 1) * sizeof(int32_t));
   c->used_dev = (uint8_t*)dev_alloc(c, (size_t)n);
   c->kernel_status = (int*)dev_alloc(c, sizeof(int));
@@ -440,7 +463,7 @@ int swarm_init(swarm_ctx** out, int32_t n, int64_t d, swarm_topology topo, uint6
   bool ok = c->X && c->codes && c->exps && c->adj_dev && c->scalars && c->pot_partial && c->pot_out &&
             c->pairs_out_dev && c->used_dev && c->stage_dev && c->kernel_status;
   ok = ok && cudaMallocHost(&c->stage_host, c->stage_slot_bytes * kStageSlots) == cudaSuccess;
-  ok = ok && cudaMallocHost((void**)&c->pot_host, sizeof(double)) == cudaSuccess;
+  ok = ok && cudaMallocHost((void**)&c->pot_host, 4 * sizeof(double)) == cudaSuccess;
   ok = ok && cudaMallocHost((void**)&c->kernel_status_host, sizeof(int)) == cudaSuccess;
   ok = ok && cudaMemsetAsync(c->kernel_status, 0, sizeof(int), c->stream) == cudaSuccess;
   ok = ok && cudaMallocHost((void**)&c->pairs_out_host, (2 * max_pairs + 1) * sizeof(int32_t)) == cudaSuccess;
@@ -630,6 +653,7 @@ int swarm_interact(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, int32_
   if (!(quant || (bits == 32 && mode == SWARM_BLOCKING))) return SWARM_EINVAL;
   if (mode == SWARM_NONBLOCKING && !c->cfg.nonblocking) return SWARM_ESTATE;
   if (mode == SWARM_REGISTERS && c->cfg.nonblocking != 2) return SWARM_ESTATE;
+  if (mode == SWARM_BLOCKING && c->track) return SWARM_ESTATE;   // no outdated model to track
   if (npairs > c->n / 2) return SWARM_EPAIR;
   int rc = validate_pairs(c, pairs, npairs);
   if (rc != SWARM_OK) return rc;
@@ -687,6 +711,59 @@ int swarm_interact(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, int32_
     for (int i = 0; i < c->n; ++i) c->tau[i] += 1;
     c->tau[pairs[p].a] = 0;
   }
+  if (c->track) {
+    std::vector<int32_t> init((size_t)npairs);
+    for (int p = 0; p < npairs; ++p) init[p] = pairs[p].a;
+    rc = record_initiations(c, init.data(), npairs);
+    if (rc != SWARM_OK) return rc;
+  }
+  return SWARM_OK;
+}
+
+int swarm_track_staleness(swarm_ctx* c, int32_t enable) {
+  if (!c) return SWARM_EINVAL;
+  DeviceGuard guard(c->device);
+  if (!enable) {
+    SW_CUDA(c, cudaStreamSynchronize(c->stream));
+    dev_free(c, c->mu_hist); c->mu_hist = nullptr;
+    dev_free(c, c->a_hist); c->a_hist = nullptr;
+    dev_free(c, c->aux_partial); c->aux_partial = nullptr;
+    c->track = false;
+    return SWARM_OK;
+  }
+  if (!c->cfg.nonblocking || c->b_stale) return SWARM_ESTATE;
+  if (!c->track) {
+    const size_t parts = (size_t)potential_partials(c->d);
+    c->mu_hist = (float*)dev_alloc(c, (size_t)c->n * c->pitch * sizeof(float));
+    c->a_hist = (double*)dev_alloc(c, (size_t)c->n * sizeof(double));
+    c->aux_partial = (double*)dev_alloc(c, (size_t)std::max(kInlineNodes, 2) * parts * sizeof(double));
+    if (!c->mu_hist || !c->a_hist || !c->aux_partial) {
+      dev_free(c, c->mu_hist); c->mu_hist = nullptr;
+      dev_free(c, c->a_hist); c->a_hist = nullptr;
+      dev_free(c, c->aux_partial); c->aux_partial = nullptr;
+      return SWARM_ENOMEM;
+    }
+    SW_CUDA(c, cudaMemsetAsync(c->mu_hist, 0, (size_t)c->n * c->pitch * sizeof(float), c->stream));
+    c->track = true;
+  }
+  std::vector<int32_t> all((size_t)c->n);
+  for (int i = 0; i < c->n; ++i) all[i] = i;
+  const int rc = record_initiations(c, all.data(), c->n);
+  if (rc != SWARM_OK) return rc;
+  std::fill(c->tau.begin(), c->tau.end(), 0u);
+  return SWARM_OK;
+}
+
+int swarm_aux_potentials(swarm_ctx* c, double* out3) {
+  if (!c || !out3) return SWARM_EINVAL;
+  if (!c->track) return SWARM_ESTATE;
+  DeviceGuard guard(c->device);
+  int nl = 0;
+  SW_CUDA(c, launch_aux_potentials(view_of(c), c->mu_hist, c->a_hist, c->aux_partial, c->pot_out, c->stream, &nl));
+  c->launches += nl;
+  SW_CUDA(c, cudaMemcpyAsync(c->pot_host, c->pot_out, 3 * sizeof(double), cudaMemcpyDeviceToHost, c->stream));
+  SW_CUDA(c, cudaStreamSynchronize(c->stream));
+  out3[0] = c->pot_host[0]; out3[1] = c->pot_host[1]; out3[2] = c->pot_host[2];
   return SWARM_OK;
 }
 
@@ -801,6 +878,12 @@ static int tensor_access(swarm_ctx* c, int32_t which, int32_t node, void* host, 
     case SWARM_T_OEXPS:
       if (!c->oexps) return SWARM_ESTATE;
       dev = c->oexps + (size_t)node * c->nblk; want = (size_t)c->nblk; break;
+    case SWARM_T_MU_RECORD:
+      if (!c->track) return SWARM_ESTATE;
+      dev = c->mu_hist + (size_t)node * c->pitch; want = d * 4; break;
+    case SWARM_T_A_RECORD:
+      if (!c->track) return SWARM_ESTATE;
+      dev = c->a_hist + node; want = 8; break;
     case SWARM_T_CLOCKS: {
       if (bytes != 8) return SWARM_EINVAL;
       uint32_t* v = (uint32_t*)host;

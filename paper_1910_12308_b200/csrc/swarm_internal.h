@@ -117,6 +117,13 @@ cudaError_t launch_mean_model(const StoreView& s, float* out_dev, cudaStream_t s
 cudaError_t launch_potential(const StoreView& s, double* partial_dev, double* out_dev, cudaStream_t st,
                              int* launches);
 int64_t potential_partials(int64_t d);
+// Staleness tracking. mu_hist_dev: [n][pitch] mean-model records; a_hist_dev: n doubles;
+// partial_dev: list.n * potential_partials(d) doubles (record) or 2 * potential_partials(d) (query).
+cudaError_t launch_staleness_record(const StoreView& s, float* mu_hist_dev, const NodeList& list,
+                                    double* partial_dev, double* a_hist_dev, cudaStream_t st, int* launches);
+// out_dev: three doubles (Gamma-hat, A_t, B_t).
+cudaError_t launch_aux_potentials(const StoreView& s, const float* mu_hist_dev, const double* a_hist_dev,
+                                  double* partial_dev, double* out_dev, cudaStream_t st, int* launches);
 
 // Row conversion helpers for get/set of bf16 data.
 cudaError_t launch_bf16_to_f32(const void* src, float* dst, int64_t count, cudaStream_t st, int* launches);
