@@ -29,6 +29,11 @@ WORKLOADS = {
     # n = 64 nodes, d = 2^20, ring, 32 disjoint pairs per launch, 4-bit codes, averaging only.
     "ring64_d1m_b4": dict(n=64, d=1 << 20, topology="ring", degree=0, pairs=32, bits=4, mode=0, H=0, lr=0.0, seed=2,
                           cfg=dict(offset_std=float(np.sqrt(0.1)))),
+    # the same with code widths that do not divide a byte (codes regrouped into aligned words by warp shuffles)
+    "ring64_d1m_b3": dict(n=64, d=1 << 20, topology="ring", degree=0, pairs=32, bits=3, mode=0, H=0, lr=0.0, seed=2,
+                          cfg=dict(offset_std=float(np.sqrt(0.1)))),
+    "ring64_d1m_b7": dict(n=64, d=1 << 20, topology="ring", degree=0, pairs=32, bits=7, mode=0, H=0, lr=0.0, seed=2,
+                          cfg=dict(offset_std=float(np.sqrt(0.1)))),
     # n = 16 nodes, d = 25,557,032 (ResNet-50 sized), complete graph, 8 pairs, synthetic-gradient steps.
     "complete16_resnet50_b8": dict(n=16, d=25_557_032, topology="complete", degree=0, pairs=8, bits=8, mode=0, H=2,
                                    lr=0.05, seed=4, cfg=dict(objective=1, grad_std=float(np.sqrt(1e-3)),

@@ -27,8 +27,9 @@
  *                 adopted at its last initiation (Algorithm 1: \hat X^i)
  *   codes[n][nblk*1024] bytes: the node's communication buffer; at b bits per
  *                 coordinate the first nblk*128*b bytes are meaningful. Within a
- *                 1024-coordinate block the code of local coordinate k occupies bits
- *                 [(k mod (8/b))*b, +b) of byte (k*b) div 8; codes past d are zero.
+ *                 1024-coordinate block the codes form a little-endian bit stream: the code of
+ *                 local coordinate k occupies bits [k*b, (k+1)*b) of the block's 128*b bytes
+ *                 (stream bit t = bit t mod 8 of byte t div 8); codes past d are zero.
  *   exps[n][nblk] int8 lattice exponents e (step 2^e) of each block of the buffer
  *   nblk = ceil(d / 1024)
  */
@@ -117,8 +118,9 @@ int swarm_local_steps_geometric(swarm_ctx *ctx, const int32_t *node_ids_host, in
                                 int32_t *out_steps_host);
 
 /* Algorithm 1, interaction lines; Corollary 1 for Enc/Dec. `pairs_host` holds npairs disjoint
- * directed edges of G. bits in {2, 4, 8}: lattice quantizer with that many bits per
- * coordinate; bits = 32 (blocking only): identity quantizer (Corollary 2).
+ * directed edges of G. bits in {2, ..., 8}: lattice quantizer with that many bits per
+ * coordinate (one bit leaves no decoding window: L = 2^(b-1) - 1 = 0); bits = 32 (blocking only):
+ * identity quantizer (Corollary 2).
  *   SWARM_BLOCKING: per 1024-block the common exponent e is taken from the exact range of
  *     X^a - X^b; both models are encoded into their own buffers, each side decodes the
  *     partner's buffer with its own model as key, and both adopt Q(X^a)/2 + Q(X^b)/2.

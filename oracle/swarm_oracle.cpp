@@ -197,19 +197,21 @@ uint32_t sr_uniform(const Rng& rng, uint32_t owner, uint32_t w, int64_t k) {
   return (k % 2 == 0) ? (word & 0xFFFFu) : (word >> 16);
 }
 
-// Little-endian packing inside a block: code of local coordinate k occupies bits
-// [(k mod (8/b)) * b, +b) of byte (k * b) div 8.
+// Packing inside a block: a little-endian bit stream, the code of local coordinate k occupies bits
+// [k*b, (k+1)*b) of the block's 128*b bytes (bit t of the stream is bit t mod 8 of byte t div 8).
 void put_code(uint8_t* block_bytes, int k, uint32_t c, int bits) {
-  const int per_byte = 8 / bits;
-  const int byte = (k * bits) / 8;
-  const int shift = (k % per_byte) * bits;
-  block_bytes[byte] = (uint8_t)(block_bytes[byte] | (c << shift));
+  for (int t = 0; t < bits; ++t) {
+    const int pos = k * bits + t;
+    if ((c >> t) & 1u) block_bytes[pos / 8] = (uint8_t)(block_bytes[pos / 8] | (1u << (pos % 8)));
+  }
 }
 uint32_t get_code(const uint8_t* block_bytes, int k, int bits) {
-  const int per_byte = 8 / bits;
-  const int byte = (k * bits) / 8;
-  const int shift = (k % per_byte) * bits;
-  return (block_bytes[byte] >> shift) & ((1u << bits) - 1u);
+  uint32_t c = 0;
+  for (int t = 0; t < bits; ++t) {
+    const int pos = k * bits + t;
+    c |= (uint32_t)((block_bytes[pos / 8] >> (pos % 8)) & 1u) << t;
+  }
+  return c;
 }
 
 // ---------------------------------------------------------------------------
@@ -889,7 +891,7 @@ int orc_local_steps_geometric(void* h, const int32_t* nodes, int32_t count, int3
 int orc_interact(void* h, const int32_t* pairs, int32_t npairs, int32_t bits, int32_t mode, int32_t threads) {
   Swarm& s = *(Swarm*)h;
   if (npairs < 0 || mode < 0 || mode > 2) return -1;
-  if (!(bits == 2 || bits == 4 || bits == 8 || (bits == 32 && mode == 0))) return -1;
+  if (!((bits >= 2 && bits <= 8) || (bits == 32 && mode == 0))) return -1;
   if (mode == 1 && !s.cfg.nonblocking) return -4;
   if (mode == 2 && s.cfg.nonblocking != 2) return -4;
   if (mode == 0 && s.track) return -4;   // a blocking exchange has no outdated model to track
@@ -970,7 +972,7 @@ int orc_aux_potentials(void* h, double* out) {
 
 int orc_register_publish(void* h, int32_t bits) {
   Swarm& s = *(Swarm*)h;
-  if (s.cfg.nonblocking != 2 || !(bits == 2 || bits == 4 || bits == 8)) return -1;
+  if (s.cfg.nonblocking != 2 || (bits < 2 || bits > 8)) return -1;
   register_publish(s, bits);
   return 0;
 }
@@ -983,7 +985,7 @@ int32_t* orc_p_mode(void* h) { return &((Swarm*)h)->p_mode; }
 
 int orc_publish(void* h, int32_t bits) {
   Swarm& s = *(Swarm*)h;
-  if (!s.cfg.nonblocking || !(bits == 2 || bits == 4 || bits == 8)) return -1;
+  if (!s.cfg.nonblocking || (bits < 2 || bits > 8)) return -1;
   publish(s, bits);
   return 0;
 }

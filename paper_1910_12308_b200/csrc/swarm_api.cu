@@ -649,7 +649,7 @@ int swarm_local_steps_geometric(swarm_ctx* c, const int32_t* node_ids, int32_t c
 int swarm_interact(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, int32_t bits, int32_t mode) {
   if (!c || npairs < 0 || (npairs > 0 && !pairs)) return SWARM_EINVAL;
   if (mode != SWARM_BLOCKING && mode != SWARM_NONBLOCKING && mode != SWARM_REGISTERS) return SWARM_EINVAL;
-  const bool quant = bits == 2 || bits == 4 || bits == 8;
+  const bool quant = bits >= 2 && bits <= 8;
   if (!(quant || (bits == 32 && mode == SWARM_BLOCKING))) return SWARM_EINVAL;
   if (mode == SWARM_NONBLOCKING && !c->cfg.nonblocking) return SWARM_ESTATE;
   if (mode == SWARM_REGISTERS && c->cfg.nonblocking != 2) return SWARM_ESTATE;
@@ -768,7 +768,7 @@ int swarm_aux_potentials(swarm_ctx* c, double* out3) {
 }
 
 int swarm_register_publish(swarm_ctx* c, int32_t bits) {
-  if (!c || !(bits == 2 || bits == 4 || bits == 8)) return SWARM_EINVAL;
+  if (!c || (bits < 2 || bits > 8)) return SWARM_EINVAL;
   if (c->cfg.nonblocking != 2) return SWARM_ESTATE;
   DeviceGuard guard(c->device);
   return do_register_publish(c, bits);
@@ -786,7 +786,7 @@ int swarm_set_buffer_mode(swarm_ctx* c, int32_t mode) {
 }
 
 int swarm_publish(swarm_ctx* c, int32_t bits) {
-  if (!c || !(bits == 2 || bits == 4 || bits == 8)) return SWARM_EINVAL;
+  if (!c || (bits < 2 || bits > 8)) return SWARM_EINVAL;
   if (!c->cfg.nonblocking) return SWARM_ESTATE;
   DeviceGuard guard(c->device);
   return do_publish(c, bits);
@@ -895,7 +895,7 @@ static int tensor_access(swarm_ctx* c, int32_t which, int32_t node, void* host, 
       if (bytes != 12) return SWARM_EINVAL;
       uint32_t* v = (uint32_t*)host;
       if (write) {
-        if (!(v[2] == 0 || v[2] == 2 || v[2] == 4 || v[2] == 8)) return SWARM_EINVAL;
+        if (v[2] == 1 || v[2] > 8) return SWARM_EINVAL;
         c->w[node] = v[0]; c->ls[node] = v[1]; c->pbits[node] = (int32_t)v[2];
       } else {
         v[0] = c->w[node]; v[1] = c->ls[node]; v[2] = (uint32_t)c->pbits[node];

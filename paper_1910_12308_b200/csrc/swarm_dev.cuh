@@ -207,18 +207,45 @@ __device__ __forceinline__ void st256(float* p, const f8& r) {
                : "memory");
 }
 
-// Eight packed codes of one lane: BITS bytes at `p` (aligned to BITS bytes).
+// Eight packed codes of one lane: BITS bytes at `p` = (the warp's 32*BITS-byte run) + lane*BITS. A block's
+// codes are a little-endian bit stream (code of local coordinate k at bits [k*BITS, (k+1)*BITS)), so a lane's
+// 8 coordinates always fill whole bytes. Widths 2, 4, 8 give naturally aligned 2-, 4-, 8-byte accesses.
+// Widths 3, 5, 6, 7 are called by all 32 lanes together: the store regroups the run into aligned 32-bit
+// words through shuffles (each word takes bytes from at most two neighbouring lanes); the load reads the two
+// aligned 8-byte words that cover the lane's bytes (rows keep >= 128 spare bytes behind the last run).
 template <int BITS>
-__device__ __forceinline__ void store_codes(uint8_t* p, uint64_t packed) {
+__device__ __forceinline__ void store_codes(uint8_t* p, int lane, uint64_t packed) {
   if constexpr (BITS == 8) *reinterpret_cast<uint2*>(p) = make_uint2((uint32_t)packed, (uint32_t)(packed >> 32));
   else if constexpr (BITS == 4) *reinterpret_cast<uint32_t*>(p) = (uint32_t)packed;
-  else *reinterpret_cast<uint16_t*>(p) = (uint16_t)packed;
+  else if constexpr (BITS == 2) *reinterpret_cast<uint16_t*>(p) = (uint16_t)packed;
+  else {
+    uint32_t* run = reinterpret_cast<uint32_t*>(p - lane * BITS);
+    constexpr int kWords = 8 * BITS;                 // 32-bit words in the run
+#pragma unroll
+    for (int r = 0; r < (kWords + 31) / 32; ++r) {
+      const int w = r * 32 + lane;
+      const int src = (4 * w) / BITS;                // lane holding the word's first byte
+      const int off = 4 * w - src * BITS;            // ... at this byte of its BITS bytes
+      const uint64_t p0 = __shfl_sync(0xFFFFFFFFu, packed, min(src, 31));
+      const uint64_t p1 = __shfl_sync(0xFFFFFFFFu, packed, min(src + 1, 31));
+      const uint64_t both = (p0 >> (8 * off)) | (p1 << (8 * (BITS - off)));
+      if (w < kWords) run[w] = (uint32_t)both;
+    }
+  }
 }
 template <int BITS>
 __device__ __forceinline__ uint64_t load_codes(const uint8_t* p) {
   if constexpr (BITS == 8) { const uint2 v = *reinterpret_cast<const uint2*>(p); return (uint64_t)v.x | ((uint64_t)v.y << 32); }
   else if constexpr (BITS == 4) return *reinterpret_cast<const uint32_t*>(p);
-  else return *reinterpret_cast<const uint16_t*>(p);
+  else if constexpr (BITS == 2) return *reinterpret_cast<const uint16_t*>(p);
+  else {
+    const uintptr_t addr = reinterpret_cast<uintptr_t>(p);
+    const uint64_t* q = reinterpret_cast<const uint64_t*>(addr & ~(uintptr_t)7);
+    const int sh = (int)(addr & 7) * 8;
+    const uint64_t lo = q[0], hi = q[1];
+    const uint64_t v = sh ? ((lo >> sh) | (hi << (64 - sh))) : lo;
+    return v & ((1ull << (8 * BITS)) - 1ull);
+  }
 }
 
 // Warp-wide maximum of non-negative floats (bit pattern order equals value order).

@@ -107,8 +107,8 @@ interact_blocking_kernel(StoreView s, const PairList pairs, int64_t total_warps)
     }
     st256(xa + j * kSubCoords, out);
     st256(xb + j * kSubCoords, out);
-    store_codes<BITS>(ca + j * (kSubCoords * BITS / 8), pka);
-    store_codes<BITS>(cb + j * (kSubCoords * BITS / 8), pkb);
+    store_codes<BITS>(ca + j * (kSubCoords * BITS / 8), lane, pka);
+    store_codes<BITS>(cb + j * (kSubCoords * BITS / 8), lane, pkb);
   }
   if (lane == 0) {
     s.exps[(int64_t)pd.a * s.nblk + blk] = (int8_t)e;
@@ -238,8 +238,8 @@ interact_nonblocking_kernel(StoreView s, const PairList pairs, int64_t total_war
     }
     st256(xa + j * kSubCoords, nx[j]);
     st256(ba + j * kSubCoords, nx[j]);
-    store_codes<BITS>(ca + j * (kSubCoords * BITS / 8), pka);
-    store_codes<BITS>(cb + j * (kSubCoords * BITS / 8), pkb);
+    store_codes<BITS>(ca + j * (kSubCoords * BITS / 8), lane, pka);
+    store_codes<BITS>(cb + j * (kSubCoords * BITS / 8), lane, pkb);
   }
   if (lane == 0) { *ea_p = (int8_t)e; *eb_p = (int8_t)e; }
 }
@@ -311,7 +311,7 @@ publish_encode_kernel(StoreView s, const uint32_t* __restrict__ wctr, int64_t to
       int32_t cell;
       pk |= (uint64_t)((uint32_t)encode_index(v[j].v[i], inv_step, sr_u16(r, i), cell) & mask) << (i * BITS);
     }
-    store_codes<BITS>(c + j * (kSubCoords * BITS / 8), pk);
+    store_codes<BITS>(c + j * (kSubCoords * BITS / 8), lane, pk);
   }
 }
 
@@ -445,7 +445,7 @@ interact_registers_kernel(StoreView s, const PairList pairs, int64_t total_warps
       pkb |= (uint64_t)((uint32_t)encode_index(av[j].v[i], ipb_new, sr_u16(rb, i), cell) & mask) << (i * BITS);
     }
     *reinterpret_cast<uint4*>(oa + j * kSubCoords) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
-    store_codes<BITS>(cb + j * (kSubCoords * BITS / 8), pkb);
+    store_codes<BITS>(cb + j * (kSubCoords * BITS / 8), lane, pkb);
   }
   rho_a = warp_max_nonneg(rho_a);
   M_a = warp_max_nonneg(M_a);
@@ -463,7 +463,7 @@ interact_registers_kernel(StoreView s, const PairList pairs, int64_t total_warps
     }
     st256(xa + j * kSubCoords, nx[j]);
     st256(ba + j * kSubCoords, nx[j]);
-    store_codes<BITS>(ca + j * (kSubCoords * BITS / 8), pka);
+    store_codes<BITS>(ca + j * (kSubCoords * BITS / 8), lane, pka);
   }
   if (lane == 0) {
     s.oexps[(int64_t)pd.a * s.nblk + blk] = (int8_t)eo;
@@ -523,7 +523,7 @@ register_publish_encode_kernel(StoreView s, const uint32_t* __restrict__ wctr, i
       int32_t cell;
       pk |= (uint64_t)((uint32_t)encode_index(v[j].v[i], ip, sr_u16(r, i), cell) & mask) << (i * BITS);
     }
-    store_codes<BITS>(c + j * (kSubCoords * BITS / 8), pk);
+    store_codes<BITS>(c + j * (kSubCoords * BITS / 8), lane, pk);
   }
   if (lane == 0) s.exps[node * s.nblk + blk] = (int8_t)ep;
 }
@@ -532,6 +532,16 @@ register_publish_encode_kernel(StoreView s, const uint32_t* __restrict__ wctr, i
 // Launch wrappers
 // -----------------------------------------------------------------------------------------
 static inline unsigned ctas_for(int64_t warps) { return (unsigned)((warps + kWarpsPerCta - 1) / kWarpsPerCta); }
+
+// Code widths with a compiled kernel: SWARM_FOR_WIDTH(bits, BODY) runs BODY with the constant W = bits.
+#define SWARM_WIDTH_CASE(w, ...) case w: { constexpr int W = w; __VA_ARGS__; } break;
+#define SWARM_FOR_WIDTH(bits, ...)                                                          \
+  switch (bits) {                                                                           \
+    SWARM_WIDTH_CASE(2, __VA_ARGS__) SWARM_WIDTH_CASE(3, __VA_ARGS__) SWARM_WIDTH_CASE(4, __VA_ARGS__) \
+    SWARM_WIDTH_CASE(5, __VA_ARGS__) SWARM_WIDTH_CASE(6, __VA_ARGS__) SWARM_WIDTH_CASE(7, __VA_ARGS__) \
+    SWARM_WIDTH_CASE(8, __VA_ARGS__)                                                        \
+    default: return cudaErrorInvalidValue;                                                  \
+  }
 
 template <typename Kernel>
 static cudaError_t launch_dependent(Kernel kernel, dim3 grid, dim3 block, cudaStream_t st, const StoreView& s,
@@ -555,12 +565,10 @@ cudaError_t launch_interact_blocking(const StoreView& s, const PairList& pairs, 
   const int64_t warps = (int64_t)npairs * s.nblk;
   const dim3 grid(ctas_for(warps)), block(kWarpsPerCta * 32);
   cudaError_t e = cudaSuccess;
-  switch (bits) {
-    case 2: e = launch_dependent(interact_blocking_kernel<2>, grid, block, st, s, pairs, warps); break;
-    case 4: e = launch_dependent(interact_blocking_kernel<4>, grid, block, st, s, pairs, warps); break;
-    case 8: e = launch_dependent(interact_blocking_kernel<8>, grid, block, st, s, pairs, warps); break;
-    case 32: interact_identity_kernel<<<grid, block, 0, st>>>(s, pairs, warps); break;
-    default: return cudaErrorInvalidValue;
+  if (bits == 32) {
+    interact_identity_kernel<<<grid, block, 0, st>>>(s, pairs, warps);
+  } else {
+    SWARM_FOR_WIDTH(bits, e = launch_dependent(interact_blocking_kernel<W>, grid, block, st, s, pairs, warps))
   }
   ++*launches;
   return e != cudaSuccess ? e : cudaGetLastError();
@@ -572,12 +580,7 @@ cudaError_t launch_interact_nonblocking(const StoreView& s, const PairList& pair
   const int64_t warps = (int64_t)npairs * s.nblk;
   const dim3 grid(ctas_for(warps)), block(kWarpsPerCta * 32);
   cudaError_t e = cudaSuccess;
-  switch (bits) {
-    case 2: e = launch_dependent(interact_nonblocking_kernel<2>, grid, block, st, s, pairs, warps); break;
-    case 4: e = launch_dependent(interact_nonblocking_kernel<4>, grid, block, st, s, pairs, warps); break;
-    case 8: e = launch_dependent(interact_nonblocking_kernel<8>, grid, block, st, s, pairs, warps); break;
-    default: return cudaErrorInvalidValue;
-  }
+  SWARM_FOR_WIDTH(bits, e = launch_dependent(interact_nonblocking_kernel<W>, grid, block, st, s, pairs, warps))
   ++*launches;
   return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -587,21 +590,8 @@ cudaError_t launch_publish(const StoreView& s, const uint32_t* wctr_dev, int bit
   const dim3 grid_r(ctas_for(s.nblk));
   const int64_t warps = (int64_t)s.n * s.nblk;
   const dim3 grid_e(ctas_for(warps));
-  switch (bits) {
-    case 2:
-      publish_range_kernel<2><<<grid_r, block, 0, st>>>(s, s.exps);
-      publish_encode_kernel<2><<<grid_e, block, 0, st>>>(s, wctr_dev, warps);
-      break;
-    case 4:
-      publish_range_kernel<4><<<grid_r, block, 0, st>>>(s, s.exps);
-      publish_encode_kernel<4><<<grid_e, block, 0, st>>>(s, wctr_dev, warps);
-      break;
-    case 8:
-      publish_range_kernel<8><<<grid_r, block, 0, st>>>(s, s.exps);
-      publish_encode_kernel<8><<<grid_e, block, 0, st>>>(s, wctr_dev, warps);
-      break;
-    default: return cudaErrorInvalidValue;
-  }
+  SWARM_FOR_WIDTH(bits, publish_range_kernel<W><<<grid_r, block, 0, st>>>(s, s.exps);
+                        publish_encode_kernel<W><<<grid_e, block, 0, st>>>(s, wctr_dev, warps))
   *launches += 2;
   return cudaGetLastError();
 }
@@ -612,12 +602,7 @@ cudaError_t launch_interact_registers(const StoreView& s, const PairList& pairs,
   const int64_t warps = (int64_t)npairs * s.nblk;
   const dim3 grid(ctas_for(warps)), block(kWarpsPerCta * 32);
   cudaError_t e = cudaSuccess;
-  switch (bits) {
-    case 2: e = launch_dependent(interact_registers_kernel<2>, grid, block, st, s, pairs, warps); break;
-    case 4: e = launch_dependent(interact_registers_kernel<4>, grid, block, st, s, pairs, warps); break;
-    case 8: e = launch_dependent(interact_registers_kernel<8>, grid, block, st, s, pairs, warps); break;
-    default: return cudaErrorInvalidValue;
-  }
+  SWARM_FOR_WIDTH(bits, e = launch_dependent(interact_registers_kernel<W>, grid, block, st, s, pairs, warps))
   ++*launches;
   return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -630,12 +615,7 @@ cudaError_t launch_register_publish(const StoreView& s, const uint32_t* wctr_dev
   const dim3 grid_e(ctas_for(warps));
   // the own registers of a block share the step of an 8-bit code of the spread of all snapshots
   publish_range_kernel<kOwnResolutionBits><<<grid_r, block, 0, st>>>(s, s.oexps);
-  switch (bits) {
-    case 2: register_publish_encode_kernel<2><<<grid_e, block, 0, st>>>(s, wctr_dev, warps); break;
-    case 4: register_publish_encode_kernel<4><<<grid_e, block, 0, st>>>(s, wctr_dev, warps); break;
-    case 8: register_publish_encode_kernel<8><<<grid_e, block, 0, st>>>(s, wctr_dev, warps); break;
-    default: return cudaErrorInvalidValue;
-  }
+  SWARM_FOR_WIDTH(bits, register_publish_encode_kernel<W><<<grid_e, block, 0, st>>>(s, wctr_dev, warps))
   *launches += 2;
   return cudaGetLastError();
 }

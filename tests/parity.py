@@ -65,7 +65,7 @@ def assert_store_equal(orc, gpu, bits=None, nodes=None, check_B=True):
         if orc.own is not None and int(orc.p_mode[0]) == 2:
             assert np.array_equal(gpu.get(g.T_OWN, i), orc.own[i]), f"own register[{i}] differs"
             assert np.array_equal(gpu.get(g.T_OEXPS, i), orc.oexps[i]), f"own exponents[{i}] differ"
-        if bits in (2, 4, 8) and orc.pbits[i] == bits:
+        if bits is not None and 2 <= bits <= 8 and orc.pbits[i] == bits:
             nbytes = orc.nblk * 128 * bits
             assert np.array_equal(gpu.get(g.T_CODES, i)[:nbytes], orc.codes[i, :nbytes]), f"codes[{i}] differ"
             assert np.array_equal(gpu.get(g.T_EXPS, i), orc.exps[i]), f"exps[{i}] differ"

@@ -81,7 +81,7 @@ def test_pair_schedule_is_bit_exact(topo, deg, n, P):
 
 # ---- blocking interaction ------------------------------------------------------------------------
 
-@pytest.mark.parametrize("bits", [2, 4, 8, 32])
+@pytest.mark.parametrize("bits", [2, 3, 4, 5, 6, 7, 8, 32])
 @pytest.mark.parametrize("d", [1, 7, 1024, 1030, 2049, 5000])
 def test_blocking_interaction_bit_exact(bits, d):
     n = 6
@@ -95,7 +95,7 @@ def test_blocking_interaction_bit_exact(bits, d):
         assert_store_equal(orc, gpu, bits)
 
 
-@pytest.mark.parametrize("bits", [2, 4, 8])
+@pytest.mark.parametrize("bits", [2, 3, 4, 5, 6, 7, 8])
 def test_blocking_interaction_special_values(bits):
     """Identical models, zeros, huge and tiny magnitudes, and widely separated models."""
     n, d = 4, 3000
@@ -135,7 +135,7 @@ def test_blocking_interaction_on_ring_and_many_rounds():
 
 # ---- non-blocking interaction --------------------------------------------------------------------
 
-@pytest.mark.parametrize("bits", [2, 4, 8])
+@pytest.mark.parametrize("bits", [2, 3, 4, 5, 6, 7, 8])
 @pytest.mark.parametrize("d", [5, 1024, 3001])
 def test_publish_and_nonblocking_interaction_bit_exact(bits, d):
     n = 6
@@ -188,7 +188,7 @@ def test_nonblocking_far_key_alias_matches():
 
 # ---- two-register protocol -----------------------------------------------------------------------
 
-@pytest.mark.parametrize("bits", [2, 4, 8])
+@pytest.mark.parametrize("bits", [2, 3, 4, 5, 6, 7, 8])
 @pytest.mark.parametrize("d", [5, 1024, 3001])
 def test_register_protocol_bit_exact(bits, d):
     n = 6
@@ -371,7 +371,7 @@ def test_rejected_calls_change_nothing():
     assert gpu.interact([[0, 0]], 8) == -3
     assert gpu.interact([[0, 3]], 8) == -3
     assert gpu.interact([[0, 6]], 8) == -2
-    assert gpu.interact([[0, 1]], 3) == -1
+    assert gpu.interact([[0, 1]], 1) == -1 and gpu.interact([[0, 1]], 9) == -1 and gpu.interact([[0, 1]], 16) == -1
     assert gpu.interact([[0, 1]], 8, 3) == -1
     assert gpu.interact([[0, 1]], 8, g.REGISTERS) == -4
     assert gpu.interact([[0, 1]], 32, g.NONBLOCKING) == -1

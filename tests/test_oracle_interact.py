@@ -46,7 +46,7 @@ def test_exact_averaging_preserves_mean_and_drops_gamma(n):
         assert s.potential() == 0.0
 
 
-@pytest.mark.parametrize("bits", [2, 4, 8])
+@pytest.mark.parametrize("bits", [2, 3, 4, 5, 7, 8])
 def test_quantized_interaction_satisfies_the_gamma_change_identity(bits):
     """Delta = -||Xi-Xj||^2/2 + <Xi-mu + Xj-mu, Si+Sj> + (n-2)/n^2 ||Si+Sj||^2
                + ||(n-1)/n Si - Sj/n||^2 + ||(n-1)/n Sj - Si/n||^2,   Si = Sj = X' - (Xi+Xj)/2."""
@@ -138,7 +138,8 @@ def test_pair_validation():
     assert s.interact([[0, 0]], 8) == -3
     assert s.interact([[0, 3]], 8) == -3              # not adjacent on the ring
     assert s.interact([[0, 6]], 8) == -2
-    assert s.interact([[0, 1]], 3) == -1
+    assert s.interact([[0, 1]], 1) == -1             # one bit leaves no decoding window (L = 0)
+    assert s.interact([[0, 1]], 9) == -1 and s.interact([[0, 1]], 16) == -1
     assert s.interact([[0, 1]], 8, o.NONBLOCKING) == -4
 
 
@@ -150,7 +151,7 @@ def make_nb(n=4, d=2100, bits=8, seed=1, topo="complete"):
     return s
 
 
-@pytest.mark.parametrize("bits", [2, 4, 8])
+@pytest.mark.parametrize("bits", [2, 3, 4, 5, 7, 8])
 def test_publish_encodes_base_with_the_spread_of_all_bases(bits):
     s = make_nb(bits=bits)
     assert np.array_equal(s.B, s.X)

@@ -7,7 +7,7 @@ import pytest
 
 from oracle import swarm_oracle as o
 
-BITS = (2, 4, 8)
+BITS = (2, 3, 4, 5, 6, 7, 8)
 
 
 def L_of(b):

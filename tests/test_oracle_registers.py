@@ -36,7 +36,7 @@ def steps(exps, d):
     return np.repeat(2.0 ** exps.astype(np.float64), 1024)[:d]
 
 
-@pytest.mark.parametrize("bits", [2, 4, 8])
+@pytest.mark.parametrize("bits", [2, 3, 4, 6, 8])
 def test_register_publish_chain_decodes_every_snapshot(bits):
     s = make(offset_std=0.3)
     assert s.register_publish(bits) == 0
