@@ -321,7 +321,14 @@ def run_ours(args, wl, name):
     launches = [sched.next() for _ in range(K + W)]
     npairs_total = sum(len(p) for p in launches[W:])
 
+    # elementwise (synthetic) objective, on request: the nodes of the pairs step inside the interaction kernel
+    fused = (wl["H"] > 0 and wl["cfg"].get("objective") == 1 and not wl.get("step_all") and args.fused)
+
     def step(pairs):
+        if fused:
+            rc = sw.step(pairs, wl["H"], wl["lr"], wl["bits"], wl["mode"], True)
+            assert rc == 0, rc
+            return
         if wl["H"] > 0:
             rc = sw.local_steps(stepping_nodes(wl, pairs), wl["H"], wl["lr"])
             assert rc == 0, rc
@@ -345,7 +352,7 @@ def run_ours(args, wl, name):
     H, lr, bits, mode = wl["H"], wl["lr"], wl["bits"], wl["mode"]
     probe_every = 8                       # the interaction kernel is bracketed by events on every 8th step
     probes = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-              for _ in range(0, K, probe_every)] if H > 0 else []
+              for _ in range(0, K, probe_every)] if (H > 0 and not fused) else []
     # ---- device-resident timing
     for pairs in launches[:W]:
         step(pairs)
@@ -358,7 +365,9 @@ def run_ours(args, wl, name):
     ok = 0
     ev0.record(stream)
     for i, (_, pp, npp, _, nn, ncount) in enumerate(calls):
-        if H > 0:
+        if fused:
+            ok |= L.swarm_step(h, pp, npp, H, lr, bits, mode, 1)
+        elif H > 0:
             ok |= L.swarm_local_steps(h, nn, ncount, H, lr)
             if i % probe_every == 0:
                 e_a, e_b = probes[i // probe_every]
@@ -385,6 +394,8 @@ def run_ours(args, wl, name):
     else:
         kern_ms = ms_local / K
     per_launch_bytes = interaction_bytes(wl["d"], wl["bits"], wl["mode"]) * npairs_total / K
+    if fused and wl["mode"] != 0:
+        per_launch_bytes += 8 * wl["d"] * npairs_total / K      # the responder's model is read and written too
     achieved = per_launch_bytes / (kern_ms * 1e-3) / 1e9
     peak, peak_kind = measured_peak()
 
@@ -421,10 +432,12 @@ def run_ours(args, wl, name):
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
         "config": {"workload": name, **{k: wl[k] for k in ("n", "d", "topology", "pairs", "bits", "mode", "H")},
+                   "fused_local_steps": bool(fused),
                    "l2": "inputs larger than L2: every launch streams all models it touches from HBM",
                    "replicas": world},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(gpu_launches),
-        "roofline": {"bound": "hbm", "kernel": ["interact_blocking_kernel", "interact_nonblocking_kernel", "interact_registers_kernel"][wl["mode"]],
+        "roofline": {"bound": "hbm", "kernel": ["interact_blocking_kernel", "interact_nonblocking_kernel", "interact_registers_kernel"][wl["mode"]]
+                     + (" (local steps fused)" if fused else ""),
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": peak_kind, "frac_of_8000": achieved / 8000.0, "traffic": TRAFFIC.get(name),
                      "algorithmic_bytes_per_launch": per_launch_bytes, "kernel_ms": kern_ms},
@@ -474,6 +487,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--fused", action="store_true",
+                    help="synthetic-objective workloads: one swarm_step call per step (local steps inside the "
+                         "interaction kernel) instead of swarm_local_steps + swarm_interact; measured slower, "
+                         "because the step is bound by instruction issue, not by HBM")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

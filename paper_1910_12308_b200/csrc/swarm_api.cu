@@ -646,7 +646,10 @@ int swarm_local_steps_geometric(swarm_ctx* c, const int32_t* node_ids, int32_t c
   return SWARM_OK;
 }
 
-int swarm_interact(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, int32_t bits, int32_t mode) {
+// One interaction launch; fused_H > 0 runs that many synthetic-gradient local steps of the initiators (and of
+// the responders when `responders` is set) inside the interaction kernel first.
+static int interact_impl(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, int32_t bits, int32_t mode,
+                         int32_t fused_H, float lr, int32_t responders) {
   if (!c || npairs < 0 || (npairs > 0 && !pairs)) return SWARM_EINVAL;
   if (mode != SWARM_BLOCKING && mode != SWARM_NONBLOCKING && mode != SWARM_REGISTERS) return SWARM_EINVAL;
   const bool quant = bits >= 2 && bits <= 8;
@@ -682,15 +685,22 @@ int swarm_interact(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, int32_
     pd[p].a = pairs[p].a; pd[p].b = pairs[p].b;
     pd[p].wa = c->w[pairs[p].a]; pd[p].wb = c->w[pairs[p].b];
     pd[p].woa = c->wo[pairs[p].a]; pd[p].pad = 0;
+    pd[p].lsa = c->ls[pairs[p].a]; pd[p].lsb = c->ls[pairs[p].b];
   }
+  FusedSteps fs{};
+  fs.H = fused_H; fs.responders = responders ? 1 : 0; fs.lr = lr; fs.grad_std = c->cfg.grad_std; fs.scalars = c->scalars;
   if (slot >= 0) {
     rc = stage_commit(c, slot, (size_t)npairs * sizeof(PairDesc));
     if (rc != SWARM_OK) return rc;
   }
   int nl = 0;
-  if (mode == SWARM_BLOCKING) SW_CUDA(c, launch_interact_blocking(view_of(c), list, npairs, bits, c->stream, &nl));
-  else if (mode == SWARM_NONBLOCKING) SW_CUDA(c, launch_interact_nonblocking(view_of(c), list, npairs, bits, c->stream, &nl));
-  else SW_CUDA(c, launch_interact_registers(view_of(c), list, npairs, bits, c->stream, &nl));
+  if (mode == SWARM_BLOCKING) SW_CUDA(c, launch_interact_blocking(view_of(c), list, npairs, bits, fs, c->stream, &nl));
+  else if (mode == SWARM_NONBLOCKING) SW_CUDA(c, launch_interact_nonblocking(view_of(c), list, npairs, bits, fs, c->stream, &nl));
+  else SW_CUDA(c, launch_interact_registers(view_of(c), list, npairs, bits, fs, c->stream, &nl));
+  for (int p = 0; p < npairs && fused_H > 0; ++p) {
+    c->ls[pairs[p].a] += (uint32_t)fused_H;
+    if (responders) c->ls[pairs[p].b] += (uint32_t)fused_H;
+  }
   c->launches += nl;
   if (slot >= 0) {
     rc = stage_release(c, slot);
@@ -718,6 +728,41 @@ int swarm_interact(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, int32_
     if (rc != SWARM_OK) return rc;
   }
   return SWARM_OK;
+}
+
+int swarm_interact(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, int32_t bits, int32_t mode) {
+  return interact_impl(c, pairs, npairs, bits, mode, 0, 0.0f, 0);
+}
+
+int swarm_step(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, int32_t H, float lr, int32_t bits, int32_t mode,
+               int32_t step_responders) {
+  if (!c || H < 0 || npairs < 0 || (npairs > 0 && !pairs)) return SWARM_EINVAL;
+  if (H == 0) return interact_impl(c, pairs, npairs, bits, mode, 0, 0.0f, 0);
+  if (c->cfg.objective == SWARM_OBJ_NONE) return SWARM_ESTATE;
+  // Elementwise objective: the steps run inside the interaction kernel. A publish that the interaction
+  // triggers runs before the fused steps; that is the same as after them unless it first refreshes stale
+  // snapshots from the models, so that one case takes the two-call route.
+  if (c->cfg.objective == SWARM_OBJ_SYNTH && !(mode != SWARM_BLOCKING && c->b_stale))
+    return interact_impl(c, pairs, npairs, bits, mode, H, lr, step_responders);
+  // objectives whose gradient couples all coordinates: the two calls in sequence, after the checks that
+  // the interaction would make (so that a refused call leaves the models untouched)
+  if (mode != SWARM_BLOCKING && mode != SWARM_NONBLOCKING && mode != SWARM_REGISTERS) return SWARM_EINVAL;
+  if (!((bits >= 2 && bits <= 8) || (bits == 32 && mode == SWARM_BLOCKING))) return SWARM_EINVAL;
+  if (mode == SWARM_NONBLOCKING && !c->cfg.nonblocking) return SWARM_ESTATE;
+  if (mode == SWARM_REGISTERS && c->cfg.nonblocking != 2) return SWARM_ESTATE;
+  if (mode == SWARM_BLOCKING && c->track) return SWARM_ESTATE;
+  if (npairs > c->n / 2) return SWARM_EPAIR;
+  int rc = validate_pairs(c, pairs, npairs);
+  if (rc != SWARM_OK) return rc;
+  std::vector<int32_t> nodes;
+  nodes.reserve((size_t)npairs * 2);
+  for (int p = 0; p < npairs; ++p) {
+    nodes.push_back(pairs[p].a);
+    if (step_responders) nodes.push_back(pairs[p].b);
+  }
+  rc = swarm_local_steps(c, nodes.data(), (int32_t)nodes.size(), H, lr);
+  if (rc != SWARM_OK) return rc;
+  return interact_impl(c, pairs, npairs, bits, mode, 0, 0.0f, 0);
 }
 
 int swarm_track_staleness(swarm_ctx* c, int32_t enable) {

@@ -207,6 +207,21 @@ __device__ __forceinline__ void st256(float* p, const f8& r) {
                : "memory");
 }
 
+// One synthetic-gradient local step x <- x - lr * (c + grad_std * z) on the 8 consecutive coordinates of
+// coordinate group g8 (first coordinate / 8): two generator calls, every operation rounded on its own.
+// The one definition serves the stand-alone local-step kernel and the steps fused into an interaction.
+__device__ __forceinline__ void synth_step8(f8& v, uint32_t g8, uint32_t node, uint32_t event, float lr,
+                                            float grad_std, float c, const PhiloxRoundKeys& rk) {
+  float z[8];
+  normal4_fast(2u * g8, node, event, kStreamSynthGrad, rk, z);
+  normal4_fast(2u * g8 + 1u, node, event, kStreamSynthGrad, rk, z + 4);
+#pragma unroll
+  for (int t = 0; t < 8; ++t) {
+    const float grad = __fadd_rn(c, __fmul_rn(grad_std, z[t]));
+    v.v[t] = __fsub_rn(v.v[t], __fmul_rn(lr, grad));
+  }
+}
+
 // Eight packed codes of one lane: BITS bytes at `p` = (the warp's 32*BITS-byte run) + lane*BITS. A block's
 // codes are a little-endian bit stream (code of local coordinate k at bits [k*BITS, (k+1)*BITS)), so a lane's
 // 8 coordinates always fill whole bytes. Widths 2, 4, 8 give naturally aligned 2-, 4-, 8-byte accesses.

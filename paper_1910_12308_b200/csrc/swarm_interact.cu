@@ -31,15 +31,48 @@ __device__ __forceinline__ void grid_dependency_signal() { asm volatile("griddep
 constexpr int kSub = 4;          // sub-blocks per block
 constexpr int kSubCoords = 256;  // coordinates per sub-block
 
+// Local steps fused into an interaction (synthetic objective): H steps on the lane's 4 x 8 coordinates of
+// block blk of `node`, then the padding behind coordinate d of the last block is put back to zero.
+__device__ __forceinline__ void fused_steps_block(f8 (&v)[kSub], const StoreView& s, const FusedSteps& fs, int node,
+                                                  uint32_t event, int64_t blk, int lane) {
+  const float c = fs.scalars[node * 3 + 1];
+  const PhiloxRoundKeys rk = philox_round_keys(s.key0, s.key1);
+  const uint32_t g0 = (uint32_t)(blk * (kBlockCoords / 8) + lane);
+  for (int q = 0; q < fs.H; ++q) {
+#pragma unroll
+    for (int j = 0; j < kSub; ++j)
+      synth_step8(v[j], g0 + j * (kSubCoords / 8), (uint32_t)node, event + (uint32_t)q, fs.lr, fs.grad_std, c, rk);
+  }
+  if (blk == s.nblk - 1) {
+#pragma unroll
+    for (int j = 0; j < kSub; ++j)
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        if (blk * kBlockCoords + j * kSubCoords + lane * 8 + i >= s.d) v[j].v[i] = 0.0f;
+  }
+}
+
+// The responder's local steps when the interaction itself does not touch its model.
+__device__ __forceinline__ void fused_steps_responder(const StoreView& s, const FusedSteps& fs, const PairDesc& pd,
+                                                      int64_t blk, int lane) {
+  float* xb = s.X + (int64_t)pd.b * s.pitch + blk * kBlockCoords + lane * 8;
+  f8 vb[kSub];
+#pragma unroll
+  for (int j = 0; j < kSub; ++j) vb[j] = ld256(xb + j * kSubCoords);
+  fused_steps_block(vb, s, fs, pd.b, pd.lsb, blk, lane);
+#pragma unroll
+  for (int j = 0; j < kSub; ++j) st256(xb + j * kSubCoords, vb[j]);
+}
+
 // -----------------------------------------------------------------------------------------
 // Blocking interaction: both models are present. Per block: exact range of X^a - X^b gives
 // the common exponent; both are encoded into their buffers; each side decodes the partner's
 // codes against its own model and both adopt Q(X^a)/2 + Q(X^b)/2.
 // Traffic per coordinate: 8 B read, 8 B written, 2*b/8 B of codes written.
 // -----------------------------------------------------------------------------------------
-template <int BITS>
-__global__ void __launch_bounds__(kWarpsPerCta * 32)
-interact_blocking_kernel(StoreView s, const PairList pairs, int64_t total_warps) {
+template <int BITS, bool FUSED>
+__global__ void __launch_bounds__(kWarpsPerCta * 32, FUSED ? 4 : 1)
+interact_blocking_kernel(StoreView s, const PairList pairs, int64_t total_warps, const FusedSteps fs) {
   grid_dependency_signal();
   grid_dependency_wait();
   const int lane = threadIdx.x & 31;
@@ -66,6 +99,10 @@ interact_blocking_kernel(StoreView s, const PairList pairs, int64_t total_warps)
   for (int j = 0; j < kSub; ++j) va[j] = ld256(xa + j * kSubCoords);
 #pragma unroll
   for (int j = 0; j < kSub; ++j) vb[j] = ld256(xb + j * kSubCoords);
+  if constexpr (FUSED) {
+    fused_steps_block(va, s, fs, pd.a, pd.lsa, blk, lane);
+    if (fs.responders) fused_steps_block(vb, s, fs, pd.b, pd.lsb, blk, lane);
+  }
 
   float rho = 0.0f, M = 0.0f;
 #pragma unroll
@@ -118,7 +155,7 @@ interact_blocking_kernel(StoreView s, const PairList pairs, int64_t total_warps)
 
 // Identity quantizer (Corollary 2): plain averaging, buffers untouched.
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
-interact_identity_kernel(StoreView s, const PairList pairs, int64_t total_warps) {
+interact_identity_kernel(StoreView s, const PairList pairs, int64_t total_warps, const FusedSteps fs) {
   const int lane = threadIdx.x & 31;
   const int64_t warp = (int64_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
   if (warp >= total_warps) return;
@@ -132,6 +169,10 @@ interact_identity_kernel(StoreView s, const PairList pairs, int64_t total_warps)
   for (int j = 0; j < kSub; ++j) va[j] = ld256(xa + j * kSubCoords);
 #pragma unroll
   for (int j = 0; j < kSub; ++j) vb[j] = ld256(xb + j * kSubCoords);
+  if (fs.H > 0) {
+    fused_steps_block(va, s, fs, pd.a, pd.lsa, blk, lane);
+    if (fs.responders) fused_steps_block(vb, s, fs, pd.b, pd.lsb, blk, lane);
+  }
 #pragma unroll
   for (int j = 0; j < kSub; ++j) {
     f8 out;
@@ -151,9 +192,9 @@ interact_identity_kernel(StoreView s, const PairList pairs, int64_t total_warps)
 // rho' = 2 max|own - oth| + max|D| over the block.
 // Traffic per coordinate: 8 B + 2*b/8 B read, 8 B + 2*b/8 B written.
 // -----------------------------------------------------------------------------------------
-template <int BITS>
-__global__ void __launch_bounds__(kWarpsPerCta * 32)
-interact_nonblocking_kernel(StoreView s, const PairList pairs, int64_t total_warps) {
+template <int BITS, bool FUSED>
+__global__ void __launch_bounds__(kWarpsPerCta * 32, FUSED ? 4 : 1)
+interact_nonblocking_kernel(StoreView s, const PairList pairs, int64_t total_warps, const FusedSteps fs) {
   grid_dependency_signal();
   grid_dependency_wait();
   const int lane = threadIdx.x & 31;
@@ -187,6 +228,10 @@ interact_nonblocking_kernel(StoreView s, const PairList pairs, int64_t total_war
   uint64_t pa[kSub], pb[kSub];
 #pragma unroll
   for (int j = 0; j < kSub; ++j) nx[j] = ld256(xa + j * kSubCoords);
+  if constexpr (FUSED) {
+    if (fs.responders) fused_steps_responder(s, fs, pd, blk, lane);
+    fused_steps_block(nx, s, fs, pd.a, pd.lsa, blk, lane);
+  }
 #pragma unroll
   for (int j = 0; j < kSub; ++j) av[j] = ld256(ba + j * kSubCoords);
 #pragma unroll
@@ -336,9 +381,9 @@ __device__ __forceinline__ uint32_t own_code(const uint4& v, int i) {
   return (i & 1) ? (word >> 16) : (word & 0xFFFFu);
 }
 
-template <int BITS>
+template <int BITS, bool FUSED>
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
-interact_registers_kernel(StoreView s, const PairList pairs, int64_t total_warps) {
+interact_registers_kernel(StoreView s, const PairList pairs, int64_t total_warps, const FusedSteps fs) {
   grid_dependency_signal();
   grid_dependency_wait();
   const int lane = threadIdx.x & 31;
@@ -379,6 +424,10 @@ interact_registers_kernel(StoreView s, const PairList pairs, int64_t total_warps
   uint64_t pa[kSub], pb[kSub];
 #pragma unroll
   for (int j = 0; j < kSub; ++j) nx[j] = ld256(xa + j * kSubCoords);
+  if constexpr (FUSED) {
+    if (fs.responders) fused_steps_responder(s, fs, pd, blk, lane);
+    fused_steps_block(nx, s, fs, pd.a, pd.lsa, blk, lane);
+  }
 #pragma unroll
   for (int j = 0; j < kSub; ++j) av[j] = ld256(ba + j * kSubCoords);
 #pragma unroll
@@ -545,7 +594,7 @@ static inline unsigned ctas_for(int64_t warps) { return (unsigned)((warps + kWar
 
 template <typename Kernel>
 static cudaError_t launch_dependent(Kernel kernel, dim3 grid, dim3 block, cudaStream_t st, const StoreView& s,
-                                    const PairList& pairs, int64_t warps) {
+                                    const PairList& pairs, int64_t warps, const FusedSteps& fs) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
@@ -556,31 +605,33 @@ static cudaError_t launch_dependent(Kernel kernel, dim3 grid, dim3 block, cudaSt
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kernel, s, pairs, warps);
+  return cudaLaunchKernelEx(&cfg, kernel, s, pairs, warps, fs);
 }
 
 cudaError_t launch_interact_blocking(const StoreView& s, const PairList& pairs, int npairs, int bits,
-                                     cudaStream_t st, int* launches) {
+                                     const FusedSteps& fs, cudaStream_t st, int* launches) {
   if (npairs == 0) return cudaSuccess;
   const int64_t warps = (int64_t)npairs * s.nblk;
   const dim3 grid(ctas_for(warps)), block(kWarpsPerCta * 32);
   cudaError_t e = cudaSuccess;
   if (bits == 32) {
-    interact_identity_kernel<<<grid, block, 0, st>>>(s, pairs, warps);
+    interact_identity_kernel<<<grid, block, 0, st>>>(s, pairs, warps, fs);
   } else {
-    SWARM_FOR_WIDTH(bits, e = launch_dependent(interact_blocking_kernel<W>, grid, block, st, s, pairs, warps))
+    SWARM_FOR_WIDTH(bits, e = (fs.H > 0 ? launch_dependent(interact_blocking_kernel<W, true>, grid, block, st, s, pairs, warps, fs)
+                                         : launch_dependent(interact_blocking_kernel<W, false>, grid, block, st, s, pairs, warps, fs)))
   }
   ++*launches;
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_interact_nonblocking(const StoreView& s, const PairList& pairs, int npairs, int bits,
-                                        cudaStream_t st, int* launches) {
+                                        const FusedSteps& fs, cudaStream_t st, int* launches) {
   if (npairs == 0) return cudaSuccess;
   const int64_t warps = (int64_t)npairs * s.nblk;
   const dim3 grid(ctas_for(warps)), block(kWarpsPerCta * 32);
   cudaError_t e = cudaSuccess;
-  SWARM_FOR_WIDTH(bits, e = launch_dependent(interact_nonblocking_kernel<W>, grid, block, st, s, pairs, warps))
+  SWARM_FOR_WIDTH(bits, e = (fs.H > 0 ? launch_dependent(interact_nonblocking_kernel<W, true>, grid, block, st, s, pairs, warps, fs)
+                                         : launch_dependent(interact_nonblocking_kernel<W, false>, grid, block, st, s, pairs, warps, fs)))
   ++*launches;
   return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -597,12 +648,13 @@ cudaError_t launch_publish(const StoreView& s, const uint32_t* wctr_dev, int bit
 }
 
 cudaError_t launch_interact_registers(const StoreView& s, const PairList& pairs, int npairs, int bits,
-                                      cudaStream_t st, int* launches) {
+                                      const FusedSteps& fs, cudaStream_t st, int* launches) {
   if (npairs == 0) return cudaSuccess;
   const int64_t warps = (int64_t)npairs * s.nblk;
   const dim3 grid(ctas_for(warps)), block(kWarpsPerCta * 32);
   cudaError_t e = cudaSuccess;
-  SWARM_FOR_WIDTH(bits, e = launch_dependent(interact_registers_kernel<W>, grid, block, st, s, pairs, warps))
+  SWARM_FOR_WIDTH(bits, e = (fs.H > 0 ? launch_dependent(interact_registers_kernel<W, true>, grid, block, st, s, pairs, warps, fs)
+                                         : launch_dependent(interact_registers_kernel<W, false>, grid, block, st, s, pairs, warps, fs)))
   ++*launches;
   return e != cudaSuccess ? e : cudaGetLastError();
 }

@@ -12,7 +12,16 @@ struct PairDesc {
   int32_t a, b;        // initiator, responder
   uint32_t wa, wb;     // write counters of the two buffers before this interaction
   uint32_t woa;        // write counter of the initiator's own register (two-register protocol)
+  uint32_t lsa, lsb;   // local-step counters of the two nodes (steps fused into the interaction)
   uint32_t pad;
+};
+
+// Synthetic-gradient local steps taken inside an interaction kernel before the exchange (H = 0: none).
+struct FusedSteps {
+  int32_t H;
+  int32_t responders;  // 1: the responder of each pair steps too; 0: initiators only
+  float lr, grad_std;
+  const float* scalars; // [n][3] per-node offset, drift, shift
 };
 
 // One node of a local-step launch.
@@ -75,14 +84,14 @@ struct LsqView {
 
 // --- swarm_interact.cu -------------------------------------------------------------------
 cudaError_t launch_interact_blocking(const StoreView& s, const PairList& pairs, int npairs, int bits,
-                                     cudaStream_t st, int* launches);
+                                     const FusedSteps& fs, cudaStream_t st, int* launches);
 cudaError_t launch_interact_nonblocking(const StoreView& s, const PairList& pairs, int npairs, int bits,
-                                        cudaStream_t st, int* launches);
+                                        const FusedSteps& fs, cudaStream_t st, int* launches);
 // wctr_dev: n write counters (uint32) used for the rounding uniforms of each node's buffer.
 cudaError_t launch_publish(const StoreView& s, const uint32_t* wctr_dev, int bits, cudaStream_t st, int* launches);
 // Two-register protocol. wctr_dev: n write counters of the current registers followed by n of the own registers.
 cudaError_t launch_interact_registers(const StoreView& s, const PairList& pairs, int npairs, int bits,
-                                      cudaStream_t st, int* launches);
+                                      const FusedSteps& fs, cudaStream_t st, int* launches);
 cudaError_t launch_register_publish(const StoreView& s, const uint32_t* wctr_dev, int bits, cudaStream_t st,
                                     int* launches);
 
