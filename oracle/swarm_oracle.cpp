@@ -254,7 +254,8 @@ struct Swarm {
   int32_t b_stale = 0;
   // two-register protocol (Section 3, "The Communication Registers"): the register a node writes
   // itself holds a 16-bit encoding of its snapshot; `codes` is then the register others write.
-  std::vector<uint16_t> own;         // n * d
+  std::vector<uint8_t> own;          // n * nblk * 2048: per block 1024 low bytes, then 1024 high bytes
+  int32_t own_prefix = 16;           // bits of a partner's own register that a reader consumes (8 or 16)
   std::vector<int8_t> oexps;         // n * nblk
   std::vector<uint32_t> wo;          // write counters of the own registers
   std::vector<uint32_t> tau;         // interactions since the node last initiated
@@ -275,6 +276,11 @@ struct Swarm {
   float* x(int i) { return X.data() + (int64_t)i * d; }
   float* base(int i) { return B.data() + (int64_t)i * d; }
   uint8_t* code_row(int i) { return codes.data() + (int64_t)i * nblk * kBlock; }
+  // own register: the 16-bit colour of coordinate k is split over two byte planes of its block, so that
+  // a reader which needs only the 8-bit prefix (the low byte) touches half of the register
+  uint8_t* own_lo(int i, int64_t k) { return own.data() + ((int64_t)i * nblk + k / kBlock) * 2 * kBlock + k % kBlock; }
+  uint32_t own_get(int i, int64_t k) { const uint8_t* p = own_lo(i, k); return (uint32_t)p[0] | ((uint32_t)p[kBlock] << 8); }
+  void own_put(int i, int64_t k, uint32_t c) { uint8_t* p = own_lo(i, k); p[0] = (uint8_t)c; p[kBlock] = (uint8_t)(c >> 8); }
   int8_t* exp_row(int i) { return exps.data() + (int64_t)i * nblk; }
   int group_of(int i) const { return groups == n ? i : i / (n / groups); }
 };
@@ -368,7 +374,8 @@ void init_state(Swarm& s) {
   s.w.assign(n, 0); s.ls.assign(n, 0);
   s.launch = 0; s.b_stale = 0; s.p_mode = 0;
   s.tau.assign(n, 0); s.wo.assign(n, 0);
-  if (c.nonblocking == 2) { s.own.assign((size_t)n * d, 0); s.oexps.assign((size_t)n * s.nblk, 0); }
+  s.own_prefix = 16;
+  if (c.nonblocking == 2) { s.own.assign((size_t)n * s.nblk * 2 * kBlock, 0); s.oexps.assign((size_t)n * s.nblk, 0); }
   else { s.own.clear(); s.oexps.clear(); }
 
   s.A.clear(); s.bvec.clear(); s.xstar.clear(); s.groups = 0;
@@ -599,6 +606,12 @@ void interact_nonblocking(Swarm& s, int a, int b, int bits) {
 //   current register of node k  P_k = Enc_b(X_k)     written by whoever last interacted with k,
 //                                                    scaled by the exact distance to its decoding
 //                                                    key Q(X^_k) (the writer knows that key)
+// Variable rate (Corollary 1, second case, and "Counting Communication Cost"): the long code sits in
+// the writer's own register and a reader consumes only a prefix sized by its distance. The b-bit colour
+// of a lattice point is the low b bits of its 16-bit colour, so the prefix is the low-order part; the
+// register stores the low bytes of a block before the high bytes, and a reader that trusts its key to be
+// within 127 steps reads the first half only (own_prefix = 8). A node decoding its own register (key =
+// the very snapshot that was encoded, less than one step away) always uses the 8-bit prefix.
 // ---------------------------------------------------------------------------
 constexpr int kOwnBits = 16;
 constexpr int kOwnResolutionBits = 8;
@@ -613,10 +626,9 @@ uint32_t own_uniform(const Rng& rng, uint32_t owner, uint32_t w, int64_t k) {
 // Write O_i = Enc16(v) for one block with exponent eo, return the written lattice points in qhat.
 void write_own_block(Swarm& s, int i, int64_t blk, const float* v, int len, int eo, float* qhat) {
   const int64_t k0 = blk * kBlock;
-  uint16_t* o = s.own.data() + (int64_t)i * s.d + k0;
   for (int k = 0; k < len; ++k) {
     const int32_t q = enc_q(v[k], eo, own_uniform(s.rng, (uint32_t)i, s.wo[i], k0 + k));
-    o[k] = (uint16_t)code_of(q, kOwnBits);
+    s.own_put(i, k0 + k, code_of(q, kOwnBits));
     qhat[k] = (float)q * pow2f(eo);
   }
   s.oexps[(int64_t)i * s.nblk + blk] = (int8_t)eo;
@@ -677,16 +689,16 @@ void interact_registers(Swarm& s, int a, int b, int bits) {
     const int len = (int)std::min<int64_t>(kBlock, d - k0);
     const uint8_t* ca = s.code_row(a) + blk * block_bytes;
     const uint8_t* cb = s.code_row(b) + blk * block_bytes;
-    const uint16_t* oa = s.own.data() + (int64_t)a * d + k0;
-    const uint16_t* ob = s.own.data() + (int64_t)b * d + k0;
+    const int pfx = s.own_prefix;
+    const uint32_t pmask = (1u << pfx) - 1u;
     const int eoa = s.oexps[(int64_t)a * s.nblk + blk], eob = s.oexps[(int64_t)b * s.nblk + blk];
     const int epa = s.exp_row(a)[blk], epb = s.exp_row(b)[blk];
     float spread = 0.0f, dmax = 0.0f, M = 0.0f;
     for (int k = 0; k < len; ++k) {
       const float snap = ba[k0 + k];
-      const float qhat_a = dec(snap, oa[k], eoa, kOwnBits);                   // Q(X^_a): local, key = own snapshot
+      const float qhat_a = dec(snap, s.own_get(a, k0 + k) & 0xFFu, eoa, 8);   // Q(X^_a): local, key = own snapshot
       const float Qa = dec(qhat_a, get_code(ca, k, bits), epa, bits);         // Q(X_a)  <- Dec(Q(X^_a), Enc(X_a))
-      qhat_b[k] = dec(snap, ob[k], eob, kOwnBits);                            // Q(X^_b) <- Dec(X^_a, Enc(X^_b))
+      qhat_b[k] = dec(snap, s.own_get(b, k0 + k) & pmask, eob, pfx);          // Q(X^_b) <- Dec(X^_a, prefix of Enc(X^_b))
       const float Qb = dec(qhat_b[k], get_code(cb, k, bits), epb, bits);      // Q(X_b)  <- Dec(Q(X^_b), Enc(X_b))
       const float av = 0.5f * (Qa + Qb);
       const float D = snap - xa[k0 + k];                                      // pending local update (eta * h)
@@ -977,7 +989,15 @@ int orc_register_publish(void* h, int32_t bits) {
   return 0;
 }
 
-uint16_t* orc_own(void* h) { Swarm& s = *(Swarm*)h; return s.own.empty() ? nullptr : s.own.data(); }
+uint8_t* orc_own(void* h) { Swarm& s = *(Swarm*)h; return s.own.empty() ? nullptr : s.own.data(); }
+int orc_set_own_prefix(void* h, int32_t bits) {
+  Swarm& s = *(Swarm*)h;
+  if (bits != 8 && bits != 16) return -1;
+  if (s.cfg.nonblocking != 2) return -4;
+  s.own_prefix = bits;
+  return 0;
+}
+int32_t orc_get_own_prefix(void* h) { return ((Swarm*)h)->own_prefix; }
 int8_t* orc_oexps(void* h) { Swarm& s = *(Swarm*)h; return s.oexps.empty() ? nullptr : s.oexps.data(); }
 uint32_t* orc_wo(void* h) { return ((Swarm*)h)->wo.data(); }
 uint32_t* orc_tau(void* h) { return ((Swarm*)h)->tau.data(); }

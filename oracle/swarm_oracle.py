@@ -64,7 +64,7 @@ def lib():
         "orc_interact": (C.c_int, [vp, i32p, C.c_int32, C.c_int32, C.c_int32, C.c_int32]),
         "orc_publish": (C.c_int, [vp, C.c_int32]),
         "orc_register_publish": (C.c_int, [vp, C.c_int32]),
-        "orc_own": (u16p, [vp]), "orc_oexps": (i8p, [vp]), "orc_wo": (u32p, [vp]), "orc_tau": (u32p, [vp]),
+        "orc_own": (u8p, [vp]), "orc_set_own_prefix": (C.c_int, [vp, C.c_int32]), "orc_get_own_prefix": (C.c_int32, [vp]), "orc_oexps": (i8p, [vp]), "orc_wo": (u32p, [vp]), "orc_tau": (u32p, [vp]),
         "orc_p_mode": (i32p, [vp]),
         "orc_mean_model": (None, [vp, f32p]),
         "orc_potential": (C.c_double, [vp]),
@@ -236,8 +236,25 @@ class OracleSwarm:
         return _view(lib().orc_b_stale(self._h), (1,), np.int32)
 
     @property
+    def own_bytes(self):
+        """Own registers as stored: per node and block 1024 low bytes, then 1024 high bytes (live view)."""
+        return _view(lib().orc_own(self._h), (self.n, self.nblk * 2048), np.uint8)
+
+    @property
     def own(self):
-        return _view(lib().orc_own(self._h), (self.n, self.d), np.uint16)
+        """16-bit colours per coordinate, assembled from the two byte planes (a copy)."""
+        raw = self.own_bytes
+        if raw is None:
+            return None
+        planes = raw.reshape(self.n, self.nblk, 2, 1024).astype(np.uint16)
+        return (planes[:, :, 0, :] | (planes[:, :, 1, :] << 8)).reshape(self.n, self.nblk * 1024)[:, : self.d]
+
+    def set_own_prefix(self, bits):
+        return int(lib().orc_set_own_prefix(self._h, bits))
+
+    @property
+    def own_prefix(self):
+        return int(lib().orc_get_own_prefix(self._h))
 
     @property
     def oexps(self):

@@ -116,3 +116,94 @@ def test_staleness_clocks_and_mode_switches():
     plain.configure(objective=1, nonblocking=1)
     assert plain.interact([[0, 1]], 8, o.REGISTERS) == -4
     assert plain.register_publish(8) == -1
+
+
+# ---- variable rate: a reader consumes a prefix of the partner's own register (Corollary 1, second case) ----
+
+def test_colours_nest_so_a_prefix_is_a_shorter_code():
+    """The b-bit colour of a lattice point is the low b bits of its 16-bit colour; decoding the prefix gives
+    the full decode exactly when the key lies within the prefix's own window."""
+    rng = np.random.default_rng(0)
+    e = -7
+    step = 2.0 ** e
+    for _ in range(400):
+        q = int(rng.integers(-10**6, 10**6))
+        c16 = o.code(q, 16)
+        for b in (8, 4):
+            assert o.code(q, b) == c16 & ((1 << b) - 1)
+        L8 = 127
+        for off in (0, 1, -1, L8, -L8, L8 + 1, -(L8 + 1), L8 + 2, 300, -5000):
+            key = (q - off) * step + 0.25 * step           # key cell = q - off, i.e. q = cell + off
+            full = o.dec(key, c16, e, 16)
+            short = o.dec(key, c16 & 0xFF, e, 8)
+            assert full == q * step
+            if -L8 <= off <= L8 + 1:                        # q inside [cell - L, cell + L + 1]
+                assert short == full
+            else:
+                assert short != full and (short - full) / step % 256 == 0
+
+
+def far_reader():
+    """Nodes 0 and 1 start close together and node 2 a fixed offset away; after one interaction of 0 with 1
+    the own register of 0 has a finer step, and node 2 sits more than 127 but less than 32767 of those steps
+    away."""
+    s = make(n=3, d=1500, seed=4, offset_std=0.0, drift_std=0.0, grad_std=0.0, init_std=0.001)
+    s.X[2] += np.float32(0.05)
+    s.B[:] = s.X
+    s.register_publish(8)
+    s.interact([[0, 1]], 8, o.REGISTERS)
+    dist_steps = np.abs(s.B[2].astype(np.float64) - s.B[0]) / steps(s.oexps[0], s.d)
+    assert dist_steps.min() > 200 and dist_steps.max() < 30000
+    return s
+
+
+def test_prefix_reader_within_range_matches_the_full_register_and_fails_beyond():
+    near16, near8 = make(offset_std=0.05), make(offset_std=0.05)
+    assert near8.set_own_prefix(8) == 0 and near8.own_prefix == 8 and near16.own_prefix == 16
+    # nodes that keep talking to the same partner stay within the guard distance of each other's snapshots
+    # (that distance sets the own register's step): the 8-bit prefix is all such a reader needs
+    for pairs in ([[0, 1], [2, 3]], [[1, 0], [3, 2]], [[0, 1], [3, 2]], [[1, 0], [2, 3]]):
+        for s in (near16, near8):
+            s.local_steps([p[0] for p in pairs], 2, 0.05)
+            assert s.interact(pairs, 8, o.REGISTERS) == 0
+    assert np.array_equal(near16.X, near8.X) and np.array_equal(near16.own_bytes, near8.own_bytes)
+    assert np.array_equal(near16.codes, near8.codes)
+    # beyond 127 steps the 8-bit prefix aliases (by whole multiples of 256 steps); the full register does not
+    far16, far8 = far_reader(), far_reader()
+    far8.set_own_prefix(8)
+    for s in (far16, far8):
+        assert s.interact([[2, 0]], 8, o.REGISTERS) == 0
+    mid = 0.5 * (far16.B[0].astype(np.float64) + 0.05 + far16.B[0])          # about half way between 2 and 0
+    assert np.abs(far16.X[2] - mid).max() < 0.01
+    assert np.abs(far8.X[2].astype(np.float64) - far16.X[2]).max() > 0.005
+
+
+def test_prefix_reader_never_touches_the_high_bytes_of_its_partner():
+    ref, scr = make(offset_std=0.05), make(offset_std=0.05)
+    for s in (ref, scr):
+        s.set_own_prefix(8)
+        s.local_steps([1], 2, 0.05)
+        s.register_publish(8)
+    planes = scr.own_bytes.reshape(scr.n, scr.nblk, 2, 1024)
+    planes[:, :, 1, :] ^= 0xA5                               # garbage in every high byte, own and partner's
+    for s in (ref, scr):
+        assert s.interact([[1, 3]], 8, o.REGISTERS) == 0
+    assert np.array_equal(ref.X, scr.X) and np.array_equal(ref.codes, scr.codes)
+    assert np.array_equal(ref.own[1], scr.own[1])                            # a's register is rewritten in full
+    # with the full register the same garbage changes what the reader decodes
+    full = make(offset_std=0.05)
+    full.local_steps([1], 2, 0.05)
+    full.register_publish(8)
+    full.own_bytes.reshape(full.n, full.nblk, 2, 1024)[3, :, 1, :] ^= 0xA5
+    assert full.interact([[1, 3]], 8, o.REGISTERS) == 0
+    assert not np.array_equal(full.X[1], ref.X[1])
+
+
+def test_own_prefix_argument_checks():
+    s = make()
+    assert s.set_own_prefix(12) == -1 and s.set_own_prefix(8) == 0
+    s.configure(objective=1, nonblocking=2)
+    assert s.own_prefix == 16                                # a new configuration goes back to the full register
+    plain = o.OracleSwarm(4, 16, "complete")
+    plain.configure(objective=1, nonblocking=1)
+    assert plain.set_own_prefix(8) == -4
