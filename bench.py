@@ -96,9 +96,10 @@ def interaction_bytes(d, bits, mode):
         return d * 16 + 2 * d * bits // 8 + 2 * nblk
     if mode == 1:
         return d * 16 + 4 * d * bits // 8 + 4 * nblk
-    # two registers: model + snapshot read and written, two own registers read and one written (16 bits),
-    # two current registers read and written
-    return d * 16 + d * 6 + 4 * d * bits // 8 + 7 * nblk
+    # two registers: model + snapshot read and written; own registers: the 8-bit prefix of the initiator's,
+    # the 16 bits of the responder's (default prefix) read, the initiator's 16 bits written; two current
+    # registers read and written
+    return d * 16 + d * 5 + 4 * d * bits // 8 + 7 * nblk
 
 
 class PairSchedule:

@@ -196,6 +196,18 @@ int swarm_publish(swarm_ctx *ctx, int32_t bits);
  * Errors: ESTATE unless configured with nonblocking = 2, EINVAL. */
 int swarm_register_publish(swarm_ctx *ctx, int32_t bits);
 
+/* Corollary 1, second case, and "Counting Communication Cost": the long code lives in the writer's own
+ * register and a reader consumes only a prefix sized by its distance to the encoded vector. The b-bit
+ * colour of a lattice point is the low b bits of its 16-bit colour, and the register keeps the low bytes of
+ * a block before the high bytes, so a reader with `bits` = 8 reads the first half of its partner's own
+ * register only; correct while its snapshot is within 127 register steps of the partner's (partners that
+ * keep meeting are; a distant third node needs 16). Beyond that the decode aliases by multiples of 256
+ * steps (defined behaviour, as for every decode outside its window). Default 16; every swarm_configure
+ * resets it. A node decoding its own register always uses the 8-bit prefix (its key is the encoded
+ * snapshot itself). Errors: EINVAL (bits not 8 or 16), ESTATE (configuration without own registers). */
+int swarm_set_own_prefix(swarm_ctx *ctx, int32_t bits);
+int swarm_get_own_prefix(swarm_ctx *ctx, int32_t *bits_host);
+
 /* State access (checkpointing, test injection). `which` selects the array, `node` the row
  * (ignored for whole-context arrays). bytes must equal the row size exactly. Both synchronise. */
 enum {
@@ -209,7 +221,8 @@ enum {
   SWARM_T_XSTAR = 7,    /* d floats, node ignored                    */
   SWARM_T_SCALARS = 8,  /* 3 floats: offset o_i, drift c_i, shift mu_i */
   SWARM_T_COUNTERS = 9, /* 3 uint32: buffer write counter, local-step counter, code width of the buffer */
-  SWARM_T_OWN = 10,     /* d uint16: own register (ESTATE unless nonblocking = 2)                           */
+  SWARM_T_OWN = 10,     /* nblk*2048 bytes: own register, per block 1024 low bytes then 1024 high bytes of
+                           the 16-bit colours (ESTATE unless nonblocking = 2)                               */
   SWARM_T_OEXPS = 11,   /* nblk int8: exponents of the own register                                         */
   SWARM_T_CLOCKS = 12,  /* 2 uint32: write counter of the own register, staleness clock tau                 */
   SWARM_T_MU_RECORD = 13, /* d floats: mean model at the node's last initiation (ESTATE unless tracking)    */

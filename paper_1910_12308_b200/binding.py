@@ -26,7 +26,7 @@ TOPOLOGY = {"complete": TOPO_COMPLETE, "ring": TOPO_RING, "regular": TOPO_REGULA
 
 EXPORTS = [
     "swarm_set_allocator", "swarm_init", "swarm_local_steps", "swarm_local_steps_geometric", "swarm_interact", "swarm_step", "swarm_mean_model",
-    "swarm_potential", "swarm_track_staleness", "swarm_aux_potentials", "swarm_configure", "swarm_sample_pairs", "swarm_publish", "swarm_register_publish", "swarm_get_buffer_mode",
+    "swarm_potential", "swarm_track_staleness", "swarm_aux_potentials", "swarm_configure", "swarm_sample_pairs", "swarm_publish", "swarm_register_publish", "swarm_set_own_prefix", "swarm_get_own_prefix", "swarm_get_buffer_mode",
     "swarm_set_buffer_mode", "swarm_get_tensor",
     "swarm_set_tensor", "swarm_get_state", "swarm_set_state", "swarm_model_ptr", "swarm_set_stream",
     "swarm_sync", "swarm_potential_static", "swarm_kernel_launches", "swarm_last_cuda_error", "swarm_strerror", "swarm_destroy",
@@ -93,6 +93,8 @@ def load():
         "swarm_sample_pairs": (C.c_int, [vp, i32, C.POINTER(SwarmPair), C.POINTER(i32)]),
         "swarm_publish": (C.c_int, [vp, i32]),
         "swarm_register_publish": (C.c_int, [vp, i32]),
+        "swarm_set_own_prefix": (C.c_int, [vp, i32]),
+        "swarm_get_own_prefix": (C.c_int, [vp, C.POINTER(i32)]),
         "swarm_get_buffer_mode": (C.c_int, [vp, C.POINTER(i32)]),
         "swarm_set_buffer_mode": (C.c_int, [vp, i32]),
         "swarm_get_tensor": (C.c_int, [vp, i32, i32, vp, C.c_size_t]),
@@ -241,6 +243,15 @@ class Swarm:
         self._check(self._L.swarm_potential(self._h, C.byref(g)), "swarm_potential")
         return g.value
 
+    def set_own_prefix(self, bits):
+        """Bits (8 or 16) of a partner's own register that a reader consumes; returns the C code."""
+        return int(self._L.swarm_set_own_prefix(self._h, bits))
+
+    def get_own_prefix(self):
+        v = C.c_int32()
+        self._check(self._L.swarm_get_own_prefix(self._h, C.byref(v)), "swarm_get_own_prefix")
+        return v.value
+
     def track_staleness(self, enable=True):
         """Start (or stop) recording what the auxiliary potentials need; returns the C code."""
         return int(self._L.swarm_track_staleness(self._h, 1 if enable else 0))
@@ -302,7 +313,7 @@ class Swarm:
             T_X: (np.float32, self.d), T_B: (np.float32, self.d), T_CODES: (np.uint8, self.nblk * 1024),
             T_EXPS: (np.int8, self.nblk), T_ADJ: (np.int32, self.degree), T_A: (np.float32, m * self.d),
             T_BVEC: (np.float32, m), T_XSTAR: (np.float32, self.d), T_SCALARS: (np.float32, 3),
-            T_COUNTERS: (np.uint32, 3), T_OWN: (np.uint16, self.d), T_OEXPS: (np.int8, self.nblk),
+            T_COUNTERS: (np.uint32, 3), T_OWN: (np.uint8, self.nblk * 2048), T_OEXPS: (np.int8, self.nblk),
             T_CLOCKS: (np.uint32, 2), T_MU_RECORD: (np.float32, self.d), T_A_RECORD: (np.float64, 1),
         }[which]
 

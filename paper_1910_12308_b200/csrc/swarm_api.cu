@@ -53,7 +53,8 @@ struct swarm_ctx {
   float* B = nullptr;
   uint8_t* codes = nullptr;
   int8_t* exps = nullptr;
-  uint16_t* own = nullptr;           // two-register protocol: own registers [n][pitch]
+  uint8_t* own = nullptr;            // two-register protocol: own registers [n][nblk][2048] (low-byte plane, high-byte plane)
+  int32_t own_prefix = 16;           // bits of a partner's own register that a reader consumes
   int8_t* oexps = nullptr;           // [n][nblk]
   int32_t* adj_dev = nullptr;
   float* scalars = nullptr;          // n * 3
@@ -119,6 +120,7 @@ StoreView view_of(const swarm_ctx* c) {
   s.X = c->X; s.B = c->B; s.codes = c->codes; s.exps = c->exps; s.own = c->own; s.oexps = c->oexps;
   s.pitch = c->pitch; s.d = c->d; s.nblk = c->nblk; s.n = c->n;
   s.key0 = (uint32_t)c->seed; s.key1 = (uint32_t)(c->seed >> 32);
+  s.own_prefix = c->own_prefix;
   return s;
 }
 LsqView lsq_of(const swarm_ctx* c) {
@@ -239,7 +241,7 @@ int apply_config(swarm_ctx* c, const swarm_config& cfg) {
     if (!c->B) return SWARM_ENOMEM;
   }
   if (cfg.nonblocking == 2) {
-    c->own = (uint16_t*)dev_alloc(c, (size_t)n * c->pitch * sizeof(uint16_t));
+    c->own = (uint8_t*)dev_alloc(c, (size_t)n * c->nblk * 2 * kBlockCoords);
     c->oexps = (int8_t*)dev_alloc(c, (size_t)n * c->nblk);
     if (!c->own || !c->oexps) return SWARM_ENOMEM;
   }
@@ -264,7 +266,7 @@ int apply_config(swarm_ctx* c, const swarm_config& cfg) {
   SW_CUDA(c, cudaMemsetAsync(c->codes, 0, (size_t)n * c->nblk * kBlockCoords, c->stream));
   SW_CUDA(c, cudaMemsetAsync(c->exps, 0, (size_t)n * c->nblk, c->stream));
   if (c->own) {
-    SW_CUDA(c, cudaMemsetAsync(c->own, 0, (size_t)n * c->pitch * sizeof(uint16_t), c->stream));
+    SW_CUDA(c, cudaMemsetAsync(c->own, 0, (size_t)n * c->nblk * 2 * kBlockCoords, c->stream));
     SW_CUDA(c, cudaMemsetAsync(c->oexps, 0, (size_t)n * c->nblk, c->stream));
   }
   SW_CUDA(c, launch_node_scalars(c->scalars, n, cfg.offset_std, cfg.drift_std, s.key0, s.key1, c->stream, &nl));
@@ -283,6 +285,7 @@ int apply_config(swarm_ctx* c, const swarm_config& cfg) {
   c->launch_ctr = 0;
   c->b_stale = 0;
   c->p_mode = 0;
+  c->own_prefix = 16;
   return SWARM_OK;
 }
 
@@ -819,6 +822,18 @@ int swarm_register_publish(swarm_ctx* c, int32_t bits) {
   return do_register_publish(c, bits);
 }
 
+int swarm_set_own_prefix(swarm_ctx* c, int32_t bits) {
+  if (!c || (bits != 8 && bits != 16)) return SWARM_EINVAL;
+  if (c->cfg.nonblocking != 2) return SWARM_ESTATE;
+  c->own_prefix = bits;
+  return SWARM_OK;
+}
+int swarm_get_own_prefix(swarm_ctx* c, int32_t* bits) {
+  if (!c || !bits) return SWARM_EINVAL;
+  *bits = c->own_prefix;
+  return SWARM_OK;
+}
+
 int swarm_get_buffer_mode(swarm_ctx* c, int32_t* mode) {
   if (!c || !mode) return SWARM_EINVAL;
   *mode = c->p_mode;
@@ -919,7 +934,7 @@ static int tensor_access(swarm_ctx* c, int32_t which, int32_t node, void* host, 
     case SWARM_T_SCALARS: dev = c->scalars + (size_t)node * 3; want = 12; break;
     case SWARM_T_OWN:
       if (!c->own) return SWARM_ESTATE;
-      dev = c->own + (size_t)node * c->pitch; want = d * 2; break;
+      dev = c->own + (size_t)node * c->nblk * 2 * kBlockCoords; want = (size_t)c->nblk * 2 * kBlockCoords; break;
     case SWARM_T_OEXPS:
       if (!c->oexps) return SWARM_ESTATE;
       dev = c->oexps + (size_t)node * c->nblk; want = (size_t)c->nblk; break;

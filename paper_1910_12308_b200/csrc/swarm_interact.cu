@@ -376,9 +376,25 @@ publish_encode_kernel(StoreView s, const uint32_t* __restrict__ wctr, int64_t to
 constexpr int kOwnBits = 16;
 constexpr int kOwnResolutionBits = 8;
 
-__device__ __forceinline__ uint32_t own_code(const uint4& v, int i) {
-  const uint32_t word = (i < 2) ? v.x : (i < 4) ? v.y : (i < 6) ? v.z : v.w;
-  return (i & 1) ? (word >> 16) : (word & 0xFFFFu);
+// Own registers are stored in two byte planes per 1024-coordinate block (1024 low bytes, then 1024 high
+// bytes of the 16-bit colours), so that a reader which needs only the 8-bit prefix touches the first
+// plane alone. A lane's 8 coordinates of a sub-block are 8 consecutive bytes in each plane.
+constexpr int kOwnBlockBytes = 2 * kBlockCoords;
+__device__ __forceinline__ uint32_t plane_byte(const uint2& v, int i) {
+  return (((i < 4) ? v.x : v.y) >> ((i & 3) * 8)) & 0xFFu;
+}
+// Decode with a prefix of `bits` (8 or 16, warp-uniform) of a 16-bit colour.
+__device__ __forceinline__ float decode_prefix(float key, uint32_t c, int bits, float inv_step, float step) {
+  const int32_t cell = __float2int_rd(__fmul_rn(key, inv_step));
+  const uint32_t mask = (1u << bits) - 1u;
+  int32_t delta = (int32_t)((c - (uint32_t)cell) & mask);
+  if (delta > (int32_t)(1u << (bits - 1))) delta -= (int32_t)(mask + 1u);
+  return __fmul_rn(__int2float_rn((int32_t)((uint32_t)cell + (uint32_t)delta)), step);
+}
+// Split eight 16-bit colours (two per word) into their low-byte and high-byte planes.
+__device__ __forceinline__ void split_planes(const uint32_t (&ow)[4], uint2& lo, uint2& hi) {
+  lo.x = __byte_perm(ow[0], ow[1], 0x6420); hi.x = __byte_perm(ow[0], ow[1], 0x7531);
+  lo.y = __byte_perm(ow[2], ow[3], 0x6420); hi.y = __byte_perm(ow[2], ow[3], 0x7531);
 }
 
 template <int BITS, bool FUSED>
@@ -401,10 +417,10 @@ interact_registers_kernel(StoreView s, const PairList pairs, int64_t total_warps
       const int64_t k2 = blk2 * kBlockCoords;
       prefetch_l2(s.X + (int64_t)p2.a * s.pitch + k2 + lane * 32);                      // 32 lines of 128 B
       prefetch_l2(s.B + (int64_t)p2.a * s.pitch + k2 + lane * 32);
-      if (lane < 16) {                                                                   // 2 KiB of 16-bit codes each
-        prefetch_l2(s.own + (int64_t)p2.a * s.pitch + k2 + lane * 64);
-        prefetch_l2(s.own + (int64_t)p2.b * s.pitch + k2 + lane * 64);
-      }
+      if (lane < 8)                                                                      // a's low-byte plane (1 KiB)
+        prefetch_l2(s.own + ((int64_t)p2.a * s.nblk + blk2) * kOwnBlockBytes + lane * 128);
+      if (lane < s.own_prefix)                                                           // b's plane(s): 8 or 16 lines
+        prefetch_l2(s.own + ((int64_t)p2.b * s.nblk + blk2) * kOwnBlockBytes + lane * 128);
       if (lane < BITS) {
         prefetch_l2(s.codes + (int64_t)p2.a * s.nblk * kBlockCoords + blk2 * (kBlockCoords * BITS / 8) + lane * 128);
         prefetch_l2(s.codes + (int64_t)p2.b * s.nblk * kBlockCoords + blk2 * (kBlockCoords * BITS / 8) + lane * 128);
@@ -414,13 +430,14 @@ interact_registers_kernel(StoreView s, const PairList pairs, int64_t total_warps
   const int64_t koff = blk * kBlockCoords + lane * 8;
   float* xa = s.X + (int64_t)pd.a * s.pitch + koff;
   float* ba = s.B + (int64_t)pd.a * s.pitch + koff;
-  uint16_t* oa = s.own + (int64_t)pd.a * s.pitch + koff;
-  const uint16_t* ob = s.own + (int64_t)pd.b * s.pitch + koff;
+  uint8_t* oa = s.own + ((int64_t)pd.a * s.nblk + blk) * kOwnBlockBytes + lane * 8;       // low plane; high at +1024
+  const uint8_t* ob = s.own + ((int64_t)pd.b * s.nblk + blk) * kOwnBlockBytes + lane * 8;
+  const int prefix = s.own_prefix;
   uint8_t* ca = s.codes + (int64_t)pd.a * s.nblk * kBlockCoords + blk * (kBlockCoords * BITS / 8) + lane * BITS;
   uint8_t* cb = s.codes + (int64_t)pd.b * s.nblk * kBlockCoords + blk * (kBlockCoords * BITS / 8) + lane * BITS;
 
   f8 nx[kSub], av[kSub];       // loaded as X^a / B^a, overwritten with new model / average
-  uint4 va[kSub], vb[kSub];
+  uint2 va[kSub], vb[kSub], vbh[kSub];   // low bytes of a's and b's own registers, high bytes of b's
   uint64_t pa[kSub], pb[kSub];
 #pragma unroll
   for (int j = 0; j < kSub; ++j) nx[j] = ld256(xa + j * kSubCoords);
@@ -432,8 +449,9 @@ interact_registers_kernel(StoreView s, const PairList pairs, int64_t total_warps
   for (int j = 0; j < kSub; ++j) av[j] = ld256(ba + j * kSubCoords);
 #pragma unroll
   for (int j = 0; j < kSub; ++j) {
-    va[j] = *reinterpret_cast<const uint4*>(oa + j * kSubCoords);
-    vb[j] = *reinterpret_cast<const uint4*>(ob + j * kSubCoords);
+    va[j] = *reinterpret_cast<const uint2*>(oa + j * kSubCoords);
+    vb[j] = *reinterpret_cast<const uint2*>(ob + j * kSubCoords);
+    vbh[j] = prefix == 16 ? *reinterpret_cast<const uint2*>(ob + kBlockCoords + j * kSubCoords) : make_uint2(0u, 0u);
     pa[j] = load_codes<BITS>(ca + j * (kSubCoords * BITS / 8));
     pb[j] = load_codes<BITS>(cb + j * (kSubCoords * BITS / 8));
   }
@@ -449,9 +467,9 @@ interact_registers_kernel(StoreView s, const PairList pairs, int64_t total_warps
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const float snap = av[j].v[i];
-      const float qhat_a = decode_value<kOwnBits>(snap, own_code(va[j], i), io_a, so_a);
+      const float qhat_a = decode_value<8>(snap, plane_byte(va[j], i), io_a, so_a);    // own key: < 1 step away
       const float Qa = decode_value<BITS>(qhat_a, (uint32_t)(pa[j] >> (i * BITS)) & mask, ip_a, sp_a);
-      const float qhat_b = decode_value<kOwnBits>(snap, own_code(vb[j], i), io_b, so_b);
+      const float qhat_b = decode_prefix(snap, plane_byte(vb[j], i) | (plane_byte(vbh[j], i) << 8), prefix, io_b, so_b);
       const float Qb = decode_value<BITS>(qhat_b, (uint32_t)(pb[j] >> (i * BITS)) & mask, ip_b, sp_b);
       const float avg = __fmul_rn(0.5f, __fadd_rn(Qa, Qb));
       const float D = __fsub_rn(snap, nx[j].v[i]);
@@ -493,7 +511,10 @@ interact_registers_kernel(StoreView s, const PairList pairs, int64_t total_warps
       M_a = fmaxf(M_a, fmaxf(fabsf(nx[j].v[i]), fabsf(qhat_new)));
       pkb |= (uint64_t)((uint32_t)encode_index(av[j].v[i], ipb_new, sr_u16(rb, i), cell) & mask) << (i * BITS);
     }
-    *reinterpret_cast<uint4*>(oa + j * kSubCoords) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+    uint2 lo, hi;
+    split_planes(ow, lo, hi);
+    *reinterpret_cast<uint2*>(oa + j * kSubCoords) = lo;
+    *reinterpret_cast<uint2*>(oa + kBlockCoords + j * kSubCoords) = hi;
     store_codes<BITS>(cb + j * (kSubCoords * BITS / 8), lane, pkb);
   }
   rho_a = warp_max_nonneg(rho_a);
@@ -533,7 +554,7 @@ register_publish_encode_kernel(StoreView s, const uint32_t* __restrict__ wctr, i
   const int64_t blk = warp - node * s.nblk;
   const int64_t koff = blk * kBlockCoords + lane * 8;
   const float* row = s.B + node * s.pitch + koff;
-  uint16_t* o = s.own + node * s.pitch + koff;
+  uint8_t* o = s.own + (node * s.nblk + blk) * kOwnBlockBytes + lane * 8;
   uint8_t* c = s.codes + node * s.nblk * kBlockCoords + blk * (kBlockCoords * BITS / 8) + lane * BITS;
   const int eo = s.oexps[node * s.nblk + blk];
   const float so = pow2f_exact(eo), io = pow2f_exact(-eo);
@@ -557,7 +578,10 @@ register_publish_encode_kernel(StoreView s, const uint32_t* __restrict__ wctr, i
       rho = fmaxf(rho, fabsf(__fsub_rn(v[j].v[i], qhat)));
       M = fmaxf(M, fmaxf(fabsf(v[j].v[i]), fabsf(qhat)));
     }
-    *reinterpret_cast<uint4*>(o + j * kSubCoords) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+    uint2 lo, hi;
+    split_planes(ow, lo, hi);
+    *reinterpret_cast<uint2*>(o + j * kSubCoords) = lo;
+    *reinterpret_cast<uint2*>(o + kBlockCoords + j * kSubCoords) = hi;
   }
   rho = warp_max_nonneg(rho);
   M = warp_max_nonneg(M);

@@ -66,13 +66,15 @@ struct StoreView {
   float* B;            // [n][pitch] or nullptr
   uint8_t* codes;      // [n][nblk * 1024]
   int8_t* exps;        // [n][nblk]
-  uint16_t* own;       // [n][pitch] own registers (two-register protocol) or nullptr
+  uint8_t* own;        // [n][nblk][2048] own registers (two-register protocol) or nullptr: per block the low
+                       // bytes of the 1024 16-bit colours, then their high bytes
   int8_t* oexps;       // [n][nblk] exponents of the own registers
   int64_t pitch;       // elements per row, multiple of 1024
   int64_t d;
   int64_t nblk;
   int32_t n;
   uint32_t key0, key1; // generator key (seed low / high word)
+  int32_t own_prefix;  // bits of a partner's own register that a reader consumes: 8 or 16
 };
 
 struct LsqView {

@@ -33,8 +33,8 @@ def inject(orc, gpu, what=("X", "B", "P", "counters", "data")):
         if "P" in what:
             gpu.set(g.T_CODES, i, orc.codes[i])
             gpu.set(g.T_EXPS, i, orc.exps[i])
-        if "P" in what and orc.own is not None:
-            gpu.set(g.T_OWN, i, orc.own[i])
+        if "P" in what and orc.own_bytes is not None:
+            gpu.set(g.T_OWN, i, orc.own_bytes[i])
             gpu.set(g.T_OEXPS, i, orc.oexps[i])
         if "counters" in what:
             gpu.set(g.T_COUNTERS, i, [orc.w[i], orc.ls[i], orc.pbits[i]])
@@ -62,8 +62,8 @@ def assert_store_equal(orc, gpu, bits=None, nodes=None, check_B=True):
         w, ls, pb = gpu.get(g.T_COUNTERS, i)
         assert (w, ls, pb) == (orc.w[i], orc.ls[i], orc.pbits[i]), f"counters[{i}]"
         assert tuple(gpu.get(g.T_CLOCKS, i)) == (orc.wo[i], orc.tau[i]), f"clocks[{i}]"
-        if orc.own is not None and int(orc.p_mode[0]) == 2:
-            assert np.array_equal(gpu.get(g.T_OWN, i), orc.own[i]), f"own register[{i}] differs"
+        if orc.own_bytes is not None and int(orc.p_mode[0]) == 2:
+            assert np.array_equal(gpu.get(g.T_OWN, i), orc.own_bytes[i]), f"own register[{i}] differs"
             assert np.array_equal(gpu.get(g.T_OEXPS, i), orc.oexps[i]), f"own exponents[{i}] differ"
         if bits is not None and 2 <= bits <= 8 and orc.pbits[i] == bits:
             nbytes = orc.nblk * 128 * bits

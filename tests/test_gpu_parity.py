@@ -210,6 +210,38 @@ def test_register_protocol_bit_exact(bits, d):
         assert_store_equal(orc, gpu, bits)
 
 
+@pytest.mark.parametrize("bits", [3, 8])
+def test_register_protocol_with_8_bit_prefix_reads(bits):
+    """Readers consume only the low-byte plane of their partner's own register (in range and aliasing alike)."""
+    n, d = 6, 3001
+    cfg = dict(objective=1, nonblocking=2, grad_std=0.03, drift_std=0.1, offset_std=0.2)
+    orc, gpu = make_pair(n, d, "complete", seed=31, **cfg)
+    inject(orc, gpu)
+    assert orc.set_own_prefix(8) == 0 and gpu.set_own_prefix(8) == 0 and gpu.get_own_prefix() == 8
+    assert gpu.set_own_prefix(12) == g.EINVAL
+    rng = np.random.default_rng(bits)
+    for rnd in range(8):
+        nodes = rng.permutation(n)[:3]
+        assert orc.local_steps(nodes, 2, 0.05) == 0 and gpu.local_steps(nodes, 2, 0.05) == 0
+        inject(orc, gpu, what=("X",))
+        pairs = disjoint_pairs(orc, rng, int(rng.integers(1, 4)))
+        assert orc.interact(pairs, bits, o.REGISTERS) == 0
+        assert gpu.interact(pairs, bits, g.REGISTERS) == 0
+        assert_store_equal(orc, gpu, bits)
+    # garbage in the high-byte planes of everybody else changes nothing for a prefix reader
+    before = gpu.get(g.T_X, 0).copy()
+    ref_pairs = [[0, 1]]
+    orc_x = orc.X.copy()
+    for i in range(1, n):
+        row = gpu.get(g.T_OWN, i).reshape(-1, 2, 1024)
+        row[:, 1, :] ^= 0x5A
+        gpu.set(g.T_OWN, i, row.reshape(-1))
+    assert orc.interact(ref_pairs, bits, o.REGISTERS) == 0 and gpu.interact(ref_pairs, bits, g.REGISTERS) == 0
+    assert np.array_equal(gpu.get(g.T_X, 0).view(np.uint32), orc.X[0].view(np.uint32))
+    gpu.configure(**cfg)
+    assert gpu.get_own_prefix() == 16
+
+
 def test_register_protocol_mode_switches_and_far_snapshots():
     n, d = 4, 2100
     cfg = dict(objective=1, nonblocking=2, grad_std=0.0, drift_std=0.0, offset_std=0.05)
