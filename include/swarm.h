@@ -152,6 +152,18 @@ int swarm_interact(swarm_ctx *ctx, const swarm_pair *pairs_host, int32_t npairs,
 int swarm_step(swarm_ctx *ctx, const swarm_pair *pairs_host, int32_t npairs, int32_t H, float lr, int32_t bits,
                int32_t mode, int32_t step_responders);
 
+/* Section 3, "Sequential model": nsteps interactions one after the other, pairs_host[t] being the pair of
+ * time step t (consecutive pairs may share nodes). Same results, bit for bit, as
+ *     for t: swarm_step(ctx, &pairs_host[t], 1, H, lr, bits, SWARM_BLOCKING, step_responders).
+ * For short models (row pitch <= 8192) with fp32 least-squares or logistic data and a minibatch of at most
+ * 32 rows the whole sequence runs in ONE kernel launch (a thread-block cluster walks the steps; launch
+ * latency, which dominates such steps, is paid once per 64 steps or more); otherwise the library issues the
+ * steps one by one. Refused (ESTATE) while staleness tracking is on, like every blocking exchange.
+ * Errors: EINVAL (nsteps < 0, H < 0, bits, NULL), ERANGE, EPAIR (a pair that is not an edge), ESTATE; all pairs
+ * are checked before anything runs. */
+int swarm_run_sequence(swarm_ctx *ctx, const swarm_pair *pairs_host, int32_t nsteps, int32_t H, float lr,
+                       int32_t bits, int32_t step_responders);
+
 /* Section 4: mu = (1/n) sum_i X^i, written to out_dev (d floats, device memory). */
 int swarm_mean_model(swarm_ctx *ctx, float *out_dev);
 

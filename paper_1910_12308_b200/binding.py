@@ -25,7 +25,7 @@ T_X, T_B, T_CODES, T_EXPS, T_ADJ, T_A, T_BVEC, T_XSTAR, T_SCALARS, T_COUNTERS, T
 TOPOLOGY = {"complete": TOPO_COMPLETE, "ring": TOPO_RING, "regular": TOPO_REGULAR}
 
 EXPORTS = [
-    "swarm_set_allocator", "swarm_init", "swarm_local_steps", "swarm_local_steps_geometric", "swarm_interact", "swarm_step", "swarm_mean_model",
+    "swarm_set_allocator", "swarm_init", "swarm_local_steps", "swarm_local_steps_geometric", "swarm_interact", "swarm_step", "swarm_run_sequence", "swarm_mean_model",
     "swarm_potential", "swarm_track_staleness", "swarm_aux_potentials", "swarm_configure", "swarm_sample_pairs", "swarm_publish", "swarm_register_publish", "swarm_set_own_prefix", "swarm_get_own_prefix", "swarm_get_buffer_mode",
     "swarm_set_buffer_mode", "swarm_get_tensor",
     "swarm_set_tensor", "swarm_get_state", "swarm_set_state", "swarm_model_ptr", "swarm_set_stream",
@@ -85,6 +85,7 @@ def load():
         "swarm_local_steps_geometric": (C.c_int, [vp, C.POINTER(i32), i32, i32, f32, C.POINTER(i32)]),
         "swarm_interact": (C.c_int, [vp, C.POINTER(SwarmPair), i32, i32, i32]),
         "swarm_step": (C.c_int, [vp, C.POINTER(SwarmPair), i32, i32, f32, i32, i32, i32]),
+        "swarm_run_sequence": (C.c_int, [vp, C.POINTER(SwarmPair), i32, i32, f32, i32, i32]),
         "swarm_mean_model": (C.c_int, [vp, vp]),
         "swarm_potential": (C.c_int, [vp, C.POINTER(C.c_double)]),
         "swarm_track_staleness": (C.c_int, [vp, i32]),
@@ -230,6 +231,12 @@ class Swarm:
         interactions, in one call; returns the C code."""
         arr, ptr = _pairs_array(pairs)
         return self._L.swarm_step(self._h, ptr, len(arr), H, lr, bits, mode, 1 if step_responders else 0)
+
+    def run_sequence(self, pairs, H, lr, bits, step_responders=True):
+        """One interaction per time step, pairs[t] at step t, local steps before each (sequential gossip);
+        a single kernel launch for short models with fp32 least-squares data. Returns the C code."""
+        arr, ptr = _pairs_array(pairs)
+        return self._L.swarm_run_sequence(self._h, ptr, len(arr), H, lr, bits, 1 if step_responders else 0)
 
     def mean_model(self, out=None):
         import torch

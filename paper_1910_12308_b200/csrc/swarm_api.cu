@@ -768,6 +768,75 @@ int swarm_step(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, int32_t H,
   return interact_impl(c, pairs, npairs, bits, mode, 0, 0.0f, 0);
 }
 
+int swarm_run_sequence(swarm_ctx* c, const swarm_pair* pairs, int32_t nsteps, int32_t H, float lr, int32_t bits,
+                       int32_t step_responders) {
+  if (!c || nsteps < 0 || H < 0 || (nsteps > 0 && !pairs)) return SWARM_EINVAL;
+  if (!((bits >= 2 && bits <= 8) || bits == 32)) return SWARM_EINVAL;
+  if (H > 0 && c->cfg.objective == SWARM_OBJ_NONE) return SWARM_ESTATE;
+  if (c->track) return SWARM_ESTATE;
+  for (int t = 0; t < nsteps; ++t) {
+    const int rc = validate_pairs(c, pairs + t, 1);
+    if (rc != SWARM_OK) return rc;
+  }
+  if (nsteps == 0) return SWARM_OK;
+  DeviceGuard guard(c->device);
+  const StoreView s = view_of(c);
+  const LsqView l = lsq_of(c);
+  const bool lsq = c->cfg.objective == SWARM_OBJ_LSQ || c->cfg.objective == SWARM_OBJ_LOGISTIC;
+  if (!(lsq && H > 0 && bits != 32 && !c->tc_partial && lsq_sequence_supported(s, l))) {
+    // no single-launch form for this configuration: the steps one by one
+    for (int t = 0; t < nsteps; ++t) {
+      const int rc = swarm_step(c, pairs + t, 1, H, lr, bits, SWARM_BLOCKING, step_responders);
+      if (rc != SWARM_OK) return rc;
+    }
+    return SWARM_OK;
+  }
+  // One launch per slice of the sequence. The host knows how every counter evolves (each step advances the
+  // two buffers' write counters by one and the stepping nodes' local-step counters by H), so the descriptors
+  // of all steps are written up front and the kernel needs no counters of its own.
+  const int max_slice = (int)std::max<size_t>(kInlinePairs, c->stage_slot_bytes / sizeof(PairDesc));
+  for (int base = 0; base < nsteps; base += max_slice) {
+    const int count = std::min(max_slice, nsteps - base);
+    void *host = nullptr, *dev = nullptr;
+    int slot = -1;
+    PairList list{};
+    list.n = count;
+    PairDesc* pd = list.inl;
+    if (count > kInlinePairs) {
+      const int rc = stage_acquire(c, (size_t)count * sizeof(PairDesc), &host, &dev, &slot);
+      if (rc != SWARM_OK) return rc;
+      pd = (PairDesc*)host;
+      list.ptr = (const PairDesc*)dev;
+    }
+    for (int t = 0; t < count; ++t) {
+      const int a = pairs[base + t].a, b = pairs[base + t].b;
+      pd[t].a = a; pd[t].b = b;
+      pd[t].wa = c->w[a]; pd[t].wb = c->w[b]; pd[t].woa = c->wo[a];
+      pd[t].lsa = c->ls[a]; pd[t].lsb = c->ls[b]; pd[t].pad = 0;
+      c->w[a] += 1; c->w[b] += 1;
+      c->pbits[a] = bits; c->pbits[b] = bits;
+      c->ls[a] += (uint32_t)H;
+      if (step_responders) c->ls[b] += (uint32_t)H;
+      for (int i = 0; i < c->n; ++i) c->tau[i] += 1;
+      c->tau[a] = 0;
+    }
+    if (slot >= 0) {
+      const int rc = stage_commit(c, slot, (size_t)count * sizeof(PairDesc));
+      if (rc != SWARM_OK) return rc;
+    }
+    int nl = 0;
+    SW_CUDA(c, launch_lsq_sequence(s, l, list, H, lr, bits, step_responders ? 1 : 0, c->stream, &nl));
+    c->launches += nl;
+    if (slot >= 0) {
+      const int rc = stage_release(c, slot);
+      if (rc != SWARM_OK) return rc;
+    }
+  }
+  c->p_mode = 0;
+  if (c->cfg.nonblocking) c->b_stale = 1;
+  return SWARM_OK;
+}
+
 int swarm_track_staleness(swarm_ctx* c, int32_t enable) {
   if (!c) return SWARM_EINVAL;
   DeviceGuard guard(c->device);

@@ -1,0 +1,114 @@
+// Per-block bodies shared by the interaction kernels and the single-launch sequence kernel: one warp
+// handles one 1024-coordinate block of one pair; a lane owns 8 consecutive coordinates in each of the
+// block's four 256-coordinate sub-blocks.
+#pragma once
+#include "swarm_dev.cuh"
+#include "swarm_internal.h"
+
+namespace swarm {
+
+constexpr int kSub = 4;          // sub-blocks per block
+constexpr int kSubCoords = 256;  // coordinates per sub-block
+
+// Local steps fused into an interaction (synthetic objective): H steps on the lane's 4 x 8 coordinates of
+// block blk of `node`, then the padding behind coordinate d of the last block is put back to zero.
+__device__ __forceinline__ void fused_steps_block(f8 (&v)[kSub], const StoreView& s, const FusedSteps& fs, int node,
+                                                  uint32_t event, int64_t blk, int lane) {
+  const float c = fs.scalars[node * 3 + 1];
+  const PhiloxRoundKeys rk = philox_round_keys(s.key0, s.key1);
+  const uint32_t g0 = (uint32_t)(blk * (kBlockCoords / 8) + lane);
+  for (int q = 0; q < fs.H; ++q) {
+#pragma unroll
+    for (int j = 0; j < kSub; ++j)
+      synth_step8(v[j], g0 + j * (kSubCoords / 8), (uint32_t)node, event + (uint32_t)q, fs.lr, fs.grad_std, c, rk);
+  }
+  if (blk == s.nblk - 1) {
+#pragma unroll
+    for (int j = 0; j < kSub; ++j)
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        if (blk * kBlockCoords + j * kSubCoords + lane * 8 + i >= s.d) v[j].v[i] = 0.0f;
+  }
+}
+
+// The responder's local steps when the interaction itself does not touch its model.
+__device__ __forceinline__ void fused_steps_responder(const StoreView& s, const FusedSteps& fs, const PairDesc& pd,
+                                                      int64_t blk, int lane) {
+  float* xb = s.X + (int64_t)pd.b * s.pitch + blk * kBlockCoords + lane * 8;
+  f8 vb[kSub];
+#pragma unroll
+  for (int j = 0; j < kSub; ++j) vb[j] = ld256(xb + j * kSubCoords);
+  fused_steps_block(vb, s, fs, pd.b, pd.lsb, blk, lane);
+#pragma unroll
+  for (int j = 0; j < kSub; ++j) st256(xb + j * kSubCoords, vb[j]);
+}
+
+// Blocking interaction of one block (Algorithm 1, interaction lines, with both models present): exact
+// range of X^a - X^b gives the common exponent; both models are encoded into their buffers; each side
+// decodes the partner's codes against its own model and both adopt Q(X^a)/2 + Q(X^b)/2.
+template <int BITS, bool FUSED>
+__device__ __forceinline__ void blocking_block(const StoreView& s, const PairDesc& pd, int64_t blk, int lane,
+                                               const FusedSteps& fs) {
+  float* xa = s.X + (int64_t)pd.a * s.pitch + blk * kBlockCoords + lane * 8;
+  float* xb = s.X + (int64_t)pd.b * s.pitch + blk * kBlockCoords + lane * 8;
+
+  f8 va[kSub], vb[kSub];
+#pragma unroll
+  for (int j = 0; j < kSub; ++j) va[j] = ld256(xa + j * kSubCoords);
+#pragma unroll
+  for (int j = 0; j < kSub; ++j) vb[j] = ld256(xb + j * kSubCoords);
+  if constexpr (FUSED) {
+    fused_steps_block(va, s, fs, pd.a, pd.lsa, blk, lane);
+    if (fs.responders) fused_steps_block(vb, s, fs, pd.b, pd.lsb, blk, lane);
+  }
+
+  float rho = 0.0f, M = 0.0f;
+#pragma unroll
+  for (int j = 0; j < kSub; ++j)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      rho = fmaxf(rho, fabsf(__fsub_rn(va[j].v[i], vb[j].v[i])));
+      M = fmaxf(M, fmaxf(fabsf(va[j].v[i]), fabsf(vb[j].v[i])));
+    }
+  rho = warp_max_nonneg(rho);
+  M = warp_max_nonneg(M);
+  const int e = exponent_rule<BITS>(rho, M);
+  const float step = pow2f_exact(e), inv_step = pow2f_exact(-e);
+
+  constexpr uint32_t mask = (1u << BITS) - 1u;
+  const uint32_t group0 = (uint32_t)(blk * (kBlockCoords / 8) + lane);   // generator call index of sub-block 0
+  uint8_t* ca = s.codes + (int64_t)pd.a * s.nblk * kBlockCoords + blk * (kBlockCoords * BITS / 8) + lane * BITS;
+  uint8_t* cb = s.codes + (int64_t)pd.b * s.nblk * kBlockCoords + blk * (kBlockCoords * BITS / 8) + lane * BITS;
+
+#pragma unroll
+  for (int j = 0; j < kSub; ++j) {
+    const uint32_t g = group0 + j * (kSubCoords / 8);
+    const uint4 ra = philox4x32_10(g, (uint32_t)pd.a, pd.wa, kStreamRounding, s.key0, s.key1);
+    const uint4 rb = philox4x32_10(g, (uint32_t)pd.b, pd.wb, kStreamRounding, s.key0, s.key1);
+    uint64_t pka = 0, pkb = 0;
+    f8 out;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      int32_t cell_a, cell_b;
+      const int32_t qa = encode_index(va[j].v[i], inv_step, sr_u16(ra, i), cell_a);
+      const int32_t qb = encode_index(vb[j].v[i], inv_step, sr_u16(rb, i), cell_b);
+      const uint32_t code_a = (uint32_t)qa & mask, code_b = (uint32_t)qb & mask;
+      pka |= (uint64_t)code_a << (i * BITS);
+      pkb |= (uint64_t)code_b << (i * BITS);
+      // b decodes a's codes with X^b as key and vice versa; the key's cell is already known
+      const float Qa = __fmul_rn(__int2float_rn(decode_index<BITS>(code_a, cell_b)), step);
+      const float Qb = __fmul_rn(__int2float_rn(decode_index<BITS>(code_b, cell_a)), step);
+      out.v[i] = __fmul_rn(0.5f, __fadd_rn(Qa, Qb));
+    }
+    st256(xa + j * kSubCoords, out);
+    st256(xb + j * kSubCoords, out);
+    store_codes<BITS>(ca + j * (kSubCoords * BITS / 8), lane, pka);
+    store_codes<BITS>(cb + j * (kSubCoords * BITS / 8), lane, pkb);
+  }
+  if (lane == 0) {
+    s.exps[(int64_t)pd.a * s.nblk + blk] = (int8_t)e;
+    s.exps[(int64_t)pd.b * s.nblk + blk] = (int8_t)e;
+  }
+}
+
+}  // namespace swarm

@@ -110,6 +110,12 @@ cudaError_t launch_local_synth(const StoreView& s, const NodeList& nodes, int co
 cudaError_t launch_local_lsq(const StoreView& s, const LsqView& l, const NodeList& nodes, int count, int H,
                              float lr, float* partial_dev, cudaStream_t st, int* launches);
 int64_t lsq_chunks(int64_t d);
+// Sequential gossip in one launch (short models, fp32 least-squares data, batch <= 32): steps.n steps of one
+// pair each; per step the pair's nodes (the initiator only if responders == 0) take H local steps, then the
+// pair interacts in blocking mode at `bits` bits. The descriptors carry the counters of every step.
+bool lsq_sequence_supported(const StoreView& s, const LsqView& l);
+cudaError_t launch_lsq_sequence(const StoreView& s, const LsqView& l, const PairList& steps, int H, float lr, int bits,
+                                int responders, cudaStream_t st, int* launches);
 
 // --- swarm_lsq_tc.cu (bf16 data, batch <= 64) ----------------------------------------------
 size_t lsq_tc_partial_bytes(int64_t pitch, int units);

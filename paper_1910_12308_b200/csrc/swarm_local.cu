@@ -6,6 +6,7 @@
 
 #include "swarm_dev.cuh"
 #include "swarm_internal.h"
+#include "swarm_blocks.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -249,90 +250,159 @@ __device__ __forceinline__ float4 load4_as_float<__nv_bfloat16>(const __nv_bfloa
                      __uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xFFFF0000u));
 }
 
+// Shared-memory scratch of the short-model least-squares steps, for up to two nodes handled at once.
+struct SmallShared {
+  int rows[2][kSmallMaxBatch];
+  float red[2][kSmallThreads / 32][kSmallMaxBatch];
+  float part[2][kSmallMaxBatch];       // this CTA's partial dot products (read by the whole cluster)
+  float resid[2][kSmallMaxBatch];
+};
+
+// H least-squares steps of nn (1 or 2) nodes, executed by a whole cluster; the nodes share the cluster
+// barriers but each keeps the arithmetic order of a node handled alone. Models are read from and written
+// back to global memory; the caller orders those accesses against other CTAs' work.
+template <typename T>
+__device__ __forceinline__ void lsq_small_steps(cg::cluster_group& cluster, const StoreView& s, const LsqView& l,
+                                                int nn, const int (&node)[2], const uint32_t (&event)[2], int H,
+                                                float lr, int csize, int iters, SmallShared& sh) {
+  const int rank = (int)cluster.block_rank();
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int64_t base = (int64_t)rank * iters * (kSmallThreads * 4) + tid * 4;   // first coordinate of this thread
+  float4 x[2][2];
+#pragma unroll
+  for (int u = 0; u < 2; ++u) {
+    x[u][0] = x[u][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (u < nn) {
+      const float* xrow = s.X + (int64_t)node[u] * s.pitch + base;
+      x[u][0] = *reinterpret_cast<const float4*>(xrow);
+      if (iters > 1) x[u][1] = *reinterpret_cast<const float4*>(xrow + kSmallThreads * 4);
+    }
+  }
+  const float scale = lr / (float)l.batch;
+
+  for (int q = 0; q < H; ++q) {
+    if (tid < l.batch)
+      for (int u = 0; u < nn; ++u)
+        sh.rows[u][tid] = minibatch_row(tid, node[u] / l.nodes_per_group, event[u] + (uint32_t)q, l.m, s.key0, s.key1);
+    __syncthreads();
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      if (u >= nn) continue;
+      const T* A = reinterpret_cast<const T*>(l.A) + (int64_t)(node[u] / l.nodes_per_group) * l.m * s.pitch + base;
+      // groups of 8 sampled rows: all loads of a group are issued before the first reduction
+      for (int s0 = 0; s0 < l.batch; s0 += 8) {
+        float4 a0[8], a1[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const bool on = s0 + j < l.batch;
+          const T* row = A + (int64_t)sh.rows[u][on ? s0 + j : 0] * s.pitch;
+          a0[j] = on ? load4_as_float<T>(row) : make_float4(0.f, 0.f, 0.f, 0.f);
+          a1[j] = (on && iters > 1) ? load4_as_float<T>(row + kSmallThreads * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          float acc = a0[j].x * x[u][0].x;
+          acc = fmaf(a0[j].y, x[u][0].y, acc); acc = fmaf(a0[j].z, x[u][0].z, acc); acc = fmaf(a0[j].w, x[u][0].w, acc);
+          acc = fmaf(a1[j].x, x[u][1].x, acc); acc = fmaf(a1[j].y, x[u][1].y, acc);
+          acc = fmaf(a1[j].z, x[u][1].z, acc); acc = fmaf(a1[j].w, x[u][1].w, acc);
+          acc = warp_sum(acc);
+          if (lane == 0 && s0 + j < l.batch) sh.red[u][warp][s0 + j] = acc;
+        }
+      }
+    }
+    __syncthreads();
+    if (tid < l.batch)
+      for (int u = 0; u < nn; ++u) {
+        float tot = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kSmallThreads / 32; ++w) tot += sh.red[u][w][tid];
+        sh.part[u][tid] = tot;
+      }
+    cluster.sync();                              // every CTA's partial sums are in place
+    if (tid < l.batch)
+      for (int u = 0; u < nn; ++u) {
+        float tot = 0.0f;
+        for (int r = 0; r < csize; ++r) tot += *cluster.map_shared_rank(&sh.part[u][tid], r);
+        const float* labels = l.bvec + (int64_t)node[u] * l.m;
+        sh.resid[u][tid] = row_residual(tot, labels[sh.rows[u][tid]], l.logistic);
+      }
+    __syncthreads();
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      if (u >= nn) continue;
+      const T* A = reinterpret_cast<const T*>(l.A) + (int64_t)(node[u] / l.nodes_per_group) * l.m * s.pitch + base;
+      float4 g0 = make_float4(0.f, 0.f, 0.f, 0.f), g1 = g0;
+      for (int s0 = 0; s0 < l.batch; s0 += 8) {
+        float4 a0[8], a1[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const bool on = s0 + j < l.batch;
+          const T* row = A + (int64_t)sh.rows[u][on ? s0 + j : 0] * s.pitch;
+          a0[j] = on ? load4_as_float<T>(row) : make_float4(0.f, 0.f, 0.f, 0.f);
+          a1[j] = (on && iters > 1) ? load4_as_float<T>(row + kSmallThreads * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const float rs = s0 + j < l.batch ? sh.resid[u][s0 + j] : 0.0f;
+          g0.x = fmaf(rs, a0[j].x, g0.x); g0.y = fmaf(rs, a0[j].y, g0.y); g0.z = fmaf(rs, a0[j].z, g0.z); g0.w = fmaf(rs, a0[j].w, g0.w);
+          g1.x = fmaf(rs, a1[j].x, g1.x); g1.y = fmaf(rs, a1[j].y, g1.y); g1.z = fmaf(rs, a1[j].z, g1.z); g1.w = fmaf(rs, a1[j].w, g1.w);
+        }
+      }
+      x[u][0].x -= scale * g0.x; x[u][0].y -= scale * g0.y; x[u][0].z -= scale * g0.z; x[u][0].w -= scale * g0.w;
+      x[u][1].x -= scale * g1.x; x[u][1].y -= scale * g1.y; x[u][1].z -= scale * g1.z; x[u][1].w -= scale * g1.w;
+    }
+    cluster.sync();                              // all remote reads of part[] are done before it is rewritten
+  }
+  // data rows are zero past d, so coordinates past d have stayed zero
+#pragma unroll
+  for (int u = 0; u < 2; ++u) {
+    if (u >= nn) continue;
+    float* xrow = s.X + (int64_t)node[u] * s.pitch + base;
+    *reinterpret_cast<float4*>(xrow) = x[u][0];
+    if (iters > 1) *reinterpret_cast<float4*>(xrow + kSmallThreads * 4) = x[u][1];
+  }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kSmallThreads)
 lsq_small_kernel(StoreView s, LsqView l, const NodeList nodes, int H, float lr, int csize, int iters) {
   cg::cluster_group cluster = cg::this_cluster();
-  const int rank = (int)cluster.block_rank();
+  __shared__ SmallShared sh;
   const NodeDesc nd = nodes.get(blockIdx.x / csize);
-  const int group = nd.node / l.nodes_per_group;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int64_t base = (int64_t)rank * iters * (kSmallThreads * 4) + tid * 4;   // first coordinate of this thread
-  float* xrow = s.X + (int64_t)nd.node * s.pitch + base;
-  const T* A = reinterpret_cast<const T*>(l.A) + (int64_t)group * l.m * s.pitch + base;
-  const float* labels = l.bvec + (int64_t)nd.node * l.m;
+  const int node[2] = {nd.node, nd.node};
+  const uint32_t event[2] = {nd.event, nd.event};
+  lsq_small_steps<T>(cluster, s, l, 1, node, event, H, lr, csize, iters, sh);
+}
 
-  __shared__ int rows[kSmallMaxBatch];
-  __shared__ float red[kSmallThreads / 32][kSmallMaxBatch];
-  __shared__ float part[kSmallMaxBatch];       // this CTA's partial dot products (read by the whole cluster)
-  __shared__ float resid[kSmallMaxBatch];
-
-  float4 x[2];
-  x[0] = *reinterpret_cast<const float4*>(xrow);
-  x[1] = iters > 1 ? *reinterpret_cast<const float4*>(xrow + kSmallThreads * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-  const float scale = lr / (float)l.batch;
-
-  for (int q = 0; q < H; ++q) {
-    if (tid < l.batch) rows[tid] = minibatch_row(tid, group, nd.event + (uint32_t)q, l.m, s.key0, s.key1);
-    __syncthreads();
-    // groups of 8 sampled rows: all loads of a group are issued before the first reduction
-    for (int s0 = 0; s0 < l.batch; s0 += 8) {
-      float4 a0[8], a1[8];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const bool on = s0 + j < l.batch;
-        const T* row = A + (int64_t)rows[on ? s0 + j : 0] * s.pitch;
-        a0[j] = on ? load4_as_float<T>(row) : make_float4(0.f, 0.f, 0.f, 0.f);
-        a1[j] = (on && iters > 1) ? load4_as_float<T>(row + kSmallThreads * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-      }
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        float acc = a0[j].x * x[0].x;
-        acc = fmaf(a0[j].y, x[0].y, acc); acc = fmaf(a0[j].z, x[0].z, acc); acc = fmaf(a0[j].w, x[0].w, acc);
-        acc = fmaf(a1[j].x, x[1].x, acc); acc = fmaf(a1[j].y, x[1].y, acc);
-        acc = fmaf(a1[j].z, x[1].z, acc); acc = fmaf(a1[j].w, x[1].w, acc);
-        acc = warp_sum(acc);
-        if (lane == 0 && s0 + j < l.batch) red[warp][s0 + j] = acc;
-      }
-    }
-    __syncthreads();
-    if (tid < l.batch) {
-      float tot = 0.0f;
-#pragma unroll
-      for (int w = 0; w < kSmallThreads / 32; ++w) tot += red[w][tid];
-      part[tid] = tot;
-    }
-    cluster.sync();                              // every CTA's partial sums are in place
-    if (tid < l.batch) {
-      float tot = 0.0f;
-      for (int r = 0; r < csize; ++r) tot += *cluster.map_shared_rank(&part[tid], r);
-      resid[tid] = row_residual(tot, labels[rows[tid]], l.logistic);
-    }
-    __syncthreads();
-    float4 g0 = make_float4(0.f, 0.f, 0.f, 0.f), g1 = g0;
-    for (int s0 = 0; s0 < l.batch; s0 += 8) {
-      float4 a0[8], a1[8];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const bool on = s0 + j < l.batch;
-        const T* row = A + (int64_t)rows[on ? s0 + j : 0] * s.pitch;
-        a0[j] = on ? load4_as_float<T>(row) : make_float4(0.f, 0.f, 0.f, 0.f);
-        a1[j] = (on && iters > 1) ? load4_as_float<T>(row + kSmallThreads * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-      }
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const float rs = s0 + j < l.batch ? resid[s0 + j] : 0.0f;
-        g0.x = fmaf(rs, a0[j].x, g0.x); g0.y = fmaf(rs, a0[j].y, g0.y); g0.z = fmaf(rs, a0[j].z, g0.z); g0.w = fmaf(rs, a0[j].w, g0.w);
-        g1.x = fmaf(rs, a1[j].x, g1.x); g1.y = fmaf(rs, a1[j].y, g1.y); g1.z = fmaf(rs, a1[j].z, g1.z); g1.w = fmaf(rs, a1[j].w, g1.w);
-      }
-    }
-    x[0].x -= scale * g0.x; x[0].y -= scale * g0.y; x[0].z -= scale * g0.z; x[0].w -= scale * g0.w;
-    x[1].x -= scale * g1.x; x[1].y -= scale * g1.y; x[1].z -= scale * g1.z; x[1].w -= scale * g1.w;
-    cluster.sync();                              // all remote reads of part[] are done before it is rewritten
+// -----------------------------------------------------------------------------------------
+// Sequential gossip on short models in one launch (Section 3, "Sequential model": one interaction per
+// time step). A single cluster walks the list of steps; in each, the two nodes of the pair take their H
+// least-squares steps (the cluster-wide routine above, both nodes sharing its barriers), then the warps
+// of the cluster take one 1024-coordinate block of the blocking interaction each. Models travel between
+// the two phases through global memory; the cluster barriers (release / acquire at cluster scope, after a
+// device-scope fence) order those accesses. Every CTA executes the same number of barriers.
+// -----------------------------------------------------------------------------------------
+template <int BITS>
+__global__ void __launch_bounds__(kSmallThreads)
+lsq_sequence_kernel(StoreView s, LsqView l, const PairList steps, int H, float lr, int csize, int iters,
+                    int responders) {
+  cg::cluster_group cluster = cg::this_cluster();
+  __shared__ SmallShared sh;
+  const int rank = (int)cluster.block_rank();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int64_t blk = (int64_t)rank * (kSmallThreads / 32) + warp;
+  FusedSteps none{};
+  for (int t = 0; t < steps.n; ++t) {
+    const PairDesc pd = steps.get(t);
+    const int node[2] = {pd.a, pd.b};
+    const uint32_t event[2] = {pd.lsa, pd.lsb};
+    lsq_small_steps<float>(cluster, s, l, responders ? 2 : 1, node, event, H, lr, csize, iters, sh);
+    __threadfence();
+    cluster.sync();                              // both models are complete in global memory
+    if (blk < s.nblk) blocking_block<BITS, false>(s, pd, blk, lane, none);
+    __threadfence();
+    cluster.sync();                              // the averaged models are in place for the next step
   }
-  // data rows are zero past d, so coordinates past d have stayed zero
-  *reinterpret_cast<float4*>(xrow) = x[0];
-  if (iters > 1) *reinterpret_cast<float4*>(xrow + kSmallThreads * 4) = x[1];
 }
 
 // -----------------------------------------------------------------------------------------
@@ -475,6 +545,43 @@ cudaError_t launch_local_lsq(const StoreView& s, const LsqView& l, const NodeLis
     *launches += 2;
   }
   return cudaGetLastError();
+}
+
+bool lsq_sequence_supported(const StoreView& s, const LsqView& l) {
+  return s.pitch <= kSmallMaxPitch && l.batch <= kSmallMaxBatch && l.dtype == 0;
+}
+
+cudaError_t launch_lsq_sequence(const StoreView& s, const LsqView& l, const PairList& steps, int H, float lr, int bits,
+                                int responders, cudaStream_t st, int* launches) {
+  if (steps.n == 0) return cudaSuccess;
+  if (!lsq_sequence_supported(s, l)) return cudaErrorInvalidValue;
+  const int slices512 = (int)(s.pitch / (kSmallThreads * 4));
+  const int csize = slices512 <= 8 ? slices512 : slices512 / 2;
+  const int iters = slices512 <= 8 ? 1 : 2;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)csize);            // one cluster walks the whole sequence
+  cfg.blockDim = dim3(kSmallThreads);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)csize;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaErrorInvalidValue;
+  switch (bits) {
+    case 2: e = cudaLaunchKernelEx(&cfg, lsq_sequence_kernel<2>, s, l, steps, H, lr, csize, iters, responders); break;
+    case 3: e = cudaLaunchKernelEx(&cfg, lsq_sequence_kernel<3>, s, l, steps, H, lr, csize, iters, responders); break;
+    case 4: e = cudaLaunchKernelEx(&cfg, lsq_sequence_kernel<4>, s, l, steps, H, lr, csize, iters, responders); break;
+    case 5: e = cudaLaunchKernelEx(&cfg, lsq_sequence_kernel<5>, s, l, steps, H, lr, csize, iters, responders); break;
+    case 6: e = cudaLaunchKernelEx(&cfg, lsq_sequence_kernel<6>, s, l, steps, H, lr, csize, iters, responders); break;
+    case 7: e = cudaLaunchKernelEx(&cfg, lsq_sequence_kernel<7>, s, l, steps, H, lr, csize, iters, responders); break;
+    case 8: e = cudaLaunchKernelEx(&cfg, lsq_sequence_kernel<8>, s, l, steps, H, lr, csize, iters, responders); break;
+    default: return cudaErrorInvalidValue;
+  }
+  ++*launches;
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_sample_pairs(const int32_t* adj_dev, int n, int degree, int max_pairs, uint32_t launch_ctr,
