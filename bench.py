@@ -75,7 +75,7 @@ WORKLOADS = {
                                              lsq_groups=2, lsq_noise_std=float(np.sqrt(0.1)))),
     # small case the CPU checker finishes in seconds
     "complete8_d4096_b8_lsq": dict(n=8, d=4096, topology="complete", degree=0, pairs=1, bits=8, mode=0, H=2, lr=0.05,
-                                   seed=0, cfg=dict(objective=2, lsq_m=64, lsq_batch=16, lsq_dtype=0, lsq_groups=0,
+                                   seed=0, sequence=True, cfg=dict(objective=2, lsq_m=64, lsq_batch=16, lsq_dtype=0, lsq_groups=0,
                                                     lsq_noise_std=float(np.sqrt(0.1)))),
 }
 DEFAULT_WORKLOAD = "ring64_d1m_b4"
@@ -325,6 +325,9 @@ def run_ours(args, wl, name):
     # elementwise (synthetic) objective, on request: the nodes of the pairs step inside the interaction kernel
     fused = (wl["H"] > 0 and wl["cfg"].get("objective") == 1 and not wl.get("step_all") and args.fused)
 
+    # sequential gossip on short models: the whole timed region is one swarm_run_sequence call
+    sequence = bool(wl.get("sequence")) and wl["pairs"] == 1 and wl["mode"] == 0 and not args.stepwise
+
     def step(pairs):
         if fused:
             rc = sw.step(pairs, wl["H"], wl["lr"], wl["bits"], wl["mode"], True)
@@ -365,6 +368,11 @@ def run_ours(args, wl, name):
     ev_mid = []
     ok = 0
     ev0.record(stream)
+    if sequence:
+        seq = np.ascontiguousarray(np.concatenate(launches[W:]), dtype=np.int32)
+        ok |= L.swarm_run_sequence(h, seq.ctypes.data_as(C.POINTER(g.SwarmPair)), len(seq), H, lr, bits, 1)
+        calls = []
+        probes = []
     for i, (_, pp, npp, _, nn, ncount) in enumerate(calls):
         if fused:
             ok |= L.swarm_step(h, pp, npp, H, lr, bits, mode, 1)
@@ -433,7 +441,7 @@ def run_ours(args, wl, name):
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
         "config": {"workload": name, **{k: wl[k] for k in ("n", "d", "topology", "pairs", "bits", "mode", "H")},
-                   "fused_local_steps": bool(fused),
+                   "fused_local_steps": bool(fused), "single_launch_sequence": bool(sequence),
                    "l2": "inputs larger than L2: every launch streams all models it touches from HBM",
                    "replicas": world},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(gpu_launches),
@@ -488,6 +496,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--stepwise", action="store_true",
+                    help="sequential small-model workload: two calls per step instead of one swarm_run_sequence "
+                         "call for the whole timed region")
     ap.add_argument("--fused", action="store_true",
                     help="synthetic-objective workloads: one swarm_step call per step (local steps inside the "
                          "interaction kernel) instead of swarm_local_steps + swarm_interact; measured slower, "

@@ -111,4 +111,62 @@ __device__ __forceinline__ void blocking_block(const StoreView& s, const PairDes
   }
 }
 
+// The same interaction with the block spread over four warps of one CTA (warp j takes sub-block j): for
+// launches too small to fill the GPU, where the length of one warp's instruction chain is what counts.
+// `red` holds 8 floats of shared memory; the four warps meet at named barrier `bar_id` (128 threads).
+// Results are identical to blocking_block: the block maxima are order-independent and every coordinate
+// keeps its rounding uniform.
+template <int BITS>
+__device__ __forceinline__ void blocking_subblock(const StoreView& s, const PairDesc& pd, int64_t blk, int j, int lane,
+                                                  float* red, int bar_id) {
+  float* xa = s.X + (int64_t)pd.a * s.pitch + blk * kBlockCoords + j * kSubCoords + lane * 8;
+  float* xb = s.X + (int64_t)pd.b * s.pitch + blk * kBlockCoords + j * kSubCoords + lane * 8;
+  const f8 va = ld256(xa), vb = ld256(xb);
+  float rho = 0.0f, M = 0.0f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    rho = fmaxf(rho, fabsf(__fsub_rn(va.v[i], vb.v[i])));
+    M = fmaxf(M, fmaxf(fabsf(va.v[i]), fabsf(vb.v[i])));
+  }
+  rho = warp_max_nonneg(rho);
+  M = warp_max_nonneg(M);
+  if (lane == 0) { red[j] = rho; red[4 + j] = M; }
+  asm volatile("bar.sync %0, 128;" :: "r"(bar_id) : "memory");
+  rho = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+  M = fmaxf(fmaxf(red[4], red[5]), fmaxf(red[6], red[7]));
+  const int e = exponent_rule<BITS>(rho, M);
+  const float step = pow2f_exact(e), inv_step = pow2f_exact(-e);
+  constexpr uint32_t mask = (1u << BITS) - 1u;
+  const uint32_t g = (uint32_t)(blk * (kBlockCoords / 8) + j * (kSubCoords / 8) + lane);
+  uint8_t* ca = s.codes + (int64_t)pd.a * s.nblk * kBlockCoords + blk * (kBlockCoords * BITS / 8) +
+                j * (kSubCoords * BITS / 8) + lane * BITS;
+  uint8_t* cb = s.codes + (int64_t)pd.b * s.nblk * kBlockCoords + blk * (kBlockCoords * BITS / 8) +
+                j * (kSubCoords * BITS / 8) + lane * BITS;
+  const uint4 ra = philox4x32_10(g, (uint32_t)pd.a, pd.wa, kStreamRounding, s.key0, s.key1);
+  const uint4 rb = philox4x32_10(g, (uint32_t)pd.b, pd.wb, kStreamRounding, s.key0, s.key1);
+  uint64_t pka = 0, pkb = 0;
+  f8 out;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    int32_t cell_a, cell_b;
+    const int32_t qa = encode_index(va.v[i], inv_step, sr_u16(ra, i), cell_a);
+    const int32_t qb = encode_index(vb.v[i], inv_step, sr_u16(rb, i), cell_b);
+    const uint32_t code_a = (uint32_t)qa & mask, code_b = (uint32_t)qb & mask;
+    pka |= (uint64_t)code_a << (i * BITS);
+    pkb |= (uint64_t)code_b << (i * BITS);
+    const float Qa = __fmul_rn(__int2float_rn(decode_index<BITS>(code_a, cell_b)), step);
+    const float Qb = __fmul_rn(__int2float_rn(decode_index<BITS>(code_b, cell_a)), step);
+    out.v[i] = __fmul_rn(0.5f, __fadd_rn(Qa, Qb));
+  }
+  st256(xa, out);
+  st256(xb, out);
+  store_codes<BITS>(ca, lane, pka);
+  store_codes<BITS>(cb, lane, pkb);
+  if (j == 0 && lane == 0) {
+    s.exps[(int64_t)pd.a * s.nblk + blk] = (int8_t)e;
+    s.exps[(int64_t)pd.b * s.nblk + blk] = (int8_t)e;
+  }
+  // red[] is rewritten only after the next cluster-wide barrier of the caller
+}
+
 }  // namespace swarm

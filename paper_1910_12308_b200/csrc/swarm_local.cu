@@ -250,157 +250,193 @@ __device__ __forceinline__ float4 load4_as_float<__nv_bfloat16>(const __nv_bfloa
                      __uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xFFFF0000u));
 }
 
-// Shared-memory scratch of the short-model least-squares steps, for up to two nodes handled at once.
+// Shared-memory scratch of the short-model least-squares steps of one node.
+constexpr int kRowsAhead = 8;            // local steps whose minibatches are drawn together
 struct SmallShared {
-  int rows[2][kSmallMaxBatch];
-  float red[2][kSmallThreads / 32][kSmallMaxBatch];
-  float part[2][kSmallMaxBatch];       // this CTA's partial dot products (read by the whole cluster)
-  float resid[2][kSmallMaxBatch];
+  int rows[kRowsAhead][kSmallMaxBatch];
+  float label[kRowsAhead][kSmallMaxBatch];
+  float red[kSmallThreads / 32][kSmallMaxBatch];
+  float part[kSmallMaxBatch];          // this CTA's partial dot products (read by the whole cluster)
+  float resid[kSmallMaxBatch];
 };
 
-// H least-squares steps of nn (1 or 2) nodes, executed by a whole cluster; the nodes share the cluster
-// barriers but each keeps the arithmetic order of a node handled alone. Models are read from and written
-// back to global memory; the caller orders those accesses against other CTAs' work.
-template <typename T>
-__device__ __forceinline__ void lsq_small_steps(cg::cluster_group& cluster, const StoreView& s, const LsqView& l,
-                                                int nn, const int (&node)[2], const uint32_t (&event)[2], int H,
-                                                float lr, int csize, int iters, SmallShared& sh) {
-  const int rank = (int)cluster.block_rank();
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int64_t base = (int64_t)rank * iters * (kSmallThreads * 4) + tid * 4;   // first coordinate of this thread
-  float4 x[2][2];
+// Barrier among the `count` threads that use barrier `id` (a multiple of 32 threads, whole warps).
+__device__ __forceinline__ void named_barrier(int id, int count) {
+  asm volatile("bar.sync %0, %1;" :: "r"(id), "r"(count) : "memory");
+}
+
+// Sums over the 32 lanes of G per-lane values at once: at each level a lane keeps one half of its values and
+// hands the other half to its partner, so G rows cost G + 1 (G = 16) shuffles instead of 5 G. Lane and partner
+// are paired as in the xor butterfly of warp_sum (offsets 16, 8, 4, 2, 1), so every sum has the same
+// association, hence the same rounding. Lanes with an even index end up holding the sum of row `row`.
+template <int G>
+__device__ __forceinline__ float reduce_rows(float (&v)[G], int lane, int& row) {
+  row = 0;
+  int offset = 16;
 #pragma unroll
-  for (int u = 0; u < 2; ++u) {
-    x[u][0] = x[u][1] = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (u < nn) {
-      const float* xrow = s.X + (int64_t)node[u] * s.pitch + base;
-      x[u][0] = *reinterpret_cast<const float4*>(xrow);
-      if (iters > 1) x[u][1] = *reinterpret_cast<const float4*>(xrow + kSmallThreads * 4);
+  for (int width = G; width > 1; width >>= 1) {
+    const int half = width >> 1;
+    const bool upper = (lane & offset) != 0;
+#pragma unroll
+    for (int i = 0; i < half; ++i) {
+      const float send = upper ? v[i] : v[i + half];
+      const float keep = upper ? v[i + half] : v[i];
+      v[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, offset);
     }
+    if (upper) row += half;
+    offset >>= 1;
+  }
+  for (; offset > 0; offset >>= 1) v[0] += __shfl_xor_sync(0xFFFFFFFFu, v[0], offset);
+  return v[0];
+}
+
+// H least-squares steps of one node by kSmallThreads threads of every CTA of a cluster (ltid = 0..127 within
+// the CTA; they share named barrier bar_id). Threads with active == false only take part in the cluster
+// barriers, so that several thread groups of a CTA (each with its own node, scratch and named barrier) can
+// run side by side. ITERS = slices of 512 coordinates per CTA. The model is read from and written back to
+// global memory; the caller orders those accesses against other CTAs' work.
+template <typename T, int ITERS>
+__device__ __forceinline__ void lsq_small_steps(cg::cluster_group& cluster, const StoreView& s, const LsqView& l,
+                                                bool active, int node, uint32_t event, int H, float lr, int csize,
+                                                int ltid, int bar_id, SmallShared& sh) {
+  constexpr int G = 16 / ITERS;                  // sampled rows whose loads are in flight together
+  const int rank = (int)cluster.block_rank();
+  const int warp = ltid >> 5, lane = ltid & 31;
+  const int64_t base = (int64_t)rank * ITERS * (kSmallThreads * 4) + ltid * 4;   // first coordinate of this thread
+  const int group = node / l.nodes_per_group;
+  float* xrow = s.X + (int64_t)node * s.pitch + base;
+  const T* A = reinterpret_cast<const T*>(l.A) + (int64_t)group * l.m * s.pitch + base;
+  const float* labels = l.bvec + (int64_t)node * l.m;
+  const bool one_group = l.batch <= G;           // then the rows loaded for the dot products serve the update too
+
+  float4 x[2];
+  x[0] = x[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (active) {
+    x[0] = *reinterpret_cast<const float4*>(xrow);
+    if (ITERS > 1) x[1] = *reinterpret_cast<const float4*>(xrow + kSmallThreads * 4);
   }
   const float scale = lr / (float)l.batch;
+  float4 a0[G], a1[G];
+
+  const int* rows_q = sh.rows[0];
+  auto load_group = [&](int s0) {
+#pragma unroll
+    for (int j = 0; j < G; ++j) {
+      const bool on = s0 + j < l.batch;
+      const T* row = A + (int64_t)rows_q[on ? s0 + j : 0] * s.pitch;
+      a0[j] = on ? load4_as_float<T>(row) : make_float4(0.f, 0.f, 0.f, 0.f);
+      a1[j] = (on && ITERS > 1) ? load4_as_float<T>(row + kSmallThreads * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  };
 
   for (int q = 0; q < H; ++q) {
-    if (tid < l.batch)
-      for (int u = 0; u < nn; ++u)
-        sh.rows[u][tid] = minibatch_row(tid, node[u] / l.nodes_per_group, event[u] + (uint32_t)q, l.m, s.key0, s.key1);
-    __syncthreads();
+    const int qq = q % kRowsAhead;
+    if (active && qq == 0) {
+      // minibatches (they depend on counters only) and their labels for the next kRowsAhead steps
+      const int ahead = min(kRowsAhead, H - q) * l.batch;
+      for (int idx = ltid; idx < ahead; idx += kSmallThreads) {
+        const int dq = idx / l.batch, si = idx - dq * l.batch;
+        const int r = minibatch_row(si, group, event + (uint32_t)(q + dq), l.m, s.key0, s.key1);
+        sh.rows[dq][si] = r;
+        sh.label[dq][si] = labels[r];
+      }
+      named_barrier(bar_id, kSmallThreads);
+    }
+    rows_q = sh.rows[qq];
+    if (active) {
+      for (int s0 = 0; s0 < l.batch; s0 += G) {
+        load_group(s0);
+        float acc[G];
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      if (u >= nn) continue;
-      const T* A = reinterpret_cast<const T*>(l.A) + (int64_t)(node[u] / l.nodes_per_group) * l.m * s.pitch + base;
-      // groups of 8 sampled rows: all loads of a group are issued before the first reduction
-      for (int s0 = 0; s0 < l.batch; s0 += 8) {
-        float4 a0[8], a1[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const bool on = s0 + j < l.batch;
-          const T* row = A + (int64_t)sh.rows[u][on ? s0 + j : 0] * s.pitch;
-          a0[j] = on ? load4_as_float<T>(row) : make_float4(0.f, 0.f, 0.f, 0.f);
-          a1[j] = (on && iters > 1) ? load4_as_float<T>(row + kSmallThreads * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int j = 0; j < G; ++j) {
+          acc[j] = a0[j].x * x[0].x;
+          acc[j] = fmaf(a0[j].y, x[0].y, acc[j]); acc[j] = fmaf(a0[j].z, x[0].z, acc[j]); acc[j] = fmaf(a0[j].w, x[0].w, acc[j]);
+          acc[j] = fmaf(a1[j].x, x[1].x, acc[j]); acc[j] = fmaf(a1[j].y, x[1].y, acc[j]);
+          acc[j] = fmaf(a1[j].z, x[1].z, acc[j]); acc[j] = fmaf(a1[j].w, x[1].w, acc[j]);
         }
+        int row;
+        const float tot = reduce_rows<G>(acc, lane, row);
+        if ((lane & 1) == 0 && s0 + row < l.batch) sh.red[warp][s0 + row] = tot;
+      }
+      named_barrier(bar_id, kSmallThreads);
+      if (ltid < l.batch) {
+        float tot = 0.0f;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          float acc = a0[j].x * x[u][0].x;
-          acc = fmaf(a0[j].y, x[u][0].y, acc); acc = fmaf(a0[j].z, x[u][0].z, acc); acc = fmaf(a0[j].w, x[u][0].w, acc);
-          acc = fmaf(a1[j].x, x[u][1].x, acc); acc = fmaf(a1[j].y, x[u][1].y, acc);
-          acc = fmaf(a1[j].z, x[u][1].z, acc); acc = fmaf(a1[j].w, x[u][1].w, acc);
-          acc = warp_sum(acc);
-          if (lane == 0 && s0 + j < l.batch) sh.red[u][warp][s0 + j] = acc;
-        }
+        for (int w = 0; w < kSmallThreads / 32; ++w) tot += sh.red[w][ltid];
+        sh.part[ltid] = tot;
       }
     }
-    __syncthreads();
-    if (tid < l.batch)
-      for (int u = 0; u < nn; ++u) {
-        float tot = 0.0f;
-#pragma unroll
-        for (int w = 0; w < kSmallThreads / 32; ++w) tot += sh.red[u][w][tid];
-        sh.part[u][tid] = tot;
-      }
     cluster.sync();                              // every CTA's partial sums are in place
-    if (tid < l.batch)
-      for (int u = 0; u < nn; ++u) {
+    if (active) {
+      if (ltid < l.batch) {
+        float v[8];                              // remote reads issued together, summed in rank order
+#pragma unroll
+        for (int r = 0; r < 8; ++r) v[r] = r < csize ? *cluster.map_shared_rank(&sh.part[ltid], r) : 0.0f;
         float tot = 0.0f;
-        for (int r = 0; r < csize; ++r) tot += *cluster.map_shared_rank(&sh.part[u][tid], r);
-        const float* labels = l.bvec + (int64_t)node[u] * l.m;
-        sh.resid[u][tid] = row_residual(tot, labels[sh.rows[u][tid]], l.logistic);
+#pragma unroll
+        for (int r = 0; r < 8; ++r) if (r < csize) tot += v[r];
+        sh.resid[ltid] = row_residual(tot, sh.label[qq][ltid], l.logistic);
       }
-    __syncthreads();
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      if (u >= nn) continue;
-      const T* A = reinterpret_cast<const T*>(l.A) + (int64_t)(node[u] / l.nodes_per_group) * l.m * s.pitch + base;
+      named_barrier(bar_id, kSmallThreads);
       float4 g0 = make_float4(0.f, 0.f, 0.f, 0.f), g1 = g0;
-      for (int s0 = 0; s0 < l.batch; s0 += 8) {
-        float4 a0[8], a1[8];
+      for (int s0 = 0; s0 < l.batch; s0 += G) {
+        if (!one_group) load_group(s0);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const bool on = s0 + j < l.batch;
-          const T* row = A + (int64_t)sh.rows[u][on ? s0 + j : 0] * s.pitch;
-          a0[j] = on ? load4_as_float<T>(row) : make_float4(0.f, 0.f, 0.f, 0.f);
-          a1[j] = (on && iters > 1) ? load4_as_float<T>(row + kSmallThreads * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const float rs = s0 + j < l.batch ? sh.resid[u][s0 + j] : 0.0f;
+        for (int j = 0; j < G; ++j) {
+          const float rs = s0 + j < l.batch ? sh.resid[s0 + j] : 0.0f;
           g0.x = fmaf(rs, a0[j].x, g0.x); g0.y = fmaf(rs, a0[j].y, g0.y); g0.z = fmaf(rs, a0[j].z, g0.z); g0.w = fmaf(rs, a0[j].w, g0.w);
           g1.x = fmaf(rs, a1[j].x, g1.x); g1.y = fmaf(rs, a1[j].y, g1.y); g1.z = fmaf(rs, a1[j].z, g1.z); g1.w = fmaf(rs, a1[j].w, g1.w);
         }
       }
-      x[u][0].x -= scale * g0.x; x[u][0].y -= scale * g0.y; x[u][0].z -= scale * g0.z; x[u][0].w -= scale * g0.w;
-      x[u][1].x -= scale * g1.x; x[u][1].y -= scale * g1.y; x[u][1].z -= scale * g1.z; x[u][1].w -= scale * g1.w;
+      x[0].x -= scale * g0.x; x[0].y -= scale * g0.y; x[0].z -= scale * g0.z; x[0].w -= scale * g0.w;
+      x[1].x -= scale * g1.x; x[1].y -= scale * g1.y; x[1].z -= scale * g1.z; x[1].w -= scale * g1.w;
     }
     cluster.sync();                              // all remote reads of part[] are done before it is rewritten
   }
   // data rows are zero past d, so coordinates past d have stayed zero
-#pragma unroll
-  for (int u = 0; u < 2; ++u) {
-    if (u >= nn) continue;
-    float* xrow = s.X + (int64_t)node[u] * s.pitch + base;
-    *reinterpret_cast<float4*>(xrow) = x[u][0];
-    if (iters > 1) *reinterpret_cast<float4*>(xrow + kSmallThreads * 4) = x[u][1];
+  if (active) {
+    *reinterpret_cast<float4*>(xrow) = x[0];
+    if (ITERS > 1) *reinterpret_cast<float4*>(xrow + kSmallThreads * 4) = x[1];
   }
 }
 
-template <typename T>
+template <typename T, int ITERS>
 __global__ void __launch_bounds__(kSmallThreads)
-lsq_small_kernel(StoreView s, LsqView l, const NodeList nodes, int H, float lr, int csize, int iters) {
+lsq_small_kernel(StoreView s, LsqView l, const NodeList nodes, int H, float lr, int csize) {
   cg::cluster_group cluster = cg::this_cluster();
   __shared__ SmallShared sh;
   const NodeDesc nd = nodes.get(blockIdx.x / csize);
-  const int node[2] = {nd.node, nd.node};
-  const uint32_t event[2] = {nd.event, nd.event};
-  lsq_small_steps<T>(cluster, s, l, 1, node, event, H, lr, csize, iters, sh);
+  lsq_small_steps<T, ITERS>(cluster, s, l, true, nd.node, nd.event, H, lr, csize, threadIdx.x, 1, sh);
 }
 
 // -----------------------------------------------------------------------------------------
 // Sequential gossip on short models in one launch (Section 3, "Sequential model": one interaction per
-// time step). A single cluster walks the list of steps; in each, the two nodes of the pair take their H
-// least-squares steps (the cluster-wide routine above, both nodes sharing its barriers), then the warps
-// of the cluster take one 1024-coordinate block of the blocking interaction each. Models travel between
-// the two phases through global memory; the cluster barriers (release / acquire at cluster scope, after a
-// device-scope fence) order those accesses. Every CTA executes the same number of barriers.
+// time step). A single cluster of 256-thread CTAs walks the list of steps. In each step the two halves of
+// every CTA take the H least-squares steps of the initiator and of the responder side by side (the
+// cluster-wide routine above; a half idles when only the initiator steps); then CTA r < nblk performs the
+// blocking interaction of block r, one sub-block per warp. Models travel between the two phases through
+// global memory; the cluster barriers (release / acquire at cluster scope) order those accesses, all of
+// which are made by CTAs of this one cluster. Every thread executes the same number of cluster barriers.
 // -----------------------------------------------------------------------------------------
-template <int BITS>
-__global__ void __launch_bounds__(kSmallThreads)
-lsq_sequence_kernel(StoreView s, LsqView l, const PairList steps, int H, float lr, int csize, int iters,
-                    int responders) {
+constexpr int kSeqThreads = 2 * kSmallThreads;
+
+template <int BITS, int ITERS>
+__global__ void __launch_bounds__(kSeqThreads)
+lsq_sequence_kernel(StoreView s, LsqView l, const PairList steps, int H, float lr, int csize, int responders) {
   cg::cluster_group cluster = cg::this_cluster();
-  __shared__ SmallShared sh;
+  __shared__ SmallShared sh[2];
+  __shared__ float red[8];
   const int rank = (int)cluster.block_rank();
+  const int half = threadIdx.x / kSmallThreads, ltid = threadIdx.x % kSmallThreads;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int64_t blk = (int64_t)rank * (kSmallThreads / 32) + warp;
-  FusedSteps none{};
   for (int t = 0; t < steps.n; ++t) {
     const PairDesc pd = steps.get(t);
-    const int node[2] = {pd.a, pd.b};
-    const uint32_t event[2] = {pd.lsa, pd.lsb};
-    lsq_small_steps<float>(cluster, s, l, responders ? 2 : 1, node, event, H, lr, csize, iters, sh);
-    __threadfence();
+    const int node = half == 0 ? pd.a : pd.b;
+    const uint32_t event = half == 0 ? pd.lsa : pd.lsb;
+    lsq_small_steps<float, ITERS>(cluster, s, l, half == 0 || responders != 0, node, event, H, lr, csize, ltid,
+                                  1 + half, sh[half]);
     cluster.sync();                              // both models are complete in global memory
-    if (blk < s.nblk) blocking_block<BITS, false>(s, pd, blk, lane, none);
-    __threadfence();
+    if (rank < s.nblk && warp < 4) blocking_subblock<BITS>(s, pd, rank, warp, lane, red, 3);
     cluster.sync();                              // the averaged models are in place for the next step
   }
 }
@@ -527,8 +563,13 @@ cudaError_t launch_local_lsq(const StoreView& s, const LsqView& l, const NodeLis
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaError_t e;
-    if (l.dtype == 1) e = cudaLaunchKernelEx(&cfg, lsq_small_kernel<__nv_bfloat16>, s, l, nodes, H, lr, csize, iters);
-    else e = cudaLaunchKernelEx(&cfg, lsq_small_kernel<float>, s, l, nodes, H, lr, csize, iters);
+    if (l.dtype == 1) {
+      e = iters == 1 ? cudaLaunchKernelEx(&cfg, lsq_small_kernel<__nv_bfloat16, 1>, s, l, nodes, H, lr, csize)
+                     : cudaLaunchKernelEx(&cfg, lsq_small_kernel<__nv_bfloat16, 2>, s, l, nodes, H, lr, csize);
+    } else {
+      e = iters == 1 ? cudaLaunchKernelEx(&cfg, lsq_small_kernel<float, 1>, s, l, nodes, H, lr, csize)
+                     : cudaLaunchKernelEx(&cfg, lsq_small_kernel<float, 2>, s, l, nodes, H, lr, csize);
+    }
     ++*launches;
     return e != cudaSuccess ? e : cudaGetLastError();
   }
@@ -560,7 +601,7 @@ cudaError_t launch_lsq_sequence(const StoreView& s, const LsqView& l, const Pair
   const int iters = slices512 <= 8 ? 1 : 2;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)csize);            // one cluster walks the whole sequence
-  cfg.blockDim = dim3(kSmallThreads);
+  cfg.blockDim = dim3(kSeqThreads);
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -570,16 +611,17 @@ cudaError_t launch_lsq_sequence(const StoreView& s, const LsqView& l, const Pair
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   cudaError_t e = cudaErrorInvalidValue;
+#define SWARM_SEQ_CASE(w)                                                                                      \
+  case w:                                                                                                      \
+    e = iters == 1 ? cudaLaunchKernelEx(&cfg, lsq_sequence_kernel<w, 1>, s, l, steps, H, lr, csize, responders) \
+                   : cudaLaunchKernelEx(&cfg, lsq_sequence_kernel<w, 2>, s, l, steps, H, lr, csize, responders); \
+    break;
   switch (bits) {
-    case 2: e = cudaLaunchKernelEx(&cfg, lsq_sequence_kernel<2>, s, l, steps, H, lr, csize, iters, responders); break;
-    case 3: e = cudaLaunchKernelEx(&cfg, lsq_sequence_kernel<3>, s, l, steps, H, lr, csize, iters, responders); break;
-    case 4: e = cudaLaunchKernelEx(&cfg, lsq_sequence_kernel<4>, s, l, steps, H, lr, csize, iters, responders); break;
-    case 5: e = cudaLaunchKernelEx(&cfg, lsq_sequence_kernel<5>, s, l, steps, H, lr, csize, iters, responders); break;
-    case 6: e = cudaLaunchKernelEx(&cfg, lsq_sequence_kernel<6>, s, l, steps, H, lr, csize, iters, responders); break;
-    case 7: e = cudaLaunchKernelEx(&cfg, lsq_sequence_kernel<7>, s, l, steps, H, lr, csize, iters, responders); break;
-    case 8: e = cudaLaunchKernelEx(&cfg, lsq_sequence_kernel<8>, s, l, steps, H, lr, csize, iters, responders); break;
+    SWARM_SEQ_CASE(2) SWARM_SEQ_CASE(3) SWARM_SEQ_CASE(4) SWARM_SEQ_CASE(5) SWARM_SEQ_CASE(6) SWARM_SEQ_CASE(7)
+    SWARM_SEQ_CASE(8)
     default: return cudaErrorInvalidValue;
   }
+#undef SWARM_SEQ_CASE
   ++*launches;
   return e != cudaSuccess ? e : cudaGetLastError();
 }
