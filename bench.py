@@ -485,7 +485,7 @@ def run_ours(args, wl, name):
 
 # ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel (see profiles/);
 # None until a capture of the current kernel exists.
-TRAFFIC = {"ring64_d1m_b4": 512.5e6}
+TRAFFIC = {"ring64_d1m_b4": 511.1e6}
 
 
 def main():
