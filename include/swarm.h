@@ -241,6 +241,11 @@ enum {
   SWARM_T_A_RECORD = 14   /* 1 double: ||snapshot - mean||^2 at the node's last initiation                  */
 };
 int swarm_get_tensor(swarm_ctx *ctx, int32_t which, int32_t node, void *dst_host, size_t bytes);
+/* The same read queued on the context's stream without waiting: dst_host (pinned memory, or the copy is
+ * not asynchronous) holds the row once swarm_sync, or any other synchronising call issued later, returns.
+ * For callers that consume a result of every step without stalling the launch pipeline. Only rows kept
+ * in device memory: EINVAL for SWARM_T_ADJ, SWARM_T_COUNTERS, SWARM_T_CLOCKS, SWARM_T_A. */
+int swarm_get_tensor_async(swarm_ctx *ctx, int32_t which, int32_t node, void *dst_pinned_host, size_t bytes);
 int swarm_set_tensor(swarm_ctx *ctx, int32_t which, int32_t node, const void *src_host, size_t bytes);
 
 /* Whole-context counters: launch counter of the pair sampler and the "snapshots stale" flag. */

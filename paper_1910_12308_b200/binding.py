@@ -27,7 +27,7 @@ TOPOLOGY = {"complete": TOPO_COMPLETE, "ring": TOPO_RING, "regular": TOPO_REGULA
 EXPORTS = [
     "swarm_set_allocator", "swarm_init", "swarm_local_steps", "swarm_local_steps_geometric", "swarm_interact", "swarm_step", "swarm_run_sequence", "swarm_mean_model",
     "swarm_potential", "swarm_track_staleness", "swarm_aux_potentials", "swarm_configure", "swarm_sample_pairs", "swarm_publish", "swarm_register_publish", "swarm_set_own_prefix", "swarm_get_own_prefix", "swarm_get_buffer_mode",
-    "swarm_set_buffer_mode", "swarm_get_tensor",
+    "swarm_set_buffer_mode", "swarm_get_tensor", "swarm_get_tensor_async",
     "swarm_set_tensor", "swarm_get_state", "swarm_set_state", "swarm_model_ptr", "swarm_set_stream",
     "swarm_sync", "swarm_potential_static", "swarm_kernel_launches", "swarm_last_cuda_error", "swarm_strerror", "swarm_destroy",
 ]
@@ -99,6 +99,7 @@ def load():
         "swarm_get_buffer_mode": (C.c_int, [vp, C.POINTER(i32)]),
         "swarm_set_buffer_mode": (C.c_int, [vp, i32]),
         "swarm_get_tensor": (C.c_int, [vp, i32, i32, vp, C.c_size_t]),
+        "swarm_get_tensor_async": (C.c_int, [vp, i32, i32, vp, C.c_size_t]),
         "swarm_set_tensor": (C.c_int, [vp, i32, i32, vp, C.c_size_t]),
         "swarm_get_state": (C.c_int, [vp, C.POINTER(u32), C.POINTER(i32)]),
         "swarm_set_state": (C.c_int, [vp, u32, i32]),
@@ -329,6 +330,13 @@ class Swarm:
         out = np.empty(count, dtype=dt)
         self._check(self._L.swarm_get_tensor(self._h, which, node, out.ctypes.data, out.nbytes), "swarm_get_tensor")
         return out
+
+    def get_async(self, which, node, out):
+        """Queue the read of a row into `out` (a pinned torch tensor or array of the row's size) without
+        waiting; the data is there after sync(). Returns the C code."""
+        ptr = out.data_ptr() if hasattr(out, "data_ptr") else out.ctypes.data
+        nbytes = out.numel() * out.element_size() if hasattr(out, "numel") else out.nbytes
+        return int(self._L.swarm_get_tensor_async(self._h, which, node, ptr, nbytes))
 
     def set(self, which, node, values):
         dt, count = self._row_spec(which)

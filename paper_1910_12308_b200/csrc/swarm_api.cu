@@ -974,8 +974,12 @@ int swarm_set_state(swarm_ctx* c, uint32_t launch, int32_t b_stale) {
   return SWARM_OK;
 }
 
-static int tensor_access(swarm_ctx* c, int32_t which, int32_t node, void* host, size_t bytes, bool write) {
+static int tensor_access(swarm_ctx* c, int32_t which, int32_t node, void* host, size_t bytes, bool write,
+                         bool wait = true) {
   if (!c || !host) return SWARM_EINVAL;
+  // rows that live in host mirrors or need a conversion pass have no asynchronous form
+  if (!wait && (which == SWARM_T_ADJ || which == SWARM_T_COUNTERS || which == SWARM_T_CLOCKS || which == SWARM_T_A))
+    return SWARM_EINVAL;
   const bool per_node = which != SWARM_T_XSTAR && which != SWARM_T_A;
   if (per_node && (node < 0 || node >= c->n)) return SWARM_ERANGE;
   DeviceGuard guard(c->device);
@@ -1066,12 +1070,15 @@ static int tensor_access(swarm_ctx* c, int32_t which, int32_t node, void* host, 
   // the copy is ordered after earlier work by the stream; one synchronisation at the end is enough
   if (write) SW_CUDA(c, cudaMemcpyAsync(dev, host, bytes, cudaMemcpyHostToDevice, c->stream));
   else SW_CUDA(c, cudaMemcpyAsync(host, dev, bytes, cudaMemcpyDeviceToHost, c->stream));
-  SW_CUDA(c, cudaStreamSynchronize(c->stream));
+  if (wait) SW_CUDA(c, cudaStreamSynchronize(c->stream));
   return SWARM_OK;
 }
 
 int swarm_get_tensor(swarm_ctx* c, int32_t which, int32_t node, void* dst, size_t bytes) {
   return tensor_access(c, which, node, dst, bytes, false);
+}
+int swarm_get_tensor_async(swarm_ctx* c, int32_t which, int32_t node, void* dst, size_t bytes) {
+  return tensor_access(c, which, node, dst, bytes, false, false);
 }
 int swarm_set_tensor(swarm_ctx* c, int32_t which, int32_t node, const void* src, size_t bytes) {
   return tensor_access(c, which, node, const_cast<void*>(src), bytes, true);

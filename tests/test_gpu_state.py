@@ -72,3 +72,19 @@ def test_non_default_stream():
     assert np.array_equal(sw.get_all(g.T_X), ref.get_all(g.T_X))
     assert np.array_equal(mu.cpu().numpy(), ref.mean_model().cpu().numpy())
     assert sw.potential() == ref.potential()
+
+
+def test_asynchronous_row_read_arrives_after_sync():
+    import torch
+    sw = g.Swarm(4, 3000, "complete", 0, 2)
+    sw.configure(objective=1, grad_std=0.1, offset_std=0.2)
+    out = torch.zeros(3000, dtype=torch.float32).pin_memory()
+    exps = torch.zeros(sw.nblk, dtype=torch.int8).pin_memory()
+    assert sw.interact([[0, 1]], 8) == 0
+    assert sw.get_async(g.T_X, 1, out) == 0 and sw.get_async(g.T_EXPS, 1, exps) == 0
+    sw.sync()
+    assert np.array_equal(out.numpy(), sw.get(g.T_X, 1)) and np.array_equal(exps.numpy(), sw.get(g.T_EXPS, 1))
+    small = torch.zeros(3, dtype=torch.uint32).pin_memory() if hasattr(torch, "uint32") else np.zeros(3, np.uint32)
+    assert sw.get_async(g.T_COUNTERS, 0, small) == g.EINVAL          # host-side rows have no asynchronous form
+    assert sw.get_async(g.T_X, 9, out) == g.ERANGE
+    assert sw.get_async(g.T_X, 0, exps) == g.EINVAL                  # size mismatch
