@@ -27,7 +27,8 @@ def random_sequence(n, steps, seed):
 
 
 @pytest.mark.parametrize("responders", [True, False])
-@pytest.mark.parametrize("d,bits,steps", [(4096, 8, 150), (1500, 3, 40), (8192, 4, 30), (5000, 8, 70), (700, 6, 10)])
+@pytest.mark.parametrize("d,bits,steps", [(4096, 8, 150), (1500, 3, 40), (8192, 4, 30), (5000, 8, 70), (700, 6, 10),
+                                           (900, 2, 12), (2100, 5, 12), (3000, 7, 12)])
 def test_sequence_equals_the_steps_one_by_one(d, bits, steps, responders):
     n = 8
     two = g.Swarm(n, d, "complete", 0, 21)
