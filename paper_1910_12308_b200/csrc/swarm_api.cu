@@ -67,7 +67,8 @@ struct swarm_ctx {
   int* kernel_status = nullptr;      // set by a kernel whose bounded wait expired
   int* kernel_status_host = nullptr; // pinned
   double* pot_partial = nullptr;
-  double* pot_out = nullptr;         // 4 doubles
+  double* pot_out = nullptr;         // 4 doubles, then the ticket counter of the potential kernel
+  double* pot_host_dev = nullptr;    // device-visible address of pot_host (nullptr: not mapped)
   // auxiliary potentials of the staleness analysis (off until swarm_track_staleness)
   bool track = false;
   float* mu_hist = nullptr;          // [n][pitch] mean model at each node's last initiation
@@ -458,7 +459,7 @@ int swarm_init(swarm_ctx** out, int32_t n, int64_t d, swarm_topology topo, uint6
   c->adj_dev = (int32_t*)dev_alloc(c, c->adj.size() * sizeof(int32_t));
   c->scalars = (float*)dev_alloc(c, (size_t)n * 3 * sizeof(float));
   c->pot_partial = (double*)dev_alloc(c, (size_t)potential_partials(d) * sizeof(double));
-  c->pot_out = (double*)dev_alloc(c, 4 * sizeof(double));
+  c->pot_out = (double*)dev_alloc(c, 5 * sizeof(double));
   c->pairs_out_dev = (int32_t*)dev_alloc(c, (2 * max_pairs + 1) * sizeof(int32_t));
   c->used_dev = (uint8_t*)dev_alloc(c, (size_t)n);
   c->kernel_status = (int*)dev_alloc(c, sizeof(int));
@@ -467,6 +468,12 @@ int swarm_init(swarm_ctx** out, int32_t n, int64_t d, swarm_topology topo, uint6
             c->pairs_out_dev && c->used_dev && c->stage_dev && c->kernel_status;
   ok = ok && cudaMallocHost(&c->stage_host, c->stage_slot_bytes * kStageSlots) == cudaSuccess;
   ok = ok && cudaMallocHost((void**)&c->pot_host, 4 * sizeof(double)) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(c->pot_out, 0, 5 * sizeof(double), c->stream) == cudaSuccess;
+  if (ok) {   // the potential kernel writes its result straight to the pinned host word when that is mapped
+    void* mapped = nullptr;
+    if (cudaHostGetDevicePointer(&mapped, c->pot_host, 0) == cudaSuccess) c->pot_host_dev = (double*)mapped;
+    else cudaGetLastError();
+  }
   ok = ok && cudaMallocHost((void**)&c->kernel_status_host, sizeof(int)) == cudaSuccess;
   ok = ok && cudaMemsetAsync(c->kernel_status, 0, sizeof(int), c->stream) == cudaSuccess;
   ok = ok && cudaMallocHost((void**)&c->pairs_out_host, (2 * max_pairs + 1) * sizeof(int32_t)) == cudaSuccess;
@@ -934,9 +941,11 @@ int swarm_potential(swarm_ctx* c, double* out_gamma) {
   if (!c || !out_gamma) return SWARM_EINVAL;
   DeviceGuard guard(c->device);
   int nl = 0;
-  SW_CUDA(c, launch_potential(view_of(c), c->pot_partial, c->pot_out, c->stream, &nl));
+  SW_CUDA(c, launch_potential(view_of(c), c->pot_partial, (unsigned int*)(c->pot_out + 4), c->pot_out, c->pot_host_dev,
+                              c->stream, &nl));
   c->launches += nl;
-  SW_CUDA(c, cudaMemcpyAsync(c->pot_host, c->pot_out, sizeof(double), cudaMemcpyDeviceToHost, c->stream));
+  if (!c->pot_host_dev)
+    SW_CUDA(c, cudaMemcpyAsync(c->pot_host, c->pot_out, sizeof(double), cudaMemcpyDeviceToHost, c->stream));
   SW_CUDA(c, cudaStreamSynchronize(c->stream));
   *out_gamma = *c->pot_host;
   return SWARM_OK;

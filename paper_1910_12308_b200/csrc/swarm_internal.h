@@ -130,9 +130,10 @@ cudaError_t launch_sample_pairs(const int32_t* adj_dev, int n, int degree, int m
 
 // --- swarm_reduce.cu ---------------------------------------------------------------------
 cudaError_t launch_mean_model(const StoreView& s, float* out_dev, cudaStream_t st, int* launches);
-// partial_dev: potential_partials(d) doubles of scratch; out_dev: one double.
-cudaError_t launch_potential(const StoreView& s, double* partial_dev, double* out_dev, cudaStream_t st,
-                             int* launches);
+// partial_dev: potential_partials(d) doubles of scratch; ticket_dev: one zero-initialised counter (left at
+// zero); out_dev: one double; out_host_mapped: device-visible address of a pinned host double, or nullptr.
+cudaError_t launch_potential(const StoreView& s, double* partial_dev, unsigned int* ticket_dev, double* out_dev,
+                             double* out_host_mapped, cudaStream_t st, int* launches);
 int64_t potential_partials(int64_t d);
 // Staleness tracking. mu_hist_dev: [n][pitch] mean-model records; a_hist_dev: n doubles;
 // partial_dev: list.n * potential_partials(d) doubles (record) or 2 * potential_partials(d) (query).

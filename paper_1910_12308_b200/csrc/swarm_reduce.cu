@@ -1,11 +1,14 @@
 // Mean model mu = (1/n) sum_i X^i and potential Gamma = sum_i ||X^i - mu||^2 (Section 4).
 // Both stream X[n][d] once: a thread owns 4 adjacent columns and walks down the n rows.
+#include <algorithm>
+
 #include "swarm_dev.cuh"
 #include "swarm_internal.h"
 
 namespace swarm {
 
 constexpr int kRedThreads = 128;
+constexpr int kPotentialMaxCtas = 148 * 16;   // one resident wave of 128-thread CTAs on 148 SMs
 constexpr int kRowUnroll = 8;
 
 // mu[k]: rows summed in double in row order, divided by n, rounded once.
@@ -37,13 +40,18 @@ mean_model_kernel(StoreView s, float* __restrict__ out) {
 
 // Per column, with the first row as shift (exact in double): s_i = x_i - x_0,
 // Gamma_col = sum s_i^2 - (sum s_i)^2 / n. The shift keeps the subtraction benign when the
-// models are close to each other but far from the origin. CTA partials go to scratch and are
-// summed by a second, single-CTA kernel in index order.
+// models are close to each other but far from the origin. CTA partials go to scratch.
+// The CTA that finishes last (a ticket counter tells) sums the partials in a fixed pattern, so the result
+// does not depend on which CTA that is, writes it to out_dev and, when out_host is given (pinned host
+// memory mapped into the device's address space), to the host directly, and resets the ticket.
 __global__ void __launch_bounds__(kRedThreads)
-potential_partial_kernel(StoreView s, double* __restrict__ partial) {
-  const int64_t c4 = (int64_t)blockIdx.x * kRedThreads + threadIdx.x;
+potential_partial_kernel(StoreView s, double* __restrict__ partial, unsigned int* __restrict__ ticket,
+                         double* __restrict__ out_dev, double* __restrict__ out_host) {
   double gamma = 0.0;
-  if (c4 * 4 < s.d) {
+  // a fixed number of CTAs walks the column groups, so the sum of a CTA (and with it the result) depends on
+  // the grid size only, and the last CTA has few partials to add up
+  for (int64_t c4 = (int64_t)blockIdx.x * kRedThreads + threadIdx.x; c4 * 4 < s.d;
+       c4 += (int64_t)gridDim.x * kRedThreads) {
     const float* col = s.X + c4 * 4;
     const float4 x0 = *reinterpret_cast<const float4*>(col);
     const double b0 = x0.x, b1 = x0.y, b2 = x0.z, b3 = x0.w;
@@ -72,6 +80,7 @@ potential_partial_kernel(StoreView s, double* __restrict__ partial) {
       gamma += sq[t] - sm[t] * sm[t] * inv_n;
   }
   __shared__ double red[kRedThreads / 32];
+  __shared__ bool last;
   gamma = warp_sum(gamma);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = gamma;
   __syncthreads();
@@ -80,21 +89,25 @@ potential_partial_kernel(StoreView s, double* __restrict__ partial) {
 #pragma unroll
     for (int w = 0; w < kRedThreads / 32; ++w) tot += red[w];
     partial[blockIdx.x] = tot;
+    __threadfence();                                     // the partial is visible before the ticket is taken
+    last = atomicAdd(ticket, 1u) == gridDim.x - 1;
   }
-}
-
-__global__ void __launch_bounds__(1024)
-potential_final_kernel(const double* __restrict__ partial, int64_t count, double* __restrict__ out) {
+  __syncthreads();
+  if (!last) return;
+  __threadfence();
   double acc = 0.0;
-  for (int64_t i = threadIdx.x; i < count; i += 1024) acc += partial[i];
-  __shared__ double red[32];
+  for (int64_t i = threadIdx.x; i < (int64_t)gridDim.x; i += kRedThreads) acc += __ldcg(partial + i);
   acc = warp_sum(acc);
+  __syncthreads();                                       // red[] was read above
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
   __syncthreads();
-  if (threadIdx.x < 32) {
-    double v = red[threadIdx.x];
-    v = warp_sum(v);
-    if (threadIdx.x == 0) *out = v;
+  if (threadIdx.x == 0) {
+    double tot = 0.0;
+#pragma unroll
+    for (int w = 0; w < kRedThreads / 32; ++w) tot += red[w];
+    *out_dev = tot;
+    if (out_host) *out_host = tot;
+    *ticket = 0u;
   }
 }
 
@@ -238,12 +251,11 @@ cudaError_t launch_mean_model(const StoreView& s, float* out_dev, cudaStream_t s
   return cudaGetLastError();
 }
 
-cudaError_t launch_potential(const StoreView& s, double* partial_dev, double* out_dev, cudaStream_t st,
-                             int* launches) {
-  const int64_t parts = potential_partials(s.d);
-  potential_partial_kernel<<<(unsigned)parts, kRedThreads, 0, st>>>(s, partial_dev);
-  potential_final_kernel<<<1, 1024, 0, st>>>(partial_dev, parts, out_dev);
-  *launches += 2;
+cudaError_t launch_potential(const StoreView& s, double* partial_dev, unsigned int* ticket_dev, double* out_dev,
+                             double* out_host_mapped, cudaStream_t st, int* launches) {
+  const int64_t parts = std::min<int64_t>(potential_partials(s.d), kPotentialMaxCtas);
+  potential_partial_kernel<<<(unsigned)parts, kRedThreads, 0, st>>>(s, partial_dev, ticket_dev, out_dev, out_host_mapped);
+  ++*launches;
   return cudaGetLastError();
 }
 
