@@ -244,7 +244,9 @@ int swarm_get_tensor(swarm_ctx *ctx, int32_t which, int32_t node, void *dst_host
 /* The same read queued on the context's stream without waiting: dst_host (pinned memory, or the copy is
  * not asynchronous) holds the row once swarm_sync, or any other synchronising call issued later, returns.
  * For callers that consume a result of every step without stalling the launch pipeline. Only rows kept
- * in device memory: EINVAL for SWARM_T_ADJ, SWARM_T_COUNTERS, SWARM_T_CLOCKS, SWARM_T_A. */
+ * in device memory: EINVAL for SWARM_T_ADJ, SWARM_T_COUNTERS, SWARM_T_CLOCKS, SWARM_T_A. Rows of up to 64 KiB
+ * going to pinned memory that the device can address are written by a small kernel rather than the copy
+ * engine, which keeps back-to-back interaction launches overlapping their launch latency. */
 int swarm_get_tensor_async(swarm_ctx *ctx, int32_t which, int32_t node, void *dst_pinned_host, size_t bytes);
 int swarm_set_tensor(swarm_ctx *ctx, int32_t which, int32_t node, const void *src_host, size_t bytes);
 

@@ -1077,6 +1077,17 @@ static int tensor_access(swarm_ctx* c, int32_t which, int32_t node, void* host, 
   }
   if (bytes != want) return SWARM_EINVAL;
   // the copy is ordered after earlier work by the stream; one synchronisation at the end is enough
+  if (!write && !wait && bytes <= (64u << 10)) {
+    // short queued read into pinned memory that the device can address: a small kernel instead of the copy engine
+    void* mapped = nullptr;
+    if (cudaHostGetDevicePointer(&mapped, host, 0) == cudaSuccess && mapped) {
+      int nl = 0;
+      SW_CUDA(c, launch_row_to_host(dev, mapped, (int64_t)bytes, c->stream, &nl));
+      c->launches += nl;
+      return SWARM_OK;
+    }
+    cudaGetLastError();   // pageable or unmapped destination: the copy engine takes it
+  }
   if (write) SW_CUDA(c, cudaMemcpyAsync(dev, host, bytes, cudaMemcpyHostToDevice, c->stream));
   else SW_CUDA(c, cudaMemcpyAsync(host, dev, bytes, cudaMemcpyDeviceToHost, c->stream));
   if (wait) SW_CUDA(c, cudaStreamSynchronize(c->stream));

@@ -1,6 +1,7 @@
 // State generation, local SGD steps (Section 3, "The Communication Procedure": H sequential
 // stochastic gradient steps, each at the running iterate) and the pair sampler (Algorithm 1,
 // sampling lines).
+#include <algorithm>
 #include <cooperative_groups.h>
 #include <cuda_bf16.h>
 
@@ -482,6 +483,17 @@ sample_pairs_kernel(const int32_t* __restrict__ adj, int n, int degree, int max_
   if (threadIdx.x == 0) *out_count = count_sh;
 }
 
+// Small row read-back into pinned host memory that is mapped into the device's address space: a kernel
+// instead of a copy-engine transfer, launched as a programmatic dependent, so that a row read queued
+// between two interaction launches does not cost them the overlap of launch latency.
+__global__ void __launch_bounds__(256)
+row_to_host_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst_host, int64_t bytes) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < bytes; i += (int64_t)gridDim.x * blockDim.x)
+    dst_host[i] = src[i];
+}
+
 __global__ void bf16_to_f32_kernel(const __nv_bfloat16* src, float* dst, int64_t count) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i < count) dst[i] = __bfloat162float(src[i]);
@@ -633,6 +645,23 @@ cudaError_t launch_sample_pairs(const int32_t* adj_dev, int n, int degree, int m
                                          out_count_dev, used_dev);
   ++*launches;
   return cudaGetLastError();
+}
+
+cudaError_t launch_row_to_host(const void* src_dev, void* dst_host_mapped, int64_t bytes, cudaStream_t st,
+                               int* launches) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)std::min<int64_t>(cdiv(bytes, 256), 64));
+  cfg.blockDim = dim3(256);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, row_to_host_kernel, reinterpret_cast<const uint8_t*>(src_dev),
+                                           reinterpret_cast<uint8_t*>(dst_host_mapped), bytes);
+  ++*launches;
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_bf16_to_f32(const void* src, float* dst, int64_t count, cudaStream_t st, int* launches) {
