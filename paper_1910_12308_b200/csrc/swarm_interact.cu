@@ -279,7 +279,7 @@ publish_encode_kernel(StoreView s, const uint32_t* __restrict__ wctr, int64_t to
 //   X_a <- Q(X_a)/2 + Q(X_b)/2 - (B_a - X_a);  B_a <- X_a;  O_a, P_a <- Enc(X_a);  P_b <- Enc(average)
 // Traffic per coordinate: 8 + 4 + 2b/8 B read, 8 + 2 + 2b/8 B written.
 // -----------------------------------------------------------------------------------------
-constexpr int kOwnBits = 16;
+// own registers hold 16-bit colours (two byte planes)
 constexpr int kOwnResolutionBits = 8;
 
 // Own registers are stored in two byte planes per 1024-coordinate block (1024 low bytes, then 1024 high
