@@ -41,6 +41,13 @@ def test_argument_validation_needs_no_device():
     assert L.swarm_init(None, 4, 16, g.SwarmTopology(0, 0), 0) == -1
     assert L.swarm_interact(None, None, 0, 8, 0) == -1
     assert L.swarm_potential(None, None) == -1
+    assert L.swarm_step(None, None, 0, 1, 0.1, 8, 0, 1) == -1
+    assert L.swarm_run_sequence(None, None, 0, 1, 0.1, 8, 1) == -1
+    assert L.swarm_set_own_prefix(None, 8) == -1 and L.swarm_get_own_prefix(None, None) == -1
+    assert L.swarm_track_staleness(None, 1) == -1 and L.swarm_aux_potentials(None, None) == -1
+    assert L.swarm_get_tensor_async(None, 0, 0, None, 0) == -1
+    out = C.c_double()
+    assert L.swarm_potential_static(None, 4, 16, 16, C.addressof(out), None) == -1
 
 
 def test_no_cpu_fallback():
