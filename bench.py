@@ -34,6 +34,9 @@ WORKLOADS = {
                           cfg=dict(offset_std=float(np.sqrt(0.1)))),
     "ring64_d1m_b7": dict(n=64, d=1 << 20, topology="ring", degree=0, pairs=32, bits=7, mode=0, H=0, lr=0.0, seed=2,
                           cfg=dict(offset_std=float(np.sqrt(0.1)))),
+    # identity quantizer (Corollary 2): plain averaging, 16 bytes per coordinate pair
+    "ring64_d1m_identity": dict(n=64, d=1 << 20, topology="ring", degree=0, pairs=32, bits=32, mode=0, H=0, lr=0.0,
+                                seed=2, cfg=dict(offset_std=float(np.sqrt(0.1)))),
     # n = 16 nodes, d = 25,557,032 (ResNet-50 sized), complete graph, 8 pairs, synthetic-gradient steps.
     "complete16_resnet50_b8": dict(n=16, d=25_557_032, topology="complete", degree=0, pairs=8, bits=8, mode=0, H=2,
                                    lr=0.05, seed=4, cfg=dict(objective=1, grad_std=float(np.sqrt(1e-3)),
@@ -92,6 +95,8 @@ def interaction_bytes(d, bits, mode):
     """Algorithmic bytes one interaction must move: blocking reads two models, writes two models and
     two packed buffers; non-blocking reads model + snapshot + two buffers and writes the same."""
     nblk = (d + 1023) // 1024
+    if mode == 0 and bits == 32:
+        return d * 16
     if mode == 0:
         return d * 16 + 2 * d * bits // 8 + 2 * nblk
     if mode == 1:
@@ -453,7 +458,8 @@ def run_ours(args, wl, name):
                    "l2": "inputs larger than L2: every launch streams all models it touches from HBM",
                    "replicas": world},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(gpu_launches),
-        "roofline": {"bound": "hbm", "kernel": ["interact_blocking_kernel", "interact_nonblocking_kernel", "interact_registers_kernel"][wl["mode"]]
+        "roofline": {"bound": "hbm", "kernel": ("interact_identity_kernel" if wl["bits"] == 32 else
+                                ["interact_blocking_kernel", "interact_nonblocking_kernel", "interact_registers_kernel"][wl["mode"]])
                      + (" (local steps fused)" if fused else ""),
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": peak_kind, "frac_of_8000": achieved / 8000.0, "traffic": TRAFFIC.get(name),

@@ -62,12 +62,23 @@ interact_blocking_kernel(StoreView s, const PairList pairs, int64_t total_warps,
 // Identity quantizer (Corollary 2): plain averaging, buffers untouched.
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
 interact_identity_kernel(StoreView s, const PairList pairs, int64_t total_warps, const FusedSteps fs) {
+  grid_dependency_signal();
+  grid_dependency_wait();
   const int lane = threadIdx.x & 31;
   const int64_t warp = (int64_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
   if (warp >= total_warps) return;
   const int64_t pair = warp / s.nblk;
   const int64_t blk = warp - pair * s.nblk;
   const PairDesc pd = pairs.get(pair);
+  {
+    const int64_t w2 = warp + kPrefetchDistance;
+    if (w2 < total_warps) {
+      const int64_t pair2 = w2 / s.nblk, blk2 = w2 - pair2 * s.nblk;
+      const PairDesc p2 = pairs.get(pair2);
+      prefetch_l2(s.X + (int64_t)p2.a * s.pitch + blk2 * kBlockCoords + lane * 32);
+      prefetch_l2(s.X + (int64_t)p2.b * s.pitch + blk2 * kBlockCoords + lane * 32);
+    }
+  }
   float* xa = s.X + (int64_t)pd.a * s.pitch + blk * kBlockCoords + lane * 8;
   float* xb = s.X + (int64_t)pd.b * s.pitch + blk * kBlockCoords + lane * 8;
   f8 va[kSub], vb[kSub];
@@ -545,7 +556,7 @@ cudaError_t launch_interact_blocking(const StoreView& s, const PairList& pairs, 
   const dim3 grid(ctas_for(warps)), block(kWarpsPerCta * 32);
   cudaError_t e = cudaSuccess;
   if (bits == 32) {
-    interact_identity_kernel<<<grid, block, 0, st>>>(s, pairs, warps, fs);
+    e = launch_dependent(interact_identity_kernel, grid, block, st, s, pairs, warps, fs);
   } else {
     SWARM_FOR_WIDTH(bits, e = (fs.H > 0 ? launch_dependent(interact_blocking_kernel<W, true>, grid, block, st, s, pairs, warps, fs)
                                          : launch_dependent(interact_blocking_kernel<W, false>, grid, block, st, s, pairs, warps, fs)))
