@@ -43,6 +43,42 @@ __device__ __forceinline__ void fused_steps_responder(const StoreView& s, const 
   for (int j = 0; j < kSub; ++j) st256(xb + j * kSubCoords, vb[j]);
 }
 
+// Encode / cross-decode / average / store phase of a blocking block, in the fast or the defining form of
+// the lattice arithmetic (LatticeOps).
+template <int BITS, bool FAST>
+__device__ __forceinline__ void blocking_exchange(const f8 (&va)[kSub], const f8 (&vb)[kSub], float* xa, float* xb,
+                                                  uint8_t* ca, uint8_t* cb, uint32_t group0, const StoreView& s,
+                                                  const PairDesc& pd, int lane, int e) {
+  using Ops = LatticeOps<FAST>;
+  const float step = pow2f_exact(e), inv_step = pow2f_exact(-e);
+  const float unbias = FAST ? -__fmul_rn(kCellBias, step) : 0.0f;
+  constexpr uint32_t mask = (1u << BITS) - 1u;
+#pragma unroll
+  for (int j = 0; j < kSub; ++j) {
+    const uint32_t g = group0 + j * (kSubCoords / 8);
+    const uint4 ra = philox4x32_10(g, (uint32_t)pd.a, pd.wa, kStreamRounding, s.key0, s.key1);
+    const uint4 rb = philox4x32_10(g, (uint32_t)pd.b, pd.wb, kStreamRounding, s.key0, s.key1);
+    uint64_t pka = 0, pkb = 0;
+    f8 out;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      uint32_t cell_a, cell_b;
+      const uint32_t code_a = Ops::encode(va[j].v[i], inv_step, sr_word(ra, i), i & 1, cell_a) & mask;
+      const uint32_t code_b = Ops::encode(vb[j].v[i], inv_step, sr_word(rb, i), i & 1, cell_b) & mask;
+      pka |= (uint64_t)code_a << (i * BITS);
+      pkb |= (uint64_t)code_b << (i * BITS);
+      // b decodes a's codes with X^b as key and vice versa; the key's cell is already known
+      const float Qa = Ops::value(Ops::template decode<BITS>(code_a, cell_b), step, unbias);
+      const float Qb = Ops::value(Ops::template decode<BITS>(code_b, cell_a), step, unbias);
+      out.v[i] = __fmul_rn(0.5f, __fadd_rn(Qa, Qb));
+    }
+    st256(xa + j * kSubCoords, out);
+    st256(xb + j * kSubCoords, out);
+    store_codes<BITS>(ca + j * (kSubCoords * BITS / 8), lane, pka);
+    store_codes<BITS>(cb + j * (kSubCoords * BITS / 8), lane, pkb);
+  }
+}
+
 // Blocking interaction of one block (Algorithm 1, interaction lines, with both models present): exact
 // range of X^a - X^b gives the common exponent; both models are encoded into their buffers; each side
 // decodes the partner's codes against its own model and both adopt Q(X^a)/2 + Q(X^b)/2.
@@ -73,42 +109,42 @@ __device__ __forceinline__ void blocking_block(const StoreView& s, const PairDes
   rho = warp_max_nonneg(rho);
   M = warp_max_nonneg(M);
   const int e = exponent_rule<BITS>(rho, M);
-  const float step = pow2f_exact(e), inv_step = pow2f_exact(-e);
 
-  constexpr uint32_t mask = (1u << BITS) - 1u;
   const uint32_t group0 = (uint32_t)(blk * (kBlockCoords / 8) + lane);   // generator call index of sub-block 0
   uint8_t* ca = s.codes + (int64_t)pd.a * s.nblk * kBlockCoords + blk * (kBlockCoords * BITS / 8) + lane * BITS;
   uint8_t* cb = s.codes + (int64_t)pd.b * s.nblk * kBlockCoords + blk * (kBlockCoords * BITS / 8) + lane * BITS;
-
-#pragma unroll
-  for (int j = 0; j < kSub; ++j) {
-    const uint32_t g = group0 + j * (kSubCoords / 8);
-    const uint4 ra = philox4x32_10(g, (uint32_t)pd.a, pd.wa, kStreamRounding, s.key0, s.key1);
-    const uint4 rb = philox4x32_10(g, (uint32_t)pd.b, pd.wb, kStreamRounding, s.key0, s.key1);
-    uint64_t pka = 0, pkb = 0;
-    f8 out;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      int32_t cell_a, cell_b;
-      const int32_t qa = encode_index(va[j].v[i], inv_step, sr_u16(ra, i), cell_a);
-      const int32_t qb = encode_index(vb[j].v[i], inv_step, sr_u16(rb, i), cell_b);
-      const uint32_t code_a = (uint32_t)qa & mask, code_b = (uint32_t)qb & mask;
-      pka |= (uint64_t)code_a << (i * BITS);
-      pkb |= (uint64_t)code_b << (i * BITS);
-      // b decodes a's codes with X^b as key and vice versa; the key's cell is already known
-      const float Qa = __fmul_rn(__int2float_rn(decode_index<BITS>(code_a, cell_b)), step);
-      const float Qb = __fmul_rn(__int2float_rn(decode_index<BITS>(code_b, cell_a)), step);
-      out.v[i] = __fmul_rn(0.5f, __fadd_rn(Qa, Qb));
-    }
-    st256(xa + j * kSubCoords, out);
-    st256(xb + j * kSubCoords, out);
-    store_codes<BITS>(ca + j * (kSubCoords * BITS / 8), lane, pka);
-    store_codes<BITS>(cb + j * (kSubCoords * BITS / 8), lane, pkb);
-  }
+  if (fast_range(M, pow2f_exact(-e), e)) blocking_exchange<BITS, true>(va, vb, xa, xb, ca, cb, group0, s, pd, lane, e);
+  else blocking_exchange<BITS, false>(va, vb, xa, xb, ca, cb, group0, s, pd, lane, e);
   if (lane == 0) {
     s.exps[(int64_t)pd.a * s.nblk + blk] = (int8_t)e;
     s.exps[(int64_t)pd.b * s.nblk + blk] = (int8_t)e;
   }
+}
+
+template <int BITS, bool FAST>
+__device__ __forceinline__ void subblock_exchange(const f8& va, const f8& vb, float* xa, float* xb, uint8_t* ca,
+                                                  uint8_t* cb, const uint4& ra, const uint4& rb, int lane, int e) {
+  using Ops = LatticeOps<FAST>;
+  const float step = pow2f_exact(e), inv_step = pow2f_exact(-e);
+  const float unbias = FAST ? -__fmul_rn(kCellBias, step) : 0.0f;
+  constexpr uint32_t mask = (1u << BITS) - 1u;
+  uint64_t pka = 0, pkb = 0;
+  f8 out;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    uint32_t cell_a, cell_b;
+    const uint32_t code_a = Ops::encode(va.v[i], inv_step, sr_word(ra, i), i & 1, cell_a) & mask;
+    const uint32_t code_b = Ops::encode(vb.v[i], inv_step, sr_word(rb, i), i & 1, cell_b) & mask;
+    pka |= (uint64_t)code_a << (i * BITS);
+    pkb |= (uint64_t)code_b << (i * BITS);
+    const float Qa = Ops::value(Ops::template decode<BITS>(code_a, cell_b), step, unbias);
+    const float Qb = Ops::value(Ops::template decode<BITS>(code_b, cell_a), step, unbias);
+    out.v[i] = __fmul_rn(0.5f, __fadd_rn(Qa, Qb));
+  }
+  st256(xa, out);
+  st256(xb, out);
+  store_codes<BITS>(ca, lane, pka);
+  store_codes<BITS>(cb, lane, pkb);
 }
 
 // The same interaction with the block spread over four warps of one CTA (warp j takes sub-block j): for
@@ -135,8 +171,6 @@ __device__ __forceinline__ void blocking_subblock(const StoreView& s, const Pair
   rho = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
   M = fmaxf(fmaxf(red[4], red[5]), fmaxf(red[6], red[7]));
   const int e = exponent_rule<BITS>(rho, M);
-  const float step = pow2f_exact(e), inv_step = pow2f_exact(-e);
-  constexpr uint32_t mask = (1u << BITS) - 1u;
   const uint32_t g = (uint32_t)(blk * (kBlockCoords / 8) + j * (kSubCoords / 8) + lane);
   uint8_t* ca = s.codes + (int64_t)pd.a * s.nblk * kBlockCoords + blk * (kBlockCoords * BITS / 8) +
                 j * (kSubCoords * BITS / 8) + lane * BITS;
@@ -144,24 +178,8 @@ __device__ __forceinline__ void blocking_subblock(const StoreView& s, const Pair
                 j * (kSubCoords * BITS / 8) + lane * BITS;
   const uint4 ra = philox4x32_10(g, (uint32_t)pd.a, pd.wa, kStreamRounding, s.key0, s.key1);
   const uint4 rb = philox4x32_10(g, (uint32_t)pd.b, pd.wb, kStreamRounding, s.key0, s.key1);
-  uint64_t pka = 0, pkb = 0;
-  f8 out;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    int32_t cell_a, cell_b;
-    const int32_t qa = encode_index(va.v[i], inv_step, sr_u16(ra, i), cell_a);
-    const int32_t qb = encode_index(vb.v[i], inv_step, sr_u16(rb, i), cell_b);
-    const uint32_t code_a = (uint32_t)qa & mask, code_b = (uint32_t)qb & mask;
-    pka |= (uint64_t)code_a << (i * BITS);
-    pkb |= (uint64_t)code_b << (i * BITS);
-    const float Qa = __fmul_rn(__int2float_rn(decode_index<BITS>(code_a, cell_b)), step);
-    const float Qb = __fmul_rn(__int2float_rn(decode_index<BITS>(code_b, cell_a)), step);
-    out.v[i] = __fmul_rn(0.5f, __fadd_rn(Qa, Qb));
-  }
-  st256(xa, out);
-  st256(xb, out);
-  store_codes<BITS>(ca, lane, pka);
-  store_codes<BITS>(cb, lane, pkb);
+  if (fast_range(M, pow2f_exact(-e), e)) subblock_exchange<BITS, true>(va, vb, xa, xb, ca, cb, ra, rb, lane, e);
+  else subblock_exchange<BITS, false>(va, vb, xa, xb, ca, cb, ra, rb, lane, e);
   if (j == 0 && lane == 0) {
     s.exps[(int64_t)pd.a * s.nblk + blk] = (int8_t)e;
     s.exps[(int64_t)pd.b * s.nblk + blk] = (int8_t)e;

@@ -164,22 +164,85 @@ __device__ __forceinline__ int32_t encode_index(float x, float inv_step, uint32_
   return (int32_t)((uint32_t)cell + (u16 < thr ? 1u : 0u));
 }
 
-// Lattice index congruent to colour c (mod 2^b) in the window [cell - L, cell + L + 1]
-// around the key's cell.
-template <int BITS>
-__device__ __forceinline__ int32_t decode_index(uint32_t c, int32_t cell) {
-  constexpr uint32_t mask = (1u << BITS) - 1u;
-  int32_t delta = (int32_t)((c - (uint32_t)cell) & mask);
-  if (delta > (1 << (BITS - 1))) delta -= (1 << BITS);
-  return (int32_t)((uint32_t)cell + (uint32_t)delta);
+// ---------------------------------------------------------------------------------------
+// The same lattice arithmetic without conversion instructions. Float<->integer conversions and
+// floorf share one quarter-rate unit, which the 8..18 conversions per coordinate of the interaction
+// kernels keep busier than HBM does. While every scaled value t = x * 2^-e and every lattice index
+// of a block stays inside (-2^22, 2^22), the same results come from full-rate float adds:
+//   s = t + 1.5*2^23 rounded toward -inf is floor(t) + 1.5*2^23 exactly (ulp 1 in [2^23, 2^24)), its bit
+//   pattern is 0x4B400000 + floor(t): a lattice cell "biased" by 0x4B400000. The bias has no low 22
+//   bits, so colours (cell & mask) and the window arithmetic of the decoder work on biased cells
+//   unchanged, and a biased index i turns into the value (i - bias) * 2^e with one exact fused
+//   multiply-add: as_float(i) * 2^e - 1.5*2^23 * 2^e.
+//   floor(frac * 2^16) is compared with the 16-bit uniform as 2^23 + floor(.) against 2^23 + u, both
+//   as bit patterns: frac * 2^16 + 2^23 rounded toward zero, and the uniform's half word spliced under
+//   the exponent byte with one byte permute.
+// LatticeOps<true> is that form (the caller checks the range, warp-uniformly, per block);
+// LatticeOps<false> is the defining form with saturating conversions. Both give bit-identical
+// results wherever the fast form is valid.
+// ---------------------------------------------------------------------------------------
+constexpr float kCellBias = 12582912.0f;            // 1.5 * 2^23
+constexpr float kFastRange = 2097152.0f;            // 2^21: bound on |x| * 2^-e for the fast form (half the
+                                                    // exact limit, which leaves room for the decode window)
+constexpr int kFastExpMax = 100;                    // keeps 1.5*2^23 * 2^e finite
+
+template <bool FAST>
+struct LatticeOps {
+  // (biased) cell of a key: floor(key * 2^-e)
+  static __device__ __forceinline__ uint32_t cell(float key, float inv_step) {
+    const float t = __fmul_rn(key, inv_step);
+    if constexpr (FAST) return __float_as_uint(__fadd_rd(t, kCellBias));
+    else return (uint32_t)__float2int_rd(t);
+  }
+  // (biased) lattice index of x after stochastic rounding with half `hi` (0 low, 1 high) of generator
+  // word `w`; `cell` receives the (biased) cell of x.
+  static __device__ __forceinline__ uint32_t encode(float x, float inv_step, uint32_t w, int hi, uint32_t& cell_out) {
+    const float t = __fmul_rn(x, inv_step);
+    if constexpr (FAST) {
+      const float sft = __fadd_rd(t, kCellBias);
+      const float f = __fsub_rn(sft, kCellBias);
+      const float frac = __fsub_rn(t, f);
+      const uint32_t thr = __float_as_uint(__fmaf_rz(frac, 65536.0f, 8388608.0f));   // 0x4B000000 + floor(frac * 2^16)
+      const uint32_t u = __byte_perm(w, 0x4B000000u, hi ? 0x7632 : 0x7610);          // 0x4B000000 + uniform
+      cell_out = __float_as_uint(sft);
+      return cell_out + (u < thr ? 1u : 0u);
+    } else {
+      const float f = floorf(t);
+      const float frac = __fsub_rn(t, f);
+      const uint32_t thr = __float2uint_rz(__fmul_rn(frac, 65536.0f));
+      const uint32_t u = hi ? (w >> 16) : (w & 0xFFFFu);
+      cell_out = (uint32_t)__float2int_rd(t);
+      return cell_out + (u < thr ? 1u : 0u);
+    }
+  }
+  // (biased) index congruent to colour c (mod 2^BITS) in the window [cell - L, cell + L + 1]:
+  // cell - L + ((c - cell + L) mod 2^BITS), L = 2^(BITS-1) - 1.
+  template <int BITS>
+  static __device__ __forceinline__ uint32_t decode(uint32_t c, uint32_t cell_in) {
+    constexpr uint32_t mask = (1u << BITS) - 1u, L = (1u << (BITS - 1)) - 1u;
+    return cell_in - L + ((c - cell_in + L) & mask);
+  }
+  static __device__ __forceinline__ uint32_t decode_bits(uint32_t c, uint32_t cell_in, int bits) {
+    const uint32_t mask = (1u << bits) - 1u, L = (1u << (bits - 1)) - 1u;
+    return cell_in - L + ((c - cell_in + L) & mask);
+  }
+  // value of a (biased) index; `unbias` = -1.5*2^23 * step (fast form only)
+  static __device__ __forceinline__ float value(uint32_t idx, float step, float unbias) {
+    if constexpr (FAST) return __fmaf_rn(__uint_as_float(idx), step, unbias);
+    else return __fmul_rn(__int2float_rn((int32_t)idx), step);
+  }
+};
+
+// Whether the fast form covers a block: largest magnitude `maxabs` scaled by 2^-e stays below 2^21.
+__device__ __forceinline__ bool fast_range(float maxabs, float inv_step, int e) {
+  return __fmul_rn(maxabs, inv_step) < kFastRange && e <= kFastExpMax;
 }
 
-template <int BITS>
-__device__ __forceinline__ float decode_value(float key, uint32_t c, float inv_step, float step) {
-  const int32_t cell = __float2int_rd(__fmul_rn(key, inv_step));
-  return __fmul_rn(__int2float_rn(decode_index<BITS>(c, cell)), step);
+// Generator word holding the 16-bit rounding uniform of coordinate i (0..7) of a call covering 8
+// consecutive coordinates (low half for even i, high half for odd i).
+__device__ __forceinline__ uint32_t sr_word(const uint4& w, int i) {
+  return (i < 2) ? w.x : (i < 4) ? w.y : (i < 6) ? w.z : w.w;
 }
-
 // 16-bit rounding uniform i (0..7) of a generator call covering 8 consecutive coordinates.
 __device__ __forceinline__ uint32_t sr_u16(const uint4& w, int i) {
   const uint32_t word = (i < 2) ? w.x : (i < 4) ? w.y : (i < 6) ? w.z : w.w;

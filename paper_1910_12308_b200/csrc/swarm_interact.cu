@@ -100,6 +100,68 @@ interact_identity_kernel(StoreView s, const PairList pairs, int64_t total_warps,
   }
 }
 
+// Decode phase of a non-blocking block: nx holds X^a and av the snapshot B^a (the key) on entry; on return
+// nx holds the new model and av the average. Block maxima for the guard rule come back warp-reduced.
+template <int BITS, bool FAST>
+__device__ __forceinline__ void nonblocking_decode(f8 (&nx)[kSub], f8 (&av)[kSub], const uint64_t (&pa)[kSub],
+                                                   const uint64_t (&pb)[kSub], int e_own, int e_oth, float& spread_out,
+                                                   float& dmax_out, float& M_out) {
+  using Ops = LatticeOps<FAST>;
+  const float step_own = pow2f_exact(e_own), inv_own = pow2f_exact(-e_own);
+  const float step_oth = pow2f_exact(e_oth), inv_oth = pow2f_exact(-e_oth);
+  const float unb_own = FAST ? -__fmul_rn(kCellBias, step_own) : 0.0f;
+  const float unb_oth = FAST ? -__fmul_rn(kCellBias, step_oth) : 0.0f;
+  constexpr uint32_t mask = (1u << BITS) - 1u;
+  float spread = 0.0f, dmax = 0.0f, M = 0.0f;
+#pragma unroll
+  for (int j = 0; j < kSub; ++j)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float key = av[j].v[i];
+      const uint32_t code_own = (uint32_t)(pa[j] >> (i * BITS)) & mask, code_oth = (uint32_t)(pb[j] >> (i * BITS)) & mask;
+      const float own = Ops::value(Ops::template decode<BITS>(code_own, Ops::cell(key, inv_own)), step_own, unb_own);
+      const float oth = Ops::value(Ops::template decode<BITS>(code_oth, Ops::cell(key, inv_oth)), step_oth, unb_oth);
+      const float avg = __fmul_rn(0.5f, __fadd_rn(own, oth));
+      const float D = __fsub_rn(key, nx[j].v[i]);
+      const float x_new = __fsub_rn(avg, D);
+      spread = fmaxf(spread, fabsf(__fsub_rn(own, oth)));
+      dmax = fmaxf(dmax, fabsf(D));
+      M = fmaxf(M, fmaxf(fabsf(x_new), fabsf(avg)));
+      nx[j].v[i] = x_new;
+      av[j].v[i] = avg;
+    }
+  spread_out = warp_max_nonneg(spread);
+  dmax_out = warp_max_nonneg(dmax);
+  M_out = warp_max_nonneg(M);
+}
+
+// Encode phase: the new model goes to X^a, B^a and (encoded) to a's buffer, the average (encoded) to b's.
+template <int BITS, bool FAST>
+__device__ __forceinline__ void nonblocking_encode(const f8 (&nx)[kSub], const f8 (&av)[kSub], float* xa, float* ba,
+                                                   uint8_t* ca, uint8_t* cb, uint32_t group0, const StoreView& s,
+                                                   const PairDesc& pd, int lane, int e) {
+  using Ops = LatticeOps<FAST>;
+  const float inv_step = pow2f_exact(-e);
+  constexpr uint32_t mask = (1u << BITS) - 1u;
+#pragma unroll
+  for (int j = 0; j < kSub; ++j) {
+    const uint32_t g = group0 + j * (kSubCoords / 8);
+    const uint4 ra = philox4x32_10(g, (uint32_t)pd.a, pd.wa, kStreamRounding, s.key0, s.key1);
+    const uint4 rb = philox4x32_10(g, (uint32_t)pd.b, pd.wb, kStreamRounding, s.key0, s.key1);
+    uint64_t pka = 0, pkb = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      uint32_t cell;
+      pka |= (uint64_t)(Ops::encode(nx[j].v[i], inv_step, sr_word(ra, i), i & 1, cell) & mask) << (i * BITS);
+      pkb |= (uint64_t)(Ops::encode(av[j].v[i], inv_step, sr_word(rb, i), i & 1, cell) & mask) << (i * BITS);
+    }
+    st256(xa + j * kSubCoords, nx[j]);
+    st256(ba + j * kSubCoords, nx[j]);
+    store_codes<BITS>(ca + j * (kSubCoords * BITS / 8), lane, pka);
+    store_codes<BITS>(cb + j * (kSubCoords * BITS / 8), lane, pkb);
+  }
+}
+
 // -----------------------------------------------------------------------------------------
 // Non-blocking interaction (the single-buffer form of Algorithm 1): the initiator a decodes
 // its own buffer and the responder's buffer with its base snapshot B^a as key, averages,
@@ -157,52 +219,26 @@ interact_nonblocking_kernel(StoreView s, const PairList pairs, int64_t total_war
     pb[j] = load_codes<BITS>(cb + j * (kSubCoords * BITS / 8));
   }
   const int e_own = *ea_p, e_oth = *eb_p;
-  const float step_own = pow2f_exact(e_own), inv_own = pow2f_exact(-e_own);
-  const float step_oth = pow2f_exact(e_oth), inv_oth = pow2f_exact(-e_oth);
 
-  constexpr uint32_t mask = (1u << BITS) - 1u;
-  float spread = 0.0f, dmax = 0.0f, M = 0.0f;
+  // largest key magnitude of the block: decides, for the whole warp, which form of the lattice arithmetic
+  // the decodes take
+  float kmax = 0.0f;
 #pragma unroll
   for (int j = 0; j < kSub; ++j)
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const float key = av[j].v[i];
-      const float own = decode_value<BITS>(key, (uint32_t)(pa[j] >> (i * BITS)) & mask, inv_own, step_own);
-      const float oth = decode_value<BITS>(key, (uint32_t)(pb[j] >> (i * BITS)) & mask, inv_oth, step_oth);
-      const float avg = __fmul_rn(0.5f, __fadd_rn(own, oth));
-      const float D = __fsub_rn(key, nx[j].v[i]);
-      const float x_new = __fsub_rn(avg, D);
-      spread = fmaxf(spread, fabsf(__fsub_rn(own, oth)));
-      dmax = fmaxf(dmax, fabsf(D));
-      M = fmaxf(M, fmaxf(fabsf(x_new), fabsf(avg)));
-      nx[j].v[i] = x_new;
-      av[j].v[i] = avg;
-    }
-  spread = warp_max_nonneg(spread);
-  dmax = warp_max_nonneg(dmax);
-  M = warp_max_nonneg(M);
+    for (int i = 0; i < 8; ++i) kmax = fmaxf(kmax, fabsf(av[j].v[i]));
+  kmax = warp_max_nonneg(kmax);
+  float spread, dmax, M;
+  if (fast_range(kmax, pow2f_exact(-e_own), e_own) && fast_range(kmax, pow2f_exact(-e_oth), e_oth))
+    nonblocking_decode<BITS, true>(nx, av, pa, pb, e_own, e_oth, spread, dmax, M);
+  else
+    nonblocking_decode<BITS, false>(nx, av, pa, pb, e_own, e_oth, spread, dmax, M);
   const float rho = __fadd_rn(__fmul_rn(2.0f, spread), dmax);
   const int e = exponent_rule<BITS>(rho, M);
-  const float inv_step = pow2f_exact(-e);
 
   const uint32_t group0 = (uint32_t)(blk * (kBlockCoords / 8) + lane);
-#pragma unroll
-  for (int j = 0; j < kSub; ++j) {
-    const uint32_t g = group0 + j * (kSubCoords / 8);
-    const uint4 ra = philox4x32_10(g, (uint32_t)pd.a, pd.wa, kStreamRounding, s.key0, s.key1);
-    const uint4 rb = philox4x32_10(g, (uint32_t)pd.b, pd.wb, kStreamRounding, s.key0, s.key1);
-    uint64_t pka = 0, pkb = 0;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      int32_t cell;
-      pka |= (uint64_t)((uint32_t)encode_index(nx[j].v[i], inv_step, sr_u16(ra, i), cell) & mask) << (i * BITS);
-      pkb |= (uint64_t)((uint32_t)encode_index(av[j].v[i], inv_step, sr_u16(rb, i), cell) & mask) << (i * BITS);
-    }
-    st256(xa + j * kSubCoords, nx[j]);
-    st256(ba + j * kSubCoords, nx[j]);
-    store_codes<BITS>(ca + j * (kSubCoords * BITS / 8), lane, pka);
-    store_codes<BITS>(cb + j * (kSubCoords * BITS / 8), lane, pkb);
-  }
+  if (fast_range(M, pow2f_exact(-e), e)) nonblocking_encode<BITS, true>(nx, av, xa, ba, ca, cb, group0, s, pd, lane, e);
+  else nonblocking_encode<BITS, false>(nx, av, xa, ba, ca, cb, group0, s, pd, lane, e);
   if (lane == 0) { *ea_p = (int8_t)e; *eb_p = (int8_t)e; }
 }
 
@@ -300,18 +336,116 @@ constexpr int kOwnBlockBytes = 2 * kBlockCoords;
 __device__ __forceinline__ uint32_t plane_byte(const uint2& v, int i) {
   return (((i < 4) ? v.x : v.y) >> ((i & 3) * 8)) & 0xFFu;
 }
-// Decode with a prefix of `bits` (8 or 16, warp-uniform) of a 16-bit colour.
-__device__ __forceinline__ float decode_prefix(float key, uint32_t c, int bits, float inv_step, float step) {
-  const int32_t cell = __float2int_rd(__fmul_rn(key, inv_step));
-  const uint32_t mask = (1u << bits) - 1u;
-  int32_t delta = (int32_t)((c - (uint32_t)cell) & mask);
-  if (delta > (int32_t)(1u << (bits - 1))) delta -= (int32_t)(mask + 1u);
-  return __fmul_rn(__int2float_rn((int32_t)((uint32_t)cell + (uint32_t)delta)), step);
-}
 // Split eight 16-bit colours (two per word) into their low-byte and high-byte planes.
 __device__ __forceinline__ void split_planes(const uint32_t (&ow)[4], uint2& lo, uint2& hi) {
   lo.x = __byte_perm(ow[0], ow[1], 0x6420); hi.x = __byte_perm(ow[0], ow[1], 0x7531);
   lo.y = __byte_perm(ow[2], ow[3], 0x6420); hi.y = __byte_perm(ow[2], ow[3], 0x7531);
+}
+
+// Decode chain of a two-register block. On entry nx = X^a, av = snapshot B^a; on return nx = new model,
+// av = average. Returns the warp-reduced block maxima for the exponents of the three writes.
+template <int BITS, bool FAST>
+__device__ __forceinline__ void registers_decode(f8 (&nx)[kSub], f8 (&av)[kSub], const uint2 (&va)[kSub],
+                                                 const uint2 (&vb)[kSub], const uint2 (&vbh)[kSub],
+                                                 const uint64_t (&pa)[kSub], const uint64_t (&pb)[kSub], int prefix,
+                                                 int eoa, int eob, int epa, int epb, float& spread_out, float& dmax_out,
+                                                 float& M_out, float& rho_b_out, float& M_b_out) {
+  using Ops = LatticeOps<FAST>;
+  const float so_a = pow2f_exact(eoa), io_a = pow2f_exact(-eoa), so_b = pow2f_exact(eob), io_b = pow2f_exact(-eob);
+  const float sp_a = pow2f_exact(epa), ip_a = pow2f_exact(-epa), sp_b = pow2f_exact(epb), ip_b = pow2f_exact(-epb);
+  const float uo_a = FAST ? -__fmul_rn(kCellBias, so_a) : 0.0f, uo_b = FAST ? -__fmul_rn(kCellBias, so_b) : 0.0f;
+  const float up_a = FAST ? -__fmul_rn(kCellBias, sp_a) : 0.0f, up_b = FAST ? -__fmul_rn(kCellBias, sp_b) : 0.0f;
+  constexpr uint32_t mask = (1u << BITS) - 1u;
+  float spread = 0.0f, dmax = 0.0f, M = 0.0f, rho_b = 0.0f, M_b = 0.0f;
+#pragma unroll
+  for (int j = 0; j < kSub; ++j)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float snap = av[j].v[i];
+      // own key: less than one step away, the 8-bit prefix always suffices
+      const float qhat_a = Ops::value(Ops::template decode<8>(plane_byte(va[j], i), Ops::cell(snap, io_a)), so_a, uo_a);
+      const float Qa = Ops::value(Ops::template decode<BITS>((uint32_t)(pa[j] >> (i * BITS)) & mask, Ops::cell(qhat_a, ip_a)), sp_a, up_a);
+      const float qhat_b = Ops::value(Ops::decode_bits(plane_byte(vb[j], i) | (plane_byte(vbh[j], i) << 8),
+                                                       Ops::cell(snap, io_b), prefix), so_b, uo_b);
+      const float Qb = Ops::value(Ops::template decode<BITS>((uint32_t)(pb[j] >> (i * BITS)) & mask, Ops::cell(qhat_b, ip_b)), sp_b, up_b);
+      const float avg = __fmul_rn(0.5f, __fadd_rn(Qa, Qb));
+      const float D = __fsub_rn(snap, nx[j].v[i]);
+      const float x_new = __fsub_rn(avg, D);
+      spread = fmaxf(spread, fabsf(__fsub_rn(Qa, Qb)));
+      dmax = fmaxf(dmax, fabsf(D));
+      M = fmaxf(M, fmaxf(fabsf(x_new), fabsf(avg)));
+      rho_b = fmaxf(rho_b, fabsf(__fsub_rn(avg, qhat_b)));        // distance of the average to b's decoding key
+      M_b = fmaxf(M_b, fmaxf(fabsf(avg), fabsf(qhat_b)));
+      nx[j].v[i] = x_new;
+      av[j].v[i] = avg;
+    }
+  spread_out = warp_max_nonneg(spread);
+  dmax_out = warp_max_nonneg(dmax);
+  M_out = warp_max_nonneg(M);
+  rho_b_out = warp_max_nonneg(rho_b);
+  M_b_out = warp_max_nonneg(M_b);
+}
+
+// Writes a's own register (16-bit colours of the new model, two byte planes) and b's current register
+// (b-bit colours of the average); returns the distance of the new model to the lattice point just written.
+template <int BITS, bool FAST>
+__device__ __forceinline__ void registers_encode_own(const f8 (&nx)[kSub], const f8 (&av)[kSub], uint8_t* oa, uint8_t* cb,
+                                                     uint32_t group0, const StoreView& s, const PairDesc& pd, int lane,
+                                                     int eo, int ep_b, float& rho_a_out, float& M_a_out) {
+  using Ops = LatticeOps<FAST>;
+  const float so = pow2f_exact(eo), io = pow2f_exact(-eo), ipb_new = pow2f_exact(-ep_b);
+  const float uo = FAST ? -__fmul_rn(kCellBias, so) : 0.0f;
+  constexpr uint32_t mask = (1u << BITS) - 1u;
+  float rho_a = 0.0f, M_a = 0.0f;
+#pragma unroll
+  for (int j = 0; j < kSub; ++j) {
+    const uint32_t g = group0 + j * (kSubCoords / 8);
+    const uint4 ro = philox4x32_10(g, (uint32_t)pd.a, pd.woa, kStreamOwnRounding, s.key0, s.key1);
+    const uint4 rb = philox4x32_10(g, (uint32_t)pd.b, pd.wb, kStreamRounding, s.key0, s.key1);
+    uint32_t ow[4] = {0u, 0u, 0u, 0u};
+    uint64_t pkb = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      uint32_t cell;
+      const uint32_t q = Ops::encode(nx[j].v[i], io, sr_word(ro, i), i & 1, cell);
+      ow[i >> 1] |= (q & 0xFFFFu) << ((i & 1) * 16);
+      const float qhat_new = Ops::value(q, so, uo);
+      rho_a = fmaxf(rho_a, fabsf(__fsub_rn(nx[j].v[i], qhat_new)));
+      M_a = fmaxf(M_a, fmaxf(fabsf(nx[j].v[i]), fabsf(qhat_new)));
+      pkb |= (uint64_t)(Ops::encode(av[j].v[i], ipb_new, sr_word(rb, i), i & 1, cell) & mask) << (i * BITS);
+    }
+    uint2 lo, hi;
+    split_planes(ow, lo, hi);
+    *reinterpret_cast<uint2*>(oa + j * kSubCoords) = lo;
+    *reinterpret_cast<uint2*>(oa + kBlockCoords + j * kSubCoords) = hi;
+    store_codes<BITS>(cb + j * (kSubCoords * BITS / 8), lane, pkb);
+  }
+  rho_a_out = warp_max_nonneg(rho_a);
+  M_a_out = warp_max_nonneg(M_a);
+}
+
+// Writes the new model to X^a and B^a and its b-bit colours to a's current register.
+template <int BITS, bool FAST>
+__device__ __forceinline__ void registers_encode_current(const f8 (&nx)[kSub], float* xa, float* ba, uint8_t* ca,
+                                                         uint32_t group0, const StoreView& s, const PairDesc& pd,
+                                                         int lane, int ep_a) {
+  using Ops = LatticeOps<FAST>;
+  const float ipa_new = pow2f_exact(-ep_a);
+  constexpr uint32_t mask = (1u << BITS) - 1u;
+#pragma unroll
+  for (int j = 0; j < kSub; ++j) {
+    const uint32_t g = group0 + j * (kSubCoords / 8);
+    const uint4 ra = philox4x32_10(g, (uint32_t)pd.a, pd.wa, kStreamRounding, s.key0, s.key1);
+    uint64_t pka = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      uint32_t cell;
+      pka |= (uint64_t)(Ops::encode(nx[j].v[i], ipa_new, sr_word(ra, i), i & 1, cell) & mask) << (i * BITS);
+    }
+    st256(xa + j * kSubCoords, nx[j]);
+    st256(ba + j * kSubCoords, nx[j]);
+    store_codes<BITS>(ca + j * (kSubCoords * BITS / 8), lane, pka);
+  }
 }
 
 template <int BITS, bool FUSED>
@@ -374,84 +508,35 @@ interact_registers_kernel(StoreView s, const PairList pairs, int64_t total_warps
   }
   const int eoa = s.oexps[(int64_t)pd.a * s.nblk + blk], eob = s.oexps[(int64_t)pd.b * s.nblk + blk];
   const int epa = s.exps[(int64_t)pd.a * s.nblk + blk], epb = s.exps[(int64_t)pd.b * s.nblk + blk];
-  const float so_a = pow2f_exact(eoa), io_a = pow2f_exact(-eoa), so_b = pow2f_exact(eob), io_b = pow2f_exact(-eob);
-  const float sp_a = pow2f_exact(epa), ip_a = pow2f_exact(-epa), sp_b = pow2f_exact(epb), ip_b = pow2f_exact(-epb);
 
-  constexpr uint32_t mask = (1u << BITS) - 1u;
-  float spread = 0.0f, dmax = 0.0f, M = 0.0f, rho_b = 0.0f, M_b = 0.0f;
+  // largest key magnitude of the block and bounds on the decoded own-register values (a key plus the decode
+  // window): they decide, for the whole warp, which form of the lattice arithmetic the decode chain takes
+  float kmax = 0.0f;
 #pragma unroll
   for (int j = 0; j < kSub; ++j)
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const float snap = av[j].v[i];
-      const float qhat_a = decode_value<8>(snap, plane_byte(va[j], i), io_a, so_a);    // own key: < 1 step away
-      const float Qa = decode_value<BITS>(qhat_a, (uint32_t)(pa[j] >> (i * BITS)) & mask, ip_a, sp_a);
-      const float qhat_b = decode_prefix(snap, plane_byte(vb[j], i) | (plane_byte(vbh[j], i) << 8), prefix, io_b, so_b);
-      const float Qb = decode_value<BITS>(qhat_b, (uint32_t)(pb[j] >> (i * BITS)) & mask, ip_b, sp_b);
-      const float avg = __fmul_rn(0.5f, __fadd_rn(Qa, Qb));
-      const float D = __fsub_rn(snap, nx[j].v[i]);
-      const float x_new = __fsub_rn(avg, D);
-      spread = fmaxf(spread, fabsf(__fsub_rn(Qa, Qb)));
-      dmax = fmaxf(dmax, fabsf(D));
-      M = fmaxf(M, fmaxf(fabsf(x_new), fabsf(avg)));
-      rho_b = fmaxf(rho_b, fabsf(__fsub_rn(avg, qhat_b)));        // distance of the average to b's decoding key
-      M_b = fmaxf(M_b, fmaxf(fabsf(avg), fabsf(qhat_b)));
-      nx[j].v[i] = x_new;
-      av[j].v[i] = avg;
-    }
-  spread = warp_max_nonneg(spread);
-  dmax = warp_max_nonneg(dmax);
-  M = warp_max_nonneg(M);
-  rho_b = warp_max_nonneg(rho_b);
-  M_b = warp_max_nonneg(M_b);
+    for (int i = 0; i < 8; ++i) kmax = fmaxf(kmax, fabsf(av[j].v[i]));
+  kmax = warp_max_nonneg(kmax);
+  const float qa_max = __fmaf_rn(130.0f, pow2f_exact(eoa), kmax);
+  const float qb_max = __fmaf_rn(prefix == 16 ? 32770.0f : 130.0f, pow2f_exact(eob), kmax);
+  const bool fast_chain = fast_range(kmax, pow2f_exact(-eoa), eoa) && fast_range(kmax, pow2f_exact(-eob), eob) &&
+                          fast_range(qa_max, pow2f_exact(-epa), epa) && fast_range(qb_max, pow2f_exact(-epb), epb);
+  float spread, dmax, M, rho_b, M_b;
+  if (fast_chain) registers_decode<BITS, true>(nx, av, va, vb, vbh, pa, pb, prefix, eoa, eob, epa, epb, spread, dmax, M, rho_b, M_b);
+  else registers_decode<BITS, false>(nx, av, va, vb, vbh, pa, pb, prefix, eoa, eob, epa, epb, spread, dmax, M, rho_b, M_b);
   const int eo = exponent_rule<kOwnResolutionBits>(__fadd_rn(__fmul_rn(2.0f, spread), dmax), M);
   const int ep_b = exponent_rule<BITS>(rho_b, M_b);
-  const float so = pow2f_exact(eo), io = pow2f_exact(-eo), ipb_new = pow2f_exact(-ep_b);
 
   // own register of a (16 bits) and current register of b; distance of the new model to its own key
   const uint32_t group0 = (uint32_t)(blk * (kBlockCoords / 8) + lane);
-  float rho_a = 0.0f, M_a = 0.0f;
-#pragma unroll
-  for (int j = 0; j < kSub; ++j) {
-    const uint32_t g = group0 + j * (kSubCoords / 8);
-    const uint4 ro = philox4x32_10(g, (uint32_t)pd.a, pd.woa, kStreamOwnRounding, s.key0, s.key1);
-    const uint4 rb = philox4x32_10(g, (uint32_t)pd.b, pd.wb, kStreamRounding, s.key0, s.key1);
-    uint32_t ow[4] = {0u, 0u, 0u, 0u};
-    uint64_t pkb = 0;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      int32_t cell;
-      const int32_t q = encode_index(nx[j].v[i], io, sr_u16(ro, i), cell);
-      ow[i >> 1] |= ((uint32_t)q & 0xFFFFu) << ((i & 1) * 16);
-      const float qhat_new = __fmul_rn(__int2float_rn(q), so);
-      rho_a = fmaxf(rho_a, fabsf(__fsub_rn(nx[j].v[i], qhat_new)));
-      M_a = fmaxf(M_a, fmaxf(fabsf(nx[j].v[i]), fabsf(qhat_new)));
-      pkb |= (uint64_t)((uint32_t)encode_index(av[j].v[i], ipb_new, sr_u16(rb, i), cell) & mask) << (i * BITS);
-    }
-    uint2 lo, hi;
-    split_planes(ow, lo, hi);
-    *reinterpret_cast<uint2*>(oa + j * kSubCoords) = lo;
-    *reinterpret_cast<uint2*>(oa + kBlockCoords + j * kSubCoords) = hi;
-    store_codes<BITS>(cb + j * (kSubCoords * BITS / 8), lane, pkb);
-  }
-  rho_a = warp_max_nonneg(rho_a);
-  M_a = warp_max_nonneg(M_a);
+  float rho_a, M_a;
+  if (fast_range(M, pow2f_exact(-eo), eo) && fast_range(M_b, pow2f_exact(-ep_b), ep_b))
+    registers_encode_own<BITS, true>(nx, av, oa, cb, group0, s, pd, lane, eo, ep_b, rho_a, M_a);
+  else
+    registers_encode_own<BITS, false>(nx, av, oa, cb, group0, s, pd, lane, eo, ep_b, rho_a, M_a);
   const int ep_a = exponent_rule<BITS>(rho_a, M_a);
-  const float ipa_new = pow2f_exact(-ep_a);
-#pragma unroll
-  for (int j = 0; j < kSub; ++j) {
-    const uint32_t g = group0 + j * (kSubCoords / 8);
-    const uint4 ra = philox4x32_10(g, (uint32_t)pd.a, pd.wa, kStreamRounding, s.key0, s.key1);
-    uint64_t pka = 0;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      int32_t cell;
-      pka |= (uint64_t)((uint32_t)encode_index(nx[j].v[i], ipa_new, sr_u16(ra, i), cell) & mask) << (i * BITS);
-    }
-    st256(xa + j * kSubCoords, nx[j]);
-    st256(ba + j * kSubCoords, nx[j]);
-    store_codes<BITS>(ca + j * (kSubCoords * BITS / 8), lane, pka);
-  }
+  if (fast_range(M_a, pow2f_exact(-ep_a), ep_a)) registers_encode_current<BITS, true>(nx, xa, ba, ca, group0, s, pd, lane, ep_a);
+  else registers_encode_current<BITS, false>(nx, xa, ba, ca, group0, s, pd, lane, ep_a);
   if (lane == 0) {
     s.oexps[(int64_t)pd.a * s.nblk + blk] = (int8_t)eo;
     s.exps[(int64_t)pd.a * s.nblk + blk] = (int8_t)ep_a;

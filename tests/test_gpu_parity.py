@@ -186,6 +186,66 @@ def test_nonblocking_far_key_alias_matches():
         assert_store_equal(orc, gpu, bits)
 
 
+# ---- magnitude / distance ratios around the kernels' conversion-free range ----------------------
+
+def _ranged_models(n, d, rng):
+    """Models whose 1024-blocks have magnitude-to-distance ratios 2^2 ... 2^30 (both signs, some blocks
+    exactly on powers of two): scaled values x * 2^-e run from a few units up to the 2^23 limit of the
+    exponent rule, across the 2^21 bound below which the kernels use float adds instead of conversions."""
+    nblk = (d + 1023) // 1024
+    X = np.zeros((n, d), dtype=np.float32)
+    for k in range(nblk):
+        lo, hi = k * 1024, min(d, (k + 1) * 1024)
+        ratio = 2.0 ** (2 + 2 * (k % 15))
+        base = (-1.0) ** k * (0.37 if k % 3 else 0.5) * 2.0 ** (k % 7 - 3)
+        noise = rng.normal(size=(n, hi - lo))
+        X[:, lo:hi] = (base * (1.0 + noise / ratio)).astype(np.float32)
+        if k % 4 == 1:                      # mixed signs inside the block
+            X[:, lo:hi:2] *= np.float32(-1.0)
+    return X
+
+
+@pytest.mark.parametrize("bits", [2, 4, 5, 8])
+def test_blocking_interaction_across_magnitude_ratios(bits):
+    n, d = 6, 16 * 1024 + 37
+    orc, gpu = make_pair(n, d, "complete", seed=5)
+    rng = np.random.default_rng(900 + bits)
+    orc.X[:] = _ranged_models(n, d, rng)
+    inject(orc, gpu)
+    for rnd in range(4):
+        pairs = disjoint_pairs(orc, rng, 3)
+        assert orc.interact(pairs, bits) == 0 and gpu.interact(pairs, bits) == 0
+        assert_store_equal(orc, gpu, bits)
+
+
+@pytest.mark.parametrize("mode", [1, 2])
+@pytest.mark.parametrize("bits", [2, 4, 7, 8])
+def test_one_way_interactions_across_magnitude_ratios(bits, mode):
+    """Single-buffer and two-register interactions on the same wide-ranged models, with and without pending
+    local updates, including keys that moved away from what the buffers encode."""
+    n, d = 6, 16 * 1024 + 37
+    cfg = dict(objective=1, nonblocking=mode, grad_std=0.0, drift_std=0.0)
+    orc, gpu = make_pair(n, d, "complete", seed=6, **cfg)
+    rng = np.random.default_rng(950 + 10 * bits + mode)
+    orc.X[:] = _ranged_models(n, d, rng)
+    orc.B[:] = orc.X
+    inject(orc, gpu)
+    publish = (lambda s_: s_.publish(bits)) if mode == 1 else (lambda s_: s_.register_publish(bits))
+    assert publish(orc) == 0 and publish(gpu) == 0
+    assert_store_equal(orc, gpu, bits)
+    for rnd in range(5):
+        if rnd >= 2:                         # pending updates of very different relative sizes
+            scale = np.float32(2.0 ** -(4 * rnd))
+            orc.X[:] = (orc.X * (1.0 + scale * rng.normal(size=orc.X.shape))).astype(np.float32)
+        if rnd == 4:                         # a snapshot far from its published encoding
+            orc.B[0, 2048:4096] *= np.float32(1.5)
+            orc.X[0] = orc.B[0]
+        inject(orc, gpu, what=("X", "B"))
+        pairs = disjoint_pairs(orc, rng, 3)
+        assert orc.interact(pairs, bits, mode) == 0 and gpu.interact(pairs, bits, mode) == 0
+        assert_store_equal(orc, gpu, bits)
+
+
 # ---- two-register protocol -----------------------------------------------------------------------
 
 @pytest.mark.parametrize("bits", [2, 3, 4, 5, 6, 7, 8])
