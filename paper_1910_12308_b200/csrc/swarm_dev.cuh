@@ -174,9 +174,11 @@ __device__ __forceinline__ int32_t encode_index(float x, float inv_step, uint32_
 //   bits, so colours (cell & mask) and the window arithmetic of the decoder work on biased cells
 //   unchanged, and a biased index i turns into the value (i - bias) * 2^e with one exact fused
 //   multiply-add: as_float(i) * 2^e - 1.5*2^23 * 2^e.
-//   floor(frac * 2^16) is compared with the 16-bit uniform as 2^23 + floor(.) against 2^23 + u, both
-//   as bit patterns: frac * 2^16 + 2^23 rounded toward zero, and the uniform's half word spliced under
-//   the exponent byte with one byte permute.
+//   The rounding decision u < floor(frac * 2^16) is the same as (u + 1) / 2^16 <= frac, so the index is
+//   floor(t) + floor(z) with z = 1 + frac - (u + 1) / 2^16 in [0, 2): z comes from one fused multiply-add
+//   rounded toward -inf (which cannot cross the integer 1), the uniform enters as a float by splicing its
+//   half word under the exponent byte of 2^23 with one byte permute, and adding z to s, again rounded
+//   toward -inf, lands on s + floor(z). One integer-pipe instruction per encoded coordinate is left.
 // LatticeOps<true> is that form (the caller checks the range, warp-uniformly, per block);
 // LatticeOps<false> is the defining form with saturating conversions. Both give bit-identical
 // results wherever the fast form is valid.
@@ -201,11 +203,12 @@ struct LatticeOps {
     if constexpr (FAST) {
       const float sft = __fadd_rd(t, kCellBias);
       const float f = __fsub_rn(sft, kCellBias);
-      const float frac = __fsub_rn(t, f);
-      const uint32_t thr = __float_as_uint(__fmaf_rz(frac, 65536.0f, 8388608.0f));   // 0x4B000000 + floor(frac * 2^16)
-      const uint32_t u = __byte_perm(w, 0x4B000000u, hi ? 0x7632 : 0x7610);          // 0x4B000000 + uniform
+      const float frac = __fsub_rn(t, f);                                              // in [0, 1]
+      const float um = __uint_as_float(__byte_perm(w, 0x4B000000u, hi ? 0x7632 : 0x7610));   // 2^23 + uniform
+      const float un = __fsub_rn(um, 8454143.0f);                                      // uniform - 65535, exact
+      const float z = __fmaf_rd(un, -0x1p-16f, frac);                                  // 1 + frac - (u + 1) / 2^16, rounded down
       cell_out = __float_as_uint(sft);
-      return cell_out + (u < thr ? 1u : 0u);
+      return __float_as_uint(__fadd_rd(sft, z));                                       // sft + floor(z), floor(z) in {0, 1}
     } else {
       const float f = floorf(t);
       const float frac = __fsub_rn(t, f);
