@@ -186,6 +186,29 @@ def test_nonblocking_far_key_alias_matches():
         assert_store_equal(orc, gpu, bits)
 
 
+# ---- launches with more pairs / nodes than fit the kernel parameters --------------------------------
+
+@pytest.mark.parametrize("mode,bits", [(0, 4), (1, 2), (2, 8)])
+def test_launch_of_128_pairs_on_256_nodes(mode, bits):
+    """The 256-node workload's launch shape (random 8-regular graph, up to 128 disjoint pairs from the
+    sampler, every node stepping before the launch) at a short model: descriptor lists longer than 64
+    entries travel through device memory instead of the kernel parameters."""
+    n, d = 256, 2100
+    cfg = dict(objective=1, nonblocking=mode, grad_std=0.02, drift_std=0.1, offset_std=0.05)
+    orc, gpu = make_pair(n, d, "regular", 8, seed=5, **cfg)
+    inject(orc, gpu)
+    for rnd in range(3):
+        nodes = np.arange(n, dtype=np.int32)
+        assert orc.local_steps(nodes, 2, 0.05) == 0 and gpu.local_steps(nodes, 2, 0.05) == 0
+        for i in range(0, n, 17):
+            assert rel_err(gpu.get(g.T_X, i), orc.X[i]) < TOL
+        inject(orc, gpu, what=("X",))
+        pairs = orc.sample_pairs(128)
+        assert np.array_equal(gpu.sample_pairs(128), pairs) and len(pairs) > 64
+        assert orc.interact(pairs, bits, mode) == 0 and gpu.interact(pairs, bits, mode) == 0
+        assert_store_equal(orc, gpu, bits)
+
+
 # ---- magnitude / distance ratios around the kernels' conversion-free range ----------------------
 
 def _ranged_models(n, d, rng):
