@@ -465,6 +465,19 @@ def run_ours(args, wl, name):
                      "peak_kind": peak_kind, "frac_of_8000": achieved / 8000.0, "traffic": TRAFFIC.get(name),
                      "algorithmic_bytes_per_launch": per_launch_bytes, "kernel_ms": kern_ms},
     }
+    if wl["mode"] == 2 and not fused:
+        # the two-register kernel is bound by instruction issue, not by HBM: report it against the issue rate
+        # (148 SMs x 4 schedulers x SM clock) with its warp instructions per 1024-block from the ncu capture
+        nblk = (wl["d"] + 1023) // 1024
+        instr = REGISTER_KERNEL_INSTR_PER_BLOCK * nblk * npairs_total / K
+        rate = instr / (kern_ms * 1e-3) / 1e12
+        issue_peak = 148 * 4 * (clocks["sm_max_mhz"] or 1965) * 1e6 / 1e12
+        hbm = out["roofline"]
+        out["roofline"] = {"bound": "alu", "kernel": hbm["kernel"], "achieved": rate, "peak": issue_peak,
+                           "unit": "T warp-instructions/s", "frac": rate / issue_peak, "traffic": TRAFFIC.get(name),
+                           "warp_instructions_per_launch": instr, "kernel_ms": kern_ms,
+                           "hbm": {k: hbm[k] for k in ("achieved", "peak", "unit", "frac", "peak_kind", "frac_of_8000",
+                                                       "algorithmic_bytes_per_launch")}}
     # mean model and potential (one HBM pass over all n models each), timed on their own
     reps = 20
     mu = torch.empty(wl["d"], dtype=torch.float32, device="cuda")
@@ -499,7 +512,9 @@ def run_ours(args, wl, name):
 
 # ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel (see profiles/);
 # None until a capture of the current kernel exists.
-TRAFFIC = {"ring64_d1m_b4": 511.1e6}
+TRAFFIC = {"ring64_d1m_b4": 512.1e6}
+# smsp__inst_executed.sum per 1024-coordinate block of interact_registers_kernel<8> (see profiles/)
+REGISTER_KERNEL_INSTR_PER_BLOCK = 3607
 
 
 def main():
