@@ -11,6 +11,12 @@ LIB = os.path.join(HERE, "libswarm_oracle.so")
 
 
 def build(force: bool = False) -> str:
+    # SWARM_ORACLE_LIBRARY names an already built library to load instead of the in-tree one. Only the
+    # mutation tests set it: they compile copies of the source with a mistake planted in each and check
+    # that the pins reject every copy.
+    override = os.environ.get("SWARM_ORACLE_LIBRARY")
+    if override:
+        return override
     if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= os.path.getmtime(SRC):
         return LIB
     cmd = ["g++", "-O2", "-std=c++17", "-ffp-contract=off", "-fno-fast-math", "-fPIC", "-shared",
