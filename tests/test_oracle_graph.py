@@ -100,6 +100,15 @@ def test_sampled_pairs_are_disjoint_and_adjacent(topo, k, n):
     assert total > 50 * n // 4
 
 
+def test_batch_draw_stops_after_sixteen_attempts_per_requested_pair():
+    """A launch of up to P pairs makes at most 16 P draws. On the complete graph with n = 16, P = 8 an independent
+    simulation of that process (numpy, 2000 launches) finds 7.51 pairs per launch on average; it would find 6.43
+    with 4 P draws and 7.98 with 64 P."""
+    s = o.OracleSwarm(16, 4, "complete", seed=9)
+    found = [len(s.sample_pairs(8)) for _ in range(600)]
+    assert max(found) == 8 and abs(np.mean(found) - 7.51) < 0.12
+
+
 def test_single_pair_follows_the_edge_law():
     """With one pair per launch the draw is Algorithm 1's: P[(i -> j)] = 1 / (n * rho_i)."""
     n, k = 6, 2

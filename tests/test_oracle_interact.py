@@ -217,6 +217,24 @@ def test_nonblocking_without_pending_update_matches_blocking_average_of_decoded_
     assert np.array_equal(s.X[1], np.float32(0.5) * (own + oth))
 
 
+def test_nonblocking_write_scales_both_written_vectors_below_2_to_23():
+    """The exponent of a one-way write must keep both vectors it encodes (the new model and the average) below
+    2^23 lattice steps, or their scaled values stop being exact. Here the average is exactly 1 and the new model
+    just below 1, with a pending update of 2^-20: the distance alone would allow a step of 2^-26, the new model
+    alone one of 2^-23, the average needs 2^-22."""
+    s = make_nb(n=4, d=1024)
+    s.X[:] = np.float32(1.0)
+    s.B[:] = np.float32(1.0)
+    assert s.publish(8) == 0
+    assert s.exps[:, 0].tolist() == [-22] * 4                       # zero spread: only the magnitude rule acts
+    s.X[0] = np.float32(1.0 - 2.0**-20)                             # pending update D = B - X = 2^-20
+    assert s.interact([[0, 1]], 8, o.NONBLOCKING) == 0
+    assert np.all(s.X[0] == np.float32(1.0 - 2.0**-20))             # average 1 minus D
+    e = int(s.exps[0, 0])
+    assert int(s.exps[1, 0]) == e
+    assert 1.0 * 2.0**-e < 2.0**23 and 1.0 * 2.0**-(e - 1) >= 2.0**23   # least step that keeps the average exact
+
+
 def test_nonblocking_swarm_contracts_gamma():
     """Statistical sanity only: repeated one-way interactions pull the models together (coordinates
     whose key distance left the decode window stay aliased: the quantization-failure event)."""

@@ -64,11 +64,14 @@ def test_lsq_step_is_minus_lr_times_minibatch_gradient_by_finite_differences():
 def test_lsq_rows_are_uniform_with_replacement_and_shared_inside_a_data_group():
     s = lsq(n=4, d=8, m=7, batch=6, groups=2)
     counts = np.zeros(7)
+    repeats = 0
     for ev in range(2000):
         r = s.minibatch_rows(0, ev)
         assert r.min() >= 0 and r.max() < 7
         counts[r] += 1
+        repeats += int(r[0] == r[1]) + int(r[2] == r[3]) + int(r[3] == r[4])
         assert np.array_equal(r, s.minibatch_rows(1, ev))        # same group, same event
+    assert abs(repeats / 6000 - 1 / 7) < 0.02                    # draws are independent: two agree with probability 1/m
     assert not np.array_equal(s.minibatch_rows(0, 0), s.minibatch_rows(2, 0))
     exp = counts.sum() / 7
     assert ((counts - exp) ** 2 / exp).sum() < 30
@@ -187,6 +190,12 @@ def test_logistic_labels_and_gradient_by_finite_differences():
     score = s.A[0].astype(np.float64) @ s.xstar.astype(np.float64) + float(s.shift[0])
     sure = np.abs(score) > 0.9                               # label noise (std 0.2) cannot flip these
     assert sure.sum() >= 3 and np.array_equal(s.bvec[0][sure], (score[sure] > 0).astype(np.float32))
+    # without label noise the class is exactly the sign of the score (threshold 0, not 1/2)
+    clean = logistic(n=2, d=8, m=400, batch=6, seed=4, noise=0.0)
+    sc = clean.A[1].astype(np.float64) @ clean.xstar.astype(np.float64) + float(clean.shift[1])
+    away = np.abs(sc) > 1e-4
+    assert ((sc > 0) & (sc < 0.5)).sum() >= 10
+    assert np.array_equal(clean.bvec[1][away], (sc[away] > 0).astype(np.float32))
     rows = s.minibatch_rows(0, 0)
     x0 = s.X[0].astype(np.float64).copy()
     A, y = s.A[0].astype(np.float64)[rows], s.bvec[0].astype(np.float64)[rows]

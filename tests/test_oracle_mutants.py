@@ -77,6 +77,39 @@ MUTANTS = [
      ["test_oracle_interact.py"]),
     ("mean_model_is_a_sum", "out[k] = (float)(acc / (double)s.n);", "out[k] = (float)(acc);",
      ["test_oracle_interact.py", "test_oracle_staleness.py"]),
+    ("guard_distance_counts_the_spread_once", "const float rho = 2.0f * spread + dmax;\n    const int e = exponent_rule(rho, M, bits);",
+     "const float rho = spread + dmax;\n    const int e = exponent_rule(rho, M, bits);", ["test_oracle_interact.py"]),
+    ("one_way_write_scaled_by_the_new_model_alone", "M = std::max(M, std::max(std::fabs(nx), std::fabs(av)));\n    }\n    const float rho = 2.0f * spread + dmax;\n    const int e = exponent_rule(rho, M, bits);",
+     "M = std::max(M, std::fabs(nx));\n    }\n    const float rho = 2.0f * spread + dmax;\n    const int e = exponent_rule(rho, M, bits);",
+     ["test_oracle_interact.py"]),
+    ("responder_register_scaled_to_the_wrong_key", "write_current_block(s, b, blk, avg.data(), qhat_b.data(), len, bits);",
+     "write_current_block(s, b, blk, avg.data(), qhat_new.data(), len, bits);", ["test_oracle_registers.py"]),
+    ("own_register_resolution_follows_the_code_width", "const int eo = exponent_rule(rho, M, kOwnResolutionBits);\n    write_own_block(s, a,",
+     "const int eo = exponent_rule(rho, M, bits);\n    write_own_block(s, a,", ["test_oracle_registers.py"]),
+    ("rounding_uniform_halves_swapped", "return (k % 2 == 0) ? (word & 0xFFFFu) : (word >> 16);\n}\n\n// Packing",
+     "return (k % 2 == 1) ? (word & 0xFFFFu) : (word >> 16);\n}\n\n// Packing", ["test_oracle_rng.py"]),
+    ("initial_models_without_the_node_offset", "xi[k] = p + s.offset[i];", "xi[k] = p;", ["test_oracle_rng.py", "test_oracle_interact.py"]),
+    ("labels_without_the_node_shift", "const float score = (float)(acc + (double)s.shift[i] + (double)noise);",
+     "const float score = (float)(acc + (double)noise);", ["test_oracle_local_steps.py"]),
+    ("logistic_class_threshold_one_half", "(score > 0.0f ? 1.0f : 0.0f)", "(score > 0.5f ? 1.0f : 0.0f)", ["test_oracle_local_steps.py"]),
+    ("minibatch_rows_share_one_word", "rows[t] = (int32_t)uniform_int(wd[t % 4], (uint32_t)s.cfg.lsq_m);",
+     "rows[t] = (int32_t)uniform_int(wd[0], (uint32_t)s.cfg.lsq_m);", ["test_oracle_local_steps.py"]),
+    ("write_counter_of_the_responder_not_advanced", "s.w[a] += 1; s.w[b] += 1;\n  s.pbits[a] = bits; s.pbits[b] = bits;",
+     "s.w[a] += 1;\n  s.pbits[a] = bits; s.pbits[b] = bits;", ["test_oracle_interact.py"]),
+    ("magnitude_rule_one_bit_short", "e = std::max(e, fm - 23);", "e = std::max(e, fm - 24);", ["test_oracle_quantizer.py"]),
+    ("publish_range_from_the_maximum_alone", "lo = std::min(lo, v); hi = std::max(hi, v);\n        M = std::max(M, std::fabs(v));\n      }\n      rho = std::max(rho, hi - lo);\n    }\n    const int e = exponent_rule(rho, M, bits);",
+     "hi = std::max(hi, v);\n        M = std::max(M, std::fabs(v));\n      }\n      rho = std::max(rho, hi - lo);\n    }\n    const int e = exponent_rule(rho, M, bits);",
+     ["test_oracle_interact.py"]),
+    ("data_matrix_scaled_by_one_over_d", "const float inv_sqrt_d = (float)(1.0 / std::sqrt((double)d));",
+     "const float inv_sqrt_d = (float)(1.0 / (double)d);", ["test_oracle_local_steps.py"]),
+    ("key_that_is_not_a_number_gets_cell_one", "if (std::isnan(f)) return 0;", "if (std::isnan(f)) return 1;", ["test_oracle_quantizer.py"]),
+    ("saturation_dropped", "if (f >= 2147483648.0f) return std::numeric_limits<int32_t>::max();", "if (f >= 2147483648.0f) return 0;",
+     ["test_oracle_quantizer.py"]),
+    ("sampler_gives_up_after_four_attempts_per_pair", "attempt < 16LL * max_pairs", "attempt < 4LL * max_pairs", ["test_oracle_graph.py"]),
+    ("ring_neighbours_in_the_other_order", "s.adj[(size_t)i * 2 + 0] = (i + n - 1) % n;\n      s.adj[(size_t)i * 2 + 1] = (i + 1) % n;",
+     "s.adj[(size_t)i * 2 + 1] = (i + n - 1) % n;\n      s.adj[(size_t)i * 2 + 0] = (i + 1) % n;", ["test_oracle_graph.py"]),
+    ("geometric_count_capped_at_three", "constexpr int kMaxGeometricTrials = 1024;", "constexpr int kMaxGeometricTrials = 3;",
+     ["test_oracle_local_steps.py"]),
 ]
 
 

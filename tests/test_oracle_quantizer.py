@@ -133,6 +133,9 @@ def test_saturating_conversion_for_distant_keys():
         delta -= 256
     q = (qy + delta + 2**31) % 2**32 - 2**31
     assert got == float(np.float32(q)) * 2.0**e
+    # a key that is not a number has cell 0 (as the float-to-integer conversion of the CUDA side defines it)
+    for c in range(256):
+        assert o.dec(float("nan"), c, e, b) == o.dec(0.0, c, e, b)
 
 
 @pytest.mark.parametrize("b", BITS)

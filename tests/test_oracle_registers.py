@@ -82,6 +82,13 @@ def test_register_interaction_follows_algorithm_1(bits):
     assert np.all(np.abs(decode_current(s, qhat_b, 3, bits).astype(np.float64) - avg) < steps(s.exps[3], s.d))
     assert s.wo.tolist() == [1, 2, 1, 1] and s.w.tolist() == [1, 2, 1, 2]
     assert s.tau.tolist() == [1, 0, 1, 1]
+    # the own register's step is that of an 8-bit code of the guard distance 2 max|Q(X_a) - Q(X_b)| + max|eta h|,
+    # whatever the width of the current registers: 127 steps cover the distance, 127 half-steps would not
+    for blk in range(s.nblk):
+        k = slice(blk * 1024, min(s.d, (blk + 1) * 1024))
+        guard = 2.0 * float(np.abs(Qa[k] - Qb[k]).max()) + float(np.abs(D[k]).max())
+        step = 2.0 ** int(s.oexps[1, blk])
+        assert 127 * step >= guard > 127 * step / 2
 
 
 def test_registers_remove_the_aliasing_plateau_of_the_single_buffer_form():
