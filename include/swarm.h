@@ -20,6 +20,10 @@
  *   - One context is bound to the CUDA device that was current at swarm_init and is
  *     not thread-safe.
  *   - All kernels are compiled for sm_100a only; there is no CPU path.
+ *   - Models and snapshots are expected to be finite. Magnitudes up to the largest float, subnormals and
+ *     decode keys arbitrarily far from the encoded value are defined behaviour (saturating conversions,
+ *     aliased lattice points); a 1024-coordinate block that holds a NaN or an infinity yields unspecified
+ *     values for that block (never a fault: no address depends on model data).
  *
  * Memory layout (row-major, every row padded to a multiple of 1024 elements)
  *   X[n][pitch]   fp32 live models
