@@ -36,7 +36,7 @@ __device__ __forceinline__ void grid_dependency_signal() { asm volatile("griddep
 // Traffic per coordinate: 8 B read, 8 B written, 2*b/8 B of codes written.
 // -----------------------------------------------------------------------------------------
 template <int BITS, bool FUSED>
-__global__ void __launch_bounds__(kWarpsPerCta * 32, FUSED ? 4 : 0)
+__global__ void __launch_bounds__(kWarpsPerCta * 32, 4)   // 128 registers: four CTAs per SM at every code width
 interact_blocking_kernel(StoreView s, const PairList pairs, int64_t total_warps, const FusedSteps fs) {
   grid_dependency_signal();
   grid_dependency_wait();
