@@ -245,13 +245,15 @@ enum {
   SWARM_T_A_RECORD = 14   /* 1 double: ||snapshot - mean||^2 at the node's last initiation                  */
 };
 int swarm_get_tensor(swarm_ctx *ctx, int32_t which, int32_t node, void *dst_host, size_t bytes);
-/* The same read queued on the context's stream without waiting: dst_host (pinned memory, or the copy is
- * not asynchronous) holds the row once swarm_sync, or any other synchronising call issued later, returns.
- * For callers that consume a result of every step without stalling the launch pipeline. Only rows kept
- * in device memory: EINVAL for SWARM_T_ADJ, SWARM_T_COUNTERS, SWARM_T_CLOCKS, SWARM_T_A. Rows of up to 64 KiB
- * going to pinned memory that the device can address are written by a small kernel rather than the copy
- * engine, which keeps back-to-back interaction launches overlapping their launch latency. */
-int swarm_get_tensor_async(swarm_ctx *ctx, int32_t which, int32_t node, void *dst_pinned_host, size_t bytes);
+/* The same read queued on the context's stream without waiting: dst_host (any host memory, which must stay
+ * valid until then) holds the row once swarm_sync, or any other synchronising call issued later (swarm_potential,
+ * swarm_get_tensor, swarm_sample_pairs, ...), returns. For callers that consume a result of every step without
+ * stalling the launch pipeline. Only rows kept in device memory: EINVAL for SWARM_T_ADJ, SWARM_T_COUNTERS,
+ * SWARM_T_CLOCKS, SWARM_T_A. Rows of up to 64 KiB are copied at once, by a small kernel, into a 1 MiB ring inside
+ * the context (the row's value is the one at this point of the stream) and travel to the host in one transfer
+ * at that later call; when the ring is full the call itself synchronises first. Longer rows are copied by the
+ * copy engine straight to dst_host (pinned memory, or that copy is not asynchronous). */
+int swarm_get_tensor_async(swarm_ctx *ctx, int32_t which, int32_t node, void *dst_host, size_t bytes);
 int swarm_set_tensor(swarm_ctx *ctx, int32_t which, int32_t node, const void *src_host, size_t bytes);
 
 /* Whole-context counters: launch counter of the pair sampler and the "snapshots stale" flag. */

@@ -20,6 +20,8 @@ swarm_free_fn g_free = nullptr;
 void* g_alloc_user = nullptr;
 
 constexpr int kStageSlots = 8;
+constexpr size_t kReadQueueBytes = 1u << 20;     // device ring (and pinned mirror) of queued row reads
+constexpr size_t kReadQueueMaxRow = 64u << 10;   // longer rows take the copy engine
 
 }  // namespace
 
@@ -86,6 +88,15 @@ struct swarm_ctx {
   int stage_next = 0;
   double* pot_host = nullptr;        // pinned
   int32_t* pairs_out_host = nullptr; // pinned
+
+  // queued row reads (swarm_get_tensor_async): a small kernel copies the row into a device ring, which keeps the
+  // chain of programmatic dependent launches intact; the used part of the ring travels to its pinned mirror in one
+  // transfer at the next synchronising call, after which the host hands the rows to their destinations
+  struct QueuedRead { void* dst; size_t off, bytes; };
+  uint8_t* rq_dev = nullptr;
+  uint8_t* rq_host = nullptr;        // pinned
+  size_t rq_used = 0;
+  std::vector<QueuedRead> rq;
 };
 
 namespace {
@@ -102,6 +113,23 @@ int fail_cuda(swarm_ctx* c, cudaError_t e) { c->last_cuda = (int)e; return SWARM
   do {                                                       \
     cudaError_t e__ = (call);                                \
     if (e__ != cudaSuccess) return fail_cuda((ctx), e__);    \
+  } while (0)
+
+// Every wait on the context's stream goes through here: rows queued by swarm_get_tensor_async ride along
+// (one transfer of the ring's used part) and are handed to their destinations once the stream is idle.
+int ctx_sync(swarm_ctx* c) {
+  if (!c->rq.empty())
+    SW_CUDA(c, cudaMemcpyAsync(c->rq_host, c->rq_dev, c->rq_used, cudaMemcpyDeviceToHost, c->stream));
+  SW_CUDA(c, cudaStreamSynchronize(c->stream));
+  for (const auto& q : c->rq) std::memcpy(q.dst, c->rq_host + q.off, q.bytes);
+  c->rq.clear();
+  c->rq_used = 0;
+  return SWARM_OK;
+}
+#define SW_SYNC(ctx)                                         \
+  do {                                                       \
+    const int rc__ = ctx_sync(ctx);                          \
+    if (rc__ != SWARM_OK) return rc__;                       \
   } while (0)
 
 void* dev_alloc(swarm_ctx* c, size_t bytes) {
@@ -424,6 +452,8 @@ void swarm_destroy(swarm_ctx* c) {
   dev_free(c, c->X); dev_free(c, c->codes); dev_free(c, c->exps); dev_free(c, c->adj_dev);
   dev_free(c, c->scalars); dev_free(c, c->pot_partial); dev_free(c, c->pot_out);
   dev_free(c, c->pairs_out_dev); dev_free(c, c->used_dev); dev_free(c, c->stage_dev); dev_free(c, c->kernel_status);
+  dev_free(c, c->rq_dev);
+  if (c->rq_host) cudaFreeHost(c->rq_host);
   if (c->kernel_status_host) cudaFreeHost(c->kernel_status_host);
   if (c->stage_host) cudaFreeHost(c->stage_host);
   if (c->pot_host) cudaFreeHost(c->pot_host);
@@ -464,8 +494,10 @@ int swarm_init(swarm_ctx** out, int32_t n, int64_t d, swarm_topology topo, uint6
   c->used_dev = (uint8_t*)dev_alloc(c, (size_t)n);
   c->kernel_status = (int*)dev_alloc(c, sizeof(int));
   c->stage_dev = dev_alloc(c, c->stage_slot_bytes * kStageSlots);
+  c->rq_dev = (uint8_t*)dev_alloc(c, kReadQueueBytes);
   bool ok = c->X && c->codes && c->exps && c->adj_dev && c->scalars && c->pot_partial && c->pot_out &&
-            c->pairs_out_dev && c->used_dev && c->stage_dev && c->kernel_status;
+            c->pairs_out_dev && c->used_dev && c->stage_dev && c->kernel_status && c->rq_dev;
+  ok = ok && cudaMallocHost((void**)&c->rq_host, kReadQueueBytes) == cudaSuccess;
   ok = ok && cudaMallocHost(&c->stage_host, c->stage_slot_bytes * kStageSlots) == cudaSuccess;
   ok = ok && cudaMallocHost((void**)&c->pot_host, 4 * sizeof(double)) == cudaSuccess;
   ok = ok && cudaMemsetAsync(c->pot_out, 0, 5 * sizeof(double), c->stream) == cudaSuccess;
@@ -498,17 +530,17 @@ int swarm_configure(swarm_ctx* c, const swarm_config* cfg) {
   int rc = validate_config(c, cfg);
   if (rc != SWARM_OK) return rc;
   DeviceGuard guard(c->device);
-  SW_CUDA(c, cudaStreamSynchronize(c->stream));
+  SW_SYNC(c);
   rc = apply_config(c, *cfg);
   if (rc != SWARM_OK) return rc;
-  SW_CUDA(c, cudaStreamSynchronize(c->stream));
+  SW_SYNC(c);
   return SWARM_OK;
 }
 
 int swarm_set_stream(swarm_ctx* c, void* cuda_stream) {
   if (!c) return SWARM_EINVAL;
   DeviceGuard guard(c->device);
-  SW_CUDA(c, cudaStreamSynchronize(c->stream));
+  SW_SYNC(c);
   c->stream = (cudaStream_t)cuda_stream;
   return SWARM_OK;
 }
@@ -517,7 +549,7 @@ int swarm_sync(swarm_ctx* c) {
   if (!c) return SWARM_EINVAL;
   DeviceGuard guard(c->device);
   SW_CUDA(c, cudaMemcpyAsync(c->kernel_status_host, c->kernel_status, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
-  SW_CUDA(c, cudaStreamSynchronize(c->stream));
+  SW_SYNC(c);
   if (*c->kernel_status_host != 0) return fail_cuda(c, cudaErrorLaunchTimeout);   // a bounded device wait expired
   return SWARM_OK;
 }
@@ -848,7 +880,7 @@ int swarm_track_staleness(swarm_ctx* c, int32_t enable) {
   if (!c) return SWARM_EINVAL;
   DeviceGuard guard(c->device);
   if (!enable) {
-    SW_CUDA(c, cudaStreamSynchronize(c->stream));
+    SW_SYNC(c);
     dev_free(c, c->mu_hist); c->mu_hist = nullptr;
     dev_free(c, c->a_hist); c->a_hist = nullptr;
     dev_free(c, c->aux_partial); c->aux_partial = nullptr;
@@ -886,7 +918,7 @@ int swarm_aux_potentials(swarm_ctx* c, double* out3) {
   SW_CUDA(c, launch_aux_potentials(view_of(c), c->mu_hist, c->a_hist, c->aux_partial, c->pot_out, c->stream, &nl));
   c->launches += nl;
   SW_CUDA(c, cudaMemcpyAsync(c->pot_host, c->pot_out, 3 * sizeof(double), cudaMemcpyDeviceToHost, c->stream));
-  SW_CUDA(c, cudaStreamSynchronize(c->stream));
+  SW_SYNC(c);
   out3[0] = c->pot_host[0]; out3[1] = c->pot_host[1]; out3[2] = c->pot_host[2];
   return SWARM_OK;
 }
@@ -946,7 +978,7 @@ int swarm_potential(swarm_ctx* c, double* out_gamma) {
   c->launches += nl;
   if (!c->pot_host_dev)
     SW_CUDA(c, cudaMemcpyAsync(c->pot_host, c->pot_out, sizeof(double), cudaMemcpyDeviceToHost, c->stream));
-  SW_CUDA(c, cudaStreamSynchronize(c->stream));
+  SW_SYNC(c);
   *out_gamma = *c->pot_host;
   return SWARM_OK;
 }
@@ -963,7 +995,7 @@ int swarm_sample_pairs(swarm_ctx* c, int32_t max_pairs, swarm_pair* out_pairs, i
   c->launches += nl;
   SW_CUDA(c, cudaMemcpyAsync(c->pairs_out_host, c->pairs_out_dev, (2 * max_slots + 1) * sizeof(int32_t),
                              cudaMemcpyDeviceToHost, c->stream));
-  SW_CUDA(c, cudaStreamSynchronize(c->stream));
+  SW_SYNC(c);
   const int count = c->pairs_out_host[2 * max_slots];
   for (int p = 0; p < count; ++p) { out_pairs[p].a = c->pairs_out_host[2 * p]; out_pairs[p].b = c->pairs_out_host[2 * p + 1]; }
   *out_count = count;
@@ -1049,7 +1081,7 @@ static int tensor_access(swarm_ctx* c, int32_t which, int32_t node, void* host, 
       if (node < 0 || node >= c->groups) return SWARM_ERANGE;
       const size_t m = (size_t)c->cfg.lsq_m;
       if (bytes != m * d * 4) return SWARM_EINVAL;
-      SW_CUDA(c, cudaStreamSynchronize(c->stream));
+      SW_SYNC(c);
       int nl = 0;
       for (size_t r = 0; r < m; ++r) {
         char* hrow = (char*)host + r * d * 4;
@@ -1066,31 +1098,32 @@ static int tensor_access(swarm_ctx* c, int32_t which, int32_t node, void* host, 
             SW_CUDA(c, launch_bf16_to_f32(drow, c->convert_tmp, (int64_t)d, c->stream, &nl));
             SW_CUDA(c, cudaMemcpyAsync(hrow, c->convert_tmp, d * 4, cudaMemcpyDeviceToHost, c->stream));
           }
-          SW_CUDA(c, cudaStreamSynchronize(c->stream));   // convert_tmp and pageable host memory are reused per row
+          SW_SYNC(c);   // convert_tmp and pageable host memory are reused per row
         }
       }
       c->launches += nl;
-      SW_CUDA(c, cudaStreamSynchronize(c->stream));
+      SW_SYNC(c);
       return SWARM_OK;
     }
     default: return SWARM_EINVAL;
   }
   if (bytes != want) return SWARM_EINVAL;
   // the copy is ordered after earlier work by the stream; one synchronisation at the end is enough
-  if (!write && !wait && bytes <= (64u << 10)) {
-    // short queued read into pinned memory that the device can address: a small kernel instead of the copy engine
-    void* mapped = nullptr;
-    if (cudaHostGetDevicePointer(&mapped, host, 0) == cudaSuccess && mapped) {
-      int nl = 0;
-      SW_CUDA(c, launch_row_to_host(dev, mapped, (int64_t)bytes, c->stream, &nl));
-      c->launches += nl;
-      return SWARM_OK;
-    }
-    cudaGetLastError();   // pageable or unmapped destination: the copy engine takes it
+  if (!write && !wait && bytes <= kReadQueueMaxRow) {
+    // short queued read: into the ring now (a small dependent kernel, no copy engine between two launches),
+    // to `host` at the next synchronising call
+    const size_t need = (bytes + 15) / 16 * 16;
+    if (c->rq_used + need > kReadQueueBytes) SW_SYNC(c);          // ring full: deliver what is queued first
+    int nl = 0;
+    SW_CUDA(c, launch_row_copy(dev, c->rq_dev + c->rq_used, (int64_t)bytes, c->stream, &nl));
+    c->launches += nl;
+    c->rq.push_back({host, c->rq_used, bytes});
+    c->rq_used += need;
+    return SWARM_OK;
   }
   if (write) SW_CUDA(c, cudaMemcpyAsync(dev, host, bytes, cudaMemcpyHostToDevice, c->stream));
   else SW_CUDA(c, cudaMemcpyAsync(host, dev, bytes, cudaMemcpyDeviceToHost, c->stream));
-  if (wait) SW_CUDA(c, cudaStreamSynchronize(c->stream));
+  if (wait) SW_SYNC(c);
   return SWARM_OK;
 }
 

@@ -143,10 +143,9 @@ cudaError_t launch_staleness_record(const StoreView& s, float* mu_hist_dev, cons
 cudaError_t launch_aux_potentials(const StoreView& s, const float* mu_hist_dev, const double* a_hist_dev,
                                   double* partial_dev, double* out_dev, cudaStream_t st, int* launches);
 
-// Read-back of a short row by a kernel writing to mapped pinned host memory (keeps the launch pipeline
-// of programmatic dependents intact, which a copy-engine transfer between two launches would not).
-cudaError_t launch_row_to_host(const void* src_dev, void* dst_host_mapped, int64_t bytes, cudaStream_t st,
-                               int* launches);
+// Device-to-device copy of a short row by a small dependent kernel (keeps the launch pipeline of programmatic
+// dependents intact, which a copy-engine transfer between two launches would not).
+cudaError_t launch_row_copy(const void* src_dev, void* dst_dev, int64_t bytes, cudaStream_t st, int* launches);
 
 // Row conversion helpers for get/set of bf16 data.
 cudaError_t launch_bf16_to_f32(const void* src, float* dst, int64_t count, cudaStream_t st, int* launches);

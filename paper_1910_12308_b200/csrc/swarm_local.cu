@@ -483,15 +483,22 @@ sample_pairs_kernel(const int32_t* __restrict__ adj, int n, int degree, int max_
   if (threadIdx.x == 0) *out_count = count_sh;
 }
 
-// Small row read-back into pinned host memory that is mapped into the device's address space: a kernel
-// instead of a copy-engine transfer, launched as a programmatic dependent, so that a row read queued
-// between two interaction launches does not cost them the overlap of launch latency.
+// Small device-to-device row copy (queued row reads): a kernel instead of a copy-engine transfer, launched as
+// a programmatic dependent, so that a row read queued between two interaction launches does not cost them
+// the overlap of launch latency.
 __global__ void __launch_bounds__(256)
-row_to_host_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst_host, int64_t bytes) {
+row_copy_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, int64_t bytes) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < bytes; i += (int64_t)gridDim.x * blockDim.x)
-    dst_host[i] = src[i];
+  const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x, stride = (int64_t)gridDim.x * blockDim.x;
+  if (((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15) == 0) {
+    const int64_t vecs = bytes / 16;
+    for (int64_t i = t; i < vecs; i += stride)
+      reinterpret_cast<uint4*>(dst)[i] = reinterpret_cast<const uint4*>(src)[i];
+    for (int64_t i = vecs * 16 + t; i < bytes; i += stride) dst[i] = src[i];
+  } else {
+    for (int64_t i = t; i < bytes; i += stride) dst[i] = src[i];
+  }
 }
 
 __global__ void bf16_to_f32_kernel(const __nv_bfloat16* src, float* dst, int64_t count) {
@@ -647,10 +654,9 @@ cudaError_t launch_sample_pairs(const int32_t* adj_dev, int n, int degree, int m
   return cudaGetLastError();
 }
 
-cudaError_t launch_row_to_host(const void* src_dev, void* dst_host_mapped, int64_t bytes, cudaStream_t st,
-                               int* launches) {
+cudaError_t launch_row_copy(const void* src_dev, void* dst_dev, int64_t bytes, cudaStream_t st, int* launches) {
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)std::min<int64_t>(cdiv(bytes, 256), 64));
+  cfg.gridDim = dim3((unsigned)std::min<int64_t>(cdiv(bytes, 16 * 256), 16));
   cfg.blockDim = dim3(256);
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
@@ -658,8 +664,8 @@ cudaError_t launch_row_to_host(const void* src_dev, void* dst_host_mapped, int64
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  const cudaError_t e = cudaLaunchKernelEx(&cfg, row_to_host_kernel, reinterpret_cast<const uint8_t*>(src_dev),
-                                           reinterpret_cast<uint8_t*>(dst_host_mapped), bytes);
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, row_copy_kernel, reinterpret_cast<const uint8_t*>(src_dev),
+                                           reinterpret_cast<uint8_t*>(dst_dev), bytes);
   ++*launches;
   return e != cudaSuccess ? e : cudaGetLastError();
 }

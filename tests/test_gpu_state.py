@@ -88,3 +88,28 @@ def test_asynchronous_row_read_arrives_after_sync():
     assert sw.get_async(g.T_COUNTERS, 0, small) == g.EINVAL          # host-side rows have no asynchronous form
     assert sw.get_async(g.T_X, 9, out) == g.ERANGE
     assert sw.get_async(g.T_X, 0, exps) == g.EINVAL                  # size mismatch
+
+
+def test_queued_row_reads_keep_the_value_of_their_point_in_the_stream():
+    """A queued read returns the row as it was when queued, even if later launches change it before the
+    synchronising call; any synchronising call delivers (here the potential), destinations need not be pinned,
+    and more rows than the context's ring holds are still all delivered."""
+    sw = g.Swarm(4, 5000, "complete", 0, 3)
+    sw.configure(offset_std=0.2)
+    before = sw.get(g.T_X, 0).copy()
+    first = np.zeros(5000, dtype=np.float32)                         # pageable memory
+    assert sw.get_async(g.T_X, 0, first) == 0
+    assert sw.interact([[0, 1]], 8) == 0                             # changes row 0 after the read was queued
+    second = np.zeros(5000, dtype=np.float32)
+    assert sw.get_async(g.T_X, 0, second) == 0
+    sw.potential()                                                   # synchronises: both rows are there
+    assert np.array_equal(first, before)
+    assert np.array_equal(second, sw.get(g.T_X, 0)) and not np.array_equal(first, second)
+    # 80 rows of 20,000 bytes exceed the 1 MiB ring: the call that finds it full delivers the queued ones first
+    outs = [np.zeros(5000, dtype=np.float32) for _ in range(80)]
+    rows = [sw.get(g.T_X, i % 4) for i in range(4)]
+    for i, o_ in enumerate(outs):
+        assert sw.get_async(g.T_X, i % 4, o_) == 0
+    sw.sync()
+    for i, o_ in enumerate(outs):
+        assert np.array_equal(o_, rows[i % 4])
