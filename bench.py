@@ -464,7 +464,7 @@ def run_ours(args, wl, name):
                                 ["interact_blocking_kernel", "interact_nonblocking_kernel", "interact_registers_kernel"][wl["mode"]])
                      + (" (local steps fused)" if fused else ""),
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_kind": peak_kind, "frac_of_8000": achieved / 8000.0, "traffic": TRAFFIC.get(name),
+                     "peak_kind": peak_kind, "frac_of_8000": achieved / 8000.0, "traffic": traffic_of(name, npairs_total / K),
                      "algorithmic_bytes_per_launch": per_launch_bytes, "kernel_ms": kern_ms},
     }
     if wl["mode"] == 2 and not fused:
@@ -476,7 +476,7 @@ def run_ours(args, wl, name):
         issue_peak = 148 * 4 * (clocks["sm_max_mhz"] or 1965) * 1e6 / 1e12
         hbm = out["roofline"]
         out["roofline"] = {"bound": "alu", "kernel": hbm["kernel"], "achieved": rate, "peak": issue_peak,
-                           "unit": "T warp-instructions/s", "frac": rate / issue_peak, "traffic": TRAFFIC.get(name),
+                           "unit": "T warp-instructions/s", "frac": rate / issue_peak, "traffic": traffic_of(name, npairs_total / K),
                            "warp_instructions_per_launch": instr, "kernel_ms": kern_ms,
                            "hbm": {k: hbm[k] for k in ("achieved", "peak", "unit", "frac", "peak_kind", "frac_of_8000",
                                                        "algorithmic_bytes_per_launch")}}
@@ -556,8 +556,20 @@ def run_ours(args, wl, name):
 # ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel (see profiles/);
 # None until a capture of the current kernel exists.
 TRAFFIC = {"ring64_d1m_b4": 512.1e6}
+# the same per pair of a launch, for workloads whose launches differ in their number of pairs: captured on a reduced
+# copy (8 nodes, 3 pairs per launch) for the single-buffer kernel and on the full workload (14 pairs) for the
+# two-register kernel; traffic is proportional to the pairs of a launch (every pair streams its own rows once)
+TRAFFIC_PER_PAIR = {"regular32_resnet18_b8_nb": 214.8e6, "regular32_resnet18_b8_reg": 288.1e6}
 # smsp__inst_executed.sum per 1024-coordinate block of interact_registers_kernel<8> (see profiles/)
 REGISTER_KERNEL_INSTR_PER_BLOCK = 3607
+
+
+def traffic_of(name, pairs_per_launch):
+    if name in TRAFFIC:
+        return TRAFFIC[name]
+    if name in TRAFFIC_PER_PAIR:
+        return TRAFFIC_PER_PAIR[name] * pairs_per_launch
+    return None
 
 
 def main():
