@@ -73,6 +73,54 @@ def test_large_model_sampled_pair_bit_exact(d, bits, mode):
     assert not gpu.get(g.T_CODES, 1)[d * bits // 8: orc.nblk * 128 * bits].any()
 
 
+@pytest.mark.parametrize("workload", ["regular32_resnet18_b8_nb", "complete16_resnet50_b4", "regular256_d1m_b2_lsq_nb"])
+def test_full_store_launch_checked_on_the_pair_with_the_highest_node(workload):
+    """The benchmark's store and launch shape at full size (32 x 11.7 M, 16 x 25.6 M and 256 x 1 M coordinates: row
+    offsets beyond 2^31 bytes, up to 128 pairs per launch from the benchmark's own schedule); the oracle recomputes
+    the pair that contains the last node. The objective is the synthetic one in all three (the least-squares data
+    of the 256-node workload is covered at 32 nodes below), with the oracle's own initial state switched off: its
+    rows for the checked pair are copies of the CUDA state."""
+    import bench
+    wl = bench.WORKLOADS[workload]
+    n, d, bits, mode = wl["n"], wl["d"], wl["bits"], wl["mode"]
+    cfg = dict(objective=1, nonblocking=mode, grad_std=float(np.sqrt(1e-3)), drift_std=float(np.sqrt(0.05)))
+    gpu = g.Swarm(n, d, wl["topology"], wl["degree"], wl["seed"])
+    gpu.configure(**cfg)
+    sched = bench.PairSchedule(wl, gpu.get_all(g.T_ADJ))
+    pairs = sched.next()
+    assert len(pairs) >= wl["pairs"] * 3 // 4
+    if mode == 1:
+        assert gpu.publish(bits) == 0
+    assert gpu.local_steps(pairs.reshape(-1), 2, 0.05) == 0       # pending updates for the one-way exchange
+    sample = [p for p in pairs.tolist() if n - 1 in p] or [pairs[-1].tolist()]
+    a, b = sample[0]
+    orc = o.OracleSwarm(n, d, wl["topology"], wl["degree"], wl["seed"])
+    orc.configure(objective=1, nonblocking=mode, grad_std=0.0, drift_std=0.0, init_std=0.0)
+    for i in (a, b):
+        orc.X[i] = gpu.get(g.T_X, i)
+        orc.w[i] = gpu.get(g.T_COUNTERS, i)[0]
+        if mode == 1:
+            orc.B[i] = gpu.get(g.T_B, i)
+            orc.codes[i] = gpu.get(g.T_CODES, i)
+            orc.exps[i] = gpu.get(g.T_EXPS, i)
+    if mode == 1:
+        orc.pbits[:] = bits
+        orc.p_mode[0] = 1
+    assert gpu.interact(pairs, bits, mode) == 0
+    assert orc.interact([[a, b]], bits, mode) == 0
+    for i in (a, b):
+        assert np.array_equal(gpu.get(g.T_X, i).view(np.uint32), orc.X[i].view(np.uint32)), i
+        assert np.array_equal(gpu.get(g.T_CODES, i)[: orc.nblk * 128 * bits], orc.packed_codes(i, bits)), i
+        assert np.array_equal(gpu.get(g.T_EXPS, i), orc.exps[i]), i
+        if mode == 1:
+            assert np.array_equal(gpu.get(g.T_B, i).view(np.uint32), orc.B[i].view(np.uint32)), i
+    # a bystander of the launch with a high node id kept its rows unless it was in a pair
+    touched = set(pairs.reshape(-1).tolist())
+    idle = [i for i in range(n - 1, -1, -1) if i not in touched]
+    if idle:
+        assert gpu.get(g.T_COUNTERS, idle[0])[0] == (1 if mode == 1 else 0)
+
+
 def test_config1_trajectory_teacher_forced():
     """n = 8, d = 4096, least squares 64 x 4096, H = 2, batch 16, lr = 0.05, 8-bit, one pair per
     interaction, seed 0: local steps within tolerance, interactions bit-exact."""
