@@ -77,7 +77,7 @@ def test_large_model_sampled_pair_bit_exact(d, bits, mode):
 def test_full_store_launch_checked_on_the_pair_with_the_highest_node(workload):
     """The benchmark's store and launch shape at full size (32 x 11.7 M, 16 x 25.6 M and 256 x 1 M coordinates: row
     offsets beyond 2^31 bytes, up to 128 pairs per launch from the benchmark's own schedule); the oracle recomputes
-    the pair that contains the last node. The objective is the synthetic one in all three (the least-squares data
+    the pair that contains the last node, and that node's local steps. The objective is the synthetic one in all three (the least-squares data
     of the 256-node workload is covered at 32 nodes below), with the oracle's own initial state switched off: its
     rows for the checked pair are copies of the CUDA state."""
     import bench
@@ -91,11 +91,18 @@ def test_full_store_launch_checked_on_the_pair_with_the_highest_node(workload):
     assert len(pairs) >= wl["pairs"] * 3 // 4
     if mode == 1:
         assert gpu.publish(bits) == 0
-    assert gpu.local_steps(pairs.reshape(-1), 2, 0.05) == 0       # pending updates for the one-way exchange
     sample = [p for p in pairs.tolist() if n - 1 in p] or [pairs[-1].tolist()]
     a, b = sample[0]
+    last = max(a, b)
+    x_before = gpu.get(g.T_X, last).copy()
+    assert gpu.local_steps(pairs.reshape(-1), 2, 0.05) == 0       # pending updates for the one-way exchange
     orc = o.OracleSwarm(n, d, wl["topology"], wl["degree"], wl["seed"])
-    orc.configure(objective=1, nonblocking=mode, grad_std=0.0, drift_std=0.0, init_std=0.0)
+    orc.configure(objective=1, nonblocking=mode, grad_std=cfg["grad_std"], drift_std=cfg["drift_std"], init_std=0.0)
+    # the last node's two local steps, recomputed from its row before the steps
+    orc.X[last] = x_before
+    orc.drift[last] = gpu.get(g.T_SCALARS, last)[1]
+    assert orc.local_steps([last], 2, 0.05) == 0
+    assert rel_err(gpu.get(g.T_X, last), orc.X[last]) < 1e-6
     for i in (a, b):
         orc.X[i] = gpu.get(g.T_X, i)
         orc.w[i] = gpu.get(g.T_COUNTERS, i)[0]
