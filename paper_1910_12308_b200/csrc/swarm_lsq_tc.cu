@@ -124,17 +124,18 @@ __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bflo
 //   A    : 2 atoms x [64 rows x 128 B]   (K-major, 128B swizzle, 8-row groups 1024 B apart)  16 KiB
 // plus two operand buffers Xhi/Xlo: 2 atoms x [16 rows x 128 B] each. The fp32 models are loaded one
 // tile ahead into registers (8 coordinates per thread) and converted to bf16 hi/lo straight into the
-// operand buffers. Five stages of A: 97 KiB per CTA, two CTAs per SM so that one CTA's barrier and
-// operand conversion hide behind the other's copies.
+// operand buffers. Three stages of A: 65 KiB per CTA, three CTAs per SM, so that one CTA's barrier and
+// operand conversion hide behind the copies of the other two (measured against five stages and two CTAs per
+// SM at the 256-node workload: 5 % off the whole step).
 // =================================================================================================
 constexpr int kResTile = 128;
 constexpr int kResAtoms = kResTile / 64;
-constexpr int kResStages = 5;
+constexpr int kResStages = 3;
 constexpr int kResABytes = kResAtoms * kTcBatch * 128;         // 16384
 constexpr int kResXopBytes = kResAtoms * kUnitNodes * 128;     // 4096 (one of hi / lo)
 constexpr int kResSmem = kResStages * kResABytes + 2 * 2 * kResXopBytes + 1024 /*align*/ + 64;
 
-__global__ void __launch_bounds__(kTcThreads, 2)
+__global__ void __launch_bounds__(kTcThreads, 3)
 lsq_tc_residual_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, int step, float* __restrict__ partial,
                        int64_t chunk_coords, int64_t nchunks, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
@@ -308,7 +309,7 @@ lsq_tc_finalize_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units
 //   [half h of 64 coordinates][8 groups of 8 sampled rows][8 rows x 128 B], 128B swizzle
 //   (leading byte offset = 8192 between halves, stride byte offset = 1024 between row groups).
 // B operand = resid hi / lo, K-major [16 nodes x 64 rows] (one swizzle atom each).
-// Accumulators: 128 lanes x 16 columns, two buffers.
+// Accumulators: 128 lanes x 16 columns, two buffers. Four stages: 70 KiB per CTA, three CTAs per SM (72 registers).
 // =================================================================================================
 constexpr int kUpdTile = 128;
 constexpr int kUpdStages = 4;
@@ -316,7 +317,7 @@ constexpr int kUpdABytes = kTcBatch * kUpdTile * 2;             // 16384
 constexpr int kUpdRBytes = kUnitNodes * 128;                   // 2048 (one of hi / lo)
 constexpr int kUpdSmem = kUpdStages * kUpdABytes + 2 * kUpdRBytes + 1024 + 64;
 
-__global__ void __launch_bounds__(kTcThreads, 2)
+__global__ void __launch_bounds__(kTcThreads, 3)
 lsq_tc_update_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, int step, float lr,
                      const __nv_bfloat16* __restrict__ resid, int64_t chunk_coords, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
