@@ -17,6 +17,11 @@
  *     call changes no state and no counter.
  *   - Device work is asynchronous on the context's stream and ordered by call order.
  *     swarm_potential, swarm_get_tensor, swarm_sample_pairs and swarm_sync wait for it.
+ *   - Device-side waits are bounded (only the tensor-core local-step kernels have any). A kernel whose wait
+ *     runs out raises a status word, writes no result and returns; later kernels of the context that would
+ *     build on its result return at once. Every synchronising call checks that word: from then on each of them
+ *     returns SWARM_ECUDA with swarm_last_cuda_error() == cudaErrorLaunchTimeout (the models are in an
+ *     undefined state) until swarm_configure rebuilds the context from its seed.
  *   - One context is bound to the CUDA device that was current at swarm_init and is
  *     not thread-safe.
  *   - All kernels are compiled for sm_100a only; there is no CPU path.
@@ -195,7 +200,10 @@ int swarm_aux_potentials(swarm_ctx *ctx, double *out3_host);
  * ---------------------------------------------------------------------------------------- */
 
 /* Apply a workload description and rebuild the state from the seed (models, per-node scalars,
- * data, counters). Errors: EINVAL, ENOMEM, ECUDA. */
+ * data, counters). The buffers of the previous configuration are released first. If the new ones cannot be
+ * allocated the call returns ENOMEM and leaves the context in the default configuration of swarm_init (no
+ * objective, no snapshots, init_std = 0.1, state rebuilt from the seed), never with a configuration whose
+ * buffers are missing. Errors: EINVAL (nothing changed), ENOMEM, ECUDA. */
 int swarm_configure(swarm_ctx *ctx, const swarm_config *cfg_host);
 
 /* Algorithm 1, sampling lines: draw up to max_pairs disjoint pairs for the next launch
@@ -274,7 +282,8 @@ int swarm_model_ptr(swarm_ctx *ctx, float **x_dev, int64_t *pitch);
  * framework that passes only raw pointers -- and therefore cannot create a context (contexts allocate
  * their scratch) or tolerate cudaMalloc's device-wide synchronisation and late failure.
  *   x_dev          n rows of d floats, row i at x_dev + i*pitch (device memory, read only; pitch >= d,
- *                  in elements; rows 16-byte aligned and pitch a multiple of 4 take the fast path)
+ *                  in elements; when x_dev is 16-byte aligned and pitch a multiple of 4 every row is, and the
+ *                  rows are read with 128-bit loads; any other float-aligned base or pitch is read element by element)
  *   out_gamma_dev  one double in device memory, written asynchronously on cuda_stream
  *   cuda_stream    cudaStream_t (NULL = default stream) on the current device
  * Gamma = sum_i ||X^i - mu||^2 as in swarm_potential, same arithmetic. The per-CTA partial sums live in a
@@ -283,13 +292,21 @@ int swarm_model_ptr(swarm_ctx *ctx, float **x_dev, int64_t *pitch);
  * launched. All calls share that array: calls on one stream are ordered and safe, calls that may overlap
  * on the same GPU race on it. The first call made with a given device current looks up the array's
  * device address (no allocation); make that first call before starting any stream capture.
- * Errors: EINVAL (NULL pointer, n < 2, d < 1, pitch < d, d > SWARM_STATIC_MAX_D), ECUDA. */
+ * Errors: EINVAL (NULL pointer, x_dev not 4-byte or out_gamma_dev not 8-byte aligned, n < 2, d < 1, pitch < d,
+ * d > SWARM_STATIC_MAX_D), ECUDA. */
 #define SWARM_STATIC_MAX_D 33554432
 int swarm_potential_static(const float *x_dev, int32_t n, int64_t d, int64_t pitch, double *out_gamma_dev,
                            void *cuda_stream);
 
 int swarm_set_stream(swarm_ctx *ctx, void *cuda_stream);   /* cudaStream_t; NULL = default stream */
 int swarm_sync(swarm_ctx *ctx);
+/* Failure detection (the paper has no counterpart): the number of polls after which a device-side wait gives
+ * up (see "Device-side waits are bounded" above). polls < 0 restores the default (2^22 polls; one poll may
+ * itself block for a hardware-defined time, so this is seconds). polls = 0 makes every such wait give up at
+ * once, which is how the error path is exercised on a healthy GPU without faulting or hanging it: the
+ * kernel still waits, bounded by the default, for its own tensor-core work before it releases tensor memory.
+ * Errors: EINVAL (NULL, polls >= 2^32). */
+int swarm_set_wait_limit(swarm_ctx *ctx, int64_t polls);
 int64_t swarm_kernel_launches(swarm_ctx *ctx);             /* kernels launched so far by this context */
 int swarm_last_cuda_error(swarm_ctx *ctx);                 /* cudaError_t of the last SWARM_ECUDA       */
 const char *swarm_strerror(int code);

@@ -29,7 +29,7 @@ EXPORTS = [
     "swarm_potential", "swarm_track_staleness", "swarm_aux_potentials", "swarm_configure", "swarm_sample_pairs", "swarm_publish", "swarm_register_publish", "swarm_set_own_prefix", "swarm_get_own_prefix", "swarm_get_buffer_mode",
     "swarm_set_buffer_mode", "swarm_get_tensor", "swarm_get_tensor_async",
     "swarm_set_tensor", "swarm_get_state", "swarm_set_state", "swarm_model_ptr", "swarm_set_stream",
-    "swarm_sync", "swarm_potential_static", "swarm_kernel_launches", "swarm_last_cuda_error", "swarm_strerror", "swarm_destroy",
+    "swarm_sync", "swarm_set_wait_limit", "swarm_potential_static", "swarm_kernel_launches", "swarm_last_cuda_error", "swarm_strerror", "swarm_destroy",
 ]
 
 
@@ -107,6 +107,7 @@ def load():
         "swarm_potential_static": (C.c_int, [vp, i32, i64, i64, vp, vp]),
         "swarm_set_stream": (C.c_int, [vp, vp]),
         "swarm_sync": (C.c_int, [vp]),
+        "swarm_set_wait_limit": (C.c_int, [vp, i64]),
         "swarm_kernel_launches": (i64, [vp]),
         "swarm_last_cuda_error": (C.c_int, [vp]),
         "swarm_strerror": (C.c_char_p, [C.c_int]),
@@ -305,6 +306,13 @@ class Swarm:
 
     def sync(self):
         self._check(self._L.swarm_sync(self._h), "swarm_sync")
+
+    def set_wait_limit(self, polls):
+        """Polls after which a device-side wait gives up (negative = default, 0 = at once); returns the C code."""
+        return int(self._L.swarm_set_wait_limit(self._h, polls))
+
+    def last_cuda_error(self):
+        return int(self._L.swarm_last_cuda_error(self._h))
 
     def kernel_launches(self):
         return int(self._L.swarm_kernel_launches(self._h))

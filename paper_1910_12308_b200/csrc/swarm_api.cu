@@ -4,6 +4,7 @@
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -15,6 +16,8 @@ using namespace swarm;
 
 namespace {
 
+// process-wide allocator hook: read by swarm_init, written by swarm_set_allocator, under g_alloc_mutex
+std::mutex g_alloc_mutex;
 swarm_alloc_fn g_alloc = nullptr;
 swarm_free_fn g_free = nullptr;
 void* g_alloc_user = nullptr;
@@ -68,6 +71,9 @@ struct swarm_ctx {
   void* tc_resid = nullptr;          // tensor-core path: residuals as bf16 hi / lo
   int* kernel_status = nullptr;      // set by a kernel whose bounded wait expired
   int* kernel_status_host = nullptr; // pinned
+  bool status_pending = false;       // kernels with bounded waits were launched since the status word was last read
+  bool poisoned = false;             // a bounded wait expired: the state is undefined until swarm_configure
+  uint32_t wait_limit = 0;           // polls per bounded device wait
   double* pot_partial = nullptr;
   double* pot_out = nullptr;         // 4 doubles, then the ticket counter of the potential kernel
   double* pot_host_dev = nullptr;    // device-visible address of pot_host (nullptr: not mapped)
@@ -117,13 +123,22 @@ int fail_cuda(swarm_ctx* c, cudaError_t e) { c->last_cuda = (int)e; return SWARM
 
 // Every wait on the context's stream goes through here: rows queued by swarm_get_tensor_async ride along
 // (one transfer of the ring's used part) and are handed to their destinations once the stream is idle.
-int ctx_sync(swarm_ctx* c) {
+// The status word of the kernels with bounded waits travels the same way when such kernels ran since it was last
+// read; once it has been seen set, every synchronising call reports the expired wait (cudaErrorLaunchTimeout).
+int ctx_sync(swarm_ctx* c, bool report_expired_wait = true) {
   if (!c->rq.empty())
     SW_CUDA(c, cudaMemcpyAsync(c->rq_host, c->rq_dev, c->rq_used, cudaMemcpyDeviceToHost, c->stream));
+  if (c->status_pending)
+    SW_CUDA(c, cudaMemcpyAsync(c->kernel_status_host, c->kernel_status, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
   SW_CUDA(c, cudaStreamSynchronize(c->stream));
   for (const auto& q : c->rq) std::memcpy(q.dst, c->rq_host + q.off, q.bytes);
   c->rq.clear();
   c->rq_used = 0;
+  if (c->status_pending) {
+    c->status_pending = false;
+    if (*c->kernel_status_host != 0) c->poisoned = true;
+  }
+  if (c->poisoned && report_expired_wait) return fail_cuda(c, cudaErrorLaunchTimeout);
   return SWARM_OK;
 }
 #define SW_SYNC(ctx)                                         \
@@ -259,12 +274,10 @@ int stage_release(swarm_ctx* c, int slot) {
   return SWARM_OK;
 }
 
-int apply_config(swarm_ctx* c, const swarm_config& cfg) {
-  free_objective(c);
-  c->cfg = cfg;
+// Device buffers that a configuration needs beyond the ones every context has.
+int alloc_objective(swarm_ctx* c, const swarm_config& cfg) {
   const int n = c->n;
   const size_t row_bytes = (size_t)c->pitch * sizeof(float);
-  int nl = 0;
   if (cfg.nonblocking) {
     c->B = (float*)dev_alloc(c, (size_t)n * row_bytes);
     if (!c->B) return SWARM_ENOMEM;
@@ -290,10 +303,39 @@ int apply_config(swarm_ctx* c, const swarm_config& cfg) {
       if (!c->tc_partial || !c->tc_resid) return SWARM_ENOMEM;
     }
   }
+  return SWARM_OK;
+}
+
+swarm_config default_config() {
+  swarm_config def{};
+  def.objective = SWARM_OBJ_NONE; def.nonblocking = 0; def.init_std = 0.1f;
+  return def;
+}
+
+// Rebuilds the whole state from the seed under `wanted`. The old objective buffers are released first (a data
+// matrix can be most of the device's memory, so old and new are never held together). When an allocation
+// fails, what was allocated is released again and the context is rebuilt under the default configuration (no
+// objective, no snapshots: what swarm_init leaves, which needs no further memory), so that it never holds a
+// configuration whose buffers are missing; the call then returns SWARM_ENOMEM.
+int apply_config(swarm_ctx* c, const swarm_config& wanted) {
+  free_objective(c);
+  swarm_config cfg = wanted;
+  int result = alloc_objective(c, cfg);
+  if (result != SWARM_OK) {
+    free_objective(c);
+    cfg = default_config();
+  }
+  c->cfg = cfg;
+  const int n = c->n;
+  const size_t row_bytes = (size_t)c->pitch * sizeof(float);
+  int nl = 0;
   StoreView s = view_of(c);
   SW_CUDA(c, cudaMemsetAsync(c->X, 0, (size_t)n * row_bytes, c->stream));
   SW_CUDA(c, cudaMemsetAsync(c->codes, 0, (size_t)n * c->nblk * kBlockCoords, c->stream));
   SW_CUDA(c, cudaMemsetAsync(c->exps, 0, (size_t)n * c->nblk, c->stream));
+  SW_CUDA(c, cudaMemsetAsync(c->kernel_status, 0, sizeof(int), c->stream));
+  c->status_pending = false;
+  c->poisoned = false;
   if (c->own) {
     SW_CUDA(c, cudaMemsetAsync(c->own, 0, (size_t)n * c->nblk * 2 * kBlockCoords, c->stream));
     SW_CUDA(c, cudaMemsetAsync(c->oexps, 0, (size_t)n * c->nblk, c->stream));
@@ -315,7 +357,7 @@ int apply_config(swarm_ctx* c, const swarm_config& cfg) {
   c->b_stale = 0;
   c->p_mode = 0;
   c->own_prefix = 16;
-  return SWARM_OK;
+  return result;
 }
 
 int validate_config(const swarm_ctx* c, const swarm_config* cfg) {
@@ -427,6 +469,7 @@ extern "C" {
 
 int swarm_set_allocator(swarm_alloc_fn alloc_fn, swarm_free_fn free_fn, void* user) {
   if ((alloc_fn == nullptr) != (free_fn == nullptr)) return SWARM_EINVAL;
+  std::lock_guard<std::mutex> lock(g_alloc_mutex);
   g_alloc = alloc_fn; g_free = free_fn; g_alloc_user = user;
   return SWARM_OK;
 }
@@ -473,8 +516,12 @@ int swarm_init(swarm_ctx** out, int32_t n, int64_t d, swarm_topology topo, uint6
   c->nblk = (d + kBlockCoords - 1) / kBlockCoords;
   c->pitch = c->nblk * kBlockCoords;
   c->topo_kind = topo.kind; c->degree = topo.degree;
-  c->custom_alloc = g_alloc != nullptr;
-  c->alloc_fn = g_alloc; c->free_fn = g_free; c->alloc_user = g_alloc_user;
+  {
+    std::lock_guard<std::mutex> lock(g_alloc_mutex);
+    c->custom_alloc = g_alloc != nullptr;
+    c->alloc_fn = g_alloc; c->free_fn = g_free; c->alloc_user = g_alloc_user;
+  }
+  c->wait_limit = lsq_tc_default_wait_limit();
   if (!build_graph(c)) { delete c; return SWARM_EINVAL; }
   c->w.assign(n, 0); c->ls.assign(n, 0); c->pbits.assign(n, 0); c->wo.assign(n, 0); c->tau.assign(n, 0);
 
@@ -516,9 +563,7 @@ int swarm_init(swarm_ctx** out, int32_t n, int64_t d, swarm_topology topo, uint6
   cudaError_t e = cudaMemcpyAsync(c->adj_dev, c->adj.data(), c->adj.size() * sizeof(int32_t), cudaMemcpyHostToDevice,
                                   c->stream);
   if (e != cudaSuccess) { swarm_destroy(c); return SWARM_ECUDA; }
-  swarm_config def{};
-  def.objective = SWARM_OBJ_NONE; def.nonblocking = 0; def.init_std = 0.1f;
-  int rc = apply_config(c, def);
+  int rc = apply_config(c, default_config());
   if (rc == SWARM_OK && cudaStreamSynchronize(c->stream) != cudaSuccess) rc = SWARM_ECUDA;
   if (rc != SWARM_OK) { swarm_destroy(c); return rc; }
   *out = c;
@@ -530,11 +575,11 @@ int swarm_configure(swarm_ctx* c, const swarm_config* cfg) {
   int rc = validate_config(c, cfg);
   if (rc != SWARM_OK) return rc;
   DeviceGuard guard(c->device);
-  SW_SYNC(c);
-  rc = apply_config(c, *cfg);
+  rc = ctx_sync(c, false);          // a context whose bounded wait expired is rebuilt here, not refused
   if (rc != SWARM_OK) return rc;
+  rc = apply_config(c, *cfg);
   SW_SYNC(c);
-  return SWARM_OK;
+  return rc;
 }
 
 int swarm_set_stream(swarm_ctx* c, void* cuda_stream) {
@@ -548,9 +593,13 @@ int swarm_set_stream(swarm_ctx* c, void* cuda_stream) {
 int swarm_sync(swarm_ctx* c) {
   if (!c) return SWARM_EINVAL;
   DeviceGuard guard(c->device);
-  SW_CUDA(c, cudaMemcpyAsync(c->kernel_status_host, c->kernel_status, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
-  SW_SYNC(c);
-  if (*c->kernel_status_host != 0) return fail_cuda(c, cudaErrorLaunchTimeout);   // a bounded device wait expired
+  SW_SYNC(c);      // also reports a bounded device wait that expired
+  return SWARM_OK;
+}
+
+int swarm_set_wait_limit(swarm_ctx* c, int64_t polls) {
+  if (!c || polls > (int64_t)UINT32_MAX) return SWARM_EINVAL;
+  c->wait_limit = polls < 0 ? lsq_tc_default_wait_limit() : (uint32_t)polls;
   return SWARM_OK;
 }
 
@@ -606,7 +655,8 @@ int swarm_local_steps(swarm_ctx* c, const int32_t* node_ids, int32_t count, int3
     if (rc != SWARM_OK) return rc;
     int nl = 0;
     SW_CUDA(c, launch_local_lsq_tc(view_of(c), lsq_of(c), (const LsqUnit*)dev, (int)units.size(), H, lr, c->tc_partial,
-                                   c->tc_resid, c->kernel_status, c->stream, &nl));
+                                   c->tc_resid, c->kernel_status, c->wait_limit, c->stream, &nl));
+    c->status_pending = true;
     c->launches += nl;
     rc = stage_release(c, slot);
     if (rc != SWARM_OK) return rc;

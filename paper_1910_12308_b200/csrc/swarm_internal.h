@@ -120,10 +120,12 @@ cudaError_t launch_lsq_sequence(const StoreView& s, const LsqView& l, const Pair
 // --- swarm_lsq_tc.cu (bf16 data, batch <= 64) ----------------------------------------------
 size_t lsq_tc_partial_bytes(int64_t pitch, int units);
 size_t lsq_tc_resid_bytes(int units);
-// status_dev: one int, set to 1 if a bounded wait inside a kernel expired.
+// status_dev: one int, set to 1 if a bounded wait inside a kernel expired (kernels that find it set return at
+// once); wait_limit: polls after which a wait on a tensor-core commit gives up.
 cudaError_t launch_local_lsq_tc(const StoreView& s, const LsqView& l, const LsqUnit* units_dev, int nunits, int H,
-                                float lr, float* partial_dev, void* resid_dev, int* status_dev, cudaStream_t st,
-                                int* launches);
+                                float lr, float* partial_dev, void* resid_dev, int* status_dev, uint32_t wait_limit,
+                                cudaStream_t st, int* launches);
+uint32_t lsq_tc_default_wait_limit();
 cudaError_t launch_sample_pairs(const int32_t* adj_dev, int n, int degree, int max_pairs, uint32_t launch_ctr,
                                 uint32_t key0, uint32_t key1, int32_t* out_pairs_dev, int32_t* out_count_dev,
                                 uint8_t* used_dev, cudaStream_t st, int* launches);

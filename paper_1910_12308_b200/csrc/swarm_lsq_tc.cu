@@ -18,8 +18,14 @@
 //                           writes resid as bf16 hi/lo
 //   lsq_tc_update_kernel    CTA = (k-chunk, unit): D = A_S^T resid per 128-coordinate tile, x -= scale * D
 // Operand tiles are staged with cp.async into the 128-byte-swizzled shared-memory layouts the MMA
-// descriptors name. Every wait on an mbarrier is bounded; on expiry the kernel raises a status word,
-// drains its copies, frees its tensor memory and returns.
+// descriptors name. Every wait on an mbarrier is bounded (spin_limit polls). A wait's outcome is made
+// warp-uniform by a vote and CTA-uniform at the tile loop's barrier, so all threads of a CTA leave the loop
+// together; the CTA then raises the status word, drains its copies, waits (bounded by the full default limit,
+// whatever spin_limit says) for the last MMA commit so that no MMA is in flight, frees its tensor memory and
+// returns without writing results. Kernels that find the status word set on entry return at once, so a step
+// that gave up is not built upon.
+#include <mutex>
+
 #include <cuda_bf16.h>
 
 #include "swarm_dev.cuh"
@@ -53,11 +59,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
                : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait: false when the limit expired.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
-  return false;
+// Bounded wait, called by whole warps: false for every lane when the limit expired in any lane.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t limit) {
+  bool done = false;
+  for (uint32_t i = 0; i < limit && !done; ++i) done = mbar_try_wait(bar, parity);
+  return __all_sync(0xFFFFFFFFu, done);
+}
+// True (for the whole CTA) when an earlier kernel on this context gave up; called by all threads.
+__device__ __forceinline__ bool status_raised(const int* status, int* flag_smem) {
+  if (threadIdx.x == 0) *flag_smem = *reinterpret_cast<const volatile int*>(status);
+  __syncthreads();
+  return *flag_smem != 0;
 }
 __device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t cols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(slot_smem), "r"(cols) : "memory");
@@ -137,7 +149,9 @@ constexpr int kResSmem = kResStages * kResABytes + 2 * 2 * kResXopBytes + 1024 /
 
 __global__ void __launch_bounds__(kTcThreads, 3)
 lsq_tc_residual_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, int step, float* __restrict__ partial,
-                       int64_t chunk_coords, int64_t nchunks, int* __restrict__ status) {
+                       int64_t chunk_coords, int64_t nchunks, int* __restrict__ status, uint32_t spin_limit) {
+  __shared__ int poisoned;
+  if (status_raised(status, &poisoned)) return;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* sA = smem;                                           // stages of A
@@ -204,16 +218,17 @@ lsq_tc_residual_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units
     }
   };
 
-  bool ok = true;
+  bool ok = true;                  // this warp's waits so far
+  int committed = -1;              // last tile whose MMAs were committed (the same in every thread)
   for (int t = 0; t < kResStages - 1; ++t) issue_loads(t);
   constexpr uint32_t idesc = instr_desc_bf16(kTcBatch, kUnitNodes, 0, 0);
   float4 xcur[2], xnext[2];
   load_x(0, xcur);
-  for (int t = 0; t < ntiles && ok; ++t) {
+  for (int t = 0; t < ntiles; ++t) {
     const int st = t % kResStages, buf = t & 1;
     load_x(t + 1, xnext);                                   // consumed one iteration later
     cp_async_wait<kResStages - 2>();                        // this thread's copies of tile t have landed
-    if (t >= 2) ok = mbar_wait(smem_u32(&bars[buf]), ((t >> 1) - 1) & 1);   // operand buffer free again
+    if (t >= 2) ok = mbar_wait(smem_u32(&bars[buf]), ((t >> 1) - 1) & 1, spin_limit) && ok;   // operand buffer free again
     // fp32 -> bf16 hi/lo into the swizzled operand layout
     {
       const int r = xr, c8 = xc8;                           // c8: group of 8 coordinates = one 16-byte bf16 chunk
@@ -233,8 +248,9 @@ lsq_tc_residual_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units
     }
     fence_proxy_async();                                    // generic-proxy writes (cp.async, st.shared) -> MMA reads
     tc_fence_before();
-    __syncthreads();
-    if (tid == 0 && ok) {
+    ok = __syncthreads_and(ok);                             // the loop's one barrier also makes the give-up decision CTA-uniform
+    if (!ok) break;
+    if (tid == 0) {
       tc_fence_after();
       const uint32_t a_base = smem_u32(sA + st * kResABytes);
       const uint32_t h_base = smem_u32(sXop + (buf * 2 + 0) * kResXopBytes);
@@ -251,16 +267,24 @@ lsq_tc_residual_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units
         }
       tc_commit(smem_u32(&bars[buf]));
     }
-    // refill the stage that tile t-1 used (its MMAs were committed one iteration ago)
-    if (t >= 1 && ok) ok = mbar_wait(smem_u32(&bars[(t - 1) & 1]), ((t - 1) >> 1) & 1);
-    issue_loads(t + kResStages - 1);
+    committed = t;
+    // refill the stage that tile t-1 used (its MMAs were committed one iteration ago); a warp whose wait
+    // expired leaves that stage alone and reports at the next barrier
+    if (t >= 1) ok = mbar_wait(smem_u32(&bars[(t - 1) & 1]), ((t - 1) >> 1) & 1, spin_limit);
+    if (ok) issue_loads(t + kResStages - 1); else cp_async_commit();
     xcur[0] = xnext[0]; xcur[1] = xnext[1];
   }
   cp_async_wait<0>();
-  if (ok && ntiles > 0) ok = mbar_wait(smem_u32(&bars[(ntiles - 1) & 1]), ((ntiles - 1) >> 1) & 1);
-  if (ok && ntiles > 1) ok = mbar_wait(smem_u32(&bars[(ntiles - 2) & 1]), ((ntiles - 2) >> 1) & 1);
+  if (ok && committed >= 0) ok = mbar_wait(smem_u32(&bars[committed & 1]), (committed >> 1) & 1, spin_limit);
+  if (ok && committed >= 1) ok = mbar_wait(smem_u32(&bars[(committed - 1) & 1]), ((committed - 1) >> 1) & 1, spin_limit);
+  ok = __syncthreads_and(ok);
+  if (!ok) {
+    if (tid == 0) atomicExch(status, 1);
+    // gave up: the last commit covers every MMA issued before it; wait for it with the full default bound
+    // so that tensor memory is not released under an MMA
+    if (committed >= 0) mbar_wait(smem_u32(&bars[committed & 1]), (committed >> 1) & 1, kSpinLimit);
+  }
   tc_fence_after();
-  if (!ok && tid == 0) atomicExch(status, 1);
   // accumulator rows 16q..16q+15 live in lanes 32q..32q+15: warps 0..3, lanes 0..15
   if (warp < 4) {
     float v[16];
@@ -285,7 +309,8 @@ lsq_tc_residual_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units
 // =================================================================================================
 __global__ void __launch_bounds__(kTcBatch * kUnitNodes)
 lsq_tc_finalize_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, int step, const float* __restrict__ partial,
-                       int64_t nchunks, __nv_bfloat16* __restrict__ resid) {
+                       int64_t nchunks, __nv_bfloat16* __restrict__ resid, const int* __restrict__ status) {
+  if (*reinterpret_cast<const volatile int*>(status) != 0) return;    // the partials of a step that gave up are not complete
   const LsqUnit u = units[blockIdx.x];
   const int sidx = threadIdx.x / kUnitNodes, j = threadIdx.x % kUnitNodes;
   const float* p = partial + (int64_t)blockIdx.x * nchunks * (kTcBatch * kUnitNodes) + threadIdx.x;
@@ -319,7 +344,10 @@ constexpr int kUpdSmem = kUpdStages * kUpdABytes + 2 * kUpdRBytes + 1024 + 64;
 
 __global__ void __launch_bounds__(kTcThreads, 3)
 lsq_tc_update_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, int step, float lr,
-                     const __nv_bfloat16* __restrict__ resid, int64_t chunk_coords, int* __restrict__ status) {
+                     const __nv_bfloat16* __restrict__ resid, int64_t chunk_coords, int* __restrict__ status,
+                     uint32_t spin_limit) {
+  __shared__ int poisoned;
+  if (status_raised(status, &poisoned)) return;               // no model is touched after a step gave up
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* sA = smem;
@@ -399,17 +427,19 @@ lsq_tc_update_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
       xin[q] = (tile < ntiles && jbase + q < u.count) ? s.X[(int64_t)unodes[jbase + q] * s.pitch + k] : 0.0f;
   };
 
-  bool ok = true;
+  bool ok = true;                  // this warp's waits so far
+  int committed = -1;              // last tile whose MMAs were committed (the same in every thread)
   for (int t = 0; t < kUpdStages - 1; ++t) issue_loads(t);
   constexpr uint32_t idesc = instr_desc_bf16(kUpdTile, kUnitNodes, 1, 0);
   float xprev[8], xcur[8];
-  for (int t = 0; t < ntiles && ok; ++t) {
+  for (int t = 0; t < ntiles; ++t) {
     const int st = t % kUpdStages, buf = t & 1;
     load_x(t, xcur);                                        // consumed one iteration later
     cp_async_wait<kUpdStages - 2>();
     fence_proxy_async();
     tc_fence_before();
-    __syncthreads();                                        // tile t landed; epilogue of tile t-2 has drained buffer `buf`
+    ok = __syncthreads_and(ok);                             // tile t landed; epilogue of tile t-2 has drained buffer `buf`;
+    if (!ok) break;                                         // and the give-up decision is CTA-uniform
     if (tid == 0) {
       tc_fence_after();
       const uint32_t a_base = smem_u32(sA + st * kUpdABytes);
@@ -424,23 +454,31 @@ lsq_tc_update_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
       }
       tc_commit(smem_u32(&bars[buf]));
     }
+    committed = t;
     if (t >= 1) {
-      ok = mbar_wait(smem_u32(&bars[(t - 1) & 1]), ((t - 1) >> 1) & 1);
+      ok = mbar_wait(smem_u32(&bars[(t - 1) & 1]), ((t - 1) >> 1) & 1, spin_limit);
       tc_fence_after();
       if (ok) epilogue(t - 1, xprev);
       tc_fence_before();
     }
 #pragma unroll
     for (int q = 0; q < 8; ++q) xprev[q] = xcur[q];
-    issue_loads(t + kUpdStages - 1);                        // stage of tile t-1: its MMAs have completed
+    if (ok) issue_loads(t + kUpdStages - 1);                // stage of tile t-1: its MMAs have completed
+    else cp_async_commit();
   }
   cp_async_wait<0>();
-  if (ok && ntiles > 0) {
-    ok = mbar_wait(smem_u32(&bars[(ntiles - 1) & 1]), ((ntiles - 1) >> 1) & 1);
+  if (ok && committed >= 0) {
+    ok = mbar_wait(smem_u32(&bars[committed & 1]), (committed >> 1) & 1, spin_limit);
     tc_fence_after();
-    if (ok) epilogue(ntiles - 1, xprev);
+    if (ok) epilogue(committed, xprev);
   }
-  if (!ok && tid == 0) atomicExch(status, 1);
+  ok = __syncthreads_and(ok);
+  if (!ok) {
+    if (tid == 0) atomicExch(status, 1);
+    // gave up: wait for the last commit (it covers every MMA issued before it) with the full default bound,
+    // so that tensor memory is not released under an MMA
+    if (committed >= 0) mbar_wait(smem_u32(&bars[committed & 1]), (committed >> 1) & 1, kSpinLimit);
+  }
   tc_fence_before();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem_d, 32);
@@ -460,12 +498,16 @@ int64_t lsq_tc_chunks(int64_t pitch) {
 size_t lsq_tc_partial_bytes(int64_t pitch, int units) { return (size_t)units * lsq_tc_chunks(pitch) * kTcBatch * kUnitNodes * 4; }
 size_t lsq_tc_resid_bytes(int units) { return (size_t)units * 2 * kUnitNodes * kTcBatch * 2; }
 
+uint32_t lsq_tc_default_wait_limit() { return kSpinLimit; }
+
 cudaError_t launch_local_lsq_tc(const StoreView& s, const LsqView& l, const LsqUnit* units_dev, int nunits, int H,
-                                float lr, float* partial_dev, void* resid_dev, int* status_dev, cudaStream_t st,
-                                int* launches) {
+                                float lr, float* partial_dev, void* resid_dev, int* status_dev, uint32_t wait_limit,
+                                cudaStream_t st, int* launches) {
   if (nunits == 0 || H == 0) return cudaSuccess;
   if (l.batch > kTcBatch || l.dtype != 1) return cudaErrorInvalidValue;
   static bool attr_set[64] = {};
+  static std::mutex attr_mutex;                   // contexts on different threads may reach this together
+  std::lock_guard<std::mutex> lock(attr_mutex);
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev >= 0 && dev < 64 && !attr_set[dev]) {
@@ -478,11 +520,13 @@ cudaError_t launch_local_lsq_tc(const StoreView& s, const LsqView& l, const LsqU
   const int64_t chunk = lsq_tc_chunk_coords(s.pitch), nchunks = lsq_tc_chunks(s.pitch);
   const dim3 grid((unsigned)nchunks, nunits);
   for (int q = 0; q < H; ++q) {
-    lsq_tc_residual_kernel<<<grid, kTcThreads, kResSmem, st>>>(s, l, units_dev, q, partial_dev, chunk, nchunks, status_dev);
+    lsq_tc_residual_kernel<<<grid, kTcThreads, kResSmem, st>>>(s, l, units_dev, q, partial_dev, chunk, nchunks, status_dev,
+                                                               wait_limit);
     lsq_tc_finalize_kernel<<<nunits, kTcBatch * kUnitNodes, 0, st>>>(s, l, units_dev, q, partial_dev, nchunks,
-                                                                     reinterpret_cast<__nv_bfloat16*>(resid_dev));
+                                                                     reinterpret_cast<__nv_bfloat16*>(resid_dev), status_dev);
     lsq_tc_update_kernel<<<grid, kTcThreads, kUpdSmem, st>>>(s, l, units_dev, q, lr,
-                                                             reinterpret_cast<const __nv_bfloat16*>(resid_dev), chunk, status_dev);
+                                                             reinterpret_cast<const __nv_bfloat16*>(resid_dev), chunk, status_dev,
+                                                             wait_limit);
     *launches += 3;
   }
   return cudaGetLastError();

@@ -38,14 +38,15 @@ std::mutex g_setup_mutex;
 
 // Same arithmetic as the context-based kernel: per column the first row is the shift (exact in double),
 // Gamma_col = sum s^2 - (sum s)^2 / n with s = x_i - x_0; columns past d are skipped.
+// `vec` (decided on the host): every row starts on a 16-byte boundary, so four columns travel as one 128-bit load.
 __global__ void __launch_bounds__(kThreads)
-static_potential_partial_kernel(const float* __restrict__ x, int n, int64_t d, int64_t pitch,
+static_potential_partial_kernel(const float* __restrict__ x, int n, int64_t d, int64_t pitch, int vec,
                                 double* __restrict__ partial) {
   const int64_t c4 = (int64_t)blockIdx.x * kThreads + threadIdx.x;
   double gamma = 0.0;
   if (c4 * 4 < d) {
     const float* col = x + c4 * 4;
-    const bool whole = c4 * 4 + 3 < d && (pitch & 3) == 0;   // vector path needs 16-byte aligned rows
+    const bool whole = vec != 0 && c4 * 4 + 3 < d;
     double b[4], sm[4] = {0.0, 0.0, 0.0, 0.0}, sq[4] = {0.0, 0.0, 0.0, 0.0};
     auto load = [&](int64_t row, float v[4]) {
       const float* p = col + row * pitch;
@@ -120,6 +121,7 @@ static_potential_final_kernel(const double* __restrict__ partial, int64_t count,
 extern "C" int swarm_potential_static(const float* x_dev, int32_t n, int64_t d, int64_t pitch,
                                       double* out_gamma_dev, void* cuda_stream) {
   if (!x_dev || !out_gamma_dev || n < 2 || d < 1 || pitch < d) return SWARM_EINVAL;
+  if (((uintptr_t)x_dev & 3) != 0 || ((uintptr_t)out_gamma_dev & 7) != 0) return SWARM_EINVAL;   // not a float / double address
   if (d > SWARM_STATIC_MAX_D) return SWARM_EINVAL;      // beyond the capacity of the fixed scratch array
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return SWARM_ECUDA;
@@ -138,7 +140,10 @@ extern "C" int swarm_potential_static(const float* x_dev, int32_t n, int64_t d, 
   }
   const int64_t parts = ((d + 3) / 4 + kThreads - 1) / kThreads;      // <= kMaxPartials by the check above
   cudaStream_t st = (cudaStream_t)cuda_stream;
-  static_potential_partial_kernel<<<(unsigned)parts, kThreads, 0, st>>>(x_dev, n, d, pitch, partial);
+  // 128-bit loads only when every row starts on a 16-byte boundary: base address and row pitch both count
+  // (a view into a larger tensor can have an aligned pitch and a base that is off by one float)
+  const int vec = (((uintptr_t)x_dev & 15) == 0 && (pitch & 3) == 0) ? 1 : 0;
+  static_potential_partial_kernel<<<(unsigned)parts, kThreads, 0, st>>>(x_dev, n, d, pitch, vec, partial);
   static_potential_final_kernel<<<1, 1024, 0, st>>>(partial, parts, out_gamma_dev);
   return cudaGetLastError() == cudaSuccess ? SWARM_OK : SWARM_ECUDA;
 }

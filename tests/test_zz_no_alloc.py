@@ -53,3 +53,27 @@ def test_static_potential_on_a_plain_tensor_and_size_limit():
     assert g.potential_static(x.data_ptr(), n, d, d - 1, out.data_ptr(), None) == -1
     torch.cuda.synchronize()
     assert float(out.item()) == -5.0
+
+
+@pytest.mark.parametrize("offset,d,pitch", [(1, 1000, 1004), (2, 4099, 4100), (3, 17, 20), (4, 1000, 1004), (1, 1000, 1001)])
+def test_static_potential_on_a_view_that_starts_off_a_16_byte_boundary(offset, d, pitch):
+    """A slice of a larger tensor: the pitch may be a multiple of four floats while the first row starts one,
+    two or three floats past a 16-byte boundary. Such rows are read element by element; offset 4 is aligned
+    again and takes the 128-bit loads."""
+    import torch
+    torch.manual_seed(offset)
+    n = 7
+    store = (torch.randn(n * pitch + 8, device="cuda") * 2 - 30).contiguous()
+    assert store.data_ptr() % 16 == 0
+    view = store[offset: offset + n * pitch].view(n, pitch)[:, :d]
+    out = torch.zeros(1, dtype=torch.float64, device="cuda")
+    for _ in range(2):
+        assert g.potential_static(store.data_ptr() + 4 * offset, n, d, pitch, out.data_ptr(),
+                                  torch.cuda.current_stream()) == 0
+        torch.cuda.synchronize()
+        xd = view.double()
+        want = float(((xd - xd.mean(0)) ** 2).sum().item())
+        assert abs(float(out.item()) - want) <= 1e-9 * want
+    # addresses that cannot be a float or a double are refused before anything is launched
+    assert g.potential_static(store.data_ptr() + 2, n, d, pitch, out.data_ptr(), None) == -1
+    assert g.potential_static(store.data_ptr(), n, d, pitch, out.data_ptr() + 4, None) == -1
