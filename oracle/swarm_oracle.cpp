@@ -610,8 +610,10 @@ void interact_nonblocking(Swarm& s, int a, int b, int bits) {
 // the writer's own register and a reader consumes only a prefix sized by its distance. The b-bit colour
 // of a lattice point is the low b bits of its 16-bit colour, so the prefix is the low-order part; the
 // register stores the low bytes of a block before the high bytes, and a reader that trusts its key to be
-// within 127 steps reads the first half only (own_prefix = 8). A node decoding its own register (key =
-// the very snapshot that was encoded, less than one step away) always uses the 8-bit prefix.
+// within 127 steps reads the first half only (prefix = 8). The prefix is the reader's: every interaction
+// states how many bits of its responder's own register its initiator consumes (own_prefix is the default for
+// launches that state none). A node decoding its own register (key = the very snapshot that was encoded,
+// less than one step away) always uses the 8-bit prefix.
 // ---------------------------------------------------------------------------
 constexpr int kOwnBits = 16;
 constexpr int kOwnResolutionBits = 8;
@@ -679,7 +681,7 @@ void register_publish(Swarm& s, int bits) {
   s.p_mode = 2;
 }
 
-void interact_registers(Swarm& s, int a, int b, int bits) {
+void interact_registers(Swarm& s, int a, int b, int bits, int pfx) {
   const int64_t d = s.d;
   float* xa = s.x(a); float* ba = s.base(a);
   const size_t block_bytes = (size_t)kBlock * bits / 8;
@@ -689,7 +691,6 @@ void interact_registers(Swarm& s, int a, int b, int bits) {
     const int len = (int)std::min<int64_t>(kBlock, d - k0);
     const uint8_t* ca = s.code_row(a) + blk * block_bytes;
     const uint8_t* cb = s.code_row(b) + blk * block_bytes;
-    const int pfx = s.own_prefix;
     const uint32_t pmask = (1u << pfx) - 1u;
     const int eoa = s.oexps[(int64_t)a * s.nblk + blk], eob = s.oexps[(int64_t)b * s.nblk + blk];
     const int epa = s.exp_row(a)[blk], epb = s.exp_row(b)[blk];
@@ -900,9 +901,16 @@ int orc_local_steps_geometric(void* h, const int32_t* nodes, int32_t count, int3
 
 // pairs: npairs x (initiator, responder). threads > 1 splits the (disjoint, hence
 // independent) pairs over plain std::thread workers.
-int orc_interact(void* h, const int32_t* pairs, int32_t npairs, int32_t bits, int32_t mode, int32_t threads) {
+// prefixes (may be null: the context's default for every pair): per pair the number of bits, 8 or 16, of the
+// responder's own register that the initiator reads (two-register mode only).
+int orc_interact_prefixed(void* h, const int32_t* pairs, const int32_t* prefixes, int32_t npairs, int32_t bits,
+                          int32_t mode, int32_t threads) {
   Swarm& s = *(Swarm*)h;
   if (npairs < 0 || mode < 0 || mode > 2) return -1;
+  if (prefixes) {
+    if (mode != 2) return -1;
+    for (int p = 0; p < npairs; ++p) if (prefixes[p] != 8 && prefixes[p] != 16) return -1;
+  }
   if (!((bits >= 2 && bits <= 8) || (bits == 32 && mode == 0))) return -1;
   if (mode == 1 && !s.cfg.nonblocking) return -4;
   if (mode == 2 && s.cfg.nonblocking != 2) return -4;
@@ -914,7 +922,7 @@ int orc_interact(void* h, const int32_t* pairs, int32_t npairs, int32_t bits, in
   auto run = [&](int p) {
     if (mode == 0) interact_blocking(s, pairs[2 * p], pairs[2 * p + 1], bits);
     else if (mode == 1) interact_nonblocking(s, pairs[2 * p], pairs[2 * p + 1], bits);
-    else interact_registers(s, pairs[2 * p], pairs[2 * p + 1], bits);
+    else interact_registers(s, pairs[2 * p], pairs[2 * p + 1], bits, prefixes ? prefixes[p] : s.own_prefix);
   };
   if (threads <= 1 || npairs <= 1) {
     for (int p = 0; p < npairs; ++p) run(p);
@@ -943,6 +951,10 @@ int orc_interact(void* h, const int32_t* pairs, int32_t npairs, int32_t bits, in
     for (int p = 0; p < npairs; ++p) record_initiation(s, pairs[2 * p], mu.data());
   }
   return 0;
+}
+
+int orc_interact(void* h, const int32_t* pairs, int32_t npairs, int32_t bits, int32_t mode, int32_t threads) {
+  return orc_interact_prefixed(h, pairs, nullptr, npairs, bits, mode, threads);
 }
 
 // Start (or stop) tracking the auxiliary potentials: every node counts as having initiated just now.

@@ -62,6 +62,7 @@ def lib():
         "orc_local_steps": (C.c_int, [vp, i32p, C.c_int32, C.c_int32, C.c_float]),
         "orc_local_steps_geometric": (C.c_int, [vp, i32p, C.c_int32, C.c_int32, C.c_float, i32p]),
         "orc_interact": (C.c_int, [vp, i32p, C.c_int32, C.c_int32, C.c_int32, C.c_int32]),
+        "orc_interact_prefixed": (C.c_int, [vp, i32p, i32p, C.c_int32, C.c_int32, C.c_int32, C.c_int32]),
         "orc_publish": (C.c_int, [vp, C.c_int32]),
         "orc_register_publish": (C.c_int, [vp, C.c_int32]),
         "orc_own": (u8p, [vp]), "orc_set_own_prefix": (C.c_int, [vp, C.c_int32]), "orc_get_own_prefix": (C.c_int32, [vp]), "orc_oexps": (i8p, [vp]), "orc_wo": (u32p, [vp]), "orc_tau": (u32p, [vp]),
@@ -337,6 +338,17 @@ class OracleSwarm:
         pairs = np.ascontiguousarray(pairs, dtype=np.int32).reshape(-1, 2)
         return int(lib().orc_interact(self._h, pairs.ctypes.data_as(C.POINTER(C.c_int32)), len(pairs), bits, mode,
                                       threads))
+
+    def interact_prefixed(self, pairs, prefixes, bits, threads=1):
+        """Two-register interactions in which the initiator of pairs[p] reads prefixes[p] (8 or 16) bits of its
+        responder's own register."""
+        pairs = np.ascontiguousarray(pairs, dtype=np.int32).reshape(-1, 2)
+        prefixes = np.ascontiguousarray(prefixes, dtype=np.int32)
+        if len(prefixes) != len(pairs):
+            raise ValueError("one prefix per pair")
+        return int(lib().orc_interact_prefixed(self._h, pairs.ctypes.data_as(C.POINTER(C.c_int32)),
+                                               prefixes.ctypes.data_as(C.POINTER(C.c_int32)), len(pairs), bits,
+                                               REGISTERS, threads))
 
     def publish(self, bits):
         return int(lib().orc_publish(self._h, bits))

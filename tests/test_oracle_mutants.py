@@ -57,6 +57,8 @@ MUTANTS = [
     ("register_update_sign", "const float nx = av - D;\n      avg[k] = av; new_x[k] = nx;\n      spread = std::max(spread, std::fabs(Qa - Qb));",
      "const float nx = av + D;\n      avg[k] = av; new_x[k] = nx;\n      spread = std::max(spread, std::fabs(Qa - Qb));",
      ["test_oracle_registers.py"]),
+    ("every_reader_gets_the_first_readers_prefix", "bits, prefixes ? prefixes[p] : s.own_prefix);",
+     "bits, prefixes ? prefixes[0] : s.own_prefix);", ["test_oracle_registers.py"]),
     ("clock_of_the_initiator_not_reset", "s.tau[pairs[2 * p]] = 0;", "s.tau[pairs[2 * p + 1]] = 0;",
      ["test_oracle_registers.py", "test_oracle_graph.py", "test_oracle_staleness.py"]),
     ("lsq_gradient_not_averaged_over_the_batch", "g /= (double)bsz;", "", ["test_oracle_local_steps.py"]),

@@ -214,3 +214,75 @@ def test_own_prefix_argument_checks():
     plain = o.OracleSwarm(4, 16, "complete")
     plain.configure(objective=1, nonblocking=1)
     assert plain.set_own_prefix(8) == -4
+
+
+# ---- the prefix is the reader's: each interaction of a launch states its own (Corollary 1, second case;
+# ---- "Counting Communication Cost": a reader uses the first bits in proportion to its distance) ----
+
+def decode_own_prefix(s, reader, owner, prefix):
+    mask = (1 << prefix) - 1
+    return np.array([o.dec(float(s.B[reader, k]), int(s.own[owner, k]) & mask, int(s.oexps[owner, k // 1024]), prefix)
+                     for k in range(s.d)], dtype=np.float32)
+
+
+def near_and_far_readers():
+    """Nodes 0, 1 and 3, 4 are close pairs that have just met (fine own registers); node 2 sits 0.05 away from
+    all of them: hundreds of own-register steps, far outside an 8-bit window, well inside the 16-bit one."""
+    s = make(n=5, d=1500, seed=4, offset_std=0.0, drift_std=0.0, grad_std=0.0, init_std=0.001)
+    s.X[2] += np.float32(0.05)
+    s.B[:] = s.X
+    s.register_publish(8)
+    assert s.interact([[0, 1], [3, 4]], 8, o.REGISTERS) == 0
+    dist_steps = np.abs(s.B[2].astype(np.float64) - s.B[0]) / steps(s.oexps[0], s.d)
+    assert dist_steps.min() > 200 and dist_steps.max() < 30000
+    near_steps = np.abs(s.B[4].astype(np.float64) - s.B[3]) / steps(s.oexps[3], s.d)
+    assert near_steps.max() < 100
+    return s
+
+
+def test_a_launch_mixes_readers_with_different_prefixes():
+    launch = [[2, 0], [4, 3]]                          # a far reader and a near reader
+    ref, default = near_and_far_readers(), near_and_far_readers()
+    assert ref.interact_prefixed(launch, [16, 16], 8) == 0
+    assert default.interact(launch, 8, o.REGISTERS) == 0             # the context's default prefix is 16
+    for name in ("X", "B", "own_bytes", "codes", "exps", "oexps", "w", "wo", "tau"):
+        assert np.array_equal(getattr(ref, name), getattr(default, name)), name
+    # the near reader needs 8 bits only: same launch, same result, half of its partner's register read
+    mixed = near_and_far_readers()
+    assert mixed.interact_prefixed(launch, [16, 8], 8) == 0
+    for name in ("X", "B", "own_bytes", "codes", "exps", "oexps", "w", "wo", "tau"):
+        assert np.array_equal(getattr(ref, name), getattr(mixed, name)), name
+    # the other way round the far reader aliases; the near reader's interaction is not affected by it
+    wrong = near_and_far_readers()
+    before = near_and_far_readers()
+    short, full = decode_own_prefix(before, 2, 0, 8), decode_own_prefix(before, 2, 0, 16)
+    st = steps(before.oexps[0], before.d)
+    q = np.round(full.astype(np.float64) / st)
+    cell = np.floor(before.B[2].astype(np.float64) / st)
+    inside = (q - cell >= -127) & (q - cell <= 128)                  # the 8-bit window around the reader's cell
+    assert not inside.any()
+    assert np.array_equal(short == full, inside)
+    off = (short.astype(np.float64) - full) / st
+    assert np.all(off % 256 == 0) and np.all(off != 0)
+    assert wrong.interact_prefixed(launch, [8, 16], 8) == 0
+    for i in (3, 4, 0, 1):
+        assert np.array_equal(wrong.X[i], ref.X[i]) and np.array_equal(wrong.B[i], ref.B[i])
+    assert np.array_equal(wrong.own_bytes[4], ref.own_bytes[4]) and np.array_equal(wrong.codes[3], ref.codes[3])
+    # node 2's update restated from unit decodes with the short prefix
+    Qa = decode_current(before, decode_own_prefix(before, 2, 2, 8), 2, 8)
+    Qb = decode_current(before, short, 0, 8)
+    assert np.array_equal(wrong.X[2], np.float32(0.5) * (Qa + Qb) - (before.B[2] - before.X[2]))
+    assert np.abs(wrong.X[2].astype(np.float64) - ref.X[2]).max() > 0.005
+
+
+def test_context_default_prefix_is_the_prefix_of_every_pair():
+    launch = [[1, 0], [4, 3]]
+    a, b = near_and_far_readers(), near_and_far_readers()
+    assert a.set_own_prefix(8) == 0
+    assert a.interact(launch, 8, o.REGISTERS) == 0
+    assert b.interact_prefixed(launch, [8, 8], 8) == 0 and b.own_prefix == 16
+    for name in ("X", "B", "own_bytes", "codes", "exps", "oexps"):
+        assert np.array_equal(getattr(a, name), getattr(b, name)), name
+    assert b.interact_prefixed(launch, [8, 12], 8) == -1
+    with pytest.raises(ValueError):
+        b.interact_prefixed(launch, [8], 8)
