@@ -435,11 +435,11 @@ void local_step_synth(Swarm& s, int i, float lr) {
   }
 }
 
-void local_step_lsq(Swarm& s, int i, float lr) {
-  const int m = s.cfg.lsq_m, bsz = s.cfg.lsq_batch;
+// One minibatch step of node i on the given rows of its data matrix (Section 3, "The Communication
+// Procedure": x <- x - lr * g~(x), g~ the gradient of the minibatch objective at the running iterate).
+void lsq_step_on_rows(Swarm& s, int i, const int32_t* rows, int bsz, float lr) {
+  const int m = s.cfg.lsq_m;
   const int64_t d = s.d;
-  std::vector<int32_t> rows(bsz);
-  minibatch_rows(s, i, s.ls[i], rows.data());
   const float* Ag = s.A.data() + (size_t)s.group_of(i) * m * d;
   float* xi = s.x(i);
   std::vector<double> resid(bsz);
@@ -458,6 +458,12 @@ void local_step_lsq(Swarm& s, int i, float lr) {
     g /= (double)bsz;
     xi[k] = (float)((double)xi[k] - (double)lr * g);
   }
+}
+
+void local_step_lsq(Swarm& s, int i, float lr) {
+  std::vector<int32_t> rows(s.cfg.lsq_batch);
+  minibatch_rows(s, i, s.ls[i], rows.data());
+  lsq_step_on_rows(s, i, rows.data(), s.cfg.lsq_batch, lr);
 }
 
 // Number of local steps of a node as a geometric random variable of mean H (Section 3, "Sequential
@@ -874,6 +880,18 @@ int orc_local_steps(void* h, const int32_t* nodes, int32_t count, int32_t H, flo
       s.ls[i] += 1;
     }
   }
+  return 0;
+}
+
+// One least-squares (or logistic) step of `node` on an explicit list of rows of its data matrix instead of
+// the rows its counter would draw; the step counter advances as for a drawn minibatch. For checks of a
+// single step of a large swarm on a small copy of the rows it touched.
+int orc_local_step_on_rows(void* h, int32_t node, const int32_t* rows, int32_t count, float lr) {
+  Swarm& s = *(Swarm*)h;
+  if (s.cfg.objective < 2 || node < 0 || node >= s.n || count < 1) return -1;
+  for (int t = 0; t < count; ++t) if (rows[t] < 0 || rows[t] >= s.cfg.lsq_m) return -2;
+  lsq_step_on_rows(s, node, rows, count, lr);
+  s.ls[node] += 1;
   return 0;
 }
 

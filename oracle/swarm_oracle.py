@@ -60,6 +60,7 @@ def lib():
         "orc_minibatch_rows": (C.c_int, [vp, C.c_int32, C.c_uint32, i32p]),
         "orc_sample_pairs": (C.c_int, [vp, C.c_int32, i32p, i32p]),
         "orc_local_steps": (C.c_int, [vp, i32p, C.c_int32, C.c_int32, C.c_float]),
+        "orc_local_step_on_rows": (C.c_int, [vp, C.c_int32, i32p, C.c_int32, C.c_float]),
         "orc_local_steps_geometric": (C.c_int, [vp, i32p, C.c_int32, C.c_int32, C.c_float, i32p]),
         "orc_interact": (C.c_int, [vp, i32p, C.c_int32, C.c_int32, C.c_int32, C.c_int32]),
         "orc_interact_prefixed": (C.c_int, [vp, i32p, i32p, C.c_int32, C.c_int32, C.c_int32, C.c_int32]),
@@ -325,6 +326,11 @@ class OracleSwarm:
     def local_steps(self, nodes, H, lr):
         nodes = np.ascontiguousarray(nodes, dtype=np.int32)
         return int(lib().orc_local_steps(self._h, nodes.ctypes.data_as(C.POINTER(C.c_int32)), len(nodes), H, lr))
+
+    def local_step_on_rows(self, node, rows, lr):
+        """One least-squares step of `node` on the listed rows of its data matrix (its counter advances by one)."""
+        rows = np.ascontiguousarray(rows, dtype=np.int32)
+        return int(lib().orc_local_step_on_rows(self._h, node, rows.ctypes.data_as(C.POINTER(C.c_int32)), len(rows), lr))
 
     def local_steps_geometric(self, nodes, mean_h, lr):
         """Returns (rc, steps taken per listed node)."""

@@ -157,6 +157,12 @@ def test_geometric_step_counts_have_the_stated_moments():
         var = H * H - H                                  # variance of the geometric law
         assert abs(draws.mean() - H) < 5 * np.sqrt(var / N)
         assert abs((draws**2).mean() - (2 * H * H - H)) < 0.08 * (2 * H * H - H)
+        # appendix lemmas on the step count: sum_K Pr[H_i = K] K^3 <= 6 H^3 and sum_K Pr[H_i = K] K^4 <= 24 H^4.
+        # Closed forms of the geometric law with success probability 1/H: E[K^3] = 6H^3 - 6H^2 + H and
+        # E[K^4] = 24H^4 - 36H^3 + 14H^2 - H; the sample moments must sit at those and under the bounds
+        m3, m4 = 6 * H**3 - 6 * H**2 + H, 24 * H**4 - 36 * H**3 + 14 * H**2 - H
+        assert abs((draws**3).mean() - m3) < 0.15 * m3 and (draws**3).mean() <= 6 * H**3
+        assert abs((draws**4).mean() - m4) < 0.30 * m4 and (draws**4).mean() <= 24 * H**4
         assert abs((draws == 1).mean() - 1 / H) < 5 * np.sqrt((1 / H) * (1 - 1 / H) / N)
         assert abs((draws == 2).mean() - (1 - 1 / H) / H) < 5 * np.sqrt(0.25 / N)
 
@@ -224,3 +230,25 @@ def test_logistic_sgd_reduces_the_loss():
     assert loss(s.X[1].astype(np.float64)) < 0.6 * l0
     pred = (A @ s.X[1].astype(np.float64)) > 0
     assert (pred == (y > 0.5)).mean() > 0.85
+
+
+def test_step_on_explicit_rows_is_the_step_the_counter_would_draw():
+    """local_step_on_rows with the rows of minibatch_rows is local_steps; with one explicit row it is the
+    by-hand update x' = x - lr (<a, x> - b) a; the counter advances either way."""
+    s1, s2 = lsq(n=3, d=40, m=12, batch=5, noise=0.2, seed=6), lsq(n=3, d=40, m=12, batch=5, noise=0.2, seed=6)
+    for step in range(3):
+        rows = s1.minibatch_rows(2, step)
+        assert s1.local_steps([2], 1, 0.1) == 0
+        assert s2.local_step_on_rows(2, rows, 0.1) == 0
+    assert np.array_equal(s1.X, s2.X) and s1.ls.tolist() == s2.ls.tolist() == [0, 0, 3]
+    x0 = s2.X[1].astype(np.float64).copy()
+    a = s2.A[1, 7].astype(np.float64)
+    assert s2.local_step_on_rows(1, [7], 0.25) == 0
+    assert np.array_equal(s2.X[1], (x0 - 0.25 * (a @ x0 - float(s2.bvec[1, 7])) * a).astype(np.float32))
+    # two explicit rows: the mean of the two single-row gradients
+    x0 = s2.X[0].astype(np.float64).copy()
+    A = s2.A[0].astype(np.float64)
+    g = 0.5 * sum((A[r] @ x0 - float(s2.bvec[0, r])) * A[r] for r in (3, 3))   # a row may repeat (drawn with replacement)
+    assert s2.local_step_on_rows(0, [3, 3], 0.5) == 0
+    assert np.array_equal(s2.X[0], (x0 - 0.5 * g).astype(np.float32))
+    assert s2.local_step_on_rows(0, [12], 0.1) == -2 and s2.local_step_on_rows(3, [0], 0.1) == -1
