@@ -61,6 +61,13 @@ WORKLOADS = {
     "regular8_resnet18_b8_reg": dict(n=8, d=11_689_512, topology="regular", degree=4, pairs=4, bits=8, mode=2, H=3,
                                      lr=0.05, seed=3, cfg=dict(objective=1, nonblocking=2,
                                                                grad_std=float(np.sqrt(1e-3)))),
+    # ring of 64 nodes through the two-register protocol: every reader consumes all 16 bits of its partner's own
+    # register (the default), or only the 8-bit prefix (ring neighbours keep meeting, so their snapshots stay within
+    # the 8-bit window of each other's own registers): bytes moved per interaction 22 d + 2 d bits/8 against 21 d + ...
+    "ring64_d1m_b8_reg": dict(n=64, d=1 << 20, topology="ring", degree=0, pairs=32, bits=8, mode=2, H=2, lr=0.05, seed=2,
+                              cfg=dict(objective=1, nonblocking=2, grad_std=float(np.sqrt(1e-3)))),
+    "ring64_d1m_b8_reg_p8": dict(n=64, d=1 << 20, topology="ring", degree=0, pairs=32, bits=8, mode=2, H=2, lr=0.05,
+                                 seed=2, prefix=8, cfg=dict(objective=1, nonblocking=2, grad_std=float(np.sqrt(1e-3)))),
     # reduced copy (8 nodes, 4 pairs) for profiler captures that must stay small
     "regular8_resnet18_b8_nb": dict(n=8, d=11_689_512, topology="regular", degree=4, pairs=4, bits=8, mode=1, H=3,
                                     lr=0.05, seed=3, cfg=dict(objective=1, nonblocking=1,
@@ -93,7 +100,7 @@ def stepping_nodes(wl, pairs):
     return pairs.reshape(-1)
 
 
-def interaction_bytes(d, bits, mode):
+def interaction_bytes(d, bits, mode, prefix=16):
     """Algorithmic bytes one interaction must move: blocking reads two models, writes two models and
     two packed buffers; non-blocking reads model + snapshot + two buffers and writes the same."""
     nblk = (d + 1023) // 1024
@@ -104,9 +111,8 @@ def interaction_bytes(d, bits, mode):
     if mode == 1:
         return d * 16 + 4 * d * bits // 8 + 4 * nblk
     # two registers: model + snapshot read and written; own registers: the 8-bit prefix of the initiator's,
-    # the 16 bits of the responder's (default prefix) read, the initiator's 16 bits written; two current
-    # registers read and written
-    return d * 16 + d * 5 + 4 * d * bits // 8 + 7 * nblk
+    # `prefix` bits of the responder's read, the initiator's 16 bits written; two current registers read and written
+    return d * 16 + d * (3 + prefix // 8) + 4 * d * bits // 8 + 7 * nblk
 
 
 class PairSchedule:
@@ -311,6 +317,252 @@ def run_reference(args, wl, name):
 # ---------------------------------------------------------------------------------------------------
 # CUDA arm
 # ---------------------------------------------------------------------------------------------------
+KERNEL_SOURCES = ("swarm_interact.cu", "swarm_blocks.cuh", "swarm_dev.cuh", "swarm_internal.h")
+# the five workloads of the measurement table: small least squares, ring averaging, ResNet-18-sized non-blocking,
+# ResNet-50-sized blocking at two code widths, 256 nodes with tensor-core least squares
+TABLE_WORKLOADS = ("complete8_d4096_b8_lsq", "ring64_d1m_b4", "regular32_resnet18_b8_nb", "complete16_resnet50_b4",
+                   "complete16_resnet50_b8", "regular256_d1m_b2_lsq_nb")
+
+
+def kernel_source_hash():
+    """sha256 over the sources that define the interaction kernels: profiler counters recorded under profiles/
+    carry the hash of the sources they were captured from and are dropped once it no longer matches."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_1910_12308_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def profiler_counters(name):
+    """Counters of the dominant kernel of workload `name` from profiles/kernel_counters.json ({} when there is no
+    capture of the kernels as they are now)."""
+    try:
+        rec = json.load(open(os.path.join(ROOT, "profiles", "kernel_counters.json")))[name]
+    except Exception:
+        return {}
+    return rec if rec.get("source_sha256_16") == kernel_source_hash() else {}
+
+
+def traffic_of(name, pairs_per_launch):
+    """ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, or None."""
+    rec = profiler_counters(name)
+    if "dram_bytes_per_launch" in rec:
+        return rec["dram_bytes_per_launch"]
+    if "dram_bytes_per_pair" in rec:       # launches whose number of pairs varies: every pair streams its own rows once
+        return rec["dram_bytes_per_pair"] * pairs_per_launch
+    return None
+
+
+def kernel_name(wl, fused=False):
+    base = ("interact_identity_kernel" if wl["bits"] == 32 else
+            ["interact_blocking_kernel", "interact_nonblocking_kernel", "interact_registers_kernel"][wl["mode"]])
+    return base + (" (local steps fused)" if fused else "")
+
+
+class Runner:
+    """One workload on the current device: context, pair schedule and the timed loop over the C ABI."""
+
+    def __init__(self, g, torch, wl, name, seed_shift, stream, args):
+        self.g, self.torch, self.wl, self.name, self.stream = g, torch, wl, name, stream
+        self.sw = g.Swarm(wl["n"], wl["d"], wl["topology"], wl["degree"], wl["seed"] + seed_shift, stream=stream)
+        if wl["cfg"]:
+            self.sw.configure(**wl["cfg"])
+        self.sched = PairSchedule(wl, self.sw.get_all(g.T_ADJ))
+        # elementwise (synthetic) objective, on request: the nodes of the pairs step inside the interaction kernel
+        self.fused = bool(wl["H"] > 0 and wl["cfg"].get("objective") == 1 and not wl.get("step_all") and args.fused)
+        # sequential gossip on short models: the whole timed region is one swarm_run_sequence call
+        self.sequence = bool(wl.get("sequence")) and wl["pairs"] == 1 and wl["mode"] == 0 and not args.stepwise
+
+    def step(self, pairs):
+        """One step through the public binding (what a user calls)."""
+        sw, wl = self.sw, self.wl
+        if self.fused:
+            rc = sw.step(pairs, wl["H"], wl["lr"], wl["bits"], wl["mode"], True)
+            assert rc == 0, rc
+            return
+        if wl["H"] > 0:
+            rc = sw.local_steps(stepping_nodes(wl, pairs), wl["H"], wl["lr"])
+            assert rc == 0, rc
+        if wl.get("prefix"):
+            rc = sw.interact_prefixed(pairs, np.full(len(pairs), wl["prefix"], dtype=np.int32), wl["bits"])
+        else:
+            rc = sw.interact(pairs, wl["bits"], wl["mode"])
+        assert rc == 0, rc
+
+    def timed(self, launches, barrier, probe_every=8):
+        """Times len(launches) steps with CUDA events on the context's stream, models resident in HBM. Arguments
+        are marshalled before the timed region; the loop only crosses the C ABI. Returns (ms for all steps,
+        average ms of the interaction kernel, kernels launched)."""
+        import ctypes as C
+        g, torch, wl, sw, stream = self.g, self.torch, self.wl, self.sw, self.stream
+        L, h = sw._L, sw._h
+        H, lr, bits, mode = wl["H"], wl["lr"], wl["bits"], wl["mode"]
+        K = len(launches)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ok, ev_mid = 0, []
+        l0 = sw.kernel_launches()
+        if self.sequence:
+            seq = np.ascontiguousarray(np.concatenate(launches), dtype=np.int32)
+            ptr = seq.ctypes.data_as(C.POINTER(g.SwarmPair))
+            ev0.record(stream)
+            ok |= L.swarm_run_sequence(h, ptr, len(seq), H, lr, bits, 1)
+            ev1.record(stream)
+        else:
+            prefixes = np.full(wl["n"], wl.get("prefix", 16), dtype=np.int32)
+            pf_ptr = prefixes.ctypes.data_as(C.POINTER(C.c_int32))
+
+            def interact(pp, npp):
+                if wl.get("prefix"):
+                    return L.swarm_interact_prefixed(h, pp, pf_ptr, npp, bits)
+                return L.swarm_interact(h, pp, npp, bits, mode)
+            calls = []
+            for pairs in launches:
+                pa = np.ascontiguousarray(pairs, dtype=np.int32)
+                na = np.ascontiguousarray(stepping_nodes(wl, pairs), dtype=np.int32)
+                calls.append((pa, pa.ctypes.data_as(C.POINTER(g.SwarmPair)), len(pa), na,
+                              na.ctypes.data_as(C.POINTER(C.c_int32)), len(na)))
+            self.calls = calls
+            probes = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                      for _ in range(0, K, probe_every)] if (H > 0 and not self.fused) else []
+            ev0.record(stream)
+            for i, (_, pp, npp, _, nn, ncount) in enumerate(calls):
+                if self.fused:
+                    ok |= L.swarm_step(h, pp, npp, H, lr, bits, mode, 1)
+                elif H > 0:
+                    ok |= L.swarm_local_steps(h, nn, ncount, H, lr)
+                    if i % probe_every == 0:       # the interaction kernel is bracketed by events on every 8th step
+                        e_a, e_b = probes[i // probe_every]
+                        e_a.record(stream)
+                        ok |= interact(pp, npp)
+                        e_b.record(stream)
+                        ev_mid.append((e_a, e_b))
+                    else:
+                        ok |= interact(pp, npp)
+                else:
+                    ok |= interact(pp, npp)
+            ev1.record(stream)
+        barrier()
+        assert ok == 0, "a call in the timed region failed"
+        ms = ev0.elapsed_time(ev1)
+        if ev_mid:
+            kern_ms = sum(a.elapsed_time(b) for a, b in ev_mid) / len(ev_mid)
+            kern_pairs = float(np.mean([len(launches[i]) for i in range(0, K, probe_every)]))
+        else:
+            kern_ms, kern_pairs = ms / K, float(np.mean([len(p) for p in launches]))
+        return ms, kern_ms, kern_pairs, sw.kernel_launches() - l0
+
+    def kernel_bytes(self, pairs_per_launch):
+        """Algorithmic bytes one launch of the interaction kernel moves."""
+        wl = self.wl
+        b = interaction_bytes(wl["d"], wl["bits"], wl["mode"], wl.get("prefix", 16)) * pairs_per_launch
+        if self.fused and wl["mode"] != 0:
+            b += 8 * wl["d"] * pairs_per_launch             # the responder's model is read and written too
+        return b
+
+    def end_to_end(self, launches, seconds, barrier):
+        """The same steps through the public binding with host buffers inside the timed region: every step's pair
+        list comes from pinned host memory, a result of every step (the block exponents that the first initiator
+        published) is read back to pinned host memory, and the potential is read (synchronising, which also delivers
+        the queued rows) every 32 steps. Runs for at least `seconds` and at least len(launches) steps.
+        Returns (pairs processed, ms, host-to-device bytes per step, device-to-host bytes per step)."""
+        g, torch, wl, sw, stream = self.g, self.torch, self.wl, self.sw, self.stream
+        nblk = (wl["d"] + 1023) // 1024
+        pinned = [torch.from_numpy(np.ascontiguousarray(p, dtype=np.int32).copy()).pin_memory() for p in launches]
+        chunk = 64 if self.sequence else 1        # sequential gossip: 64 time steps per call (one kernel launch)
+        if self.sequence:
+            flat = torch.from_numpy(np.ascontiguousarray(np.concatenate(launches), dtype=np.int32).copy()).pin_memory()
+            nchunks_have = max(1, len(flat) // chunk)
+        ring = torch.empty((32, nblk), dtype=torch.int8).pin_memory()     # results of the last 32 steps
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+        def one(i):
+            if self.sequence:
+                c0 = (i % nchunks_have) * chunk
+                pairs = flat[c0:c0 + chunk].numpy()
+                rc = sw.run_sequence(pairs, wl["H"], wl["lr"], wl["bits"], True)
+                assert rc == 0, rc
+                first = int(pairs[-1, 0])
+                done = len(pairs)
+            else:
+                pairs = pinned[i % len(pinned)].numpy()
+                self.step(pairs)
+                first = int(pairs[0, 0])
+                done = len(pairs)
+            rc = sw.get_async(g.T_EXPS, first, ring[i % 32])
+            assert rc == 0, rc
+            return done, pairs.nbytes
+
+        # warm the path: first launch of the row-read kernel, first queued read, first potential
+        one(0)
+        sw.potential()
+        barrier()
+        t0 = time.perf_counter()
+        one(1)
+        sw.sync()
+        per_step = max(time.perf_counter() - t0, 1e-6)
+        steps = max(-(-len(launches) // chunk), int(seconds / per_step) + 1)
+        steps = min((steps + 31) // 32 * 32, 200000)          # whole groups of 32: the last potential read ends the run
+        barrier()
+        done = h2d = d2h = checksum = 0
+        t0 = time.perf_counter()
+        ev0.record(stream)
+        for i in range(steps):
+            dn, nb = one(i + 2)
+            done += dn
+            h2d += nb
+            d2h += nblk
+            if i % 32 == 31:
+                sw.potential()
+                d2h += 8
+                checksum += int(ring.sum())
+        ev1.record(stream)
+        barrier()
+        ms = max(ev0.elapsed_time(ev1), (time.perf_counter() - t0) * 1e3)
+        return done, ms, h2d / steps, d2h / steps, steps
+
+    def close(self):
+        self.sw.close()
+
+
+def table_entry(g, torch, wl, name, args, stream, peak, local_rank):
+    """A short run (at least 0.25 s of timed steps) of one workload: interactions/s of the whole step, the fused
+    interaction kernel's time, its algorithmic GB/s and fraction of the measured copy bandwidth, clocks."""
+    r = Runner(g, torch, wl, name, 0, stream, args)
+
+    def barrier():
+        torch.cuda.synchronize()
+    warm = [r.sched.next() for _ in range(5)]
+    for p in warm:
+        r.step(p)
+    barrier()
+    probe = [r.sched.next() for _ in range(8)]
+    ms, _, _, _ = r.timed(probe, barrier)
+    K = int(min(20000, max(16, 0.25 / max(ms / len(probe) * 1e-3, 1e-7))))
+    launches = [r.sched.next() for _ in range(K)]
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ms, kern_ms, kern_pairs, nl = r.timed(launches, barrier)
+    clocks = sampler.stop()
+    pairs_total = sum(len(p) for p in launches)
+    entry = {"interactions_per_s": pairs_total / (ms * 1e-3), "steps": K, "seconds": ms * 1e-3, "ms_per_step": ms / K,
+             "pairs_per_launch": pairs_total / K, "gpu_launches": int(nl), "clocks": clocks,
+             "config": {k: wl[k] for k in ("n", "d", "topology", "pairs", "bits", "mode", "H")}}
+    if r.sequence:
+        entry.update({"kernel": "lsq_sequence_kernel", "single_launch_sequence": True, "bound": "latency",
+                      "us_per_whole_step": 1e3 * ms / K})
+    else:
+        gbs = r.kernel_bytes(kern_pairs) / (kern_ms * 1e-3) / 1e9
+        entry.update({"kernel": kernel_name(wl), "interaction_kernel_ms": kern_ms,
+                      "interaction_only_per_s": kern_pairs / (kern_ms * 1e-3), "algorithmic_GBps": gbs,
+                      "frac": gbs / peak, "frac_of_8000": gbs / 8000.0})
+    r.close()
+    del r
+    torch.cuda.empty_cache()
+    return entry
+
+
 def run_ours(args, wl, name):
     import torch
     from paper_1910_12308_b200 import binding as g
@@ -320,180 +572,108 @@ def run_ours(args, wl, name):
         raise RuntimeError("bench: no CUDA device (the library has no CPU path)")
     torch.cuda.set_device(local_rank)
     use_dist = world > 1
+    dist = None
     if use_dist:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     stream = torch.cuda.current_stream()
-    sw = g.Swarm(wl["n"], wl["d"], wl["topology"], wl["degree"], wl["seed"] + 1000 * rank, stream=stream)
-    if wl["cfg"]:
-        sw.configure(**wl["cfg"])
-    adj = sw.get_all(g.T_ADJ)
-    sched = PairSchedule(wl, adj)
+    r = Runner(g, torch, wl, name, 1000 * rank, stream, args)
+    sw, fused, sequence = r.sw, r.fused, r.sequence
     K, W = args.steps, args.warmup
-    launches = [sched.next() for _ in range(K + W)]
+    launches = [r.sched.next() for _ in range(K + W)]
     npairs_total = sum(len(p) for p in launches[W:])
-
-    # elementwise (synthetic) objective, on request: the nodes of the pairs step inside the interaction kernel
-    fused = (wl["H"] > 0 and wl["cfg"].get("objective") == 1 and not wl.get("step_all") and args.fused)
-
-    # sequential gossip on short models: the whole timed region is one swarm_run_sequence call
-    sequence = bool(wl.get("sequence")) and wl["pairs"] == 1 and wl["mode"] == 0 and not args.stepwise
-
-    def step(pairs):
-        if fused:
-            rc = sw.step(pairs, wl["H"], wl["lr"], wl["bits"], wl["mode"], True)
-            assert rc == 0, rc
-            return
-        if wl["H"] > 0:
-            rc = sw.local_steps(stepping_nodes(wl, pairs), wl["H"], wl["lr"])
-            assert rc == 0, rc
-        rc = sw.interact(pairs, wl["bits"], wl["mode"])
-        assert rc == 0, rc
 
     def barrier():
         if use_dist:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # arguments are marshalled once, outside the timed region; the loop only crosses the C ABI
-    import ctypes as C
-    L, h = sw._L, sw._h
-    calls = []
-    for pairs in launches[W:]:
-        pa = np.ascontiguousarray(pairs, dtype=np.int32)
-        na = np.ascontiguousarray(stepping_nodes(wl, pairs), dtype=np.int32)
-        calls.append((pa, pa.ctypes.data_as(C.POINTER(g.SwarmPair)), len(pa), na,
-                      na.ctypes.data_as(C.POINTER(C.c_int32)), len(na)))
-    H, lr, bits, mode = wl["H"], wl["lr"], wl["bits"], wl["mode"]
-    probe_every = 8                       # the interaction kernel is bracketed by events on every 8th step
-    probes = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-              for _ in range(0, K, probe_every)] if (H > 0 and not fused) else []
-    # ---- device-resident timing
+    # ---- device-resident timing: W untimed steps, then exactly K timed steps
     for pairs in launches[:W]:
-        step(pairs)
+        r.step(pairs)
     barrier()
     sampler = ClockSampler(local_rank)
     sampler.start()
-    l0 = sw.kernel_launches()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev_mid = []
-    ok = 0
-    ev0.record(stream)
-    if sequence:
-        seq = np.ascontiguousarray(np.concatenate(launches[W:]), dtype=np.int32)
-        ok |= L.swarm_run_sequence(h, seq.ctypes.data_as(C.POINTER(g.SwarmPair)), len(seq), H, lr, bits, 1)
-        calls = []
-        probes = []
-    for i, (_, pp, npp, _, nn, ncount) in enumerate(calls):
-        if fused:
-            ok |= L.swarm_step(h, pp, npp, H, lr, bits, mode, 1)
-        elif H > 0:
-            ok |= L.swarm_local_steps(h, nn, ncount, H, lr)
-            if i % probe_every == 0:
-                e_a, e_b = probes[i // probe_every]
-                e_a.record(stream)
-                ok |= L.swarm_interact(h, pp, npp, bits, mode)
-                e_b.record(stream)
-                ev_mid.append((e_a, e_b))
-            else:
-                ok |= L.swarm_interact(h, pp, npp, bits, mode)
-        else:
-            ok |= L.swarm_interact(h, pp, npp, bits, mode)
-    ev1.record(stream)
-    barrier()
-    assert ok == 0, "a call in the timed region failed"
+    ms_local, kern_ms, kern_pairs, gpu_launches = r.timed(launches[W:], barrier)
     clocks = sampler.stop()
-    gpu_launches = sw.kernel_launches() - l0
-    ms_local = ev0.elapsed_time(ev1)
     ms, pairs_all = aggregate_over_ranks(ms_local, npairs_total, dist if use_dist else None, "cuda")
     value = pairs_all / (ms * 1e-3)
 
     # fused interaction kernel: average launch duration inside the timed region
-    if ev_mid:
-        kern_ms = sum(a.elapsed_time(b) for a, b in ev_mid) / len(ev_mid)
-    else:
-        kern_ms = ms_local / K
-    per_launch_bytes = interaction_bytes(wl["d"], wl["bits"], wl["mode"]) * npairs_total / K
-    if fused and wl["mode"] != 0:
-        per_launch_bytes += 8 * wl["d"] * npairs_total / K      # the responder's model is read and written too
+    per_launch_bytes = r.kernel_bytes(kern_pairs)
     achieved = per_launch_bytes / (kern_ms * 1e-3) / 1e9
     peak, peak_kind = measured_peak()
 
-    # ---- end to end through the C ABI with host buffers: pair lists come from pinned host memory,
-    # the step's result (block exponents of the first initiator) is read back into pinned memory every step
-    # (asynchronously, consumed in batches of 32), the potential every 32 steps (synchronising).
-    e2e_steps = min(K, 2000)
-    pinned = [torch.from_numpy(p.copy()).pin_memory() for p in launches[W:W + e2e_steps]]
-    barrier()
-    d2h = 0
-    nblk = (wl["d"] + 1023) // 1024
-    ring = torch.empty((32, nblk), dtype=torch.int8).pin_memory()     # results of the last 32 steps
-    checksum = 0
-    t0 = time.perf_counter()
-    ev0.record(stream)
-    for i, pt in enumerate(pinned):
-        pairs = pt.numpy()
-        step(pairs)
-        # the step's result is read back every step, queued behind the step on the same stream; the host
-        # consumes the last 32 results at each synchronising potential read
-        rc = sw.get_async(g.T_EXPS, int(pairs[0, 0]), ring[i % 32])
-        assert rc == 0, rc
-        d2h += nblk
-        if i % 32 == 31:
-            sw.potential()
-            d2h += 8
-            checksum += int(ring.sum())
-    ev1.record(stream)
-    barrier()
-    checksum += int(ring.sum())
-    e2e_ms = ev0.elapsed_time(ev1)
-    wall_ms = (time.perf_counter() - t0) * 1e3
-    e2e_ms = max(e2e_ms, wall_ms)
-    e2e_pairs = sum(len(p) for p in launches[W:W + e2e_steps])
+    # ---- end to end through the public binding with host buffers (see Runner.end_to_end)
+    e2e_pairs, e2e_ms, h2d, d2h, e2e_steps = r.end_to_end(launches[W:], args.e2e_seconds, barrier)
     e2e_ms, e2e_pairs_all = aggregate_over_ranks(e2e_ms, e2e_pairs, dist if use_dist else None, "cuda")
-    e2e = {"value": e2e_pairs_all / (e2e_ms * 1e-3), "unit": UNIT,
-           "h2d_bytes_per_step": int(np.mean([len(p) * 16 for p in launches[W:W + e2e_steps]])),
-           "d2h_bytes_per_step": int(d2h / e2e_steps)}
+    e2e = {"value": e2e_pairs_all / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(round(h2d)),
+           "d2h_bytes_per_step": int(round(d2h)), "steps": e2e_steps, "seconds": e2e_ms * 1e-3,
+           "calls_per_step": ("swarm_run_sequence (64 time steps per call)" if sequence else
+                              ("swarm_step" if fused else ("swarm_local_steps, swarm_interact" if wl["H"] > 0
+                                                           else "swarm_interact")))
+           + ", swarm_get_tensor_async; swarm_potential every 32 steps"}
 
+    traffic = traffic_of(name, kern_pairs)
+    roofline = {"bound": "hbm", "kernel": kernel_name(wl, fused),
+                "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "what": "algorithmic bytes per launch / CUDA-event time of the launch (not DRAM traffic)",
+                "peak_kind": peak_kind, "frac_of_8000": achieved / 8000.0, "traffic": traffic,
+                "algorithmic_bytes_per_launch": per_launch_bytes, "kernel_ms": kern_ms}
+    if traffic is not None:
+        # what reached DRAM in the profiler's capture, at the launch time measured here
+        roofline["dram_GBps"] = traffic / (kern_ms * 1e-3) / 1e9
+        roofline["dram_frac"] = roofline["dram_GBps"] / peak
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
         "config": {"workload": name, **{k: wl[k] for k in ("n", "d", "topology", "pairs", "bits", "mode", "H")},
                    "fused_local_steps": bool(fused), "single_launch_sequence": bool(sequence),
-                   "l2": "inputs larger than L2: every launch streams all models it touches from HBM",
+                   "l2": ("inputs larger than L2: the models a launch touches (%.0f MB) exceed the 126 MB L2, so every "
+                          "launch reads them from HBM; part of the lines it rewrites is still in L2 when it ends"
+                          % (2 * kern_pairs * wl["d"] * 4 / 1e6)) if wl["d"] * kern_pairs * 8 > 126e6 else
+                         "L2 flushed by nothing: the working set fits in L2 (latency-bound workload, no HBM roofline)",
                    "replicas": world},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": int(gpu_launches),
-        "roofline": {"bound": "hbm", "kernel": ("interact_identity_kernel" if wl["bits"] == 32 else
-                                ["interact_blocking_kernel", "interact_nonblocking_kernel", "interact_registers_kernel"][wl["mode"]])
-                     + (" (local steps fused)" if fused else ""),
-                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_kind": peak_kind, "frac_of_8000": achieved / 8000.0, "traffic": traffic_of(name, npairs_total / K),
-                     "algorithmic_bytes_per_launch": per_launch_bytes, "kernel_ms": kern_ms},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(gpu_launches), "roofline": roofline,
     }
-    if wl["mode"] == 2 and not fused:
-        # the two-register kernel is bound by instruction issue, not by HBM: report it against the issue rate
-        # (148 SMs x 4 schedulers x SM clock) with its warp instructions per 1024-block from the ncu capture
+    counters = profiler_counters(name)
+    if wl["mode"] == 2 and not fused and "warp_instructions_per_block" in counters:
+        # the two-register kernel is bound by instruction issue where it does not reach the HBM rate: also report it
+        # against the issue rate (148 SMs x 4 schedulers x SM clock) with its warp instructions per 1024-block
         nblk = (wl["d"] + 1023) // 1024
-        instr = REGISTER_KERNEL_INSTR_PER_BLOCK * nblk * npairs_total / K
+        instr = counters["warp_instructions_per_block"] * nblk * kern_pairs
         rate = instr / (kern_ms * 1e-3) / 1e12
         issue_peak = 148 * 4 * (clocks["sm_max_mhz"] or 1965) * 1e6 / 1e12
-        hbm = out["roofline"]
-        out["roofline"] = {"bound": "alu", "kernel": hbm["kernel"], "achieved": rate, "peak": issue_peak,
-                           "unit": "T warp-instructions/s", "frac": rate / issue_peak, "traffic": traffic_of(name, npairs_total / K),
-                           "warp_instructions_per_launch": instr, "kernel_ms": kern_ms,
-                           "hbm": {k: hbm[k] for k in ("achieved", "peak", "unit", "frac", "peak_kind", "frac_of_8000",
-                                                       "algorithmic_bytes_per_launch")}}
+        out["roofline"]["issue"] = {"achieved": rate, "peak": issue_peak, "unit": "T warp-instructions/s",
+                                    "frac": rate / issue_peak, "warp_instructions_per_launch": instr}
     # the same launches for about two seconds: long enough for the board to settle at its power limit, which the
     # timed region above (a burst of K launches) is not; reported beside the burst figure, with the clock seen
-    if calls and H == 0 and not fused and rank == 0 and world == 1:
+    if not sequence and wl["H"] == 0 and not fused and rank == 0 and world == 1:
+        L, h, ok = sw._L, sw._h, 0
+        bits, mode = wl["bits"], wl["mode"]
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         reps = max(1, int(2.0 / max(ms_local * 1e-3, 1e-6)))
+        # An averaging-only swarm contracts: kept going for hundreds of thousands of interactions it reaches
+        # consensus, where the lattice steps are set by the magnitude rule and the kernels take the defining form of
+        # the lattice arithmetic (another instruction stream than the workload's). The workload is 10^4 interactions
+        # from the initial state, so the models are put back to that state every 10^4 interactions (one
+        # device-to-device copy on the same stream, inside the timed loop and counted in its time).
+        sw.configure(**wl["cfg"])
+        xt = sw.model_tensor()
+        x_init = xt.clone()
+        restore_every = max(1, int(round(1e4 / max(kern_pairs, 1))))
+        barrier()
         sampler2 = ClockSampler(local_rank)
         sampler2.start()
+        done_launches = 0
         ev0.record(stream)
         for _ in range(reps):
-            for (_, pp, npp, _, _, _) in calls:
+            for (_, pp, npp, _, _, _) in r.calls:
                 ok |= L.swarm_interact(h, pp, npp, bits, mode)
+                done_launches += 1
+                if done_launches % restore_every == 0:
+                    xt.copy_(x_init)
         ev1.record(stream)
         barrier()
         assert ok == 0
@@ -502,7 +682,9 @@ def run_ours(args, wl, name):
         s_gbs = per_launch_bytes / (s_ms * 1e-3) / 1e9
         out["sustained"] = {"launches": reps * K, "seconds": ev0.elapsed_time(ev1) * 1e-3,
                             "value": npairs_total * reps / (ev0.elapsed_time(ev1) * 1e-3), "unit": UNIT,
-                            "kernel_ms": s_ms, "achieved": s_gbs, "frac": s_gbs / peak, "clocks": clk2}
+                            "kernel_ms": s_ms, "achieved": s_gbs, "frac": s_gbs / peak, "clocks": clk2,
+                            "models_restored_every_launches": restore_every}
+        del x_init
         # yardstick under the same conditions: a plain device copy (library kernel) kept up for as long
         a = torch.empty(1 << 28, dtype=torch.float32, device="cuda")
         b = torch.empty_like(a)
@@ -527,6 +709,7 @@ def run_ours(args, wl, name):
 
     # mean model and potential (one HBM pass over all n models each), timed on their own
     reps = 20
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     mu = torch.empty(wl["d"], dtype=torch.float32, device="cuda")
     L, h = sw._L, sw._h
     for name_k, call in (("mean_model", lambda: L.swarm_mean_model(h, mu.data_ptr())),
@@ -542,6 +725,25 @@ def run_ours(args, wl, name):
         t_ms = ev0.elapsed_time(ev1) / reps
         out.setdefault("aux_kernels", {})[name_k] = {
             "ms": t_ms, "GB/s": 4.0 * wl["n"] * wl["d"] / (t_ms * 1e-3) / 1e9, "bytes": 4 * wl["n"] * wl["d"]}
+    r.close()
+    del r, mu
+    torch.cuda.empty_cache()
+    if rank == 0 and world == 1 and not args.no_table:
+        # short runs of the five workloads of the measurement table, in the same process and on the same board
+        table = {}
+        for nm in TABLE_WORKLOADS:
+            if nm == name and not (fused or args.stepwise):
+                table[nm] = {"interactions_per_s": value, "steps": K, "seconds": ms * 1e-3, "ms_per_step": ms / K,
+                             "pairs_per_launch": npairs_total / K, "kernel": kernel_name(wl),
+                             "interaction_kernel_ms": kern_ms, "algorithmic_GBps": achieved, "frac": achieved / peak,
+                             "frac_of_8000": achieved / 8000.0, "clocks": clocks, "same_as": "the timed region above"}
+                if sequence:
+                    table[nm] = {"interactions_per_s": value, "steps": K, "seconds": ms * 1e-3, "bound": "latency",
+                                 "kernel": "lsq_sequence_kernel", "us_per_whole_step": 1e3 * ms / K, "clocks": clocks,
+                                 "same_as": "the timed region above"}
+                continue
+            table[nm] = table_entry(g, torch, WORKLOADS[nm], nm, args, stream, peak, local_rank)
+        out["workloads"] = table
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v, T, nl, tt, swl = time_oracle(wl, budget_s=10.0, max_launches=40)
         v1, _, nl1, tt1, _ = time_oracle(wl, budget_s=3.0, max_launches=1, threads=1)
@@ -557,25 +759,6 @@ def run_ours(args, wl, name):
         print(json.dumps(out))
 
 
-# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel (see profiles/);
-# None until a capture of the current kernel exists.
-TRAFFIC = {"ring64_d1m_b4": 512.1e6}
-# the same per pair of a launch, for workloads whose launches differ in their number of pairs: captured on a reduced
-# copy (8 nodes, 3 pairs per launch) for the single-buffer kernel and on the full workload (14 pairs) for the
-# two-register kernel; traffic is proportional to the pairs of a launch (every pair streams its own rows once)
-TRAFFIC_PER_PAIR = {"regular32_resnet18_b8_nb": 214.8e6, "regular32_resnet18_b8_reg": 288.1e6}
-# smsp__inst_executed.sum per 1024-coordinate block of interact_registers_kernel<8> (see profiles/)
-REGISTER_KERNEL_INSTR_PER_BLOCK = 3607
-
-
-def traffic_of(name, pairs_per_launch):
-    if name in TRAFFIC:
-        return TRAFFIC[name]
-    if name in TRAFFIC_PER_PAIR:
-        return TRAFFIC_PER_PAIR[name] * pairs_per_launch
-    return None
-
-
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -584,6 +767,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-seconds", type=float, default=0.3,
+                    help="least duration of the end-to-end loop (it always runs at least --steps steps)")
+    ap.add_argument("--no-table", action="store_true",
+                    help="skip the short runs of the other workloads of the measurement table (\"workloads\" object)")
     ap.add_argument("--stepwise", action="store_true",
                     help="sequential small-model workload: two calls per step instead of one swarm_run_sequence "
                          "call for the whole timed region")

@@ -232,6 +232,17 @@ int swarm_register_publish(swarm_ctx *ctx, int32_t bits);
 int swarm_set_own_prefix(swarm_ctx *ctx, int32_t bits);
 int swarm_get_own_prefix(swarm_ctx *ctx, int32_t *bits_host);
 
+/* The same passages, per reader: swarm_interact in SWARM_REGISTERS mode in which the initiator of
+ * pairs_host[p] reads prefixes_host[p] bits (8 or 16) of its responder's own register, whatever
+ * swarm_set_own_prefix says (that setting is the prefix of every pair of a plain swarm_interact). A launch can
+ * thus mix partners that keep meeting (8 bits: half of the partner's own register crosses the memory system)
+ * with a reader whose snapshot is far from its partner's (16 bits). The prefix is the reader's statement about
+ * its distance; the construction has no check value, so a prefix that is too short aliases (defined
+ * behaviour, see swarm_set_own_prefix). prefixes_host: npairs int32 values, host memory, read during the call.
+ * Errors: those of swarm_interact; EINVAL for a prefix other than 8 or 16 or a NULL list with npairs > 0. */
+int swarm_interact_prefixed(swarm_ctx *ctx, const swarm_pair *pairs_host, const int32_t *prefixes_host,
+                            int32_t npairs, int32_t bits);
+
 /* State access (checkpointing, test injection). `which` selects the array, `node` the row
  * (ignored for whole-context arrays). bytes must equal the row size exactly. Both synchronise. */
 enum {
@@ -263,6 +274,10 @@ int swarm_get_tensor(swarm_ctx *ctx, int32_t which, int32_t node, void *dst_host
  * copy engine straight to dst_host (pinned memory, or that copy is not asynchronous). */
 int swarm_get_tensor_async(swarm_ctx *ctx, int32_t which, int32_t node, void *dst_host, size_t bytes);
 int swarm_set_tensor(swarm_ctx *ctx, int32_t which, int32_t node, const void *src_host, size_t bytes);
+/* Rows row0 .. row0 + nrows - 1 of least-squares data matrix `matrix` as floats (bf16 storage is widened), nrows * d
+ * floats into dst_host; a whole matrix (SWARM_T_A) can be gigabytes. bytes must equal nrows * d * 4. Synchronises.
+ * Errors: ESTATE (no least-squares data), ERANGE (matrix, rows), EINVAL. */
+int swarm_get_data_rows(swarm_ctx *ctx, int32_t matrix, int32_t row0, int32_t nrows, float *dst_host, size_t bytes);
 
 /* Whole-context counters: launch counter of the pair sampler and the "snapshots stale" flag. */
 int swarm_get_state(swarm_ctx *ctx, uint32_t *launch_host, int32_t *b_stale_host);

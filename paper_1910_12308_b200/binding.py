@@ -25,9 +25,9 @@ T_X, T_B, T_CODES, T_EXPS, T_ADJ, T_A, T_BVEC, T_XSTAR, T_SCALARS, T_COUNTERS, T
 TOPOLOGY = {"complete": TOPO_COMPLETE, "ring": TOPO_RING, "regular": TOPO_REGULAR}
 
 EXPORTS = [
-    "swarm_set_allocator", "swarm_init", "swarm_local_steps", "swarm_local_steps_geometric", "swarm_interact", "swarm_step", "swarm_run_sequence", "swarm_mean_model",
+    "swarm_set_allocator", "swarm_init", "swarm_local_steps", "swarm_local_steps_geometric", "swarm_interact", "swarm_interact_prefixed", "swarm_step", "swarm_run_sequence", "swarm_mean_model",
     "swarm_potential", "swarm_track_staleness", "swarm_aux_potentials", "swarm_configure", "swarm_sample_pairs", "swarm_publish", "swarm_register_publish", "swarm_set_own_prefix", "swarm_get_own_prefix", "swarm_get_buffer_mode",
-    "swarm_set_buffer_mode", "swarm_get_tensor", "swarm_get_tensor_async",
+    "swarm_set_buffer_mode", "swarm_get_tensor", "swarm_get_data_rows", "swarm_get_tensor_async",
     "swarm_set_tensor", "swarm_get_state", "swarm_set_state", "swarm_model_ptr", "swarm_set_stream",
     "swarm_sync", "swarm_set_wait_limit", "swarm_potential_static", "swarm_kernel_launches", "swarm_last_cuda_error", "swarm_strerror", "swarm_destroy",
 ]
@@ -65,7 +65,8 @@ class SwarmError(RuntimeError):
 
 
 def library_path():
-    return os.path.join(_HERE, "libswarm_b200.so")
+    """The in-tree library; SWARM_B200_LIBRARY names another build of it to load instead (for comparing builds)."""
+    return os.environ.get("SWARM_B200_LIBRARY") or os.path.join(_HERE, "libswarm_b200.so")
 
 
 def load():
@@ -84,6 +85,7 @@ def load():
         "swarm_local_steps": (C.c_int, [vp, C.POINTER(i32), i32, i32, f32]),
         "swarm_local_steps_geometric": (C.c_int, [vp, C.POINTER(i32), i32, i32, f32, C.POINTER(i32)]),
         "swarm_interact": (C.c_int, [vp, C.POINTER(SwarmPair), i32, i32, i32]),
+        "swarm_interact_prefixed": (C.c_int, [vp, C.POINTER(SwarmPair), C.POINTER(i32), i32, i32]),
         "swarm_step": (C.c_int, [vp, C.POINTER(SwarmPair), i32, i32, f32, i32, i32, i32]),
         "swarm_run_sequence": (C.c_int, [vp, C.POINTER(SwarmPair), i32, i32, f32, i32, i32]),
         "swarm_mean_model": (C.c_int, [vp, vp]),
@@ -100,6 +102,7 @@ def load():
         "swarm_set_buffer_mode": (C.c_int, [vp, i32]),
         "swarm_get_tensor": (C.c_int, [vp, i32, i32, vp, C.c_size_t]),
         "swarm_get_tensor_async": (C.c_int, [vp, i32, i32, vp, C.c_size_t]),
+        "swarm_get_data_rows": (C.c_int, [vp, i32, i32, i32, vp, C.c_size_t]),
         "swarm_set_tensor": (C.c_int, [vp, i32, i32, vp, C.c_size_t]),
         "swarm_get_state": (C.c_int, [vp, C.POINTER(u32), C.POINTER(i32)]),
         "swarm_set_state": (C.c_int, [vp, u32, i32]),
@@ -228,6 +231,15 @@ class Swarm:
         arr, ptr = _pairs_array(pairs)
         return self._L.swarm_interact(self._h, ptr, len(arr), bits, mode)
 
+    def interact_prefixed(self, pairs, prefixes, bits):
+        """Two-register interactions; the initiator of pairs[p] reads prefixes[p] (8 or 16) bits of its
+        responder's own register. Returns the C code."""
+        arr, ptr = _pairs_array(pairs)
+        pf = np.ascontiguousarray(prefixes, dtype=np.int32)
+        if len(pf) != len(arr):
+            raise ValueError("one prefix per pair")
+        return self._L.swarm_interact_prefixed(self._h, ptr, pf.ctypes.data_as(C.POINTER(C.c_int32)), len(arr), bits)
+
     def step(self, pairs, H, lr, bits, mode=BLOCKING, step_responders=True):
         """H local steps of the nodes in `pairs` (initiators only if step_responders is false), then the
         interactions, in one call; returns the C code."""
@@ -322,6 +334,17 @@ class Swarm:
         self._check(self._L.swarm_model_ptr(self._h, C.byref(p), C.byref(pitch)), "swarm_model_ptr")
         return p.value, pitch.value
 
+    def model_tensor(self):
+        """The live models as an (n, pitch) float32 torch tensor over the library's own memory (contexts whose
+        device memory comes from PyTorch only): for callers that read or restore models in place, on the
+        context's stream. Valid until the next configure / close."""
+        import torch
+        ptr, pitch = self.model_ptr()
+        block = _torch_blocks.get(ptr)
+        if block is None:
+            raise RuntimeError("swarm: the models of this context are not backed by a torch allocation")
+        return block[: self.n * pitch * 4].view(torch.float32).view(self.n, pitch)
+
     # -- state access
     def _row_spec(self, which):
         m = self.cfg.lsq_m
@@ -337,6 +360,13 @@ class Swarm:
         dt, count = self._row_spec(which)
         out = np.empty(count, dtype=dt)
         self._check(self._L.swarm_get_tensor(self._h, which, node, out.ctypes.data, out.nbytes), "swarm_get_tensor")
+        return out
+
+    def get_data_rows(self, matrix, row0, nrows):
+        """Rows row0 .. row0 + nrows - 1 of a least-squares data matrix as an (nrows, d) float array."""
+        out = np.empty((nrows, self.d), dtype=np.float32)
+        self._check(self._L.swarm_get_data_rows(self._h, matrix, row0, nrows, out.ctypes.data, out.nbytes),
+                    "swarm_get_data_rows")
         return out
 
     def get_async(self, which, node, out):

@@ -164,7 +164,8 @@ StoreView view_of(const swarm_ctx* c) {
   s.X = c->X; s.B = c->B; s.codes = c->codes; s.exps = c->exps; s.own = c->own; s.oexps = c->oexps;
   s.pitch = c->pitch; s.d = c->d; s.nblk = c->nblk; s.n = c->n;
   s.key0 = (uint32_t)c->seed; s.key1 = (uint32_t)(c->seed >> 32);
-  s.own_prefix = c->own_prefix;
+  s.rk = philox_round_keys(s.key0, s.key1);
+  division_magic((uint64_t)c->nblk, &s.nblk_magic, &s.nblk_shift);
   return s;
 }
 LsqView lsq_of(const swarm_ctx* c) {
@@ -741,9 +742,14 @@ int swarm_local_steps_geometric(swarm_ctx* c, const int32_t* node_ids, int32_t c
 // One interaction launch; fused_H > 0 runs that many synthetic-gradient local steps of the initiators (and of
 // the responders when `responders` is set) inside the interaction kernel first.
 static int interact_impl(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, int32_t bits, int32_t mode,
-                         int32_t fused_H, float lr, int32_t responders) {
+                         int32_t fused_H, float lr, int32_t responders, const int32_t* prefixes = nullptr) {
   if (!c || npairs < 0 || (npairs > 0 && !pairs)) return SWARM_EINVAL;
   if (mode != SWARM_BLOCKING && mode != SWARM_NONBLOCKING && mode != SWARM_REGISTERS) return SWARM_EINVAL;
+  if (prefixes) {
+    if (mode != SWARM_REGISTERS) return SWARM_EINVAL;
+    for (int p = 0; p < npairs; ++p)
+      if (prefixes[p] != 8 && prefixes[p] != 16) return SWARM_EINVAL;
+  }
   const bool quant = bits >= 2 && bits <= 8;
   if (!(quant || (bits == 32 && mode == SWARM_BLOCKING))) return SWARM_EINVAL;
   if (mode == SWARM_NONBLOCKING && !c->cfg.nonblocking) return SWARM_ESTATE;
@@ -776,7 +782,7 @@ static int interact_impl(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, 
   for (int p = 0; p < npairs; ++p) {
     pd[p].a = pairs[p].a; pd[p].b = pairs[p].b;
     pd[p].wa = c->w[pairs[p].a]; pd[p].wb = c->w[pairs[p].b];
-    pd[p].woa = c->wo[pairs[p].a]; pd[p].pad = 0;
+    pd[p].woa = c->wo[pairs[p].a]; pd[p].prefix = (uint32_t)(prefixes ? prefixes[p] : c->own_prefix);
     pd[p].lsa = c->ls[pairs[p].a]; pd[p].lsb = c->ls[pairs[p].b];
   }
   FusedSteps fs{};
@@ -826,6 +832,12 @@ int swarm_interact(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, int32_
   return interact_impl(c, pairs, npairs, bits, mode, 0, 0.0f, 0);
 }
 
+int swarm_interact_prefixed(swarm_ctx* c, const swarm_pair* pairs, const int32_t* prefixes, int32_t npairs,
+                            int32_t bits) {
+  if (npairs > 0 && !prefixes) return SWARM_EINVAL;
+  return interact_impl(c, pairs, npairs, bits, SWARM_REGISTERS, 0, 0.0f, 0, prefixes);
+}
+
 int swarm_step(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, int32_t H, float lr, int32_t bits, int32_t mode,
                int32_t step_responders) {
   if (!c || H < 0 || npairs < 0 || (npairs > 0 && !pairs)) return SWARM_EINVAL;
@@ -872,7 +884,7 @@ int swarm_run_sequence(swarm_ctx* c, const swarm_pair* pairs, int32_t nsteps, in
   const StoreView s = view_of(c);
   const LsqView l = lsq_of(c);
   const bool lsq = c->cfg.objective == SWARM_OBJ_LSQ || c->cfg.objective == SWARM_OBJ_LOGISTIC;
-  if (!(lsq && H > 0 && bits != 32 && !c->tc_partial && lsq_sequence_supported(s, l))) {
+  if (!(lsq && bits != 32 && !c->tc_partial && lsq_sequence_supported(s, l))) {
     // no single-launch form for this configuration: the steps one by one
     for (int t = 0; t < nsteps; ++t) {
       const int rc = swarm_step(c, pairs + t, 1, H, lr, bits, SWARM_BLOCKING, step_responders);
@@ -901,7 +913,7 @@ int swarm_run_sequence(swarm_ctx* c, const swarm_pair* pairs, int32_t nsteps, in
       const int a = pairs[base + t].a, b = pairs[base + t].b;
       pd[t].a = a; pd[t].b = b;
       pd[t].wa = c->w[a]; pd[t].wb = c->w[b]; pd[t].woa = c->wo[a];
-      pd[t].lsa = c->ls[a]; pd[t].lsb = c->ls[b]; pd[t].pad = 0;
+      pd[t].lsa = c->ls[a]; pd[t].lsb = c->ls[b]; pd[t].prefix = 16;
       c->w[a] += 1; c->w[b] += 1;
       c->pbits[a] = bits; c->pbits[b] = bits;
       c->ls[a] += (uint32_t)H;
@@ -1174,6 +1186,32 @@ static int tensor_access(swarm_ctx* c, int32_t which, int32_t node, void* host, 
   if (write) SW_CUDA(c, cudaMemcpyAsync(dev, host, bytes, cudaMemcpyHostToDevice, c->stream));
   else SW_CUDA(c, cudaMemcpyAsync(host, dev, bytes, cudaMemcpyDeviceToHost, c->stream));
   if (wait) SW_SYNC(c);
+  return SWARM_OK;
+}
+
+int swarm_get_data_rows(swarm_ctx* c, int32_t matrix, int32_t row0, int32_t nrows, float* dst, size_t bytes) {
+  if (!c || !dst || nrows < 0) return SWARM_EINVAL;
+  if (!c->A) return SWARM_ESTATE;
+  if (matrix < 0 || matrix >= c->groups) return SWARM_ERANGE;
+  if (row0 < 0 || (int64_t)row0 + nrows > c->cfg.lsq_m) return SWARM_ERANGE;
+  const size_t d = (size_t)c->d;
+  if (bytes != (size_t)nrows * d * 4) return SWARM_EINVAL;
+  DeviceGuard guard(c->device);
+  SW_SYNC(c);
+  int nl = 0;
+  for (int32_t r = 0; r < nrows; ++r) {
+    char* hrow = (char*)dst + (size_t)r * d * 4;
+    const size_t row = (size_t)matrix * c->cfg.lsq_m + (size_t)(row0 + r);
+    if (c->cfg.lsq_dtype == SWARM_F32) {
+      SW_CUDA(c, cudaMemcpyAsync(hrow, (const float*)c->A + row * c->pitch, d * 4, cudaMemcpyDeviceToHost, c->stream));
+    } else {
+      SW_CUDA(c, launch_bf16_to_f32((const uint16_t*)c->A + row * c->pitch, c->convert_tmp, (int64_t)d, c->stream, &nl));
+      SW_CUDA(c, cudaMemcpyAsync(hrow, c->convert_tmp, d * 4, cudaMemcpyDeviceToHost, c->stream));
+      SW_SYNC(c);   // convert_tmp is reused per row
+    }
+  }
+  c->launches += nl;
+  SW_SYNC(c);
   return SWARM_OK;
 }
 

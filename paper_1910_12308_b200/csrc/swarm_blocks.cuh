@@ -15,7 +15,7 @@ constexpr int kSubCoords = 256;  // coordinates per sub-block
 __device__ __forceinline__ void fused_steps_block(f8 (&v)[kSub], const StoreView& s, const FusedSteps& fs, int node,
                                                   uint32_t event, int64_t blk, int lane) {
   const float c = fs.scalars[node * 3 + 1];
-  const PhiloxRoundKeys rk = philox_round_keys(s.key0, s.key1);
+  const PhiloxRoundKeys& rk = s.rk;
   const uint32_t g0 = (uint32_t)(blk * (kBlockCoords / 8) + lane);
   for (int q = 0; q < fs.H; ++q) {
 #pragma unroll
@@ -43,40 +43,77 @@ __device__ __forceinline__ void fused_steps_responder(const StoreView& s, const 
   for (int j = 0; j < kSub; ++j) st256(xb + j * kSubCoords, vb[j]);
 }
 
-// Encode / cross-decode / average / store phase of a blocking block, in the fast or the defining form of
-// the lattice arithmetic (LatticeOps).
-template <int BITS, bool FAST>
+// Encode / cross-decode / average of the 8 coordinate pairs a lane owns in one sub-block, in the fast or the
+// defining form of the lattice arithmetic (LatticeOps). ra, rb: the generator calls that hold the rounding
+// uniforms of the two buffers. ELIDE (fast form only) leaves the cross-decodes out: when the block's range
+// satisfies rho < L * 2^e strictly, |X^a - X^b| < L * 2^e holds for the exact difference of every coordinate
+// pair (rho is a maximum of rounded differences, and rounding to nearest cannot carry a value from L * 2^e or
+// above to below it), so the two scaled values differ by less than L, their floors by at most L, and the
+// encoder's index, floor or floor + 1, lies in the decoder's window [cell - L, cell + L + 1] around the
+// partner's cell: Dec returns the encoder's own lattice point (Corollary 1, the case where the writer knows
+// the distance to the decoding key). At equality, or with the exponent clamped, the decode stays.
+struct ExchangeScale {
+  float step, inv_step, unbias, half_step, half_unbias;
+};
+template <bool FAST>
+__device__ __forceinline__ ExchangeScale exchange_scale(int e) {
+  ExchangeScale sc;
+  sc.step = pow2f_exact(e);
+  sc.inv_step = pow2f_exact(-e);
+  sc.unbias = FAST ? -__fmul_rn(kCellBias, sc.step) : 0.0f;
+  sc.half_step = __fmul_rn(0.5f, sc.step);                  // 2^(e-1): a subnormal for e = -126, still exact
+  sc.half_unbias = __fmul_rn(0.5f, sc.unbias);
+  return sc;
+}
+template <int BITS, bool FAST, bool ELIDE>
+__device__ __forceinline__ void exchange8(const f8& va, const f8& vb, const uint4& ra, const uint4& rb,
+                                          const ExchangeScale& sc, f8& out, uint64_t& pka, uint64_t& pkb) {
+  using Ops = LatticeOps<FAST>;
+  static_assert(FAST || !ELIDE, "the decode is left out in the fast form only");
+  uint32_t ia[8], ib[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    uint32_t cell_a, cell_b;
+    ia[i] = Ops::encode(va.v[i], sc.inv_step, sr_word(ra, i), i & 1, cell_a);
+    ib[i] = Ops::encode(vb.v[i], sc.inv_step, sr_word(rb, i), i & 1, cell_b);
+    // b decodes a's codes with X^b as key and vice versa; the key's cell is already known
+    if constexpr (ELIDE) {
+      out.v[i] = Ops::mean_of_own(ia[i], ib[i], sc.half_step, sc.half_unbias);
+    } else {
+      const float Qa = Ops::value(Ops::template decode<BITS>(ia[i], cell_b), sc.step, sc.unbias);
+      const float Qb = Ops::value(Ops::template decode<BITS>(ib[i], cell_a), sc.step, sc.unbias);
+      out.v[i] = __fmul_rn(0.5f, __fadd_rn(Qa, Qb));
+    }
+  }
+  pka = pack_colours<BITS>(ia);
+  pkb = pack_colours<BITS>(ib);
+}
+
+template <int BITS, bool FAST, bool ELIDE>
 __device__ __forceinline__ void blocking_exchange(const f8 (&va)[kSub], const f8 (&vb)[kSub], float* xa, float* xb,
                                                   uint8_t* ca, uint8_t* cb, uint32_t group0, const StoreView& s,
                                                   const PairDesc& pd, int lane, int e) {
-  using Ops = LatticeOps<FAST>;
-  const float step = pow2f_exact(e), inv_step = pow2f_exact(-e);
-  const float unbias = FAST ? -__fmul_rn(kCellBias, step) : 0.0f;
-  constexpr uint32_t mask = (1u << BITS) - 1u;
+  const ExchangeScale sc = exchange_scale<FAST>(e);
 #pragma unroll
   for (int j = 0; j < kSub; ++j) {
     const uint32_t g = group0 + j * (kSubCoords / 8);
-    const uint4 ra = philox4x32_10(g, (uint32_t)pd.a, pd.wa, kStreamRounding, s.key0, s.key1);
-    const uint4 rb = philox4x32_10(g, (uint32_t)pd.b, pd.wb, kStreamRounding, s.key0, s.key1);
-    uint64_t pka = 0, pkb = 0;
+    const uint4 ra = philox4x32_10(g, (uint32_t)pd.a, pd.wa, kStreamRounding, s.rk);
+    const uint4 rb = philox4x32_10(g, (uint32_t)pd.b, pd.wb, kStreamRounding, s.rk);
+    uint64_t pka, pkb;
     f8 out;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      uint32_t cell_a, cell_b;
-      const uint32_t code_a = Ops::encode(va[j].v[i], inv_step, sr_word(ra, i), i & 1, cell_a) & mask;
-      const uint32_t code_b = Ops::encode(vb[j].v[i], inv_step, sr_word(rb, i), i & 1, cell_b) & mask;
-      pka |= (uint64_t)code_a << (i * BITS);
-      pkb |= (uint64_t)code_b << (i * BITS);
-      // b decodes a's codes with X^b as key and vice versa; the key's cell is already known
-      const float Qa = Ops::value(Ops::template decode<BITS>(code_a, cell_b), step, unbias);
-      const float Qb = Ops::value(Ops::template decode<BITS>(code_b, cell_a), step, unbias);
-      out.v[i] = __fmul_rn(0.5f, __fadd_rn(Qa, Qb));
-    }
+    exchange8<BITS, FAST, ELIDE>(va[j], vb[j], ra, rb, sc, out, pka, pkb);
     st256(xa + j * kSubCoords, out);
     st256(xb + j * kSubCoords, out);
     store_codes<BITS>(ca + j * (kSubCoords * BITS / 8), lane, pka);
     store_codes<BITS>(cb + j * (kSubCoords * BITS / 8), lane, pkb);
   }
+}
+
+// Whether a blocking block may leave the cross-decodes out: rho < L * 2^e strictly (see exchange8).
+template <int BITS>
+__device__ __forceinline__ bool decode_elidable(float rho, int e) {
+  constexpr float L = (float)((1 << (BITS - 1)) - 1);
+  return rho < __fmul_rn(L, pow2f_exact(e));
 }
 
 // Blocking interaction of one block (Algorithm 1, interaction lines, with both models present): exact
@@ -113,34 +150,25 @@ __device__ __forceinline__ void blocking_block(const StoreView& s, const PairDes
   const uint32_t group0 = (uint32_t)(blk * (kBlockCoords / 8) + lane);   // generator call index of sub-block 0
   uint8_t* ca = s.codes + (int64_t)pd.a * s.nblk * kBlockCoords + blk * (kBlockCoords * BITS / 8) + lane * BITS;
   uint8_t* cb = s.codes + (int64_t)pd.b * s.nblk * kBlockCoords + blk * (kBlockCoords * BITS / 8) + lane * BITS;
-  if (fast_range(M, pow2f_exact(-e), e)) blocking_exchange<BITS, true>(va, vb, xa, xb, ca, cb, group0, s, pd, lane, e);
-  else blocking_exchange<BITS, false>(va, vb, xa, xb, ca, cb, group0, s, pd, lane, e);
+  if (fast_range(M, pow2f_exact(-e), e)) {
+    if (decode_elidable<BITS>(rho, e)) blocking_exchange<BITS, true, true>(va, vb, xa, xb, ca, cb, group0, s, pd, lane, e);
+    else blocking_exchange<BITS, true, false>(va, vb, xa, xb, ca, cb, group0, s, pd, lane, e);
+  } else {
+    blocking_exchange<BITS, false, false>(va, vb, xa, xb, ca, cb, group0, s, pd, lane, e);
+  }
   if (lane == 0) {
     s.exps[(int64_t)pd.a * s.nblk + blk] = (int8_t)e;
     s.exps[(int64_t)pd.b * s.nblk + blk] = (int8_t)e;
   }
 }
 
-template <int BITS, bool FAST>
+template <int BITS, bool FAST, bool ELIDE>
 __device__ __forceinline__ void subblock_exchange(const f8& va, const f8& vb, float* xa, float* xb, uint8_t* ca,
                                                   uint8_t* cb, const uint4& ra, const uint4& rb, int lane, int e) {
-  using Ops = LatticeOps<FAST>;
-  const float step = pow2f_exact(e), inv_step = pow2f_exact(-e);
-  const float unbias = FAST ? -__fmul_rn(kCellBias, step) : 0.0f;
-  constexpr uint32_t mask = (1u << BITS) - 1u;
-  uint64_t pka = 0, pkb = 0;
+  const ExchangeScale sc = exchange_scale<FAST>(e);
+  uint64_t pka, pkb;
   f8 out;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    uint32_t cell_a, cell_b;
-    const uint32_t code_a = Ops::encode(va.v[i], inv_step, sr_word(ra, i), i & 1, cell_a) & mask;
-    const uint32_t code_b = Ops::encode(vb.v[i], inv_step, sr_word(rb, i), i & 1, cell_b) & mask;
-    pka |= (uint64_t)code_a << (i * BITS);
-    pkb |= (uint64_t)code_b << (i * BITS);
-    const float Qa = Ops::value(Ops::template decode<BITS>(code_a, cell_b), step, unbias);
-    const float Qb = Ops::value(Ops::template decode<BITS>(code_b, cell_a), step, unbias);
-    out.v[i] = __fmul_rn(0.5f, __fadd_rn(Qa, Qb));
-  }
+  exchange8<BITS, FAST, ELIDE>(va, vb, ra, rb, sc, out, pka, pkb);
   st256(xa, out);
   st256(xb, out);
   store_codes<BITS>(ca, lane, pka);
@@ -176,10 +204,14 @@ __device__ __forceinline__ void blocking_subblock(const StoreView& s, const Pair
                 j * (kSubCoords * BITS / 8) + lane * BITS;
   uint8_t* cb = s.codes + (int64_t)pd.b * s.nblk * kBlockCoords + blk * (kBlockCoords * BITS / 8) +
                 j * (kSubCoords * BITS / 8) + lane * BITS;
-  const uint4 ra = philox4x32_10(g, (uint32_t)pd.a, pd.wa, kStreamRounding, s.key0, s.key1);
-  const uint4 rb = philox4x32_10(g, (uint32_t)pd.b, pd.wb, kStreamRounding, s.key0, s.key1);
-  if (fast_range(M, pow2f_exact(-e), e)) subblock_exchange<BITS, true>(va, vb, xa, xb, ca, cb, ra, rb, lane, e);
-  else subblock_exchange<BITS, false>(va, vb, xa, xb, ca, cb, ra, rb, lane, e);
+  const uint4 ra = philox4x32_10(g, (uint32_t)pd.a, pd.wa, kStreamRounding, s.rk);
+  const uint4 rb = philox4x32_10(g, (uint32_t)pd.b, pd.wb, kStreamRounding, s.rk);
+  if (fast_range(M, pow2f_exact(-e), e)) {
+    if (decode_elidable<BITS>(rho, e)) subblock_exchange<BITS, true, true>(va, vb, xa, xb, ca, cb, ra, rb, lane, e);
+    else subblock_exchange<BITS, true, false>(va, vb, xa, xb, ca, cb, ra, rb, lane, e);
+  } else {
+    subblock_exchange<BITS, false, false>(va, vb, xa, xb, ca, cb, ra, rb, lane, e);
+  }
   if (j == 0 && lane == 0) {
     s.exps[(int64_t)pd.a * s.nblk + blk] = (int8_t)e;
     s.exps[(int64_t)pd.b * s.nblk + blk] = (int8_t)e;

@@ -5,6 +5,8 @@
 #include <cstdint>
 #include <cuda_runtime.h>
 
+#include "swarm_internal.h"
+
 namespace swarm {
 
 constexpr int kBlockCoords = 1024;   // coordinates sharing one lattice exponent
@@ -39,9 +41,8 @@ __host__ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1
   return make_uint4(c0, c1, c2, c3);
 }
 
-// The ten round keys of a generator key, for kernels that call the generator inside a run-time loop
-// (computed once per thread instead of once per call).
-struct PhiloxRoundKeys { uint32_t k0[10], k1[10]; };
+// The ten round keys of a generator key (struct in swarm_internal.h): the kernels on the hot path take them
+// ready-made from their parameters instead of deriving them in every call.
 __host__ __device__ __forceinline__ PhiloxRoundKeys philox_round_keys(uint32_t k0, uint32_t k1) {
   PhiloxRoundKeys rk;
 #pragma unroll
@@ -167,49 +168,50 @@ __device__ __forceinline__ int32_t encode_index(float x, float inv_step, uint32_
 // ---------------------------------------------------------------------------------------
 // The same lattice arithmetic without conversion instructions. Float<->integer conversions and
 // floorf share one quarter-rate unit, which the 8..18 conversions per coordinate of the interaction
-// kernels keep busier than HBM does. While every scaled value t = x * 2^-e and every lattice index
-// of a block stays inside (-2^22, 2^22), the same results come from full-rate float adds:
-//   s = t + 1.5*2^23 rounded toward -inf is floor(t) + 1.5*2^23 exactly (ulp 1 in [2^23, 2^24)), its bit
-//   pattern is 0x4B400000 + floor(t): a lattice cell "biased" by 0x4B400000. The bias has no low 22
-//   bits, so colours (cell & mask) and the window arithmetic of the decoder work on biased cells
-//   unchanged, and a biased index i turns into the value (i - bias) * 2^e with one exact fused
-//   multiply-add: as_float(i) * 2^e - 1.5*2^23 * 2^e.
-//   The rounding decision u < floor(frac * 2^16) is the same as (u + 1) / 2^16 <= frac, so the index is
-//   floor(t) + floor(z) with z = 1 + frac - (u + 1) / 2^16 in [0, 2): z comes from one fused multiply-add
-//   rounded toward -inf (which cannot cross the integer 1), the uniform enters as a float by splicing its
-//   half word under the exponent byte of 2^23 with one byte permute, and adding z to s, again rounded
-//   toward -inf, lands on s + floor(z). One integer-pipe instruction per encoded coordinate is left.
+// kernels keep busier than HBM does. While the lattice exponent is e <= 0 (then t = x * 2^-e is an exact
+// product, subnormal x included) and every scaled value and lattice index of a block stays inside
+// (-2^21, 2^21), the same results come from full-rate fused multiply-adds and adds with directed rounding:
+//   s = fma(x, 2^-e, C) rounded toward -inf, C an integer in [2^23, 2^24) - 2^21, is floor(t) + C exactly
+//   (ulp 1 in [2^23, 2^24)). With C = 1.5 * 2^23 its bit pattern is 0x4B400000 + floor(t): a lattice cell
+//   "biased" by 0x4B400000. The bias has no low 22 bits, so colours (cell & mask) and the window arithmetic
+//   of the decoder work on biased cells unchanged, and a biased index i turns into the value
+//   (i - bias) * 2^e with one exact fused multiply-add: as_float(i) * 2^e - 1.5*2^23 * 2^e.
+//   Encoder: with C = 1.5 * 2^23 + 192, frac = fma(x, 2^-e, C - s) is RN(t - floor t), the definition's
+//   fraction (it can round up to 1 for a tiny negative t, as there). The 16-bit uniform u becomes the float
+//   um = 192 + u / 2^16 by splicing its half word under the bytes 0x43 0x40 with one byte permute; 192 keeps
+//   um - frac inside [128, 256), where floats are spaced 2^-16, so um - frac rounded toward +inf is
+//   192 + (u - thr) / 2^16 with thr = floor(frac * 2^16), the definition's threshold, and s minus that,
+//   again rounded toward +inf, is floor(t) + 1.5 * 2^23 + [u < thr]: the biased lattice index.
+//   Six instructions, none of them a conversion.
 // LatticeOps<true> is that form (the caller checks the range, warp-uniformly, per block);
 // LatticeOps<false> is the defining form with saturating conversions. Both give bit-identical
 // results wherever the fast form is valid.
 // ---------------------------------------------------------------------------------------
 constexpr float kCellBias = 12582912.0f;            // 1.5 * 2^23
+constexpr uint32_t kCellBiasBits = 0x4B400000u;
+constexpr float kEncBias = 12583104.0f;             // 1.5 * 2^23 + 192: running sum of the encoder
 constexpr float kFastRange = 2097152.0f;            // 2^21: bound on |x| * 2^-e for the fast form (half the
                                                     // exact limit, which leaves room for the decode window)
-constexpr int kFastExpMax = 100;                    // keeps 1.5*2^23 * 2^e finite
 
 template <bool FAST>
 struct LatticeOps {
   // (biased) cell of a key: floor(key * 2^-e)
   static __device__ __forceinline__ uint32_t cell(float key, float inv_step) {
-    const float t = __fmul_rn(key, inv_step);
-    if constexpr (FAST) return __float_as_uint(__fadd_rd(t, kCellBias));
-    else return (uint32_t)__float2int_rd(t);
+    if constexpr (FAST) return __float_as_uint(__fmaf_rd(key, inv_step, kCellBias));
+    else return (uint32_t)__float2int_rd(__fmul_rn(key, inv_step));
   }
   // (biased) lattice index of x after stochastic rounding with half `hi` (0 low, 1 high) of generator
   // word `w`; `cell` receives the (biased) cell of x.
   static __device__ __forceinline__ uint32_t encode(float x, float inv_step, uint32_t w, int hi, uint32_t& cell_out) {
-    const float t = __fmul_rn(x, inv_step);
     if constexpr (FAST) {
-      const float sft = __fadd_rd(t, kCellBias);
-      const float f = __fsub_rn(sft, kCellBias);
-      const float frac = __fsub_rn(t, f);                                              // in [0, 1]
-      const float um = __uint_as_float(__byte_perm(w, 0x4B000000u, hi ? 0x7632 : 0x7610));   // 2^23 + uniform
-      const float un = __fsub_rn(um, 8454143.0f);                                      // uniform - 65535, exact
-      const float z = __fmaf_rd(un, -0x1p-16f, frac);                                  // 1 + frac - (u + 1) / 2^16, rounded down
-      cell_out = __float_as_uint(sft);
-      return __float_as_uint(__fadd_rd(sft, z));                                       // sft + floor(z), floor(z) in {0, 1}
+      const float sft = __fmaf_rd(x, inv_step, kEncBias);                              // floor(t) + kEncBias
+      const float frac = __fmaf_rn(x, inv_step, __fsub_rn(kEncBias, sft));             // RN(t - floor t), in [0, 1]
+      const float um = __uint_as_float(__byte_perm(w, 0x43400000u, hi ? 0x7632 : 0x7610));   // 192 + u / 2^16
+      const float gap = __fsub_ru(um, frac);                                           // 192 + (u - thr) / 2^16
+      cell_out = __float_as_uint(sft) - 192u;
+      return __float_as_uint(__fsub_ru(sft, gap));                                     // floor(t) + bias + [u < thr]
     } else {
+      const float t = __fmul_rn(x, inv_step);
       const float f = floorf(t);
       const float frac = __fsub_rn(t, f);
       const uint32_t thr = __float2uint_rz(__fmul_rn(frac, 65536.0f));
@@ -219,7 +221,7 @@ struct LatticeOps {
     }
   }
   // (biased) index congruent to colour c (mod 2^BITS) in the window [cell - L, cell + L + 1]:
-  // cell - L + ((c - cell + L) mod 2^BITS), L = 2^(BITS-1) - 1.
+  // cell - L + ((c - cell + L) mod 2^BITS), L = 2^(BITS-1) - 1. Bits of c above the colour are ignored.
   template <int BITS>
   static __device__ __forceinline__ uint32_t decode(uint32_t c, uint32_t cell_in) {
     constexpr uint32_t mask = (1u << BITS) - 1u, L = (1u << (BITS - 1)) - 1u;
@@ -234,11 +236,50 @@ struct LatticeOps {
     if constexpr (FAST) return __fmaf_rn(__uint_as_float(idx), step, unbias);
     else return __fmul_rn(__int2float_rn((int32_t)idx), step);
   }
+  // Fast form: half the sum of the values of two biased indices of magnitude <= 2^21 each (an encoder's own
+  // output), (qa + qb) * 2^(e-1). That is what RN(0.5 * RN(Qa + Qb)) comes to, because each product and the sum
+  // are exact and (qa + qb) * 2^(e-1) is a float for every e >= -126 (a subnormal at worst). One integer
+  // add-add (the sum of two biased patterns minus one bias is the biased sum while |qa + qb| <= 2^22) and one
+  // fused multiply-add; `half_step` = 2^(e-1), `half_unbias` = -1.5*2^23 * 2^(e-1).
+  static __device__ __forceinline__ float mean_of_own(uint32_t ia, uint32_t ib, float half_step, float half_unbias) {
+    static_assert(FAST, "biased indices only");
+    return __fmaf_rn(__uint_as_float(ia + ib - kCellBiasBits), half_step, half_unbias);
+  }
 };
 
-// Whether the fast form covers a block: largest magnitude `maxabs` scaled by 2^-e stays below 2^21.
+// Eight colours (the low BITS bits of eight lattice indices, coordinate order) as one little-endian bit
+// stream of 8 * BITS bits. Widths 2, 4 and 8 merge neighbours with shift-and-select steps that leave
+// garbage above each partial byte and drop it with byte permutes.
+template <int BITS>
+__device__ __forceinline__ uint64_t pack_colours(const uint32_t (&q)[8]) {
+  if constexpr (BITS == 8) {
+    const uint32_t lo = __byte_perm(__byte_perm(q[0], q[1], 0x0040), __byte_perm(q[2], q[3], 0x0040), 0x5410);
+    const uint32_t hi = __byte_perm(__byte_perm(q[4], q[5], 0x0040), __byte_perm(q[6], q[7], 0x0040), 0x5410);
+    return (uint64_t)lo | ((uint64_t)hi << 32);
+  } else if constexpr (BITS == 4) {
+    uint32_t b[4];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) b[t] = (q[2 * t] & 0xFu) | (q[2 * t + 1] << 4);         // byte t (garbage above bit 7)
+    return __byte_perm(__byte_perm(b[0], b[1], 0x0040), __byte_perm(b[2], b[3], 0x0040), 0x5410);
+  } else if constexpr (BITS == 2) {
+    uint32_t n[4];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) n[t] = (q[2 * t] & 0x3u) | (q[2 * t + 1] << 2);         // nibble t (garbage above bit 3)
+    const uint32_t b0 = (n[0] & 0xFu) | (n[1] << 4), b1 = (n[2] & 0xFu) | (n[3] << 4);
+    return __byte_perm(b0, b1, 0x0040) & 0xFFFFu;
+  } else {
+    constexpr uint32_t mask = (1u << BITS) - 1u;
+    uint64_t pk = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) pk |= (uint64_t)(q[i] & mask) << (i * BITS);
+    return pk;
+  }
+}
+
+// Whether the fast form covers a block: e <= 0 (exact scaling) and the largest magnitude `maxabs` scaled by
+// 2^-e stays below 2^21.
 __device__ __forceinline__ bool fast_range(float maxabs, float inv_step, int e) {
-  return __fmul_rn(maxabs, inv_step) < kFastRange && e <= kFastExpMax;
+  return __fmul_rn(maxabs, inv_step) < kFastRange && e <= 0;
 }
 
 // Generator word holding the 16-bit rounding uniform of coordinate i (0..7) of a call covering 8

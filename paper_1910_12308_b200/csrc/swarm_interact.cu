@@ -27,6 +27,18 @@ __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefe
 constexpr int64_t kPrefetchDistance = 444;            // warps ahead; swept 148..2368 on B200 (best 300..600)
 constexpr int64_t kPrefetchDistanceRegisters = 296;   // the register-protocol kernel keeps fewer warps resident
 
+// The (pair, block) that the warp `ahead` warp indices after this one works on; false past the end of the
+// launch. A launch has fewer than 2^31 warps (checked by the launch wrappers), for which the multiplier and
+// shift in the store view give the exact quotient by the number of blocks per row.
+__device__ __forceinline__ bool warp_slot(int64_t total_warps, const StoreView& s, uint32_t ahead, uint32_t& pair,
+                                          uint32_t& blk) {
+  const uint32_t warp = blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5) + ahead;
+  if (warp >= (uint32_t)total_warps) return false;
+  pair = s.nblk_magic ? __umulhi(warp, s.nblk_magic) >> s.nblk_shift : warp;
+  blk = warp - pair * (uint32_t)s.nblk;
+  return true;
+}
+
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_dependency_signal() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 // -----------------------------------------------------------------------------------------
@@ -41,15 +53,14 @@ interact_blocking_kernel(StoreView s, const PairList pairs, int64_t total_warps,
   grid_dependency_signal();
   grid_dependency_wait();
   const int lane = threadIdx.x & 31;
-  const int64_t warp = (int64_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
-  if (warp >= total_warps) return;
-  const int64_t pair = warp / s.nblk;
-  const int64_t blk = warp - pair * s.nblk;
+  uint32_t pair, blk32;
+  if (!warp_slot(total_warps, s, 0, pair, blk32)) return;
+  const int64_t blk = blk32;
   const PairDesc pd = pairs.get(pair);
   {
-    const int64_t w2 = warp + kPrefetchDistance;
-    if (w2 < total_warps) {
-      const int64_t pair2 = w2 / s.nblk, blk2 = w2 - pair2 * s.nblk;
+    uint32_t pair2, blk2_32;
+    if (warp_slot(total_warps, s, (uint32_t)kPrefetchDistance, pair2, blk2_32)) {
+      const int64_t blk2 = blk2_32;
       const PairDesc p2 = pairs.get(pair2);
       prefetch_l2(s.X + (int64_t)p2.a * s.pitch + blk2 * kBlockCoords + lane * 32);     // 32 lines of 128 B
       prefetch_l2(s.X + (int64_t)p2.b * s.pitch + blk2 * kBlockCoords + lane * 32);
@@ -65,15 +76,14 @@ interact_identity_kernel(StoreView s, const PairList pairs, int64_t total_warps,
   grid_dependency_signal();
   grid_dependency_wait();
   const int lane = threadIdx.x & 31;
-  const int64_t warp = (int64_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
-  if (warp >= total_warps) return;
-  const int64_t pair = warp / s.nblk;
-  const int64_t blk = warp - pair * s.nblk;
+  uint32_t pair, blk32;
+  if (!warp_slot(total_warps, s, 0, pair, blk32)) return;
+  const int64_t blk = blk32;
   const PairDesc pd = pairs.get(pair);
   {
-    const int64_t w2 = warp + kPrefetchDistance;
-    if (w2 < total_warps) {
-      const int64_t pair2 = w2 / s.nblk, blk2 = w2 - pair2 * s.nblk;
+    uint32_t pair2, blk2_32;
+    if (warp_slot(total_warps, s, (uint32_t)kPrefetchDistance, pair2, blk2_32)) {
+      const int64_t blk2 = blk2_32;
       const PairDesc p2 = pairs.get(pair2);
       prefetch_l2(s.X + (int64_t)p2.a * s.pitch + blk2 * kBlockCoords + lane * 32);
       prefetch_l2(s.X + (int64_t)p2.b * s.pitch + blk2 * kBlockCoords + lane * 32);
@@ -111,14 +121,14 @@ __device__ __forceinline__ void nonblocking_decode(f8 (&nx)[kSub], f8 (&av)[kSub
   const float step_oth = pow2f_exact(e_oth), inv_oth = pow2f_exact(-e_oth);
   const float unb_own = FAST ? -__fmul_rn(kCellBias, step_own) : 0.0f;
   const float unb_oth = FAST ? -__fmul_rn(kCellBias, step_oth) : 0.0f;
-  constexpr uint32_t mask = (1u << BITS) - 1u;
   float spread = 0.0f, dmax = 0.0f, M = 0.0f;
 #pragma unroll
   for (int j = 0; j < kSub; ++j)
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const float key = av[j].v[i];
-      const uint32_t code_own = (uint32_t)(pa[j] >> (i * BITS)) & mask, code_oth = (uint32_t)(pb[j] >> (i * BITS)) & mask;
+      // colours with whatever follows them in the stream above: the decoder reads the low BITS bits only
+      const uint32_t code_own = (uint32_t)(pa[j] >> (i * BITS)), code_oth = (uint32_t)(pb[j] >> (i * BITS));
       const float own = Ops::value(Ops::template decode<BITS>(code_own, Ops::cell(key, inv_own)), step_own, unb_own);
       const float oth = Ops::value(Ops::template decode<BITS>(code_oth, Ops::cell(key, inv_oth)), step_oth, unb_oth);
       const float avg = __fmul_rn(0.5f, __fadd_rn(own, oth));
@@ -142,23 +152,22 @@ __device__ __forceinline__ void nonblocking_encode(const f8 (&nx)[kSub], const f
                                                    const PairDesc& pd, int lane, int e) {
   using Ops = LatticeOps<FAST>;
   const float inv_step = pow2f_exact(-e);
-  constexpr uint32_t mask = (1u << BITS) - 1u;
 #pragma unroll
   for (int j = 0; j < kSub; ++j) {
     const uint32_t g = group0 + j * (kSubCoords / 8);
-    const uint4 ra = philox4x32_10(g, (uint32_t)pd.a, pd.wa, kStreamRounding, s.key0, s.key1);
-    const uint4 rb = philox4x32_10(g, (uint32_t)pd.b, pd.wb, kStreamRounding, s.key0, s.key1);
-    uint64_t pka = 0, pkb = 0;
+    const uint4 ra = philox4x32_10(g, (uint32_t)pd.a, pd.wa, kStreamRounding, s.rk);
+    const uint4 rb = philox4x32_10(g, (uint32_t)pd.b, pd.wb, kStreamRounding, s.rk);
+    uint32_t qa[8], qb[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       uint32_t cell;
-      pka |= (uint64_t)(Ops::encode(nx[j].v[i], inv_step, sr_word(ra, i), i & 1, cell) & mask) << (i * BITS);
-      pkb |= (uint64_t)(Ops::encode(av[j].v[i], inv_step, sr_word(rb, i), i & 1, cell) & mask) << (i * BITS);
+      qa[i] = Ops::encode(nx[j].v[i], inv_step, sr_word(ra, i), i & 1, cell);
+      qb[i] = Ops::encode(av[j].v[i], inv_step, sr_word(rb, i), i & 1, cell);
     }
     st256(xa + j * kSubCoords, nx[j]);
     st256(ba + j * kSubCoords, nx[j]);
-    store_codes<BITS>(ca + j * (kSubCoords * BITS / 8), lane, pka);
-    store_codes<BITS>(cb + j * (kSubCoords * BITS / 8), lane, pkb);
+    store_codes<BITS>(ca + j * (kSubCoords * BITS / 8), lane, pack_colours<BITS>(qa));
+    store_codes<BITS>(cb + j * (kSubCoords * BITS / 8), lane, pack_colours<BITS>(qb));
   }
 }
 
@@ -177,15 +186,14 @@ interact_nonblocking_kernel(StoreView s, const PairList pairs, int64_t total_war
   grid_dependency_signal();
   grid_dependency_wait();
   const int lane = threadIdx.x & 31;
-  const int64_t warp = (int64_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
-  if (warp >= total_warps) return;
-  const int64_t pair = warp / s.nblk;
-  const int64_t blk = warp - pair * s.nblk;
+  uint32_t pair, blk32;
+  if (!warp_slot(total_warps, s, 0, pair, blk32)) return;
+  const int64_t blk = blk32;
   const PairDesc pd = pairs.get(pair);
   {
-    const int64_t w2 = warp + kPrefetchDistance;
-    if (w2 < total_warps) {
-      const int64_t pair2 = w2 / s.nblk, blk2 = w2 - pair2 * s.nblk;
+    uint32_t pair2, blk2_32;
+    if (warp_slot(total_warps, s, (uint32_t)kPrefetchDistance, pair2, blk2_32)) {
+      const int64_t blk2 = blk2_32;
       const PairDesc p2 = pairs.get(pair2);
       prefetch_l2(s.X + (int64_t)p2.a * s.pitch + blk2 * kBlockCoords + lane * 32);     // 32 lines of 128 B
       prefetch_l2(s.B + (int64_t)p2.a * s.pitch + blk2 * kBlockCoords + lane * 32);
@@ -302,7 +310,7 @@ publish_encode_kernel(StoreView s, const uint32_t* __restrict__ wctr, int64_t to
   for (int j = 0; j < kSub; ++j) v[j] = ld256(row + j * kSubCoords);
 #pragma unroll
   for (int j = 0; j < kSub; ++j) {
-    const uint4 r = philox4x32_10(group0 + j * (kSubCoords / 8), (uint32_t)node, w, kStreamRounding, s.key0, s.key1);
+    const uint4 r = philox4x32_10(group0 + j * (kSubCoords / 8), (uint32_t)node, w, kStreamRounding, s.rk);
     uint64_t pk = 0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -333,8 +341,14 @@ constexpr int kOwnResolutionBits = 8;
 // bytes of the 16-bit colours), so that a reader which needs only the 8-bit prefix touches the first
 // plane alone. A lane's 8 coordinates of a sub-block are 8 consecutive bytes in each plane.
 constexpr int kOwnBlockBytes = 2 * kBlockCoords;
+// Byte i of a lane's 8 plane bytes in the low byte of the result; whatever follows it stays above (decoders read
+// the low bits they need).
 __device__ __forceinline__ uint32_t plane_byte(const uint2& v, int i) {
-  return (((i < 4) ? v.x : v.y) >> ((i & 3) * 8)) & 0xFFu;
+  return ((i < 4) ? v.x : v.y) >> ((i & 3) * 8);
+}
+// 16-bit colour i from the low-byte and high-byte planes in the low half of the result (upper half: garbage).
+__device__ __forceinline__ uint32_t plane_colour16(const uint2& lo, const uint2& hi, int i) {
+  return __byte_perm((i < 4) ? lo.x : lo.y, (i < 4) ? hi.x : hi.y, (i & 3) | ((4 + (i & 3)) << 4));
 }
 // Split eight 16-bit colours (two per word) into their low-byte and high-byte planes.
 __device__ __forceinline__ void split_planes(const uint32_t (&ow)[4], uint2& lo, uint2& hi) {
@@ -343,20 +357,21 @@ __device__ __forceinline__ void split_planes(const uint32_t (&ow)[4], uint2& lo,
 }
 
 // Decode chain of a two-register block. On entry nx = X^a, av = snapshot B^a; on return nx = new model,
-// av = average. Returns the warp-reduced block maxima for the exponents of the three writes.
+// av = average. Returns the warp-reduced block maxima for the exponents of the three writes. The magnitude
+// bounds max(|new model|, |average|) and max(|average|, |Q(X^_b)|) are put together after the reduction from the
+// maxima of the three vectors (max is exact, so the grouping does not matter): one max per vector and coordinate.
 template <int BITS, bool FAST>
 __device__ __forceinline__ void registers_decode(f8 (&nx)[kSub], f8 (&av)[kSub], const uint2 (&va)[kSub],
                                                  const uint2 (&vb)[kSub], const uint2 (&vbh)[kSub],
                                                  const uint64_t (&pa)[kSub], const uint64_t (&pb)[kSub], int prefix,
                                                  int eoa, int eob, int epa, int epb, float& spread_out, float& dmax_out,
-                                                 float& M_out, float& rho_b_out, float& M_b_out) {
+                                                 float& M_out, float& rho_b_out, float& M_b_out, float& m_new_out) {
   using Ops = LatticeOps<FAST>;
   const float so_a = pow2f_exact(eoa), io_a = pow2f_exact(-eoa), so_b = pow2f_exact(eob), io_b = pow2f_exact(-eob);
   const float sp_a = pow2f_exact(epa), ip_a = pow2f_exact(-epa), sp_b = pow2f_exact(epb), ip_b = pow2f_exact(-epb);
   const float uo_a = FAST ? -__fmul_rn(kCellBias, so_a) : 0.0f, uo_b = FAST ? -__fmul_rn(kCellBias, so_b) : 0.0f;
   const float up_a = FAST ? -__fmul_rn(kCellBias, sp_a) : 0.0f, up_b = FAST ? -__fmul_rn(kCellBias, sp_b) : 0.0f;
-  constexpr uint32_t mask = (1u << BITS) - 1u;
-  float spread = 0.0f, dmax = 0.0f, M = 0.0f, rho_b = 0.0f, M_b = 0.0f;
+  float spread = 0.0f, dmax = 0.0f, rho_b = 0.0f, m_new = 0.0f, m_avg = 0.0f, m_qb = 0.0f;
 #pragma unroll
   for (int j = 0; j < kSub; ++j)
 #pragma unroll
@@ -364,26 +379,29 @@ __device__ __forceinline__ void registers_decode(f8 (&nx)[kSub], f8 (&av)[kSub],
       const float snap = av[j].v[i];
       // own key: less than one step away, the 8-bit prefix always suffices
       const float qhat_a = Ops::value(Ops::template decode<8>(plane_byte(va[j], i), Ops::cell(snap, io_a)), so_a, uo_a);
-      const float Qa = Ops::value(Ops::template decode<BITS>((uint32_t)(pa[j] >> (i * BITS)) & mask, Ops::cell(qhat_a, ip_a)), sp_a, up_a);
-      const float qhat_b = Ops::value(Ops::decode_bits(plane_byte(vb[j], i) | (plane_byte(vbh[j], i) << 8),
-                                                       Ops::cell(snap, io_b), prefix), so_b, uo_b);
-      const float Qb = Ops::value(Ops::template decode<BITS>((uint32_t)(pb[j] >> (i * BITS)) & mask, Ops::cell(qhat_b, ip_b)), sp_b, up_b);
+      const float Qa = Ops::value(Ops::template decode<BITS>((uint32_t)(pa[j] >> (i * BITS)), Ops::cell(qhat_a, ip_a)), sp_a, up_a);
+      const float qhat_b = Ops::value(Ops::decode_bits(plane_colour16(vb[j], vbh[j], i), Ops::cell(snap, io_b), prefix), so_b, uo_b);
+      const float Qb = Ops::value(Ops::template decode<BITS>((uint32_t)(pb[j] >> (i * BITS)), Ops::cell(qhat_b, ip_b)), sp_b, up_b);
       const float avg = __fmul_rn(0.5f, __fadd_rn(Qa, Qb));
       const float D = __fsub_rn(snap, nx[j].v[i]);
       const float x_new = __fsub_rn(avg, D);
       spread = fmaxf(spread, fabsf(__fsub_rn(Qa, Qb)));
       dmax = fmaxf(dmax, fabsf(D));
-      M = fmaxf(M, fmaxf(fabsf(x_new), fabsf(avg)));
+      m_new = fmaxf(m_new, fabsf(x_new));
+      m_avg = fmaxf(m_avg, fabsf(avg));
+      m_qb = fmaxf(m_qb, fabsf(qhat_b));
       rho_b = fmaxf(rho_b, fabsf(__fsub_rn(avg, qhat_b)));        // distance of the average to b's decoding key
-      M_b = fmaxf(M_b, fmaxf(fabsf(avg), fabsf(qhat_b)));
       nx[j].v[i] = x_new;
       av[j].v[i] = avg;
     }
   spread_out = warp_max_nonneg(spread);
   dmax_out = warp_max_nonneg(dmax);
-  M_out = warp_max_nonneg(M);
   rho_b_out = warp_max_nonneg(rho_b);
-  M_b_out = warp_max_nonneg(M_b);
+  m_new = warp_max_nonneg(m_new);
+  m_avg = warp_max_nonneg(m_avg);
+  M_out = fmaxf(m_new, m_avg);
+  M_b_out = fmaxf(m_avg, warp_max_nonneg(m_qb));
+  m_new_out = m_new;
 }
 
 // Writes a's own register (16-bit colours of the new model, two byte planes) and b's current register
@@ -391,37 +409,37 @@ __device__ __forceinline__ void registers_decode(f8 (&nx)[kSub], f8 (&av)[kSub],
 template <int BITS, bool FAST>
 __device__ __forceinline__ void registers_encode_own(const f8 (&nx)[kSub], const f8 (&av)[kSub], uint8_t* oa, uint8_t* cb,
                                                      uint32_t group0, const StoreView& s, const PairDesc& pd, int lane,
-                                                     int eo, int ep_b, float& rho_a_out, float& M_a_out) {
+                                                     int eo, int ep_b, float m_new, float& rho_a_out, float& M_a_out) {
   using Ops = LatticeOps<FAST>;
   const float so = pow2f_exact(eo), io = pow2f_exact(-eo), ipb_new = pow2f_exact(-ep_b);
   const float uo = FAST ? -__fmul_rn(kCellBias, so) : 0.0f;
-  constexpr uint32_t mask = (1u << BITS) - 1u;
-  float rho_a = 0.0f, M_a = 0.0f;
+  float rho_a = 0.0f, m_q = 0.0f;    // m_new: the block maximum of |new model|, known from the decode phase
 #pragma unroll
   for (int j = 0; j < kSub; ++j) {
     const uint32_t g = group0 + j * (kSubCoords / 8);
-    const uint4 ro = philox4x32_10(g, (uint32_t)pd.a, pd.woa, kStreamOwnRounding, s.key0, s.key1);
-    const uint4 rb = philox4x32_10(g, (uint32_t)pd.b, pd.wb, kStreamRounding, s.key0, s.key1);
-    uint32_t ow[4] = {0u, 0u, 0u, 0u};
-    uint64_t pkb = 0;
+    const uint4 ro = philox4x32_10(g, (uint32_t)pd.a, pd.woa, kStreamOwnRounding, s.rk);
+    const uint4 rb = philox4x32_10(g, (uint32_t)pd.b, pd.wb, kStreamRounding, s.rk);
+    uint32_t qo[8], qb[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       uint32_t cell;
-      const uint32_t q = Ops::encode(nx[j].v[i], io, sr_word(ro, i), i & 1, cell);
-      ow[i >> 1] |= (q & 0xFFFFu) << ((i & 1) * 16);
-      const float qhat_new = Ops::value(q, so, uo);
+      qo[i] = Ops::encode(nx[j].v[i], io, sr_word(ro, i), i & 1, cell);
+      const float qhat_new = Ops::value(qo[i], so, uo);
       rho_a = fmaxf(rho_a, fabsf(__fsub_rn(nx[j].v[i], qhat_new)));
-      M_a = fmaxf(M_a, fmaxf(fabsf(nx[j].v[i]), fabsf(qhat_new)));
-      pkb |= (uint64_t)(Ops::encode(av[j].v[i], ipb_new, sr_word(rb, i), i & 1, cell) & mask) << (i * BITS);
+      m_q = fmaxf(m_q, fabsf(qhat_new));
+      qb[i] = Ops::encode(av[j].v[i], ipb_new, sr_word(rb, i), i & 1, cell);
     }
+    uint32_t ow[4];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) ow[t] = __byte_perm(qo[2 * t], qo[2 * t + 1], 0x5410);   // two 16-bit colours per word
     uint2 lo, hi;
     split_planes(ow, lo, hi);
     *reinterpret_cast<uint2*>(oa + j * kSubCoords) = lo;
     *reinterpret_cast<uint2*>(oa + kBlockCoords + j * kSubCoords) = hi;
-    store_codes<BITS>(cb + j * (kSubCoords * BITS / 8), lane, pkb);
+    store_codes<BITS>(cb + j * (kSubCoords * BITS / 8), lane, pack_colours<BITS>(qb));
   }
   rho_a_out = warp_max_nonneg(rho_a);
-  M_a_out = warp_max_nonneg(M_a);
+  M_a_out = fmaxf(m_new, warp_max_nonneg(m_q));
 }
 
 // Writes the new model to X^a and B^a and its b-bit colours to a's current register.
@@ -431,20 +449,19 @@ __device__ __forceinline__ void registers_encode_current(const f8 (&nx)[kSub], f
                                                          int lane, int ep_a) {
   using Ops = LatticeOps<FAST>;
   const float ipa_new = pow2f_exact(-ep_a);
-  constexpr uint32_t mask = (1u << BITS) - 1u;
 #pragma unroll
   for (int j = 0; j < kSub; ++j) {
     const uint32_t g = group0 + j * (kSubCoords / 8);
-    const uint4 ra = philox4x32_10(g, (uint32_t)pd.a, pd.wa, kStreamRounding, s.key0, s.key1);
-    uint64_t pka = 0;
+    const uint4 ra = philox4x32_10(g, (uint32_t)pd.a, pd.wa, kStreamRounding, s.rk);
+    uint32_t qa[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       uint32_t cell;
-      pka |= (uint64_t)(Ops::encode(nx[j].v[i], ipa_new, sr_word(ra, i), i & 1, cell) & mask) << (i * BITS);
+      qa[i] = Ops::encode(nx[j].v[i], ipa_new, sr_word(ra, i), i & 1, cell);
     }
     st256(xa + j * kSubCoords, nx[j]);
     st256(ba + j * kSubCoords, nx[j]);
-    store_codes<BITS>(ca + j * (kSubCoords * BITS / 8), lane, pka);
+    store_codes<BITS>(ca + j * (kSubCoords * BITS / 8), lane, pack_colours<BITS>(qa));
   }
 }
 
@@ -454,23 +471,22 @@ interact_registers_kernel(StoreView s, const PairList pairs, int64_t total_warps
   grid_dependency_signal();
   grid_dependency_wait();
   const int lane = threadIdx.x & 31;
-  const int64_t warp = (int64_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
-  if (warp >= total_warps) return;
-  const int64_t pair = warp / s.nblk;
-  const int64_t blk = warp - pair * s.nblk;
+  uint32_t pair, blk32;
+  if (!warp_slot(total_warps, s, 0, pair, blk32)) return;
+  const int64_t blk = blk32;
   const PairDesc pd = pairs.get(pair);
 
   {
-    const int64_t w2 = warp + kPrefetchDistanceRegisters;
-    if (w2 < total_warps) {
-      const int64_t pair2 = w2 / s.nblk, blk2 = w2 - pair2 * s.nblk;
+    uint32_t pair2, blk2_32;
+    if (warp_slot(total_warps, s, (uint32_t)kPrefetchDistanceRegisters, pair2, blk2_32)) {
+      const int64_t blk2 = blk2_32;
       const PairDesc p2 = pairs.get(pair2);
       const int64_t k2 = blk2 * kBlockCoords;
       prefetch_l2(s.X + (int64_t)p2.a * s.pitch + k2 + lane * 32);                      // 32 lines of 128 B
       prefetch_l2(s.B + (int64_t)p2.a * s.pitch + k2 + lane * 32);
       if (lane < 8)                                                                      // a's low-byte plane (1 KiB)
         prefetch_l2(s.own + ((int64_t)p2.a * s.nblk + blk2) * kOwnBlockBytes + lane * 128);
-      if (lane < s.own_prefix)                                                           // b's plane(s): 8 or 16 lines
+      if (lane < (int)p2.prefix)                                                         // b's plane(s): 8 or 16 lines
         prefetch_l2(s.own + ((int64_t)p2.b * s.nblk + blk2) * kOwnBlockBytes + lane * 128);
       if (lane < BITS) {
         prefetch_l2(s.codes + (int64_t)p2.a * s.nblk * kBlockCoords + blk2 * (kBlockCoords * BITS / 8) + lane * 128);
@@ -483,7 +499,7 @@ interact_registers_kernel(StoreView s, const PairList pairs, int64_t total_warps
   float* ba = s.B + (int64_t)pd.a * s.pitch + koff;
   uint8_t* oa = s.own + ((int64_t)pd.a * s.nblk + blk) * kOwnBlockBytes + lane * 8;       // low plane; high at +1024
   const uint8_t* ob = s.own + ((int64_t)pd.b * s.nblk + blk) * kOwnBlockBytes + lane * 8;
-  const int prefix = s.own_prefix;
+  const int prefix = (int)pd.prefix;      // the reader's statement about its distance to b's snapshot
   uint8_t* ca = s.codes + (int64_t)pd.a * s.nblk * kBlockCoords + blk * (kBlockCoords * BITS / 8) + lane * BITS;
   uint8_t* cb = s.codes + (int64_t)pd.b * s.nblk * kBlockCoords + blk * (kBlockCoords * BITS / 8) + lane * BITS;
 
@@ -521,9 +537,9 @@ interact_registers_kernel(StoreView s, const PairList pairs, int64_t total_warps
   const float qb_max = __fmaf_rn(prefix == 16 ? 32770.0f : 130.0f, pow2f_exact(eob), kmax);
   const bool fast_chain = fast_range(kmax, pow2f_exact(-eoa), eoa) && fast_range(kmax, pow2f_exact(-eob), eob) &&
                           fast_range(qa_max, pow2f_exact(-epa), epa) && fast_range(qb_max, pow2f_exact(-epb), epb);
-  float spread, dmax, M, rho_b, M_b;
-  if (fast_chain) registers_decode<BITS, true>(nx, av, va, vb, vbh, pa, pb, prefix, eoa, eob, epa, epb, spread, dmax, M, rho_b, M_b);
-  else registers_decode<BITS, false>(nx, av, va, vb, vbh, pa, pb, prefix, eoa, eob, epa, epb, spread, dmax, M, rho_b, M_b);
+  float spread, dmax, M, rho_b, M_b, m_new;
+  if (fast_chain) registers_decode<BITS, true>(nx, av, va, vb, vbh, pa, pb, prefix, eoa, eob, epa, epb, spread, dmax, M, rho_b, M_b, m_new);
+  else registers_decode<BITS, false>(nx, av, va, vb, vbh, pa, pb, prefix, eoa, eob, epa, epb, spread, dmax, M, rho_b, M_b, m_new);
   const int eo = exponent_rule<kOwnResolutionBits>(__fadd_rn(__fmul_rn(2.0f, spread), dmax), M);
   const int ep_b = exponent_rule<BITS>(rho_b, M_b);
 
@@ -531,9 +547,9 @@ interact_registers_kernel(StoreView s, const PairList pairs, int64_t total_warps
   const uint32_t group0 = (uint32_t)(blk * (kBlockCoords / 8) + lane);
   float rho_a, M_a;
   if (fast_range(M, pow2f_exact(-eo), eo) && fast_range(M_b, pow2f_exact(-ep_b), ep_b))
-    registers_encode_own<BITS, true>(nx, av, oa, cb, group0, s, pd, lane, eo, ep_b, rho_a, M_a);
+    registers_encode_own<BITS, true>(nx, av, oa, cb, group0, s, pd, lane, eo, ep_b, m_new, rho_a, M_a);
   else
-    registers_encode_own<BITS, false>(nx, av, oa, cb, group0, s, pd, lane, eo, ep_b, rho_a, M_a);
+    registers_encode_own<BITS, false>(nx, av, oa, cb, group0, s, pd, lane, eo, ep_b, m_new, rho_a, M_a);
   const int ep_a = exponent_rule<BITS>(rho_a, M_a);
   if (fast_range(M_a, pow2f_exact(-ep_a), ep_a)) registers_encode_current<BITS, true>(nx, xa, ba, ca, group0, s, pd, lane, ep_a);
   else registers_encode_current<BITS, false>(nx, xa, ba, ca, group0, s, pd, lane, ep_a);
@@ -569,7 +585,7 @@ register_publish_encode_kernel(StoreView s, const uint32_t* __restrict__ wctr, i
   float rho = 0.0f, M = 0.0f;
 #pragma unroll
   for (int j = 0; j < kSub; ++j) {
-    const uint4 ro = philox4x32_10(group0 + j * (kSubCoords / 8), (uint32_t)node, wo, kStreamOwnRounding, s.key0, s.key1);
+    const uint4 ro = philox4x32_10(group0 + j * (kSubCoords / 8), (uint32_t)node, wo, kStreamOwnRounding, s.rk);
     uint32_t ow[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -591,7 +607,7 @@ register_publish_encode_kernel(StoreView s, const uint32_t* __restrict__ wctr, i
   const float ip = pow2f_exact(-ep);
 #pragma unroll
   for (int j = 0; j < kSub; ++j) {
-    const uint4 r = philox4x32_10(group0 + j * (kSubCoords / 8), (uint32_t)node, w, kStreamRounding, s.key0, s.key1);
+    const uint4 r = philox4x32_10(group0 + j * (kSubCoords / 8), (uint32_t)node, w, kStreamRounding, s.rk);
     uint64_t pk = 0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -607,6 +623,7 @@ register_publish_encode_kernel(StoreView s, const uint32_t* __restrict__ wctr, i
 // Launch wrappers
 // -----------------------------------------------------------------------------------------
 static inline unsigned ctas_for(int64_t warps) { return (unsigned)((warps + kWarpsPerCta - 1) / kWarpsPerCta); }
+constexpr int64_t kMaxLaunchWarps = (int64_t)1 << 31;   // the kernels index warps, and the warp a prefetch looks at, in 32 bits
 
 // Code widths with a compiled kernel: SWARM_FOR_WIDTH(bits, BODY) runs BODY with the constant W = bits.
 #define SWARM_WIDTH_CASE(w, ...) case w: { constexpr int W = w; __VA_ARGS__; } break;
@@ -638,6 +655,7 @@ cudaError_t launch_interact_blocking(const StoreView& s, const PairList& pairs, 
                                      const FusedSteps& fs, cudaStream_t st, int* launches) {
   if (npairs == 0) return cudaSuccess;
   const int64_t warps = (int64_t)npairs * s.nblk;
+  if (warps + kPrefetchDistance >= kMaxLaunchWarps) return cudaErrorInvalidValue;
   const dim3 grid(ctas_for(warps)), block(kWarpsPerCta * 32);
   cudaError_t e = cudaSuccess;
   if (bits == 32) {
@@ -654,6 +672,7 @@ cudaError_t launch_interact_nonblocking(const StoreView& s, const PairList& pair
                                         const FusedSteps& fs, cudaStream_t st, int* launches) {
   if (npairs == 0) return cudaSuccess;
   const int64_t warps = (int64_t)npairs * s.nblk;
+  if (warps + kPrefetchDistance >= kMaxLaunchWarps) return cudaErrorInvalidValue;
   const dim3 grid(ctas_for(warps)), block(kWarpsPerCta * 32);
   cudaError_t e = cudaSuccess;
   SWARM_FOR_WIDTH(bits, e = (fs.H > 0 ? launch_dependent(interact_nonblocking_kernel<W, true>, grid, block, st, s, pairs, warps, fs)
@@ -677,6 +696,7 @@ cudaError_t launch_interact_registers(const StoreView& s, const PairList& pairs,
                                       const FusedSteps& fs, cudaStream_t st, int* launches) {
   if (npairs == 0) return cudaSuccess;
   const int64_t warps = (int64_t)npairs * s.nblk;
+  if (warps + kPrefetchDistance >= kMaxLaunchWarps) return cudaErrorInvalidValue;
   const dim3 grid(ctas_for(warps)), block(kWarpsPerCta * 32);
   cudaError_t e = cudaSuccess;
   SWARM_FOR_WIDTH(bits, e = (fs.H > 0 ? launch_dependent(interact_registers_kernel<W, true>, grid, block, st, s, pairs, warps, fs)

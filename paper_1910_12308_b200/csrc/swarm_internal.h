@@ -13,7 +13,7 @@ struct PairDesc {
   uint32_t wa, wb;     // write counters of the two buffers before this interaction
   uint32_t woa;        // write counter of the initiator's own register (two-register protocol)
   uint32_t lsa, lsb;   // local-step counters of the two nodes (steps fused into the interaction)
-  uint32_t pad;
+  uint32_t prefix;     // two-register protocol: bits (8 or 16) of the responder's own register that the initiator reads
 };
 
 // Synthetic-gradient local steps taken inside an interaction kernel before the exchange (H = 0: none).
@@ -61,6 +61,10 @@ struct LsqUnit {
   int32_t pad;
 };
 
+// The ten round keys of the generator key (round r uses key + r * Weyl constant): computed once on the host and
+// carried in the kernel parameters, where the generator reads them as constants.
+struct PhiloxRoundKeys { uint32_t k0[10], k1[10]; };
+
 struct StoreView {
   float* X;            // [n][pitch]
   float* B;            // [n][pitch] or nullptr
@@ -74,8 +78,22 @@ struct StoreView {
   int64_t nblk;
   int32_t n;
   uint32_t key0, key1; // generator key (seed low / high word)
-  int32_t own_prefix;  // bits of a partner's own register that a reader consumes: 8 or 16
+  PhiloxRoundKeys rk;  // its round keys
+  // warp index -> (pair, block) without a division: for w < 2^31, w / nblk = umulhi(w, nblk_magic) >> nblk_shift
+  // (nblk_magic = 0: nblk is 1 and the quotient is w itself)
+  uint32_t nblk_magic, nblk_shift;
 };
+
+// Multiplier and shift with floor(w / divisor) = umulhi(w, magic) >> shift for every w < 2^31 (divisor >= 2):
+// with L = ceil(log2 divisor) and magic = floor(2^(31 + L) / divisor) + 1 the product w * magic / 2^(31 + L) exceeds
+// w / divisor by less than 2^-L <= 1 / divisor, which cannot reach the next integer.
+inline void division_magic(uint64_t divisor, uint32_t* magic, uint32_t* shift) {
+  if (divisor < 2) { *magic = 0; *shift = 0; return; }
+  uint32_t L = 0;
+  while (((uint64_t)1 << L) < divisor) ++L;
+  *magic = (uint32_t)((((uint64_t)1 << (31 + L)) / divisor) + 1);
+  *shift = L - 1;
+}
 
 struct LsqView {
   const void* A;       // [groups][m][pitch] fp32 or bf16

@@ -116,9 +116,8 @@ local_synth_kernel(StoreView s, const NodeList nodes, int H, float lr, float gra
   const float c = scalars[nd.node * 3 + 1];
   float* p = s.X + (int64_t)nd.node * s.pitch + g8 * 8;
   f8 v = ld256(p);
-  const PhiloxRoundKeys rk = philox_round_keys(s.key0, s.key1);
   for (int q = 0; q < H; ++q)
-    synth_step8(v, (uint32_t)g8, (uint32_t)nd.node, nd.event + (uint32_t)q, lr, grad_std, c, rk);
+    synth_step8(v, (uint32_t)g8, (uint32_t)nd.node, nd.event + (uint32_t)q, lr, grad_std, c, s.rk);
   if (g8 * 8 + 8 > s.d) {                                    // keep the row padding zero
 #pragma unroll
     for (int t = 0; t < 8; ++t) if (g8 * 8 + t >= s.d) v.v[t] = 0.0f;

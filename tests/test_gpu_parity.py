@@ -325,6 +325,62 @@ def test_register_protocol_with_8_bit_prefix_reads(bits):
     assert gpu.get_own_prefix() == 16
 
 
+@pytest.mark.parametrize("bits", [2, 5, 8])
+def test_register_protocol_with_a_prefix_per_reader(bits):
+    """Launches that mix 8-bit and 16-bit readers (each pair states its own prefix), near partners and far ones,
+    in range and aliasing alike; more than 64 pairs per launch too (descriptors through the staging ring)."""
+    n, d = 10, 3001
+    cfg = dict(objective=1, nonblocking=2, grad_std=0.03, drift_std=0.1, offset_std=0.2)
+    orc, gpu = make_pair(n, d, "complete", seed=33, **cfg)
+    inject(orc, gpu)
+    rng = np.random.default_rng(bits)
+    for rnd in range(8):
+        nodes = rng.permutation(n)[:4]
+        assert orc.local_steps(nodes, 2, 0.05) == 0 and gpu.local_steps(nodes, 2, 0.05) == 0
+        inject(orc, gpu, what=("X",))
+        pairs = disjoint_pairs(orc, rng, int(rng.integers(1, 6)))
+        prefixes = rng.choice([8, 16], size=len(pairs)).astype(np.int32)
+        assert orc.interact_prefixed(pairs, prefixes, bits) == 0
+        assert gpu.interact_prefixed(pairs, prefixes, bits) == 0
+        assert_store_equal(orc, gpu, bits)
+    # an 8-bit reader does not touch its partner's high bytes, the 16-bit reader in the same launch does
+    valid = (np.arange(orc.nblk * 1024) < d).reshape(-1, 1024)       # not the padding behind coordinate d
+    for i in range(n):
+        row = gpu.get(g.T_OWN, i).reshape(-1, 2, 1024).copy()
+        row[:, 1, :][valid] ^= 0x3C
+        gpu.set(g.T_OWN, i, row.reshape(-1))
+        orc.own_bytes[i] = row.reshape(-1)
+    pairs, prefixes = [[0, 1], [2, 3]], [8, 16]
+    x0 = orc.X[0].copy()
+    assert orc.interact_prefixed(pairs, prefixes, bits) == 0 and gpu.interact_prefixed(pairs, prefixes, bits) == 0
+    assert_store_equal(orc, gpu, bits)
+    assert gpu.get_own_prefix() == 16
+    # argument checks: nothing runs, nothing changes
+    w_before = [tuple(gpu.get(g.T_COUNTERS, i)) for i in range(n)]
+    assert gpu.interact_prefixed([[4, 5]], [12], bits) == g.EINVAL
+    assert gpu._L.swarm_interact_prefixed(gpu._h, None, None, 1, bits) == g.EINVAL
+    assert gpu.interact_prefixed([[4, 4]], [8], bits) == g.EPAIR
+    assert [tuple(gpu.get(g.T_COUNTERS, i)) for i in range(n)] == w_before
+    plain = g.Swarm(4, 64)
+    plain.configure(objective=1, nonblocking=1)
+    assert plain.interact_prefixed([[0, 1]], [8], 8) == g.ESTATE
+
+
+def test_prefix_per_reader_in_a_launch_of_100_pairs():
+    n, d, bits = 200, 1500, 4
+    cfg = dict(objective=1, nonblocking=2, grad_std=0.03, offset_std=0.02)
+    orc, gpu = make_pair(n, d, "regular", 6, seed=35, **cfg)
+    inject(orc, gpu)
+    rng = np.random.default_rng(5)
+    for rnd in range(3):
+        pairs = disjoint_pairs(orc, rng, 100)
+        assert len(pairs) > 64
+        prefixes = rng.choice([8, 16], size=len(pairs)).astype(np.int32)
+        assert orc.interact_prefixed(pairs, prefixes, bits) == 0
+        assert gpu.interact_prefixed(pairs, prefixes, bits) == 0
+        assert_store_equal(orc, gpu, bits)
+
+
 def test_register_protocol_mode_switches_and_far_snapshots():
     n, d = 4, 2100
     cfg = dict(objective=1, nonblocking=2, grad_std=0.0, drift_std=0.0, offset_std=0.05)

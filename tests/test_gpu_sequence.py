@@ -76,6 +76,33 @@ def test_sequence_against_the_oracle_within_a_few_lattice_steps():
     assert gpu.potential() == pytest.approx(orc.potential(), rel=0.05)
 
 
+@pytest.mark.parametrize("H,lr", [(0, 0.05), (2, 0.0)])
+@pytest.mark.parametrize("d,bits", [(4096, 8), (1500, 3), (8192, 4), (700, 2)])
+def test_sequence_of_pure_interactions_matches_the_oracle_bit_for_bit(d, bits, H, lr):
+    """Without local steps (H = 0), or with steps of size zero, a sequence is a chain of blocking interactions on
+    shared nodes: everything in it is exact or a single rounding, so the single launch must reproduce the oracle's
+    models, codes, exponents and counters bit for bit."""
+    n = 8
+    orc, gpu = make_pair(n, d, "complete", seed=8, **LSQ)
+    inject(orc, gpu)
+    seq = random_sequence(n, 90, d + bits)
+    for a, b in seq:
+        if H > 0:
+            assert orc.local_steps([a, b], H, lr) == 0
+        assert orc.interact([[a, b]], bits) == 0
+    before = gpu.kernel_launches()
+    assert gpu.run_sequence(seq, H, lr, bits, True) == 0
+    assert gpu.kernel_launches() - before == 2          # 64 steps per launch
+    for i in range(n):
+        assert np.array_equal(gpu.get(g.T_X, i).view(np.uint32), orc.X[i].view(np.uint32)), i
+        nbytes = orc.nblk * 128 * bits
+        assert np.array_equal(gpu.get(g.T_CODES, i)[:nbytes], orc.codes[i, :nbytes]), i
+        assert np.array_equal(gpu.get(g.T_EXPS, i), orc.exps[i]), i
+        assert tuple(gpu.get(g.T_COUNTERS, i)) == (orc.w[i], orc.ls[i], orc.pbits[i])
+        assert tuple(gpu.get(g.T_CLOCKS, i)) == (orc.wo[i], orc.tau[i])
+    assert gpu.potential() == pytest.approx(orc.potential(), rel=1e-9)
+
+
 def test_sequence_falls_back_to_single_steps_elsewhere():
     n, d = 6, 3000
     for cfg, bits in ((dict(objective=1, grad_std=0.05, drift_std=0.2), 8), (dict(LSQ), 32),

@@ -252,6 +252,11 @@ def test_a_launch_mixes_readers_with_different_prefixes():
     assert mixed.interact_prefixed(launch, [16, 8], 8) == 0
     for name in ("X", "B", "own_bytes", "codes", "exps", "oexps", "w", "wo", "tau"):
         assert np.array_equal(getattr(ref, name), getattr(mixed, name)), name
+    # the prefix travels with its pair, wherever the pair stands in the list
+    swapped = near_and_far_readers()
+    assert swapped.interact_prefixed(launch[::-1], [8, 16], 8) == 0
+    for name in ("X", "B", "own_bytes", "codes", "exps", "oexps", "w", "wo"):
+        assert np.array_equal(getattr(ref, name), getattr(swapped, name)), name
     # the other way round the far reader aliases; the near reader's interaction is not affected by it
     wrong = near_and_far_readers()
     before = near_and_far_readers()
