@@ -357,21 +357,22 @@ __device__ __forceinline__ void split_planes(const uint32_t (&ow)[4], uint2& lo,
 }
 
 // Decode chain of a two-register block. On entry nx = X^a, av = snapshot B^a; on return nx = new model,
-// av = average. Returns the warp-reduced block maxima for the exponents of the three writes. The magnitude
-// bounds max(|new model|, |average|) and max(|average|, |Q(X^_b)|) are put together after the reduction from the
-// maxima of the three vectors (max is exact, so the grouping does not matter): one max per vector and coordinate.
-template <int BITS, bool FAST>
+// av = average. Returns the warp-reduced block maxima for the exponents of the three writes. FAST_LAST: the form
+// of the lattice arithmetic in the last decode (b's current register, keyed by Q(X^_b)).
+template <int BITS, bool FAST, bool FAST_LAST>
 __device__ __forceinline__ void registers_decode(f8 (&nx)[kSub], f8 (&av)[kSub], const uint2 (&va)[kSub],
                                                  const uint2 (&vb)[kSub], const uint2 (&vbh)[kSub],
                                                  const uint64_t (&pa)[kSub], const uint64_t (&pb)[kSub], int prefix,
                                                  int eoa, int eob, int epa, int epb, float& spread_out, float& dmax_out,
-                                                 float& M_out, float& rho_b_out, float& M_b_out, float& m_new_out) {
+                                                 float& M_out, float& rho_b_out, float& M_b_out) {
   using Ops = LatticeOps<FAST>;
+  using LastOps = LatticeOps<FAST_LAST>;
+  static_assert(FAST || !FAST_LAST, "the last decode follows the others into the defining form");
   const float so_a = pow2f_exact(eoa), io_a = pow2f_exact(-eoa), so_b = pow2f_exact(eob), io_b = pow2f_exact(-eob);
   const float sp_a = pow2f_exact(epa), ip_a = pow2f_exact(-epa), sp_b = pow2f_exact(epb), ip_b = pow2f_exact(-epb);
   const float uo_a = FAST ? -__fmul_rn(kCellBias, so_a) : 0.0f, uo_b = FAST ? -__fmul_rn(kCellBias, so_b) : 0.0f;
-  const float up_a = FAST ? -__fmul_rn(kCellBias, sp_a) : 0.0f, up_b = FAST ? -__fmul_rn(kCellBias, sp_b) : 0.0f;
-  float spread = 0.0f, dmax = 0.0f, rho_b = 0.0f, m_new = 0.0f, m_avg = 0.0f, m_qb = 0.0f;
+  const float up_a = FAST ? -__fmul_rn(kCellBias, sp_a) : 0.0f, up_b = FAST_LAST ? -__fmul_rn(kCellBias, sp_b) : 0.0f;
+  float spread = 0.0f, dmax = 0.0f, M = 0.0f, rho_b = 0.0f, M_b = 0.0f;
 #pragma unroll
   for (int j = 0; j < kSub; ++j)
 #pragma unroll
@@ -381,27 +382,23 @@ __device__ __forceinline__ void registers_decode(f8 (&nx)[kSub], f8 (&av)[kSub],
       const float qhat_a = Ops::value(Ops::template decode<8>(plane_byte(va[j], i), Ops::cell(snap, io_a)), so_a, uo_a);
       const float Qa = Ops::value(Ops::template decode<BITS>((uint32_t)(pa[j] >> (i * BITS)), Ops::cell(qhat_a, ip_a)), sp_a, up_a);
       const float qhat_b = Ops::value(Ops::decode_bits(plane_colour16(vb[j], vbh[j], i), Ops::cell(snap, io_b), prefix), so_b, uo_b);
-      const float Qb = Ops::value(Ops::template decode<BITS>((uint32_t)(pb[j] >> (i * BITS)), Ops::cell(qhat_b, ip_b)), sp_b, up_b);
+      const float Qb = LastOps::value(LastOps::template decode<BITS>((uint32_t)(pb[j] >> (i * BITS)), LastOps::cell(qhat_b, ip_b)), sp_b, up_b);
       const float avg = __fmul_rn(0.5f, __fadd_rn(Qa, Qb));
       const float D = __fsub_rn(snap, nx[j].v[i]);
       const float x_new = __fsub_rn(avg, D);
       spread = fmaxf(spread, fabsf(__fsub_rn(Qa, Qb)));
       dmax = fmaxf(dmax, fabsf(D));
-      m_new = fmaxf(m_new, fabsf(x_new));
-      m_avg = fmaxf(m_avg, fabsf(avg));
-      m_qb = fmaxf(m_qb, fabsf(qhat_b));
+      M = fmaxf(M, fmaxf(fabsf(x_new), fabsf(avg)));             // (three-input maxima: one instruction each)
       rho_b = fmaxf(rho_b, fabsf(__fsub_rn(avg, qhat_b)));        // distance of the average to b's decoding key
+      M_b = fmaxf(M_b, fmaxf(fabsf(avg), fabsf(qhat_b)));
       nx[j].v[i] = x_new;
       av[j].v[i] = avg;
     }
   spread_out = warp_max_nonneg(spread);
   dmax_out = warp_max_nonneg(dmax);
+  M_out = warp_max_nonneg(M);
   rho_b_out = warp_max_nonneg(rho_b);
-  m_new = warp_max_nonneg(m_new);
-  m_avg = warp_max_nonneg(m_avg);
-  M_out = fmaxf(m_new, m_avg);
-  M_b_out = fmaxf(m_avg, warp_max_nonneg(m_qb));
-  m_new_out = m_new;
+  M_b_out = warp_max_nonneg(M_b);
 }
 
 // Writes a's own register (16-bit colours of the new model, two byte planes) and b's current register
@@ -409,11 +406,11 @@ __device__ __forceinline__ void registers_decode(f8 (&nx)[kSub], f8 (&av)[kSub],
 template <int BITS, bool FAST>
 __device__ __forceinline__ void registers_encode_own(const f8 (&nx)[kSub], const f8 (&av)[kSub], uint8_t* oa, uint8_t* cb,
                                                      uint32_t group0, const StoreView& s, const PairDesc& pd, int lane,
-                                                     int eo, int ep_b, float m_new, float& rho_a_out, float& M_a_out) {
+                                                     int eo, int ep_b, float& rho_a_out, float& M_a_out) {
   using Ops = LatticeOps<FAST>;
   const float so = pow2f_exact(eo), io = pow2f_exact(-eo), ipb_new = pow2f_exact(-ep_b);
   const float uo = FAST ? -__fmul_rn(kCellBias, so) : 0.0f;
-  float rho_a = 0.0f, m_q = 0.0f;    // m_new: the block maximum of |new model|, known from the decode phase
+  float rho_a = 0.0f, M_a = 0.0f;
 #pragma unroll
   for (int j = 0; j < kSub; ++j) {
     const uint32_t g = group0 + j * (kSubCoords / 8);
@@ -426,7 +423,7 @@ __device__ __forceinline__ void registers_encode_own(const f8 (&nx)[kSub], const
       qo[i] = Ops::encode(nx[j].v[i], io, sr_word(ro, i), i & 1, cell);
       const float qhat_new = Ops::value(qo[i], so, uo);
       rho_a = fmaxf(rho_a, fabsf(__fsub_rn(nx[j].v[i], qhat_new)));
-      m_q = fmaxf(m_q, fabsf(qhat_new));
+      M_a = fmaxf(M_a, fmaxf(fabsf(nx[j].v[i]), fabsf(qhat_new)));
       qb[i] = Ops::encode(av[j].v[i], ipb_new, sr_word(rb, i), i & 1, cell);
     }
     uint32_t ow[4];
@@ -439,7 +436,7 @@ __device__ __forceinline__ void registers_encode_own(const f8 (&nx)[kSub], const
     store_codes<BITS>(cb + j * (kSubCoords * BITS / 8), lane, pack_colours<BITS>(qb));
   }
   rho_a_out = warp_max_nonneg(rho_a);
-  M_a_out = fmaxf(m_new, warp_max_nonneg(m_q));
+  M_a_out = warp_max_nonneg(M_a);
 }
 
 // Writes the new model to X^a and B^a and its b-bit colours to a's current register.
@@ -525,8 +522,12 @@ interact_registers_kernel(StoreView s, const PairList pairs, int64_t total_warps
   const int eoa = s.oexps[(int64_t)pd.a * s.nblk + blk], eob = s.oexps[(int64_t)pd.b * s.nblk + blk];
   const int epa = s.exps[(int64_t)pd.a * s.nblk + blk], epb = s.exps[(int64_t)pd.b * s.nblk + blk];
 
-  // largest key magnitude of the block and bounds on the decoded own-register values (a key plus the decode
-  // window): they decide, for the whole warp, which form of the lattice arithmetic the decode chain takes
+  // Which form of the lattice arithmetic the decode chain takes is decided for the whole warp from bounds on the
+  // keys: the snapshot (largest magnitude kmax) for the two own registers; for a's current register Q(X^_a),
+  // which the 8-bit own decode leaves within 130 own steps of the snapshot; for b's current register Q(X^_b), which
+  // can lie anywhere in the reader's window (32768 own steps with the full register: usually too far for the bound
+  // to pass, though the value itself never is). That last decode therefore takes its form on its own: with the
+  // full register it normally runs in the defining form (two conversions) while the other three stay fast.
   float kmax = 0.0f;
 #pragma unroll
   for (int j = 0; j < kSub; ++j)
@@ -535,11 +536,16 @@ interact_registers_kernel(StoreView s, const PairList pairs, int64_t total_warps
   kmax = warp_max_nonneg(kmax);
   const float qa_max = __fmaf_rn(130.0f, pow2f_exact(eoa), kmax);
   const float qb_max = __fmaf_rn(prefix == 16 ? 32770.0f : 130.0f, pow2f_exact(eob), kmax);
-  const bool fast_chain = fast_range(kmax, pow2f_exact(-eoa), eoa) && fast_range(kmax, pow2f_exact(-eob), eob) &&
-                          fast_range(qa_max, pow2f_exact(-epa), epa) && fast_range(qb_max, pow2f_exact(-epb), epb);
-  float spread, dmax, M, rho_b, M_b, m_new;
-  if (fast_chain) registers_decode<BITS, true>(nx, av, va, vb, vbh, pa, pb, prefix, eoa, eob, epa, epb, spread, dmax, M, rho_b, M_b, m_new);
-  else registers_decode<BITS, false>(nx, av, va, vb, vbh, pa, pb, prefix, eoa, eob, epa, epb, spread, dmax, M, rho_b, M_b, m_new);
+  const bool fast_keys = fast_range(kmax, pow2f_exact(-eoa), eoa) && fast_range(kmax, pow2f_exact(-eob), eob) &&
+                         fast_range(qa_max, pow2f_exact(-epa), epa);
+  const bool fast_last = fast_range(qb_max, pow2f_exact(-epb), epb);
+  float spread, dmax, M, rho_b, M_b;
+  if (fast_keys && fast_last)
+    registers_decode<BITS, true, true>(nx, av, va, vb, vbh, pa, pb, prefix, eoa, eob, epa, epb, spread, dmax, M, rho_b, M_b);
+  else if (fast_keys)
+    registers_decode<BITS, true, false>(nx, av, va, vb, vbh, pa, pb, prefix, eoa, eob, epa, epb, spread, dmax, M, rho_b, M_b);
+  else
+    registers_decode<BITS, false, false>(nx, av, va, vb, vbh, pa, pb, prefix, eoa, eob, epa, epb, spread, dmax, M, rho_b, M_b);
   const int eo = exponent_rule<kOwnResolutionBits>(__fadd_rn(__fmul_rn(2.0f, spread), dmax), M);
   const int ep_b = exponent_rule<BITS>(rho_b, M_b);
 
@@ -547,9 +553,9 @@ interact_registers_kernel(StoreView s, const PairList pairs, int64_t total_warps
   const uint32_t group0 = (uint32_t)(blk * (kBlockCoords / 8) + lane);
   float rho_a, M_a;
   if (fast_range(M, pow2f_exact(-eo), eo) && fast_range(M_b, pow2f_exact(-ep_b), ep_b))
-    registers_encode_own<BITS, true>(nx, av, oa, cb, group0, s, pd, lane, eo, ep_b, m_new, rho_a, M_a);
+    registers_encode_own<BITS, true>(nx, av, oa, cb, group0, s, pd, lane, eo, ep_b, rho_a, M_a);
   else
-    registers_encode_own<BITS, false>(nx, av, oa, cb, group0, s, pd, lane, eo, ep_b, m_new, rho_a, M_a);
+    registers_encode_own<BITS, false>(nx, av, oa, cb, group0, s, pd, lane, eo, ep_b, rho_a, M_a);
   const int ep_a = exponent_rule<BITS>(rho_a, M_a);
   if (fast_range(M_a, pow2f_exact(-ep_a), ep_a)) registers_encode_current<BITS, true>(nx, xa, ba, ca, group0, s, pd, lane, ep_a);
   else registers_encode_current<BITS, false>(nx, xa, ba, ca, group0, s, pd, lane, ep_a);
