@@ -154,9 +154,10 @@ int swarm_interact(swarm_ctx *ctx, const swarm_pair *pairs_host, int32_t npairs,
 /* Algorithm 1, one whole step of a launch: the initiator of every pair (and its responder when
  * step_responders != 0) takes H local steps with learning rate lr, then the pairs interact. Same
  * results, bit for bit, as swarm_local_steps on those nodes followed by swarm_interact(pairs, bits, mode).
- * With SWARM_OBJ_SYNTH the steps run inside the interaction kernel, so the models make one trip through
- * HBM instead of two and the launch is one kernel; with the least-squares objectives, whose gradient
- * couples all coordinates of a model, the library runs the two calls in sequence. H = 0 is swarm_interact.
+ * With SWARM_OBJ_SYNTH and a blocking or single-buffer exchange the steps run inside the interaction kernel, so
+ * the models make one trip through HBM instead of two and the launch is one kernel; with the two-register
+ * exchange, and with the least-squares objectives, whose gradient couples all coordinates of a model, the
+ * library runs the two calls in sequence. H = 0 is swarm_interact.
  * Errors: those of the two calls; a refused call leaves the models untouched. */
 int swarm_step(swarm_ctx *ctx, const swarm_pair *pairs_host, int32_t npairs, int32_t H, float lr, int32_t bits,
                int32_t mode, int32_t step_responders);

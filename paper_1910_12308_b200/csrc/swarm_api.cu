@@ -843,10 +843,11 @@ int swarm_step(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, int32_t H,
   if (!c || H < 0 || npairs < 0 || (npairs > 0 && !pairs)) return SWARM_EINVAL;
   if (H == 0) return interact_impl(c, pairs, npairs, bits, mode, 0, 0.0f, 0);
   if (c->cfg.objective == SWARM_OBJ_NONE) return SWARM_ESTATE;
-  // Elementwise objective: the steps run inside the interaction kernel. A publish that the interaction
-  // triggers runs before the fused steps; that is the same as after them unless it first refreshes stale
-  // snapshots from the models, so that one case takes the two-call route.
-  if (c->cfg.objective == SWARM_OBJ_SYNTH && !(mode != SWARM_BLOCKING && c->b_stale))
+  // Elementwise objective, blocking or single-buffer exchange: the steps run inside the interaction kernel. A
+  // publish that the interaction triggers runs before the fused steps; that is the same as after them unless it
+  // first refreshes stale snapshots from the models, so that one case takes the two-call route. So does the
+  // two-register exchange, whose kernel is bound by instruction issue already (measured slower with the steps in it).
+  if (c->cfg.objective == SWARM_OBJ_SYNTH && mode != SWARM_REGISTERS && !(mode != SWARM_BLOCKING && c->b_stale))
     return interact_impl(c, pairs, npairs, bits, mode, H, lr, step_responders);
   // objectives whose gradient couples all coordinates: the two calls in sequence, after the checks that
   // the interaction would make (so that a refused call leaves the models untouched)

@@ -462,7 +462,9 @@ __device__ __forceinline__ void registers_encode_current(const f8 (&nx)[kSub], f
   }
 }
 
-template <int BITS, bool FUSED>
+// (Local steps are not fused into this kernel: at 168 registers it keeps three warps per scheduler, and the steps'
+// instruction stream on top of its own ran slower than the two kernels one after the other.)
+template <int BITS>
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
 interact_registers_kernel(StoreView s, const PairList pairs, int64_t total_warps, const FusedSteps fs) {
   grid_dependency_signal();
@@ -505,10 +507,6 @@ interact_registers_kernel(StoreView s, const PairList pairs, int64_t total_warps
   uint64_t pa[kSub], pb[kSub];
 #pragma unroll
   for (int j = 0; j < kSub; ++j) nx[j] = ld256(xa + j * kSubCoords);
-  if constexpr (FUSED) {
-    if (fs.responders) fused_steps_responder(s, fs, pd, blk, lane);
-    fused_steps_block(nx, s, fs, pd.a, pd.lsa, blk, lane);
-  }
 #pragma unroll
   for (int j = 0; j < kSub; ++j) av[j] = ld256(ba + j * kSubCoords);
 #pragma unroll
@@ -705,8 +703,8 @@ cudaError_t launch_interact_registers(const StoreView& s, const PairList& pairs,
   if (warps + kPrefetchDistance >= kMaxLaunchWarps) return cudaErrorInvalidValue;
   const dim3 grid(ctas_for(warps)), block(kWarpsPerCta * 32);
   cudaError_t e = cudaSuccess;
-  SWARM_FOR_WIDTH(bits, e = (fs.H > 0 ? launch_dependent(interact_registers_kernel<W, true>, grid, block, st, s, pairs, warps, fs)
-                                         : launch_dependent(interact_registers_kernel<W, false>, grid, block, st, s, pairs, warps, fs)))
+  if (fs.H > 0) return cudaErrorInvalidValue;       // the caller runs the local steps as a kernel of their own
+  SWARM_FOR_WIDTH(bits, e = launch_dependent(interact_registers_kernel<W>, grid, block, st, s, pairs, warps, fs))
   ++*launches;
   return e != cudaSuccess ? e : cudaGetLastError();
 }
