@@ -43,9 +43,9 @@ __device__ __forceinline__ void fused_steps_responder(const StoreView& s, const 
   for (int j = 0; j < kSub; ++j) st256(xb + j * kSubCoords, vb[j]);
 }
 
-// Encode / cross-decode / average of the 8 coordinate pairs a lane owns in one sub-block, in the fast or the
+// Encode / cross-decode / average of the 8 coordinate pairs a lane owns in one sub-block, in a fast or the
 // defining form of the lattice arithmetic (LatticeOps). ra, rb: the generator calls that hold the rounding
-// uniforms of the two buffers. ELIDE (fast form only) leaves the cross-decodes out: when the block's range
+// uniforms of the two buffers. ELIDE (fast forms only) leaves the cross-decodes out: when the block's range
 // satisfies rho < L * 2^e strictly, |X^a - X^b| < L * 2^e holds for the exact difference of every coordinate
 // pair (rho is a maximum of rounded differences, and rounding to nearest cannot carry a value from L * 2^e or
 // above to below it), so the two scaled values differ by less than L, their floors by at most L, and the
@@ -55,21 +55,21 @@ __device__ __forceinline__ void fused_steps_responder(const StoreView& s, const 
 struct ExchangeScale {
   float step, inv_step, unbias, half_step, half_unbias;
 };
-template <bool FAST>
+template <int MODE>
 __device__ __forceinline__ ExchangeScale exchange_scale(int e) {
   ExchangeScale sc;
   sc.step = pow2f_exact(e);
   sc.inv_step = pow2f_exact(-e);
-  sc.unbias = FAST ? -__fmul_rn(kCellBias, sc.step) : 0.0f;
+  sc.unbias = MODE != kDefining ? -__fmul_rn(kCellBias, sc.step) : 0.0f;
   sc.half_step = __fmul_rn(0.5f, sc.step);                  // 2^(e-1): a subnormal for e = -126, still exact
   sc.half_unbias = __fmul_rn(0.5f, sc.unbias);
   return sc;
 }
-template <int BITS, bool FAST, bool ELIDE>
+template <int BITS, int MODE, bool ELIDE>
 __device__ __forceinline__ void exchange8(const f8& va, const f8& vb, const uint4& ra, const uint4& rb,
                                           const ExchangeScale& sc, f8& out, uint64_t& pka, uint64_t& pkb) {
-  using Ops = LatticeOps<FAST>;
-  static_assert(FAST || !ELIDE, "the decode is left out in the fast form only");
+  using Ops = LatticeOps<MODE>;
+  static_assert(MODE != kDefining || !ELIDE, "the decode is left out in the fast forms only");
   uint32_t ia[8], ib[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
@@ -89,11 +89,11 @@ __device__ __forceinline__ void exchange8(const f8& va, const f8& vb, const uint
   pkb = pack_colours<BITS>(ib);
 }
 
-template <int BITS, bool FAST, bool ELIDE>
+template <int BITS, int MODE, bool ELIDE>
 __device__ __forceinline__ void blocking_exchange(const f8 (&va)[kSub], const f8 (&vb)[kSub], float* xa, float* xb,
                                                   uint8_t* ca, uint8_t* cb, uint32_t group0, const StoreView& s,
                                                   const PairDesc& pd, int lane, int e) {
-  const ExchangeScale sc = exchange_scale<FAST>(e);
+  const ExchangeScale sc = exchange_scale<MODE>(e);
 #pragma unroll
   for (int j = 0; j < kSub; ++j) {
     const uint32_t g = group0 + j * (kSubCoords / 8);
@@ -101,7 +101,7 @@ __device__ __forceinline__ void blocking_exchange(const f8 (&va)[kSub], const f8
     const uint4 rb = philox4x32_10(g, (uint32_t)pd.b, pd.wb, kStreamRounding, s.rk);
     uint64_t pka, pkb;
     f8 out;
-    exchange8<BITS, FAST, ELIDE>(va[j], vb[j], ra, rb, sc, out, pka, pkb);
+    exchange8<BITS, MODE, ELIDE>(va[j], vb[j], ra, rb, sc, out, pka, pkb);
     st256(xa + j * kSubCoords, out);
     st256(xb + j * kSubCoords, out);
     store_codes<BITS>(ca + j * (kSubCoords * BITS / 8), lane, pka);
@@ -150,25 +150,26 @@ __device__ __forceinline__ void blocking_block(const StoreView& s, const PairDes
   const uint32_t group0 = (uint32_t)(blk * (kBlockCoords / 8) + lane);   // generator call index of sub-block 0
   uint8_t* ca = s.codes + (int64_t)pd.a * s.nblk * kBlockCoords + blk * (kBlockCoords * BITS / 8) + lane * BITS;
   uint8_t* cb = s.codes + (int64_t)pd.b * s.nblk * kBlockCoords + blk * (kBlockCoords * BITS / 8) + lane * BITS;
-  if (fast_range(M, pow2f_exact(-e), e)) {
-    if (decode_elidable<BITS>(rho, e)) blocking_exchange<BITS, true, true>(va, vb, xa, xb, ca, cb, group0, s, pd, lane, e);
-    else blocking_exchange<BITS, true, false>(va, vb, xa, xb, ca, cb, group0, s, pd, lane, e);
-  } else {
-    blocking_exchange<BITS, false, false>(va, vb, xa, xb, ca, cb, group0, s, pd, lane, e);
-  }
+  const int mode = lattice_mode(M, pow2f_exact(-e), e);
+  const bool elide = mode != kDefining && decode_elidable<BITS>(rho, e);
+  if (mode == kFastFma && elide) blocking_exchange<BITS, kFastFma, true>(va, vb, xa, xb, ca, cb, group0, s, pd, lane, e);
+  else if (mode == kFastFma) blocking_exchange<BITS, kFastFma, false>(va, vb, xa, xb, ca, cb, group0, s, pd, lane, e);
+  else if (mode == kFastMul && elide) blocking_exchange<BITS, kFastMul, true>(va, vb, xa, xb, ca, cb, group0, s, pd, lane, e);
+  else if (mode == kFastMul) blocking_exchange<BITS, kFastMul, false>(va, vb, xa, xb, ca, cb, group0, s, pd, lane, e);
+  else blocking_exchange<BITS, kDefining, false>(va, vb, xa, xb, ca, cb, group0, s, pd, lane, e);
   if (lane == 0) {
     s.exps[(int64_t)pd.a * s.nblk + blk] = (int8_t)e;
     s.exps[(int64_t)pd.b * s.nblk + blk] = (int8_t)e;
   }
 }
 
-template <int BITS, bool FAST, bool ELIDE>
+template <int BITS, int MODE, bool ELIDE>
 __device__ __forceinline__ void subblock_exchange(const f8& va, const f8& vb, float* xa, float* xb, uint8_t* ca,
                                                   uint8_t* cb, const uint4& ra, const uint4& rb, int lane, int e) {
-  const ExchangeScale sc = exchange_scale<FAST>(e);
+  const ExchangeScale sc = exchange_scale<MODE>(e);
   uint64_t pka, pkb;
   f8 out;
-  exchange8<BITS, FAST, ELIDE>(va, vb, ra, rb, sc, out, pka, pkb);
+  exchange8<BITS, MODE, ELIDE>(va, vb, ra, rb, sc, out, pka, pkb);
   st256(xa, out);
   st256(xb, out);
   store_codes<BITS>(ca, lane, pka);
@@ -206,12 +207,13 @@ __device__ __forceinline__ void blocking_subblock(const StoreView& s, const Pair
                 j * (kSubCoords * BITS / 8) + lane * BITS;
   const uint4 ra = philox4x32_10(g, (uint32_t)pd.a, pd.wa, kStreamRounding, s.rk);
   const uint4 rb = philox4x32_10(g, (uint32_t)pd.b, pd.wb, kStreamRounding, s.rk);
-  if (fast_range(M, pow2f_exact(-e), e)) {
-    if (decode_elidable<BITS>(rho, e)) subblock_exchange<BITS, true, true>(va, vb, xa, xb, ca, cb, ra, rb, lane, e);
-    else subblock_exchange<BITS, true, false>(va, vb, xa, xb, ca, cb, ra, rb, lane, e);
-  } else {
-    subblock_exchange<BITS, false, false>(va, vb, xa, xb, ca, cb, ra, rb, lane, e);
-  }
+  const int mode = lattice_mode(M, pow2f_exact(-e), e);
+  const bool elide = mode != kDefining && decode_elidable<BITS>(rho, e);
+  if (mode == kFastFma && elide) subblock_exchange<BITS, kFastFma, true>(va, vb, xa, xb, ca, cb, ra, rb, lane, e);
+  else if (mode == kFastFma) subblock_exchange<BITS, kFastFma, false>(va, vb, xa, xb, ca, cb, ra, rb, lane, e);
+  else if (mode == kFastMul && elide) subblock_exchange<BITS, kFastMul, true>(va, vb, xa, xb, ca, cb, ra, rb, lane, e);
+  else if (mode == kFastMul) subblock_exchange<BITS, kFastMul, false>(va, vb, xa, xb, ca, cb, ra, rb, lane, e);
+  else subblock_exchange<BITS, kDefining, false>(va, vb, xa, xb, ca, cb, ra, rb, lane, e);
   if (j == 0 && lane == 0) {
     s.exps[(int64_t)pd.a * s.nblk + blk] = (int8_t)e;
     s.exps[(int64_t)pd.b * s.nblk + blk] = (int8_t)e;

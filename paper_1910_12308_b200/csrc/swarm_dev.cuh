@@ -168,44 +168,58 @@ __device__ __forceinline__ int32_t encode_index(float x, float inv_step, uint32_
 // ---------------------------------------------------------------------------------------
 // The same lattice arithmetic without conversion instructions. Float<->integer conversions and
 // floorf share one quarter-rate unit, which the 8..18 conversions per coordinate of the interaction
-// kernels keep busier than HBM does. While the lattice exponent is e <= 0 (then t = x * 2^-e is an exact
-// product, subnormal x included) and every scaled value and lattice index of a block stays inside
-// (-2^21, 2^21), the same results come from full-rate fused multiply-adds and adds with directed rounding:
-//   s = fma(x, 2^-e, C) rounded toward -inf, C an integer in [2^23, 2^24) - 2^21, is floor(t) + C exactly
-//   (ulp 1 in [2^23, 2^24)). With C = 1.5 * 2^23 its bit pattern is 0x4B400000 + floor(t): a lattice cell
+// kernels keep busier than HBM does. While every scaled value and lattice index of a block stays inside
+// (-2^21, 2^21) and the exponent is at most 100, the same results come from full-rate instructions with
+// directed rounding:
+//   s = t + C rounded toward -inf, C an integer in [2^23, 2^24) - 2^21, is floor(t) + C exactly (floats are
+//   spaced 1 in [2^23, 2^24)). With C = 1.5 * 2^23 its bit pattern is 0x4B400000 + floor(t): a lattice cell
 //   "biased" by 0x4B400000. The bias has no low 22 bits, so colours (cell & mask) and the window arithmetic
 //   of the decoder work on biased cells unchanged, and a biased index i turns into the value
 //   (i - bias) * 2^e with one exact fused multiply-add: as_float(i) * 2^e - 1.5*2^23 * 2^e.
-//   Encoder: with C = 1.5 * 2^23 + 192, frac = fma(x, 2^-e, C - s) is RN(t - floor t), the definition's
-//   fraction (it can round up to 1 for a tiny negative t, as there). The 16-bit uniform u becomes the float
+//   Encoder: with C = 1.5 * 2^23 + 192, frac = t + (C - s) is RN(t - floor t), the definition's fraction (it
+//   can round up to 1 for a tiny negative t, as there). The 16-bit uniform u becomes the float
 //   um = 192 + u / 2^16 by splicing its half word under the bytes 0x43 0x40 with one byte permute; 192 keeps
 //   um - frac inside [128, 256), where floats are spaced 2^-16, so um - frac rounded toward +inf is
 //   192 + (u - thr) / 2^16 with thr = floor(frac * 2^16), the definition's threshold, and s minus that,
 //   again rounded toward +inf, is floor(t) + 1.5 * 2^23 + [u < thr]: the biased lattice index.
-//   Six instructions, none of them a conversion.
-// LatticeOps<true> is that form (the caller checks the range, warp-uniformly, per block);
-// LatticeOps<false> is the defining form with saturating conversions. Both give bit-identical
-// results wherever the fast form is valid.
+// Two fast forms. For e <= 0 the scaled value t = x * 2^-e is an exact product (subnormal x included), so the
+// multiply folds into the adds: s = fma(x, 2^-e, C) and frac = fma(x, 2^-e, C - s), six instructions per encoded
+// coordinate (kFastFma). For 0 < e <= 100 a tiny x can make the product inexact (a subnormal result), and the
+// definition rounds it before taking the floor, so t is formed by a multiply of its own first: seven
+// instructions (kFastMul, valid for every e <= 100). LatticeOps<kDefining> is the defining form with saturating
+// conversions. All give bit-identical results wherever a fast form is valid; the caller picks the form,
+// warp-uniformly, per block.
 // ---------------------------------------------------------------------------------------
 constexpr float kCellBias = 12582912.0f;            // 1.5 * 2^23
 constexpr uint32_t kCellBiasBits = 0x4B400000u;
 constexpr float kEncBias = 12583104.0f;             // 1.5 * 2^23 + 192: running sum of the encoder
-constexpr float kFastRange = 2097152.0f;            // 2^21: bound on |x| * 2^-e for the fast form (half the
+constexpr float kFastRange = 2097152.0f;            // 2^21: bound on |x| * 2^-e for the fast forms (half the
                                                     // exact limit, which leaves room for the decode window)
+constexpr int kFastExpMax = 100;                    // keeps 1.5*2^23 * 2^e finite
+enum : int { kDefining = 0, kFastFma = 1, kFastMul = 2 };
 
-template <bool FAST>
+template <int MODE>
 struct LatticeOps {
+  static constexpr bool kFast = MODE != kDefining;
+  // x * 2^-e plus an integer constant, rounded toward -inf: floor(t) + c
+  static __device__ __forceinline__ float floor_plus(float x, float inv_step, float c, float& t_out) {
+    if constexpr (MODE == kFastFma) { t_out = 0.0f; return __fmaf_rd(x, inv_step, c); }
+    else { t_out = __fmul_rn(x, inv_step); return __fadd_rd(t_out, c); }
+  }
   // (biased) cell of a key: floor(key * 2^-e)
   static __device__ __forceinline__ uint32_t cell(float key, float inv_step) {
-    if constexpr (FAST) return __float_as_uint(__fmaf_rd(key, inv_step, kCellBias));
+    if constexpr (kFast) { float t; return __float_as_uint(floor_plus(key, inv_step, kCellBias, t)); }
     else return (uint32_t)__float2int_rd(__fmul_rn(key, inv_step));
   }
   // (biased) lattice index of x after stochastic rounding with half `hi` (0 low, 1 high) of generator
   // word `w`; `cell` receives the (biased) cell of x.
   static __device__ __forceinline__ uint32_t encode(float x, float inv_step, uint32_t w, int hi, uint32_t& cell_out) {
-    if constexpr (FAST) {
-      const float sft = __fmaf_rd(x, inv_step, kEncBias);                              // floor(t) + kEncBias
-      const float frac = __fmaf_rn(x, inv_step, __fsub_rn(kEncBias, sft));             // RN(t - floor t), in [0, 1]
+    if constexpr (kFast) {
+      float t;
+      const float sft = floor_plus(x, inv_step, kEncBias, t);                          // floor(t) + kEncBias
+      const float neg_floor = __fsub_rn(kEncBias, sft);
+      const float frac = MODE == kFastFma ? __fmaf_rn(x, inv_step, neg_floor)          // RN(t - floor t), in [0, 1]
+                                          : __fadd_rn(t, neg_floor);
       const float um = __uint_as_float(__byte_perm(w, 0x43400000u, hi ? 0x7632 : 0x7610));   // 192 + u / 2^16
       const float gap = __fsub_ru(um, frac);                                           // 192 + (u - thr) / 2^16
       cell_out = __float_as_uint(sft) - 192u;
@@ -231,18 +245,18 @@ struct LatticeOps {
     const uint32_t mask = (1u << bits) - 1u, L = (1u << (bits - 1)) - 1u;
     return cell_in - L + ((c - cell_in + L) & mask);
   }
-  // value of a (biased) index; `unbias` = -1.5*2^23 * step (fast form only)
+  // value of a (biased) index; `unbias` = -1.5*2^23 * step (fast forms only)
   static __device__ __forceinline__ float value(uint32_t idx, float step, float unbias) {
-    if constexpr (FAST) return __fmaf_rn(__uint_as_float(idx), step, unbias);
+    if constexpr (kFast) return __fmaf_rn(__uint_as_float(idx), step, unbias);
     else return __fmul_rn(__int2float_rn((int32_t)idx), step);
   }
-  // Fast form: half the sum of the values of two biased indices of magnitude <= 2^21 each (an encoder's own
+  // Fast forms: half the sum of the values of two biased indices of magnitude <= 2^21 each (an encoder's own
   // output), (qa + qb) * 2^(e-1). That is what RN(0.5 * RN(Qa + Qb)) comes to, because each product and the sum
   // are exact and (qa + qb) * 2^(e-1) is a float for every e >= -126 (a subnormal at worst). One integer
   // add-add (the sum of two biased patterns minus one bias is the biased sum while |qa + qb| <= 2^22) and one
   // fused multiply-add; `half_step` = 2^(e-1), `half_unbias` = -1.5*2^23 * 2^(e-1).
   static __device__ __forceinline__ float mean_of_own(uint32_t ia, uint32_t ib, float half_step, float half_unbias) {
-    static_assert(FAST, "biased indices only");
+    static_assert(kFast, "biased indices only");
     return __fmaf_rn(__uint_as_float(ia + ib - kCellBiasBits), half_step, half_unbias);
   }
 };
@@ -276,11 +290,27 @@ __device__ __forceinline__ uint64_t pack_colours(const uint32_t (&q)[8]) {
   }
 }
 
-// Whether the fast form covers a block: e <= 0 (exact scaling) and the largest magnitude `maxabs` scaled by
-// 2^-e stays below 2^21.
-__device__ __forceinline__ bool fast_range(float maxabs, float inv_step, int e) {
-  return __fmul_rn(maxabs, inv_step) < kFastRange && e <= 0;
+// The form of the lattice arithmetic that covers a block whose largest magnitude is `maxabs` at exponent e:
+// a fast form while maxabs * 2^-e stays below 2^21 and e <= 100, the fused one for e <= 0.
+__device__ __forceinline__ int lattice_mode(float maxabs, float inv_step, int e) {
+  if (!(__fmul_rn(maxabs, inv_step) < kFastRange) || e > kFastExpMax) return kDefining;
+  return e <= 0 ? kFastFma : kFastMul;
 }
+// For kernels that are built without the multiply form (their fast path is the fused one or none).
+__device__ __forceinline__ int lattice_mode_fused_only(float maxabs, float inv_step, int e) {
+  return lattice_mode(maxabs, inv_step, e) == kFastFma ? kFastFma : kDefining;
+}
+// The form that serves two scalings at once.
+__device__ __forceinline__ int lattice_mode_both(int m1, int m2) {
+  return (m1 == kDefining || m2 == kDefining) ? kDefining : ((m1 == kFastFma && m2 == kFastFma) ? kFastFma : kFastMul);
+}
+// Runs CALL with the compile-time constant M set to the run-time form `mode`.
+#define SWARM_LATTICE_DISPATCH(mode, ...)                                   \
+  switch (mode) {                                                           \
+    case kFastFma: { constexpr int M = kFastFma; __VA_ARGS__; } break;      \
+    case kFastMul: { constexpr int M = kFastMul; __VA_ARGS__; } break;      \
+    default: { constexpr int M = kDefining; __VA_ARGS__; } break;           \
+  }
 
 // Generator word holding the 16-bit rounding uniform of coordinate i (0..7) of a call covering 8
 // consecutive coordinates (low half for even i, high half for odd i).

@@ -112,15 +112,15 @@ interact_identity_kernel(StoreView s, const PairList pairs, int64_t total_warps,
 
 // Decode phase of a non-blocking block: nx holds X^a and av the snapshot B^a (the key) on entry; on return
 // nx holds the new model and av the average. Block maxima for the guard rule come back warp-reduced.
-template <int BITS, bool FAST>
+template <int BITS, int MODE>
 __device__ __forceinline__ void nonblocking_decode(f8 (&nx)[kSub], f8 (&av)[kSub], const uint64_t (&pa)[kSub],
                                                    const uint64_t (&pb)[kSub], int e_own, int e_oth, float& spread_out,
                                                    float& dmax_out, float& M_out) {
-  using Ops = LatticeOps<FAST>;
+  using Ops = LatticeOps<MODE>;
   const float step_own = pow2f_exact(e_own), inv_own = pow2f_exact(-e_own);
   const float step_oth = pow2f_exact(e_oth), inv_oth = pow2f_exact(-e_oth);
-  const float unb_own = FAST ? -__fmul_rn(kCellBias, step_own) : 0.0f;
-  const float unb_oth = FAST ? -__fmul_rn(kCellBias, step_oth) : 0.0f;
+  const float unb_own = Ops::kFast ? -__fmul_rn(kCellBias, step_own) : 0.0f;
+  const float unb_oth = Ops::kFast ? -__fmul_rn(kCellBias, step_oth) : 0.0f;
   float spread = 0.0f, dmax = 0.0f, M = 0.0f;
 #pragma unroll
   for (int j = 0; j < kSub; ++j)
@@ -146,11 +146,11 @@ __device__ __forceinline__ void nonblocking_decode(f8 (&nx)[kSub], f8 (&av)[kSub
 }
 
 // Encode phase: the new model goes to X^a, B^a and (encoded) to a's buffer, the average (encoded) to b's.
-template <int BITS, bool FAST>
+template <int BITS, int MODE>
 __device__ __forceinline__ void nonblocking_encode(const f8 (&nx)[kSub], const f8 (&av)[kSub], float* xa, float* ba,
                                                    uint8_t* ca, uint8_t* cb, uint32_t group0, const StoreView& s,
                                                    const PairDesc& pd, int lane, int e) {
-  using Ops = LatticeOps<FAST>;
+  using Ops = LatticeOps<MODE>;
   const float inv_step = pow2f_exact(-e);
 #pragma unroll
   for (int j = 0; j < kSub; ++j) {
@@ -181,7 +181,7 @@ __device__ __forceinline__ void nonblocking_encode(const f8 (&nx)[kSub], const f
 // Traffic per coordinate: 8 B + 2*b/8 B read, 8 B + 2*b/8 B written.
 // -----------------------------------------------------------------------------------------
 template <int BITS, bool FUSED>
-__global__ void __launch_bounds__(kWarpsPerCta * 32, FUSED ? 4 : 0)
+__global__ void __launch_bounds__(kWarpsPerCta * 32, 4)     // 128 registers: four CTAs per SM
 interact_nonblocking_kernel(StoreView s, const PairList pairs, int64_t total_warps, const FusedSteps fs) {
   grid_dependency_signal();
   grid_dependency_wait();
@@ -236,17 +236,15 @@ interact_nonblocking_kernel(StoreView s, const PairList pairs, int64_t total_war
 #pragma unroll
     for (int i = 0; i < 8; ++i) kmax = fmaxf(kmax, fabsf(av[j].v[i]));
   kmax = warp_max_nonneg(kmax);
-  float spread, dmax, M;
-  if (fast_range(kmax, pow2f_exact(-e_own), e_own) && fast_range(kmax, pow2f_exact(-e_oth), e_oth))
-    nonblocking_decode<BITS, true>(nx, av, pa, pb, e_own, e_oth, spread, dmax, M);
-  else
-    nonblocking_decode<BITS, false>(nx, av, pa, pb, e_own, e_oth, spread, dmax, M);
+  float spread, dmax, M_blk;
+  const int dec_mode = lattice_mode_both(lattice_mode(kmax, pow2f_exact(-e_own), e_own), lattice_mode(kmax, pow2f_exact(-e_oth), e_oth));
+  SWARM_LATTICE_DISPATCH(dec_mode, nonblocking_decode<BITS, M>(nx, av, pa, pb, e_own, e_oth, spread, dmax, M_blk))
   const float rho = __fadd_rn(__fmul_rn(2.0f, spread), dmax);
-  const int e = exponent_rule<BITS>(rho, M);
+  const int e = exponent_rule<BITS>(rho, M_blk);
 
   const uint32_t group0 = (uint32_t)(blk * (kBlockCoords / 8) + lane);
-  if (fast_range(M, pow2f_exact(-e), e)) nonblocking_encode<BITS, true>(nx, av, xa, ba, ca, cb, group0, s, pd, lane, e);
-  else nonblocking_encode<BITS, false>(nx, av, xa, ba, ca, cb, group0, s, pd, lane, e);
+  SWARM_LATTICE_DISPATCH(lattice_mode(M_blk, pow2f_exact(-e), e),
+                         nonblocking_encode<BITS, M>(nx, av, xa, ba, ca, cb, group0, s, pd, lane, e))
   if (lane == 0) { *ea_p = (int8_t)e; *eb_p = (int8_t)e; }
 }
 
@@ -359,19 +357,19 @@ __device__ __forceinline__ void split_planes(const uint32_t (&ow)[4], uint2& lo,
 // Decode chain of a two-register block. On entry nx = X^a, av = snapshot B^a; on return nx = new model,
 // av = average. Returns the warp-reduced block maxima for the exponents of the three writes. FAST_LAST: the form
 // of the lattice arithmetic in the last decode (b's current register, keyed by Q(X^_b)).
-template <int BITS, bool FAST, bool FAST_LAST>
+template <int BITS, int MODE, int MODE_LAST>
 __device__ __forceinline__ void registers_decode(f8 (&nx)[kSub], f8 (&av)[kSub], const uint2 (&va)[kSub],
                                                  const uint2 (&vb)[kSub], const uint2 (&vbh)[kSub],
                                                  const uint64_t (&pa)[kSub], const uint64_t (&pb)[kSub], int prefix,
                                                  int eoa, int eob, int epa, int epb, float& spread_out, float& dmax_out,
                                                  float& M_out, float& rho_b_out, float& M_b_out) {
-  using Ops = LatticeOps<FAST>;
-  using LastOps = LatticeOps<FAST_LAST>;
-  static_assert(FAST || !FAST_LAST, "the last decode follows the others into the defining form");
+  using Ops = LatticeOps<MODE>;
+  using LastOps = LatticeOps<MODE_LAST>;
+  static_assert(MODE != kDefining || MODE_LAST == kDefining, "the last decode follows the others into the defining form");
   const float so_a = pow2f_exact(eoa), io_a = pow2f_exact(-eoa), so_b = pow2f_exact(eob), io_b = pow2f_exact(-eob);
   const float sp_a = pow2f_exact(epa), ip_a = pow2f_exact(-epa), sp_b = pow2f_exact(epb), ip_b = pow2f_exact(-epb);
-  const float uo_a = FAST ? -__fmul_rn(kCellBias, so_a) : 0.0f, uo_b = FAST ? -__fmul_rn(kCellBias, so_b) : 0.0f;
-  const float up_a = FAST ? -__fmul_rn(kCellBias, sp_a) : 0.0f, up_b = FAST_LAST ? -__fmul_rn(kCellBias, sp_b) : 0.0f;
+  const float uo_a = Ops::kFast ? -__fmul_rn(kCellBias, so_a) : 0.0f, uo_b = Ops::kFast ? -__fmul_rn(kCellBias, so_b) : 0.0f;
+  const float up_a = Ops::kFast ? -__fmul_rn(kCellBias, sp_a) : 0.0f, up_b = LastOps::kFast ? -__fmul_rn(kCellBias, sp_b) : 0.0f;
   float spread = 0.0f, dmax = 0.0f, M = 0.0f, rho_b = 0.0f, M_b = 0.0f;
 #pragma unroll
   for (int j = 0; j < kSub; ++j)
@@ -403,13 +401,13 @@ __device__ __forceinline__ void registers_decode(f8 (&nx)[kSub], f8 (&av)[kSub],
 
 // Writes a's own register (16-bit colours of the new model, two byte planes) and b's current register
 // (b-bit colours of the average); returns the distance of the new model to the lattice point just written.
-template <int BITS, bool FAST>
+template <int BITS, int MODE>
 __device__ __forceinline__ void registers_encode_own(const f8 (&nx)[kSub], const f8 (&av)[kSub], uint8_t* oa, uint8_t* cb,
                                                      uint32_t group0, const StoreView& s, const PairDesc& pd, int lane,
                                                      int eo, int ep_b, float& rho_a_out, float& M_a_out) {
-  using Ops = LatticeOps<FAST>;
+  using Ops = LatticeOps<MODE>;
   const float so = pow2f_exact(eo), io = pow2f_exact(-eo), ipb_new = pow2f_exact(-ep_b);
-  const float uo = FAST ? -__fmul_rn(kCellBias, so) : 0.0f;
+  const float uo = Ops::kFast ? -__fmul_rn(kCellBias, so) : 0.0f;
   float rho_a = 0.0f, M_a = 0.0f;
 #pragma unroll
   for (int j = 0; j < kSub; ++j) {
@@ -440,11 +438,11 @@ __device__ __forceinline__ void registers_encode_own(const f8 (&nx)[kSub], const
 }
 
 // Writes the new model to X^a and B^a and its b-bit colours to a's current register.
-template <int BITS, bool FAST>
+template <int BITS, int MODE>
 __device__ __forceinline__ void registers_encode_current(const f8 (&nx)[kSub], float* xa, float* ba, uint8_t* ca,
                                                          uint32_t group0, const StoreView& s, const PairDesc& pd,
                                                          int lane, int ep_a) {
-  using Ops = LatticeOps<FAST>;
+  using Ops = LatticeOps<MODE>;
   const float ipa_new = pow2f_exact(-ep_a);
 #pragma unroll
   for (int j = 0; j < kSub; ++j) {
@@ -534,29 +532,33 @@ interact_registers_kernel(StoreView s, const PairList pairs, int64_t total_warps
   kmax = warp_max_nonneg(kmax);
   const float qa_max = __fmaf_rn(130.0f, pow2f_exact(eoa), kmax);
   const float qb_max = __fmaf_rn(prefix == 16 ? 32770.0f : 130.0f, pow2f_exact(eob), kmax);
-  const bool fast_keys = fast_range(kmax, pow2f_exact(-eoa), eoa) && fast_range(kmax, pow2f_exact(-eob), eob) &&
-                         fast_range(qa_max, pow2f_exact(-epa), epa);
-  const bool fast_last = fast_range(qb_max, pow2f_exact(-epb), epb);
+  // (This kernel is built with the fused fast form only: with the multiply form as a third set of variants it ran
+  // 3 % slower on its main workload, for the sake of blocks with positive exponents, which take the defining form.)
+  const int mode_keys = lattice_mode_both(
+      lattice_mode_both(lattice_mode_fused_only(kmax, pow2f_exact(-eoa), eoa), lattice_mode_fused_only(kmax, pow2f_exact(-eob), eob)),
+      lattice_mode_fused_only(qa_max, pow2f_exact(-epa), epa));
+  const int mode_last = lattice_mode_fused_only(qb_max, pow2f_exact(-epb), epb);
   float spread, dmax, M, rho_b, M_b;
-  if (fast_keys && fast_last)
-    registers_decode<BITS, true, true>(nx, av, va, vb, vbh, pa, pb, prefix, eoa, eob, epa, epb, spread, dmax, M, rho_b, M_b);
-  else if (fast_keys)
-    registers_decode<BITS, true, false>(nx, av, va, vb, vbh, pa, pb, prefix, eoa, eob, epa, epb, spread, dmax, M, rho_b, M_b);
-  else
-    registers_decode<BITS, false, false>(nx, av, va, vb, vbh, pa, pb, prefix, eoa, eob, epa, epb, spread, dmax, M, rho_b, M_b);
+#define SWARM_CHAIN(MK, ML) registers_decode<BITS, MK, ML>(nx, av, va, vb, vbh, pa, pb, prefix, eoa, eob, epa, epb, spread, dmax, M, rho_b, M_b)
+  if (mode_keys == kFastFma && mode_last == kFastFma) SWARM_CHAIN(kFastFma, kFastFma);
+  else if (mode_keys == kFastFma) SWARM_CHAIN(kFastFma, kDefining);
+  else SWARM_CHAIN(kDefining, kDefining);
+#undef SWARM_CHAIN
   const int eo = exponent_rule<kOwnResolutionBits>(__fadd_rn(__fmul_rn(2.0f, spread), dmax), M);
   const int ep_b = exponent_rule<BITS>(rho_b, M_b);
 
   // own register of a (16 bits) and current register of b; distance of the new model to its own key
   const uint32_t group0 = (uint32_t)(blk * (kBlockCoords / 8) + lane);
   float rho_a, M_a;
-  if (fast_range(M, pow2f_exact(-eo), eo) && fast_range(M_b, pow2f_exact(-ep_b), ep_b))
-    registers_encode_own<BITS, true>(nx, av, oa, cb, group0, s, pd, lane, eo, ep_b, rho_a, M_a);
+  if (lattice_mode_both(lattice_mode_fused_only(M, pow2f_exact(-eo), eo), lattice_mode_fused_only(M_b, pow2f_exact(-ep_b), ep_b)) == kFastFma)
+    registers_encode_own<BITS, kFastFma>(nx, av, oa, cb, group0, s, pd, lane, eo, ep_b, rho_a, M_a);
   else
-    registers_encode_own<BITS, false>(nx, av, oa, cb, group0, s, pd, lane, eo, ep_b, rho_a, M_a);
+    registers_encode_own<BITS, kDefining>(nx, av, oa, cb, group0, s, pd, lane, eo, ep_b, rho_a, M_a);
   const int ep_a = exponent_rule<BITS>(rho_a, M_a);
-  if (fast_range(M_a, pow2f_exact(-ep_a), ep_a)) registers_encode_current<BITS, true>(nx, xa, ba, ca, group0, s, pd, lane, ep_a);
-  else registers_encode_current<BITS, false>(nx, xa, ba, ca, group0, s, pd, lane, ep_a);
+  if (lattice_mode_fused_only(M_a, pow2f_exact(-ep_a), ep_a) == kFastFma)
+    registers_encode_current<BITS, kFastFma>(nx, xa, ba, ca, group0, s, pd, lane, ep_a);
+  else
+    registers_encode_current<BITS, kDefining>(nx, xa, ba, ca, group0, s, pd, lane, ep_a);
   if (lane == 0) {
     s.oexps[(int64_t)pd.a * s.nblk + blk] = (int8_t)eo;
     s.exps[(int64_t)pd.a * s.nblk + blk] = (int8_t)ep_a;

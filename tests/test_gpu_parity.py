@@ -269,6 +269,51 @@ def test_one_way_interactions_across_magnitude_ratios(bits, mode):
         assert_store_equal(orc, gpu, bits)
 
 
+def _large_scale_models(n, d, rng):
+    """Models whose block ranges exceed the decoding window at step 1, so that lattice exponents are positive
+    (1 ... 40), with magnitudes from the range itself up to 2^20 times it; every block also holds zeros, subnormals
+    and tiny negative values, whose scaled values x * 2^-e are inexact products that round to -0 or to a subnormal."""
+    nblk = (d + 1023) // 1024
+    X = np.zeros((n, d), dtype=np.float32)
+    tiny = np.array([0.0, -0.0, 1e-45, -1e-45, 3e-42, -3e-42, 1e-39, -1e-39, -2e-38, 1e-30, -1e-30], dtype=np.float32)
+    for k in range(nblk):
+        lo, hi = k * 1024, min(d, (k + 1) * 1024)
+        spread = 2.0 ** (3 + 3 * (k % 13))
+        base = (-1.0) ** k * spread * 2.0 ** (2 * (k % 11))
+        X[:, lo:hi] = (base + spread * rng.normal(size=(n, hi - lo))).astype(np.float32)
+        idx = rng.choice(hi - lo, size=min(24, hi - lo), replace=False)
+        X[:, lo + idx] = tiny[rng.integers(0, len(tiny), size=(n, len(idx)))]
+    return X
+
+
+@pytest.mark.parametrize("mode", [0, 1, 2])
+@pytest.mark.parametrize("bits", [2, 4, 8])
+def test_interactions_with_positive_lattice_exponents(bits, mode):
+    """Blocks whose lattice step is 2, 4, ... 2^40: the scaled value is then no longer an exact product for tiny
+    coordinates, and the kernels must round it exactly as the definition does before taking the floor."""
+    n, d = 6, 14 * 1024 + 301
+    cfg = dict(objective=1, nonblocking=mode, grad_std=0.0, drift_std=0.0)
+    orc, gpu = make_pair(n, d, "complete", seed=8, **cfg)
+    rng = np.random.default_rng(700 + 10 * bits + mode)
+    orc.X[:] = _large_scale_models(n, d, rng)
+    if mode:
+        orc.B[:] = orc.X
+    inject(orc, gpu)
+    if mode:
+        publish = (lambda s_: s_.publish(bits)) if mode == 1 else (lambda s_: s_.register_publish(bits))
+        assert publish(orc) == 0 and publish(gpu) == 0
+        assert_store_equal(orc, gpu, bits)
+    assert int(orc.exps.max()) > 0 or mode == 0
+    for rnd in range(4):
+        if mode and rnd >= 1:                # pending updates, tiny coordinates included
+            orc.X[:] = (orc.X * (1.0 + np.float32(2.0 ** -(3 * rnd)) * rng.normal(size=orc.X.shape))).astype(np.float32)
+            inject(orc, gpu, what=("X",))
+        pairs = disjoint_pairs(orc, rng, 3)
+        assert orc.interact(pairs, bits, mode) == 0 and gpu.interact(pairs, bits, mode) == 0
+        assert_store_equal(orc, gpu, bits)
+    assert int(orc.exps.max()) > 3
+
+
 # ---- two-register protocol -----------------------------------------------------------------------
 
 @pytest.mark.parametrize("bits", [2, 3, 4, 5, 6, 7, 8])
