@@ -11,9 +11,17 @@ constexpr int kRedThreads = 128;
 constexpr int kPotentialMaxCtas = 148 * 16;   // one resident wave of 128-thread CTAs on 148 SMs
 constexpr int kRowUnroll = 8;
 
+// Programmatic dependent launch (see swarm_interact.cu): the two kernels below may become resident while their
+// predecessor in the stream drains; they touch no global memory before the wait returns.
+__device__ __forceinline__ void dependent_launch_prologue() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // mu[k]: rows summed in double in row order, divided by n, rounded once.
 __global__ void __launch_bounds__(kRedThreads)
 mean_model_kernel(StoreView s, float* __restrict__ out) {
+  dependent_launch_prologue();
   const int64_t c4 = (int64_t)blockIdx.x * kRedThreads + threadIdx.x;
   if (c4 * 4 >= s.d) return;
   const float* col = s.X + c4 * 4;
@@ -47,6 +55,7 @@ mean_model_kernel(StoreView s, float* __restrict__ out) {
 __global__ void __launch_bounds__(kRedThreads)
 potential_partial_kernel(StoreView s, double* __restrict__ partial, unsigned int* __restrict__ ticket,
                          double* __restrict__ out_dev, double* __restrict__ out_host) {
+  dependent_launch_prologue();
   double gamma = 0.0;
   // a fixed number of CTAs walks the column groups, so the sum of a CTA (and with it the result) depends on
   // the grid size only, and the last CTA has few partials to add up
@@ -245,18 +254,31 @@ cudaError_t launch_aux_potentials(const StoreView& s, const float* mu_hist, cons
 
 int64_t potential_partials(int64_t d) { return ((d + 3) / 4 + kRedThreads - 1) / kRedThreads; }
 
+template <typename Kernel, typename... Args>
+static cudaError_t launch_dependent(Kernel kernel, unsigned grid, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kRedThreads);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, args...);
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
 cudaError_t launch_mean_model(const StoreView& s, float* out_dev, cudaStream_t st, int* launches) {
-  mean_model_kernel<<<(unsigned)potential_partials(s.d), kRedThreads, 0, st>>>(s, out_dev);
   ++*launches;
-  return cudaGetLastError();
+  return launch_dependent(mean_model_kernel, (unsigned)potential_partials(s.d), st, s, out_dev);
 }
 
 cudaError_t launch_potential(const StoreView& s, double* partial_dev, unsigned int* ticket_dev, double* out_dev,
                              double* out_host_mapped, cudaStream_t st, int* launches) {
   const int64_t parts = std::min<int64_t>(potential_partials(s.d), kPotentialMaxCtas);
-  potential_partial_kernel<<<(unsigned)parts, kRedThreads, 0, st>>>(s, partial_dev, ticket_dev, out_dev, out_host_mapped);
   ++*launches;
-  return cudaGetLastError();
+  return launch_dependent(potential_partial_kernel, (unsigned)parts, st, s, partial_dev, ticket_dev, out_dev, out_host_mapped);
 }
 
 }  // namespace swarm
