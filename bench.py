@@ -31,6 +31,10 @@ WORKLOADS = {
     # n = 64 nodes, d = 2^20, ring, 32 disjoint pairs per launch, 4-bit codes, averaging only.
     "ring64_d1m_b4": dict(n=64, d=1 << 20, topology="ring", degree=0, pairs=32, bits=4, mode=0, H=0, lr=0.0, seed=2,
                           cfg=dict(offset_std=float(np.sqrt(0.1)))),
+    # the same store with the launches drawn by the library's pair sampler (Algorithm 1's draw with rejection of
+    # pairs that touch a node already paired in the launch: 27-28 of the 32 possible pairs on average)
+    "ring64_d1m_b4_sampled": dict(n=64, d=1 << 20, topology="ring", degree=0, pairs=32, bits=4, mode=0, H=0, lr=0.0, seed=2,
+                                  sampler=True, cfg=dict(offset_std=float(np.sqrt(0.1)))),
     # the same with code widths that do not divide a byte (codes regrouped into aligned words by warp shuffles)
     "ring64_d1m_b3": dict(n=64, d=1 << 20, topology="ring", degree=0, pairs=32, bits=3, mode=0, H=0, lr=0.0, seed=2,
                           cfg=dict(offset_std=float(np.sqrt(0.1)))),
@@ -117,14 +121,19 @@ def interaction_bytes(d, bits, mode, prefix=16):
 
 class PairSchedule:
     """Deterministic full matchings for the launch shapes of the workloads (host-side list making
-    only; the library validates disjointness and adjacency)."""
+    only; the library validates disjointness and adjacency). With `sampler` (an object with sample_pairs(P): the
+    CUDA context or the oracle) the launches are the method's own draws instead."""
 
-    def __init__(self, wl, adj):
+    def __init__(self, wl, adj, sampler=None):
         self.wl, self.adj, self.rng = wl, adj, np.random.default_rng(wl["seed"])
         self.step = 0
+        self.sampler = sampler if wl.get("sampler") else None
 
     def next(self):
         wl, n, P = self.wl, self.wl["n"], self.wl["pairs"]
+        if self.sampler is not None:
+            self.step += 1
+            return np.ascontiguousarray(self.sampler.sample_pairs(P), dtype=np.int32)
         if wl["topology"] == "ring":
             parity = self.step & 1
             flips = self.rng.integers(0, 2, P)
@@ -254,7 +263,7 @@ def time_oracle(wl, budget_s, max_launches, threads=None):
     orc = o.OracleSwarm(wl["n"], wl["d"], wl["topology"], wl["degree"], wl["seed"])
     if wl["cfg"]:
         orc.configure(**wl["cfg"])
-    sched = PairSchedule(wl, orc.adj)
+    sched = PairSchedule(wl, orc.adj, orc)
     done, t_total, launches = 0, 0.0, 0
     while launches < max_launches and (t_total < budget_s or launches == 0):
         pairs = sched.next()[:P]
@@ -282,7 +291,7 @@ def run_reference(args, wl, name):
     orc = o.OracleSwarm(wl["n"], wl["d"], wl["topology"], wl["degree"], wl["seed"])
     if wl["cfg"]:
         orc.configure(**wl["cfg"])
-    sched = PairSchedule(wl, orc.adj)
+    sched = PairSchedule(wl, orc.adj, orc)
 
     def step(p, T):
         pairs = sched.next()[:p]
@@ -369,7 +378,7 @@ class Runner:
         self.sw = g.Swarm(wl["n"], wl["d"], wl["topology"], wl["degree"], wl["seed"] + seed_shift, stream=stream)
         if wl["cfg"]:
             self.sw.configure(**wl["cfg"])
-        self.sched = PairSchedule(wl, self.sw.get_all(g.T_ADJ))
+        self.sched = PairSchedule(wl, self.sw.get_all(g.T_ADJ), self.sw)
         # elementwise (synthetic) objective: the nodes of the pairs step inside the interaction kernel (swarm_step),
         # unless two calls per step are asked for
         self.fused = bool(wl["H"] > 0 and wl["cfg"].get("objective") == 1 and not wl.get("step_all")
@@ -467,7 +476,8 @@ class Runner:
         """The same steps through the public binding with host buffers inside the timed region: every step's pair
         list comes from pinned host memory, a result of every step (the block exponents that the first initiator
         published) is read back to pinned host memory, and the potential is read (synchronising, which also delivers
-        the queued rows) every 32 steps. Runs for at least `seconds` and at least len(launches) steps.
+        the queued rows) every 1000 interactions, at least every 32 steps. Runs for at least `seconds` and at least
+        len(launches) steps.
         Returns (pairs processed, ms, host-to-device bytes per step, device-to-host bytes per step)."""
         g, torch, wl, sw, stream = self.g, self.torch, self.wl, self.sw, self.stream
         nblk = (wl["d"] + 1023) // 1024
@@ -508,19 +518,23 @@ class Runner:
         steps = max(-(-len(launches) // chunk), int(seconds / per_step) + 1)
         steps = min((steps + 31) // 32 * 32, 200000)          # whole groups of 32: the last potential read ends the run
         barrier()
-        done = h2d = d2h = checksum = 0
+        done = h2d = d2h = checksum = since = reads = 0
         t0 = time.perf_counter()
         ev0.record(stream)
         for i in range(steps):
             dn, nb = one(i + 33)
             done += dn
+            since += dn
             h2d += nb
             d2h += nblk
-            if i % 32 == 31:
+            if since >= 1000 or i % 32 == 31:
                 sw.potential()
+                since = 0
+                reads += 1
                 d2h += 8
                 checksum += int(ring.sum())
         ev1.record(stream)
+        self.potential_reads_per_step = reads / steps
         barrier()
         ms = max(ev0.elapsed_time(ev1), (time.perf_counter() - t0) * 1e3)
         return done, ms, h2d / steps, d2h / steps, steps
@@ -632,7 +646,8 @@ def run_ours(args, wl, name):
            "calls_per_step": ("swarm_run_sequence (64 time steps per call)" if sequence else
                               ("swarm_step" if fused else ("swarm_local_steps, swarm_interact" if wl["H"] > 0
                                                            else "swarm_interact")))
-           + ", swarm_get_tensor_async; swarm_potential every 32 steps"}
+           + ", swarm_get_tensor_async; swarm_potential every 1000 interactions (%.3f reads per step)"
+           % r.potential_reads_per_step}
 
     traffic = traffic_of(name, kern_pairs)
     roofline = {"bound": "hbm", "kernel": kernel_name(wl, fused),

@@ -212,3 +212,31 @@ def test_config5_full_size_tensor_core_steps_on_the_last_data_matrix():
         assert rel_err(got, orc.X[j]) < 1e-6, node
     assert gpu._L.swarm_get_data_rows(gpu._h, groups, 0, 1, x0[0].ctypes.data, d * 4) == g.ERANGE
     assert gpu._L.swarm_get_data_rows(gpu._h, 0, m, 1, x0[0].ctypes.data, d * 4) == g.ERANGE
+
+
+@pytest.mark.parametrize("workload", ["regular32_resnet18_b8_nb", "complete16_resnet50_b4", "complete16_resnet50_b8"])
+def test_one_call_step_equals_the_two_calls_at_the_full_store(workload):
+    """The benchmark runs these workloads through swarm_step (local steps inside the interaction kernel). At the
+    full store and with the benchmark's own launch lists, three such steps must leave every model, snapshot, buffer
+    and counter of the swarm bit-identical to swarm_local_steps + swarm_interact, which the tests above tie to the
+    oracle."""
+    import bench
+    wl = bench.WORKLOADS[workload]
+    n, d, bits, mode = wl["n"], wl["d"], wl["bits"], wl["mode"]
+    one = g.Swarm(n, d, wl["topology"], wl["degree"], wl["seed"])
+    two = g.Swarm(n, d, wl["topology"], wl["degree"], wl["seed"])
+    one.configure(**wl["cfg"])
+    two.configure(**wl["cfg"])
+    sched = bench.PairSchedule(wl, one.get_all(g.T_ADJ))
+    for _ in range(3):
+        pairs = sched.next()
+        assert two.local_steps(pairs.reshape(-1), wl["H"], wl["lr"]) == 0
+        assert two.interact(pairs, bits, mode) == 0
+        before = one.kernel_launches()
+        assert one.step(pairs, wl["H"], wl["lr"], bits, mode, True) == 0
+    assert one.kernel_launches() - before == 1
+    rows = (g.T_X, g.T_CODES, g.T_EXPS, g.T_COUNTERS) + ((g.T_B,) if mode else ())
+    for i in range(n):
+        for which in rows:
+            assert np.array_equal(one.get(which, i).view(np.uint8), two.get(which, i).view(np.uint8)), (which, i)
+    assert one.potential() == two.potential()
