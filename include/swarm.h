@@ -114,6 +114,12 @@ int swarm_init(swarm_ctx **out, int32_t n, int64_t d, swarm_topology topo, uint6
  * gradient steps of size lr on its own objective, every gradient evaluated at the running
  * iterate (\tilde h^q = \tilde g_i(X - sum_{s<q} lr \tilde h^s)); the steps are applied in
  * place to X^i. node_ids_host: `count` distinct ids (host). H >= 0.
+ * Least squares and logistic regression on bf16 data with minibatches of at most 64 rows: the rows of a
+ * node's next steps are known in advance and a step moves the model along its sampled rows only, so up to
+ * four consecutive steps are evaluated from one pass over the model (their scores <a, x> against the model
+ * before the first of them, corrected step by step with inner products of data rows, which the library keeps
+ * as the data matrices' Gram matrices when these take at most 256 MiB) and applied in one pass. The iterates
+ * are the same sequential ones; the model is rounded to fp32 once per group instead of once per step.
  * Errors: ESTATE (no objective), EINVAL (H < 0, count < 0, duplicate id), ERANGE. */
 int swarm_local_steps(swarm_ctx *ctx, const int32_t *node_ids_host, int32_t count, int32_t H, float lr);
 

@@ -69,6 +69,7 @@ struct swarm_ctx {
   float* lsq_partial = nullptr;      // n * batch * chunks
   float* tc_partial = nullptr;       // tensor-core path: split-K partials of the residuals
   void* tc_resid = nullptr;          // tensor-core path: residuals as bf16 hi / lo
+  float* gram = nullptr;             // tensor-core path: Gram matrices of the data matrices (nullptr: not kept)
   int* kernel_status = nullptr;      // set by a kernel whose bounded wait expired
   int* kernel_status_host = nullptr; // pinned
   bool status_pending = false;       // kernels with bounded waits were launched since the status word was last read
@@ -170,7 +171,7 @@ StoreView view_of(const swarm_ctx* c) {
 }
 LsqView lsq_of(const swarm_ctx* c) {
   LsqView l;
-  l.A = c->A; l.bvec = c->bvec; l.m = c->cfg.lsq_m; l.batch = c->cfg.lsq_batch; l.dtype = c->cfg.lsq_dtype;
+  l.A = c->A; l.bvec = c->bvec; l.gram = c->gram; l.m = c->cfg.lsq_m; l.batch = c->cfg.lsq_batch; l.dtype = c->cfg.lsq_dtype;
   l.groups = c->groups; l.nodes_per_group = c->nodes_per_group;
   l.logistic = c->cfg.objective == SWARM_OBJ_LOGISTIC ? 1 : 0;
   return l;
@@ -242,6 +243,7 @@ void free_objective(swarm_ctx* c) {
   dev_free(c, c->lsq_partial); c->lsq_partial = nullptr;
   dev_free(c, c->tc_partial); c->tc_partial = nullptr;
   dev_free(c, c->tc_resid); c->tc_resid = nullptr;
+  dev_free(c, c->gram); c->gram = nullptr;
   dev_free(c, c->convert_tmp); c->convert_tmp = nullptr;
   dev_free(c, c->B); c->B = nullptr;
   dev_free(c, c->own); c->own = nullptr;
@@ -302,6 +304,11 @@ int alloc_objective(swarm_ctx* c, const swarm_config& cfg) {
       c->tc_partial = (float*)dev_alloc(c, lsq_tc_partial_bytes(c->pitch, n));
       c->tc_resid = dev_alloc(c, lsq_tc_resid_bytes(n));
       if (!c->tc_partial || !c->tc_resid) return SWARM_ENOMEM;
+      const size_t gram_bytes = lsq_tc_gram_bytes(c->groups, cfg.lsq_m);
+      if (gram_bytes) {
+        c->gram = (float*)dev_alloc(c, gram_bytes);
+        if (!c->gram) return SWARM_ENOMEM;
+      }
     }
   }
   return SWARM_OK;
@@ -347,6 +354,7 @@ int apply_config(swarm_ctx* c, const swarm_config& wanted) {
   if (cfg.objective == SWARM_OBJ_LSQ || cfg.objective == SWARM_OBJ_LOGISTIC) {
     LsqView l = lsq_of(c);
     SW_CUDA(c, launch_lsq_data(s, l, c->A, c->xstar, c->bvec, c->scalars, cfg.lsq_noise_std, c->stream, &nl));
+    SW_CUDA(c, launch_lsq_gram(c->A, cfg.lsq_m, c->pitch, 0, c->groups, c->gram, c->stream, &nl));
   }
   c->launches += nl;
   std::fill(c->w.begin(), c->w.end(), 0u);
@@ -1164,6 +1172,8 @@ static int tensor_access(swarm_ctx* c, int32_t which, int32_t node, void* host, 
           SW_SYNC(c);   // convert_tmp and pageable host memory are reused per row
         }
       }
+      // rewritten rows change the matrix's Gram matrix, which the grouped local steps read
+      if (write) SW_CUDA(c, launch_lsq_gram(c->A, c->cfg.lsq_m, c->pitch, node, 1, c->gram, c->stream, &nl));
       c->launches += nl;
       SW_SYNC(c);
       return SWARM_OK;

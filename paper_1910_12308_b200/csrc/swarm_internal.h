@@ -98,6 +98,7 @@ inline void division_magic(uint64_t divisor, uint32_t* magic, uint32_t* shift) {
 struct LsqView {
   const void* A;       // [groups][m][pitch] fp32 or bf16
   const float* bvec;   // [n][m]
+  const float* gram;   // [groups][m][m] Gram matrices A A^T of the bf16 data matrices, or nullptr when not kept
   int32_t m, batch, dtype, groups, nodes_per_group;
   int32_t logistic;    // 1: residual = sigmoid(<a, x>) - y with labels in {0, 1}; 0: residual = <a, x> - b
 };
@@ -138,6 +139,13 @@ cudaError_t launch_lsq_sequence(const StoreView& s, const LsqView& l, const Pair
 // --- swarm_lsq_tc.cu (bf16 data, batch <= 64) ----------------------------------------------
 size_t lsq_tc_partial_bytes(int64_t pitch, int units);
 size_t lsq_tc_resid_bytes(int units);
+// Bytes of the Gram matrices of `matrices` data matrices of m rows; 0 when they are too large to keep (local steps
+// then go one at a time instead of in groups).
+size_t lsq_tc_gram_bytes(int matrices, int m);
+// gram_dev[first_matrix .. first_matrix + matrices) = A A^T of those bf16 data matrices (row padding must be zero).
+cudaError_t launch_lsq_gram(const void* A_dev, int m, int64_t pitch, int first_matrix, int matrices, float* gram_dev,
+                            cudaStream_t st, int* launches);
+// H steps of every unit, in groups of up to four steps per pair of passes when l.gram is set (one step otherwise).
 // status_dev: one int, set to 1 if a bounded wait inside a kernel expired (kernels that find it set return at
 // once); wait_limit: polls after which a wait on a tensor-core commit gives up.
 cudaError_t launch_local_lsq_tc(const StoreView& s, const LsqView& l, const LsqUnit* units_dev, int nunits, int H,

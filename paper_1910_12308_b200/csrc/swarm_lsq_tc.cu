@@ -4,22 +4,35 @@
 // Section 3, "The Communication Procedure": x <- x - lr * g~(x), g~ = (1/B) sum_s (<a_s, x> - b_s) a_s
 // over the B sampled rows a_s. For a unit of up to 16 nodes with the same rows this is two skinny
 // contractions per step:
-//   residuals  R[s][j] = sum_k A[r_s][k] * X_j[k]          (64 x 16 output, K = d)
+//   scores     P[s][j] = sum_k A[r_s][k] * X_j[k]          (64 x 16 output, K = d)
 //   update     X_j[k] -= (lr/B) * sum_s resid[s][j] A[r_s][k]   (d x 16 output, K = 64)
 // Both stream the sampled rows once per unit (instead of once per node) and are HBM-bound; the
 // tensor cores keep the 2*64*16 flops per coordinate off the critical path.
 //
+// Steps in groups. A node's G consecutive steps q = 0 .. G-1 (G <= 4) draw row sets S_q that are known in
+// advance, and each step moves x along the sampled rows only: x_q = x_0 - (lr/B) sum_{p<q} A_{S_p}^T resid_p.
+// The scores of step q are therefore
+//   A_{S_q} x_q = A_{S_q} x_0 - (lr/B) sum_{p<q} (A_{S_q} A_{S_p}^T) resid_p,
+// where A_{S_q} A_{S_p}^T is a 64 x 64 block of the data matrix's Gram matrix A A^T (m x m, a constant of
+// the data, computed once when the data is made). One pass over the models then gives the scores of all G
+// steps against x_0, a small kernel walks the recursion, and one pass applies all G updates:
+// (G * rows + models) + (G * rows + 2 * models) bytes instead of G * (2 * rows + 3 * models).
+// The result differs from G separately rounded steps only in rounding (the models are rounded once instead
+// of G times). Without a Gram matrix (too large to keep) G = 1.
+//
 // Precision: fp32 operands are split into bf16 hi + bf16 lo (x = hi + lo up to 2^-17 relative), both
 // halves multiplied against the same data tile, accumulated in fp32.
 //
-// Three kernels per step:
-//   lsq_tc_residual_kernel  CTA = (k-chunk, unit): split-K partial R into scratch
-//   lsq_tc_finalize_kernel  CTA = unit: sums the chunk partials in chunk order, subtracts labels,
-//                           writes resid as bf16 hi/lo
-//   lsq_tc_update_kernel    CTA = (k-chunk, unit): D = A_S^T resid per 128-coordinate tile, x -= scale * D
+// Three kernels per group of steps:
+//   lsq_tc_scores_kernel    CTA = (k-chunk, unit): split-K partial scores of the G steps into scratch
+//   lsq_tc_finalize_kernel  CTA = unit: sums the chunk partials in chunk order, applies the Gram
+//                           corrections step by step, subtracts labels, writes resid as bf16 hi/lo
+//   lsq_tc_update_kernel    CTA = (k-chunk, unit): D = sum_q A_{S_q}^T resid_q per 128-coordinate tile,
+//                           x -= scale * D
 // Operand tiles are staged with cp.async into the 128-byte-swizzled shared-memory layouts the MMA
-// descriptors name. Every wait on an mbarrier is bounded (spin_limit polls). A wait's outcome is made
-// warp-uniform by a vote and CTA-uniform at the tile loop's barrier, so all threads of a CTA leave the loop
+// descriptors name; a stage holds the rows of one step for one tile, and the stages of a tile follow one
+// another. Every wait on an mbarrier is bounded (spin_limit polls). A wait's outcome is made
+// warp-uniform by a vote and CTA-uniform at the stage loop's barrier, so all threads of a CTA leave the loop
 // together; the CTA then raises the status word, drains its copies, waits (bounded by the full default limit,
 // whatever spin_limit says) for the last MMA commit so that no MMA is in flight, frees its tensor memory and
 // returns without writing results. Kernels that find the status word set on entry return at once, so a step
@@ -131,14 +144,35 @@ __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bflo
 
 }  // namespace
 
+constexpr int kTcMaxGroup = 4;            // steps folded into one pair of passes
+
+// The rows of steps step0 .. step0 + G - 1 of a unit (slots beyond the batch size hold row 0 and are never read
+// as data: their tiles are zero and their residuals are zero).
+template <int G>
+__device__ __forceinline__ void draw_rows(int* rows, const LsqView& l, int group, uint32_t event0, const StoreView& s) {
+  for (int i = threadIdx.x; i < G * kTcBatch; i += blockDim.x) {
+    const int q = i / kTcBatch, sidx = i % kTcBatch;
+    rows[i] = sidx < l.batch ? tc_minibatch_row(sidx, group, event0 + (uint32_t)q, l.m, s.key0, s.key1) : 0;
+  }
+}
+
 // =================================================================================================
-// Residual partials. Tile = 128 coordinates (2 swizzle atoms of 64). Shared memory per stage:
+// Score partials. Tile = 128 coordinates (2 swizzle atoms of 64). Shared memory per stage:
 //   A    : 2 atoms x [64 rows x 128 B]   (K-major, 128B swizzle, 8-row groups 1024 B apart)  16 KiB
-// plus two operand buffers Xhi/Xlo: 2 atoms x [16 rows x 128 B] each. The fp32 models are loaded one
+// plus two operand buffers of 2 atoms x [32 rows x 128 B]: rows 0..15 the bf16 hi halves of the 16 nodes' models,
+// rows 16..31 the lo halves, so that one MMA (N = 32) multiplies a data tile against both; the two products are
+// added in the epilogue. Stage f holds the rows of step f % G for tile f / G; the model tile is converted once
+// per tile and multiplied against the G stages of the tile, step q accumulating into tensor-memory columns
+// 32 q .. 32 q + 31. The MMAs of a stage are issued after the copies of a later stage, so that the issuing thread's
+// warp does not fall behind with its copies. The fp32 models are loaded one
 // tile ahead into registers (8 coordinates per thread) and converted to bf16 hi/lo straight into the
 // operand buffers. Three stages of A: 65 KiB per CTA, three CTAs per SM, so that one CTA's barrier and
-// operand conversion hide behind the copies of the other two (measured against five stages and two CTAs per
-// SM at the 256-node workload: 5 % off the whole step).
+// operand conversion hide behind the copies of the other two. (Measured on the 256-node workload and dropped: a
+// fourth stage with a single operand buffer, which each new tile must wait for, 3 % slower; L2 prefetches of the
+// rows of a stage 2 to 8 stages further on, 6 % slower.)
+// Order of completion: the wait at the end of iteration f covers the commit of stage f - 1, and commits complete
+// in order; so when iteration f starts, every MMA up to stage f - 2 has completed, among them (G >= 1) all that
+// read the operand buffer which a new tile is about to overwrite (the tile two before).
 // =================================================================================================
 constexpr int kResTile = 128;
 constexpr int kResAtoms = kResTile / 64;
@@ -147,9 +181,11 @@ constexpr int kResABytes = kResAtoms * kTcBatch * 128;         // 16384
 constexpr int kResXopBytes = kResAtoms * kUnitNodes * 128;     // 4096 (one of hi / lo)
 constexpr int kResSmem = kResStages * kResABytes + 2 * 2 * kResXopBytes + 1024 /*align*/ + 64;
 
+template <int G>
 __global__ void __launch_bounds__(kTcThreads, 3)
-lsq_tc_residual_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, int step, float* __restrict__ partial,
-                       int64_t chunk_coords, int64_t nchunks, int* __restrict__ status, uint32_t spin_limit) {
+lsq_tc_scores_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, int step, float* __restrict__ partial,
+                     int64_t chunk_coords, int64_t nchunks, int* __restrict__ status, uint32_t spin_limit) {
+  constexpr uint32_t kCols = G == 1 ? 32 : G == 2 ? 64 : 128;   // tensor-memory columns: 32 per step, a power of two
   __shared__ int poisoned;
   if (status_raised(status, &poisoned)) return;
   extern __shared__ uint8_t smem_raw[];
@@ -158,26 +194,26 @@ lsq_tc_residual_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units
   uint8_t* sXop = sA + kResStages * kResABytes;                 // [buf][hi|lo]
   uint64_t* bars = (uint64_t*)(sXop + 4 * kResXopBytes);        // mma_done[2]
   uint32_t* tmem_slot = (uint32_t*)(bars + 2);
-  __shared__ int rows[kTcBatch];
+  __shared__ int rows[G * kTcBatch];
   __shared__ int unodes[kUnitNodes];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const LsqUnit* up = units + blockIdx.y;
   struct { int group, count; } u = {up->group, up->count};
-  const uint32_t event = up->event + (uint32_t)step;
   if (tid < kUnitNodes) unodes[tid] = up->nodes[tid];
   const int64_t kbase = (int64_t)blockIdx.x * chunk_coords;
   const int64_t kend = min(kbase + chunk_coords, s.pitch);
   const int ntiles = (int)((kend - kbase) / kResTile);
+  const int nstages = ntiles * G;
   const __nv_bfloat16* A = reinterpret_cast<const __nv_bfloat16*>(l.A) + (int64_t)u.group * l.m * s.pitch;
 
-  if (tid < kTcBatch) rows[tid] = tid < l.batch ? tc_minibatch_row(tid, u.group, event, l.m, s.key0, s.key1) : 0;
+  draw_rows<G>(rows, l, u.group, up->event + (uint32_t)step, s);
   if (tid == 0) {
     mbar_init(smem_u32(&bars[0]), 1);
     mbar_init(smem_u32(&bars[1]), 1);
     fence_mbar_init();
   }
-  if (warp == 0) { tmem_alloc(smem_u32(tmem_slot), 32); tmem_relinquish(); }
+  if (warp == 0) { tmem_alloc(smem_u32(tmem_slot), kCols); tmem_relinquish(); }
   // rows of the minibatch tile beyond the batch size are never copied: they must read as zero
   if (l.batch < kTcBatch)
     for (int i = tid; i < kResStages * kResABytes / 16; i += kTcThreads) reinterpret_cast<uint4*>(sA)[i] = make_uint4(0, 0, 0, 0);
@@ -186,9 +222,10 @@ lsq_tc_residual_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units
   tc_fence_after();
   const uint32_t tmem_d = *tmem_slot;
 
-  auto issue_loads = [&](int tile) {
-    if (tile < ntiles) {
-      const int st = tile % kResStages;
+  auto issue_loads = [&](int f) {
+    if (f < nstages) {
+      const int tile = f / G, q = f - tile * G;
+      const int st = f % kResStages;
       const int64_t k0 = kbase + (int64_t)tile * kResTile;
       // A: 64 rows x 16 chunks of 16 B; thread -> (row = idx / 16, chunk = idx % 16)
       const uint32_t a_base = smem_u32(sA + st * kResABytes);
@@ -199,7 +236,7 @@ lsq_tc_residual_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units
         if (r < l.batch) {
           const int atom = c >> 3, cc = c & 7;
           const uint32_t dst = a_base + atom * (kTcBatch * 128) + (r >> 3) * 1024 + (r & 7) * 128 + ((cc ^ (r & 7)) << 4);
-          cp_async16(dst, A + (int64_t)rows[r] * s.pitch + k0 + c * 8);
+          cp_async16(dst, A + (int64_t)rows[q * kTcBatch + r] * s.pitch + k0 + c * 8);
         }
       }
     }
@@ -219,60 +256,61 @@ lsq_tc_residual_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units
   };
 
   bool ok = true;                  // this warp's waits so far
-  int committed = -1;              // last tile whose MMAs were committed (the same in every thread)
-  for (int t = 0; t < kResStages - 1; ++t) issue_loads(t);
-  constexpr uint32_t idesc = instr_desc_bf16(kTcBatch, kUnitNodes, 0, 0);
+  int committed = -1;              // last stage whose MMAs were committed (the same in every thread)
+  for (int f = 0; f < kResStages - 1; ++f) issue_loads(f);
+  constexpr uint32_t idesc = instr_desc_bf16(kTcBatch, 2 * kUnitNodes, 0, 0);   // N = 32: hi and lo side by side
   float4 xcur[2], xnext[2];
   load_x(0, xcur);
-  for (int t = 0; t < ntiles; ++t) {
-    const int st = t % kResStages, buf = t & 1;
-    load_x(t + 1, xnext);                                   // consumed one iteration later
-    cp_async_wait<kResStages - 2>();                        // this thread's copies of tile t have landed
-    if (t >= 2) ok = mbar_wait(smem_u32(&bars[buf]), ((t >> 1) - 1) & 1, spin_limit) && ok;   // operand buffer free again
-    // fp32 -> bf16 hi/lo into the swizzled operand layout
-    {
+  for (int f = 0; f < nstages; ++f) {
+    const int t = f / G, q = f - t * G;
+    const int st = f % kResStages, buf = t & 1;
+    if (q == 0) load_x(t + 1, xnext);                       // consumed one tile later
+    cp_async_wait<kResStages - 2>();                        // this thread's copies of stage f have landed
+    if (q == 0 && ok) {
+      // fp32 -> bf16 hi/lo into the swizzled operand layout
       const int r = xr, c8 = xc8;                           // c8: group of 8 coordinates = one 16-byte bf16 chunk
       __align__(16) __nv_bfloat16 hi[8], lo[8];
 #pragma unroll
-      for (int q = 0; q < 2; ++q) {
-        const float4 v = xcur[q];
-        split_bf16(v.x, hi[q * 4 + 0], lo[q * 4 + 0]);
-        split_bf16(v.y, hi[q * 4 + 1], lo[q * 4 + 1]);
-        split_bf16(v.z, hi[q * 4 + 2], lo[q * 4 + 2]);
-        split_bf16(v.w, hi[q * 4 + 3], lo[q * 4 + 3]);
+      for (int p = 0; p < 2; ++p) {
+        const float4 v = xcur[p];
+        split_bf16(v.x, hi[p * 4 + 0], lo[p * 4 + 0]);
+        split_bf16(v.y, hi[p * 4 + 1], lo[p * 4 + 1]);
+        split_bf16(v.z, hi[p * 4 + 2], lo[p * 4 + 2]);
+        split_bf16(v.w, hi[p * 4 + 3], lo[p * 4 + 3]);
       }
+      // operand rows 0..15 = hi of the 16 nodes, rows 16..31 = lo (two 8-row groups further on)
       const int atom = c8 >> 3, cc = c8 & 7;
-      const int off = atom * (kUnitNodes * 128) + (r >> 3) * 1024 + (r & 7) * 128 + ((cc ^ (r & 7)) << 4);
-      *reinterpret_cast<uint4*>(sXop + (buf * 2 + 0) * kResXopBytes + off) = *reinterpret_cast<const uint4*>(hi);
-      *reinterpret_cast<uint4*>(sXop + (buf * 2 + 1) * kResXopBytes + off) = *reinterpret_cast<const uint4*>(lo);
+      const int off = buf * (2 * kResXopBytes) + atom * (2 * kUnitNodes * 128) + (r >> 3) * 1024 + (r & 7) * 128 +
+                      ((cc ^ (r & 7)) << 4);
+      *reinterpret_cast<uint4*>(sXop + off) = *reinterpret_cast<const uint4*>(hi);
+      *reinterpret_cast<uint4*>(sXop + off + 2048) = *reinterpret_cast<const uint4*>(lo);
+      xcur[0] = xnext[0]; xcur[1] = xnext[1];
     }
     fence_proxy_async();                                    // generic-proxy writes (cp.async, st.shared) -> MMA reads
     tc_fence_before();
     ok = __syncthreads_and(ok);                             // the loop's one barrier also makes the give-up decision CTA-uniform
     if (!ok) break;
+    // refill the stage that stage f-1 used (its MMAs were committed one iteration ago) before this stage's MMAs
+    // are issued, so that the issue does not hold back warp 0's copies; a warp whose wait expired leaves that stage
+    // alone and reports at the next barrier
+    if (f >= 1) ok = mbar_wait(smem_u32(&bars[(f - 1) & 1]), ((f - 1) >> 1) & 1, spin_limit);
+    if (ok) issue_loads(f + kResStages - 1); else cp_async_commit();
     if (tid == 0) {
       tc_fence_after();
       const uint32_t a_base = smem_u32(sA + st * kResABytes);
-      const uint32_t h_base = smem_u32(sXop + (buf * 2 + 0) * kResXopBytes);
-      const uint32_t l_base = smem_u32(sXop + (buf * 2 + 1) * kResXopBytes);
+      const uint32_t x_base = smem_u32(sXop + buf * (2 * kResXopBytes));
+      const uint32_t d_addr = tmem_d + (uint32_t)(q * 2 * kUnitNodes);
 #pragma unroll
       for (int atom = 0; atom < kResAtoms; ++atom)
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks) {                    // 16 coordinates (32 bytes) per MMA
           const uint64_t da = smem_desc_sw128(a_base + atom * (kTcBatch * 128) + ks * 32, 16, 1024);
-          const uint64_t dh = smem_desc_sw128(h_base + atom * (kUnitNodes * 128) + ks * 32, 16, 1024);
-          const uint64_t dl = smem_desc_sw128(l_base + atom * (kUnitNodes * 128) + ks * 32, 16, 1024);
-          tc_mma(tmem_d, da, dh, idesc, (t | atom | ks) != 0);
-          tc_mma(tmem_d, da, dl, idesc, 1);
+          const uint64_t dx = smem_desc_sw128(x_base + atom * (2 * kUnitNodes * 128) + ks * 32, 16, 1024);
+          tc_mma(d_addr, da, dx, idesc, (t | atom | ks) != 0);
         }
-      tc_commit(smem_u32(&bars[buf]));
+      tc_commit(smem_u32(&bars[f & 1]));
     }
-    committed = t;
-    // refill the stage that tile t-1 used (its MMAs were committed one iteration ago); a warp whose wait
-    // expired leaves that stage alone and reports at the next barrier
-    if (t >= 1) ok = mbar_wait(smem_u32(&bars[(t - 1) & 1]), ((t - 1) >> 1) & 1, spin_limit);
-    if (ok) issue_loads(t + kResStages - 1); else cp_async_commit();
-    xcur[0] = xnext[0]; xcur[1] = xnext[1];
+    committed = f;
   }
   cp_async_wait<0>();
   if (ok && committed >= 0) ok = mbar_wait(smem_u32(&bars[committed & 1]), (committed >> 1) & 1, spin_limit);
@@ -285,112 +323,169 @@ lsq_tc_residual_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units
     if (committed >= 0) mbar_wait(smem_u32(&bars[committed & 1]), (committed >> 1) & 1, kSpinLimit);
   }
   tc_fence_after();
-  // accumulator rows 16q..16q+15 live in lanes 32q..32q+15: warps 0..3, lanes 0..15
+  // accumulator rows 16w..16w+15 live in lanes 32w..32w+15: warps 0..3, lanes 0..15
   if (warp < 4) {
-    float v[16];
-    tmem_ld8(tmem_d + ((uint32_t)(warp * 32) << 16), v);
-    tmem_ld8(tmem_d + ((uint32_t)(warp * 32) << 16) + 8, v + 8);
-    if (lane < 16 && ok) {
-      float* dst = partial + (((int64_t)blockIdx.y * nchunks + blockIdx.x) * kTcBatch + warp * 16 + lane) * kUnitNodes;
 #pragma unroll
-      for (int q = 0; q < 4; ++q)
-        reinterpret_cast<float4*>(dst)[q] = ntiles > 0 ? make_float4(v[q * 4], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3])
-                                                       : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int q = 0; q < G; ++q) {
+      float v[16], w[16];                                   // products with the hi halves, with the lo halves
+#pragma unroll
+      for (int p = 0; p < 2; ++p) {
+        tmem_ld8(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)(q * 2 * kUnitNodes + p * 8), v + p * 8);
+        tmem_ld8(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)(q * 2 * kUnitNodes + kUnitNodes + p * 8), w + p * 8);
+      }
+#pragma unroll
+      for (int p = 0; p < 16; ++p) v[p] += w[p];
+      if (lane < 16 && ok) {
+        float* dst = partial +
+                     ((((int64_t)blockIdx.y * nchunks + blockIdx.x) * G + q) * kTcBatch + warp * 16 + lane) * kUnitNodes;
+#pragma unroll
+        for (int p = 0; p < 4; ++p)
+          reinterpret_cast<float4*>(dst)[p] = ntiles > 0 ? make_float4(v[p * 4], v[p * 4 + 1], v[p * 4 + 2], v[p * 4 + 3])
+                                                         : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
     }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem_d, 32);
+  if (warp == 0) tmem_dealloc(tmem_d, kCols);
 }
 
 // =================================================================================================
-// Finalize: resid[s][j] = sum over chunks (in chunk order) - label, stored K-major per node as bf16
-// hi / lo: R[unit][hi|lo][j][s].
+// Finalize, one CTA per unit, thread = (sampled row s, node j). For step q = 0 .. G-1 in turn:
+//   score[s][j] = sum over chunks (in chunk order) of the partials of step q
+//                 - scale * sum_{p<q} sum_{s'} gram[row_q[s]][row_p[s']] * resid_p[s'][j]
+//   resid_q[s][j] = score - label (least squares) or sigmoid(score) - label (logistic)
+// stored K-major per node as bf16 hi / lo: R[unit][q][hi|lo][j][s]. The corrections use the residuals as the
+// update kernel will see them (hi + lo).
 // =================================================================================================
 __global__ void __launch_bounds__(kTcBatch * kUnitNodes)
-lsq_tc_finalize_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, int step, const float* __restrict__ partial,
-                       int64_t nchunks, __nv_bfloat16* __restrict__ resid, const int* __restrict__ status) {
+lsq_tc_finalize_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, int step, int G, float scale,
+                       const float* __restrict__ partial, int64_t nchunks, __nv_bfloat16* __restrict__ resid,
+                       const int* __restrict__ status) {
   if (*reinterpret_cast<const volatile int*>(status) != 0) return;    // the partials of a step that gave up are not complete
+  __shared__ int rows[kTcMaxGroup * kTcBatch];
+  __shared__ float seen[kTcMaxGroup - 1][kTcBatch][kUnitNodes];       // residuals of the earlier steps of the group
+  __shared__ float block[kTcBatch][kTcBatch + 1];                     // one 64 x 64 block of the Gram matrix
   const LsqUnit u = units[blockIdx.x];
   const int sidx = threadIdx.x / kUnitNodes, j = threadIdx.x % kUnitNodes;
-  const float* p = partial + (int64_t)blockIdx.x * nchunks * (kTcBatch * kUnitNodes) + threadIdx.x;
-  float acc = 0.0f;
-#pragma unroll 8
-  for (int64_t c = 0; c < nchunks; ++c) acc += p[c * (kTcBatch * kUnitNodes)];   // chunk order: fixed summation order
-  float r = 0.0f;
-  if (sidx < l.batch && j < u.count) {
-    const int row = tc_minibatch_row(sidx, u.group, u.event + (uint32_t)step, l.m, s.key0, s.key1);
-    r = row_residual(acc, l.bvec[(int64_t)u.nodes[j] * l.m + row], l.logistic);
+  for (int i = threadIdx.x; i < G * kTcBatch; i += blockDim.x) {
+    const int q = i / kTcBatch, r = i % kTcBatch;
+    rows[i] = r < l.batch ? tc_minibatch_row(r, u.group, u.event + (uint32_t)(step + q), l.m, s.key0, s.key1) : 0;
   }
-  __nv_bfloat16 hi, lo;
-  split_bf16(r, hi, lo);
-  __nv_bfloat16* out = resid + (int64_t)blockIdx.x * (2 * kUnitNodes * kTcBatch);
-  out[j * kTcBatch + sidx] = hi;
-  out[kUnitNodes * kTcBatch + j * kTcBatch + sidx] = lo;
+  __syncthreads();
+  const float* gram = l.gram + (int64_t)u.group * l.m * l.m;
+  const bool valid = sidx < l.batch && j < u.count;
+  // the scores of every step against the model before the group: chunk order, a fixed summation order; the
+  // steps' sums are independent of one another, which keeps four times as many loads in flight
+  float sum[kTcMaxGroup] = {0.0f, 0.0f, 0.0f, 0.0f};
+  {
+    const float* p = partial + (int64_t)blockIdx.x * nchunks * G * (kTcBatch * kUnitNodes) + threadIdx.x;
+#pragma unroll 4
+    for (int64_t c = 0; c < nchunks; ++c) {
+#pragma unroll
+      for (int q = 0; q < kTcMaxGroup; ++q)
+        if (q < G) sum[q] += p[(c * G + q) * (kTcBatch * kUnitNodes)];
+    }
+  }
+#pragma unroll
+  for (int q = 0; q < kTcMaxGroup; ++q) {
+    if (q >= G) break;
+    float acc = sum[q];
+    float corr = 0.0f;
+    for (int pq = 0; pq < q; ++pq) {
+      __syncthreads();                                                // the block's previous readers are done
+      for (int i = threadIdx.x; i < kTcBatch * kTcBatch; i += blockDim.x) {
+        const int a = i / kTcBatch, b = i % kTcBatch;
+        block[a][b] = gram[(int64_t)rows[q * kTcBatch + a] * l.m + rows[pq * kTcBatch + b]];
+      }
+      __syncthreads();
+#pragma unroll 8
+      for (int b = 0; b < kTcBatch; ++b) corr = fmaf(block[sidx][b], seen[pq][b][j], corr);
+    }
+    acc = fmaf(-scale, corr, acc);
+    float r = 0.0f;
+    if (valid) r = row_residual(acc, l.bvec[(int64_t)u.nodes[j] * l.m + rows[q * kTcBatch + sidx]], l.logistic);
+    __nv_bfloat16 hi, lo;
+    split_bf16(r, hi, lo);
+    __nv_bfloat16* out = resid + ((int64_t)blockIdx.x * G + q) * (2 * kUnitNodes * kTcBatch);
+    out[j * kTcBatch + sidx] = hi;
+    out[kUnitNodes * kTcBatch + j * kTcBatch + sidx] = lo;
+    if (q + 1 < G) seen[q][sidx][j] = __bfloat162float(hi) + __bfloat162float(lo);
+  }
 }
 
 // =================================================================================================
 // Update. Tile = 128 coordinates. A operand = A_S^T, MN-major: per stage
 //   [half h of 64 coordinates][8 groups of 8 sampled rows][8 rows x 128 B], 128B swizzle
 //   (leading byte offset = 8192 between halves, stride byte offset = 1024 between row groups).
-// B operand = resid hi / lo, K-major [16 nodes x 64 rows] (one swizzle atom each).
-// Accumulators: 128 lanes x 16 columns, two buffers. Four stages: 70 KiB per CTA, three CTAs per SM (72 registers).
+// B operand = resid of the stage's step, K-major [32 x 64 rows]: rows 0..15 the hi halves of the 16 nodes'
+// residuals, rows 16..31 the lo halves (N = 32; the two products are added in the epilogue).
+// Stage f holds the rows of step f % G for tile f / G; the G stages of a tile accumulate into one accumulator
+// (128 lanes x 32 columns, two buffers), read back once the tile's last stage has completed.
+// Four stages (three for groups of more than two steps, whose residuals take more room): at most 75 KiB per
+// CTA, three CTAs per SM (72 registers).
 // =================================================================================================
 constexpr int kUpdTile = 128;
-constexpr int kUpdStages = 4;
 constexpr int kUpdABytes = kTcBatch * kUpdTile * 2;             // 16384
 constexpr int kUpdRBytes = kUnitNodes * 128;                   // 2048 (one of hi / lo)
-constexpr int kUpdSmem = kUpdStages * kUpdABytes + 2 * kUpdRBytes + 1024 + 64;
+__host__ __device__ constexpr int upd_stages(int G) { return G <= 2 ? 4 : 3; }
+__host__ __device__ constexpr int upd_smem(int G) { return upd_stages(G) * kUpdABytes + G * 2 * kUpdRBytes + 1024 + 64; }
 
+template <int G>
 __global__ void __launch_bounds__(kTcThreads, 3)
 lsq_tc_update_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, int step, float lr,
                      const __nv_bfloat16* __restrict__ resid, int64_t chunk_coords, int* __restrict__ status,
                      uint32_t spin_limit) {
+  constexpr int kStages = upd_stages(G);
   __shared__ int poisoned;
   if (status_raised(status, &poisoned)) return;               // no model is touched after a step gave up
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* sA = smem;
-  uint8_t* sR = sA + kUpdStages * kUpdABytes;                   // hi then lo
-  uint64_t* bars = (uint64_t*)(sR + 2 * kUpdRBytes);
+  uint8_t* sR = sA + kStages * kUpdABytes;                      // per step: hi then lo
+  uint64_t* bars = (uint64_t*)(sR + G * 2 * kUpdRBytes);
   uint32_t* tmem_slot = (uint32_t*)(bars + 2);
-  __shared__ int rows[kTcBatch];
+  __shared__ int rows[G * kTcBatch];
   __shared__ int unodes[kUnitNodes];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const LsqUnit* up = units + blockIdx.y;
   struct { int group, count; } u = {up->group, up->count};
-  const uint32_t event = up->event + (uint32_t)step;
   if (tid < kUnitNodes) unodes[tid] = up->nodes[tid];
   const int64_t kbase = (int64_t)blockIdx.x * chunk_coords;
   const int64_t kend = min(kbase + chunk_coords, s.pitch);
   const int ntiles = (int)((kend - kbase) / kUpdTile);
+  const int nstages = ntiles * G;
   const __nv_bfloat16* A = reinterpret_cast<const __nv_bfloat16*>(l.A) + (int64_t)u.group * l.m * s.pitch;
   const float scale = lr / (float)l.batch;
 
-  if (tid < kTcBatch) rows[tid] = tid < l.batch ? tc_minibatch_row(tid, u.group, event, l.m, s.key0, s.key1) : 0;
+  draw_rows<G>(rows, l, u.group, up->event + (uint32_t)step, s);
   if (tid == 0) {
     mbar_init(smem_u32(&bars[0]), 1);
     mbar_init(smem_u32(&bars[1]), 1);
     fence_mbar_init();
   }
-  if (warp == 0) { tmem_alloc(smem_u32(tmem_slot), 32); tmem_relinquish(); }
+  if (warp == 0) { tmem_alloc(smem_u32(tmem_slot), 64); tmem_relinquish(); }
   if (l.batch < kTcBatch)     // sampled-row slots beyond the batch are never copied: they must read as zero
-    for (int i = tid; i < kUpdStages * kUpdABytes / 16; i += kTcThreads) reinterpret_cast<uint4*>(sA)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < kStages * kUpdABytes / 16; i += kTcThreads) reinterpret_cast<uint4*>(sA)[i] = make_uint4(0, 0, 0, 0);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_d = *tmem_slot;
 
-  // resid hi / lo: 2 x [16 rows x 8 chunks], K-major swizzled
-  if (tid < 2 * kUnitNodes * 8) {
+  // resid hi / lo of every step: 2 x [16 rows x 8 chunks], K-major swizzled (part of the first copy group)
+  {
     const int which = tid / (kUnitNodes * 8), r = (tid / 8) % kUnitNodes, c = tid & 7;
-    cp_async16(smem_u32(sR + which * kUpdRBytes + (r >> 3) * 1024 + (r & 7) * 128 + ((c ^ (r & 7)) << 4)),
-               resid + (int64_t)blockIdx.y * (2 * kUnitNodes * kTcBatch) + which * (kUnitNodes * kTcBatch) + r * kTcBatch + c * 8);
+#pragma unroll
+    for (int q = 0; q < G; ++q)
+      cp_async16(smem_u32(sR + (q * 2 + which) * kUpdRBytes + (r >> 3) * 1024 + (r & 7) * 128 + ((c ^ (r & 7)) << 4)),
+                 resid + ((int64_t)blockIdx.y * G + q) * (2 * kUnitNodes * kTcBatch) + which * (kUnitNodes * kTcBatch) +
+                     r * kTcBatch + c * 8);
   }
-  auto issue_loads = [&](int tile) {
-    if (tile < ntiles) {
-      const int st = tile % kUpdStages;
+  auto issue_loads = [&](int f) {
+    if (f < nstages) {
+      const int tile = f / G, q = f - tile * G;
+      const int st = f % kStages;
       const int64_t k0 = kbase + (int64_t)tile * kUpdTile;
       const uint32_t a_base = smem_u32(sA + st * kUpdABytes);
       // 64 rows x 16 chunks of 16 B: thread -> (row = idx / 16, chunk = idx % 16)
@@ -401,7 +496,7 @@ lsq_tc_update_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
         if (r < l.batch) {
           const int half = c >> 3, cc = c & 7;
           const uint32_t dst = a_base + half * 8192 + (r >> 3) * 1024 + (r & 7) * 128 + ((cc ^ (r & 7)) << 4);
-          cp_async16(dst, A + (int64_t)rows[r] * s.pitch + k0 + c * 8);
+          cp_async16(dst, A + (int64_t)rows[q * kTcBatch + r] * s.pitch + k0 + c * 8);
         }
       }
     }
@@ -411,66 +506,70 @@ lsq_tc_update_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
   // this thread's share of the epilogue: coordinate lane of quadrant (warp % 4), nodes 8*(warp/4)..+7
   const int quad = warp & 3, jbase = (warp >> 2) * 8;
   auto epilogue = [&](int tile, const float xin[8]) {
-    float dacc[8];
-    tmem_ld8(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)((tile & 1) * kUnitNodes + jbase), dacc);
+    float dacc[8], dlo[8];                                  // products with the hi halves of the residuals, with the lo halves
+    tmem_ld8(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)((tile & 1) * 2 * kUnitNodes + jbase), dacc);
+    tmem_ld8(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)((tile & 1) * 2 * kUnitNodes + kUnitNodes + jbase), dlo);
+#pragma unroll
+    for (int p = 0; p < 8; ++p) dacc[p] += dlo[p];
     const int64_t k = kbase + (int64_t)tile * kUpdTile + quad * 32 + lane;
     if (k < s.d) {
 #pragma unroll
-      for (int q = 0; q < 8; ++q)
-        if (jbase + q < u.count) s.X[(int64_t)unodes[jbase + q] * s.pitch + k] = xin[q] - scale * dacc[q];
+      for (int p = 0; p < 8; ++p)
+        if (jbase + p < u.count) s.X[(int64_t)unodes[jbase + p] * s.pitch + k] = xin[p] - scale * dacc[p];
     }
   };
   auto load_x = [&](int tile, float xin[8]) {
     const int64_t k = kbase + (int64_t)tile * kUpdTile + quad * 32 + lane;
 #pragma unroll
-    for (int q = 0; q < 8; ++q)
-      xin[q] = (tile < ntiles && jbase + q < u.count) ? s.X[(int64_t)unodes[jbase + q] * s.pitch + k] : 0.0f;
+    for (int p = 0; p < 8; ++p)
+      xin[p] = (tile < ntiles && jbase + p < u.count) ? s.X[(int64_t)unodes[jbase + p] * s.pitch + k] : 0.0f;
   };
 
   bool ok = true;                  // this warp's waits so far
-  int committed = -1;              // last tile whose MMAs were committed (the same in every thread)
-  for (int t = 0; t < kUpdStages - 1; ++t) issue_loads(t);
-  constexpr uint32_t idesc = instr_desc_bf16(kUpdTile, kUnitNodes, 1, 0);
+  int committed = -1;              // last stage whose MMAs were committed (the same in every thread)
+  for (int f = 0; f < kStages - 1; ++f) issue_loads(f);
+  constexpr uint32_t idesc = instr_desc_bf16(kUpdTile, 2 * kUnitNodes, 1, 0);   // N = 32: hi and lo residuals side by side
   float xprev[8], xcur[8];
-  for (int t = 0; t < ntiles; ++t) {
-    const int st = t % kUpdStages, buf = t & 1;
-    load_x(t, xcur);                                        // consumed one iteration later
-    cp_async_wait<kUpdStages - 2>();
+  for (int f = 0; f < nstages; ++f) {
+    const int t = f / G, q = f - t * G;
+    const int st = f % kStages, buf = t & 1;
+    if (q == 0) load_x(t, xcur);                            // consumed when the tile's last stage has completed
+    cp_async_wait<kStages - 2>();
     fence_proxy_async();
     tc_fence_before();
-    ok = __syncthreads_and(ok);                             // tile t landed; epilogue of tile t-2 has drained buffer `buf`;
+    ok = __syncthreads_and(ok);                             // stage f landed; epilogue of tile t-2 has drained buffer `buf`;
     if (!ok) break;                                         // and the give-up decision is CTA-uniform
     if (tid == 0) {
       tc_fence_after();
       const uint32_t a_base = smem_u32(sA + st * kUpdABytes);
-      const uint32_t h_base = smem_u32(sR), l_base = smem_u32(sR + kUpdRBytes);
+      const uint32_t r_base = smem_u32(sR + q * 2 * kUpdRBytes);   // rows 0..15 hi, rows 16..31 lo
 #pragma unroll
       for (int ks = 0; ks < 4; ++ks) {                      // 16 sampled rows per MMA = two 8-row groups
         const uint64_t da = smem_desc_sw128(a_base + ks * 2048, 8192, 1024);
-        const uint64_t dh = smem_desc_sw128(h_base + ks * 32, 16, 1024);
-        const uint64_t dl = smem_desc_sw128(l_base + ks * 32, 16, 1024);
-        tc_mma(tmem_d + buf * kUnitNodes, da, dh, idesc, ks != 0);
-        tc_mma(tmem_d + buf * kUnitNodes, da, dl, idesc, 1);
+        const uint64_t dr = smem_desc_sw128(r_base + ks * 32, 16, 1024);
+        tc_mma(tmem_d + buf * 2 * kUnitNodes, da, dr, idesc, (q | ks) != 0);
       }
-      tc_commit(smem_u32(&bars[buf]));
+      tc_commit(smem_u32(&bars[f & 1]));
     }
-    committed = t;
-    if (t >= 1) {
-      ok = mbar_wait(smem_u32(&bars[(t - 1) & 1]), ((t - 1) >> 1) & 1, spin_limit);
+    committed = f;
+    if (f >= 1) {
+      ok = mbar_wait(smem_u32(&bars[(f - 1) & 1]), ((f - 1) >> 1) & 1, spin_limit);
       tc_fence_after();
-      if (ok) epilogue(t - 1, xprev);
+      if (ok && q == 0) epilogue(t - 1, xprev);             // stage f-1 was the last of tile t-1
       tc_fence_before();
     }
+    if (q == 0) {
 #pragma unroll
-    for (int q = 0; q < 8; ++q) xprev[q] = xcur[q];
-    if (ok) issue_loads(t + kUpdStages - 1);                // stage of tile t-1: its MMAs have completed
+      for (int p = 0; p < 8; ++p) xprev[p] = xcur[p];
+    }
+    if (ok) issue_loads(f + kStages - 1);                   // stage of f-1: its MMAs have completed
     else cp_async_commit();
   }
   cp_async_wait<0>();
   if (ok && committed >= 0) {
     ok = mbar_wait(smem_u32(&bars[committed & 1]), (committed >> 1) & 1, spin_limit);
     tc_fence_after();
-    if (ok) epilogue(committed, xprev);
+    if (ok) epilogue(committed / G, xprev);
   }
   ok = __syncthreads_and(ok);
   if (!ok) {
@@ -481,11 +580,78 @@ lsq_tc_update_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem_d, 32);
+  if (warp == 0) tmem_dealloc(tmem_d, 64);
 }
 
 // =================================================================================================
-// Launch wrapper
+// Gram matrix of one data matrix: gram[i][j] = <A[i], A[j]> over the padded row (the padding is zero).
+// CTA = one 64 x 64 tile of the lower triangle (mirrored on store), thread = 4 x 4 entries; products are
+// summed in fp32 over 1024 coordinates at a time and in double across those runs, in coordinate order.
+// Runs once per data matrix (when the data is made or rewritten), not in the step.
+// =================================================================================================
+constexpr int kGramTile = 64;
+constexpr int kGramK = 32;
+
+__global__ void __launch_bounds__(256)
+lsq_gram_kernel(const __nv_bfloat16* __restrict__ A, int m, int64_t pitch, int first_matrix, float* __restrict__ gram) {
+  __shared__ __align__(16) float sa[kGramK][kGramTile + 4];
+  __shared__ __align__(16) float sb[kGramK][kGramTile + 4];
+  int ti = 0;
+  while ((ti + 1) * (ti + 2) / 2 <= (int)blockIdx.x) ++ti;       // tile (ti, tj) of the lower triangle, tj <= ti
+  const int tj = (int)blockIdx.x - ti * (ti + 1) / 2;
+  const int matrix = first_matrix + (int)blockIdx.y;
+  const __nv_bfloat16* Ag = A + (int64_t)matrix * m * pitch;
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int lrow = tid >> 2, c8 = (tid & 3) * 8;                 // staging: 64 rows x 4 groups of 8 coordinates
+  const int ri = ti * kGramTile + lrow, rj = tj * kGramTile + lrow;
+  double total[16];
+  float run[16];
+#pragma unroll
+  for (int e = 0; e < 16; ++e) { total[e] = 0.0; run[e] = 0.0f; }
+  for (int64_t k0 = 0; k0 < pitch; k0 += kGramK) {
+    uint4 va = make_uint4(0, 0, 0, 0), vb = make_uint4(0, 0, 0, 0);
+    if (ri < m) va = *reinterpret_cast<const uint4*>(Ag + (int64_t)ri * pitch + k0 + c8);
+    if (rj < m) vb = *reinterpret_cast<const uint4*>(Ag + (int64_t)rj * pitch + k0 + c8);
+    const __nv_bfloat16* ha = reinterpret_cast<const __nv_bfloat16*>(&va);
+    const __nv_bfloat16* hb = reinterpret_cast<const __nv_bfloat16*>(&vb);
+    __syncthreads();                                             // the previous slice's readers are done
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      sa[c8 + e][lrow] = __bfloat162float(ha[e]);
+      sb[c8 + e][lrow] = __bfloat162float(hb[e]);
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int k = 0; k < kGramK; ++k) {
+      const float4 a = *reinterpret_cast<const float4*>(&sa[k][ty * 4]);
+      const float4 b = *reinterpret_cast<const float4*>(&sb[k][tx * 4]);
+      const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int y = 0; y < 4; ++y)
+#pragma unroll
+        for (int x = 0; x < 4; ++x) run[y * 4 + x] = fmaf(av[y], bv[x], run[y * 4 + x]);
+    }
+    if (((k0 + kGramK) & 1023) == 0) {
+#pragma unroll
+      for (int e = 0; e < 16; ++e) { total[e] += (double)run[e]; run[e] = 0.0f; }
+    }
+  }
+  float* G = gram + (int64_t)matrix * m * m;
+#pragma unroll
+  for (int y = 0; y < 4; ++y)
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      const int i = ti * kGramTile + ty * 4 + y, j = tj * kGramTile + tx * 4 + x;
+      if (i < m && j < m) {
+        const float v = (float)(total[y * 4 + x] + (double)run[y * 4 + x]);
+        G[(int64_t)i * m + j] = v;
+        G[(int64_t)j * m + i] = v;
+      }
+    }
+}
+
+// =================================================================================================
+// Launch wrappers
 // =================================================================================================
 int64_t lsq_tc_chunk_coords(int64_t pitch) {
   // chunks of 8192 coordinates (a multiple of both tile sizes); short rows get a single chunk
@@ -495,10 +661,50 @@ int64_t lsq_tc_chunks(int64_t pitch) {
   const int64_t c = lsq_tc_chunk_coords(pitch);
   return (pitch + c - 1) / c;
 }
-size_t lsq_tc_partial_bytes(int64_t pitch, int units) { return (size_t)units * lsq_tc_chunks(pitch) * kTcBatch * kUnitNodes * 4; }
-size_t lsq_tc_resid_bytes(int units) { return (size_t)units * 2 * kUnitNodes * kTcBatch * 2; }
+size_t lsq_tc_partial_bytes(int64_t pitch, int units) {
+  return (size_t)units * lsq_tc_chunks(pitch) * kTcMaxGroup * kTcBatch * kUnitNodes * 4;
+}
+size_t lsq_tc_resid_bytes(int units) { return (size_t)units * kTcMaxGroup * 2 * kUnitNodes * kTcBatch * 2; }
+size_t lsq_tc_gram_bytes(int matrices, int m) {
+  const size_t bytes = (size_t)matrices * (size_t)m * (size_t)m * 4;
+  return bytes <= ((size_t)256 << 20) ? bytes : 0;              // larger tables are not kept: steps go one at a time
+}
 
 uint32_t lsq_tc_default_wait_limit() { return kSpinLimit; }
+
+cudaError_t launch_lsq_gram(const void* A_dev, int m, int64_t pitch, int first_matrix, int matrices, float* gram_dev,
+                            cudaStream_t st, int* launches) {
+  if (matrices == 0 || !gram_dev) return cudaSuccess;
+  const int tiles = (m + kGramTile - 1) / kGramTile;
+  const dim3 grid((unsigned)(tiles * (tiles + 1) / 2), (unsigned)matrices);
+  lsq_gram_kernel<<<grid, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(A_dev), m, pitch, first_matrix, gram_dev);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+namespace {
+
+template <int G>
+cudaError_t set_group_attributes() {
+  cudaError_t e = cudaFuncSetAttribute(lsq_tc_scores_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, kResSmem);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(lsq_tc_update_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, upd_smem(G));
+}
+
+template <int G>
+void launch_group(const StoreView& s, const LsqView& l, const LsqUnit* units_dev, int nunits, int step, float lr,
+                  float* partial_dev, __nv_bfloat16* resid_dev, int* status_dev, uint32_t wait_limit, cudaStream_t st) {
+  const int64_t chunk = lsq_tc_chunk_coords(s.pitch), nchunks = lsq_tc_chunks(s.pitch);
+  const dim3 grid((unsigned)nchunks, nunits);
+  lsq_tc_scores_kernel<G><<<grid, kTcThreads, kResSmem, st>>>(s, l, units_dev, step, partial_dev, chunk, nchunks, status_dev,
+                                                              wait_limit);
+  lsq_tc_finalize_kernel<<<nunits, kTcBatch * kUnitNodes, 0, st>>>(s, l, units_dev, step, G, lr / (float)l.batch, partial_dev,
+                                                                   nchunks, resid_dev, status_dev);
+  lsq_tc_update_kernel<G><<<grid, kTcThreads, upd_smem(G), st>>>(s, l, units_dev, step, lr, resid_dev, chunk, status_dev,
+                                                                 wait_limit);
+}
+
+}  // namespace
 
 cudaError_t launch_local_lsq_tc(const StoreView& s, const LsqView& l, const LsqUnit* units_dev, int nunits, int H,
                                 float lr, float* partial_dev, void* resid_dev, int* status_dev, uint32_t wait_limit,
@@ -511,23 +717,25 @@ cudaError_t launch_local_lsq_tc(const StoreView& s, const LsqView& l, const LsqU
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(lsq_tc_residual_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kResSmem);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(lsq_tc_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kUpdSmem);
+    cudaError_t e = set_group_attributes<1>();
+    if (e == cudaSuccess) e = set_group_attributes<2>();
+    if (e == cudaSuccess) e = set_group_attributes<3>();
+    if (e == cudaSuccess) e = set_group_attributes<4>();
     if (e != cudaSuccess) return e;
     attr_set[dev] = true;
   }
-  const int64_t chunk = lsq_tc_chunk_coords(s.pitch), nchunks = lsq_tc_chunks(s.pitch);
-  const dim3 grid((unsigned)nchunks, nunits);
-  for (int q = 0; q < H; ++q) {
-    lsq_tc_residual_kernel<<<grid, kTcThreads, kResSmem, st>>>(s, l, units_dev, q, partial_dev, chunk, nchunks, status_dev,
-                                                               wait_limit);
-    lsq_tc_finalize_kernel<<<nunits, kTcBatch * kUnitNodes, 0, st>>>(s, l, units_dev, q, partial_dev, nchunks,
-                                                                     reinterpret_cast<__nv_bfloat16*>(resid_dev), status_dev);
-    lsq_tc_update_kernel<<<grid, kTcThreads, kUpdSmem, st>>>(s, l, units_dev, q, lr,
-                                                             reinterpret_cast<const __nv_bfloat16*>(resid_dev), chunk, status_dev,
-                                                             wait_limit);
+  auto* resid = reinterpret_cast<__nv_bfloat16*>(resid_dev);
+  const int max_group = l.gram ? kTcMaxGroup : 1;
+  for (int q = 0; q < H;) {
+    const int G = H - q < max_group ? H - q : max_group;
+    switch (G) {
+      case 1: launch_group<1>(s, l, units_dev, nunits, q, lr, partial_dev, resid, status_dev, wait_limit, st); break;
+      case 2: launch_group<2>(s, l, units_dev, nunits, q, lr, partial_dev, resid, status_dev, wait_limit, st); break;
+      case 3: launch_group<3>(s, l, units_dev, nunits, q, lr, partial_dev, resid, status_dev, wait_limit, st); break;
+      default: launch_group<4>(s, l, units_dev, nunits, q, lr, partial_dev, resid, status_dev, wait_limit, st); break;
+    }
     *launches += 3;
+    q += G;
   }
   return cudaGetLastError();
 }

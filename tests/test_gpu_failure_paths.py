@@ -72,7 +72,7 @@ def test_configure_out_of_memory_leaves_the_default_configuration():
     try:
         sw = g.Swarm(n, d, "complete", seed=5, torch_memory=False)
         default_x = sw.get_all(g.T_X)
-        needed = 10      # snapshots, own registers + exponents, data, labels, x*, two scratch arrays, tensor-core scratch x 2
+        needed = 11      # snapshots, own registers + exponents, data, labels, x*, two scratch arrays, tensor-core scratch x 2, Gram matrices
         for k in range(needed + 1):
             state["budget"] = k
             if k < needed:

@@ -520,6 +520,43 @@ def test_batched_tensor_core_least_squares_steps(n, groups, d, m, batch):
         inject(orc, gpu, what=("X",))
 
 
+@pytest.mark.parametrize("H,objective", [(1, 2), (4, 2), (5, 2), (7, 2), (9, 2), (4, 3), (6, 3)])
+def test_tensor_core_steps_folded_four_at_a_time(H, objective):
+    """bf16 data: up to four consecutive steps of a unit share one pass for the scores (against the model before
+    the first of them, corrected step by step through blocks of the data's Gram matrix) and one pass for the
+    updates. Every split of H into groups (4, 4 + 1, 4 + 3, 4 + 4 + 1) must give the oracle's H separate steps.
+    Fewer rows than a minibatch draws, so that minibatches share rows and the corrections are large; a step size
+    ten times the usual one; the second data matrix rewritten through swarm_set_tensor (its Gram matrix follows)."""
+    n, d = 20, 17000
+    cfg = dict(objective=objective, lsq_m=48, lsq_batch=64, lsq_dtype=1, lsq_groups=2, lsq_noise_std=0.3, init_std=0.5)
+    orc, gpu = make_pair(n, d, seed=97, **cfg)
+    orc.A[1] = (2.0 * orc.A[1][::-1]).astype(np.float32)          # exact in bf16
+    inject(orc, gpu)
+    lr = 0.5
+    for nodes in (list(range(n)), [3, 17, 4, 11, 12]):
+        assert orc.local_steps(nodes, H, lr) == 0 and gpu.local_steps(nodes, H, lr) == 0
+        gpu.sync()
+        for i in range(n):
+            assert rel_err(gpu.get(g.T_X, i), orc.X[i]) < TOL, i
+            assert gpu.get(g.T_COUNTERS, i)[1] == orc.ls[i]
+        inject(orc, gpu, what=("X",))
+
+
+def test_tensor_core_steps_one_at_a_time_when_the_gram_matrix_is_not_kept():
+    """A data matrix of 8200 rows: its Gram matrix (269 MB) is above what the library keeps, so the steps take
+    one pair of passes each; same results within the tolerance."""
+    n, d = 4, 1024
+    cfg = dict(objective=2, lsq_m=8200, lsq_batch=64, lsq_dtype=1, lsq_groups=1, lsq_noise_std=0.3)
+    orc, gpu = make_pair(n, d, seed=98, **cfg)
+    inject(orc, gpu)
+    launches = gpu.kernel_launches()
+    assert orc.local_steps([0, 1, 2, 3], 3, 0.2) == 0 and gpu.local_steps([0, 1, 2, 3], 3, 0.2) == 0
+    gpu.sync()
+    assert gpu.kernel_launches() - launches == 9                           # three kernels per step
+    for i in range(n):
+        assert rel_err(gpu.get(g.T_X, i), orc.X[i]) < TOL, i
+
+
 @pytest.mark.parametrize("d,m,batch,dtype,groups", [(4096, 64, 16, 0, 0), (20000, 24, 40, 0, 2), (33000, 64, 64, 1, 2),
                                                    (700, 12, 5, 1, 0)])
 def test_logistic_regression_steps_within_tolerance(d, m, batch, dtype, groups):
