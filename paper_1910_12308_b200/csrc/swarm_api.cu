@@ -342,6 +342,7 @@ int apply_config(swarm_ctx* c, const swarm_config& wanted) {
   SW_CUDA(c, cudaMemsetAsync(c->codes, 0, (size_t)n * c->nblk * kBlockCoords, c->stream));
   SW_CUDA(c, cudaMemsetAsync(c->exps, 0, (size_t)n * c->nblk, c->stream));
   SW_CUDA(c, cudaMemsetAsync(c->kernel_status, 0, sizeof(int), c->stream));
+  if (c->tc_resid) SW_CUDA(c, cudaMemsetAsync(c->tc_resid, 0, lsq_tc_resid_bytes(n), c->stream));   // its ticket counters
   c->status_pending = false;
   c->poisoned = false;
   if (c->own) {
@@ -663,7 +664,7 @@ int swarm_local_steps(swarm_ctx* c, const int32_t* node_ids, int32_t count, int3
     rc = stage_commit(c, slot, bytes);
     if (rc != SWARM_OK) return rc;
     int nl = 0;
-    SW_CUDA(c, launch_local_lsq_tc(view_of(c), lsq_of(c), (const LsqUnit*)dev, (int)units.size(), H, lr, c->tc_partial,
+    SW_CUDA(c, launch_local_lsq_tc(view_of(c), lsq_of(c), (const LsqUnit*)dev, (int)units.size(), c->n, H, lr, c->tc_partial,
                                    c->tc_resid, c->kernel_status, c->wait_limit, c->stream, &nl));
     c->status_pending = true;
     c->launches += nl;

@@ -148,9 +148,10 @@ cudaError_t launch_lsq_gram(const void* A_dev, int m, int64_t pitch, int first_m
 // H steps of every unit, in groups of up to four steps per pair of passes when l.gram is set (one step otherwise).
 // status_dev: one int, set to 1 if a bounded wait inside a kernel expired (kernels that find it set return at
 // once); wait_limit: polls after which a wait on a tensor-core commit gives up.
-cudaError_t launch_local_lsq_tc(const StoreView& s, const LsqView& l, const LsqUnit* units_dev, int nunits, int H,
-                                float lr, float* partial_dev, void* resid_dev, int* status_dev, uint32_t wait_limit,
-                                cudaStream_t st, int* launches);
+// partial_dev and resid_dev: lsq_tc_partial_bytes / lsq_tc_resid_bytes for max_units units, the latter zeroed once.
+cudaError_t launch_local_lsq_tc(const StoreView& s, const LsqView& l, const LsqUnit* units_dev, int nunits, int max_units,
+                                int H, float lr, float* partial_dev, void* resid_dev, int* status_dev,
+                                uint32_t wait_limit, cudaStream_t st, int* launches);
 uint32_t lsq_tc_default_wait_limit();
 cudaError_t launch_sample_pairs(const int32_t* adj_dev, int n, int degree, int max_pairs, uint32_t launch_ctr,
                                 uint32_t key0, uint32_t key1, int32_t* out_pairs_dev, int32_t* out_count_dev,

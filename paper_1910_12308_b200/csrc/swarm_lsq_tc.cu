@@ -351,22 +351,66 @@ lsq_tc_scores_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
 }
 
 // =================================================================================================
-// Finalize, one CTA per unit, thread = (sampled row s, node j). For step q = 0 .. G-1 in turn:
-//   score[s][j] = sum over chunks (in chunk order) of the partials of step q
-//                 - scale * sum_{p<q} sum_{s'} gram[row_q[s]][row_p[s']] * resid_p[s'][j]
+// Finalize, thread = (sampled row s, node j). kFinSplit CTAs per unit each add a contiguous run of the unit's
+// chunk partials (in chunk order) and leave one second-level partial per step; the CTA of a unit that finishes
+// last (a ticket counter per unit, left at zero) adds the second-level partials in run order, so the sum has one
+// fixed association whichever CTA that is, and then walks the steps q = 0 .. G-1 in turn:
+//   score[s][j] = the sum of step q - scale * sum_{p<q} sum_{s'} gram[row_q[s]][row_p[s']] * resid_p[s'][j]
 //   resid_q[s][j] = score - label (least squares) or sigmoid(score) - label (logistic)
 // stored K-major per node as bf16 hi / lo: R[unit][q][hi|lo][j][s]. The corrections use the residuals as the
 // update kernel will see them (hi + lo).
 // =================================================================================================
+constexpr int kFinSplit = 8;
+
 __global__ void __launch_bounds__(kTcBatch * kUnitNodes)
 lsq_tc_finalize_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, int step, int G, float scale,
-                       const float* __restrict__ partial, int64_t nchunks, __nv_bfloat16* __restrict__ resid,
+                       const float* __restrict__ partial, int64_t nchunks, float* __restrict__ level2,
+                       unsigned int* __restrict__ tickets, __nv_bfloat16* __restrict__ resid,
                        const int* __restrict__ status) {
   if (*reinterpret_cast<const volatile int*>(status) != 0) return;    // the partials of a step that gave up are not complete
   __shared__ int rows[kTcMaxGroup * kTcBatch];
   __shared__ float seen[kTcMaxGroup - 1][kTcBatch][kUnitNodes];       // residuals of the earlier steps of the group
   __shared__ float block[kTcBatch][kTcBatch + 1];                     // one 64 x 64 block of the Gram matrix
-  const LsqUnit u = units[blockIdx.x];
+  __shared__ bool last;
+  const int unit = blockIdx.y, part = blockIdx.x;
+  constexpr int kCell = kTcBatch * kUnitNodes;
+  // the scores of every step against the model before the group; the steps' sums are independent of one another,
+  // which keeps G times as many loads in flight
+  float sum[kTcMaxGroup] = {0.0f, 0.0f, 0.0f, 0.0f};
+  {
+    const int64_t per = (nchunks + kFinSplit - 1) / kFinSplit;
+    const int64_t c0 = part * per, c1 = min(c0 + per, nchunks);
+    const float* p = partial + (int64_t)unit * nchunks * G * kCell + threadIdx.x;
+#pragma unroll 4
+    for (int64_t c = c0; c < c1; ++c) {
+#pragma unroll
+      for (int q = 0; q < kTcMaxGroup; ++q)
+        if (q < G) sum[q] += p[(c * G + q) * kCell];
+    }
+    float* mine = level2 + ((int64_t)unit * kFinSplit + part) * kTcMaxGroup * kCell + threadIdx.x;
+#pragma unroll
+    for (int q = 0; q < kTcMaxGroup; ++q)
+      if (q < G) mine[q * kCell] = sum[q];
+  }
+  __threadfence();                                                    // this thread's partials before the ticket
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    last = atomicAdd(&tickets[unit], 1u) == kFinSplit - 1;
+    if (last) tickets[unit] = 0;                                      // every CTA of the unit has drawn: ready for the next launch
+  }
+  __syncthreads();
+  if (!last) return;
+  __threadfence();                                                    // the other CTAs' partials after the ticket
+  {
+    const volatile float* all = level2 + (int64_t)unit * kFinSplit * kTcMaxGroup * kCell + threadIdx.x;
+#pragma unroll
+    for (int q = 0; q < kTcMaxGroup; ++q) {
+      sum[q] = 0.0f;
+      if (q < G)
+        for (int r = 0; r < kFinSplit; ++r) sum[q] += all[(r * kTcMaxGroup + q) * kCell];
+    }
+  }
+  const LsqUnit u = units[unit];
   const int sidx = threadIdx.x / kUnitNodes, j = threadIdx.x % kUnitNodes;
   for (int i = threadIdx.x; i < G * kTcBatch; i += blockDim.x) {
     const int q = i / kTcBatch, r = i % kTcBatch;
@@ -375,18 +419,6 @@ lsq_tc_finalize_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units
   __syncthreads();
   const float* gram = l.gram + (int64_t)u.group * l.m * l.m;
   const bool valid = sidx < l.batch && j < u.count;
-  // the scores of every step against the model before the group: chunk order, a fixed summation order; the
-  // steps' sums are independent of one another, which keeps four times as many loads in flight
-  float sum[kTcMaxGroup] = {0.0f, 0.0f, 0.0f, 0.0f};
-  {
-    const float* p = partial + (int64_t)blockIdx.x * nchunks * G * (kTcBatch * kUnitNodes) + threadIdx.x;
-#pragma unroll 4
-    for (int64_t c = 0; c < nchunks; ++c) {
-#pragma unroll
-      for (int q = 0; q < kTcMaxGroup; ++q)
-        if (q < G) sum[q] += p[(c * G + q) * (kTcBatch * kUnitNodes)];
-    }
-  }
 #pragma unroll
   for (int q = 0; q < kTcMaxGroup; ++q) {
     if (q >= G) break;
@@ -407,7 +439,7 @@ lsq_tc_finalize_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units
     if (valid) r = row_residual(acc, l.bvec[(int64_t)u.nodes[j] * l.m + rows[q * kTcBatch + sidx]], l.logistic);
     __nv_bfloat16 hi, lo;
     split_bf16(r, hi, lo);
-    __nv_bfloat16* out = resid + ((int64_t)blockIdx.x * G + q) * (2 * kUnitNodes * kTcBatch);
+    __nv_bfloat16* out = resid + ((int64_t)unit * G + q) * (2 * kUnitNodes * kTcBatch);
     out[j * kTcBatch + sidx] = hi;
     out[kUnitNodes * kTcBatch + j * kTcBatch + sidx] = lo;
     if (q + 1 < G) seen[q][sidx][j] = __bfloat162float(hi) + __bfloat162float(lo);
@@ -661,10 +693,17 @@ int64_t lsq_tc_chunks(int64_t pitch) {
   const int64_t c = lsq_tc_chunk_coords(pitch);
   return (pitch + c - 1) / c;
 }
-size_t lsq_tc_partial_bytes(int64_t pitch, int units) {
-  return (size_t)units * lsq_tc_chunks(pitch) * kTcMaxGroup * kTcBatch * kUnitNodes * 4;
+// Scratch of the tensor-core steps. Partials: the chunk partials of every unit, then kFinSplit second-level
+// partials per unit. Residuals: bf16 hi / lo per unit and step, then one ticket counter per unit (zero between
+// launches; the caller zeroes the buffer once).
+static size_t chunk_partial_floats(int64_t pitch, int units) {
+  return (size_t)units * lsq_tc_chunks(pitch) * kTcMaxGroup * kTcBatch * kUnitNodes;
 }
-size_t lsq_tc_resid_bytes(int units) { return (size_t)units * kTcMaxGroup * 2 * kUnitNodes * kTcBatch * 2; }
+static size_t resid_elems(int units) { return (size_t)units * kTcMaxGroup * 2 * kUnitNodes * kTcBatch; }
+size_t lsq_tc_partial_bytes(int64_t pitch, int units) {
+  return (chunk_partial_floats(pitch, units) + (size_t)units * kFinSplit * kTcMaxGroup * kTcBatch * kUnitNodes) * 4;
+}
+size_t lsq_tc_resid_bytes(int units) { return resid_elems(units) * 2 + (size_t)units * 4; }
 size_t lsq_tc_gram_bytes(int matrices, int m) {
   const size_t bytes = (size_t)matrices * (size_t)m * (size_t)m * 4;
   return bytes <= ((size_t)256 << 20) ? bytes : 0;              // larger tables are not kept: steps go one at a time
@@ -693,22 +732,23 @@ cudaError_t set_group_attributes() {
 
 template <int G>
 void launch_group(const StoreView& s, const LsqView& l, const LsqUnit* units_dev, int nunits, int step, float lr,
-                  float* partial_dev, __nv_bfloat16* resid_dev, int* status_dev, uint32_t wait_limit, cudaStream_t st) {
+                  float* partial_dev, float* level2_dev, __nv_bfloat16* resid_dev, unsigned int* tickets_dev,
+                  int* status_dev, uint32_t wait_limit, cudaStream_t st) {
   const int64_t chunk = lsq_tc_chunk_coords(s.pitch), nchunks = lsq_tc_chunks(s.pitch);
   const dim3 grid((unsigned)nchunks, nunits);
   lsq_tc_scores_kernel<G><<<grid, kTcThreads, kResSmem, st>>>(s, l, units_dev, step, partial_dev, chunk, nchunks, status_dev,
                                                               wait_limit);
-  lsq_tc_finalize_kernel<<<nunits, kTcBatch * kUnitNodes, 0, st>>>(s, l, units_dev, step, G, lr / (float)l.batch, partial_dev,
-                                                                   nchunks, resid_dev, status_dev);
+  lsq_tc_finalize_kernel<<<dim3(kFinSplit, nunits), kTcBatch * kUnitNodes, 0, st>>>(
+      s, l, units_dev, step, G, lr / (float)l.batch, partial_dev, nchunks, level2_dev, tickets_dev, resid_dev, status_dev);
   lsq_tc_update_kernel<G><<<grid, kTcThreads, upd_smem(G), st>>>(s, l, units_dev, step, lr, resid_dev, chunk, status_dev,
                                                                  wait_limit);
 }
 
 }  // namespace
 
-cudaError_t launch_local_lsq_tc(const StoreView& s, const LsqView& l, const LsqUnit* units_dev, int nunits, int H,
-                                float lr, float* partial_dev, void* resid_dev, int* status_dev, uint32_t wait_limit,
-                                cudaStream_t st, int* launches) {
+cudaError_t launch_local_lsq_tc(const StoreView& s, const LsqView& l, const LsqUnit* units_dev, int nunits, int max_units,
+                                int H, float lr, float* partial_dev, void* resid_dev, int* status_dev,
+                                uint32_t wait_limit, cudaStream_t st, int* launches) {
   if (nunits == 0 || H == 0) return cudaSuccess;
   if (l.batch > kTcBatch || l.dtype != 1) return cudaErrorInvalidValue;
   static bool attr_set[64] = {};
@@ -724,15 +764,18 @@ cudaError_t launch_local_lsq_tc(const StoreView& s, const LsqView& l, const LsqU
     if (e != cudaSuccess) return e;
     attr_set[dev] = true;
   }
+  if (nunits > max_units) return cudaErrorInvalidValue;
   auto* resid = reinterpret_cast<__nv_bfloat16*>(resid_dev);
+  auto* tickets = reinterpret_cast<unsigned int*>(resid + resid_elems(max_units));
+  float* level2 = partial_dev + chunk_partial_floats(s.pitch, max_units);
   const int max_group = l.gram ? kTcMaxGroup : 1;
   for (int q = 0; q < H;) {
     const int G = H - q < max_group ? H - q : max_group;
     switch (G) {
-      case 1: launch_group<1>(s, l, units_dev, nunits, q, lr, partial_dev, resid, status_dev, wait_limit, st); break;
-      case 2: launch_group<2>(s, l, units_dev, nunits, q, lr, partial_dev, resid, status_dev, wait_limit, st); break;
-      case 3: launch_group<3>(s, l, units_dev, nunits, q, lr, partial_dev, resid, status_dev, wait_limit, st); break;
-      default: launch_group<4>(s, l, units_dev, nunits, q, lr, partial_dev, resid, status_dev, wait_limit, st); break;
+      case 1: launch_group<1>(s, l, units_dev, nunits, q, lr, partial_dev, level2, resid, tickets, status_dev, wait_limit, st); break;
+      case 2: launch_group<2>(s, l, units_dev, nunits, q, lr, partial_dev, level2, resid, tickets, status_dev, wait_limit, st); break;
+      case 3: launch_group<3>(s, l, units_dev, nunits, q, lr, partial_dev, level2, resid, tickets, status_dev, wait_limit, st); break;
+      default: launch_group<4>(s, l, units_dev, nunits, q, lr, partial_dev, level2, resid, tickets, status_dev, wait_limit, st); break;
     }
     *launches += 3;
     q += G;
