@@ -300,10 +300,14 @@ int alloc_objective(swarm_ctx* c, const swarm_config& cfg) {
     c->lsq_partial = (float*)dev_alloc(c, (size_t)n * cfg.lsq_batch * lsq_chunks(c->d) * sizeof(float));
     c->convert_tmp = (float*)dev_alloc(c, row_bytes);
     if (!c->A || !c->bvec || !c->xstar || !c->lsq_partial || !c->convert_tmp) return SWARM_ENOMEM;
-    if (cfg.lsq_dtype == SWARM_BF16 && cfg.lsq_batch <= 64) {
+    const bool tensor_cores = cfg.lsq_dtype == SWARM_BF16 && cfg.lsq_batch <= 64;
+    if (tensor_cores) {
       c->tc_partial = (float*)dev_alloc(c, lsq_tc_partial_bytes(c->pitch, n));
       c->tc_resid = dev_alloc(c, lsq_tc_resid_bytes(n));
       if (!c->tc_partial || !c->tc_resid) return SWARM_ENOMEM;
+    }
+    // Gram matrices of the data, for the kernels that take several local steps per pass
+    if (tensor_cores || lsq_small_steps_in_pairs(c->pitch, cfg.lsq_batch)) {
       const size_t gram_bytes = lsq_tc_gram_bytes(c->groups, cfg.lsq_m);
       if (gram_bytes) {
         c->gram = (float*)dev_alloc(c, gram_bytes);
@@ -355,7 +359,7 @@ int apply_config(swarm_ctx* c, const swarm_config& wanted) {
   if (cfg.objective == SWARM_OBJ_LSQ || cfg.objective == SWARM_OBJ_LOGISTIC) {
     LsqView l = lsq_of(c);
     SW_CUDA(c, launch_lsq_data(s, l, c->A, c->xstar, c->bvec, c->scalars, cfg.lsq_noise_std, c->stream, &nl));
-    SW_CUDA(c, launch_lsq_gram(c->A, cfg.lsq_m, c->pitch, 0, c->groups, c->gram, c->stream, &nl));
+    SW_CUDA(c, launch_lsq_gram(c->A, cfg.lsq_dtype, cfg.lsq_m, c->pitch, 0, c->groups, c->gram, c->stream, &nl));
   }
   c->launches += nl;
   std::fill(c->w.begin(), c->w.end(), 0u);
@@ -1174,7 +1178,8 @@ static int tensor_access(swarm_ctx* c, int32_t which, int32_t node, void* host, 
         }
       }
       // rewritten rows change the matrix's Gram matrix, which the grouped local steps read
-      if (write) SW_CUDA(c, launch_lsq_gram(c->A, c->cfg.lsq_m, c->pitch, node, 1, c->gram, c->stream, &nl));
+      if (write)
+        SW_CUDA(c, launch_lsq_gram(c->A, c->cfg.lsq_dtype, c->cfg.lsq_m, c->pitch, node, 1, c->gram, c->stream, &nl));
       c->launches += nl;
       SW_SYNC(c);
       return SWARM_OK;

@@ -98,7 +98,7 @@ inline void division_magic(uint64_t divisor, uint32_t* magic, uint32_t* shift) {
 struct LsqView {
   const void* A;       // [groups][m][pitch] fp32 or bf16
   const float* bvec;   // [n][m]
-  const float* gram;   // [groups][m][m] Gram matrices A A^T of the bf16 data matrices, or nullptr when not kept
+  const float* gram;   // [groups][m][m] Gram matrices A A^T of the data matrices, or nullptr when not kept
   int32_t m, batch, dtype, groups, nodes_per_group;
   int32_t logistic;    // 1: residual = sigmoid(<a, x>) - y with labels in {0, 1}; 0: residual = <a, x> - b
 };
@@ -129,6 +129,9 @@ cudaError_t launch_local_synth(const StoreView& s, const NodeList& nodes, int co
 cudaError_t launch_local_lsq(const StoreView& s, const LsqView& l, const NodeList& nodes, int count, int H,
                              float lr, float* partial_dev, cudaStream_t st, int* launches);
 int64_t lsq_chunks(int64_t d);
+// True when the short-model kernels take two steps per round given the data's Gram matrix (row pitch and batch
+// size small enough that both minibatches stay in registers).
+bool lsq_small_steps_in_pairs(int64_t pitch, int batch);
 // Sequential gossip in one launch (short models, fp32 least-squares data, batch <= 32): steps.n steps of one
 // pair each; per step the pair's nodes (the initiator only if responders == 0) take H local steps, then the
 // pair interacts in blocking mode at `bits` bits. The descriptors carry the counters of every step.
@@ -142,9 +145,10 @@ size_t lsq_tc_resid_bytes(int units);
 // Bytes of the Gram matrices of `matrices` data matrices of m rows; 0 when they are too large to keep (local steps
 // then go one at a time instead of in groups).
 size_t lsq_tc_gram_bytes(int matrices, int m);
-// gram_dev[first_matrix .. first_matrix + matrices) = A A^T of those bf16 data matrices (row padding must be zero).
-cudaError_t launch_lsq_gram(const void* A_dev, int m, int64_t pitch, int first_matrix, int matrices, float* gram_dev,
-                            cudaStream_t st, int* launches);
+// gram_dev[first_matrix .. first_matrix + matrices) = A A^T of those data matrices (dtype 1: bf16, else fp32; row
+// padding must be zero).
+cudaError_t launch_lsq_gram(const void* A_dev, int dtype, int m, int64_t pitch, int first_matrix, int matrices,
+                            float* gram_dev, cudaStream_t st, int* launches);
 // H steps of every unit, in groups of up to four steps per pair of passes when l.gram is set (one step otherwise).
 // status_dev: one int, set to 1 if a bounded wait inside a kernel expired (kernels that find it set return at
 // once); wait_limit: polls after which a wait on a tensor-core commit gives up.

@@ -258,6 +258,11 @@ struct SmallShared {
   float red[kSmallThreads / 32][kSmallMaxBatch];
   float part[kSmallMaxBatch];          // this CTA's partial dot products (read by the whole cluster)
   float resid[kSmallMaxBatch];
+  // second step of a pair of steps taken in one round (batches of at most 16 rows)
+  float red2[kSmallThreads / 32][16];
+  float part2[16];
+  float resid2[16];
+  float gram[16][17];                  // <row s of the second step, row s' of the first>
 };
 
 // Barrier among the `count` threads that use barrier `id` (a multiple of 32 threads, whole warps).
@@ -295,6 +300,11 @@ __device__ __forceinline__ float reduce_rows(float (&v)[G], int lane, int& row) 
 // barriers, so that several thread groups of a CTA (each with its own node, scratch and named barrier) can
 // run side by side. ITERS = slices of 512 coordinates per CTA. The model is read from and written back to
 // global memory; the caller orders those accesses against other CTAs' work.
+// Two steps per round where the data's Gram matrix is at hand and a minibatch fits the rows a thread keeps in
+// flight: the second step's rows are known in advance, and <a, x_1> = <a, x_0> - (lr/B) sum_s' <a, a_s'> resid_0[s'],
+// so both steps' dot products are formed against x_0 in one round of loads, warp sums and cluster exchange, the
+// second step's are corrected with 16 x 16 entries of the Gram matrix (fetched alongside the rows), and the two
+// updates are applied one after the other, each rounded as in a round of its own.
 template <typename T, int ITERS>
 __device__ __forceinline__ void lsq_small_steps(cg::cluster_group& cluster, const StoreView& s, const LsqView& l,
                                                 bool active, int node, uint32_t event, int H, float lr, int csize,
@@ -329,7 +339,11 @@ __device__ __forceinline__ void lsq_small_steps(cg::cluster_group& cluster, cons
     }
   };
 
-  for (int q = 0; q < H; ++q) {
+  const bool in_pairs = l.gram != nullptr && one_group;
+  const float* gram = in_pairs ? l.gram + (int64_t)group * l.m * l.m : nullptr;
+  float4 b0[G], b1[G];                           // the second step's rows in a round of two steps
+
+  for (int q = 0; q < H;) {
     const int qq = q % kRowsAhead;
     if (active && qq == 0) {
       // minibatches (they depend on counters only) and their labels for the next kRowsAhead steps
@@ -341,6 +355,108 @@ __device__ __forceinline__ void lsq_small_steps(cg::cluster_group& cluster, cons
         sh.label[dq][si] = labels[r];
       }
       named_barrier(bar_id, kSmallThreads);
+    }
+    if (in_pairs && q + 1 < H) {
+      // ---- steps q and q + 1 in one round (q is even here, so both lie in the window drawn above)
+      const int* rows_p = sh.rows[qq + 1];
+      if (active) {
+        rows_q = sh.rows[qq];
+        float gv[2];                             // this thread's entries of the 16 x 16 Gram block
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int idx = ltid + e * kSmallThreads, a = idx / l.batch, b = idx - a * l.batch;
+          gv[e] = a < l.batch ? gram[(int64_t)rows_p[a] * l.m + rows_q[b]] : 0.0f;
+        }
+        load_group(0);
+#pragma unroll
+        for (int j = 0; j < G; ++j) {
+          const bool on = j < l.batch;
+          const T* row = A + (int64_t)rows_p[on ? j : 0] * s.pitch;
+          b0[j] = on ? load4_as_float<T>(row) : make_float4(0.f, 0.f, 0.f, 0.f);
+          b1[j] = (on && ITERS > 1) ? load4_as_float<T>(row + kSmallThreads * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        float acc[G], acc2[G];
+#pragma unroll
+        for (int j = 0; j < G; ++j) {
+          acc[j] = a0[j].x * x[0].x;
+          acc[j] = fmaf(a0[j].y, x[0].y, acc[j]); acc[j] = fmaf(a0[j].z, x[0].z, acc[j]); acc[j] = fmaf(a0[j].w, x[0].w, acc[j]);
+          acc[j] = fmaf(a1[j].x, x[1].x, acc[j]); acc[j] = fmaf(a1[j].y, x[1].y, acc[j]);
+          acc[j] = fmaf(a1[j].z, x[1].z, acc[j]); acc[j] = fmaf(a1[j].w, x[1].w, acc[j]);
+          acc2[j] = b0[j].x * x[0].x;
+          acc2[j] = fmaf(b0[j].y, x[0].y, acc2[j]); acc2[j] = fmaf(b0[j].z, x[0].z, acc2[j]); acc2[j] = fmaf(b0[j].w, x[0].w, acc2[j]);
+          acc2[j] = fmaf(b1[j].x, x[1].x, acc2[j]); acc2[j] = fmaf(b1[j].y, x[1].y, acc2[j]);
+          acc2[j] = fmaf(b1[j].z, x[1].z, acc2[j]); acc2[j] = fmaf(b1[j].w, x[1].w, acc2[j]);
+        }
+        int row, row2;
+        const float tot = reduce_rows<G>(acc, lane, row);
+        const float tot2 = reduce_rows<G>(acc2, lane, row2);
+        if ((lane & 1) == 0 && row < l.batch) { sh.red[warp][row] = tot; sh.red2[warp][row2] = tot2; }
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int idx = ltid + e * kSmallThreads, a = idx / l.batch, b = idx - a * l.batch;
+          if (a < l.batch) sh.gram[a][b] = gv[e];
+        }
+        named_barrier(bar_id, kSmallThreads);
+        // warp 0 finishes the first step's sums, warp 1 the second step's
+        if (ltid < l.batch) {
+          float t = 0.0f;
+#pragma unroll
+          for (int w = 0; w < kSmallThreads / 32; ++w) t += sh.red[w][ltid];
+          sh.part[ltid] = t;
+        } else if (ltid >= 32 && ltid - 32 < l.batch) {
+          float t = 0.0f;
+#pragma unroll
+          for (int w = 0; w < kSmallThreads / 32; ++w) t += sh.red2[w][ltid - 32];
+          sh.part2[ltid - 32] = t;
+        }
+      }
+      cluster.sync();                            // every CTA's partial sums of both steps are in place
+      if (active) {
+        float dot2 = 0.0f;
+        if (ltid < l.batch) {
+          float v[8];                            // remote reads issued together, summed in rank order
+#pragma unroll
+          for (int r = 0; r < 8; ++r) v[r] = r < csize ? *cluster.map_shared_rank(&sh.part[ltid], r) : 0.0f;
+          float t = 0.0f;
+#pragma unroll
+          for (int r = 0; r < 8; ++r) if (r < csize) t += v[r];
+          sh.resid[ltid] = row_residual(t, sh.label[qq][ltid], l.logistic);
+        } else if (ltid >= 32 && ltid - 32 < l.batch) {
+          float v[8];
+#pragma unroll
+          for (int r = 0; r < 8; ++r) v[r] = r < csize ? *cluster.map_shared_rank(&sh.part2[ltid - 32], r) : 0.0f;
+#pragma unroll
+          for (int r = 0; r < 8; ++r) if (r < csize) dot2 += v[r];
+        }
+        named_barrier(bar_id, kSmallThreads);
+        if (ltid >= 32 && ltid - 32 < l.batch) {
+          float corr = 0.0f;                     // <a, x_0 - x_1> / (lr/B) for the second step's row a
+          for (int b = 0; b < l.batch; ++b) corr = fmaf(sh.gram[ltid - 32][b], sh.resid[b], corr);
+          sh.resid2[ltid - 32] = row_residual(fmaf(-scale, corr, dot2), sh.label[qq + 1][ltid - 32], l.logistic);
+        }
+        named_barrier(bar_id, kSmallThreads);
+        float4 g0 = make_float4(0.f, 0.f, 0.f, 0.f), g1 = g0;
+#pragma unroll
+        for (int j = 0; j < G; ++j) {
+          const float rs = j < l.batch ? sh.resid[j] : 0.0f;
+          g0.x = fmaf(rs, a0[j].x, g0.x); g0.y = fmaf(rs, a0[j].y, g0.y); g0.z = fmaf(rs, a0[j].z, g0.z); g0.w = fmaf(rs, a0[j].w, g0.w);
+          g1.x = fmaf(rs, a1[j].x, g1.x); g1.y = fmaf(rs, a1[j].y, g1.y); g1.z = fmaf(rs, a1[j].z, g1.z); g1.w = fmaf(rs, a1[j].w, g1.w);
+        }
+        x[0].x -= scale * g0.x; x[0].y -= scale * g0.y; x[0].z -= scale * g0.z; x[0].w -= scale * g0.w;
+        x[1].x -= scale * g1.x; x[1].y -= scale * g1.y; x[1].z -= scale * g1.z; x[1].w -= scale * g1.w;
+        g0 = make_float4(0.f, 0.f, 0.f, 0.f); g1 = g0;
+#pragma unroll
+        for (int j = 0; j < G; ++j) {
+          const float rs = j < l.batch ? sh.resid2[j] : 0.0f;
+          g0.x = fmaf(rs, b0[j].x, g0.x); g0.y = fmaf(rs, b0[j].y, g0.y); g0.z = fmaf(rs, b0[j].z, g0.z); g0.w = fmaf(rs, b0[j].w, g0.w);
+          g1.x = fmaf(rs, b1[j].x, g1.x); g1.y = fmaf(rs, b1[j].y, g1.y); g1.z = fmaf(rs, b1[j].z, g1.z); g1.w = fmaf(rs, b1[j].w, g1.w);
+        }
+        x[0].x -= scale * g0.x; x[0].y -= scale * g0.y; x[0].z -= scale * g0.z; x[0].w -= scale * g0.w;
+        x[1].x -= scale * g1.x; x[1].y -= scale * g1.y; x[1].z -= scale * g1.z; x[1].w -= scale * g1.w;
+      }
+      cluster.sync();                            // all remote reads of part[] and part2[] are done before they are rewritten
+      q += 2;
+      continue;
     }
     rows_q = sh.rows[qq];
     if (active) {
@@ -392,6 +508,7 @@ __device__ __forceinline__ void lsq_small_steps(cg::cluster_group& cluster, cons
       x[1].x -= scale * g1.x; x[1].y -= scale * g1.y; x[1].z -= scale * g1.z; x[1].w -= scale * g1.w;
     }
     cluster.sync();                              // all remote reads of part[] are done before it is rewritten
+    ++q;
   }
   // data rows are zero past d, so coordinates past d have stayed zero
   if (active) {
@@ -558,6 +675,12 @@ cudaError_t launch_local_synth(const StoreView& s, const NodeList& nodes, int co
   local_synth_kernel<<<grid, 256, 0, st>>>(s, nodes, H, lr, grad_std, scalars_dev);
   ++*launches;
   return cudaGetLastError();
+}
+
+bool lsq_small_steps_in_pairs(int64_t pitch, int batch) {
+  if (pitch > kSmallMaxPitch) return false;
+  const int iters = pitch / (kSmallThreads * 4) <= 8 ? 1 : 2;
+  return batch <= 16 / iters;
 }
 
 cudaError_t launch_local_lsq(const StoreView& s, const LsqView& l, const NodeList& nodes, int count, int H,

@@ -616,7 +616,7 @@ lsq_tc_update_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
 }
 
 // =================================================================================================
-// Gram matrix of one data matrix: gram[i][j] = <A[i], A[j]> over the padded row (the padding is zero).
+// Gram matrix of one data matrix (bf16 or fp32): gram[i][j] = <A[i], A[j]> over the padded row (the padding is zero).
 // CTA = one 64 x 64 tile of the lower triangle (mirrored on store), thread = 4 x 4 entries; products are
 // summed in fp32 over 1024 coordinates at a time and in double across those runs, in coordinate order.
 // Runs once per data matrix (when the data is made or rewritten), not in the step.
@@ -624,15 +624,27 @@ lsq_tc_update_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
 constexpr int kGramTile = 64;
 constexpr int kGramK = 32;
 
+__device__ __forceinline__ void load8_as_float(const __nv_bfloat16* p, float v[8]) {
+  const uint4 raw = *reinterpret_cast<const uint4*>(p);
+  const __nv_bfloat16* h = reinterpret_cast<const __nv_bfloat16*>(&raw);
+#pragma unroll
+  for (int e = 0; e < 8; ++e) v[e] = __bfloat162float(h[e]);
+}
+__device__ __forceinline__ void load8_as_float(const float* p, float v[8]) {
+  const float4 lo = *reinterpret_cast<const float4*>(p), hi = *reinterpret_cast<const float4*>(p + 4);
+  v[0] = lo.x; v[1] = lo.y; v[2] = lo.z; v[3] = lo.w; v[4] = hi.x; v[5] = hi.y; v[6] = hi.z; v[7] = hi.w;
+}
+
+template <typename T>
 __global__ void __launch_bounds__(256)
-lsq_gram_kernel(const __nv_bfloat16* __restrict__ A, int m, int64_t pitch, int first_matrix, float* __restrict__ gram) {
+lsq_gram_kernel(const T* __restrict__ A, int m, int64_t pitch, int first_matrix, float* __restrict__ gram) {
   __shared__ __align__(16) float sa[kGramK][kGramTile + 4];
   __shared__ __align__(16) float sb[kGramK][kGramTile + 4];
   int ti = 0;
   while ((ti + 1) * (ti + 2) / 2 <= (int)blockIdx.x) ++ti;       // tile (ti, tj) of the lower triangle, tj <= ti
   const int tj = (int)blockIdx.x - ti * (ti + 1) / 2;
   const int matrix = first_matrix + (int)blockIdx.y;
-  const __nv_bfloat16* Ag = A + (int64_t)matrix * m * pitch;
+  const T* Ag = A + (int64_t)matrix * m * pitch;
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const int lrow = tid >> 2, c8 = (tid & 3) * 8;                 // staging: 64 rows x 4 groups of 8 coordinates
   const int ri = ti * kGramTile + lrow, rj = tj * kGramTile + lrow;
@@ -641,16 +653,14 @@ lsq_gram_kernel(const __nv_bfloat16* __restrict__ A, int m, int64_t pitch, int f
 #pragma unroll
   for (int e = 0; e < 16; ++e) { total[e] = 0.0; run[e] = 0.0f; }
   for (int64_t k0 = 0; k0 < pitch; k0 += kGramK) {
-    uint4 va = make_uint4(0, 0, 0, 0), vb = make_uint4(0, 0, 0, 0);
-    if (ri < m) va = *reinterpret_cast<const uint4*>(Ag + (int64_t)ri * pitch + k0 + c8);
-    if (rj < m) vb = *reinterpret_cast<const uint4*>(Ag + (int64_t)rj * pitch + k0 + c8);
-    const __nv_bfloat16* ha = reinterpret_cast<const __nv_bfloat16*>(&va);
-    const __nv_bfloat16* hb = reinterpret_cast<const __nv_bfloat16*>(&vb);
+    float va[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f}, vb[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    if (ri < m) load8_as_float(Ag + (int64_t)ri * pitch + k0 + c8, va);
+    if (rj < m) load8_as_float(Ag + (int64_t)rj * pitch + k0 + c8, vb);
     __syncthreads();                                             // the previous slice's readers are done
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
-      sa[c8 + e][lrow] = __bfloat162float(ha[e]);
-      sb[c8 + e][lrow] = __bfloat162float(hb[e]);
+      sa[c8 + e][lrow] = va[e];
+      sb[c8 + e][lrow] = vb[e];
     }
     __syncthreads();
 #pragma unroll 8
@@ -711,12 +721,15 @@ size_t lsq_tc_gram_bytes(int matrices, int m) {
 
 uint32_t lsq_tc_default_wait_limit() { return kSpinLimit; }
 
-cudaError_t launch_lsq_gram(const void* A_dev, int m, int64_t pitch, int first_matrix, int matrices, float* gram_dev,
-                            cudaStream_t st, int* launches) {
+cudaError_t launch_lsq_gram(const void* A_dev, int dtype, int m, int64_t pitch, int first_matrix, int matrices,
+                            float* gram_dev, cudaStream_t st, int* launches) {
   if (matrices == 0 || !gram_dev) return cudaSuccess;
   const int tiles = (m + kGramTile - 1) / kGramTile;
   const dim3 grid((unsigned)(tiles * (tiles + 1) / 2), (unsigned)matrices);
-  lsq_gram_kernel<<<grid, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(A_dev), m, pitch, first_matrix, gram_dev);
+  if (dtype == 1)
+    lsq_gram_kernel<<<grid, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(A_dev), m, pitch, first_matrix, gram_dev);
+  else
+    lsq_gram_kernel<<<grid, 256, 0, st>>>(reinterpret_cast<const float*>(A_dev), m, pitch, first_matrix, gram_dev);
   ++*launches;
   return cudaGetLastError();
 }

@@ -542,6 +542,29 @@ def test_tensor_core_steps_folded_four_at_a_time(H, objective):
         inject(orc, gpu, what=("X",))
 
 
+@pytest.mark.parametrize("d,batch,H,objective", [(700, 5, 2, 2), (4096, 16, 3, 2), (4096, 16, 5, 3), (6000, 8, 4, 2),
+                                                 (6000, 9, 4, 2), (8192, 8, 7, 3), (3000, 16, 10, 2)])
+def test_short_model_steps_taken_two_per_round(d, batch, H, objective):
+    """fp32 data, short models: where a minibatch fits the rows a thread keeps in flight (16 rows up to a row
+    pitch of 4096, 8 above) the cluster kernel takes two steps per round, the second step's inner products
+    corrected through the data's Gram matrix; an odd H ends with a round of one step, H > 8 crosses the window in
+    which minibatches are drawn ahead, batch 9 at the longer pitch stays one step per round. Fewer data rows than
+    two minibatches draw, so that the corrections are large, and a step size ten times the usual one."""
+    n, m = 6, 20
+    cfg = dict(objective=objective, lsq_m=m, lsq_batch=batch, lsq_dtype=0, lsq_groups=0, lsq_noise_std=0.3, init_std=0.5)
+    orc, gpu = make_pair(n, d, seed=131, **cfg)
+    orc.A[2] = (2.0 * orc.A[2][::-1]).astype(np.float32)          # rewritten data: the Gram matrix follows
+    inject(orc, gpu)
+    lr = 0.5
+    for nodes in (list(range(n)), [4, 2]):
+        assert orc.local_steps(nodes, H, lr) == 0 and gpu.local_steps(nodes, H, lr) == 0
+        gpu.sync()
+        for i in range(n):
+            assert rel_err(gpu.get(g.T_X, i), orc.X[i]) < TOL, i
+            assert gpu.get(g.T_COUNTERS, i)[1] == orc.ls[i]
+        inject(orc, gpu, what=("X",))
+
+
 def test_tensor_core_steps_one_at_a_time_when_the_gram_matrix_is_not_kept():
     """A data matrix of 8200 rows: its Gram matrix (269 MB) is above what the library keeps, so the steps take
     one pair of passes each; same results within the tolerance."""
