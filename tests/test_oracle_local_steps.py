@@ -103,6 +103,35 @@ def test_each_local_step_uses_the_running_iterate():
     assert s1.ls.tolist() == [0, 0, 3]
 
 
+def test_sequential_steps_equal_their_closed_form_through_the_gram_matrix():
+    """A step moves the model along its sampled rows only, x_q = x_0 - (lr/B) sum_{p<q} A_p^T r_p, so the inner
+    products of step q are A_q x_0 - (lr/B) sum_{p<q} (A_q A_p^T) r_p: H sequential steps of the oracle against
+    that recursion over blocks of A A^T, written out in double (rows repeat inside and across minibatches here:
+    10 rows, 4 draws a step)."""
+    H, lr = 4, 0.3
+    s = lsq(n=3, d=200, m=10, batch=4, noise=0.2, seed=9)
+    node = 1
+    A = s.A[node].astype(np.float64)
+    x0 = s.X[node].astype(np.float64)
+    rows = [s.minibatch_rows(node, q) for q in range(H)]
+    assert len({tuple(r.tolist()) for r in rows}) == H
+    gram = A @ A.T
+    scale = lr / 4
+    resid = []
+    for q in range(H):
+        score = A[rows[q]] @ x0
+        for p in range(q):
+            score -= scale * gram[np.ix_(rows[q], rows[p])] @ resid[p]
+        resid.append(score - s.bvec[node, rows[q]].astype(np.float64))
+    closed = x0 - scale * sum(A[rows[q]].T @ resid[q] for q in range(H))
+    assert s.local_steps([node], H, lr) == 0
+    assert np.abs(s.X[node] - closed).max() < 3e-7 * np.abs(closed).max()      # the oracle rounds x to fp32 per step
+    assert np.abs(closed - x0).max() > 1e-3 * np.abs(closed).max()
+    # without the correction terms the result is the one of H steps all taken at x_0: visibly different
+    naive = x0 - scale * sum(A[rows[q]].T @ (A[rows[q]] @ x0 - s.bvec[node, rows[q]]) for q in range(H))
+    assert np.abs(naive - closed).max() > 1e-4 * np.abs(closed).max()
+
+
 def test_synthetic_gradient_moments_and_op_order():
     n, d = 2, 40000
     s = o.OracleSwarm(n, d, "complete", seed=6)
