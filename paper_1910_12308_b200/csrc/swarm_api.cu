@@ -359,7 +359,9 @@ int apply_config(swarm_ctx* c, const swarm_config& wanted) {
   if (cfg.objective == SWARM_OBJ_LSQ || cfg.objective == SWARM_OBJ_LOGISTIC) {
     LsqView l = lsq_of(c);
     SW_CUDA(c, launch_lsq_data(s, l, c->A, c->xstar, c->bvec, c->scalars, cfg.lsq_noise_std, c->stream, &nl));
-    SW_CUDA(c, launch_lsq_gram(c->A, cfg.lsq_dtype, cfg.lsq_m, c->pitch, 0, c->groups, c->gram, c->stream, &nl));
+    SW_CUDA(c, launch_lsq_gram(c->A, cfg.lsq_dtype, cfg.lsq_m, c->pitch, 0, c->groups, c->gram, c->kernel_status,
+                               c->wait_limit, c->stream, &nl));
+    if (c->gram && cfg.lsq_dtype == SWARM_BF16) c->status_pending = true;   // its waits are bounded too
   }
   c->launches += nl;
   std::fill(c->w.begin(), c->w.end(), 0u);
@@ -1179,7 +1181,9 @@ static int tensor_access(swarm_ctx* c, int32_t which, int32_t node, void* host, 
       }
       // rewritten rows change the matrix's Gram matrix, which the grouped local steps read
       if (write)
-        SW_CUDA(c, launch_lsq_gram(c->A, c->cfg.lsq_dtype, c->cfg.lsq_m, c->pitch, node, 1, c->gram, c->stream, &nl));
+        SW_CUDA(c, launch_lsq_gram(c->A, c->cfg.lsq_dtype, c->cfg.lsq_m, c->pitch, node, 1, c->gram, c->kernel_status,
+                                   c->wait_limit, c->stream, &nl));
+      if (write && c->gram && c->cfg.lsq_dtype == SWARM_BF16) c->status_pending = true;
       c->launches += nl;
       SW_SYNC(c);
       return SWARM_OK;

@@ -145,10 +145,10 @@ size_t lsq_tc_resid_bytes(int units);
 // Bytes of the Gram matrices of `matrices` data matrices of m rows; 0 when they are too large to keep (local steps
 // then go one at a time instead of in groups).
 size_t lsq_tc_gram_bytes(int matrices, int m);
-// gram_dev[first_matrix .. first_matrix + matrices) = A A^T of those data matrices (dtype 1: bf16, else fp32; row
-// padding must be zero).
+// gram_dev[first_matrix .. first_matrix + matrices) = A A^T of those data matrices (dtype 1: bf16, on the tensor
+// cores, with bounded waits that raise *status_dev like the step kernels'; else fp32; row padding must be zero).
 cudaError_t launch_lsq_gram(const void* A_dev, int dtype, int m, int64_t pitch, int first_matrix, int matrices,
-                            float* gram_dev, cudaStream_t st, int* launches);
+                            float* gram_dev, int* status_dev, uint32_t wait_limit, cudaStream_t st, int* launches);
 // H steps of every unit, in groups of up to four steps per pair of passes when l.gram is set (one step otherwise).
 // status_dev: one int, set to 1 if a bounded wait inside a kernel expired (kernels that find it set return at
 // once); wait_limit: polls after which a wait on a tensor-core commit gives up.

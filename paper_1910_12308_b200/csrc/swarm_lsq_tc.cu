@@ -616,10 +616,148 @@ lsq_tc_update_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
 }
 
 // =================================================================================================
-// Gram matrix of one data matrix (bf16 or fp32): gram[i][j] = <A[i], A[j]> over the padded row (the padding is zero).
-// CTA = one 64 x 64 tile of the lower triangle (mirrored on store), thread = 4 x 4 entries; products are
-// summed in fp32 over 1024 coordinates at a time and in double across those runs, in coordinate order.
-// Runs once per data matrix (when the data is made or rewritten), not in the step.
+// Gram matrix of a bf16 data matrix on the tensor cores: gram = A A^T, a dense contraction with m x m outputs over
+// the row length. CTA = one 128 x 128 tile of the lower triangle (mirrored on store) over the whole row length;
+// stage = 64 coordinates of the tile's 128 + 128 rows (two K-major 128-byte-swizzled operand tiles of 16 KiB; a
+// diagonal tile uses one for both operands); M = N = 128, K = 16 per MMA. The accumulator runs in tensor memory
+// for 128 stages (8192 coordinates) at a time and is then added to per-thread double sums (thread = one row of the
+// tile x 64 columns), so the result does not depend on how a long running sum is rounded there. Waits are bounded
+// as in the step kernels. Runs once per data matrix (when the data is made or rewritten), not in the step.
+// =================================================================================================
+constexpr int kGtRows = 128;
+constexpr int kGtStages = 4;
+constexpr int kGtTileBytes = kGtRows * 128;                      // 16384
+constexpr int kGtRun = 128;                                      // stages per accumulation run in tensor memory
+constexpr int kGtSmem = kGtStages * 2 * kGtTileBytes + 1024 + 64;
+
+__global__ void __launch_bounds__(kTcThreads, 1)
+lsq_gram_tc_kernel(const __nv_bfloat16* __restrict__ A, int m, int64_t pitch, int first_matrix, float* __restrict__ gram,
+                   int* __restrict__ status, uint32_t spin_limit) {
+  __shared__ int poisoned;
+  if (status_raised(status, &poisoned)) return;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* sA = smem;                                            // per stage: the tile of rows i, then of rows j
+  uint64_t* bars = (uint64_t*)(sA + kGtStages * 2 * kGtTileBytes);
+  uint32_t* tmem_slot = (uint32_t*)(bars + 2);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  int ti = 0;
+  while ((ti + 1) * (ti + 2) / 2 <= (int)blockIdx.x) ++ti;       // tile (ti, tj) of the lower triangle, tj <= ti
+  const int tj = (int)blockIdx.x - ti * (ti + 1) / 2;
+  const bool diagonal = ti == tj;
+  const int matrix = first_matrix + (int)blockIdx.y;
+  const __nv_bfloat16* Ag = A + (int64_t)matrix * m * pitch;
+  const int i0 = ti * kGtRows, j0 = tj * kGtRows;
+  const int rows_i = min(kGtRows, m - i0), rows_j = min(kGtRows, m - j0);
+  const int nstages = (int)(pitch / 64);
+
+  if (tid == 0) {
+    mbar_init(smem_u32(&bars[0]), 1);
+    mbar_init(smem_u32(&bars[1]), 1);
+    fence_mbar_init();
+  }
+  if (warp == 0) { tmem_alloc(smem_u32(tmem_slot), 128); tmem_relinquish(); }
+  if (rows_i < kGtRows || rows_j < kGtRows)                      // rows past the matrix are never copied: they read as zero
+    for (int i = tid; i < kGtStages * 2 * kGtTileBytes / 16; i += kTcThreads) reinterpret_cast<uint4*>(sA)[i] = make_uint4(0, 0, 0, 0);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_d = *tmem_slot;
+
+  auto issue_loads = [&](int f) {
+    if (f < nstages) {
+      const uint32_t base_i = smem_u32(sA + (f % kGtStages) * 2 * kGtTileBytes), base_j = base_i + kGtTileBytes;
+      const int64_t k0 = (int64_t)f * 64;
+#pragma unroll
+      for (int it = 0; it < kGtRows * 8 / kTcThreads; ++it) {    // 128 rows x 8 chunks of 16 B per operand tile
+        const int idx = it * kTcThreads + tid;
+        const int r = idx >> 3, c = idx & 7;
+        const uint32_t off = (r >> 3) * 1024 + (r & 7) * 128 + ((c ^ (r & 7)) << 4);
+        if (r < rows_i) cp_async16(base_i + off, Ag + (int64_t)(i0 + r) * pitch + k0 + c * 8);
+        if (!diagonal && r < rows_j) cp_async16(base_j + off, Ag + (int64_t)(j0 + r) * pitch + k0 + c * 8);
+      }
+    }
+    cp_async_commit();
+  };
+
+  // this thread's share of the tile: row quad * 32 + lane, columns half * 64 .. + 63
+  const int quad = warp & 3, half = warp >> 2;
+  double total[64];
+#pragma unroll
+  for (int e = 0; e < 64; ++e) total[e] = 0.0;
+  bool ok = true;
+  int committed = -1;
+  for (int f = 0; f < kGtStages - 1; ++f) issue_loads(f);
+  constexpr uint32_t idesc = instr_desc_bf16(kGtRows, kGtRows, 0, 0);
+  for (int f = 0; f < nstages; ++f) {
+    cp_async_wait<kGtStages - 2>();                             // this thread's copies of stage f have landed
+    fence_proxy_async();
+    tc_fence_before();
+    ok = __syncthreads_and(ok);
+    if (!ok) break;
+    if (f >= 1) ok = mbar_wait(smem_u32(&bars[(f - 1) & 1]), ((f - 1) >> 1) & 1, spin_limit);
+    if (ok) issue_loads(f + kGtStages - 1); else cp_async_commit();   // into the stage of f - 1, whose MMAs have completed
+    if (tid == 0) {
+      tc_fence_after();
+      const uint32_t base_i = smem_u32(sA + (f % kGtStages) * 2 * kGtTileBytes);
+      const uint32_t base_j = diagonal ? base_i : base_i + kGtTileBytes;
+#pragma unroll
+      for (int ks = 0; ks < 4; ++ks) {                          // 16 coordinates (32 bytes) per MMA
+        const uint64_t da = smem_desc_sw128(base_i + ks * 32, 16, 1024);
+        const uint64_t db = smem_desc_sw128(base_j + ks * 32, 16, 1024);
+        tc_mma(tmem_d, da, db, idesc, ((f % kGtRun) | ks) != 0);
+      }
+      tc_commit(smem_u32(&bars[f & 1]));
+    }
+    committed = f;
+    if ((f + 1) % kGtRun == 0 || f == nstages - 1) {
+      // end of a run: once this stage's MMAs have completed, the accumulator joins the double sums; the next run's
+      // first MMA overwrites it after the next barrier, when every thread has read its part
+      const bool done = mbar_wait(smem_u32(&bars[f & 1]), (f >> 1) & 1, spin_limit);
+      ok = ok && done;
+      tc_fence_after();
+      if (ok) {
+#pragma unroll
+        for (int c8 = 0; c8 < 8; ++c8) {
+          float v[8];
+          tmem_ld8(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * 64 + c8 * 8), v);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) total[c8 * 8 + e] += (double)v[e];
+        }
+      }
+      tc_fence_before();
+    }
+  }
+  cp_async_wait<0>();
+  ok = __syncthreads_and(ok);
+  if (!ok) {
+    if (tid == 0) atomicExch(status, 1);
+    // gave up: wait for the last commit with the full default bound, so that tensor memory is not released under an MMA
+    if (committed >= 0) mbar_wait(smem_u32(&bars[committed & 1]), (committed >> 1) & 1, kSpinLimit);
+  } else {
+    float* G = gram + (int64_t)matrix * m * m;
+    const int i = i0 + quad * 32 + lane;
+    if (i < m) {
+#pragma unroll
+      for (int e = 0; e < 64; ++e) {
+        const int j = j0 + half * 64 + e;
+        if (j < m) {
+          const float v = (float)total[e];
+          G[(int64_t)i * m + j] = v;
+          G[(int64_t)j * m + i] = v;
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem_d, 128);
+}
+
+// =================================================================================================
+// Gram matrix of an fp32 data matrix (short models only, see the short-model step kernel): CTA = one 64 x 64 tile
+// of the lower triangle (mirrored on store), thread = 4 x 4 entries; products are summed in fp32 over 1024
+// coordinates at a time and in double across those runs, in coordinate order.
 // =================================================================================================
 constexpr int kGramTile = 64;
 constexpr int kGramK = 32;
@@ -721,19 +859,6 @@ size_t lsq_tc_gram_bytes(int matrices, int m) {
 
 uint32_t lsq_tc_default_wait_limit() { return kSpinLimit; }
 
-cudaError_t launch_lsq_gram(const void* A_dev, int dtype, int m, int64_t pitch, int first_matrix, int matrices,
-                            float* gram_dev, cudaStream_t st, int* launches) {
-  if (matrices == 0 || !gram_dev) return cudaSuccess;
-  const int tiles = (m + kGramTile - 1) / kGramTile;
-  const dim3 grid((unsigned)(tiles * (tiles + 1) / 2), (unsigned)matrices);
-  if (dtype == 1)
-    lsq_gram_kernel<<<grid, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(A_dev), m, pitch, first_matrix, gram_dev);
-  else
-    lsq_gram_kernel<<<grid, 256, 0, st>>>(reinterpret_cast<const float*>(A_dev), m, pitch, first_matrix, gram_dev);
-  ++*launches;
-  return cudaGetLastError();
-}
-
 namespace {
 
 template <int G>
@@ -757,13 +882,8 @@ void launch_group(const StoreView& s, const LsqView& l, const LsqUnit* units_dev
                                                                  wait_limit);
 }
 
-}  // namespace
-
-cudaError_t launch_local_lsq_tc(const StoreView& s, const LsqView& l, const LsqUnit* units_dev, int nunits, int max_units,
-                                int H, float lr, float* partial_dev, void* resid_dev, int* status_dev,
-                                uint32_t wait_limit, cudaStream_t st, int* launches) {
-  if (nunits == 0 || H == 0) return cudaSuccess;
-  if (l.batch > kTcBatch || l.dtype != 1) return cudaErrorInvalidValue;
+// Once per device: the dynamic shared-memory sizes of the tensor-core kernels.
+cudaError_t ensure_attributes() {
   static bool attr_set[64] = {};
   static std::mutex attr_mutex;                   // contexts on different threads may reach this together
   std::lock_guard<std::mutex> lock(attr_mutex);
@@ -774,8 +894,42 @@ cudaError_t launch_local_lsq_tc(const StoreView& s, const LsqView& l, const LsqU
     if (e == cudaSuccess) e = set_group_attributes<2>();
     if (e == cudaSuccess) e = set_group_attributes<3>();
     if (e == cudaSuccess) e = set_group_attributes<4>();
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(lsq_gram_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGtSmem);
     if (e != cudaSuccess) return e;
     attr_set[dev] = true;
+  }
+  return cudaSuccess;
+}
+
+}  // namespace
+
+cudaError_t launch_lsq_gram(const void* A_dev, int dtype, int m, int64_t pitch, int first_matrix, int matrices,
+                            float* gram_dev, int* status_dev, uint32_t wait_limit, cudaStream_t st, int* launches) {
+  if (matrices == 0 || !gram_dev) return cudaSuccess;
+  if (dtype == 1) {
+    const cudaError_t e = ensure_attributes();
+    if (e != cudaSuccess) return e;
+    const int tiles = (m + kGtRows - 1) / kGtRows;
+    const dim3 grid((unsigned)(tiles * (tiles + 1) / 2), (unsigned)matrices);
+    lsq_gram_tc_kernel<<<grid, kTcThreads, kGtSmem, st>>>(reinterpret_cast<const __nv_bfloat16*>(A_dev), m, pitch, first_matrix,
+                                                          gram_dev, status_dev, wait_limit);
+  } else {
+    const int tiles = (m + kGramTile - 1) / kGramTile;
+    const dim3 grid((unsigned)(tiles * (tiles + 1) / 2), (unsigned)matrices);
+    lsq_gram_kernel<<<grid, 256, 0, st>>>(reinterpret_cast<const float*>(A_dev), m, pitch, first_matrix, gram_dev);
+  }
+  ++*launches;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_local_lsq_tc(const StoreView& s, const LsqView& l, const LsqUnit* units_dev, int nunits, int max_units,
+                                int H, float lr, float* partial_dev, void* resid_dev, int* status_dev,
+                                uint32_t wait_limit, cudaStream_t st, int* launches) {
+  if (nunits == 0 || H == 0) return cudaSuccess;
+  if (l.batch > kTcBatch || l.dtype != 1) return cudaErrorInvalidValue;
+  {
+    const cudaError_t e = ensure_attributes();
+    if (e != cudaSuccess) return e;
   }
   if (nunits > max_units) return cudaErrorInvalidValue;
   auto* resid = reinterpret_cast<__nv_bfloat16*>(resid_dev);
