@@ -268,7 +268,9 @@ enum {
   SWARM_T_OEXPS = 11,   /* nblk int8: exponents of the own register                                         */
   SWARM_T_CLOCKS = 12,  /* 2 uint32: write counter of the own register, staleness clock tau                 */
   SWARM_T_MU_RECORD = 13, /* d floats: mean model at the node's last initiation (ESTATE unless tracking)    */
-  SWARM_T_A_RECORD = 14   /* 1 double: ||snapshot - mean||^2 at the node's last initiation                  */
+  SWARM_T_A_RECORD = 14,  /* 1 double: ||snapshot - mean||^2 at the node's last initiation                  */
+  SWARM_T_GRAM = 15       /* node = data-matrix id; lsq_m*lsq_m floats: the matrix's Gram matrix A A^T, kept for the
+                             local steps that are evaluated several at a time (read-only; ESTATE when not kept) */
 };
 int swarm_get_tensor(swarm_ctx *ctx, int32_t which, int32_t node, void *dst_host, size_t bytes);
 /* The same read queued on the context's stream without waiting: dst_host (any host memory, which must stay

@@ -21,7 +21,8 @@ TOPO_COMPLETE, TOPO_RING, TOPO_REGULAR = 0, 1, 2
 OBJ_NONE, OBJ_SYNTH, OBJ_LSQ, OBJ_LOGISTIC = 0, 1, 2, 3
 F32, BF16 = 0, 1
 OK, EINVAL, ERANGE, EPAIR, ESTATE, ENOMEM, ECUDA = 0, -1, -2, -3, -4, -5, -6
-T_X, T_B, T_CODES, T_EXPS, T_ADJ, T_A, T_BVEC, T_XSTAR, T_SCALARS, T_COUNTERS, T_OWN, T_OEXPS, T_CLOCKS, T_MU_RECORD, T_A_RECORD = range(15)
+(T_X, T_B, T_CODES, T_EXPS, T_ADJ, T_A, T_BVEC, T_XSTAR, T_SCALARS, T_COUNTERS, T_OWN, T_OEXPS, T_CLOCKS, T_MU_RECORD,
+ T_A_RECORD, T_GRAM) = range(16)
 TOPOLOGY = {"complete": TOPO_COMPLETE, "ring": TOPO_RING, "regular": TOPO_REGULAR}
 
 EXPORTS = [
@@ -354,6 +355,7 @@ class Swarm:
             T_BVEC: (np.float32, m), T_XSTAR: (np.float32, self.d), T_SCALARS: (np.float32, 3),
             T_COUNTERS: (np.uint32, 3), T_OWN: (np.uint8, self.nblk * 2048), T_OEXPS: (np.int8, self.nblk),
             T_CLOCKS: (np.uint32, 2), T_MU_RECORD: (np.float32, self.d), T_A_RECORD: (np.float64, 1),
+            T_GRAM: (np.float32, m * m),
         }[which]
 
     def get(self, which, node=0):

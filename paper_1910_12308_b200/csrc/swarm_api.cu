@@ -1099,7 +1099,7 @@ static int tensor_access(swarm_ctx* c, int32_t which, int32_t node, void* host, 
   // rows that live in host mirrors or need a conversion pass have no asynchronous form
   if (!wait && (which == SWARM_T_ADJ || which == SWARM_T_COUNTERS || which == SWARM_T_CLOCKS || which == SWARM_T_A))
     return SWARM_EINVAL;
-  const bool per_node = which != SWARM_T_XSTAR && which != SWARM_T_A;
+  const bool per_node = which != SWARM_T_XSTAR && which != SWARM_T_A && which != SWARM_T_GRAM;
   if (per_node && (node < 0 || node >= c->n)) return SWARM_ERANGE;
   DeviceGuard guard(c->device);
   const size_t d = (size_t)c->d;
@@ -1136,6 +1136,13 @@ static int tensor_access(swarm_ctx* c, int32_t which, int32_t node, void* host, 
     case SWARM_T_A_RECORD:
       if (!c->track) return SWARM_ESTATE;
       dev = c->a_hist + node; want = 8; break;
+    case SWARM_T_GRAM: {
+      if (!c->gram) return SWARM_ESTATE;
+      if (write) return SWARM_EINVAL;
+      if (node < 0 || node >= c->groups) return SWARM_ERANGE;
+      const size_t m = (size_t)c->cfg.lsq_m;
+      dev = c->gram + (size_t)node * m * m; want = m * m * 4; break;
+    }
     case SWARM_T_CLOCKS: {
       if (bytes != 8) return SWARM_EINVAL;
       uint32_t* v = (uint32_t*)host;

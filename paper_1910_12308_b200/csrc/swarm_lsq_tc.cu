@@ -620,14 +620,15 @@ lsq_tc_update_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
 // the row length. CTA = one 128 x 128 tile of the lower triangle (mirrored on store) over the whole row length;
 // stage = 64 coordinates of the tile's 128 + 128 rows (two K-major 128-byte-swizzled operand tiles of 16 KiB; a
 // diagonal tile uses one for both operands); M = N = 128, K = 16 per MMA. The accumulator runs in tensor memory
-// for 128 stages (8192 coordinates) at a time and is then added to per-thread double sums (thread = one row of the
-// tile x 64 columns), so the result does not depend on how a long running sum is rounded there. Waits are bounded
-// as in the step kernels. Runs once per data matrix (when the data is made or rewritten), not in the step.
+// for 32 stages (2048 coordinates, 128 MMAs) at a time and is then added to per-thread double sums (thread = one
+// row of the tile x 64 columns): the fp32 additions in tensor memory were measured to lose up to 3e-8 of the running
+// sum each, all in one direction (1.9e-6 of a diagonal entry after 64 MMAs), so a run is kept to 128 of them
+// (< 8e-6 of the entry; what reaches a residual is that times lr/B). Waits are bounded as in the step kernels. Runs once per data matrix (when the data is made or rewritten), not in the step.
 // =================================================================================================
 constexpr int kGtRows = 128;
 constexpr int kGtStages = 4;
 constexpr int kGtTileBytes = kGtRows * 128;                      // 16384
-constexpr int kGtRun = 128;                                      // stages per accumulation run in tensor memory
+constexpr int kGtRun = 32;                                       // stages per accumulation run in tensor memory
 constexpr int kGtSmem = kGtStages * 2 * kGtTileBytes + 1024 + 64;
 
 __global__ void __launch_bounds__(kTcThreads, 1)

@@ -565,6 +565,37 @@ def test_short_model_steps_taken_two_per_round(d, batch, H, objective):
         inject(orc, gpu, what=("X",))
 
 
+@pytest.mark.parametrize("d,m,dtype,groups", [(700, 48, 1, 2), (9000, 130, 1, 3), (70000, 300, 1, 1), (3000, 129, 1, 0),
+                                              (4096, 20, 0, 0), (8000, 70, 0, 2)])
+def test_gram_matrices_of_the_data(d, m, dtype, groups):
+    """The Gram matrices that the folded local steps read, against A A^T in double from the oracle's copy of the
+    data: bf16 data on the tensor cores (one, two and three 128-row tiles, ragged last tiles, off-diagonal tiles,
+    rows shorter and longer than one accumulation run of 8192 coordinates), fp32 data of short models on the CUDA
+    cores; and again after one matrix has been rewritten."""
+    n = 6
+    cfg = dict(objective=2, lsq_m=m, lsq_batch=8, lsq_dtype=dtype, lsq_groups=groups, lsq_noise_std=0.1)
+    orc, gpu = make_pair(n, d, seed=77, **cfg)
+    inject(orc, gpu)
+    ngroups = groups if groups else n
+
+    def check():
+        for grp in range(ngroups):
+            A = orc.A[grp].astype(np.float64)
+            want = A @ A.T
+            got = gpu.get(g.T_GRAM, grp).reshape(m, m)
+            assert np.array_equal(got, got.T), grp
+            # tensor cores: runs of 128 fp32 accumulations in tensor memory, each off by up to 2^-24 of the running
+            # sum in one direction, then double; CUDA cores: fp32 runs of 1024 products rounded to nearest, then double
+            assert np.abs(got - want).max() < (8e-6 if dtype == 1 else 1e-6) * np.abs(want).max(), grp
+    check()
+    last = ngroups - 1
+    orc.A[last] = (0.5 * orc.A[last][::-1]).astype(np.float32)        # exact in bf16
+    gpu.set(g.T_A, last, orc.A[last])
+    check()
+    assert gpu._L.swarm_get_tensor(gpu._h, g.T_GRAM, ngroups, np.empty(m * m, np.float32).ctypes.data, m * m * 4) == g.ERANGE
+    assert gpu._L.swarm_set_tensor(gpu._h, g.T_GRAM, 0, np.zeros(m * m, np.float32).ctypes.data, m * m * 4) == g.EINVAL
+
+
 def test_tensor_core_steps_one_at_a_time_when_the_gram_matrix_is_not_kept():
     """A data matrix of 8200 rows: its Gram matrix (269 MB) is above what the library keeps, so the steps take
     one pair of passes each; same results within the tolerance."""
