@@ -146,13 +146,16 @@ __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bflo
 
 constexpr int kTcMaxGroup = 4;            // steps folded into one pair of passes
 
-// The rows of steps step0 .. step0 + G - 1 of a unit (slots beyond the batch size hold row 0 and are never read
-// as data: their tiles are zero and their residuals are zero).
+// The rows of steps step0 .. step0 + G - 1 of a unit, as element offsets of the rows within their data matrix
+// (row * pitch), so that a copy's source address is one addition away (slots beyond the batch size hold row 0
+// and are never read as data: their tiles are zero and their residuals are zero).
 template <int G>
-__device__ __forceinline__ void draw_rows(int* rows, const LsqView& l, int group, uint32_t event0, const StoreView& s) {
+__device__ __forceinline__ void draw_rows(int64_t* row_off, const LsqView& l, int group, uint32_t event0,
+                                          const StoreView& s) {
   for (int i = threadIdx.x; i < G * kTcBatch; i += blockDim.x) {
     const int q = i / kTcBatch, sidx = i % kTcBatch;
-    rows[i] = sidx < l.batch ? tc_minibatch_row(sidx, group, event0 + (uint32_t)q, l.m, s.key0, s.key1) : 0;
+    const int row = sidx < l.batch ? tc_minibatch_row(sidx, group, event0 + (uint32_t)q, l.m, s.key0, s.key1) : 0;
+    row_off[i] = (int64_t)row * s.pitch;
   }
 }
 
@@ -194,7 +197,7 @@ lsq_tc_scores_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
   uint8_t* sXop = sA + kResStages * kResABytes;                 // [buf][hi|lo]
   uint64_t* bars = (uint64_t*)(sXop + 4 * kResXopBytes);        // mma_done[2]
   uint32_t* tmem_slot = (uint32_t*)(bars + 2);
-  __shared__ int rows[G * kTcBatch];
+  __shared__ int64_t row_off[G * kTcBatch];
   __shared__ int unodes[kUnitNodes];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -207,7 +210,7 @@ lsq_tc_scores_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
   const int nstages = ntiles * G;
   const __nv_bfloat16* A = reinterpret_cast<const __nv_bfloat16*>(l.A) + (int64_t)u.group * l.m * s.pitch;
 
-  draw_rows<G>(rows, l, u.group, up->event + (uint32_t)step, s);
+  draw_rows<G>(row_off, l, u.group, up->event + (uint32_t)step, s);
   if (tid == 0) {
     mbar_init(smem_u32(&bars[0]), 1);
     mbar_init(smem_u32(&bars[1]), 1);
@@ -222,23 +225,21 @@ lsq_tc_scores_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
   tc_fence_after();
   const uint32_t tmem_d = *tmem_slot;
 
+  // A: 64 rows x 16 chunks of 16 B per stage; this thread copies chunk tid % 16 (16 B of the 256-byte row slice) of
+  // rows tid / 16 + 16 it, it = 0..3: the same place within an 8-row group every time, 2048 B further per it
+  const int crow = tid >> 4, cchunk = tid & 15;
+  const uint32_t cdst = smem_u32(sA) + (cchunk >> 3) * (kTcBatch * 128) + (crow >> 3) * 1024 + (crow & 7) * 128 +
+                        (((cchunk & 7) ^ (crow & 7)) << 4);
+  const __nv_bfloat16* csrc = A + kbase + cchunk * 8;
   auto issue_loads = [&](int f) {
     if (f < nstages) {
       const int tile = f / G, q = f - tile * G;
-      const int st = f % kResStages;
-      const int64_t k0 = kbase + (int64_t)tile * kResTile;
-      // A: 64 rows x 16 chunks of 16 B; thread -> (row = idx / 16, chunk = idx % 16)
-      const uint32_t a_base = smem_u32(sA + st * kResABytes);
+      const uint32_t dst = cdst + (f % kResStages) * kResABytes;
+      const __nv_bfloat16* src = csrc + tile * kResTile;
+      const int64_t* off = row_off + q * kTcBatch + crow;
 #pragma unroll
-      for (int it = 0; it < kTcBatch * 16 / kTcThreads; ++it) {
-        const int idx = it * kTcThreads + tid;
-        const int r = idx >> 4, c = idx & 15;               // c: 16-byte chunk within the 256-byte row slice
-        if (r < l.batch) {
-          const int atom = c >> 3, cc = c & 7;
-          const uint32_t dst = a_base + atom * (kTcBatch * 128) + (r >> 3) * 1024 + (r & 7) * 128 + ((cc ^ (r & 7)) << 4);
-          cp_async16(dst, A + (int64_t)rows[q * kTcBatch + r] * s.pitch + k0 + c * 8);
-        }
-      }
+      for (int it = 0; it < kTcBatch * 16 / kTcThreads; ++it)
+        if (crow + 16 * it < l.batch) cp_async16(dst + it * 2048, src + off[16 * it]);
     }
     cp_async_commit();
   };
@@ -259,6 +260,7 @@ lsq_tc_scores_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
   int committed = -1;              // last stage whose MMAs were committed (the same in every thread)
   for (int f = 0; f < kResStages - 1; ++f) issue_loads(f);
   constexpr uint32_t idesc = instr_desc_bf16(kTcBatch, 2 * kUnitNodes, 0, 0);   // N = 32: hi and lo side by side
+  const uint64_t desc_a0 = smem_desc_sw128(smem_u32(sA), 16, 1024), desc_x0 = smem_desc_sw128(smem_u32(sXop), 16, 1024);
   float4 xcur[2], xnext[2];
   load_x(0, xcur);
   for (int f = 0; f < nstages; ++f) {
@@ -297,17 +299,17 @@ lsq_tc_scores_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
     if (ok) issue_loads(f + kResStages - 1); else cp_async_commit();
     if (tid == 0) {
       tc_fence_after();
-      const uint32_t a_base = smem_u32(sA + st * kResABytes);
-      const uint32_t x_base = smem_u32(sXop + buf * (2 * kResXopBytes));
+      // a descriptor's low bits hold the operand's shared-memory address / 16 (all of shared memory fits them), so
+      // the descriptors of a stage, an atom and a 16-coordinate slice are additions to the first one
+      const uint64_t da0 = desc_a0 + (uint64_t)((st * kResABytes) >> 4);
+      const uint64_t dx0 = desc_x0 + (uint64_t)((buf * 2 * kResXopBytes) >> 4);
       const uint32_t d_addr = tmem_d + (uint32_t)(q * 2 * kUnitNodes);
 #pragma unroll
       for (int atom = 0; atom < kResAtoms; ++atom)
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks) {                    // 16 coordinates (32 bytes) per MMA
-          const uint64_t da = smem_desc_sw128(a_base + atom * (kTcBatch * 128) + ks * 32, 16, 1024);
-          const uint64_t dx = smem_desc_sw128(x_base + atom * (2 * kUnitNodes * 128) + ks * 32, 16, 1024);
-          tc_mma(d_addr, da, dx, idesc, (t | atom | ks) != 0);
-        }
+        for (int ks = 0; ks < 4; ++ks)                      // 16 coordinates (32 bytes) per MMA
+          tc_mma(d_addr, da0 + (uint64_t)((atom * (kTcBatch * 128) + ks * 32) >> 4),
+                 dx0 + (uint64_t)((atom * (2 * kUnitNodes * 128) + ks * 32) >> 4), idesc, (t | atom | ks) != 0);
       tc_commit(smem_u32(&bars[f & 1]));
     }
     committed = f;
@@ -477,7 +479,7 @@ lsq_tc_update_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
   uint8_t* sR = sA + kStages * kUpdABytes;                      // per step: hi then lo
   uint64_t* bars = (uint64_t*)(sR + G * 2 * kUpdRBytes);
   uint32_t* tmem_slot = (uint32_t*)(bars + 2);
-  __shared__ int rows[G * kTcBatch];
+  __shared__ int64_t row_off[G * kTcBatch];
   __shared__ int unodes[kUnitNodes];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -491,7 +493,7 @@ lsq_tc_update_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
   const __nv_bfloat16* A = reinterpret_cast<const __nv_bfloat16*>(l.A) + (int64_t)u.group * l.m * s.pitch;
   const float scale = lr / (float)l.batch;
 
-  draw_rows<G>(rows, l, u.group, up->event + (uint32_t)step, s);
+  draw_rows<G>(row_off, l, u.group, up->event + (uint32_t)step, s);
   if (tid == 0) {
     mbar_init(smem_u32(&bars[0]), 1);
     mbar_init(smem_u32(&bars[1]), 1);
@@ -514,23 +516,21 @@ lsq_tc_update_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
                  resid + ((int64_t)blockIdx.y * G + q) * (2 * kUnitNodes * kTcBatch) + which * (kUnitNodes * kTcBatch) +
                      r * kTcBatch + c * 8);
   }
+  // 64 rows x 16 chunks of 16 B per stage; this thread copies chunk tid % 16 of rows tid / 16 + 16 it, it = 0..3:
+  // the same place within an 8-row group every time, 2048 B further per it
+  const int crow = tid >> 4, cchunk = tid & 15;
+  const uint32_t cdst = smem_u32(sA) + (cchunk >> 3) * 8192 + (crow >> 3) * 1024 + (crow & 7) * 128 +
+                        (((cchunk & 7) ^ (crow & 7)) << 4);
+  const __nv_bfloat16* csrc = A + kbase + cchunk * 8;
   auto issue_loads = [&](int f) {
     if (f < nstages) {
       const int tile = f / G, q = f - tile * G;
-      const int st = f % kStages;
-      const int64_t k0 = kbase + (int64_t)tile * kUpdTile;
-      const uint32_t a_base = smem_u32(sA + st * kUpdABytes);
-      // 64 rows x 16 chunks of 16 B: thread -> (row = idx / 16, chunk = idx % 16)
+      const uint32_t dst = cdst + (f % kStages) * kUpdABytes;
+      const __nv_bfloat16* src = csrc + tile * kUpdTile;
+      const int64_t* off = row_off + q * kTcBatch + crow;
 #pragma unroll
-      for (int it = 0; it < kTcBatch * 16 / kTcThreads; ++it) {
-        const int idx = it * kTcThreads + tid;
-        const int r = idx >> 4, c = idx & 15;
-        if (r < l.batch) {
-          const int half = c >> 3, cc = c & 7;
-          const uint32_t dst = a_base + half * 8192 + (r >> 3) * 1024 + (r & 7) * 128 + ((cc ^ (r & 7)) << 4);
-          cp_async16(dst, A + (int64_t)rows[q * kTcBatch + r] * s.pitch + k0 + c * 8);
-        }
-      }
+      for (int it = 0; it < kTcBatch * 16 / kTcThreads; ++it)
+        if (crow + 16 * it < l.batch) cp_async16(dst + it * 2048, src + off[16 * it]);
     }
     cp_async_commit();
   };
@@ -561,6 +561,7 @@ lsq_tc_update_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
   int committed = -1;              // last stage whose MMAs were committed (the same in every thread)
   for (int f = 0; f < kStages - 1; ++f) issue_loads(f);
   constexpr uint32_t idesc = instr_desc_bf16(kUpdTile, 2 * kUnitNodes, 1, 0);   // N = 32: hi and lo residuals side by side
+  const uint64_t desc_a0 = smem_desc_sw128(smem_u32(sA), 8192, 1024), desc_r0 = smem_desc_sw128(smem_u32(sR), 16, 1024);
   float xprev[8], xcur[8];
   for (int f = 0; f < nstages; ++f) {
     const int t = f / G, q = f - t * G;
@@ -573,14 +574,13 @@ lsq_tc_update_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
     if (!ok) break;                                         // and the give-up decision is CTA-uniform
     if (tid == 0) {
       tc_fence_after();
-      const uint32_t a_base = smem_u32(sA + st * kUpdABytes);
-      const uint32_t r_base = smem_u32(sR + q * 2 * kUpdRBytes);   // rows 0..15 hi, rows 16..31 lo
+      // descriptors of a stage and of a 16-row slice: additions to the first one (address / 16 in the low bits)
+      const uint64_t da0 = desc_a0 + (uint64_t)((st * kUpdABytes) >> 4);
+      const uint64_t dr0 = desc_r0 + (uint64_t)((q * 2 * kUpdRBytes) >> 4);   // rows 0..15 hi, rows 16..31 lo
 #pragma unroll
-      for (int ks = 0; ks < 4; ++ks) {                      // 16 sampled rows per MMA = two 8-row groups
-        const uint64_t da = smem_desc_sw128(a_base + ks * 2048, 8192, 1024);
-        const uint64_t dr = smem_desc_sw128(r_base + ks * 32, 16, 1024);
-        tc_mma(tmem_d + buf * 2 * kUnitNodes, da, dr, idesc, (q | ks) != 0);
-      }
+      for (int ks = 0; ks < 4; ++ks)                        // 16 sampled rows per MMA = two 8-row groups
+        tc_mma(tmem_d + buf * 2 * kUnitNodes, da0 + (uint64_t)((ks * 2048) >> 4), dr0 + (uint64_t)((ks * 32) >> 4), idesc,
+               (q | ks) != 0);
       tc_commit(smem_u32(&bars[f & 1]));
     }
     committed = f;
