@@ -230,16 +230,22 @@ lsq_tc_scores_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
   const int crow = tid >> 4, cchunk = tid & 15;
   const uint32_t cdst = smem_u32(sA) + (cchunk >> 3) * (kTcBatch * 128) + (crow >> 3) * 1024 + (crow & 7) * 128 +
                         (((cchunk & 7) ^ (crow & 7)) << 4);
-  const __nv_bfloat16* csrc = A + kbase + cchunk * 8;
-  auto issue_loads = [&](int f) {
-    if (f < nstages) {
-      const int tile = f / G, q = f - tile * G;
-      const uint32_t dst = cdst + (f % kResStages) * kResABytes;
-      const __nv_bfloat16* src = csrc + tile * kResTile;
-      const int64_t* off = row_off + q * kTcBatch + crow;
+  int cmask = 0;                                                // which of its four rows exist (batch size)
+#pragma unroll
+  for (int it = 0; it < 4; ++it) cmask |= (crow + 16 * it < l.batch) << it;
+  // the stage that the next call copies: destination, source tile, step within the tile, stage buffer, stages left
+  uint32_t ld_dst = cdst;
+  const __nv_bfloat16* ld_src = A + kbase + cchunk * 8;
+  int ld_q = 0, ld_st = 0, ld_left = nstages;
+  auto issue_loads = [&]() {
+    if (ld_left > 0) {
+      const int64_t* off = row_off + ld_q * kTcBatch + crow;
 #pragma unroll
       for (int it = 0; it < kTcBatch * 16 / kTcThreads; ++it)
-        if (crow + 16 * it < l.batch) cp_async16(dst + it * 2048, src + off[16 * it]);
+        if (cmask & (1 << it)) cp_async16(ld_dst + it * 2048, ld_src + off[16 * it]);
+      --ld_left;
+      if (++ld_q == G) { ld_q = 0; ld_src += kResTile; }
+      if (++ld_st == kResStages) { ld_st = 0; ld_dst = cdst; } else ld_dst += kResABytes;
     }
     cp_async_commit();
   };
@@ -258,14 +264,13 @@ lsq_tc_scores_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
 
   bool ok = true;                  // this warp's waits so far
   int committed = -1;              // last stage whose MMAs were committed (the same in every thread)
-  for (int f = 0; f < kResStages - 1; ++f) issue_loads(f);
+  for (int f = 0; f < kResStages - 1; ++f) issue_loads();
   constexpr uint32_t idesc = instr_desc_bf16(kTcBatch, 2 * kUnitNodes, 0, 0);   // N = 32: hi and lo side by side
   const uint64_t desc_a0 = smem_desc_sw128(smem_u32(sA), 16, 1024), desc_x0 = smem_desc_sw128(smem_u32(sXop), 16, 1024);
   float4 xcur[2], xnext[2];
   load_x(0, xcur);
-  for (int f = 0; f < nstages; ++f) {
-    const int t = f / G, q = f - t * G;
-    const int st = f % kResStages, buf = t & 1;
+  for (int f = 0, t = 0, q = 0, st = 0; f < nstages; ++f) {
+    const int buf = t & 1;
     if (q == 0) load_x(t + 1, xnext);                       // consumed one tile later
     cp_async_wait<kResStages - 2>();                        // this thread's copies of stage f have landed
     if (q == 0 && ok) {
@@ -296,7 +301,7 @@ lsq_tc_scores_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
     // are issued, so that the issue does not hold back warp 0's copies; a warp whose wait expired leaves that stage
     // alone and reports at the next barrier
     if (f >= 1) ok = mbar_wait(smem_u32(&bars[(f - 1) & 1]), ((f - 1) >> 1) & 1, spin_limit);
-    if (ok) issue_loads(f + kResStages - 1); else cp_async_commit();
+    if (ok) issue_loads(); else cp_async_commit();
     if (tid == 0) {
       tc_fence_after();
       // a descriptor's low bits hold the operand's shared-memory address / 16 (all of shared memory fits them), so
@@ -313,6 +318,8 @@ lsq_tc_scores_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
       tc_commit(smem_u32(&bars[f & 1]));
     }
     committed = f;
+    if (++q == G) { q = 0; ++t; }
+    if (++st == kResStages) st = 0;
   }
   cp_async_wait<0>();
   if (ok && committed >= 0) ok = mbar_wait(smem_u32(&bars[committed & 1]), (committed >> 1) & 1, spin_limit);
@@ -521,16 +528,22 @@ lsq_tc_update_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
   const int crow = tid >> 4, cchunk = tid & 15;
   const uint32_t cdst = smem_u32(sA) + (cchunk >> 3) * 8192 + (crow >> 3) * 1024 + (crow & 7) * 128 +
                         (((cchunk & 7) ^ (crow & 7)) << 4);
-  const __nv_bfloat16* csrc = A + kbase + cchunk * 8;
-  auto issue_loads = [&](int f) {
-    if (f < nstages) {
-      const int tile = f / G, q = f - tile * G;
-      const uint32_t dst = cdst + (f % kStages) * kUpdABytes;
-      const __nv_bfloat16* src = csrc + tile * kUpdTile;
-      const int64_t* off = row_off + q * kTcBatch + crow;
+  int cmask = 0;                                                // which of its four rows exist (batch size)
+#pragma unroll
+  for (int it = 0; it < 4; ++it) cmask |= (crow + 16 * it < l.batch) << it;
+  // the stage that the next call copies: destination, source tile, step within the tile, stage buffer, stages left
+  uint32_t ld_dst = cdst;
+  const __nv_bfloat16* ld_src = A + kbase + cchunk * 8;
+  int ld_q = 0, ld_st = 0, ld_left = nstages;
+  auto issue_loads = [&]() {
+    if (ld_left > 0) {
+      const int64_t* off = row_off + ld_q * kTcBatch + crow;
 #pragma unroll
       for (int it = 0; it < kTcBatch * 16 / kTcThreads; ++it)
-        if (crow + 16 * it < l.batch) cp_async16(dst + it * 2048, src + off[16 * it]);
+        if (cmask & (1 << it)) cp_async16(ld_dst + it * 2048, ld_src + off[16 * it]);
+      --ld_left;
+      if (++ld_q == G) { ld_q = 0; ld_src += kUpdTile; }
+      if (++ld_st == kStages) { ld_st = 0; ld_dst = cdst; } else ld_dst += kUpdABytes;
     }
     cp_async_commit();
   };
@@ -559,13 +572,12 @@ lsq_tc_update_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
 
   bool ok = true;                  // this warp's waits so far
   int committed = -1;              // last stage whose MMAs were committed (the same in every thread)
-  for (int f = 0; f < kStages - 1; ++f) issue_loads(f);
+  for (int f = 0; f < kStages - 1; ++f) issue_loads();
   constexpr uint32_t idesc = instr_desc_bf16(kUpdTile, 2 * kUnitNodes, 1, 0);   // N = 32: hi and lo residuals side by side
   const uint64_t desc_a0 = smem_desc_sw128(smem_u32(sA), 8192, 1024), desc_r0 = smem_desc_sw128(smem_u32(sR), 16, 1024);
   float xprev[8], xcur[8];
-  for (int f = 0; f < nstages; ++f) {
-    const int t = f / G, q = f - t * G;
-    const int st = f % kStages, buf = t & 1;
+  for (int f = 0, t = 0, q = 0, st = 0; f < nstages; ++f) {
+    const int buf = t & 1;
     if (q == 0) load_x(t, xcur);                            // consumed when the tile's last stage has completed
     cp_async_wait<kStages - 2>();
     fence_proxy_async();
@@ -594,8 +606,10 @@ lsq_tc_update_kernel(StoreView s, LsqView l, const LsqUnit* __restrict__ units, 
 #pragma unroll
       for (int p = 0; p < 8; ++p) xprev[p] = xcur[p];
     }
-    if (ok) issue_loads(f + kStages - 1);                   // stage of f-1: its MMAs have completed
+    if (ok) issue_loads();                                  // into the stage of f-1: its MMAs have completed
     else cp_async_commit();
+    if (++q == G) { q = 0; ++t; }
+    if (++st == kStages) st = 0;
   }
   cp_async_wait<0>();
   if (ok && committed >= 0) {
