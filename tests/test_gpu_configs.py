@@ -173,8 +173,9 @@ def test_config5_shape_tensor_core_steps_and_two_bit_interaction():
 
 def test_config5_full_size_tensor_core_steps_on_the_last_data_matrix():
     """The 256-node store at full size (16 data matrices of 512 x 2^20 bf16: row offsets up to 16 GiB into the
-    data): all nodes take two local steps on the tensor cores, as in the benchmark; the oracle recomputes the 16
-    nodes of the last data matrix from the rows that matrix's minibatches drew, read back row by row."""
+    data): all nodes take the workload's four local steps on the tensor cores, as in the benchmark (one group of four:
+    one pass for the scores, one for the updates); the oracle recomputes the 16 nodes of the last data matrix step by
+    step from the rows that matrix's minibatches drew, read back row by row."""
     import bench
     wl = bench.WORKLOADS["regular256_d1m_b2_lsq_nb"]
     n, d, cfg = wl["n"], wl["d"], wl["cfg"]
@@ -184,26 +185,29 @@ def test_config5_full_size_tensor_core_steps_on_the_last_data_matrix():
     gpu.configure(**cfg)
     unit = list(range(n - per, n))
     x0 = [gpu.get(g.T_X, i).copy() for i in unit]
-    # the rows that the last matrix's first two minibatches draw, from the oracle's own sampler: they depend on
+    # the rows that the last matrix's first four minibatches draw, from the oracle's own sampler: they depend on
     # the seed, the matrix id, the step counter, m and the batch size only, so a short-model oracle gives them
     tiny = o.OracleSwarm(n, 8, wl["topology"], wl["degree"], wl["seed"])
     tiny.configure(**dict(cfg, nonblocking=0))
-    drawn = [tiny.minibatch_rows(n - 1, step) for step in (0, 1)]
+    H = wl["H"]
+    assert H == 4
+    drawn = [tiny.minibatch_rows(n - 1, step) for step in range(H)]
     assert all(len(r) == batch and r.max() < m for r in drawn) and not np.array_equal(drawn[0], drawn[1])
-    assert gpu.local_steps(np.arange(n), 2, wl["lr"]) == 0
+    assert len(set(np.concatenate(drawn).tolist())) < H * batch       # minibatches share rows: the corrections matter
+    assert gpu.local_steps(np.arange(n), H, wl["lr"]) == 0
     gpu.sync()
-    # a 16-node oracle whose one data matrix holds exactly those rows (2 x 64) and the labels that go with them
+    # a 16-node oracle whose one data matrix holds exactly those rows (4 x 64) and the labels that go with them
     orc = o.OracleSwarm(per, d, "complete", seed=1)
-    orc.configure(objective=2, lsq_m=2 * batch, lsq_batch=batch, lsq_dtype=1, lsq_groups=1, init_std=0.0)
-    for step in (0, 1):
+    orc.configure(objective=2, lsq_m=H * batch, lsq_batch=batch, lsq_dtype=1, lsq_groups=1, init_std=0.0)
+    for step in range(H):
         for s_idx, r in enumerate(drawn[step]):
             orc.A[0, step * batch + s_idx] = gpu.get_data_rows(groups - 1, int(r), 1)[0]
     for j, node in enumerate(unit):
         labels = gpu.get(g.T_BVEC, node)
-        for step in (0, 1):
+        for step in range(H):
             orc.bvec[j, step * batch:(step + 1) * batch] = labels[drawn[step]]
         orc.X[j] = x0[j]
-    for step in (0, 1):
+    for step in range(H):
         for j in range(per):
             assert orc.local_step_on_rows(j, np.arange(step * batch, (step + 1) * batch), wl["lr"]) == 0
     for j, node in enumerate(unit):
