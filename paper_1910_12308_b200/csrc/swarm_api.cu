@@ -70,6 +70,9 @@ struct swarm_ctx {
   float* tc_partial = nullptr;       // tensor-core path: split-K partials of the residuals
   void* tc_resid = nullptr;          // tensor-core path: residuals as bf16 hi / lo
   float* gram = nullptr;             // tensor-core path: Gram matrices of the data matrices (nullptr: not kept)
+  bool sweep_backwards = false;      // direction of the next interaction launch's walk over its (pair, block) list
+  std::vector<uint64_t> touched;     // per node: when an interaction kernel last visited its rows (a running count)
+  uint64_t touch_seq = 0;
   int* kernel_status = nullptr;      // set by a kernel whose bounded wait expired
   int* kernel_status_host = nullptr; // pinned
   bool status_pending = false;       // kernels with bounded waits were launched since the status word was last read
@@ -167,6 +170,7 @@ StoreView view_of(const swarm_ctx* c) {
   s.key0 = (uint32_t)c->seed; s.key1 = (uint32_t)(c->seed >> 32);
   s.rk = philox_round_keys(s.key0, s.key1);
   division_magic((uint64_t)c->nblk, &s.nblk_magic, &s.nblk_shift);
+  s.backwards = 0;
   return s;
 }
 LsqView lsq_of(const swarm_ctx* c) {
@@ -539,7 +543,7 @@ int swarm_init(swarm_ctx** out, int32_t n, int64_t d, swarm_topology topo, uint6
   }
   c->wait_limit = lsq_tc_default_wait_limit();
   if (!build_graph(c)) { delete c; return SWARM_EINVAL; }
-  c->w.assign(n, 0); c->ls.assign(n, 0); c->pbits.assign(n, 0); c->wo.assign(n, 0); c->tau.assign(n, 0);
+  c->w.assign(n, 0); c->ls.assign(n, 0); c->pbits.assign(n, 0); c->wo.assign(n, 0); c->tau.assign(n, 0); c->touched.assign(n, 0);
 
   const size_t row_bytes = (size_t)c->pitch * sizeof(float);
   const size_t max_pairs = (size_t)n / 2;
@@ -794,11 +798,24 @@ static int interact_impl(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, 
     pd = (PairDesc*)host;
     list.ptr = (const PairDesc*)dev;
   }
-  for (int p = 0; p < npairs; ++p) {
-    pd[p].a = pairs[p].a; pd[p].b = pairs[p].b;
-    pd[p].wa = c->w[pairs[p].a]; pd[p].wb = c->w[pairs[p].b];
-    pd[p].woa = c->wo[pairs[p].a]; pd[p].prefix = (uint32_t)(prefixes ? prefixes[p] : c->own_prefix);
-    pd[p].lsa = c->ls[pairs[p].a]; pd[p].lsb = c->ls[pairs[p].b];
+  // The kernel may take the pairs of a launch in any order (they are disjoint; clocks and counters follow the
+  // caller's list order on the host). It walks its descriptor list from one end, alternating the end from launch
+  // to launch, and the descriptors are laid out so that the walk meets the pairs whose rows the previous launches
+  // touched last first: a good part of those rows is still in L2.
+  const bool backwards = c->sweep_backwards;
+  c->sweep_backwards = !c->sweep_backwards;
+  std::vector<int> walk((size_t)npairs);
+  for (int p = 0; p < npairs; ++p) walk[p] = p;
+  std::stable_sort(walk.begin(), walk.end(), [&](int x, int y) {
+    return std::max(c->touched[pairs[x].a], c->touched[pairs[x].b]) > std::max(c->touched[pairs[y].a], c->touched[pairs[y].b]);
+  });
+  for (int t = 0; t < npairs; ++t) {
+    const int p = walk[t], at = backwards ? npairs - 1 - t : t;
+    pd[at].a = pairs[p].a; pd[at].b = pairs[p].b;
+    pd[at].wa = c->w[pairs[p].a]; pd[at].wb = c->w[pairs[p].b];
+    pd[at].woa = c->wo[pairs[p].a]; pd[at].prefix = (uint32_t)(prefixes ? prefixes[p] : c->own_prefix);
+    pd[at].lsa = c->ls[pairs[p].a]; pd[at].lsb = c->ls[pairs[p].b];
+    c->touched[pairs[p].a] = c->touched[pairs[p].b] = ++c->touch_seq;
   }
   FusedSteps fs{};
   fs.H = fused_H; fs.responders = responders ? 1 : 0; fs.lr = lr; fs.grad_std = c->cfg.grad_std; fs.scalars = c->scalars;
@@ -807,9 +824,11 @@ static int interact_impl(swarm_ctx* c, const swarm_pair* pairs, int32_t npairs, 
     if (rc != SWARM_OK) return rc;
   }
   int nl = 0;
-  if (mode == SWARM_BLOCKING) SW_CUDA(c, launch_interact_blocking(view_of(c), list, npairs, bits, fs, c->stream, &nl));
-  else if (mode == SWARM_NONBLOCKING) SW_CUDA(c, launch_interact_nonblocking(view_of(c), list, npairs, bits, fs, c->stream, &nl));
-  else SW_CUDA(c, launch_interact_registers(view_of(c), list, npairs, bits, fs, c->stream, &nl));
+  StoreView sv = view_of(c);
+  sv.backwards = backwards ? 1u : 0u;
+  if (mode == SWARM_BLOCKING) SW_CUDA(c, launch_interact_blocking(sv, list, npairs, bits, fs, c->stream, &nl));
+  else if (mode == SWARM_NONBLOCKING) SW_CUDA(c, launch_interact_nonblocking(sv, list, npairs, bits, fs, c->stream, &nl));
+  else SW_CUDA(c, launch_interact_registers(sv, list, npairs, bits, fs, c->stream, &nl));
   for (int p = 0; p < npairs && fused_H > 0; ++p) {
     c->ls[pairs[p].a] += (uint32_t)fused_H;
     if (responders) c->ls[pairs[p].b] += (uint32_t)fused_H;

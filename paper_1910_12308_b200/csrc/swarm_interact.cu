@@ -32,8 +32,9 @@ constexpr int64_t kPrefetchDistanceRegisters = 296;   // the register-protocol k
 // shift in the store view give the exact quotient by the number of blocks per row.
 __device__ __forceinline__ bool warp_slot(int64_t total_warps, const StoreView& s, uint32_t ahead, uint32_t& pair,
                                           uint32_t& blk) {
-  const uint32_t warp = blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5) + ahead;
+  uint32_t warp = blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5) + ahead;
   if (warp >= (uint32_t)total_warps) return false;
+  if (s.backwards) warp = (uint32_t)total_warps - 1u - warp;
   pair = s.nblk_magic ? __umulhi(warp, s.nblk_magic) >> s.nblk_shift : warp;
   blk = warp - pair * (uint32_t)s.nblk;
   return true;

@@ -82,6 +82,9 @@ struct StoreView {
   // warp index -> (pair, block) without a division: for w < 2^31, w / nblk = umulhi(w, nblk_magic) >> nblk_shift
   // (nblk_magic = 0: nblk is 1 and the quotient is w itself)
   uint32_t nblk_magic, nblk_shift;
+  // 1: an interaction launch walks its (pair, block) list from the end. Launches alternate, so that a launch starts
+  // with the rows its predecessor touched last, a good part of which is still in L2.
+  uint32_t backwards;
 };
 
 // Multiplier and shift with floor(w / divisor) = umulhi(w, magic) >> shift for every w < 2^31 (divisor >= 2):
