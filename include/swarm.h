@@ -153,7 +153,9 @@ int swarm_local_steps_geometric(swarm_ctx *ctx, const int32_t *node_ids_host, in
  *     model and snapshot, rewrites both of its registers and writes Enc(average) to cur_b. Registers are
  *     (re)initialised from the snapshots first when they are not in this convention at `bits` bits.
  * Every call advances the staleness clocks: interactions of a launch are taken in list order, each
- * resets its initiator's clock and ages all other nodes by one.
+ * resets its initiator's clock and ages all other nodes by one. The pairs of a launch are disjoint, so the order
+ * in which the device works through them does not show in any result; the library chooses it (launches walk
+ * their pairs from alternating ends, most recently visited rows first, for the sake of the L2 cache).
  * Errors: EINVAL (bits, mode, npairs < 0, NULL), ERANGE, EPAIR, ESTATE. */
 int swarm_interact(swarm_ctx *ctx, const swarm_pair *pairs_host, int32_t npairs, int32_t bits, int32_t mode);
 
